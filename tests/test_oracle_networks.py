@@ -1,0 +1,107 @@
+"""Pins for the oracle's two networks (Eq. 2, Eq. 6; architecture of Section 4.1.3)."""
+import math
+
+import numpy as np
+from scipy.special import expit
+
+import oracle
+from paper_2608_16329_b200 import workloads as wl
+from conftest import golden_lines
+
+LN3 = math.log(3.0)
+
+
+def _golden(name):
+    for line in golden_lines("tiny_networks.txt"):
+        key, val = line.split()
+        if key == name:
+            return float(val)
+    raise KeyError(name)
+
+
+def test_parameter_counts():
+    # 1->128->128->128->32 and 128->64->64->64->64->1
+    assert wl.enc_net_size() == 128 + 128 + 2 * (128 * 128 + 128) + 32 * 128 + 32 == 37408
+    assert wl.head_net_size(128) == 128 * 64 + 64 + 3 * (64 * 64 + 64) + 64 + 1 == 20801
+
+
+def test_encoder_hand_worked_value_and_layout():
+    enc = np.array([LN3, 0.0, 0.0, 0.0,                # W1 [2][1], b1
+                    0.0, 0.0, 4.0 / 3.0, 0.0, 0.0, 0.0,  # W2 [2][2] row-major [out][in], b2
+                    1.0, 2.0, 0.5])                      # W3 [1][2], b3
+    m = oracle.Model(1, 6.0, enc, np.zeros(16), k=1, l_max=0, enc_hidden=2, enc_layers=2,
+                     head_hidden=1, head_layers=1)
+    y, _ = oracle.encoder(m, 0, 0, 1.0)
+    assert abs(y[0] - _golden("encoder_y")) < 1e-14
+
+
+def test_head_hand_worked_value_and_layout():
+    head = np.array([1.0, 0.0, -1.0, 0.0, 0.0, 0.0,      # W1 [2][2], b1
+                     0.0, -4.0, 0.0, 0.0, 0.0, 0.0,      # W2 [2][2], b2
+                     2.0, 4.0, -1.0])                    # w_out, b_out
+    m = oracle.Model(1, 6.0, np.zeros(16), head, k=2, l_max=0, enc_hidden=1, enc_layers=1,
+                     head_hidden=2, head_layers=2)
+    e = oracle.head(m, 0, np.array([LN3, 5.0]))
+    assert abs(e - _golden("head_e")) < 1e-14
+
+
+def test_encoder_reduces_to_one_layer_when_inner_layers_are_zero():
+    """With W2 = W3 = 0, b = 0 the residual layers add SiLU(0) = 0: y = W4 SiLU(w1 r + b1) + b4."""
+    rng = np.random.default_rng(0)
+    H, K = 128, 32
+    w1, b1 = rng.standard_normal(H), rng.standard_normal(H)
+    W4, b4 = rng.standard_normal((K, H)), rng.standard_normal(K)
+    zero = np.zeros(H * H + H)
+    enc = np.concatenate([w1, b1, zero, zero, W4.ravel(), b4])
+    m = oracle.Model(1, 6.0, enc, np.zeros(wl.head_net_size(128)))
+    for r in (0.7, 2.5, 5.9):
+        pre = w1 * r + b1
+        want = W4 @ (pre * expit(pre)) + b4
+        y, _ = oracle.encoder(m, 0, 0, r)
+        assert np.abs(y - want).max() < 1e-12
+
+
+def test_encoder_selects_the_ordered_pair_network():
+    enc, head = wl.make_weights(3, seed=5)
+    m = oracle.Model(3, 6.0, enc, head)
+    n = wl.enc_net_size()
+    single = oracle.Model(1, 6.0, enc[(2 * 3 + 1) * n:(2 * 3 + 2) * n], head[:wl.head_net_size(128)])
+    assert np.array_equal(oracle.encoder(m, 2, 1, 3.3)[0], oracle.encoder(single, 0, 0, 3.3)[0])
+    assert not np.allclose(oracle.encoder(m, 2, 1, 3.3)[0], oracle.encoder(m, 1, 2, 3.3)[0])
+
+
+def test_encoder_and_radial_derivatives_match_finite_differences():
+    enc, head = wl.make_weights(2, seed=7)
+    m = oracle.Model(2, 6.0, enc, head)
+    for r in (1.3, 2.9, 4.4, 5.95):
+        h = 1e-6
+        for fn in (oracle.encoder, oracle.radial):
+            _, d = fn(m, 1, 0, r)
+            fd = (fn(m, 1, 0, r + h)[0] - fn(m, 1, 0, r - h)[0]) / (2 * h)
+            assert np.abs(fd - d).max() < 1e-7 * max(1.0, np.abs(d).max())
+
+
+def test_radial_feature_vanishes_smoothly_at_the_cutoff():
+    enc, head = wl.make_weights(1, seed=9)
+    m = oracle.Model(1, 6.0, enc, head)
+    g, dg = oracle.radial(m, 0, 0, 6.0 - 1e-9)
+    assert np.abs(g).max() < 1e-15 and np.abs(dg).max() < 1e-7
+    g, dg = oracle.radial(m, 0, 0, 6.5)
+    assert not g.any() and not dg.any()
+    y, _ = oracle.encoder(m, 0, 0, 3.0)
+    g, _ = oracle.radial(m, 0, 0, 3.0)           # envelope is exactly 1/2 at r_c / 2
+    assert np.abs(g - 0.5 * y).max() < 1e-15
+
+
+def test_head_gradient_matches_finite_differences_and_selects_species():
+    enc, head = wl.make_weights(3, seed=11)
+    m = oracle.Model(3, 6.0, enc, head)
+    rng = np.random.default_rng(1)
+    G = rng.standard_normal(128)
+    e, dG = oracle.head(m, 1, G, want_grad=True)
+    assert e == oracle.head(m, 1, G)
+    assert e != oracle.head(m, 2, G)
+    for i in (0, 31, 32, 77, 127):
+        d = np.zeros(128); d[i] = 1e-6
+        fd = (oracle.head(m, 1, G + d) - oracle.head(m, 1, G - d)) / 2e-6
+        assert abs(fd - dG[i]) < 1e-8 * max(1.0, abs(dG[i]))
