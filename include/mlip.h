@@ -1,0 +1,166 @@
+/*
+ * mlip.h - C ABI of the B200 (sm_100a) small-footprint MLIP library.
+ *
+ * The library evaluates per-atom energies, forces and the virial of the
+ * pair-conditioned, irreducible-angular-basis potential (paper Section 3.1,
+ * Eq. 1-10) for periodic orthorhombic multi-component systems: a cell-binned
+ * neighbor list followed by ONE fused kernel (Section 3.4, "mega-fusion") that
+ * runs encoding, regression and derivation without writing a feature vector or
+ * any per-pair / per-atom intermediate tensor to device memory; plus a
+ * velocity-Verlet NVE step around it.
+ *
+ * Conventions
+ *   - Every function returns an int status (MLIP_OK == 0).  Nothing throws or
+ *     aborts, and no kernel traps: a device-side problem (list capacity, skin
+ *     exceeded, non-finite input, distance below the table range) raises a bit
+ *     in a device status word, the kernels finish with defined output, and the
+ *     next mlip_sync_status() reports and clears it.
+ *   - "dev" pointers are device memory on the context's device, "host" pointers
+ *     are host memory.  The caller owns every buffer it passes; the library
+ *     owns the context and its internal buffers until mlip_destroy().
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls enqueue work and return without synchronising unless stated.
+ *   - Units: Angstrom, eV, amu, fs.  Atom order of every array argument is the
+ *     caller's; the library keeps its own cell-sorted order internally.
+ *   - Only k = 32 radial channels and l_max = 3 (d = 16) are compiled in; the
+ *     encoder is 1 -> enc_hidden x enc_layers -> k, the head is
+ *     (l_max+1) k -> head_hidden x head_layers -> 1 with head_hidden = 64,
+ *     head_layers = 4 (Section 4.1.3), SiLU, identity skips around hidden
+ *     layers of equal width.
+ */
+#ifndef MLIP_H
+#define MLIP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mlip_ctx mlip_ctx;
+
+enum {
+    MLIP_OK = 0,
+    MLIP_ERR_INVALID_ARG = 1,
+    MLIP_ERR_UNSUPPORTED = 2,      /* k, l_max, network shape, species count not compiled in */
+    MLIP_ERR_BOX_TOO_SMALL = 3,    /* an edge is shorter than 2 (r_cut + skin) */
+    MLIP_ERR_NEIGHBOR_OVERFLOW = 4,/* list capacity exceeded during an in-step rebuild */
+    MLIP_ERR_SKIN_EXCEEDED = 5,    /* an atom moved more than skin/2 since the last build */
+    MLIP_ERR_NONFINITE = 6,        /* NaN/Inf or out-of-box position */
+    MLIP_ERR_TABLE_TOLERANCE = 7,  /* radial table misses the encoder by more than table_tol */
+    MLIP_ERR_NOT_BUILT = 8,        /* compute/step before build_neighbors */
+    MLIP_ERR_OOM = 9,
+    MLIP_ERR_CUDA = 10,
+    MLIP_ERR_TABLE_RANGE = 11      /* a pair came closer than table_r_min */
+};
+
+typedef struct {
+    int n_species;        /* C, 1..8 */
+    double r_cut;         /* Angstrom */
+    double skin;          /* list radius = r_cut + skin */
+    int k;                /* 32 */
+    int l_max;            /* 3 */
+    int enc_hidden, enc_layers;    /* e.g. 128, 3 */
+    int head_hidden, head_layers;  /* 64, 4 */
+    int table_knots;      /* intervals of the radial table on [table_r_min, r_cut]; 0 = default */
+    double table_r_min;   /* smallest tabulated distance; 0 = default (1.0) */
+    double table_tol;     /* accepted table error relative to max|g|; 0 = default (1e-6) */
+    int device;           /* CUDA device ordinal */
+} mlip_config;
+
+/*
+ * Create a context: uploads the networks, tabulates every ordered-pair encoder
+ * (Eq. 2: g = f_c(r) E(r; s_i, s_j), cosine envelope f_c) as a cubic B-spline
+ * in fp64 on the device and checks it against the network.  Synchronises.
+ *   enc_weights_host  [C*C] nets, net index s_i*C + s_j; each net is
+ *                     W1[h][1], b1[h], W2[h][h], b2[h], ..., Wout[k][h], bout[k], row-major [out][in]
+ *   head_weights_host [C] nets; each W1[64][128], b1, W2[64][64], b2, ..., w_out[64], b_out
+ *   mass_amu_host     [C]
+ * Errors: INVALID_ARG, UNSUPPORTED, OOM, CUDA, TABLE_TOLERANCE (context is still returned
+ * for inspection through mlip_table_error when the tolerance fails, *out otherwise NULL).
+ */
+int mlip_create(mlip_ctx **out, const mlip_config *cfg,
+                const double *enc_weights_host, size_t n_enc,
+                const double *head_weights_host, size_t n_head,
+                const double *mass_amu_host);
+
+/* Largest |spline - network| / max|network| found over all pair types (value, derivative). */
+int mlip_table_error(const mlip_ctx *ctx, double *err_value, double *err_deriv);
+
+/*
+ * Bin the atoms into cells and build the neighbor lists (Section 3.1.1: all j
+ * within the list radius, minimum image, strict d^2 < (r_cut+skin)^2 in fp64
+ * without fused multiply-add).  Copies positions and species into the context;
+ * velocities are reset to zero.  Positions must lie in [0, L).  May reallocate
+ * and synchronises once (to size the list).
+ *   pos      dev [N][3] double      species  dev [N] int32 in [0, C)
+ *   box      host [3] edge lengths (orthorhombic); each >= 2 (r_cut + skin)
+ */
+int mlip_build_neighbors(mlip_ctx *ctx, int64_t n_atoms, const double *pos, const int32_t *species,
+                         const double *box, void *stream);
+
+/*
+ * Export the lists in canonical form: caller's atom indices; for atom i and
+ * species s the neighbors of species s in ascending index order occupy
+ * nbr[seg_ptr[i*C+s] .. seg_ptr[i*C+s+1]).  Synchronises.
+ *   seg_ptr dev [N*C+1] int64, nbr dev [capacity] int32, n_entries_host out.
+ * If capacity is too small only seg_ptr and *n_entries_host are valid and
+ * MLIP_ERR_NEIGHBOR_OVERFLOW is returned.
+ */
+int mlip_get_neighbors(mlip_ctx *ctx, int64_t *seg_ptr, int32_t *nbr, int64_t capacity,
+                       int64_t *n_entries_host, void *stream);
+
+/* Replace positions (dev [N][3], caller's order) keeping the current lists. */
+int mlip_set_positions(mlip_ctx *ctx, const double *pos, void *stream);
+/* Set velocities (dev [N][3], Angstrom/fs, caller's order). */
+int mlip_set_velocities(mlip_ctx *ctx, const double *vel, void *stream);
+
+/*
+ * One fused evaluation (Eq. 1-10) at the current positions with the current
+ * lists.  Any output pointer may be NULL.
+ *   energy dev [1] double (sum of E_i)      forces dev [N][3] float, F = -dE/dr
+ *   virial dev [9] double, row-major Xi_ab = -sum_i sum_j (r_ij)_a (dE_i/dr_ij)_b
+ *   e_atom dev [N] float
+ */
+int mlip_compute(mlip_ctx *ctx, double *energy, float *forces, double *virial, float *e_atom, void *stream);
+
+/*
+ * Same evaluation with HOST buffers: copies positions in (and species at a
+ * rebuild), rebuilds the lists when `rebuild` != 0 or none exist, evaluates,
+ * copies results out and synchronises.  This is the call a host-side MD code
+ * makes once per time step.
+ */
+int mlip_compute_host(mlip_ctx *ctx, int64_t n_atoms, const double *pos_host, const int32_t *species_host,
+                      const double *box_host, int rebuild, double *energy_host, float *forces_host,
+                      double *virial_host);
+
+/*
+ * n_steps of velocity-Verlet NVE with time step dt_fs; lists are rebuilt every
+ * `rebuild_every` steps of the context's running step counter (0 = never).
+ * Needs a prior mlip_build_neighbors; evaluates forces first if none are current.
+ * Does not synchronise; device-side problems surface in mlip_sync_status().
+ */
+int mlip_step(mlip_ctx *ctx, int n_steps, double dt_fs, int rebuild_every, void *stream);
+
+/* Positions / velocities in the caller's order (dev [N][3] double, may be NULL); step counter (host). */
+int mlip_get_state(mlip_ctx *ctx, double *pos, double *vel, int64_t *step_host, void *stream);
+/* Potential energy of the last evaluation and kinetic energy now (dev [1] each, may be NULL). */
+int mlip_get_energies(mlip_ctx *ctx, double *e_pot, double *e_kin, void *stream);
+
+/* Synchronise the stream of the last call, return the first device-side error (or MLIP_OK), clear it. */
+int mlip_sync_status(mlip_ctx *ctx);
+
+/* Counters for reports: list entries, pairs inside r_cut at the last evaluation (syncs), kernels launched. */
+int mlip_get_counters(mlip_ctx *ctx, int64_t *n_list_entries, int64_t *n_pairs_in_cutoff, int64_t *n_launches);
+/* CUDA-event time of the most recent fused-kernel launch in ms (syncs on that event). */
+int mlip_last_kernel_ms(mlip_ctx *ctx, float *ms);
+
+size_t mlip_resident_bytes(const mlip_ctx *ctx);   /* device bytes the context holds */
+const char *mlip_last_error(const mlip_ctx *ctx);  /* text of the last failure (ctx may be NULL) */
+void mlip_destroy(mlip_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MLIP_H */

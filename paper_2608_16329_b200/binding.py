@@ -1,0 +1,269 @@
+"""ctypes binding of include/mlip.h: argument marshalling only.
+
+The functions carry the C entry points' names and take torch tensors (device
+memory), numpy arrays (host memory) and plain numbers; every step of the path
+runs inside the CUDA library.  Loading fails loudly if the library is missing:
+there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libmlip_b200.so")
+
+OK = 0
+ERRORS = {0: "MLIP_OK", 1: "MLIP_ERR_INVALID_ARG", 2: "MLIP_ERR_UNSUPPORTED", 3: "MLIP_ERR_BOX_TOO_SMALL",
+          4: "MLIP_ERR_NEIGHBOR_OVERFLOW", 5: "MLIP_ERR_SKIN_EXCEEDED", 6: "MLIP_ERR_NONFINITE",
+          7: "MLIP_ERR_TABLE_TOLERANCE", 8: "MLIP_ERR_NOT_BUILT", 9: "MLIP_ERR_OOM", 10: "MLIP_ERR_CUDA",
+          11: "MLIP_ERR_TABLE_RANGE"}
+CODES = {v: k for k, v in ERRORS.items()}
+
+EXPORTS = ["mlip_create", "mlip_table_error", "mlip_build_neighbors", "mlip_get_neighbors", "mlip_set_positions",
+           "mlip_set_velocities", "mlip_compute", "mlip_compute_host", "mlip_step", "mlip_get_state",
+           "mlip_get_energies", "mlip_sync_status", "mlip_get_counters", "mlip_last_kernel_ms",
+           "mlip_resident_bytes", "mlip_last_error", "mlip_destroy"]
+
+
+class MlipError(RuntimeError):
+    def __init__(self, code, message=""):
+        self.code = code
+        super().__init__(f"{ERRORS.get(code, code)}: {message}")
+
+
+class Config(ctypes.Structure):
+    _fields_ = [("n_species", ctypes.c_int), ("r_cut", ctypes.c_double), ("skin", ctypes.c_double),
+                ("k", ctypes.c_int), ("l_max", ctypes.c_int),
+                ("enc_hidden", ctypes.c_int), ("enc_layers", ctypes.c_int),
+                ("head_hidden", ctypes.c_int), ("head_layers", ctypes.c_int),
+                ("table_knots", ctypes.c_int), ("table_r_min", ctypes.c_double), ("table_tol", ctypes.c_double),
+                ("device", ctypes.c_int)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -c 'import __graft_entry__ as g; g.build()'` "
+                              "(nvcc, sm_100a). There is no fallback path.")
+        _lib = ctypes.CDLL(LIB_PATH)
+        _lib.mlip_resident_bytes.restype = ctypes.c_size_t
+        _lib.mlip_last_error.restype = ctypes.c_char_p
+        _lib.mlip_destroy.restype = None
+    return _lib
+
+
+def _dev(t):
+    """Device pointer of a CUDA torch tensor (or None)."""
+    if t is None:
+        return ctypes.c_void_p(0)
+    assert t.is_cuda and t.is_contiguous()
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _host(a):
+    if a is None:
+        return ctypes.c_void_p(0)
+    if hasattr(a, "data_ptr"):      # pinned CPU torch tensor
+        assert not a.is_cuda and a.is_contiguous()
+        return ctypes.c_void_p(a.data_ptr())
+    assert a.flags["C_CONTIGUOUS"]
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    return ctypes.c_void_p(int(stream))
+
+
+def _check(ctx, rc, allow=()):
+    if rc != OK and rc not in allow:
+        msg = lib().mlip_last_error(ctx)
+        raise MlipError(rc, msg.decode() if msg else "")
+    return rc
+
+
+def mlip_create(cfg: Config, enc_w: np.ndarray, head_w: np.ndarray, masses: np.ndarray, allow_table_error=False):
+    enc_w = np.ascontiguousarray(enc_w, dtype=np.float64)
+    head_w = np.ascontiguousarray(head_w, dtype=np.float64)
+    masses = np.ascontiguousarray(masses, dtype=np.float64)
+    ctx = ctypes.c_void_p(0)
+    rc = lib().mlip_create(ctypes.byref(ctx), ctypes.byref(cfg), _host(enc_w), ctypes.c_size_t(enc_w.size),
+                           _host(head_w), ctypes.c_size_t(head_w.size), _host(masses))
+    _check(ctx if ctx.value else None, rc, allow=(CODES["MLIP_ERR_TABLE_TOLERANCE"],) if allow_table_error else ())
+    return ctx
+
+
+def mlip_table_error(ctx):
+    a, b = ctypes.c_double(0), ctypes.c_double(0)
+    _check(ctx, lib().mlip_table_error(ctx, ctypes.byref(a), ctypes.byref(b)))
+    return a.value, b.value
+
+
+def mlip_build_neighbors(ctx, pos, species, box, stream=None):
+    box = np.ascontiguousarray(box, dtype=np.float64)
+    _check(ctx, lib().mlip_build_neighbors(ctx, ctypes.c_int64(pos.shape[0]), _dev(pos), _dev(species), _host(box), _stream(stream)))
+
+
+def mlip_get_neighbors(ctx, seg_ptr, nbr, stream=None):
+    n = ctypes.c_int64(0)
+    cap = 0 if nbr is None else nbr.numel()
+    rc = lib().mlip_get_neighbors(ctx, _dev(seg_ptr), _dev(nbr), ctypes.c_int64(cap), ctypes.byref(n), _stream(stream))
+    _check(ctx, rc, allow=(CODES["MLIP_ERR_NEIGHBOR_OVERFLOW"],))
+    return rc, n.value
+
+
+def mlip_set_positions(ctx, pos, stream=None):
+    _check(ctx, lib().mlip_set_positions(ctx, _dev(pos), _stream(stream)))
+
+
+def mlip_set_velocities(ctx, vel, stream=None):
+    _check(ctx, lib().mlip_set_velocities(ctx, _dev(vel), _stream(stream)))
+
+
+def mlip_compute(ctx, energy=None, forces=None, virial=None, e_atom=None, stream=None):
+    _check(ctx, lib().mlip_compute(ctx, _dev(energy), _dev(forces), _dev(virial), _dev(e_atom), _stream(stream)))
+
+
+def mlip_compute_host(ctx, pos, species, box, rebuild, forces_out, virial_out=None):
+    e = ctypes.c_double(0)
+    box = None if box is None else np.ascontiguousarray(box, dtype=np.float64)
+    _check(ctx, lib().mlip_compute_host(ctx, ctypes.c_int64(pos.shape[0]), _host(pos), _host(species), _host(box),
+                                        ctypes.c_int(int(rebuild)), ctypes.byref(e), _host(forces_out), _host(virial_out)))
+    return e.value
+
+
+def mlip_step(ctx, n_steps, dt_fs, rebuild_every, stream=None):
+    _check(ctx, lib().mlip_step(ctx, ctypes.c_int(n_steps), ctypes.c_double(dt_fs), ctypes.c_int(rebuild_every), _stream(stream)))
+
+
+def mlip_get_state(ctx, pos=None, vel=None, stream=None):
+    step = ctypes.c_int64(0)
+    _check(ctx, lib().mlip_get_state(ctx, _dev(pos), _dev(vel), ctypes.byref(step), _stream(stream)))
+    return step.value
+
+
+def mlip_get_energies(ctx, e_pot=None, e_kin=None, stream=None):
+    _check(ctx, lib().mlip_get_energies(ctx, _dev(e_pot), _dev(e_kin), _stream(stream)))
+
+
+def mlip_sync_status(ctx, raise_on_error=True):
+    rc = lib().mlip_sync_status(ctx)
+    if raise_on_error:
+        _check(ctx, rc)
+    return rc
+
+
+def mlip_get_counters(ctx):
+    a, b, c = ctypes.c_int64(0), ctypes.c_int64(0), ctypes.c_int64(0)
+    _check(ctx, lib().mlip_get_counters(ctx, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)))
+    return {"list_entries": a.value, "pairs_in_cutoff": b.value, "launches": c.value}
+
+
+def mlip_last_kernel_ms(ctx):
+    ms = ctypes.c_float(0)
+    _check(ctx, lib().mlip_last_kernel_ms(ctx, ctypes.byref(ms)))
+    return ms.value
+
+
+def mlip_resident_bytes(ctx):
+    return int(lib().mlip_resident_bytes(ctx))
+
+
+def mlip_last_error(ctx=None):
+    msg = lib().mlip_last_error(ctx)
+    return msg.decode() if msg else ""
+
+
+def mlip_destroy(ctx):
+    if ctx is not None and ctx.value:
+        lib().mlip_destroy(ctx)
+        ctx.value = 0
+
+
+class Potential:
+    """Convenience owner of one context; allocates outputs as torch tensors."""
+
+    def __init__(self, n_species, r_cut, skin, enc_w, head_w, masses, device=0, table_knots=0,
+                 table_r_min=0.0, table_tol=0.0, enc_hidden=128, enc_layers=3, allow_table_error=False):
+        import torch
+        self.torch = torch
+        self.device = torch.device("cuda", device)
+        self.n_species = n_species
+        self.cfg = Config(n_species, r_cut, skin, 32, 3, enc_hidden, enc_layers, 64, 4, table_knots, table_r_min,
+                          table_tol, device)
+        self.ctx = mlip_create(self.cfg, enc_w, head_w, masses, allow_table_error)
+        self.n = 0
+
+    def close(self):
+        mlip_destroy(self.ctx)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def build_neighbors(self, pos, species, box):
+        t = self.torch
+        self._pos = t.as_tensor(pos, dtype=t.float64, device=self.device).contiguous()
+        self._species = t.as_tensor(species, dtype=t.int32, device=self.device).contiguous()
+        self.n = self._pos.shape[0]
+        mlip_build_neighbors(self.ctx, self._pos, self._species, box)
+
+    def neighbors(self):
+        """Canonical lists as (seg_ptr int64 [N*C+1], nbr int32) on the device."""
+        t = self.torch
+        seg = t.empty(self.n * self.n_species + 1, dtype=t.int64, device=self.device)
+        _, total = mlip_get_neighbors(self.ctx, seg, None)
+        nbr = t.empty(max(total, 1), dtype=t.int32, device=self.device)
+        rc, total = mlip_get_neighbors(self.ctx, seg, nbr)
+        if rc != OK:
+            raise MlipError(rc, "neighbor export")
+        return seg, nbr[:total]
+
+    def compute(self, want_e_atom=False):
+        t = self.torch
+        out = {"energy": t.zeros(1, dtype=t.float64, device=self.device),
+               "forces": t.empty((self.n, 3), dtype=t.float32, device=self.device),
+               "virial": t.zeros(9, dtype=t.float64, device=self.device),
+               "e_atom": t.empty(self.n, dtype=t.float32, device=self.device) if want_e_atom else None}
+        mlip_compute(self.ctx, out["energy"], out["forces"], out["virial"], out["e_atom"])
+        return out
+
+    def set_positions(self, pos):
+        t = self.torch
+        self._pos = t.as_tensor(pos, dtype=t.float64, device=self.device).contiguous()
+        mlip_set_positions(self.ctx, self._pos)
+
+    def set_velocities(self, vel):
+        t = self.torch
+        self._vel = t.as_tensor(vel, dtype=t.float64, device=self.device).contiguous()
+        mlip_set_velocities(self.ctx, self._vel)
+
+    def step(self, n_steps, dt_fs, rebuild_every):
+        mlip_step(self.ctx, n_steps, dt_fs, rebuild_every)
+
+    def state(self):
+        t = self.torch
+        pos = t.empty((self.n, 3), dtype=t.float64, device=self.device)
+        vel = t.empty((self.n, 3), dtype=t.float64, device=self.device)
+        step = mlip_get_state(self.ctx, pos, vel)
+        return pos, vel, step
+
+    def energies(self):
+        t = self.torch
+        e = t.zeros(2, dtype=t.float64, device=self.device)
+        mlip_get_energies(self.ctx, e[0:1], e[1:2])
+        return e
+
+    def sync_status(self, raise_on_error=True):
+        return mlip_sync_status(self.ctx, raise_on_error)

@@ -1,0 +1,379 @@
+// C ABI (include/mlip.h): context life cycle, buffer management and the host-side
+// sequencing of the kernels.  No torch types, no exceptions across the boundary.
+#include <math.h>
+#include <new>
+#include <string.h>
+
+#include "common.cuh"
+#include "scan.cuh"
+
+using namespace mlip;
+
+static thread_local std::string g_last_error;
+
+static int fail(mlip_ctx *c, int code, const char *msg) {
+    if (c) c->err = msg;
+    g_last_error = msg;
+    return code;
+}
+
+template <typename T>
+static int dev_alloc(mlip_ctx *c, T **p, size_t count) {
+    *p = nullptr;
+    cudaError_t e = cudaMalloc((void **)p, sizeof(T) * (count ? count : 1));
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        c->err = std::string("cudaMalloc: ") + cudaGetErrorString(e);
+        return MLIP_ERR_OOM;
+    }
+    c->resident += sizeof(T) * (count ? count : 1);
+    return MLIP_OK;
+}
+
+template <typename T>
+static void dev_free(mlip_ctx *c, T **p, size_t count) {
+    if (*p) {
+        cudaFree(*p);
+        c->resident -= sizeof(T) * (count ? count : 1);
+        *p = nullptr;
+    }
+}
+
+static void free_atoms(mlip_ctx *c) {
+    const size_t n = (size_t)c->cap_atoms;
+    dev_free(c, &c->pos4, n); dev_free(c, &c->pos4_src, n);
+    dev_free(c, &c->vel, 3 * n); dev_free(c, &c->vel_src, 3 * n);
+    dev_free(c, &c->user_of, n); dev_free(c, &c->user_src, n);
+    dev_free(c, &c->force, n); dev_free(c, &c->disp, 3 * n);
+    dev_free(c, &c->center_order, n); dev_free(c, &c->cell_of, n);
+    dev_free(c, &c->nbr_count, n); dev_free(c, &c->nbr_off, n + 1);
+    c->cap_atoms = 0;
+}
+
+static void free_cells(mlip_ctx *c) {
+    const size_t nc = (size_t)c->cap_cells, C = (size_t)c->cfg.n_species;
+    dev_free(c, &c->cell_count, nc + 1); dev_free(c, &c->cell_start, nc + 1); dev_free(c, &c->cell_fill, nc + 1);
+    dev_free(c, &c->bin_count, C * nc + 1); dev_free(c, &c->bin_start, C * nc + 1);
+    c->cap_cells = 0;
+}
+
+static int ensure_capacity(mlip_ctx *c, int64_t n, int64_t n_cells) {
+    int rc;
+    if (n > c->cap_atoms) {
+        free_atoms(c);
+        const size_t m = (size_t)n;
+#define TRY_ALLOC(p, cnt) if ((rc = dev_alloc(c, &(p), (cnt))) != MLIP_OK) return rc
+        TRY_ALLOC(c->pos4, m); TRY_ALLOC(c->pos4_src, m);
+        TRY_ALLOC(c->vel, 3 * m); TRY_ALLOC(c->vel_src, 3 * m);
+        TRY_ALLOC(c->user_of, m); TRY_ALLOC(c->user_src, m);
+        TRY_ALLOC(c->force, m); TRY_ALLOC(c->disp, 3 * m);
+        TRY_ALLOC(c->center_order, m); TRY_ALLOC(c->cell_of, m);
+        TRY_ALLOC(c->nbr_count, m); TRY_ALLOC(c->nbr_off, m + 1);
+        c->cap_atoms = n;
+    }
+    if (n_cells > c->cap_cells) {
+        free_cells(c);
+        const size_t nc = (size_t)n_cells, C = (size_t)c->cfg.n_species;
+        TRY_ALLOC(c->cell_count, nc + 1); TRY_ALLOC(c->cell_start, nc + 1); TRY_ALLOC(c->cell_fill, nc + 1);
+        TRY_ALLOC(c->bin_count, C * nc + 1); TRY_ALLOC(c->bin_start, C * nc + 1);
+        c->cap_cells = n_cells;
+    }
+    int64_t need = scan_tmp_items(n > (int64_t)c->cfg.n_species * n_cells ? n : (int64_t)c->cfg.n_species * n_cells);
+    if (need > c->scan_tmp_cap) {
+        dev_free(c, &c->scan_tmp, (size_t)c->scan_tmp_cap);
+        TRY_ALLOC(c->scan_tmp, (size_t)need);
+        c->scan_tmp_cap = need;
+    }
+#undef TRY_ALLOC
+    return MLIP_OK;
+}
+
+static int set_grid(mlip_ctx *c, const double *box) {
+    const double rl = c->cfg.r_cut + c->cfg.skin;
+    CellGrid g;
+    int64_t n_cells = 1;
+    for (int a = 0; a < 3; ++a) {
+        if (!(box[a] >= 2.0 * rl) || !isfinite(box[a])) return fail(c, MLIP_ERR_BOX_TOO_SMALL, "box edge shorter than 2 (r_cut + skin)");
+        g.n[a] = (int)floor(box[a] / rl);
+        if (g.n[a] < 1) g.n[a] = 1;
+        g.box[a] = box[a];
+        g.half[a] = 0.5 * box[a];
+        g.inv_edge[a] = g.n[a] / box[a];
+        n_cells *= g.n[a];
+    }
+    if (n_cells > 2000000000LL) return fail(c, MLIP_ERR_UNSUPPORTED, "too many cells");
+    g.n_cells = (int)n_cells;
+    c->grid = g;
+    return MLIP_OK;
+}
+
+extern "C" {
+
+int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, size_t n_enc, const double *head_w,
+                size_t n_head, const double *mass) {
+    if (!out) return fail(nullptr, MLIP_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    if (!cfg || !enc_w || !head_w || !mass) return fail(nullptr, MLIP_ERR_INVALID_ARG, "NULL argument");
+    if (cfg->n_species < 1 || cfg->n_species > MAX_SPECIES) return fail(nullptr, MLIP_ERR_UNSUPPORTED, "n_species must be 1..8");
+    if (cfg->k != K_RADIAL || cfg->l_max != 3) return fail(nullptr, MLIP_ERR_UNSUPPORTED, "only k = 32, l_max = 3 are compiled in");
+    if (cfg->head_hidden != HEAD_H || cfg->head_layers != HEAD_L) return fail(nullptr, MLIP_ERR_UNSUPPORTED, "only a 4 x 64 head is compiled in");
+    if (cfg->enc_hidden < 1 || cfg->enc_layers < 1) return fail(nullptr, MLIP_ERR_INVALID_ARG, "bad encoder shape");
+    if (!(cfg->r_cut > 0.0) || !(cfg->skin >= 0.0)) return fail(nullptr, MLIP_ERR_INVALID_ARG, "bad r_cut or skin");
+    if (n_head != (size_t)cfg->n_species * HEAD_NET) return fail(nullptr, MLIP_ERR_INVALID_ARG, "head weight count does not match the shape");
+    for (int s = 0; s < cfg->n_species; ++s)
+        if (!(mass[s] > 0.0)) return fail(nullptr, MLIP_ERR_INVALID_ARG, "mass must be positive");
+
+    mlip_ctx *c = new (std::nothrow) mlip_ctx();
+    if (!c) return fail(nullptr, MLIP_ERR_OOM, "host allocation failed");
+    c->cfg = *cfg;
+    if (c->cfg.table_knots <= 0) c->cfg.table_knots = 256;
+    if (c->cfg.table_r_min <= 0.0) c->cfg.table_r_min = 1.0;
+    if (c->cfg.table_tol <= 0.0) c->cfg.table_tol = 1e-6;
+    if (c->cfg.table_knots > 8192 || c->cfg.table_r_min >= c->cfg.r_cut) { delete c; return fail(nullptr, MLIP_ERR_INVALID_ARG, "bad table parameters"); }
+
+    int rc = MLIP_OK;
+    cudaError_t e = cudaSetDevice(cfg->device);
+    cudaDeviceProp prop;
+    if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, cfg->device);
+    if (e != cudaSuccess) {
+        g_last_error = std::string("CUDA device unavailable: ") + cudaGetErrorString(e);
+        delete c;
+        return MLIP_ERR_CUDA;
+    }
+    c->n_sm = prop.multiProcessorCount;
+    do {
+        if ((rc = dev_alloc(c, &c->mass, (size_t)cfg->n_species)) != MLIP_OK) break;
+        if ((rc = dev_alloc(c, &c->acc, (size_t)ACC_COUNT)) != MLIP_OK) break;
+        if ((rc = dev_alloc(c, &c->pair_counter, 1)) != MLIP_OK) break;
+        if ((rc = dev_alloc(c, &c->status, 1)) != MLIP_OK) break;
+        if ((rc = dev_alloc(c, &c->tile_counter, 1)) != MLIP_OK) break;
+        if ((rc = dev_alloc(c, &c->species_start, (size_t)MAX_SPECIES + 1)) != MLIP_OK) break;
+        if ((rc = dev_alloc(c, &c->stage_out, 10)) != MLIP_OK) break;
+        if (cudaMallocHost((void **)&c->status_host, sizeof(int)) != cudaSuccess ||
+            cudaMallocHost((void **)&c->total_host, sizeof(int64_t)) != cudaSuccess ||
+            cudaEventCreate(&c->ev0) != cudaSuccess || cudaEventCreate(&c->ev1) != cudaSuccess) {
+            rc = MLIP_ERR_CUDA; c->err = "pinned host allocation or event creation failed"; break;
+        }
+        if (cudaMemcpy(c->mass, mass, sizeof(double) * cfg->n_species, cudaMemcpyHostToDevice) != cudaSuccess ||
+            cudaMemset(c->status, 0, sizeof(int)) != cudaSuccess || cudaMemset(c->acc, 0, sizeof(double) * ACC_COUNT) != cudaSuccess) {
+            rc = MLIP_ERR_CUDA; c->err = "initial upload failed"; break;
+        }
+        if ((rc = upload_head(c, head_w)) != MLIP_OK) break;
+        rc = build_tables(c, enc_w, n_enc);
+    } while (0);
+    if (rc != MLIP_OK && rc != MLIP_ERR_TABLE_TOLERANCE) {
+        g_last_error = c->err;
+        mlip_destroy(c);
+        return rc;
+    }
+    if (rc != MLIP_OK) g_last_error = c->err;
+    *out = c;
+    return rc;
+}
+
+int mlip_table_error(const mlip_ctx *c, double *err_value, double *err_deriv) {
+    if (!c) return MLIP_ERR_INVALID_ARG;
+    if (err_value) *err_value = c->table_err_value;
+    if (err_deriv) *err_deriv = c->table_err_deriv;
+    return MLIP_OK;
+}
+
+int mlip_build_neighbors(mlip_ctx *c, int64_t n, const double *pos, const int32_t *species, const double *box, void *stream) {
+    if (!c) return MLIP_ERR_INVALID_ARG;
+    if (n < 1 || n > 2000000000LL || !pos || !species || !box) return fail(c, MLIP_ERR_INVALID_ARG, "bad arguments to mlip_build_neighbors");
+    cudaStream_t s = (cudaStream_t)stream;
+    c->last_stream = s;
+    cudaSetDevice(c->cfg.device);
+    int rc = set_grid(c, box);
+    if (rc != MLIP_OK) return rc;
+    c->built = false;
+    if ((rc = ensure_capacity(c, n, c->grid.n_cells)) != MLIP_OK) return rc;
+    c->n = n;
+    if ((rc = launch_pack_source(c, pos, species, s)) != MLIP_OK) return rc;
+    double *keep = c->vel_src;   // a NULL source makes the gather reset velocities to zero
+    c->vel_src = nullptr;
+    rc = launch_build(c, true, s);
+    c->vel_src = keep;
+    if (rc != MLIP_OK) return rc;
+    c->built = true;
+    c->forces_current = false;
+    return MLIP_OK;
+}
+
+int mlip_get_neighbors(mlip_ctx *c, int64_t *seg_ptr, int32_t *nbr, int64_t capacity, int64_t *n_entries_host, void *stream) {
+    if (!c || !seg_ptr) return MLIP_ERR_INVALID_ARG;
+    if (!c->built) return fail(c, MLIP_ERR_NOT_BUILT, "no neighbor lists yet");
+    c->last_stream = (cudaStream_t)stream;
+    return launch_export(c, seg_ptr, nbr, capacity, n_entries_host, (cudaStream_t)stream);
+}
+
+int mlip_set_positions(mlip_ctx *c, const double *pos, void *stream) {
+    if (!c || !pos) return MLIP_ERR_INVALID_ARG;
+    if (!c->built) return fail(c, MLIP_ERR_NOT_BUILT, "no neighbor lists yet");
+    c->last_stream = (cudaStream_t)stream;
+    c->forces_current = false;
+    return launch_set_positions(c, pos, (cudaStream_t)stream);
+}
+
+int mlip_set_velocities(mlip_ctx *c, const double *vel, void *stream) {
+    if (!c || !vel) return MLIP_ERR_INVALID_ARG;
+    if (!c->built) return fail(c, MLIP_ERR_NOT_BUILT, "no neighbor lists yet");
+    c->last_stream = (cudaStream_t)stream;
+    return launch_set_velocities(c, vel, (cudaStream_t)stream);
+}
+
+int mlip_compute(mlip_ctx *c, double *energy, float *forces, double *virial, float *e_atom, void *stream) {
+    if (!c) return MLIP_ERR_INVALID_ARG;
+    if (!c->built) return fail(c, MLIP_ERR_NOT_BUILT, "no neighbor lists yet");
+    cudaStream_t s = (cudaStream_t)stream;
+    c->last_stream = s;
+    int rc = launch_megakernel(c, s);
+    if (rc != MLIP_OK) return rc;
+    c->forces_current = true;
+    if (energy) MLIP_CUDA_TRY(c, cudaMemcpyAsync(energy, c->acc + ACC_ENERGY, sizeof(double), cudaMemcpyDeviceToDevice, s));
+    if (virial) MLIP_CUDA_TRY(c, cudaMemcpyAsync(virial, c->acc + ACC_VIRIAL, sizeof(double) * 9, cudaMemcpyDeviceToDevice, s));
+    if (forces || e_atom) rc = launch_scatter_forces(c, forces, e_atom, s);
+    return rc;
+}
+
+int mlip_compute_host(mlip_ctx *c, int64_t n, const double *pos_host, const int32_t *species_host, const double *box_host,
+                      int rebuild, double *energy_host, float *forces_host, double *virial_host) {
+    if (!c || !pos_host || n < 1) return MLIP_ERR_INVALID_ARG;
+    cudaStream_t s = c->last_stream;
+    cudaSetDevice(c->cfg.device);
+    const bool need_build = rebuild || !c->built || n != c->n;
+    if (need_build && (!species_host || !box_host)) return fail(c, MLIP_ERR_INVALID_ARG, "species and box are needed to build the lists");
+    int rc;
+    if (n > c->stage_cap) {
+        dev_free(c, &c->stage_pos, 3 * (size_t)c->stage_cap);
+        dev_free(c, &c->stage_species, (size_t)c->stage_cap);
+        dev_free(c, &c->stage_force, 3 * (size_t)c->stage_cap);
+        c->stage_cap = 0;
+        if ((rc = dev_alloc(c, &c->stage_pos, 3 * (size_t)n)) != MLIP_OK) return rc;
+        if ((rc = dev_alloc(c, &c->stage_species, (size_t)n)) != MLIP_OK) return rc;
+        if ((rc = dev_alloc(c, &c->stage_force, 3 * (size_t)n)) != MLIP_OK) return rc;
+        c->stage_cap = n;
+    }
+    MLIP_CUDA_TRY(c, cudaMemcpyAsync(c->stage_pos, pos_host, sizeof(double) * 3 * n, cudaMemcpyHostToDevice, s));
+    if (need_build) {
+        MLIP_CUDA_TRY(c, cudaMemcpyAsync(c->stage_species, species_host, sizeof(int32_t) * n, cudaMemcpyHostToDevice, s));
+        if ((rc = mlip_build_neighbors(c, n, c->stage_pos, c->stage_species, box_host, s)) != MLIP_OK) return rc;
+    } else if ((rc = mlip_set_positions(c, c->stage_pos, s)) != MLIP_OK) return rc;
+    if ((rc = mlip_compute(c, c->stage_out, forces_host ? c->stage_force : nullptr, c->stage_out + 1, nullptr, s)) != MLIP_OK) return rc;
+    if (forces_host) MLIP_CUDA_TRY(c, cudaMemcpyAsync(forces_host, c->stage_force, sizeof(float) * 3 * n, cudaMemcpyDeviceToHost, s));
+    double out[10];
+    MLIP_CUDA_TRY(c, cudaMemcpyAsync(out, c->stage_out, sizeof out, cudaMemcpyDeviceToHost, s));
+    MLIP_CUDA_TRY(c, cudaStreamSynchronize(s));
+    if (energy_host) *energy_host = out[0];
+    if (virial_host) memcpy(virial_host, out + 1, sizeof(double) * 9);
+    return MLIP_OK;
+}
+
+int mlip_step(mlip_ctx *c, int n_steps, double dt, int rebuild_every, void *stream) {
+    if (!c || n_steps < 0 || !(dt > 0.0) || rebuild_every < 0) return MLIP_ERR_INVALID_ARG;
+    if (!c->built) return fail(c, MLIP_ERR_NOT_BUILT, "no neighbor lists yet");
+    cudaStream_t s = (cudaStream_t)stream;
+    c->last_stream = s;
+    int rc;
+    if (!c->forces_current) {
+        if ((rc = launch_megakernel(c, s)) != MLIP_OK) return rc;
+        c->forces_current = true;
+    }
+    for (int it = 0; it < n_steps; ++it) {
+        if ((rc = launch_kick_drift(c, dt, s)) != MLIP_OK) return rc;
+        c->step += 1;
+        if (rebuild_every > 0 && c->step % rebuild_every == 0) {
+            std::swap(c->pos4, c->pos4_src);
+            std::swap(c->vel, c->vel_src);
+            std::swap(c->user_of, c->user_src);
+            if ((rc = launch_build(c, false, s)) != MLIP_OK) return rc;
+        }
+        if ((rc = launch_megakernel(c, s)) != MLIP_OK) return rc;
+        if ((rc = launch_kick(c, dt, s)) != MLIP_OK) return rc;
+    }
+    return MLIP_OK;
+}
+
+int mlip_get_state(mlip_ctx *c, double *pos, double *vel, int64_t *step_host, void *stream) {
+    if (!c) return MLIP_ERR_INVALID_ARG;
+    if (!c->built) return fail(c, MLIP_ERR_NOT_BUILT, "no atoms yet");
+    c->last_stream = (cudaStream_t)stream;
+    if (step_host) *step_host = c->step;
+    if (pos || vel) return launch_get_state(c, pos, vel, (cudaStream_t)stream);
+    return MLIP_OK;
+}
+
+int mlip_get_energies(mlip_ctx *c, double *e_pot, double *e_kin, void *stream) {
+    if (!c) return MLIP_ERR_INVALID_ARG;
+    if (!c->built) return fail(c, MLIP_ERR_NOT_BUILT, "no atoms yet");
+    cudaStream_t s = (cudaStream_t)stream;
+    c->last_stream = s;
+    if (e_pot) MLIP_CUDA_TRY(c, cudaMemcpyAsync(e_pot, c->acc + ACC_ENERGY, sizeof(double), cudaMemcpyDeviceToDevice, s));
+    if (e_kin) {
+        int rc = launch_kinetic(c, s);
+        if (rc != MLIP_OK) return rc;
+        MLIP_CUDA_TRY(c, cudaMemcpyAsync(e_kin, c->acc + ACC_KINETIC, sizeof(double), cudaMemcpyDeviceToDevice, s));
+    }
+    return MLIP_OK;
+}
+
+int mlip_sync_status(mlip_ctx *c) {
+    if (!c) return MLIP_ERR_INVALID_ARG;
+    cudaStream_t s = c->last_stream;
+    MLIP_CUDA_TRY(c, cudaMemcpyAsync(c->status_host, c->status, sizeof(int), cudaMemcpyDeviceToHost, s));
+    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->status, 0, sizeof(int), s));
+    MLIP_CUDA_TRY(c, cudaStreamSynchronize(s));
+    const int f = *c->status_host;
+    if (f & FLAG_NONFINITE) return fail(c, MLIP_ERR_NONFINITE, "non-finite or out-of-box position, or species out of range");
+    if (f & FLAG_NEIGHBOR_OVERFLOW) return fail(c, MLIP_ERR_NEIGHBOR_OVERFLOW, "neighbor list capacity exceeded during a rebuild");
+    if (f & FLAG_SKIN_EXCEEDED) return fail(c, MLIP_ERR_SKIN_EXCEEDED, "an atom moved more than skin/2 since the last list build");
+    if (f & FLAG_TABLE_RANGE) return fail(c, MLIP_ERR_TABLE_RANGE, "a pair came closer than table_r_min");
+    return MLIP_OK;
+}
+
+int mlip_get_counters(mlip_ctx *c, int64_t *n_list_entries, int64_t *n_pairs, int64_t *n_launches) {
+    if (!c) return MLIP_ERR_INVALID_ARG;
+    MLIP_CUDA_TRY(c, cudaStreamSynchronize(c->last_stream));
+    if (n_list_entries) {
+        *n_list_entries = 0;
+        if (c->built) MLIP_CUDA_TRY(c, cudaMemcpy(n_list_entries, c->nbr_off + c->n, sizeof(int64_t), cudaMemcpyDeviceToHost));
+    }
+    if (n_pairs) {
+        unsigned long long v = 0;
+        MLIP_CUDA_TRY(c, cudaMemcpy(&v, c->pair_counter, sizeof v, cudaMemcpyDeviceToHost));
+        *n_pairs = (int64_t)v;
+    }
+    if (n_launches) *n_launches = c->launches;
+    return MLIP_OK;
+}
+
+int mlip_last_kernel_ms(mlip_ctx *c, float *ms) {
+    if (!c || !ms) return MLIP_ERR_INVALID_ARG;
+    if (!c->kernel_timed) return fail(c, MLIP_ERR_NOT_BUILT, "the fused kernel has not run yet");
+    MLIP_CUDA_TRY(c, cudaEventSynchronize(c->ev1));
+    MLIP_CUDA_TRY(c, cudaEventElapsedTime(ms, c->ev0, c->ev1));
+    return MLIP_OK;
+}
+
+size_t mlip_resident_bytes(const mlip_ctx *c) { return c ? c->resident : 0; }
+
+const char *mlip_last_error(const mlip_ctx *c) { return c ? c->err.c_str() : g_last_error.c_str(); }
+
+void mlip_destroy(mlip_ctx *c) {
+    if (!c) return;
+    cudaSetDevice(c->cfg.device);
+    cudaDeviceSynchronize();
+    free_atoms(c);
+    free_cells(c);
+    cudaFree(c->nbr); cudaFree(c->scan_tmp); cudaFree(c->head_w); cudaFree(c->table); cudaFree(c->mass);
+    cudaFree(c->acc); cudaFree(c->pair_counter); cudaFree(c->status); cudaFree(c->tile_counter);
+    cudaFree(c->species_start); cudaFree(c->stage_pos); cudaFree(c->stage_species); cudaFree(c->stage_force);
+    cudaFree(c->stage_out);
+    if (c->status_host) cudaFreeHost(c->status_host);
+    if (c->total_host) cudaFreeHost(c->total_host);
+    if (c->ev0) cudaEventDestroy(c->ev0);
+    if (c->ev1) cudaEventDestroy(c->ev1);
+    delete c;
+}
+
+}  // extern "C"

@@ -1,0 +1,154 @@
+// Internal declarations shared by the library's translation units.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string>
+
+#include "mlip.h"
+
+namespace mlip {
+
+constexpr int K_RADIAL = 32;   // radial channels (Section 3.2.3: k = 32)
+constexpr int D_ANG = 16;      // irreducible angular components up to l = 3 (Section 3.3.2)
+constexpr int N_INV = 128;     // (l_max + 1) * k invariants (Eq. 5)
+constexpr int HEAD_H = 64;     // head width (Section 4.1.3)
+constexpr int HEAD_L = 4;      // head hidden layers
+constexpr int MAX_SPECIES = 8;
+constexpr int HEAD_NET = N_INV * HEAD_H + HEAD_H + (HEAD_L - 1) * (HEAD_H * HEAD_H + HEAD_H) + HEAD_H + 1;
+
+// 1 eV/(Angstrom amu) in Angstrom/fs^2
+constexpr double ACC_UNIT = 1.602176634e-19 / 1.66053906660e-27 * 1e-10;
+
+// device status word bits
+enum : int {
+    FLAG_NEIGHBOR_OVERFLOW = 1 << 0,
+    FLAG_SKIN_EXCEEDED = 1 << 1,
+    FLAG_NONFINITE = 1 << 2,
+    FLAG_TABLE_RANGE = 1 << 3,
+};
+
+// accumulator slots (double)
+enum : int { ACC_ENERGY = 0, ACC_VIRIAL = 1, ACC_KINETIC = 10, ACC_COUNT = 16 };
+
+struct CellGrid {
+    int n[3];          // cells per dimension
+    double inv_edge[3];
+    double box[3];
+    double half[3];    // 0.5 * box, the minimum-image threshold
+    int n_cells;
+};
+
+// Radial table: uniform cubic B-spline per ordered species pair and channel.
+struct TableDesc {
+    const float *coef;   // [C*C][knots + 3][K_RADIAL]
+    int knots;           // number of intervals
+    float r_min;
+    float inv_h;         // 1 / interval width
+    float r_cut2;
+};
+
+struct Buffers;  // defined in api.cu
+
+}  // namespace mlip
+
+struct mlip_ctx {
+    mlip_config cfg{};
+    std::string err;
+    int n_sm = 0;
+
+    // model
+    float *head_w = nullptr;     // [C][HEAD_NET] fp32, layout see megakernel.cu
+    float *table = nullptr;      // spline coefficients
+    double *mass = nullptr;      // [C] dev
+    float *inv_mass_acc = nullptr; // unused placeholder
+    double table_err_value = 0, table_err_deriv = 0;
+    mlip::TableDesc tab{};
+
+    // system (internal order: by cell, then species, then caller index)
+    int64_t n = 0, cap_atoms = 0;
+    mlip::CellGrid grid{};
+    int64_t cap_cells = 0;
+    double4 *pos4 = nullptr;       // x, y, z, species stored as a double
+    double *vel = nullptr;         // [N][3]
+    int32_t *user_of = nullptr;    // internal -> caller index
+    float4 *force = nullptr;       // fx, fy, fz, E_i
+    float *disp = nullptr;         // [N][3] displacement since the last build
+    int32_t *center_order = nullptr;  // internal indices sorted by (species, cell)
+    int32_t species_start_host[mlip::MAX_SPECIES + 1] = {0};
+    // second set used as the source of a rebuild
+    double4 *pos4_src = nullptr;
+    double *vel_src = nullptr;
+    int32_t *user_src = nullptr;
+    // cells
+    int32_t *cell_of = nullptr;    // per source atom
+    int32_t *cell_count = nullptr, *cell_start = nullptr, *cell_fill = nullptr;   // [n_cells + 1]
+    int32_t *bin_count = nullptr, *bin_start = nullptr;                           // [C * n_cells + 1]
+    int32_t *species_start = nullptr;  // dev [C + 1]
+    // lists
+    int32_t *nbr_count = nullptr;  // [N]
+    int64_t *nbr_off = nullptr;    // [N + 1]
+    int32_t *nbr = nullptr;
+    int64_t nbr_cap = 0, n_entries = 0;
+    // scratch
+    int64_t *scan_tmp = nullptr;   // block sums for the scans
+    int64_t scan_tmp_cap = 0;
+    double *acc = nullptr;         // [ACC_COUNT]
+    unsigned long long *pair_counter = nullptr;
+    int *status = nullptr;         // device status word
+    int *tile_counter = nullptr;   // dynamic tile scheduler
+    int *status_host = nullptr;    // pinned
+    int64_t *total_host = nullptr; // pinned
+    double *stage_pos = nullptr;   // [N][3] staging for host entry point
+    int32_t *stage_species = nullptr;
+    float *stage_force = nullptr;
+    double *stage_out = nullptr;   // [10]
+    int64_t stage_cap = 0;
+
+    bool built = false, forces_current = false;
+    int64_t step = 0;
+    int64_t launches = 0;
+    size_t resident = 0;
+    cudaStream_t last_stream = nullptr;
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    bool kernel_timed = false;
+};
+
+namespace mlip {
+
+#define MLIP_CUDA_TRY(ctx, call)                                                          \
+    do {                                                                                  \
+        cudaError_t e_ = (call);                                                          \
+        if (e_ != cudaSuccess) {                                                          \
+            (ctx)->err = std::string(#call) + ": " + cudaGetErrorString(e_);              \
+            return e_ == cudaErrorMemoryAllocation ? MLIP_ERR_OOM : MLIP_ERR_CUDA;        \
+        }                                                                                 \
+    } while (0)
+
+// neighbor.cu
+int launch_pack_source(mlip_ctx *c, const double *pos, const int32_t *species, cudaStream_t s);
+int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s);
+int launch_export(mlip_ctx *c, int64_t *seg_ptr, int32_t *nbr, int64_t capacity, int64_t *n_entries_host, cudaStream_t s);
+// tables.cu
+int build_tables(mlip_ctx *c, const double *enc_w_host, size_t n_enc);
+// megakernel.cu
+int upload_head(mlip_ctx *c, const double *head_w_host);
+int launch_megakernel(mlip_ctx *c, cudaStream_t s);
+// integrate.cu
+int launch_kick_drift(mlip_ctx *c, double dt, cudaStream_t s);
+int launch_kick(mlip_ctx *c, double dt, cudaStream_t s);
+int launch_kinetic(mlip_ctx *c, cudaStream_t s);
+int launch_scatter_forces(mlip_ctx *c, float *forces, float *e_atom, cudaStream_t s);
+int launch_set_positions(mlip_ctx *c, const double *pos, cudaStream_t s);
+int launch_set_velocities(mlip_ctx *c, const double *vel, cudaStream_t s);
+int launch_get_state(mlip_ctx *c, double *pos, double *vel, cudaStream_t s);
+
+// Exact minimum-image squared distance in fp64, every operation rounded on its own
+// (no fused multiply-add), identical on host and device.
+__device__ __forceinline__ double min_image(double d, double box, double half) {
+    if (d > half) d = __dsub_rn(d, box);
+    else if (d < -half) d = __dadd_rn(d, box);
+    return d;
+}
+
+}  // namespace mlip

@@ -1,0 +1,162 @@
+// Velocity-Verlet NVE pieces and the permutation kernels between the caller's atom
+// order and the internal cell-sorted order.  Positions and velocities are fp64: at 8 M atoms
+// the box is ~450 Angstrom and a 1 fs displacement (~1e-3 Angstrom) would lose most of its
+// digits in fp32.
+#include "common.cuh"
+
+namespace mlip {
+
+// v += dt/2 a;  x += dt v;  wrap into [0, L);  track the displacement since the last list build.
+__global__ void k_kick_drift(int64_t n, double dt, CellGrid g, const double *__restrict__ mass, float skin_half2,
+                             double4 *__restrict__ pos4, double *__restrict__ vel, const float4 *__restrict__ force,
+                             float *__restrict__ disp, int *status) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    double4 p = pos4[i];
+    const float4 f = force[i];
+    const double k = 0.5 * dt * ACC_UNIT / mass[(int)p.w];
+    double v[3] = {vel[3 * i] + k * f.x, vel[3 * i + 1] + k * f.y, vel[3 * i + 2] + k * f.z};
+    double x[3] = {p.x + dt * v[0], p.y + dt * v[1], p.z + dt * v[2]};
+    float d2 = 0.f;
+#pragma unroll
+    for (int a = 0; a < 3; ++a) {
+        vel[3 * i + a] = v[a];
+        float d = disp[3 * i + a] + (float)(dt * v[a]);
+        disp[3 * i + a] = d;
+        d2 += d * d;
+        const double L = g.box[a];
+        if (x[a] >= L) x[a] -= L;
+        else if (x[a] < 0.0) x[a] += L;
+        if (!(x[a] >= 0.0 && x[a] < L)) x[a] = 0.0;   // -eps + L rounds to L; NaN is reported below
+    }
+    if (!(d2 <= skin_half2)) atomicOr(status, d2 == d2 ? FLAG_SKIN_EXCEEDED : FLAG_NONFINITE);
+    pos4[i] = make_double4(x[0], x[1], x[2], p.w);
+}
+
+// v += dt/2 a
+__global__ void k_kick(int64_t n, double dt, const double *__restrict__ mass, const double4 *__restrict__ pos4,
+                       double *__restrict__ vel, const float4 *__restrict__ force) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const float4 f = force[i];
+    const double k = 0.5 * dt * ACC_UNIT / mass[(int)pos4[i].w];
+    vel[3 * i] += k * f.x; vel[3 * i + 1] += k * f.y; vel[3 * i + 2] += k * f.z;
+}
+
+__global__ void k_kinetic(int64_t n, const double *__restrict__ mass, const double4 *__restrict__ pos4,
+                          const double *__restrict__ vel, double *acc) {
+    __shared__ double part[32];
+    double e = 0.0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        double vx = vel[3 * i], vy = vel[3 * i + 1], vz = vel[3 * i + 2];
+        e += 0.5 * mass[(int)pos4[i].w] * (vx * vx + vy * vy + vz * vz);
+    }
+    for (int o = 16; o; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = e;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        e = threadIdx.x < (blockDim.x >> 5) ? part[threadIdx.x] : 0.0;
+        for (int o = 16; o; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
+        if (threadIdx.x == 0) atomicAdd(&acc[ACC_KINETIC], e / ACC_UNIT);
+    }
+}
+
+__global__ void k_scatter_forces(int64_t n, const int32_t *__restrict__ user_of, const float4 *__restrict__ force,
+                                 float *__restrict__ forces_out, float *__restrict__ e_atom) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const float4 f = force[i];
+    const int64_t u = user_of[i];
+    if (forces_out) { forces_out[3 * u] = f.x; forces_out[3 * u + 1] = f.y; forces_out[3 * u + 2] = f.z; }
+    if (e_atom) e_atom[u] = f.w;
+}
+
+__global__ void k_set_positions(int64_t n, const int32_t *__restrict__ user_of, const double *__restrict__ pos,
+                                CellGrid g, float skin_half2, double4 *__restrict__ pos4, float *__restrict__ disp, int *status) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int64_t u = user_of[i];
+    double4 p = pos4[i];
+    const double x[3] = {pos[3 * u], pos[3 * u + 1], pos[3 * u + 2]};
+    const double old[3] = {p.x, p.y, p.z};
+    float d2 = 0.f;
+    bool ok = true;
+#pragma unroll
+    for (int a = 0; a < 3; ++a) {
+        ok = ok && (x[a] >= 0.0 && x[a] < g.box[a]);
+        float d = disp[3 * i + a] + (float)min_image(x[a] - old[a], g.box[a], g.half[a]);
+        disp[3 * i + a] = d;
+        d2 += d * d;
+    }
+    if (!ok) atomicOr(status, FLAG_NONFINITE);
+    else if (!(d2 <= skin_half2)) atomicOr(status, FLAG_SKIN_EXCEEDED);
+    pos4[i] = make_double4(x[0], x[1], x[2], p.w);
+}
+
+__global__ void k_set_velocities(int64_t n, const int32_t *__restrict__ user_of, const double *__restrict__ vel_in,
+                                 double *__restrict__ vel) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int64_t u = user_of[i];
+    vel[3 * i] = vel_in[3 * u]; vel[3 * i + 1] = vel_in[3 * u + 1]; vel[3 * i + 2] = vel_in[3 * u + 2];
+}
+
+__global__ void k_get_state(int64_t n, const int32_t *__restrict__ user_of, const double4 *__restrict__ pos4,
+                            const double *__restrict__ vel, double *__restrict__ pos_out, double *__restrict__ vel_out) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int64_t u = user_of[i];
+    if (pos_out) { double4 p = pos4[i]; pos_out[3 * u] = p.x; pos_out[3 * u + 1] = p.y; pos_out[3 * u + 2] = p.z; }
+    if (vel_out) { vel_out[3 * u] = vel[3 * i]; vel_out[3 * u + 1] = vel[3 * i + 1]; vel_out[3 * u + 2] = vel[3 * i + 2]; }
+}
+
+static inline unsigned nb(int64_t n) { return (unsigned)((n + 255) / 256); }
+static inline float skin_half2(const mlip_ctx *c) { float h = 0.5f * (float)c->cfg.skin; return h * h; }
+
+int launch_kick_drift(mlip_ctx *c, double dt, cudaStream_t s) {
+    k_kick_drift<<<nb(c->n), 256, 0, s>>>(c->n, dt, c->grid, c->mass, skin_half2(c), c->pos4, c->vel, c->force, c->disp, c->status);
+    c->launches += 1;
+    MLIP_CUDA_TRY(c, cudaGetLastError());
+    return MLIP_OK;
+}
+int launch_kick(mlip_ctx *c, double dt, cudaStream_t s) {
+    k_kick<<<nb(c->n), 256, 0, s>>>(c->n, dt, c->mass, c->pos4, c->vel, c->force);
+    c->launches += 1;
+    MLIP_CUDA_TRY(c, cudaGetLastError());
+    return MLIP_OK;
+}
+int launch_kinetic(mlip_ctx *c, cudaStream_t s) {
+    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->acc + ACC_KINETIC, 0, sizeof(double), s));
+    int64_t blocks = nb(c->n);
+    if (blocks > 1184) blocks = 1184;
+    k_kinetic<<<(unsigned)blocks, 256, 0, s>>>(c->n, c->mass, c->pos4, c->vel, c->acc);
+    c->launches += 1;
+    MLIP_CUDA_TRY(c, cudaGetLastError());
+    return MLIP_OK;
+}
+int launch_scatter_forces(mlip_ctx *c, float *forces, float *e_atom, cudaStream_t s) {
+    k_scatter_forces<<<nb(c->n), 256, 0, s>>>(c->n, c->user_of, c->force, forces, e_atom);
+    c->launches += 1;
+    MLIP_CUDA_TRY(c, cudaGetLastError());
+    return MLIP_OK;
+}
+int launch_set_positions(mlip_ctx *c, const double *pos, cudaStream_t s) {
+    k_set_positions<<<nb(c->n), 256, 0, s>>>(c->n, c->user_of, pos, c->grid, skin_half2(c), c->pos4, c->disp, c->status);
+    c->launches += 1;
+    MLIP_CUDA_TRY(c, cudaGetLastError());
+    return MLIP_OK;
+}
+int launch_set_velocities(mlip_ctx *c, const double *vel, cudaStream_t s) {
+    k_set_velocities<<<nb(c->n), 256, 0, s>>>(c->n, c->user_of, vel, c->vel);
+    c->launches += 1;
+    MLIP_CUDA_TRY(c, cudaGetLastError());
+    return MLIP_OK;
+}
+int launch_get_state(mlip_ctx *c, double *pos, double *vel, cudaStream_t s) {
+    k_get_state<<<nb(c->n), 256, 0, s>>>(c->n, c->user_of, c->pos4, c->vel, pos, vel);
+    c->launches += 1;
+    MLIP_CUDA_TRY(c, cudaGetLastError());
+    return MLIP_OK;
+}
+
+}  // namespace mlip

@@ -1,0 +1,281 @@
+// Cell binning and neighbor-list construction (Section 3.1.1: N(i) = atoms within a
+// cutoff of atom i; the paper delegates this to the MD code's binning algorithm,
+// Section 4.1.4).  Everything runs on the device:
+//   cell id per atom -> counting sort into cell order (ties broken by species, then by the
+//   caller's index, so the internal order is reproducible) -> per-species processing order
+//   -> two passes (count, fill) of a warp-per-atom scan over the 27 surrounding cells.
+// The inclusion test is fp64 with separately rounded operations, so the set of pairs is
+// identical to a plain CPU evaluation of the same expression.
+#include "common.cuh"
+#include "scan.cuh"
+
+namespace mlip {
+
+__device__ __forceinline__ int cell_coord(double x, double inv_edge, int n) {
+    int c = (int)floor(x * inv_edge);
+    return c < 0 ? 0 : (c >= n ? n - 1 : c);
+}
+
+__global__ void k_pack_source(const double *__restrict__ pos, const int32_t *__restrict__ species, int64_t n,
+                              int n_species, double4 *__restrict__ pos4, int32_t *__restrict__ user, int *status) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    int s = species[i];
+    if (s < 0 || s >= n_species) { atomicOr(status, FLAG_NONFINITE); s = 0; }
+    pos4[i] = make_double4(pos[3 * i], pos[3 * i + 1], pos[3 * i + 2], (double)s);
+    user[i] = (int32_t)i;
+}
+
+__global__ void k_cell_id(const double4 *__restrict__ pos4, int64_t n, CellGrid g, int32_t *__restrict__ cell_of,
+                          int32_t *__restrict__ cell_count, int *status) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    double4 p = pos4[i];
+    bool ok = (p.x >= 0.0 && p.x < g.box[0]) && (p.y >= 0.0 && p.y < g.box[1]) && (p.z >= 0.0 && p.z < g.box[2]);
+    if (!ok) atomicOr(status, FLAG_NONFINITE);
+    int cx = ok ? cell_coord(p.x, g.inv_edge[0], g.n[0]) : 0;
+    int cy = ok ? cell_coord(p.y, g.inv_edge[1], g.n[1]) : 0;
+    int cz = ok ? cell_coord(p.z, g.inv_edge[2], g.n[2]) : 0;
+    int c = (cx * g.n[1] + cy) * g.n[2] + cz;
+    cell_of[i] = c;
+    atomicAdd(&cell_count[c], 1);
+}
+
+__global__ void k_place(const int32_t *__restrict__ cell_of, int64_t n, const int32_t *__restrict__ cell_start,
+                        int32_t *__restrict__ cell_fill, int32_t *__restrict__ slot_src) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    int c = cell_of[i];
+    slot_src[cell_start[c] + atomicAdd(&cell_fill[c], 1)] = (int32_t)i;
+}
+
+// One thread per cell: order the cell's atoms by (species, caller index) and count them per species.
+__global__ void k_sort_cells(int n_cells, int n_species, const int32_t *__restrict__ cell_start,
+                             int32_t *__restrict__ slot_src, const double4 *__restrict__ pos4_src,
+                             const int32_t *__restrict__ user_src, int32_t *__restrict__ bin_count) {
+    int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= n_cells) return;
+    int beg = cell_start[c], end = cell_start[c + 1];
+    int cnt[MAX_SPECIES] = {0};
+    for (int a = beg; a < end; ++a) {
+        int src = slot_src[a];
+        int sa = (int)pos4_src[src].w;
+        long long key = ((long long)sa << 32) | (unsigned)user_src[src];
+        cnt[sa]++;
+        int b = a - 1;
+        while (b >= beg) {
+            int sb_src = slot_src[b];
+            long long kb = ((long long)(int)pos4_src[sb_src].w << 32) | (unsigned)user_src[sb_src];
+            if (kb <= key) break;
+            slot_src[b + 1] = sb_src;
+            --b;
+        }
+        slot_src[b + 1] = src;
+    }
+    for (int s = 0; s < n_species; ++s) bin_count[(int64_t)s * n_cells + c] = cnt[s];
+}
+
+__global__ void k_gather(int64_t n, const int32_t *__restrict__ slot_src, const double4 *__restrict__ pos4_src,
+                         const double *__restrict__ vel_src, const int32_t *__restrict__ user_src,
+                         double4 *__restrict__ pos4, double *__restrict__ vel, int32_t *__restrict__ user_of,
+                         float *__restrict__ disp) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    int src = slot_src[i];
+    pos4[i] = pos4_src[src];
+    user_of[i] = user_src[src];
+    for (int a = 0; a < 3; ++a) {
+        vel[3 * i + a] = vel_src ? vel_src[3 * (int64_t)src + a] : 0.0;
+        disp[3 * i + a] = 0.f;
+    }
+}
+
+// One thread per cell: the cell's atoms (already species-ordered) go to their (species, cell) bins.
+__global__ void k_center_order(int n_cells, int n_species, const int32_t *__restrict__ cell_start,
+                               const double4 *__restrict__ pos4, const int32_t *__restrict__ bin_start,
+                               int32_t *__restrict__ center_order, int32_t *__restrict__ species_start) {
+    int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c <= n_species) species_start[c] = c < n_species ? bin_start[(int64_t)c * n_cells] : bin_start[(int64_t)n_species * n_cells];
+    if (c >= n_cells) return;
+    int beg = cell_start[c], end = cell_start[c + 1];
+    int prev = -1, r = 0;
+    for (int a = beg; a < end; ++a) {
+        int s = (int)pos4[a].w;
+        if (s != prev) { prev = s; r = 0; }
+        center_order[bin_start[(int64_t)s * n_cells + c] + r++] = a;
+    }
+}
+
+// Warp per atom over the surrounding cells.  FILL = false counts, FILL = true writes the list.
+template <bool FILL>
+__global__ void __launch_bounds__(256) k_neighbors(int64_t n, CellGrid g, double rl2, const double4 *__restrict__ pos4,
+                                                   const int32_t *__restrict__ cell_start, int32_t *__restrict__ nbr_count,
+                                                   const int64_t *__restrict__ nbr_off, int32_t *__restrict__ nbr,
+                                                   int64_t nbr_cap, int *status) {
+    const int lane = threadIdx.x & 31;
+    int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (i >= n) return;
+    const double4 pi = pos4[i];
+    int c0[3] = {cell_coord(pi.x, g.inv_edge[0], g.n[0]), cell_coord(pi.y, g.inv_edge[1], g.n[1]),
+                 cell_coord(pi.z, g.inv_edge[2], g.n[2])};
+    int lst[3][3], nl[3];
+#pragma unroll
+    for (int a = 0; a < 3; ++a) {   // distinct periodic cells among c-1, c, c+1
+        int na = g.n[a];
+        nl[a] = na < 3 ? na : 3;
+        for (int o = 0; o < 3; ++o) {
+            int c = c0[a] + o - 1;
+            c = c < 0 ? c + na : (c >= na ? c - na : c);
+            lst[a][o] = c;
+        }
+        if (na == 2) { lst[a][0] = 0; lst[a][1] = 1; }
+        if (na == 1) lst[a][0] = 0;
+    }
+    int64_t off = 0;
+    bool writable = true;
+    if (FILL) {
+        off = nbr_off[i];
+        writable = nbr_off[i + 1] <= nbr_cap;
+        if (!writable && lane == 0) atomicOr(status, FLAG_NEIGHBOR_OVERFLOW);
+    }
+    int cnt = 0;
+    for (int x = 0; x < nl[0]; ++x)
+        for (int y = 0; y < nl[1]; ++y)
+            for (int z = 0; z < nl[2]; ++z) {
+                int c = (lst[0][x] * g.n[1] + lst[1][y]) * g.n[2] + lst[2][z];
+                int beg = cell_start[c], end = cell_start[c + 1];
+                for (int base = beg; base < end; base += 32) {
+                    int j = base + lane;
+                    bool hit = false;
+                    if (j < end && j != i) {
+                        double4 pj = pos4[j];
+                        double dx = min_image(__dsub_rn(pj.x, pi.x), g.box[0], g.half[0]);
+                        double dy = min_image(__dsub_rn(pj.y, pi.y), g.box[1], g.half[1]);
+                        double dz = min_image(__dsub_rn(pj.z, pi.z), g.box[2], g.half[2]);
+                        double d2 = __dadd_rn(__dadd_rn(__dmul_rn(dx, dx), __dmul_rn(dy, dy)), __dmul_rn(dz, dz));
+                        hit = d2 < rl2;
+                    }
+                    unsigned m = __ballot_sync(0xffffffffu, hit);
+                    if (FILL && hit && writable) nbr[off + cnt + __popc(m & ((1u << lane) - 1u))] = j;
+                    cnt += __popc(m);
+                }
+            }
+    if (!FILL && lane == 0) nbr_count[i] = cnt;
+}
+
+// ---- canonical export: caller's indices, species-segmented, ascending ----
+__global__ void k_export_count(int64_t n, int n_species, const int64_t *__restrict__ nbr_off, const int32_t *__restrict__ nbr,
+                               const double4 *__restrict__ pos4, const int32_t *__restrict__ user_of,
+                               int32_t *__restrict__ seg_count) {
+    const int lane = threadIdx.x & 31;
+    int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (i >= n) return;
+    int cnt[MAX_SPECIES] = {0};
+    for (int64_t e = nbr_off[i] + lane; e < nbr_off[i + 1]; e += 32) cnt[(int)pos4[nbr[e]].w]++;
+    int64_t row = (int64_t)user_of[i] * n_species;
+    for (int s = 0; s < n_species; ++s) {
+        int v = cnt[s];
+        for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) seg_count[row + s] = v;
+    }
+}
+
+__global__ void k_export_fill(int64_t n, int n_species, const int64_t *__restrict__ nbr_off, const int32_t *__restrict__ nbr,
+                              const double4 *__restrict__ pos4, const int32_t *__restrict__ user_of,
+                              const int64_t *__restrict__ seg_ptr, int32_t *__restrict__ out) {
+    const int lane = threadIdx.x & 31;
+    int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (i >= n) return;
+    const int64_t beg = nbr_off[i], end = nbr_off[i + 1];
+    const int64_t row = (int64_t)user_of[i] * n_species;
+    for (int64_t e = beg + lane; e < end; e += 32) {
+        int j = nbr[e];
+        int sj = (int)pos4[j].w, uj = user_of[j];
+        int rank = 0;   // entries of the same species with a smaller caller index
+        for (int64_t f = beg; f < end; ++f) {
+            int jf = nbr[f];
+            rank += ((int)pos4[jf].w == sj) && (user_of[jf] < uj);
+        }
+        out[seg_ptr[row + sj] + rank] = uj;
+    }
+}
+
+static inline unsigned blocks_for(int64_t n, int per_block) { return (unsigned)((n + per_block - 1) / per_block); }
+
+int launch_pack_source(mlip_ctx *c, const double *pos, const int32_t *species, cudaStream_t s) {
+    k_pack_source<<<blocks_for(c->n, 256), 256, 0, s>>>(pos, species, c->n, c->cfg.n_species, c->pos4_src, c->user_src, c->status);
+    c->launches += 1;
+    MLIP_CUDA_TRY(c, cudaGetLastError());
+    return MLIP_OK;
+}
+
+// Sort (pos4_src, vel_src, user_src) into cell order and build the lists.
+int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
+    const int64_t n = c->n;
+    const CellGrid &g = c->grid;
+    const int C = c->cfg.n_species;
+    const double rl = c->cfg.r_cut + c->cfg.skin;
+    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->cell_count, 0, sizeof(int32_t) * (g.n_cells + 1), s));
+    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->cell_fill, 0, sizeof(int32_t) * (g.n_cells + 1), s));
+    k_cell_id<<<blocks_for(n, 256), 256, 0, s>>>(c->pos4_src, n, g, c->cell_of, c->cell_count, c->status);
+    exclusive_scan<int32_t, int32_t>(c->cell_count, c->cell_start, g.n_cells, c->scan_tmp, s);
+    // nbr_count doubles as the slot -> source map until the lists are counted
+    int32_t *slot_src = c->nbr_count;
+    k_place<<<blocks_for(n, 256), 256, 0, s>>>(c->cell_of, n, c->cell_start, c->cell_fill, slot_src);
+    k_sort_cells<<<blocks_for(g.n_cells, 128), 128, 0, s>>>(g.n_cells, C, c->cell_start, slot_src, c->pos4_src, c->user_src, c->bin_count);
+    k_gather<<<blocks_for(n, 256), 256, 0, s>>>(n, slot_src, c->pos4_src, c->vel_src, c->user_src, c->pos4, c->vel, c->user_of, c->disp);
+    exclusive_scan<int32_t, int32_t>(c->bin_count, c->bin_start, (int64_t)C * g.n_cells, c->scan_tmp, s);
+    int nthreads_co = g.n_cells > C + 1 ? g.n_cells : C + 1;
+    k_center_order<<<blocks_for(nthreads_co, 128), 128, 0, s>>>(g.n_cells, C, c->cell_start, c->pos4, c->bin_start, c->center_order, c->species_start);
+    k_neighbors<false><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, c->cell_start, c->nbr_count, nullptr, nullptr, 0, c->status);
+    exclusive_scan<int32_t, int64_t>(c->nbr_count, c->nbr_off, n, c->scan_tmp, s);
+    c->launches += 7 + 9;
+    MLIP_CUDA_TRY(c, cudaGetLastError());
+    if (allow_sync_grow) {
+        MLIP_CUDA_TRY(c, cudaMemcpyAsync(c->total_host, c->nbr_off + n, sizeof(int64_t), cudaMemcpyDeviceToHost, s));
+        MLIP_CUDA_TRY(c, cudaStreamSynchronize(s));
+        c->n_entries = *c->total_host;
+        if (c->n_entries > c->nbr_cap) {
+            int64_t want = c->n_entries + c->n_entries / 8 + 1024;
+            if (c->nbr) { cudaFree(c->nbr); c->resident -= sizeof(int32_t) * c->nbr_cap; c->nbr = nullptr; c->nbr_cap = 0; }
+            MLIP_CUDA_TRY(c, cudaMalloc(&c->nbr, sizeof(int32_t) * want));
+            c->nbr_cap = want;
+            c->resident += sizeof(int32_t) * want;
+        }
+    }
+    k_neighbors<true><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, c->cell_start, c->nbr_count, c->nbr_off, c->nbr, c->nbr_cap, c->status);
+    c->launches += 1;
+    MLIP_CUDA_TRY(c, cudaGetLastError());
+    return MLIP_OK;
+}
+
+int launch_export(mlip_ctx *c, int64_t *seg_ptr, int32_t *nbr, int64_t capacity, int64_t *n_entries_host, cudaStream_t s) {
+    const int64_t n = c->n;
+    const int C = c->cfg.n_species;
+    // seg counts live temporarily in the bin_count-sized scratch? They need N*C ints: use a fresh buffer.
+    int32_t *seg_count = nullptr;
+    MLIP_CUDA_TRY(c, cudaMalloc(&seg_count, sizeof(int32_t) * (size_t)(n * C + 1)));
+    int64_t *tmp = nullptr;
+    MLIP_CUDA_TRY(c, cudaMalloc(&tmp, sizeof(int64_t) * (size_t)scan_tmp_items(n * C)));
+    k_export_count<<<blocks_for(n * 32, 256), 256, 0, s>>>(n, C, c->nbr_off, c->nbr, c->pos4, c->user_of, seg_count);
+    exclusive_scan<int32_t, int64_t>(seg_count, seg_ptr, n * C, tmp, s);
+    int rc = MLIP_OK;
+    cudaError_t e = cudaMemcpyAsync(c->total_host, seg_ptr + n * C, sizeof(int64_t), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e == cudaSuccess) {
+        if (n_entries_host) *n_entries_host = *c->total_host;
+        if (*c->total_host > capacity || !nbr) rc = MLIP_ERR_NEIGHBOR_OVERFLOW;
+        else {
+            k_export_fill<<<blocks_for(n * 32, 256), 256, 0, s>>>(n, C, c->nbr_off, c->nbr, c->pos4, c->user_of, seg_ptr, nbr);
+            e = cudaStreamSynchronize(s);
+        }
+    }
+    c->launches += 5;
+    cudaFree(seg_count);
+    cudaFree(tmp);
+    if (e != cudaSuccess) { c->err = cudaGetErrorString(e); return MLIP_ERR_CUDA; }
+    if (rc != MLIP_OK) c->err = "neighbor export: capacity too small";
+    return rc;
+}
+
+}  // namespace mlip

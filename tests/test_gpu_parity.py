@@ -1,0 +1,161 @@
+"""CUDA path vs the CPU oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+
+import oracle
+from helpers import canonical_equal, make_pair
+
+pytestmark = pytest.mark.gpu
+
+# fp32 kernel: energy to 1e-6 relative, forces to 1e-4 eV/Angstrom max-abs (spec tolerances)
+E_RTOL, F_ATOL = 1e-6, 1e-4
+
+
+@pytest.mark.parametrize("cfg,n_cells,skin", [(1, 4, 0.0), (1, 5, 1.0), (2, 6, 1.0), (3, 5, 1.0), (4, 8, 1.0), (5, 6, 1.0)])
+def test_neighbor_lists_bit_exact(cfg, n_cells, skin):
+    w, model, pot = make_pair(cfg, n_cells, skin)
+    pot.build_neighbors(w.pos, w.species, w.box)
+    seg, nbr = pot.neighbors()
+    pot.sync_status()
+    nl = oracle.neighbors(w.pos, w.species, w.n_species, w.box, w.r_cut + w.skin, method="brute" if w.n_atoms <= 1100 else "cell")
+    assert canonical_equal(nl, seg, nbr)
+
+
+def test_neighbor_lists_non_cubic_random_gas():
+    import paper_2608_16329_b200 as mlip
+    from paper_2608_16329_b200 import workloads as wl
+    rng = np.random.default_rng(3)
+    box = np.array([15.0, 21.5, 29.0])
+    pos = rng.uniform(0, 1, (3000, 3)) * box
+    species = rng.integers(0, 4, 3000).astype(np.int32)
+    enc, head = wl.make_weights(4, seed=1)
+    pot = mlip.Potential(4, 6.0, 1.0, enc, head, np.ones(4), table_tol=1.0)
+    pot.build_neighbors(pos, species, box)
+    seg, nbr = pot.neighbors()
+    nl = oracle.neighbors(pos, species, 4, box, 7.0)
+    assert canonical_equal(nl, seg, nbr)
+
+
+@pytest.mark.parametrize("cfg,n_cells,skin", [(1, 4, 0.0), (5, 6, 1.0), (2, 6, 1.0), (3, 5, 1.0), (4, 8, 1.0)])
+def test_energy_forces_virial_match_oracle(cfg, n_cells, skin):
+    w, model, pot = make_pair(cfg, n_cells, skin)
+    pot.build_neighbors(w.pos, w.species, w.box)
+    out = pot.compute(want_e_atom=True)
+    pot.sync_status()
+    ref = oracle.evaluate(model, w.pos, w.species, w.box)
+    e = float(out["energy"].cpu())
+    f = out["forces"].cpu().numpy().astype(np.float64)
+    ea = out["e_atom"].cpu().numpy().astype(np.float64)
+    xi = out["virial"].cpu().numpy().reshape(3, 3)
+    print(f"cfg {cfg}: N={w.n_atoms} E={e:.6f} rel dE={abs(e - ref['energy']) / abs(ref['energy']):.2e} "
+          f"max|dF|={np.abs(f - ref['forces']).max():.2e} max|dE_i|={np.abs(ea - ref['e_atom']).max():.2e} "
+          f"table err={pot_table(pot)}")
+    assert abs(e - ref["energy"]) <= E_RTOL * abs(ref["energy"])
+    assert np.abs(f - ref["forces"]).max() <= F_ATOL
+    assert np.abs(ea - ref["e_atom"]).max() <= 2e-5 * max(1.0, np.abs(ref["e_atom"]).max())
+    assert np.abs(xi - ref["virial"]).max() <= 1e-5 * np.abs(ref["virial"]).max()
+    assert abs(f.sum(0)).max() < 1e-2
+
+
+def pot_table(pot):
+    import paper_2608_16329_b200 as mlip
+    return tuple(f"{x:.1e}" for x in mlip.mlip_table_error(pot.ctx))
+
+
+def test_results_are_returned_in_the_callers_order():
+    w, model, pot = make_pair(1, 4, 0.0)
+    perm = np.random.default_rng(0).permutation(w.n_atoms)
+    pot.build_neighbors(w.pos, w.species, w.box)
+    a = pot.compute()["forces"].cpu().numpy()
+    pot.build_neighbors(w.pos[perm], w.species[perm], w.box)
+    b = pot.compute()["forces"].cpu().numpy()
+    assert np.abs(a[perm] - b).max() < 2e-5
+
+
+def test_set_positions_keeps_lists_and_matches_oracle():
+    w, model, pot = make_pair(5, 6, 1.0)
+    pot.build_neighbors(w.pos, w.species, w.box)
+    rng = np.random.default_rng(1)
+    pos = w.pos + rng.uniform(-0.2, 0.2, w.pos.shape)
+    pos -= np.floor(pos / w.box) * w.box
+    pot.set_positions(pos)
+    out = pot.compute()
+    pot.sync_status()
+    ref = oracle.evaluate(model, pos, w.species, w.box)
+    assert np.abs(out["forces"].cpu().numpy() - ref["forces"]).max() <= F_ATOL
+    assert abs(float(out["energy"].cpu()) - ref["energy"]) <= E_RTOL * abs(ref["energy"])
+
+
+def test_compute_host_matches_device_entry():
+    import paper_2608_16329_b200 as mlip
+    w, model, pot = make_pair(5, 6, 1.0)
+    pot.build_neighbors(w.pos, w.species, w.box)
+    dev = pot.compute()
+    f = np.zeros((w.n_atoms, 3), dtype=np.float32)
+    xi = np.zeros(9)
+    e = mlip.mlip_compute_host(pot.ctx, w.pos, w.species, w.box, True, f, xi)
+    assert abs(e - float(dev["energy"].cpu())) < 1e-9 * abs(e)
+    assert np.abs(f - dev["forces"].cpu().numpy()).max() < 2e-5
+    e2 = mlip.mlip_compute_host(pot.ctx, w.pos, None, None, False, f, xi)
+    assert abs(e2 - e) < 1e-9 * abs(e)
+
+
+def test_nve_tracks_the_oracle_and_conserves_energy():
+    w, model, pot = make_pair(2, 6, 1.0)
+    pot.build_neighbors(w.pos, w.species, w.box)
+    pot.set_velocities(w.vel)
+    pot.compute()
+    e0 = pot.energies().cpu().numpy()
+    ref = oracle.nve(model, w.pos, w.vel, w.species, w.masses, w.box, 10, 1.0, r_list=w.r_cut + w.skin, rebuild_every=5)
+    assert abs(e0[1] - ref["e_kin"][0]) < 1e-9 * ref["e_kin"][0]
+    pot.step(10, 1.0, 5)
+    pot.sync_status()
+    pos, vel, step = pot.state()
+    e1 = pot.energies().cpu().numpy()
+    assert step == 10
+    d = pos.cpu().numpy() - ref["pos"]
+    d -= w.box * np.round(d / w.box)
+    assert np.abs(d).max() < 1e-6
+    assert np.abs(vel.cpu().numpy() - ref["vel"]).max() < 1e-7
+    assert abs(e1.sum() - e0.sum()) < 5e-3 * np.ptp(ref["e_kin"]) + 1e-6 * abs(e0[0])
+    # 40 more steps: total energy stays put while kinetic and potential energy exchange
+    pot.step(40, 1.0, 10)
+    pot.sync_status()
+    e2 = pot.energies().cpu().numpy()
+    assert abs(e2.sum() - e0.sum()) < 0.02 * abs(e2[1] - e0[1]) + 2e-6 * abs(e0[0])
+
+
+def test_device_side_problems_become_status_codes():
+    import paper_2608_16329_b200 as mlip
+    C = mlip.binding.CODES
+    w, model, pot = make_pair(5, 6, 1.0)
+    with pytest.raises(mlip.MlipError) as err:
+        pot.compute()
+    assert err.value.code == C["MLIP_ERR_NOT_BUILT"]
+    with pytest.raises(mlip.MlipError) as err:
+        pot.build_neighbors(w.pos, w.species, np.array([10.0, 30.0, 30.0]))
+    assert err.value.code == C["MLIP_ERR_BOX_TOO_SMALL"]
+    bad = w.pos.copy(); bad[5, 1] = np.nan
+    pot.build_neighbors(bad, w.species, w.box)
+    assert pot.sync_status(raise_on_error=False) == C["MLIP_ERR_NONFINITE"]
+    pot.build_neighbors(w.pos, w.species, w.box)
+    assert pot.sync_status(raise_on_error=False) == C["MLIP_OK"]
+    moved = w.pos.copy(); moved[7] += 0.9; moved -= np.floor(moved / w.box) * w.box
+    pot.set_positions(moved)
+    assert pot.sync_status(raise_on_error=False) == C["MLIP_ERR_SKIN_EXCEEDED"]
+    close = w.pos.copy(); close[1] = close[0] + np.array([0.3, 0.0, 0.0]); close -= np.floor(close / w.box) * w.box
+    pot.build_neighbors(close, w.species, w.box)
+    pot.compute()
+    assert pot.sync_status(raise_on_error=False) == C["MLIP_ERR_TABLE_RANGE"]
+
+
+def test_table_tolerance_is_enforced():
+    import paper_2608_16329_b200 as mlip
+    from paper_2608_16329_b200 import workloads as wl
+    enc, head = wl.workload_weights(5, 6)
+    with pytest.raises(mlip.MlipError) as err:
+        mlip.Potential(6, 6.0, 1.0, enc, head, np.ones(6), table_knots=8)
+    assert err.value.code == mlip.binding.CODES["MLIP_ERR_TABLE_TOLERANCE"]
+    pot = mlip.Potential(6, 6.0, 1.0, enc, head, np.ones(6))
+    ev, ed = mlip.mlip_table_error(pot.ctx)
+    assert ev < 1e-6
