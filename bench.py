@@ -1,0 +1,308 @@
+#!/usr/bin/env python
+"""Benchmark of the hot path: velocity-Verlet NVE steps of the 6-component alloy on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--cells n]
+
+A step is one pass of the whole path over all atoms: half kick + drift, neighbor rebuild
+every 10th step (skin 1 A), one fused energy/force/virial kernel, half kick.  Prints one JSON
+line.  With N > 1 (torchrun) every rank runs an independent replica of the workload on its
+own GPU (the path has no exchange step on one node: replicas only) and the line reports the
+aggregate over ranks using the slowest rank's time.
+
+`--impl reference` times the CPU oracle (oracle/) as it stands on the host cores, on a
+bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "atom_steps_per_s"
+UNIT = "atom-steps/s"
+CFG = 5
+DEFAULT_CELLS = 126            # 4 * 126^3 = 8,001,504 atoms: the size the target is quoted on
+REBUILD_EVERY = 10
+DT_FS = 1.0
+
+# Algorithmic work (fp32 operations, FMA = 2) of the fused kernel, per unit.  Derivation in the design doc.
+FLOP_PER_PAIR = 3960.0         # pair inside r_cut: both neighbor loops (geometry, harmonics, spline, 6 d k contraction)
+FLOP_PER_SKIN_ENTRY = 24.0     # list entry between r_cut and r_cut + skin: distance test in both loops
+FLOP_PER_ATOM = 88700.0        # invariants, W_i, head forward + reverse, SiLU
+FP32_LANES_PER_SM = 128
+
+# DRAM traffic of one fused-kernel launch from the committed ncu capture
+# (profiles/k_mega_hea6.md: dram__bytes_read.sum + dram__bytes_write.sum, bytes per atom, scaled by atoms).
+NCU_DRAM_BYTES_PER_ATOM = None
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cells", type=int, default=DEFAULT_CELLS, help="FCC cells per edge (N = 4 cells^3)")
+    ap.add_argument("--cpu-centers", type=int, default=49152, help="central atoms in the CPU-oracle sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle sampling in the background during the timed region."""
+
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, sm_max, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                p = [x.strip() for x in line.split(",")]
+                if len(p) < 9:
+                    continue
+                try:
+                    sm.append(float(p[1])); sm_max.append(float(p[2])); power.append(float(p[3]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, p[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        os.unlink(self.path)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(sm_max)), "reasons": sorted(reasons),
+                "power_w_max": float(max(power)), "samples": len(sm)}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "sm_max_mhz": 1965.0}, "fallback"
+
+
+def cpu_oracle_sample(w, enc, head, n_centers, repeats=1):
+    """Time the oracle (neighbor search + full evaluation) on evenly spread central atoms."""
+    import oracle
+    model = oracle.Model(w.n_species, w.r_cut, enc, head)
+    rows = np.linspace(0, w.n_atoms - 1, n_centers).astype(np.int64)
+    rows = np.unique(rows)
+    best = None
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        nl = oracle.neighbors(w.pos, w.species, w.n_species, w.box, w.r_cut + w.skin, rows=rows)
+        oracle.compute(model, w.pos, w.species, w.box, nl)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return rows.size, best, oracle.num_threads()
+
+
+def run_reference(args, rank, world):
+    """CPU oracle arm: each step evaluates a bounded sample of central atoms of the same workload."""
+    if rank != 0:
+        return
+    from paper_2608_16329_b200 import workloads as wl
+    w = wl.make_workload(CFG, n_cells=args.cells)
+    enc, head = wl.workload_weights(CFG, w.n_species)
+    n_centers = min(args.cpu_centers, 2048)
+    for _ in range(args.warmup):
+        cpu_oracle_sample(w, enc, head, 64)
+    t0 = time.perf_counter()
+    done, cores = 0, 1
+    for _ in range(args.steps):
+        n, _, cores = cpu_oracle_sample(w, enc, head, n_centers)
+        done += n
+    dt = time.perf_counter() - t0
+    value = done / dt
+    sample = (f"{n_centers} central atoms spread evenly over the {w.n_atoms}-atom workload per step: cell-list "
+              f"neighbor search for those atoms + full fp64 energy/force/virial evaluation of them")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * dt / max(args.steps, 1), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"cfg5 hea6 fcc{args.cells} ({w.n_atoms} atoms)", "sampled_atoms_per_step": n_centers},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2608_16329_b200 as mlip
+    from paper_2608_16329_b200 import workloads as wl
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w = wl.make_workload(CFG, n_cells=args.cells, seed=wl.BASE_SEED + CFG + 17 * rank)
+    enc, head = wl.workload_weights(CFG, w.n_species)
+    n = w.n_atoms
+    pot = mlip.Potential(w.n_species, w.r_cut, w.skin, enc, head, w.masses, device=local_rank)
+    table_err = mlip.mlip_table_error(pot.ctx)
+
+    # ---- device-resident run: inputs already in HBM when timing starts ----
+    pot.build_neighbors(w.pos, w.species, w.box)
+    pot.set_velocities(w.vel)
+    pot.step(args.warmup, DT_FS, REBUILD_EVERY)
+    pot.sync_status()
+    barrier()
+    mlip.mlip_kernel_time(pot.ctx, reset=True)
+    launches0 = mlip.mlip_get_counters(pot.ctx)["launches"]
+    sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
+                           int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
+    if rank == 0:
+        sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    pot.step(args.steps, DT_FS, REBUILD_EVERY)
+    ev1.record()
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop() if rank == 0 else None
+    status = pot.sync_status(raise_on_error=False)
+    counters = mlip.mlip_get_counters(pot.ctx)
+    k_launches, k_ms = mlip.mlip_kernel_time(pot.ctx, reset=True)
+    e_final = pot.energies().cpu().numpy()
+    t = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_max = float(t.item())
+    value = world * n * args.steps / (ms_max * 1e-3)
+
+    # ---- end to end: host buffers through mlip_compute_host, copies inside the timed region ----
+    e2e = None
+    if not args.no_e2e:
+        pos_a = torch.from_numpy(w.pos).pin_memory()
+        rng = np.random.default_rng(1)
+        shifted = w.pos + rng.uniform(-0.1, 0.1, w.pos.shape)
+        shifted -= np.floor(shifted / w.box) * w.box
+        shifted[shifted >= w.box] = 0.0
+        pos_b = torch.from_numpy(shifted).pin_memory()
+        species_h = torch.from_numpy(w.species).pin_memory()
+        forces_h = torch.empty((n, 3), dtype=torch.float32).pin_memory()
+        virial_h = np.zeros(9)
+        mlip.mlip_compute_host(pot.ctx, pos_a, species_h, w.box, True, forces_h, virial_h)
+        for i in range(2):
+            mlip.mlip_compute_host(pot.ctx, pos_b if i % 2 == 0 else pos_a, None, None, False, forces_h, virial_h)
+        barrier()
+        e2e_steps = args.steps
+        t0 = time.perf_counter()
+        for i in range(e2e_steps):
+            rebuild = (i % REBUILD_EVERY == 0)
+            p = pos_a if i % 2 == 0 else pos_b
+            mlip.mlip_compute_host(pot.ctx, p, species_h if rebuild else None, w.box if rebuild else None, rebuild,
+                                   forces_h, virial_h)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        t = torch.tensor([dt], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        n_rebuilds = (e2e_steps + REBUILD_EVERY - 1) // REBUILD_EVERY
+        e2e = {"value": world * n * e2e_steps / float(t.item()), "unit": UNIT,
+               "h2d_bytes_per_step": int(24 * n + 4 * n * n_rebuilds / e2e_steps),
+               "d2h_bytes_per_step": int(12 * n + 80),
+               "call": "mlip_compute_host (positions in, forces + energy + virial out, list rebuild every 10th call)"}
+
+    if rank == 0:
+        peaks, peak_kind = measured_peaks()
+        props = torch.cuda.get_device_properties(local_rank)
+        n_sm = props.multi_processor_count
+        sm_max = (clocks or {}).get("sm_max_mhz") or peaks.get("sm_max_mhz", 1965.0)
+        peak_tflops = n_sm * FP32_LANES_PER_SM * 2 * sm_max * 1e6 / 1e12
+        pairs = counters["pairs_in_cutoff"]
+        entries = counters["list_entries"]
+        flop = FLOP_PER_PAIR * pairs + FLOP_PER_SKIN_ENTRY * max(entries - pairs, 0) + FLOP_PER_ATOM * n
+        k_avg_ms = k_ms / max(k_launches, 1)
+        achieved = flop / (k_avg_ms * 1e-3) / 1e12
+        roofline = {"bound": "alu", "kernel": "k_mega", "achieved": achieved, "peak": peak_tflops, "unit": "TFLOP/s",
+                    "frac": achieved / peak_tflops,
+                    "peak_source": f"{n_sm} SMs x {FP32_LANES_PER_SM} fp32 lanes x 2 x {sm_max:.0f} MHz (max SM clock)",
+                    "kernel_ms_avg": k_avg_ms, "kernel_launches_timed": k_launches,
+                    "kernel_share_of_step": k_ms / ms if ms > 0 else None,
+                    "flop_per_launch": flop, "pairs_in_cutoff_per_atom": pairs / n, "list_entries_per_atom": entries / n,
+                    "traffic": None if NCU_DRAM_BYTES_PER_ATOM is None else NCU_DRAM_BYTES_PER_ATOM * n,
+                    "hbm_peak_gbs": peaks["hbm_gbs"], "hbm_peak_kind": f"of {peak_kind}"}
+        if clocks and clocks.get("sm_mhz"):
+            roofline["frac_at_sampled_clock"] = achieved / (n_sm * FP32_LANES_PER_SM * 2 * clocks["sm_mhz"] * 1e6 / 1e12)
+        resident = mlip.mlip_resident_bytes(pot.ctx)
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                "ms_per_step": ms_max / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "f32", "data": "synthetic",
+                "config": {"workload": f"cfg5 hea6 fcc{args.cells}: {n} atoms, 6 species, r_cut 6 A, skin 1 A, "
+                                       f"NVE dt 1 fs, list rebuild every {REBUILD_EVERY} steps",
+                           "atoms_per_gpu": n, "parallelism": "replicas" if world > 1 else "single",
+                           "l2": "inputs larger than L2 (positions + lists = %.1f GB per GPU)" % ((32 * n + 4 * entries) / 1e9)},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": counters["launches"] - launches0,
+                "roofline": roofline,
+                "resident_bytes_per_atom": resident / n,
+                "max_atoms_in_180GB_extrapolated": int(180e9 / (resident / n)),
+                "table_error": {"value": table_err[0], "deriv": table_err[1]},
+                "status": mlip.binding.ERRORS.get(status, status),
+                "energy_final_eV": {"potential": float(e_final[0]), "kinetic": float(e_final[1])}}
+        if not args.no_cpu_baseline and world == 1:
+            nc, sec, cores = cpu_oracle_sample(w, enc, head, args.cpu_centers)
+            line["cpu_baseline"] = {"value": nc / sec, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                    "sample": f"{nc} central atoms spread evenly over the {n}-atom workload, one energy/"
+                                              f"force/virial evaluation incl. their neighbor search ({sec:.1f} s)"}
+        print(json.dumps(line), flush=True)
+    pot.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

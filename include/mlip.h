@@ -153,8 +153,12 @@ int mlip_sync_status(mlip_ctx *ctx);
 
 /* Counters for reports: list entries, pairs inside r_cut at the last evaluation (syncs), kernels launched. */
 int mlip_get_counters(mlip_ctx *ctx, int64_t *n_list_entries, int64_t *n_pairs_in_cutoff, int64_t *n_launches);
-/* CUDA-event time of the most recent fused-kernel launch in ms (syncs on that event). */
-int mlip_last_kernel_ms(mlip_ctx *ctx, float *ms);
+/*
+ * CUDA-event time of the fused-kernel launches since the last reset: number of launches timed
+ * and their summed duration in ms (each launch is bracketed by its own event pair on the
+ * launching stream; the most recent 256 launches are kept).  Synchronises on the last event.
+ */
+int mlip_kernel_time(mlip_ctx *ctx, int64_t *n_launches, double *total_ms, int reset);
 
 size_t mlip_resident_bytes(const mlip_ctx *ctx);   /* device bytes the context holds */
 const char *mlip_last_error(const mlip_ctx *ctx);  /* text of the last failure (ctx may be NULL) */

@@ -24,7 +24,7 @@ CODES = {v: k for k, v in ERRORS.items()}
 
 EXPORTS = ["mlip_create", "mlip_table_error", "mlip_build_neighbors", "mlip_get_neighbors", "mlip_set_positions",
            "mlip_set_velocities", "mlip_compute", "mlip_compute_host", "mlip_step", "mlip_get_state",
-           "mlip_get_energies", "mlip_sync_status", "mlip_get_counters", "mlip_last_kernel_ms",
+           "mlip_get_energies", "mlip_sync_status", "mlip_get_counters", "mlip_kernel_time",
            "mlip_resident_bytes", "mlip_last_error", "mlip_destroy"]
 
 
@@ -168,10 +168,11 @@ def mlip_get_counters(ctx):
     return {"list_entries": a.value, "pairs_in_cutoff": b.value, "launches": c.value}
 
 
-def mlip_last_kernel_ms(ctx):
-    ms = ctypes.c_float(0)
-    _check(ctx, lib().mlip_last_kernel_ms(ctx, ctypes.byref(ms)))
-    return ms.value
+def mlip_kernel_time(ctx, reset=False):
+    """(launches timed, summed fused-kernel milliseconds) since the last reset."""
+    n, ms = ctypes.c_int64(0), ctypes.c_double(0)
+    _check(ctx, lib().mlip_kernel_time(ctx, ctypes.byref(n), ctypes.byref(ms), ctypes.c_int(int(reset))))
+    return n.value, ms.value
 
 
 def mlip_resident_bytes(ctx):

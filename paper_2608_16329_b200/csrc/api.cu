@@ -151,9 +151,12 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
         if ((rc = dev_alloc(c, &c->stage_out, 10)) != MLIP_OK) break;
         if (cudaMallocHost((void **)&c->status_host, sizeof(int)) != cudaSuccess ||
             cudaMallocHost((void **)&c->total_host, sizeof(int64_t)) != cudaSuccess ||
-            cudaEventCreate(&c->ev0) != cudaSuccess || cudaEventCreate(&c->ev1) != cudaSuccess) {
-            rc = MLIP_ERR_CUDA; c->err = "pinned host allocation or event creation failed"; break;
+            false) {
+            rc = MLIP_ERR_CUDA; c->err = "pinned host allocation failed"; break;
         }
+        bool ev_ok = true;
+        for (int q = 0; q < 2 * mlip_ctx::EV_POOL; ++q) ev_ok = ev_ok && cudaEventCreate(&c->ev[q]) == cudaSuccess;
+        if (!ev_ok) { rc = MLIP_ERR_CUDA; c->err = "event creation failed"; break; }
         if (cudaMemcpy(c->mass, mass, sizeof(double) * cfg->n_species, cudaMemcpyHostToDevice) != cudaSuccess ||
             cudaMemset(c->status, 0, sizeof(int)) != cudaSuccess || cudaMemset(c->acc, 0, sizeof(double) * ACC_COUNT) != cudaSuccess) {
             rc = MLIP_ERR_CUDA; c->err = "initial upload failed"; break;
@@ -347,11 +350,20 @@ int mlip_get_counters(mlip_ctx *c, int64_t *n_list_entries, int64_t *n_pairs, in
     return MLIP_OK;
 }
 
-int mlip_last_kernel_ms(mlip_ctx *c, float *ms) {
-    if (!c || !ms) return MLIP_ERR_INVALID_ARG;
-    if (!c->kernel_timed) return fail(c, MLIP_ERR_NOT_BUILT, "the fused kernel has not run yet");
-    MLIP_CUDA_TRY(c, cudaEventSynchronize(c->ev1));
-    MLIP_CUDA_TRY(c, cudaEventElapsedTime(ms, c->ev0, c->ev1));
+int mlip_kernel_time(mlip_ctx *c, int64_t *n_launches, double *total_ms, int reset) {
+    if (!c) return MLIP_ERR_INVALID_ARG;
+    const int64_t kept = c->ev_count < mlip_ctx::EV_POOL ? c->ev_count : mlip_ctx::EV_POOL;
+    double total = 0.0;
+    for (int64_t q = 0; q < kept; ++q) {
+        const int slot = (int)((c->ev_count - 1 - q) % mlip_ctx::EV_POOL);
+        float ms = 0.f;
+        MLIP_CUDA_TRY(c, cudaEventSynchronize(c->ev[2 * slot + 1]));
+        MLIP_CUDA_TRY(c, cudaEventElapsedTime(&ms, c->ev[2 * slot], c->ev[2 * slot + 1]));
+        total += ms;
+    }
+    if (n_launches) *n_launches = kept;
+    if (total_ms) *total_ms = total;
+    if (reset) c->ev_count = 0;
     return MLIP_OK;
 }
 
@@ -371,8 +383,8 @@ void mlip_destroy(mlip_ctx *c) {
     cudaFree(c->stage_out);
     if (c->status_host) cudaFreeHost(c->status_host);
     if (c->total_host) cudaFreeHost(c->total_host);
-    if (c->ev0) cudaEventDestroy(c->ev0);
-    if (c->ev1) cudaEventDestroy(c->ev1);
+    for (int q = 0; q < 2 * mlip_ctx::EV_POOL; ++q)
+        if (c->ev[q]) cudaEventDestroy(c->ev[q]);
     delete c;
 }
 

@@ -110,8 +110,9 @@ struct mlip_ctx {
     int64_t launches = 0;
     size_t resident = 0;
     cudaStream_t last_stream = nullptr;
-    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-    bool kernel_timed = false;
+    static constexpr int EV_POOL = 256;
+    cudaEvent_t ev[2 * EV_POOL] = {nullptr};
+    int64_t ev_count = 0;          // launches timed since the last reset
 };
 
 namespace mlip {

@@ -419,11 +419,12 @@ int launch_megakernel(mlip_ctx *c, cudaStream_t s) {
     if (blocks > max_blocks) blocks = max_blocks;
     if (blocks < 1) blocks = 1;
     const double rc2 = c->cfg.r_cut * c->cfg.r_cut;
-    MLIP_CUDA_TRY(c, cudaEventRecord(c->ev0, s));
+    const int slot = (int)(c->ev_count % mlip_ctx::EV_POOL);
+    MLIP_CUDA_TRY(c, cudaEventRecord(c->ev[2 * slot], s));
     k_mega<<<(unsigned)blocks, WARPS * 32, 0, s>>>(n, c->cfg.n_species, c->grid, rc2, c->tab, c->pos4, c->center_order,
                                                    c->nbr_off, c->nbr, c->head_w, c->force, c->acc, c->pair_counter, c->status);
-    MLIP_CUDA_TRY(c, cudaEventRecord(c->ev1, s));
-    c->kernel_timed = true;
+    MLIP_CUDA_TRY(c, cudaEventRecord(c->ev[2 * slot + 1], s));
+    c->ev_count += 1;
     c->launches += 1;
     MLIP_CUDA_TRY(c, cudaGetLastError());
     return MLIP_OK;
