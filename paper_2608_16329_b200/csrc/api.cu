@@ -44,7 +44,7 @@ static void free_atoms(mlip_ctx *c) {
     dev_free(c, &c->pos4, n); dev_free(c, &c->pos4_src, n);
     dev_free(c, &c->vel, 3 * n); dev_free(c, &c->vel_src, 3 * n);
     dev_free(c, &c->user_of, n); dev_free(c, &c->user_src, n);
-    dev_free(c, &c->force, n); dev_free(c, &c->disp, 3 * n);
+    dev_free(c, &c->force, n); dev_free(c, &c->disp, 3 * n); dev_free(c, &c->e_atom, n);
     dev_free(c, &c->center_order, n); dev_free(c, &c->cell_of, n);
     dev_free(c, &c->nbr_count, n); dev_free(c, &c->nbr_off, n + 1);
     c->cap_atoms = 0;
@@ -66,7 +66,7 @@ static int ensure_capacity(mlip_ctx *c, int64_t n, int64_t n_cells) {
         TRY_ALLOC(c->pos4, m); TRY_ALLOC(c->pos4_src, m);
         TRY_ALLOC(c->vel, 3 * m); TRY_ALLOC(c->vel_src, 3 * m);
         TRY_ALLOC(c->user_of, m); TRY_ALLOC(c->user_src, m);
-        TRY_ALLOC(c->force, m); TRY_ALLOC(c->disp, 3 * m);
+        TRY_ALLOC(c->force, m); TRY_ALLOC(c->disp, 3 * m); TRY_ALLOC(c->e_atom, m);
         TRY_ALLOC(c->center_order, m); TRY_ALLOC(c->cell_of, m);
         TRY_ALLOC(c->nbr_count, m); TRY_ALLOC(c->nbr_off, m + 1);
         c->cap_atoms = n;

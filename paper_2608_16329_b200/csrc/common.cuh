@@ -72,7 +72,8 @@ struct mlip_ctx {
     double4 *pos4 = nullptr;       // x, y, z, species stored as a double
     double *vel = nullptr;         // [N][3]
     int32_t *user_of = nullptr;    // internal -> caller index
-    float4 *force = nullptr;       // fx, fy, fz, E_i
+    float4 *force = nullptr;       // fx, fy, fz, unused
+    float *e_atom = nullptr;       // E_i, internal order
     float *disp = nullptr;         // [N][3] displacement since the last build
     int32_t *center_order = nullptr;  // internal indices sorted by (species, cell)
     int32_t species_start_host[mlip::MAX_SPECIES + 1] = {0};

@@ -62,13 +62,13 @@ __global__ void k_kinetic(int64_t n, const double *__restrict__ mass, const doub
 }
 
 __global__ void k_scatter_forces(int64_t n, const int32_t *__restrict__ user_of, const float4 *__restrict__ force,
-                                 float *__restrict__ forces_out, float *__restrict__ e_atom) {
+                                 const float *__restrict__ e_in, float *__restrict__ forces_out, float *__restrict__ e_atom) {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     const float4 f = force[i];
     const int64_t u = user_of[i];
     if (forces_out) { forces_out[3 * u] = f.x; forces_out[3 * u + 1] = f.y; forces_out[3 * u + 2] = f.z; }
-    if (e_atom) e_atom[u] = f.w;
+    if (e_atom) e_atom[u] = e_in[i];
 }
 
 __global__ void k_set_positions(int64_t n, const int32_t *__restrict__ user_of, const double *__restrict__ pos,
@@ -135,7 +135,7 @@ int launch_kinetic(mlip_ctx *c, cudaStream_t s) {
     return MLIP_OK;
 }
 int launch_scatter_forces(mlip_ctx *c, float *forces, float *e_atom, cudaStream_t s) {
-    k_scatter_forces<<<nb(c->n), 256, 0, s>>>(c->n, c->user_of, c->force, forces, e_atom);
+    k_scatter_forces<<<nb(c->n), 256, 0, s>>>(c->n, c->user_of, c->force, c->e_atom, forces, e_atom);
     c->launches += 1;
     MLIP_CUDA_TRY(c, cudaGetLastError());
     return MLIP_OK;

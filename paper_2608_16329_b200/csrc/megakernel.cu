@@ -1,35 +1,98 @@
-// The fused evaluation kernel (Section 3.4.1 "mega-fusion": Eq. 1-10 in one launch, every
-// per-pair and per-atom intermediate kept in registers or shared memory, the radial and
-// angular features recomputed in the derivation stage instead of being kept).
+// The fused evaluation kernel (Section 3.4.1 "mega-fusion": Eq. 1-10 in one launch; every
+// per-pair and per-atom intermediate lives in registers or shared memory, and the radial and
+// angular features are recomputed in the derivation stage instead of being kept).
 //
-// Mapping, one warp per central atom:
-//   Encoding   lanes = pairs for the geometry (Eq. 1), the harmonics (Eq. 3) and the spline
-//              basis; then lanes = radial channels: each lane owns one column of the moment
-//              P_i (16 registers) and accumulates h (x) g (Eq. 4) with h broadcast from
-//              shared memory.  Invariants (Eq. 5) are then lane-local.
-//   Regression the species head (Eq. 6) forward and in reverse, two neurons per lane.
-//   Derivation W_i (Eq. 7) goes to shared memory; lanes = pairs again: each lane rebuilds
-//              g, g' for its pair, contracts them with W_i (Eq. 9 and the re-associated
-//              Eq. 8 term: U_i is never formed), projects onto the pair vector (Eq. 10) and
-//              scatters: its own sum stays in registers, the reaction goes out by atomics.
+// Work decomposition
+//   A persistent CTA (8 warps) takes tiles of 16 central atoms of ONE species from a global
+//   counter; a warp owns two atoms of the tile.
+//   Encoding    The warp scans the atom's list (lane = entry), keeps the pairs inside r_cut in a
+//               small shared queue, and every 32 queued pairs evaluates harmonics (Eq. 3) and the
+//               spline basis with lane = pair.  The moment P_i = H^T G (Eq. 4, 16 x n times
+//               n x 32) is then accumulated on the tensor pipe: mma.sync m16n8k8 TF32 with a
+//               three-term hi/lo split of both operands (error ~2^-21, fp32 accumulate), the
+//               radial values g being evaluated straight into the B fragments.
+//   Invariants  Eq. 5 from the accumulator fragments by three xor-shuffles.
+//   Regression  Eq. 6 forward and reverse for the 16 atoms at once: [16 x K] x [K x 64] layers on
+//               the tensor pipe, weights pre-split and pre-packed in fragment order.
+//   Derivation  W_i (Eq. 7) is the accumulator fragment of P_i scaled in place: by construction
+//               of the channel permutation it already is the B fragment of the next contraction.
+//               [V; T] = [G; G'] W^T (Eq. 9 and the re-associated Eq. 8 term, U_i never formed)
+//               again on the tensor pipe, 16 pairs per tile; results are transposed through
+//               shared memory to lane = pair for the projection of Eq. 10 and the scatter.
+// Everything that is not a contraction (geometry, harmonics, splines, projection) stays on the
+// fp32 pipe; positions are differenced in fp64.
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace mlip {
 
-constexpr int WARPS = 8;
-constexpr int STAGE_STRIDE = 28;   // floats per lane in the pair -> channel hand-over (16 h, 4 b, offset, pad)
+constexpr int TILE = 16;      // atoms per tile (one m16 tile of the head)
+constexpr int NW = 8;         // warps per CTA
+constexpr int PB_CAP = 64;    // queued pairs per warp
+constexpr int ST_STRIDE = 24; // encoding hand-over: 16 h, 4 b, table offset (bank-conflict-free for the fragment reads)
+constexpr int BS_STRIDE = 12; // derivation hand-over: 4 b, 4 b', table offset
+constexpr int VT_STRIDE = 40; // 16 v + 16 t per pair
+constexpr int X_STRIDE = 132; // invariants / dE/dG per atom
+constexpr int Z_STRIDE = 68;  // head activations per atom
 
-// fp32 head layout per species (floats):
-//   forward   W1t[128][64] b1[64] | W2t[64][64] b2[64] | W3t b3 | W4t b4 | w_out[64] b_out pad[3]
-//   backward  W1[64][128] | W2[64][64] | W3 | W4      (row-major [out][in], as supplied)
-constexpr int HW_FWD = N_INV * HEAD_H + HEAD_H + (HEAD_L - 1) * (HEAD_H * HEAD_H + HEAD_H) + HEAD_H + 4;
-constexpr int HW_BWD = N_INV * HEAD_H + (HEAD_L - 1) * HEAD_H * HEAD_H;
-constexpr int HW_TOTAL = HW_FWD + HW_BWD;
+constexpr int WARP_WORDS = 6 * PB_CAP + 32 * BS_STRIDE + 32 * VT_STRIDE;   // 384 + 384 + 1280 = 2048
+static_assert(32 * ST_STRIDE <= 32 * BS_STRIDE + 32 * VT_STRIDE, "encoding stage must fit the derivation buffers");
+constexpr int SP_WORDS = TILE * 16 * 32;          // moment fragments of the tile
+constexpr int SX_WORDS = TILE * X_STRIDE;
+constexpr int HEAD_WORDS = 2 * TILE * Z_STRIDE + HEAD_L * TILE * Z_STRIDE;   // activations (ping-pong) + SiLU'
+static_assert(HEAD_WORDS <= NW * WARP_WORDS, "head buffers alias the per-warp buffers");
+constexpr int SMEM_WORDS = SP_WORDS + SX_WORDS + NW * WARP_WORDS + 16;
+constexpr size_t SMEM_BYTES = sizeof(float) * SMEM_WORDS;
+
+// Pre-packed head weights per species (floats).  Fragment records are float4 {b0_hi, b1_hi, b0_lo, b1_lo}
+// per lane for the B operand of one (n-tile, k-step):
+//   forward  layer L: B[k][n] = W_L[n][k]        n-tiles 8, k-steps K_L / 8
+//   reverse  layer L: B[k][n] = W_L[k][n]        n-tiles K_L / 8, k-steps 8
+// followed by biases [4][64], w_out[64], b_out, pad.
+constexpr int KS0 = N_INV / 8, KS1 = HEAD_H / 8;
+constexpr int FWD_RECORDS = 8 * KS0 + (HEAD_L - 1) * 8 * KS1;
+constexpr int BWD_RECORDS = (N_INV / 8) * 8 + (HEAD_L - 1) * 8 * 8;
+constexpr int HP_FWD = 0;
+constexpr int HP_BWD = HP_FWD + FWD_RECORDS * 128;
+constexpr int HP_BIAS = HP_BWD + BWD_RECORDS * 128;
+constexpr int HP_WOUT = HP_BIAS + HEAD_L * HEAD_H;
+constexpr int HP_TOTAL = HP_WOUT + HEAD_H + 4;
 
 __device__ __forceinline__ float silu_f(float x, float &dsilu) {
     float s = 1.0f / (1.0f + expf(-x));
     dsilu = s * (1.0f + x * (1.0f - s));
     return x * s;
+}
+
+__device__ __forceinline__ void split_tf32(float x, uint32_t &hi, uint32_t &lo) {
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hi) : "f"(x));
+    lo = __float_as_uint(x - __uint_as_float(hi));
+}
+
+__device__ __forceinline__ void mma_tf32(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// c += A B with both operands split: A_hi B_hi + A_lo B_hi + A_hi B_lo.  The tensor pipe truncates
+// when it adds into its fp32 accumulator, so callers keep accumulation chains short (a fresh
+// accumulator per k-step, folded into the running sum by a rounded fp32 add): a long chain of
+// same-sign terms otherwise drifts by ~1e-6 relative.
+__device__ __forceinline__ void mma3(float (&c)[4], const uint32_t (&ah)[4], const uint32_t (&al)[4], uint32_t bh0, uint32_t bh1,
+                                     uint32_t bl0, uint32_t bl1) {
+    mma_tf32(c, al[0], al[1], al[2], al[3], bh0, bh1);
+    mma_tf32(c, ah[0], ah[1], ah[2], ah[3], bl0, bl1);
+    mma_tf32(c, ah[0], ah[1], ah[2], ah[3], bh0, bh1);
+}
+
+// Same product with the main and the small terms kept in separate accumulators.
+__device__ __forceinline__ void mma3s(float (&c)[4], float (&cs)[4], const uint32_t (&ah)[4], const uint32_t (&al)[4],
+                                      uint32_t bh0, uint32_t bh1, uint32_t bl0, uint32_t bl1) {
+    mma_tf32(cs, al[0], al[1], al[2], al[3], bh0, bh1);
+    mma_tf32(cs, ah[0], ah[1], ah[2], ah[3], bl0, bl1);
+    mma_tf32(c, ah[0], ah[1], ah[2], ah[3], bh0, bh1);
 }
 
 // Irreducible harmonic polynomials up to l = 3 of a unit vector (one valid solution of the
@@ -52,18 +115,16 @@ __device__ __forceinline__ void harmonics(float x, float y, float z, float *h) {
     h[15] = is10 * z * (2.0f * zz - 3.0f * xx - 3.0f * yy);
 }
 
-// Accumulate  s += sum_a h_a t_a,  tv += sum_a v_a grad h_a,  tu += sum_a l_a v_a h_a  (Euler: grad h_a . u = l_a h_a).
+// s = sum_a h_a t_a,  (tx,ty,tz) = sum_a v_a grad h_a,  tu = sum_a l_a v_a h_a  (Euler: grad h_a . u = l_a h_a).
 __device__ __forceinline__ void harmonics_project(float x, float y, float z, const float *v, const float *t,
                                                   float &s, float &tx, float &ty, float &tz, float &tu) {
     const float s2 = 1.41421356237f, is2 = 0.70710678118f, is6 = 0.40824829046f;
     const float s6 = 2.44948974278f, s15 = 1.22474487139f, is10 = 0.31622776601f;
     float xx = x * x, yy = y * y, zz = z * z, h;
     s = t[0]; tx = ty = tz = 0.f; tu = 0.f;
-    // l = 1
     s += x * t[1] + y * t[2] + z * t[3];
     tx += v[1]; ty += v[2]; tz += v[3];
     tu += x * v[1] + y * v[2] + z * v[3];
-    // l = 2
     float u2 = 0.f;
     h = s2 * x * y; s += h * t[4]; u2 += h * v[4]; tx += s2 * y * v[4]; ty += s2 * x * v[4];
     h = s2 * x * z; s += h * t[5]; u2 += h * v[5]; tx += s2 * z * v[5]; tz += s2 * x * v[5];
@@ -71,7 +132,6 @@ __device__ __forceinline__ void harmonics_project(float x, float y, float z, con
     h = is2 * (xx - yy); s += h * t[7]; u2 += h * v[7]; tx += s2 * x * v[7]; ty -= s2 * y * v[7];
     h = is6 * (2.f * zz - xx - yy); s += h * t[8]; u2 += h * v[8];
     tx -= 2.f * is6 * x * v[8]; ty -= 2.f * is6 * y * v[8]; tz += 4.f * is6 * z * v[8];
-    // l = 3
     float u3 = 0.f;
     h = s6 * x * y * z; s += h * t[9]; u3 += h * v[9];
     tx += s6 * y * z * v[9]; ty += s6 * x * z * v[9]; tz += s6 * x * y * v[9];
@@ -90,28 +150,8 @@ __device__ __forceinline__ void harmonics_project(float x, float y, float z, con
     tu += 2.f * u2 + 3.f * u3;
 }
 
-struct PairGeom {
-    float x, y, z, r, rinv;
-    int j;
-    bool valid;
-};
-
-// Eq. 1 with the periodic minimum image.  Differences are taken in fp64 (positions keep their
-// full precision in large boxes) and narrowed afterwards.
-__device__ __forceinline__ PairGeom pair_geometry(const double4 &pi, const double4 &pj, const CellGrid &g, double rc2) {
-    PairGeom p;
-    double dx = min_image(pj.x - pi.x, g.box[0], g.half[0]);
-    double dy = min_image(pj.y - pi.y, g.box[1], g.half[1]);
-    double dz = min_image(pj.z - pi.z, g.box[2], g.half[2]);
-    double d2 = dx * dx + dy * dy + dz * dz;
-    p.valid = d2 < rc2;
-    p.x = (float)dx; p.y = (float)dy; p.z = (float)dz;
-    p.r = sqrtf((float)d2);
-    p.rinv = 1.0f / p.r;
-    return p;
-}
-
-// Spline interval and cubic B-spline basis at distance r.
+// Spline interval and cubic B-spline basis (and its r-derivative) at distance r.
+template <bool DERIV>
 __device__ __forceinline__ int spline_basis(float r, const TableDesc &tab, float *b, float *db, int *status) {
     float xk = (r - tab.r_min) * tab.inv_h;
     if (xk < 0.f) { atomicOr(status, FLAG_TABLE_RANGE); xk = 0.f; }
@@ -123,7 +163,7 @@ __device__ __forceinline__ int spline_basis(float r, const TableDesc &tab, float
     b[1] = (3.f * u3 - 6.f * u2 + 4.f) * sixth;
     b[2] = (-3.f * u3 + 3.f * u2 + 3.f * u + 1.f) * sixth;
     b[3] = u3 * sixth;
-    if (db) {
+    if (DERIV) {
         db[0] = -0.5f * w * w * tab.inv_h;
         db[1] = (1.5f * u2 - 2.f * u) * tab.inv_h;
         db[2] = (-1.5f * u2 + u + 0.5f) * tab.inv_h;
@@ -132,235 +172,496 @@ __device__ __forceinline__ int spline_basis(float r, const TableDesc &tab, float
     return i;
 }
 
-__global__ void __launch_bounds__(WARPS * 32) k_mega(int64_t n, int n_species, CellGrid grid, double rc2, TableDesc tab,
-                                                     const double4 *__restrict__ pos4, const int32_t *__restrict__ center_order,
-                                                     const int64_t *__restrict__ nbr_off, const int32_t *__restrict__ nbr,
-                                                     const float *__restrict__ head_w, float4 *__restrict__ force,
-                                                     double *__restrict__ acc, unsigned long long *__restrict__ pair_counter,
-                                                     int *__restrict__ status) {
-    __shared__ __align__(16) float s_stage[WARPS][32 * STAGE_STRIDE];
-    __shared__ __align__(16) float s_W[WARPS][D_ANG * K_RADIAL];
-    __shared__ __align__(16) float s_x[WARPS][N_INV];
+struct Shared {
+    float *sP;      // [TILE][16][32] moment / W fragments
+    float *sX;      // [TILE][X_STRIDE] invariants, then dE/dG
+    float *warp;    // this warp's buffers
+    float *head;    // head activations (alias of all per-warp buffers)
+    int *ctl;       // tile hand-over
+};
 
+struct KernelArgs {
+    int64_t n;
+    int n_species;
+    CellGrid grid;
+    double rc2;
+    TableDesc tab;
+    const double4 *pos4;
+    const int32_t *center_order;
+    const int32_t *species_start;
+    const int64_t *nbr_off;
+    const int32_t *nbr;
+    const float *head_pack;
+    float4 *force;
+    float *e_atom;
+    double *acc;
+    unsigned long long *pair_counter;
+    int *status;
+    int *tile_counter;
+};
+
+// Scan the list of atom i (lane = entry), append the pairs inside r_cut to the warp's queue and
+// hand every 32 queued pairs (and the remainder) to `batch(n)`, which consumes entries [0, n).
+template <typename Batch>
+__device__ __forceinline__ int scan_pairs(const KernelArgs &k, const double4 &pi, int64_t beg, int64_t end, float *pb, int lane, Batch batch) {
+    float *px = pb, *py = pb + PB_CAP, *pz = pb + 2 * PB_CAP, *pr = pb + 3 * PB_CAP;
+    int *pj = reinterpret_cast<int *>(pb + 4 * PB_CAP), *ps = reinterpret_cast<int *>(pb + 5 * PB_CAP);
+    int nq = 0, total = 0;
+    for (int64_t base = beg; base < end; base += 32) {
+        const int64_t e = base + lane;
+        bool valid = false;
+        float x = 0.f, y = 0.f, z = 0.f, r = 1.f;
+        int j = 0, sj = 0;
+        if (e < end) {
+            j = __ldg(k.nbr + e);
+            const double4 pj4 = k.pos4[j];
+            double dx = min_image(pj4.x - pi.x, k.grid.box[0], k.grid.half[0]);
+            double dy = min_image(pj4.y - pi.y, k.grid.box[1], k.grid.half[1]);
+            double dz = min_image(pj4.z - pi.z, k.grid.box[2], k.grid.half[2]);
+            double d2 = dx * dx + dy * dy + dz * dz;
+            valid = d2 < k.rc2;
+            x = (float)dx; y = (float)dy; z = (float)dz;
+            r = sqrtf((float)d2);
+            sj = (int)pj4.w;
+        }
+        const unsigned m = __ballot_sync(0xffffffffu, valid);
+        if (valid) {
+            const int slot = nq + __popc(m & ((1u << lane) - 1u));
+            px[slot] = x; py[slot] = y; pz[slot] = z; pr[slot] = r; pj[slot] = j; ps[slot] = sj;
+        }
+        nq += __popc(m);
+        __syncwarp();
+        if (nq >= 32) {
+            batch(32);
+            total += 32;
+            // move the tail of the queue to the front
+            float tx = 0.f, ty = 0.f, tz = 0.f, tr = 1.f; int tj = 0, ts = 0;
+            const bool mv = 32 + lane < nq;
+            if (mv) { tx = px[32 + lane]; ty = py[32 + lane]; tz = pz[32 + lane]; tr = pr[32 + lane]; tj = pj[32 + lane]; ts = ps[32 + lane]; }
+            __syncwarp();
+            if (mv) { px[lane] = tx; py[lane] = ty; pz[lane] = tz; pr[lane] = tr; pj[lane] = tj; ps[lane] = ts; }
+            nq -= 32;
+            __syncwarp();
+        }
+    }
+    if (nq > 0) { batch(nq); total += nq; }
+    return total;
+}
+
+// ---------------- Encoding of one atom: returns the moment as accumulator fragments ----------------
+__device__ __forceinline__ int encode_atom(const KernelArgs &k, const double4 &pi, int si, int64_t beg, int64_t end,
+                                           float *wbuf, int lane, float (&Pf)[4][4]) {
+    const int g = lane >> 2, t = lane & 3;
+    float *pb = wbuf, *stage = wbuf + 6 * PB_CAP;
+    const int table_rows = k.tab.knots + 3;
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) Pf[a][b] = 0.f;
+
+    auto batch = [&](int n) {
+        {   // lane = pair: harmonics (Eq. 3) and spline basis
+            float h[D_ANG], b[4];
+            int off = 0;
+            if (lane < n) {
+                const float r = pb[3 * PB_CAP + lane], rinv = 1.0f / r;
+                harmonics(pb[lane] * rinv, pb[PB_CAP + lane] * rinv, pb[2 * PB_CAP + lane] * rinv, h);
+                const int iv = spline_basis<false>(r, k.tab, b, nullptr, k.status);
+                const int sj = reinterpret_cast<const int *>(pb)[5 * PB_CAP + lane];
+                off = ((si * k.n_species + sj) * table_rows + iv) * K_RADIAL;
+            } else {
+#pragma unroll
+                for (int a = 0; a < D_ANG; ++a) h[a] = 0.f;
+                b[0] = b[1] = b[2] = b[3] = 0.f;
+            }
+            float4 *row = reinterpret_cast<float4 *>(stage + lane * ST_STRIDE);
+            row[0] = make_float4(h[0], h[1], h[2], h[3]);
+            row[1] = make_float4(h[4], h[5], h[6], h[7]);
+            row[2] = make_float4(h[8], h[9], h[10], h[11]);
+            row[3] = make_float4(h[12], h[13], h[14], h[15]);
+            row[4] = make_float4(b[0], b[1], b[2], b[3]);
+            reinterpret_cast<int *>(stage)[lane * ST_STRIDE + 20] = off;
+        }
+        __syncwarp();
+        const int nks = (n + 7) >> 3;
+        for (int ks = 0; ks < nks; ++ks) {
+            // A = H^T (16 x 8 pairs): rows a = g, g + 8; columns pairs t, t + 4 of this k-step
+            const float *ra = stage + (8 * ks + t) * ST_STRIDE, *rb = ra + 4 * ST_STRIDE;
+            uint32_t ah[4], al[4];
+            split_tf32(ra[g], ah[0], al[0]);
+            split_tf32(ra[g + 8], ah[1], al[1]);
+            split_tf32(rb[g], ah[2], al[2]);
+            split_tf32(rb[g + 8], ah[3], al[3]);
+            // B = G (8 pairs x 8 channels per n-tile): this lane evaluates channels 4g .. 4g+3 (one per n-tile)
+            const float4 ba = *reinterpret_cast<const float4 *>(ra + 16), bb = *reinterpret_cast<const float4 *>(rb + 16);
+            const float4 *ta = reinterpret_cast<const float4 *>(k.tab.coef + reinterpret_cast<const int *>(ra)[20]) + g;
+            const float4 *tb = reinterpret_cast<const float4 *>(k.tab.coef + reinterpret_cast<const int *>(rb)[20]) + g;
+            const float4 a0 = __ldg(ta), a1 = __ldg(ta + 8), a2 = __ldg(ta + 16), a3 = __ldg(ta + 24);
+            const float4 b0 = __ldg(tb), b1 = __ldg(tb + 8), b2 = __ldg(tb + 16), b3 = __ldg(tb + 24);
+            float ga[4], gb[4];
+            ga[0] = ba.x * a0.x + ba.y * a1.x + ba.z * a2.x + ba.w * a3.x;
+            ga[1] = ba.x * a0.y + ba.y * a1.y + ba.z * a2.y + ba.w * a3.y;
+            ga[2] = ba.x * a0.z + ba.y * a1.z + ba.z * a2.z + ba.w * a3.z;
+            ga[3] = ba.x * a0.w + ba.y * a1.w + ba.z * a2.w + ba.w * a3.w;
+            gb[0] = bb.x * b0.x + bb.y * b1.x + bb.z * b2.x + bb.w * b3.x;
+            gb[1] = bb.x * b0.y + bb.y * b1.y + bb.z * b2.y + bb.w * b3.y;
+            gb[2] = bb.x * b0.z + bb.y * b1.z + bb.z * b2.z + bb.w * b3.z;
+            gb[3] = bb.x * b0.w + bb.y * b1.w + bb.z * b2.w + bb.w * b3.w;
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                uint32_t bh0, bl0, bh1, bl1;
+                split_tf32(ga[nt], bh0, bl0);
+                split_tf32(gb[nt], bh1, bl1);
+                float c[4] = {0.f, 0.f, 0.f, 0.f};
+                mma3(c, ah, al, bh0, bh1, bl0, bl1);   // Eq. 4, eight pairs
+                Pf[nt][0] += c[0]; Pf[nt][1] += c[1]; Pf[nt][2] += c[2]; Pf[nt][3] += c[3];
+            }
+        }
+        __syncwarp();
+    };
+    return scan_pairs(k, pi, beg, end, pb, lane, batch);
+}
+
+// ---------------- Derivation of one atom (Eq. 8-10) ----------------
+__device__ __forceinline__ void derive_atom(const KernelArgs &k, const double4 &pi, int i, int si, int64_t beg, int64_t end,
+                                            float *wbuf, int lane, const uint32_t (&Wh)[4][4], const uint32_t (&Wl)[4][4],
+                                            float (&vir)[9]) {
+    const int g = lane >> 2, t = lane & 3;
+    float *pb = wbuf, *bs = wbuf + 6 * PB_CAP, *vt = bs + 32 * BS_STRIDE;
+    const int table_rows = k.tab.knots + 3;
+    float fx = 0.f, fy = 0.f, fz = 0.f;
+
+    auto batch = [&](int n) {
+        {   // lane = pair: spline basis and its derivative
+            float b[4] = {0.f, 0.f, 0.f, 0.f}, db[4] = {0.f, 0.f, 0.f, 0.f};
+            int off = 0;
+            if (lane < n) {
+                const int iv = spline_basis<true>(pb[3 * PB_CAP + lane], k.tab, b, db, k.status);
+                const int sj = reinterpret_cast<const int *>(pb)[5 * PB_CAP + lane];
+                off = ((si * k.n_species + sj) * table_rows + iv) * K_RADIAL;
+            }
+            float4 *row = reinterpret_cast<float4 *>(bs + lane * BS_STRIDE);
+            row[0] = make_float4(b[0], b[1], b[2], b[3]);
+            row[1] = make_float4(db[0], db[1], db[2], db[3]);
+            reinterpret_cast<int *>(bs)[lane * BS_STRIDE + 8] = off;
+        }
+        __syncwarp();
+        const int nmt = (n + 15) >> 4;
+        for (int mt = 0; mt < nmt; ++mt) {
+            // A = [G; G'] (16 pairs x 32 channels): rows pairs g, g + 8; this lane evaluates channels 8t .. 8t+7
+            float V[2][4], T[2][4], Vs[2][4], Ts[2][4];   // main (hi x hi) and small (cross) terms apart
+#pragma unroll
+            for (int a = 0; a < 2; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) { V[a][b] = 0.f; T[a][b] = 0.f; Vs[a][b] = 0.f; Ts[a][b] = 0.f; }
+            float G[2][8], dG[2][8];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const float *rp = bs + (16 * mt + g + 8 * q) * BS_STRIDE;
+                const float4 b = *reinterpret_cast<const float4 *>(rp), db = *reinterpret_cast<const float4 *>(rp + 4);
+                const float4 *tc = reinterpret_cast<const float4 *>(k.tab.coef + reinterpret_cast<const int *>(rp)[8]) + 2 * t;
+                const float bw[4] = {b.x, b.y, b.z, b.w}, dbw[4] = {db.x, db.y, db.z, db.w};
+#pragma unroll
+                for (int c = 0; c < 8; ++c) { G[q][c] = 0.f; dG[q][c] = 0.f; }
+#pragma unroll
+                for (int m = 0; m < 4; ++m) {
+                    const float4 c0 = __ldg(tc + 8 * m), c1 = __ldg(tc + 8 * m + 1);
+                    const float cv[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) { G[q][c] += bw[m] * cv[c]; dG[q][c] += dbw[m] * cv[c]; }
+                }
+            }
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                uint32_t ah[4], al[4], dh[4], dl[4];
+                split_tf32(G[0][ks], ah[0], al[0]);      split_tf32(G[1][ks], ah[1], al[1]);
+                split_tf32(G[0][4 + ks], ah[2], al[2]);  split_tf32(G[1][4 + ks], ah[3], al[3]);
+                split_tf32(dG[0][ks], dh[0], dl[0]);     split_tf32(dG[1][ks], dh[1], dl[1]);
+                split_tf32(dG[0][4 + ks], dh[2], dl[2]); split_tf32(dG[1][4 + ks], dh[3], dl[3]);
+                mma3s(V[0], Vs[0], ah, al, Wh[ks][0], Wh[ks][1], Wl[ks][0], Wl[ks][1]);   // Eq. 9: rows of V, a = 0..7
+                mma3s(V[1], Vs[1], ah, al, Wh[ks][2], Wh[ks][3], Wl[ks][2], Wl[ks][3]);   //                  a = 8..15
+                mma3s(T[0], Ts[0], dh, dl, Wh[ks][0], Wh[ks][1], Wl[ks][0], Wl[ks][1]);   // W g' (Eq. 8 re-associated)
+                mma3s(T[1], Ts[1], dh, dl, Wh[ks][2], Wh[ks][3], Wl[ks][2], Wl[ks][3]);
+            }
+#pragma unroll
+            for (int a = 0; a < 2; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) { V[a][b] += Vs[a][b]; T[a][b] += Ts[a][b]; }
+            float *va = vt + (16 * mt + g) * VT_STRIDE + 2 * t, *vb = va + 8 * VT_STRIDE;
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                *reinterpret_cast<float2 *>(va + 8 * q) = make_float2(V[q][0], V[q][1]);
+                *reinterpret_cast<float2 *>(vb + 8 * q) = make_float2(V[q][2], V[q][3]);
+                *reinterpret_cast<float2 *>(va + 16 + 8 * q) = make_float2(T[q][0], T[q][1]);
+                *reinterpret_cast<float2 *>(vb + 16 + 8 * q) = make_float2(T[q][2], T[q][3]);
+            }
+        }
+        __syncwarp();
+        if (lane < n) {   // lane = pair: projection onto the pair vector (Eq. 10) and scatter
+            float v[D_ANG], tt[D_ANG];
+            const float4 *src = reinterpret_cast<const float4 *>(vt + lane * VT_STRIDE);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float4 a = src[q], b = src[4 + q];
+                v[4 * q] = a.x; v[4 * q + 1] = a.y; v[4 * q + 2] = a.z; v[4 * q + 3] = a.w;
+                tt[4 * q] = b.x; tt[4 * q + 1] = b.y; tt[4 * q + 2] = b.z; tt[4 * q + 3] = b.w;
+            }
+            const float x = pb[lane], y = pb[PB_CAP + lane], z = pb[2 * PB_CAP + lane], rinv = 1.0f / pb[3 * PB_CAP + lane];
+            const int j = reinterpret_cast<const int *>(pb)[4 * PB_CAP + lane];
+            const float ux = x * rinv, uy = y * rinv, uz = z * rinv;
+            float s, tx, ty, tz, tu;
+            harmonics_project(ux, uy, uz, v, tt, s, tx, ty, tz, tu);
+            // f_ij = (g' . u_ij) r^ + J_ang^T v_ij,  J_ang = (grad_u h)(I - u u^T) / r
+            const float qx = s * ux + (tx - tu * ux) * rinv;
+            const float qy = s * uy + (ty - tu * uy) * rinv;
+            const float qz = s * uz + (tz - tu * uz) * rinv;
+            fx += qx; fy += qy; fz += qz;
+            atomicAdd(&k.force[j].x, -qx);
+            atomicAdd(&k.force[j].y, -qy);
+            atomicAdd(&k.force[j].z, -qz);
+            vir[0] -= x * qx; vir[1] -= x * qy; vir[2] -= x * qz;
+            vir[3] -= y * qx; vir[4] -= y * qy; vir[5] -= y * qz;
+            vir[6] -= z * qx; vir[7] -= z * qy; vir[8] -= z * qz;
+        }
+        __syncwarp();
+    };
+    scan_pairs(k, pi, beg, end, pb, lane, batch);
+#pragma unroll
+    for (int o = 16; o; o >>= 1) {
+        fx += __shfl_xor_sync(0xffffffffu, fx, o);
+        fy += __shfl_xor_sync(0xffffffffu, fy, o);
+        fz += __shfl_xor_sync(0xffffffffu, fz, o);
+    }
+    if (lane == 0) {
+        atomicAdd(&k.force[i].x, fx);
+        atomicAdd(&k.force[i].y, fy);
+        atomicAdd(&k.force[i].z, fz);
+    }
+}
+
+// One layer-sized contraction of the head for the 16 atoms of the tile on the tensor pipe:
+// C[16 x 8] (n-tile nt) = A[16 x 8 nks] B, A read from shared memory through `load_a(k)`.
+template <typename LoadA>
+__device__ __forceinline__ void head_gemm(float (&c)[4], const float4 *__restrict__ rec, int nks, int lane, LoadA load_a) {
+    const int g = lane >> 2, t = lane & 3;
+    c[0] = c[1] = c[2] = c[3] = 0.f;
+#pragma unroll 4
+    for (int ks = 0; ks < nks; ++ks) {
+        uint32_t ah[4], al[4];
+        split_tf32(load_a(g, 8 * ks + t), ah[0], al[0]);
+        split_tf32(load_a(g + 8, 8 * ks + t), ah[1], al[1]);
+        split_tf32(load_a(g, 8 * ks + t + 4), ah[2], al[2]);
+        split_tf32(load_a(g + 8, 8 * ks + t + 4), ah[3], al[3]);
+        const float4 b = __ldg(rec + ks * 32 + lane);
+        float p[4] = {0.f, 0.f, 0.f, 0.f};
+        mma3(p, ah, al, __float_as_uint(b.x), __float_as_uint(b.y), __float_as_uint(b.z), __float_as_uint(b.w));
+        c[0] += p[0]; c[1] += p[1]; c[2] += p[2]; c[3] += p[3];
+    }
+}
+
+// ---------------- Regression (Eq. 6) forward and reverse for the tile ----------------
+// In: sX = invariants [atom][128].  Out: sX = dE/dG, per-atom energies written, returns nothing.
+__device__ __forceinline__ void head_tile(const KernelArgs &k, const Shared &sh, int species, int count, int first,
+                                          int warp, int lane, double &e_sum) {
+    const int g = lane >> 2, t = lane & 3;
+    const float *hp = k.head_pack + (size_t)species * HP_TOTAL;
+    const float4 *fwd = reinterpret_cast<const float4 *>(hp + HP_FWD), *bwd = reinterpret_cast<const float4 *>(hp + HP_BWD);
+    float *z0 = sh.head, *z1 = sh.head + TILE * Z_STRIDE, *sD = sh.head + 2 * TILE * Z_STRIDE;
+    const float *sX = sh.sX;
+
+    // forward: warp = n-tile (8 neurons)
+    for (int L = 0; L < HEAD_L; ++L) {
+        const float *zin = (L & 1) ? z0 : z1;   // layer L >= 1 reads what layer L-1 wrote
+        float *zout = (L & 1) ? z1 : z0;
+        float c[4];
+        if (L == 0) {
+            head_gemm(c, fwd + (size_t)(warp * KS0) * 32, KS0, lane, [&](int row, int col) { return sX[row * X_STRIDE + col]; });
+        } else {
+            const float4 *rec = fwd + (size_t)(8 * KS0 + (L - 1) * 8 * KS1 + warp * KS1) * 32;
+            head_gemm(c, rec, KS1, lane, [&](int row, int col) { return zin[row * Z_STRIDE + col]; });
+        }
+        const int n0 = 8 * warp + 2 * t;
+        const float b0 = __ldg(hp + HP_BIAS + L * HEAD_H + n0), b1 = __ldg(hp + HP_BIAS + L * HEAD_H + n0 + 1);
+        float d0, d1, d2, d3;
+        float y0 = silu_f(c[0] + b0, d0), y1 = silu_f(c[1] + b1, d1), y2 = silu_f(c[2] + b0, d2), y3 = silu_f(c[3] + b1, d3);
+        if (L > 0) {   // residual
+            y0 += zin[g * Z_STRIDE + n0]; y1 += zin[g * Z_STRIDE + n0 + 1];
+            y2 += zin[(g + 8) * Z_STRIDE + n0]; y3 += zin[(g + 8) * Z_STRIDE + n0 + 1];
+        }
+        *reinterpret_cast<float2 *>(zout + g * Z_STRIDE + n0) = make_float2(y0, y1);
+        *reinterpret_cast<float2 *>(zout + (g + 8) * Z_STRIDE + n0) = make_float2(y2, y3);
+        *reinterpret_cast<float2 *>(sD + (L * TILE + g) * Z_STRIDE + n0) = make_float2(d0, d1);
+        *reinterpret_cast<float2 *>(sD + (L * TILE + g + 8) * Z_STRIDE + n0) = make_float2(d2, d3);
+        __syncthreads();
+    }
+    // the last layer (L = 3) wrote z1.  Energies: warp w sums atoms 2w, 2w+1.
+    {
+        const float w0 = __ldg(hp + HP_WOUT + lane), w1 = __ldg(hp + HP_WOUT + 32 + lane), bo = __ldg(hp + HP_WOUT + HEAD_H);
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int a = 2 * warp + q;
+            float e = w0 * z1[a * Z_STRIDE + lane] + w1 * z1[a * Z_STRIDE + 32 + lane];
+#pragma unroll
+            for (int o = 16; o; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
+            e += bo;
+            if (lane == 0 && a < count) {
+                k.e_atom[__ldg(k.center_order + first + a)] = e;
+                e_sum += (double)e;
+            }
+        }
+    }
+    __syncthreads();
+    // reverse: dZ starts as w_out for every atom (written into z0), then layers 3, 2, 1 with their skip paths
+    for (int idx = threadIdx.x; idx < TILE * HEAD_H; idx += NW * 32)
+        z0[(idx >> 6) * Z_STRIDE + (idx & 63)] = __ldg(hp + HP_WOUT + (idx & 63));
+    __syncthreads();
+    int flip = 0;   // dZ currently in z0
+    for (int L = HEAD_L - 1; L >= 1; --L) {
+        const float *din = flip ? z1 : z0;
+        float *dout = flip ? z0 : z1;
+        const float *dact = sD + L * TILE * Z_STRIDE;
+        const float4 *rec = bwd + (size_t)((N_INV / 8) * 8 + (L - 1) * 64 + warp * 8) * 32;
+        float c[4];
+        head_gemm(c, rec, 8, lane, [&](int row, int col) { return din[row * Z_STRIDE + col] * dact[row * Z_STRIDE + col]; });
+        const int n0 = 8 * warp + 2 * t;
+        *reinterpret_cast<float2 *>(dout + g * Z_STRIDE + n0) = make_float2(c[0] + din[g * Z_STRIDE + n0], c[1] + din[g * Z_STRIDE + n0 + 1]);
+        *reinterpret_cast<float2 *>(dout + (g + 8) * Z_STRIDE + n0) =
+            make_float2(c[2] + din[(g + 8) * Z_STRIDE + n0], c[3] + din[(g + 8) * Z_STRIDE + n0 + 1]);
+        flip ^= 1;
+        __syncthreads();
+    }
+    {   // first layer: dE/dG [16 x 128], two n-tiles per warp, written over the invariants
+        const float *din = flip ? z1 : z0;
+        const float *dact = sD;
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int nt = warp + 8 * q;
+            float c[4];
+            head_gemm(c, bwd + (size_t)(nt * 8) * 32, 8, lane, [&](int row, int col) { return din[row * Z_STRIDE + col] * dact[row * Z_STRIDE + col]; });
+            const int n0 = 8 * nt + 2 * t;
+            *reinterpret_cast<float2 *>(sh.sX + g * X_STRIDE + n0) = make_float2(c[0], c[1]);
+            *reinterpret_cast<float2 *>(sh.sX + (g + 8) * X_STRIDE + n0) = make_float2(c[2], c[3]);
+        }
+    }
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(NW * 32, 2) k_mega(KernelArgs k) {
+    extern __shared__ __align__(16) float smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float *stage = s_stage[warp], *sW = s_W[warp], *sx = s_x[warp];
-    const int64_t n_warps = (int64_t)gridDim.x * WARPS;
-    const int table_rows = tab.knots + 3;
+    const int g = lane >> 2, t = lane & 3;
+    Shared sh;
+    sh.sP = smem;
+    sh.sX = smem + SP_WORDS;
+    sh.head = sh.sX + SX_WORDS;
+    sh.warp = sh.head + warp * WARP_WORDS;
+    sh.ctl = reinterpret_cast<int *>(sh.head + NW * WARP_WORDS);
+
+    // species-pure tiles: tiles of species s start at tile_first[s]
+    int tile_first[MAX_SPECIES + 1];
+    tile_first[0] = 0;
+    for (int s = 0; s < MAX_SPECIES; ++s) {
+        int cnt = s < k.n_species ? __ldg(k.species_start + s + 1) - __ldg(k.species_start + s) : 0;
+        tile_first[s + 1] = tile_first[s] + (cnt + TILE - 1) / TILE;
+    }
+    const int n_tiles = tile_first[MAX_SPECIES];
 
     double e_sum = 0.0;
     float vir[9] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     unsigned long long n_pairs = 0;
 
-    for (int64_t w = (int64_t)blockIdx.x * WARPS + warp; w < n; w += n_warps) {
-        const int i = center_order[w];
-        const double4 pi = pos4[i];
-        const int si = (int)pi.w;
-        const int64_t beg = nbr_off[i], end = nbr_off[i + 1];
+    while (true) {
+        __syncthreads();
+        if (threadIdx.x == 0) sh.ctl[0] = atomicAdd(k.tile_counter, 1);
+        __syncthreads();
+        const int tile = sh.ctl[0];
+        if (tile >= n_tiles) break;
+        int species = 0;
+        while (tile >= tile_first[species + 1]) ++species;
+        const int s_beg = __ldg(k.species_start + species), s_end = __ldg(k.species_start + species + 1);
+        const int first = s_beg + (tile - tile_first[species]) * TILE;
+        const int count = min(TILE, s_end - first);
 
-        // ---------------- Encoding ----------------
-        float P[D_ANG];
-#pragma unroll
-        for (int a = 0; a < D_ANG; ++a) P[a] = 0.f;
-        for (int64_t base = beg; base < end; base += 32) {
-            const int64_t e = base + lane;
-            bool valid = false;
-            if (e < end) {
-                const int j = nbr[e];
-                const double4 pj = pos4[j];
-                PairGeom p = pair_geometry(pi, pj, grid, rc2);
-                valid = p.valid;
-                if (valid) {
-                    float h[D_ANG], b[4];
-                    harmonics(p.x * p.rinv, p.y * p.rinv, p.z * p.rinv, h);
-                    int iv = spline_basis(p.r, tab, b, nullptr, status);
-                    int off = ((si * n_species + (int)pj.w) * table_rows + iv) * K_RADIAL;
-                    float4 *row = reinterpret_cast<float4 *>(stage + lane * STAGE_STRIDE);
-                    row[0] = make_float4(h[0], h[1], h[2], h[3]);
-                    row[1] = make_float4(h[4], h[5], h[6], h[7]);
-                    row[2] = make_float4(h[8], h[9], h[10], h[11]);
-                    row[3] = make_float4(h[12], h[13], h[14], h[15]);
-                    row[4] = make_float4(b[0], b[1], b[2], b[3]);
-                    row[5] = make_float4(__int_as_float(off), 0.f, 0.f, 0.f);
-                }
+        // ---------------- Encoding + invariants ----------------
+#pragma unroll 1
+        for (int q = 0; q < 2; ++q) {
+            const int a = 2 * warp + q;
+            float *xrow = sh.sX + a * X_STRIDE;
+            if (a >= count) {   // empty slot of a ragged tile: feed zeros to the head
+                for (int c = lane; c < N_INV; c += 32) xrow[c] = 0.f;
+                continue;
             }
-            unsigned m = __ballot_sync(0xffffffffu, valid);
-            n_pairs += __popc(m);
-            __syncwarp();
-            while (m) {
-                const int p = __ffs(m) - 1;
-                m &= m - 1;
-                const float4 *row = reinterpret_cast<const float4 *>(stage + p * STAGE_STRIDE);
-                const float4 b = row[4];
-                const int off = __float_as_int(row[5].x);
-                const float *tc = tab.coef + off + lane;
-                float g = b.x * __ldg(tc) + b.y * __ldg(tc + K_RADIAL) + b.z * __ldg(tc + 2 * K_RADIAL) + b.w * __ldg(tc + 3 * K_RADIAL);
+            const int i = __ldg(k.center_order + first + a);
+            const double4 pi = k.pos4[i];
+            float Pf[4][4];
+            n_pairs += encode_atom(k, pi, species, k.nbr_off[i], k.nbr_off[i + 1], sh.warp, lane, Pf);
+            float *prow = sh.sP + a * 16 * 32;
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const float4 h = row[q];
-                    P[4 * q + 0] += h.x * g; P[4 * q + 1] += h.y * g;
-                    P[4 * q + 2] += h.z * g; P[4 * q + 3] += h.w * g;
-                }
+            for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+                for (int r = 0; r < 4; ++r) prow[(4 * nt + r) * 32 + lane] = Pf[nt][r];
+            // Eq. 5 (C_l = I): this lane holds rows a = g, g + 8 of channels 8t + j; sum squares over the rows of a block
+            float part[4][8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float pa = Pf[j & 3][j >> 2], pb = Pf[j & 3][2 + (j >> 2)];
+                part[0][j] = g == 0 ? pa : 0.f;
+                part[1][j] = (g >= 1 && g <= 3) ? pa * pa : 0.f;
+                part[2][j] = (g >= 4 ? pa * pa : 0.f) + (g == 0 ? pb * pb : 0.f);
+                part[3][j] = g >= 1 ? pb * pb : 0.f;
             }
-            __syncwarp();
-        }
-
-        // ---------------- invariants (Eq. 5, C_l = I) ----------------
-        {
-            float g1 = P[1] * P[1] + P[2] * P[2] + P[3] * P[3];
-            float g2 = P[4] * P[4] + P[5] * P[5] + P[6] * P[6] + P[7] * P[7] + P[8] * P[8];
-            float g3 = P[9] * P[9] + P[10] * P[10] + P[11] * P[11] + P[12] * P[12] + P[13] * P[13] + P[14] * P[14] + P[15] * P[15];
-            sx[lane] = P[0]; sx[32 + lane] = g1; sx[64 + lane] = g2; sx[96 + lane] = g3;
-        }
-        __syncwarp();
-
-        // ---------------- Regression (Eq. 6): forward ----------------
-        const float *hw = head_w + (size_t)si * HW_TOTAL;
-        float dact[HEAD_L][2];   // SiLU'(pre-activation) of this lane's two neurons per layer
-        float z0, z1;
-        {
-            const float *Wt = hw, *bb = hw + N_INV * HEAD_H;
-            float a0 = __ldg(bb + lane), a1 = __ldg(bb + 32 + lane);
-#pragma unroll 8
-            for (int q = 0; q < N_INV; ++q) {
-                float x = sx[q];
-                a0 += __ldg(Wt + q * HEAD_H + lane) * x;
-                a1 += __ldg(Wt + q * HEAD_H + 32 + lane) * x;
-            }
-            z0 = silu_f(a0, dact[0][0]);
-            z1 = silu_f(a1, dact[0][1]);
-        }
-        const float *layer_w = hw + N_INV * HEAD_H + HEAD_H;
 #pragma unroll
-        for (int L = 1; L < HEAD_L; ++L) {
-            __syncwarp();
-            sx[lane] = z0; sx[32 + lane] = z1;
-            __syncwarp();
-            const float *Wt = layer_w, *bb = layer_w + HEAD_H * HEAD_H;
-            float a0 = __ldg(bb + lane), a1 = __ldg(bb + 32 + lane);
-#pragma unroll 8
-            for (int q = 0; q < HEAD_H; ++q) {
-                float x = sx[q];
-                a0 += __ldg(Wt + q * HEAD_H + lane) * x;
-                a1 += __ldg(Wt + q * HEAD_H + 32 + lane) * x;
-            }
-            float d0, d1;
-            z0 += silu_f(a0, d0);
-            z1 += silu_f(a1, d1);
-            dact[L][0] = d0; dact[L][1] = d1;
-            layer_w += HEAD_H * HEAD_H + HEAD_H;
-        }
-        const float wo0 = __ldg(layer_w + lane), wo1 = __ldg(layer_w + 32 + lane);
-        float e_i = wo0 * z0 + wo1 * z1;
+            for (int o = 4; o < 32; o <<= 1)
 #pragma unroll
-        for (int o = 16; o; o >>= 1) e_i += __shfl_xor_sync(0xffffffffu, e_i, o);
-        e_i += __ldg(layer_w + HEAD_H);
-
-        // ---------------- Regression in reverse: dE/dG ----------------
-        float dz0 = wo0, dz1 = wo1;
-        const float *bw = hw + HW_FWD + N_INV * HEAD_H + (HEAD_L - 2) * HEAD_H * HEAD_H;   // W of the last hidden layer
+                for (int l = 0; l < 4; ++l)
 #pragma unroll
-        for (int L = HEAD_L - 1; L >= 1; --L) {
-            __syncwarp();
-            sx[lane] = dz0 * dact[L][0]; sx[32 + lane] = dz1 * dact[L][1];
-            __syncwarp();
-            float a0 = 0.f, a1 = 0.f;
-#pragma unroll 8
-            for (int o = 0; o < HEAD_H; ++o) {
-                float d = sx[o];
-                a0 += __ldg(bw + o * HEAD_H + lane) * d;
-                a1 += __ldg(bw + o * HEAD_H + 32 + lane) * d;
-            }
-            dz0 += a0; dz1 += a1;
-            bw -= HEAD_H * HEAD_H;
-        }
-        __syncwarp();
-        sx[lane] = dz0 * dact[0][0]; sx[32 + lane] = dz1 * dact[0][1];
-        __syncwarp();
-        float dG[4] = {0.f, 0.f, 0.f, 0.f};
-        {
-            const float *W1 = hw + HW_FWD;
-#pragma unroll 4
-            for (int o = 0; o < HEAD_H; ++o) {
-                float d = sx[o];
+                    for (int j = 0; j < 8; ++j) part[l][j] += __shfl_xor_sync(0xffffffffu, part[l][j], o);
+            if (g == 0) {
 #pragma unroll
-                for (int q = 0; q < 4; ++q) dG[q] += __ldg(W1 + o * N_INV + 32 * q + lane) * d;
-            }
-        }
-
-        // ---------------- W_i = dE_i/dP_i (Eq. 7) ----------------
-        sW[lane] = dG[0];
-#pragma unroll
-        for (int a = 1; a < D_ANG; ++a) {
-            const float c = 2.0f * (a < 4 ? dG[1] : (a < 9 ? dG[2] : dG[3]));
-            sW[a * K_RADIAL + lane] = c * P[a];
-        }
-        __syncwarp();
-
-        // ---------------- Derivation (Eq. 8-10) ----------------
-        float fx = 0.f, fy = 0.f, fz = 0.f;
-        for (int64_t base = beg; base < end; base += 32) {
-            const int64_t e = base + lane;
-            if (e < end) {
-                const int j = nbr[e];
-                const double4 pj = pos4[j];
-                PairGeom p = pair_geometry(pi, pj, grid, rc2);
-                if (p.valid) {
-                    float b[4], db[4];
-                    int iv = spline_basis(p.r, tab, b, db, status);
-                    const float4 *tc = reinterpret_cast<const float4 *>(tab.coef + ((si * n_species + (int)pj.w) * table_rows + iv) * K_RADIAL);
-                    float v[D_ANG], t[D_ANG];
-#pragma unroll
-                    for (int a = 0; a < D_ANG; ++a) { v[a] = 0.f; t[a] = 0.f; }
-#pragma unroll
-                    for (int c4 = 0; c4 < K_RADIAL / 4; ++c4) {
-                        float4 c0 = __ldg(tc + c4), c1 = __ldg(tc + 8 + c4), c2 = __ldg(tc + 16 + c4), c3 = __ldg(tc + 24 + c4);
-                        float4 g, dg;
-                        g.x = b[0] * c0.x + b[1] * c1.x + b[2] * c2.x + b[3] * c3.x;
-                        g.y = b[0] * c0.y + b[1] * c1.y + b[2] * c2.y + b[3] * c3.y;
-                        g.z = b[0] * c0.z + b[1] * c1.z + b[2] * c2.z + b[3] * c3.z;
-                        g.w = b[0] * c0.w + b[1] * c1.w + b[2] * c2.w + b[3] * c3.w;
-                        dg.x = db[0] * c0.x + db[1] * c1.x + db[2] * c2.x + db[3] * c3.x;
-                        dg.y = db[0] * c0.y + db[1] * c1.y + db[2] * c2.y + db[3] * c3.y;
-                        dg.z = db[0] * c0.z + db[1] * c1.z + db[2] * c2.z + db[3] * c3.z;
-                        dg.w = db[0] * c0.w + db[1] * c1.w + db[2] * c2.w + db[3] * c3.w;
-#pragma unroll
-                        for (int a = 0; a < D_ANG; ++a) {
-                            const float4 wv = *reinterpret_cast<const float4 *>(sW + a * K_RADIAL + 4 * c4);
-                            v[a] += wv.x * g.x + wv.y * g.y + wv.z * g.z + wv.w * g.w;      // Eq. 9: row of V
-                            t[a] += wv.x * dg.x + wv.y * dg.y + wv.z * dg.z + wv.w * dg.w;  // W g' (Eq. 8 re-associated)
-                        }
-                    }
-                    const float ux = p.x * p.rinv, uy = p.y * p.rinv, uz = p.z * p.rinv;
-                    float s, tx, ty, tz, tu;
-                    harmonics_project(ux, uy, uz, v, t, s, tx, ty, tz, tu);
-                    // Eq. 10: f_ij = (g' . u_ij) r^ + J_ang^T v_ij,  J_ang = (grad_u h)(I - u u^T) / r
-                    const float px = s * ux + (tx - tu * ux) * p.rinv;
-                    const float py = s * uy + (ty - tu * uy) * p.rinv;
-                    const float pz = s * uz + (tz - tu * uz) * p.rinv;
-                    fx += px; fy += py; fz += pz;
-                    atomicAdd(&force[j].x, -px);
-                    atomicAdd(&force[j].y, -py);
-                    atomicAdd(&force[j].z, -pz);
-                    vir[0] -= p.x * px; vir[1] -= p.x * py; vir[2] -= p.x * pz;
-                    vir[3] -= p.y * px; vir[4] -= p.y * py; vir[5] -= p.y * pz;
-                    vir[6] -= p.z * px; vir[7] -= p.z * py; vir[8] -= p.z * pz;
+                for (int l = 0; l < 4; ++l) {
+                    *reinterpret_cast<float4 *>(xrow + 32 * l + 8 * t) = make_float4(part[l][0], part[l][1], part[l][2], part[l][3]);
+                    *reinterpret_cast<float4 *>(xrow + 32 * l + 8 * t + 4) = make_float4(part[l][4], part[l][5], part[l][6], part[l][7]);
                 }
             }
         }
+        __syncthreads();
+
+        // ---------------- Regression ----------------
+        head_tile(k, sh, species, count, first, warp, lane, e_sum);
+
+        // ---------------- Derivation ----------------
+#pragma unroll 1
+        for (int q = 0; q < 2; ++q) {
+            const int a = 2 * warp + q;
+            if (a >= count) continue;
+            const int i = __ldg(k.center_order + first + a);
+            const double4 pi = k.pos4[i];
+            // W_i = dE_i/dP_i (Eq. 7), already in B-fragment order
+            const float *xrow = sh.sX + a * X_STRIDE, *prow = sh.sP + a * 16 * 32;
+            const int la = g == 0 ? 0 : (g <= 3 ? 1 : 2), lb = g == 0 ? 2 : 3;
+            float da[8], db[8];
+            {
+                const float4 a0 = *reinterpret_cast<const float4 *>(xrow + 32 * la + 8 * t), a1 = *reinterpret_cast<const float4 *>(xrow + 32 * la + 8 * t + 4);
+                const float4 b0 = *reinterpret_cast<const float4 *>(xrow + 32 * lb + 8 * t), b1 = *reinterpret_cast<const float4 *>(xrow + 32 * lb + 8 * t + 4);
+                da[0] = a0.x; da[1] = a0.y; da[2] = a0.z; da[3] = a0.w; da[4] = a1.x; da[5] = a1.y; da[6] = a1.z; da[7] = a1.w;
+                db[0] = b0.x; db[1] = b0.y; db[2] = b0.z; db[3] = b0.w; db[4] = b1.x; db[5] = b1.y; db[6] = b1.z; db[7] = b1.w;
+            }
+            uint32_t Wh[4][4], Wl[4][4];
 #pragma unroll
-        for (int o = 16; o; o >>= 1) {
-            fx += __shfl_xor_sync(0xffffffffu, fx, o);
-            fy += __shfl_xor_sync(0xffffffffu, fy, o);
-            fz += __shfl_xor_sync(0xffffffffu, fz, o);
+            for (int ks = 0; ks < 4; ++ks) {
+                const float p0 = prow[(4 * ks + 0) * 32 + lane], p1 = prow[(4 * ks + 1) * 32 + lane];
+                const float p2 = prow[(4 * ks + 2) * 32 + lane], p3 = prow[(4 * ks + 3) * 32 + lane];
+                const float w0 = g == 0 ? da[ks] : 2.f * da[ks] * p0;          // row a = g,     channel 8t + ks
+                const float w1 = g == 0 ? da[4 + ks] : 2.f * da[4 + ks] * p1;  // row a = g,     channel 8t + 4 + ks
+                const float w2 = 2.f * db[ks] * p2;                            // row a = g + 8, channel 8t + ks
+                const float w3 = 2.f * db[4 + ks] * p3;                        // row a = g + 8, channel 8t + 4 + ks
+                split_tf32(w0, Wh[ks][0], Wl[ks][0]);
+                split_tf32(w1, Wh[ks][1], Wl[ks][1]);
+                split_tf32(w2, Wh[ks][2], Wl[ks][2]);
+                split_tf32(w3, Wh[ks][3], Wl[ks][3]);
+            }
+            derive_atom(k, pi, i, species, k.nbr_off[i], k.nbr_off[i + 1], sh.warp, lane, Wh, Wl, vir);
         }
-        if (lane == 0) {
-            atomicAdd(&force[i].x, fx);
-            atomicAdd(&force[i].y, fy);
-            atomicAdd(&force[i].z, fz);
-            force[i].w = e_i;
-            e_sum += (double)e_i;
-        }
-        __syncwarp();
     }
 
     // per-warp totals -> global accumulators
@@ -369,43 +670,67 @@ __global__ void __launch_bounds__(WARPS * 32) k_mega(int64_t n, int n_species, C
         float x = vir[q];
 #pragma unroll
         for (int o = 16; o; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
-        if (lane == 0) atomicAdd(&acc[ACC_VIRIAL + q], (double)x);
+        if (lane == 0) atomicAdd(&k.acc[ACC_VIRIAL + q], (double)x);
     }
     if (lane == 0) {
-        atomicAdd(&acc[ACC_ENERGY], e_sum);
-        atomicAdd(pair_counter, n_pairs);
+        atomicAdd(&k.acc[ACC_ENERGY], e_sum);
+        atomicAdd(k.pair_counter, n_pairs);
     }
+}
+
+// ---------------- host side ----------------
+static inline void split_host(float x, float &hi, float &lo) {
+    uint32_t u;
+    memcpy(&u, &x, 4);
+    u = (u + 0x1000u) & 0xffffe000u;   // round to nearest (ties away) at 10 mantissa bits
+    memcpy(&hi, &u, 4);
+    lo = x - hi;
 }
 
 int upload_head(mlip_ctx *c, const double *w) {
     const int C = c->cfg.n_species;
-    std::string buf_err;
-    float *host = (float *)malloc(sizeof(float) * (size_t)C * HW_TOTAL);
+    float *host = (float *)calloc((size_t)C * HP_TOTAL, sizeof(float));
     if (!host) return MLIP_ERR_OOM;
     for (int s = 0; s < C; ++s) {
         const double *src = w + (size_t)s * HEAD_NET;
-        float *fwd = host + (size_t)s * HW_TOTAL, *bwd = fwd + HW_FWD;
+        float *hp = host + (size_t)s * HP_TOTAL;
+        float *fwd = hp + HP_FWD, *bwd = hp + HP_BWD;
         int in = N_INV;
         for (int L = 0; L < HEAD_L; ++L) {
-            for (int o = 0; o < HEAD_H; ++o)
-                for (int i = 0; i < in; ++i) {
-                    fwd[i * HEAD_H + o] = (float)src[o * in + i];
-                    bwd[o * in + i] = (float)src[o * in + i];
-                }
-            for (int o = 0; o < HEAD_H; ++o) fwd[in * HEAD_H + o] = (float)src[in * HEAD_H + o];
+            const int nks = in / 8;
+            // forward: B[k][n] = W[n][k]; record (nt, ks), lane (g, t): b0 = W[8nt+g][8ks+t], b1 = W[8nt+g][8ks+t+4]
+            for (int nt = 0; nt < 8; ++nt)
+                for (int ks = 0; ks < nks; ++ks)
+                    for (int lane = 0; lane < 32; ++lane) {
+                        const int g = lane >> 2, t = lane & 3;
+                        float *rec = fwd + ((size_t)(nt * nks + ks) * 32 + lane) * 4;
+                        split_host((float)src[(8 * nt + g) * in + 8 * ks + t], rec[0], rec[2]);
+                        split_host((float)src[(8 * nt + g) * in + 8 * ks + t + 4], rec[1], rec[3]);
+                    }
+            // reverse: B[k][n] = W[k][n] (k = neuron, n = input); record (nt, ks): b0 = W[8ks+t][8nt+g], b1 = W[8ks+t+4][8nt+g]
+            for (int nt = 0; nt < in / 8; ++nt)
+                for (int ks = 0; ks < 8; ++ks)
+                    for (int lane = 0; lane < 32; ++lane) {
+                        const int g = lane >> 2, t = lane & 3;
+                        float *rec = bwd + ((size_t)(nt * 8 + ks) * 32 + lane) * 4;
+                        split_host((float)src[(8 * ks + t) * in + 8 * nt + g], rec[0], rec[2]);
+                        split_host((float)src[(8 * ks + t + 4) * in + 8 * nt + g], rec[1], rec[3]);
+                    }
+            for (int o = 0; o < HEAD_H; ++o) hp[HP_BIAS + L * HEAD_H + o] = (float)src[in * HEAD_H + o];
             src += in * HEAD_H + HEAD_H;
-            fwd += in * HEAD_H + HEAD_H;
-            bwd += in * HEAD_H;
+            fwd += (size_t)8 * nks * 128;
+            bwd += (size_t)(in / 8) * 8 * 128;
             in = HEAD_H;
         }
-        for (int o = 0; o < HEAD_H + 1; ++o) fwd[o] = (float)src[o];
-        fwd[HEAD_H + 1] = fwd[HEAD_H + 2] = fwd[HEAD_H + 3] = 0.f;
+        for (int o = 0; o < HEAD_H + 1; ++o) hp[HP_WOUT + o] = (float)src[o];
     }
-    cudaError_t e = cudaMalloc(&c->head_w, sizeof(float) * (size_t)C * HW_TOTAL);
-    if (e == cudaSuccess) e = cudaMemcpy(c->head_w, host, sizeof(float) * (size_t)C * HW_TOTAL, cudaMemcpyHostToDevice);
+    cudaError_t e = cudaMalloc(&c->head_w, sizeof(float) * (size_t)C * HP_TOTAL);
+    if (e == cudaSuccess) e = cudaMemcpy(c->head_w, host, sizeof(float) * (size_t)C * HP_TOTAL, cudaMemcpyHostToDevice);
     free(host);
     if (e != cudaSuccess) { c->err = cudaGetErrorString(e); return MLIP_ERR_CUDA; }
-    c->resident += sizeof(float) * (size_t)C * HW_TOTAL;
+    c->resident += sizeof(float) * (size_t)C * HP_TOTAL;
+    e = cudaFuncSetAttribute(k_mega, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+    if (e != cudaSuccess) { c->err = std::string("fused kernel shared memory: ") + cudaGetErrorString(e); return MLIP_ERR_CUDA; }
     return MLIP_OK;
 }
 
@@ -414,15 +739,17 @@ int launch_megakernel(mlip_ctx *c, cudaStream_t s) {
     MLIP_CUDA_TRY(c, cudaMemsetAsync(c->force, 0, sizeof(float4) * n, s));
     MLIP_CUDA_TRY(c, cudaMemsetAsync(c->acc, 0, sizeof(double) * ACC_KINETIC, s));
     MLIP_CUDA_TRY(c, cudaMemsetAsync(c->pair_counter, 0, sizeof(unsigned long long), s));
-    int64_t blocks = (n + WARPS - 1) / WARPS;
-    const int64_t max_blocks = (int64_t)c->n_sm * 8;
-    if (blocks > max_blocks) blocks = max_blocks;
-    if (blocks < 1) blocks = 1;
-    const double rc2 = c->cfg.r_cut * c->cfg.r_cut;
+    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->tile_counter, 0, sizeof(int), s));
+    const int64_t tiles_max = (n + TILE - 1) / TILE + c->cfg.n_species;
+    const int blocks = (int)std::min<int64_t>(tiles_max, (int64_t)c->n_sm * 2);
+    KernelArgs k;
+    k.n = n; k.n_species = c->cfg.n_species; k.grid = c->grid; k.rc2 = c->cfg.r_cut * c->cfg.r_cut; k.tab = c->tab;
+    k.pos4 = c->pos4; k.center_order = c->center_order; k.species_start = c->species_start;
+    k.nbr_off = c->nbr_off; k.nbr = c->nbr; k.head_pack = c->head_w; k.force = c->force; k.e_atom = c->e_atom;
+    k.acc = c->acc; k.pair_counter = c->pair_counter; k.status = c->status; k.tile_counter = c->tile_counter;
     const int slot = (int)(c->ev_count % mlip_ctx::EV_POOL);
     MLIP_CUDA_TRY(c, cudaEventRecord(c->ev[2 * slot], s));
-    k_mega<<<(unsigned)blocks, WARPS * 32, 0, s>>>(n, c->cfg.n_species, c->grid, rc2, c->tab, c->pos4, c->center_order,
-                                                   c->nbr_off, c->nbr, c->head_w, c->force, c->acc, c->pair_counter, c->status);
+    k_mega<<<blocks, NW * 32, SMEM_BYTES, s>>>(k);
     MLIP_CUDA_TRY(c, cudaEventRecord(c->ev[2 * slot + 1], s));
     c->ev_count += 1;
     c->launches += 1;
