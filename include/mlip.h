@@ -63,7 +63,7 @@ typedef struct {
     int l_max;            /* 3 */
     int enc_hidden, enc_layers;    /* e.g. 128, 3 */
     int head_hidden, head_layers;  /* 64, 4 */
-    int table_knots;      /* intervals of the radial table on [table_r_min, r_cut]; 0 = default */
+    int table_knots;      /* intervals of the radial table on [table_r_min, r_cut]; 0 = automatic: 64, doubled until table_tol holds */
     double table_r_min;   /* smallest tabulated distance; 0 = default (1.0) */
     double table_tol;     /* accepted table error relative to max|g|; 0 = default (1e-6) */
     int device;           /* CUDA device ordinal */

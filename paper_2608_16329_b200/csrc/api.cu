@@ -126,7 +126,8 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
     mlip_ctx *c = new (std::nothrow) mlip_ctx();
     if (!c) return fail(nullptr, MLIP_ERR_OOM, "host allocation failed");
     c->cfg = *cfg;
-    if (c->cfg.table_knots <= 0) c->cfg.table_knots = 256;
+    const bool auto_knots = c->cfg.table_knots <= 0;
+    if (auto_knots) c->cfg.table_knots = 64;
     if (c->cfg.table_r_min <= 0.0) c->cfg.table_r_min = 1.0;
     if (c->cfg.table_tol <= 0.0) c->cfg.table_tol = 1e-6;
     if (c->cfg.table_knots > 8192 || c->cfg.table_r_min >= c->cfg.r_cut) { delete c; return fail(nullptr, MLIP_ERR_INVALID_ARG, "bad table parameters"); }
@@ -163,6 +164,11 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
         }
         if ((rc = upload_head(c, head_w)) != MLIP_OK) break;
         rc = build_tables(c, enc_w, n_enc);
+        // automatic knot count: double until the spline meets the tolerance
+        while (auto_knots && rc == MLIP_ERR_TABLE_TOLERANCE && c->cfg.table_knots < 2048) {
+            c->cfg.table_knots *= 2;
+            rc = build_tables(c, enc_w, n_enc);
+        }
     } while (0);
     if (rc != MLIP_OK && rc != MLIP_ERR_TABLE_TOLERANCE) {
         g_last_error = c->err;

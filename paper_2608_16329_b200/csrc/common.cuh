@@ -106,7 +106,8 @@ struct mlip_ctx {
     double *stage_out = nullptr;   // [10]
     int64_t stage_cap = 0;
 
-    bool built = false, forces_current = false;
+    bool built = false, forces_current = false, kernel_ready = false;
+    size_t table_bytes = 0;
     int64_t step = 0;
     int64_t launches = 0;
     size_t resident = 0;

@@ -3,22 +3,26 @@
 // angular features are recomputed in the derivation stage instead of being kept).
 //
 // Work decomposition
-//   A persistent CTA (8 warps) takes tiles of 16 central atoms of ONE species from a global
-//   counter; a warp owns two atoms of the tile.
-//   Encoding    The warp scans the atom's list (lane = entry), keeps the pairs inside r_cut in a
-//               small shared queue, and every 32 queued pairs evaluates harmonics (Eq. 3) and the
+//   One persistent CTA of 16 warps per SM takes tiles of 16 central atoms of ONE species from a
+//   global counter; a warp owns one atom of the tile.  The radial tables of that central species
+//   (one per neighbor species) are staged in shared memory and stay there until the species of
+//   the CTA's tiles changes (tiles are handed out in species order).
+//   Encoding    The warp scans the atom's list (lane = entry), queues the pairs inside r_cut in
+//               shared memory, and every 32 queued pairs evaluates harmonics (Eq. 3) and the
 //               spline basis with lane = pair.  The moment P_i = H^T G (Eq. 4, 16 x n times
-//               n x 32) is then accumulated on the tensor pipe: mma.sync m16n8k8 TF32 with a
-//               three-term hi/lo split of both operands (error ~2^-21, fp32 accumulate), the
-//               radial values g being evaluated straight into the B fragments.
+//               n x 32) is accumulated on the tensor pipe: mma.sync m16n8k8 TF32 with a
+//               three-term hi/lo split of both operands (~2^-21 relative, fp32 accumulate), the
+//               radial values g being evaluated straight into the B fragments.  P_i stays in
+//               the accumulator registers until the derivation.
 //   Invariants  Eq. 5 from the accumulator fragments by three xor-shuffles.
-//   Regression  Eq. 6 forward and reverse for the 16 atoms at once: [16 x K] x [K x 64] layers on
-//               the tensor pipe, weights pre-split and pre-packed in fragment order.
+//   Regression  Eq. 6 forward and reverse for the 16 atoms at once as W X^T on the tensor pipe
+//               (weights pre-split and pre-packed in A-fragment order, 4-way split over the
+//               reduction dimension, elementwise epilogue over all threads).
 //   Derivation  W_i (Eq. 7) is the accumulator fragment of P_i scaled in place: by construction
 //               of the channel permutation it already is the B fragment of the next contraction.
 //               [V; T] = [G; G'] W^T (Eq. 9 and the re-associated Eq. 8 term, U_i never formed)
-//               again on the tensor pipe, 16 pairs per tile; results are transposed through
-//               shared memory to lane = pair for the projection of Eq. 10 and the scatter.
+//               on the tensor pipe, 16 pairs per tile; results are transposed through shared
+//               memory to lane = pair for the projection of Eq. 10 and the scatter.
 // Everything that is not a contraction (geometry, harmonics, splines, projection) stays on the
 // fp32 pipe; positions are differenced in fp64.
 #include <algorithm>
@@ -27,40 +31,50 @@
 
 namespace mlip {
 
-constexpr int TILE = 16;      // atoms per tile (one m16 tile of the head)
-constexpr int NW = 8;         // warps per CTA
+constexpr int TILE = 16;      // atoms per tile = warps per CTA
+constexpr int NW = 16;
 constexpr int PB_CAP = 64;    // queued pairs per warp
 constexpr int ST_STRIDE = 24; // encoding hand-over: 16 h, 4 b, table offset (bank-conflict-free for the fragment reads)
 constexpr int BS_STRIDE = 12; // derivation hand-over: 4 b, 4 b', table offset
 constexpr int VT_STRIDE = 40; // 16 v + 16 t per pair
 constexpr int X_STRIDE = 132; // invariants / dE/dG per atom
 constexpr int Z_STRIDE = 68;  // head activations per atom
+constexpr int TAB_STRIDE_SMEM = 36;   // padded table row in shared memory
 
 constexpr int WARP_WORDS = 6 * PB_CAP + 32 * BS_STRIDE + 32 * VT_STRIDE;   // 384 + 384 + 1280 = 2048
 static_assert(32 * ST_STRIDE <= 32 * BS_STRIDE + 32 * VT_STRIDE, "encoding stage must fit the derivation buffers");
-constexpr int SP_WORDS = TILE * 16 * 32;          // moment fragments of the tile
 constexpr int SX_WORDS = TILE * X_STRIDE;
-constexpr int HEAD_WORDS = 2 * TILE * Z_STRIDE + HEAD_L * TILE * Z_STRIDE;   // activations (ping-pong) + SiLU'
-static_assert(HEAD_WORDS <= NW * WARP_WORDS, "head buffers alias the per-warp buffers");
-constexpr int SMEM_WORDS = SP_WORDS + SX_WORDS + NW * WARP_WORDS + 16;
-constexpr size_t SMEM_BYTES = sizeof(float) * SMEM_WORDS;
+// head buffers (alias of the per-warp buffers)
+constexpr int HB_XS = 0;                                   // split invariants  [16][2 * X_STRIDE]
+constexpr int HB_ZS = HB_XS + TILE * 2 * X_STRIDE;         // split activations [2][16][2 * Z_STRIDE]
+constexpr int HB_SD = HB_ZS + 2 * TILE * 2 * Z_STRIDE;     // SiLU'             [4][16][Z_STRIDE]
+constexpr int HB_DZ = HB_SD + HEAD_L * TILE * Z_STRIDE;    // dE/dz             [16][Z_STRIDE]
+constexpr int HB_DP = HB_DZ + TILE * Z_STRIDE;             // split dE/dpre     [16][2 * Z_STRIDE]
+constexpr int HB_PART = HB_DP + TILE * 2 * Z_STRIDE;       // split-K partials  [4][16][Z_STRIDE] or [2][16][X_STRIDE]
+constexpr int HB_WORDS = HB_PART + 4 * TILE * Z_STRIDE;
+static_assert(2 * TILE * X_STRIDE <= 4 * TILE * Z_STRIDE, "partials of the last reverse layer");
+static_assert(HB_WORDS <= NW * WARP_WORDS, "head buffers alias the per-warp buffers");
+constexpr int FIXED_WORDS = SX_WORDS + NW * WARP_WORDS + 16;
+constexpr int SMEM_LIMIT_WORDS = 227 * 1024 / 4 - 256;
 
-// Pre-packed head weights per species (floats).  Fragment records are float4 {b0_hi, b1_hi, b0_lo, b1_lo}
-// per lane for the B operand of one (n-tile, k-step):
-//   forward  layer L: B[k][n] = W_L[n][k]        n-tiles 8, k-steps K_L / 8
-//   reverse  layer L: B[k][n] = W_L[k][n]        n-tiles K_L / 8, k-steps 8
+// Pre-packed head weights per species (floats).  A record holds the A operand of one
+// (m-tile, k-step): per lane {a0..a3 hi, a0..a3 lo}, i.e. 256 floats.
+//   forward  layer L: A[m][k] = W_L[m][k]   (m = neuron)    4 m-tiles, K_L / 8 k-steps
+//   reverse  layer L: A[m][k] = W_L[k][m]   (m = input)     K_L / 16 m-tiles, 8 k-steps
 // followed by biases [4][64], w_out[64], b_out, pad.
 constexpr int KS0 = N_INV / 8, KS1 = HEAD_H / 8;
-constexpr int FWD_RECORDS = 8 * KS0 + (HEAD_L - 1) * 8 * KS1;
-constexpr int BWD_RECORDS = (N_INV / 8) * 8 + (HEAD_L - 1) * 8 * 8;
+constexpr int FWD_RECORDS = 4 * KS0 + (HEAD_L - 1) * 4 * KS1;
+constexpr int BWD_RECORDS = (N_INV / 16) * 8 + (HEAD_L - 1) * 4 * 8;
 constexpr int HP_FWD = 0;
-constexpr int HP_BWD = HP_FWD + FWD_RECORDS * 128;
-constexpr int HP_BIAS = HP_BWD + BWD_RECORDS * 128;
+constexpr int HP_BWD = HP_FWD + FWD_RECORDS * 256;
+constexpr int HP_BIAS = HP_BWD + BWD_RECORDS * 256;
 constexpr int HP_WOUT = HP_BIAS + HEAD_L * HEAD_H;
 constexpr int HP_TOTAL = HP_WOUT + HEAD_H + 4;
 
+// SiLU and its derivative.  exp through the fast exponential: its error scales with |x| 2^-24 and
+// enters the sigmoid damped by s (1 - s), far below fp32 rounding of the surrounding sums.
 __device__ __forceinline__ float silu_f(float x, float &dsilu) {
-    float s = 1.0f / (1.0f + expf(-x));
+    const float s = __fdividef(1.0f, 1.0f + __expf(-x));
     dsilu = s * (1.0f + x * (1.0f - s));
     return x * s;
 }
@@ -68,6 +82,11 @@ __device__ __forceinline__ float silu_f(float x, float &dsilu) {
 __device__ __forceinline__ void split_tf32(float x, uint32_t &hi, uint32_t &lo) {
     asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hi) : "f"(x));
     lo = __float_as_uint(x - __uint_as_float(hi));
+}
+__device__ __forceinline__ float2 split_pair(float x) {
+    uint32_t hi, lo;
+    split_tf32(x, hi, lo);
+    return make_float2(__uint_as_float(hi), __uint_as_float(lo));
 }
 
 __device__ __forceinline__ void mma_tf32(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
@@ -86,7 +105,6 @@ __device__ __forceinline__ void mma3(float (&c)[4], const uint32_t (&ah)[4], con
     mma_tf32(c, ah[0], ah[1], ah[2], ah[3], bl0, bl1);
     mma_tf32(c, ah[0], ah[1], ah[2], ah[3], bh0, bh1);
 }
-
 // Same product with the main and the small terms kept in separate accumulators.
 __device__ __forceinline__ void mma3s(float (&c)[4], float (&cs)[4], const uint32_t (&ah)[4], const uint32_t (&al)[4],
                                       uint32_t bh0, uint32_t bh1, uint32_t bl0, uint32_t bl1) {
@@ -172,14 +190,6 @@ __device__ __forceinline__ int spline_basis(float r, const TableDesc &tab, float
     return i;
 }
 
-struct Shared {
-    float *sP;      // [TILE][16][32] moment / W fragments
-    float *sX;      // [TILE][X_STRIDE] invariants, then dE/dG
-    float *warp;    // this warp's buffers
-    float *head;    // head activations (alias of all per-warp buffers)
-    int *ctl;       // tile hand-over
-};
-
 struct KernelArgs {
     int64_t n;
     int n_species;
@@ -198,6 +208,14 @@ struct KernelArgs {
     unsigned long long *pair_counter;
     int *status;
     int *tile_counter;
+};
+
+// Where the radial tables of the current central species live: shared memory (rows padded to
+// TAB_STRIDE_SMEM, table index = neighbor species) or, when they do not fit, global memory.
+struct TableView {
+    const float *base;
+    int row_stride;     // floats per row
+    int table_stride;   // floats per neighbor species
 };
 
 // Scan the list of atom i (lane = entry), append the pairs inside r_cut to the warp's queue and
@@ -249,11 +267,11 @@ __device__ __forceinline__ int scan_pairs(const KernelArgs &k, const double4 &pi
 }
 
 // ---------------- Encoding of one atom: returns the moment as accumulator fragments ----------------
-__device__ __forceinline__ int encode_atom(const KernelArgs &k, const double4 &pi, int si, int64_t beg, int64_t end,
+__device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView &tv, const double4 &pi, int64_t beg, int64_t end,
                                            float *wbuf, int lane, float (&Pf)[4][4]) {
     const int g = lane >> 2, t = lane & 3;
     float *pb = wbuf, *stage = wbuf + 6 * PB_CAP;
-    const int table_rows = k.tab.knots + 3;
+    const int rs = tv.row_stride;
 #pragma unroll
     for (int a = 0; a < 4; ++a)
 #pragma unroll
@@ -268,7 +286,7 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const double4 &p
                 harmonics(pb[lane] * rinv, pb[PB_CAP + lane] * rinv, pb[2 * PB_CAP + lane] * rinv, h);
                 const int iv = spline_basis<false>(r, k.tab, b, nullptr, k.status);
                 const int sj = reinterpret_cast<const int *>(pb)[5 * PB_CAP + lane];
-                off = ((si * k.n_species + sj) * table_rows + iv) * K_RADIAL;
+                off = sj * tv.table_stride + iv * rs;
             } else {
 #pragma unroll
                 for (int a = 0; a < D_ANG; ++a) h[a] = 0.f;
@@ -294,10 +312,12 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const double4 &p
             split_tf32(rb[g + 8], ah[3], al[3]);
             // B = G (8 pairs x 8 channels per n-tile): this lane evaluates channels 4g .. 4g+3 (one per n-tile)
             const float4 ba = *reinterpret_cast<const float4 *>(ra + 16), bb = *reinterpret_cast<const float4 *>(rb + 16);
-            const float4 *ta = reinterpret_cast<const float4 *>(k.tab.coef + reinterpret_cast<const int *>(ra)[20]) + g;
-            const float4 *tb = reinterpret_cast<const float4 *>(k.tab.coef + reinterpret_cast<const int *>(rb)[20]) + g;
-            const float4 a0 = __ldg(ta), a1 = __ldg(ta + 8), a2 = __ldg(ta + 16), a3 = __ldg(ta + 24);
-            const float4 b0 = __ldg(tb), b1 = __ldg(tb + 8), b2 = __ldg(tb + 16), b3 = __ldg(tb + 24);
+            const float *ta = tv.base + reinterpret_cast<const int *>(ra)[20] + 4 * g;
+            const float *tb = tv.base + reinterpret_cast<const int *>(rb)[20] + 4 * g;
+            const float4 a0 = *reinterpret_cast<const float4 *>(ta), a1 = *reinterpret_cast<const float4 *>(ta + rs);
+            const float4 a2 = *reinterpret_cast<const float4 *>(ta + 2 * rs), a3 = *reinterpret_cast<const float4 *>(ta + 3 * rs);
+            const float4 b0 = *reinterpret_cast<const float4 *>(tb), b1 = *reinterpret_cast<const float4 *>(tb + rs);
+            const float4 b2 = *reinterpret_cast<const float4 *>(tb + 2 * rs), b3 = *reinterpret_cast<const float4 *>(tb + 3 * rs);
             float ga[4], gb[4];
             ga[0] = ba.x * a0.x + ba.y * a1.x + ba.z * a2.x + ba.w * a3.x;
             ga[1] = ba.x * a0.y + ba.y * a1.y + ba.z * a2.y + ba.w * a3.y;
@@ -323,12 +343,12 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const double4 &p
 }
 
 // ---------------- Derivation of one atom (Eq. 8-10) ----------------
-__device__ __forceinline__ void derive_atom(const KernelArgs &k, const double4 &pi, int i, int si, int64_t beg, int64_t end,
+__device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView &tv, const double4 &pi, int i, int64_t beg, int64_t end,
                                             float *wbuf, int lane, const uint32_t (&Wh)[4][4], const uint32_t (&Wl)[4][4],
                                             float (&vir)[9]) {
     const int g = lane >> 2, t = lane & 3;
     float *pb = wbuf, *bs = wbuf + 6 * PB_CAP, *vt = bs + 32 * BS_STRIDE;
-    const int table_rows = k.tab.knots + 3;
+    const int rs = tv.row_stride;
     float fx = 0.f, fy = 0.f, fz = 0.f;
 
     auto batch = [&](int n) {
@@ -338,7 +358,7 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const double4 &
             if (lane < n) {
                 const int iv = spline_basis<true>(pb[3 * PB_CAP + lane], k.tab, b, db, k.status);
                 const int sj = reinterpret_cast<const int *>(pb)[5 * PB_CAP + lane];
-                off = ((si * k.n_species + sj) * table_rows + iv) * K_RADIAL;
+                off = sj * tv.table_stride + iv * rs;
             }
             float4 *row = reinterpret_cast<float4 *>(bs + lane * BS_STRIDE);
             row[0] = make_float4(b[0], b[1], b[2], b[3]);
@@ -359,13 +379,13 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const double4 &
             for (int q = 0; q < 2; ++q) {
                 const float *rp = bs + (16 * mt + g + 8 * q) * BS_STRIDE;
                 const float4 b = *reinterpret_cast<const float4 *>(rp), db = *reinterpret_cast<const float4 *>(rp + 4);
-                const float4 *tc = reinterpret_cast<const float4 *>(k.tab.coef + reinterpret_cast<const int *>(rp)[8]) + 2 * t;
+                const float *tc = tv.base + reinterpret_cast<const int *>(rp)[8] + 8 * t;
                 const float bw[4] = {b.x, b.y, b.z, b.w}, dbw[4] = {db.x, db.y, db.z, db.w};
 #pragma unroll
                 for (int c = 0; c < 8; ++c) { G[q][c] = 0.f; dG[q][c] = 0.f; }
 #pragma unroll
                 for (int m = 0; m < 4; ++m) {
-                    const float4 c0 = __ldg(tc + 8 * m), c1 = __ldg(tc + 8 * m + 1);
+                    const float4 c0 = *reinterpret_cast<const float4 *>(tc + m * rs), c1 = *reinterpret_cast<const float4 *>(tc + m * rs + 4);
                     const float cv[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
 #pragma unroll
                     for (int c = 0; c < 8; ++c) { G[q][c] += bw[m] * cv[c]; dG[q][c] += dbw[m] * cv[c]; }
@@ -383,17 +403,13 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const double4 &
                 mma3s(T[0], Ts[0], dh, dl, Wh[ks][0], Wh[ks][1], Wl[ks][0], Wl[ks][1]);   // W g' (Eq. 8 re-associated)
                 mma3s(T[1], Ts[1], dh, dl, Wh[ks][2], Wh[ks][3], Wl[ks][2], Wl[ks][3]);
             }
-#pragma unroll
-            for (int a = 0; a < 2; ++a)
-#pragma unroll
-                for (int b = 0; b < 4; ++b) { V[a][b] += Vs[a][b]; T[a][b] += Ts[a][b]; }
             float *va = vt + (16 * mt + g) * VT_STRIDE + 2 * t, *vb = va + 8 * VT_STRIDE;
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
-                *reinterpret_cast<float2 *>(va + 8 * q) = make_float2(V[q][0], V[q][1]);
-                *reinterpret_cast<float2 *>(vb + 8 * q) = make_float2(V[q][2], V[q][3]);
-                *reinterpret_cast<float2 *>(va + 16 + 8 * q) = make_float2(T[q][0], T[q][1]);
-                *reinterpret_cast<float2 *>(vb + 16 + 8 * q) = make_float2(T[q][2], T[q][3]);
+                *reinterpret_cast<float2 *>(va + 8 * q) = make_float2(V[q][0] + Vs[q][0], V[q][1] + Vs[q][1]);
+                *reinterpret_cast<float2 *>(vb + 8 * q) = make_float2(V[q][2] + Vs[q][2], V[q][3] + Vs[q][3]);
+                *reinterpret_cast<float2 *>(va + 16 + 8 * q) = make_float2(T[q][0] + Ts[q][0], T[q][1] + Ts[q][1]);
+                *reinterpret_cast<float2 *>(vb + 16 + 8 * q) = make_float2(T[q][2] + Ts[q][2], T[q][3] + Ts[q][3]);
             }
         }
         __syncwarp();
@@ -439,127 +455,138 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const double4 &
     }
 }
 
-// One layer-sized contraction of the head for the 16 atoms of the tile on the tensor pipe:
-// C[16 x 8] (n-tile nt) = A[16 x 8 nks] B, A read from shared memory through `load_a(k)`.
-template <typename LoadA>
-__device__ __forceinline__ void head_gemm(float (&c)[4], const float4 *__restrict__ rec, int nks, int lane, LoadA load_a) {
+// Head contraction on the tensor pipe: C^T[16 rows of W x 16 atoms] over k-steps [ks0, ks0 + nks).
+// A records come pre-split from global memory, B = activations (hi, lo interleaved) from shared
+// memory with `bstride` floats per atom.  c[nt] covers atoms 8 nt .. 8 nt + 7.
+__device__ __forceinline__ void head_gemm(float (&c)[2][4], const float4 *__restrict__ rec, int ks0, int nks,
+                                          const float *__restrict__ act, int bstride, int lane) {
     const int g = lane >> 2, t = lane & 3;
-    c[0] = c[1] = c[2] = c[3] = 0.f;
-#pragma unroll 4
-    for (int ks = 0; ks < nks; ++ks) {
-        uint32_t ah[4], al[4];
-        split_tf32(load_a(g, 8 * ks + t), ah[0], al[0]);
-        split_tf32(load_a(g + 8, 8 * ks + t), ah[1], al[1]);
-        split_tf32(load_a(g, 8 * ks + t + 4), ah[2], al[2]);
-        split_tf32(load_a(g + 8, 8 * ks + t + 4), ah[3], al[3]);
-        const float4 b = __ldg(rec + ks * 32 + lane);
-        float p[4] = {0.f, 0.f, 0.f, 0.f};
-        mma3(p, ah, al, __float_as_uint(b.x), __float_as_uint(b.y), __float_as_uint(b.z), __float_as_uint(b.w));
-        c[0] += p[0]; c[1] += p[1]; c[2] += p[2]; c[3] += p[3];
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) c[a][b] = 0.f;
+#pragma unroll 2
+    for (int ks = ks0; ks < ks0 + nks; ++ks) {
+        const float4 ah4 = __ldg(rec + (size_t)ks * 64 + 2 * lane), al4 = __ldg(rec + (size_t)ks * 64 + 2 * lane + 1);
+        const uint32_t ah[4] = {__float_as_uint(ah4.x), __float_as_uint(ah4.y), __float_as_uint(ah4.z), __float_as_uint(ah4.w)};
+        const uint32_t al[4] = {__float_as_uint(al4.x), __float_as_uint(al4.y), __float_as_uint(al4.z), __float_as_uint(al4.w)};
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+            const float *row = act + (8 * nt + g) * bstride + 2 * (8 * ks + t);
+            const float2 b0 = *reinterpret_cast<const float2 *>(row), b1 = *reinterpret_cast<const float2 *>(row + 8);
+            float p[4] = {0.f, 0.f, 0.f, 0.f};
+            mma3(p, ah, al, __float_as_uint(b0.x), __float_as_uint(b1.x), __float_as_uint(b0.y), __float_as_uint(b1.y));
+            c[nt][0] += p[0]; c[nt][1] += p[1]; c[nt][2] += p[2]; c[nt][3] += p[3];
+        }
+    }
+}
+
+// c fragments (rows = 16 m + g, g + 8; columns = atoms) -> part[atom][row] with `pstride` floats per atom
+__device__ __forceinline__ void store_partial(const float (&c)[2][4], float *part, int pstride, int m_tile, int lane) {
+    const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt) {
+        float *p = part + (8 * nt + 2 * t) * pstride + 16 * m_tile + g;
+        p[0] = c[nt][0]; p[pstride] = c[nt][1]; p[8] = c[nt][2]; p[pstride + 8] = c[nt][3];
     }
 }
 
 // ---------------- Regression (Eq. 6) forward and reverse for the tile ----------------
-// In: sX = invariants [atom][128].  Out: sX = dE/dG, per-atom energies written, returns nothing.
-__device__ __forceinline__ void head_tile(const KernelArgs &k, const Shared &sh, int species, int count, int first,
+// In: sX = invariants [atom][128].  Out: sX = dE/dG; per-atom energies written.
+__device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float *hb, int species, int count, int first,
                                           int warp, int lane, double &e_sum) {
-    const int g = lane >> 2, t = lane & 3;
     const float *hp = k.head_pack + (size_t)species * HP_TOTAL;
     const float4 *fwd = reinterpret_cast<const float4 *>(hp + HP_FWD), *bwd = reinterpret_cast<const float4 *>(hp + HP_BWD);
-    float *z0 = sh.head, *z1 = sh.head + TILE * Z_STRIDE, *sD = sh.head + 2 * TILE * Z_STRIDE;
-    const float *sX = sh.sX;
+    float *xs = hb + HB_XS, *zs = hb + HB_ZS, *sD = hb + HB_SD, *dz = hb + HB_DZ, *dp = hb + HB_DP, *part = hb + HB_PART;
+    const int mt4 = warp & 3, kq = warp >> 2;   // forward / reverse hidden layers: 4 m-tiles x 4 k-quarters
+    const int atom = warp;                      // elementwise phases: warp = atom, lane = neuron (and neuron + 32)
 
-    // forward: warp = n-tile (8 neurons)
+    // split the invariants once
+    for (int f = lane; f < N_INV; f += 32)
+        *reinterpret_cast<float2 *>(xs + atom * 2 * X_STRIDE + 2 * f) = split_pair(sX[atom * X_STRIDE + f]);
+    __syncthreads();
+
+    float e_i = 0.f;
     for (int L = 0; L < HEAD_L; ++L) {
-        const float *zin = (L & 1) ? z0 : z1;   // layer L >= 1 reads what layer L-1 wrote
-        float *zout = (L & 1) ? z1 : z0;
-        float c[4];
-        if (L == 0) {
-            head_gemm(c, fwd + (size_t)(warp * KS0) * 32, KS0, lane, [&](int row, int col) { return sX[row * X_STRIDE + col]; });
-        } else {
-            const float4 *rec = fwd + (size_t)(8 * KS0 + (L - 1) * 8 * KS1 + warp * KS1) * 32;
-            head_gemm(c, rec, KS1, lane, [&](int row, int col) { return zin[row * Z_STRIDE + col]; });
-        }
-        const int n0 = 8 * warp + 2 * t;
-        const float b0 = __ldg(hp + HP_BIAS + L * HEAD_H + n0), b1 = __ldg(hp + HP_BIAS + L * HEAD_H + n0 + 1);
-        float d0, d1, d2, d3;
-        float y0 = silu_f(c[0] + b0, d0), y1 = silu_f(c[1] + b1, d1), y2 = silu_f(c[2] + b0, d2), y3 = silu_f(c[3] + b1, d3);
-        if (L > 0) {   // residual
-            y0 += zin[g * Z_STRIDE + n0]; y1 += zin[g * Z_STRIDE + n0 + 1];
-            y2 += zin[(g + 8) * Z_STRIDE + n0]; y3 += zin[(g + 8) * Z_STRIDE + n0 + 1];
-        }
-        *reinterpret_cast<float2 *>(zout + g * Z_STRIDE + n0) = make_float2(y0, y1);
-        *reinterpret_cast<float2 *>(zout + (g + 8) * Z_STRIDE + n0) = make_float2(y2, y3);
-        *reinterpret_cast<float2 *>(sD + (L * TILE + g) * Z_STRIDE + n0) = make_float2(d0, d1);
-        *reinterpret_cast<float2 *>(sD + (L * TILE + g + 8) * Z_STRIDE + n0) = make_float2(d2, d3);
+        const float *zin = zs + ((L + 1) & 1) * TILE * 2 * Z_STRIDE;
+        float *zout = zs + (L & 1) * TILE * 2 * Z_STRIDE;
+        float c[2][4];
+        if (L == 0) head_gemm(c, fwd + (size_t)(mt4 * KS0) * 64, kq * (KS0 / 4), KS0 / 4, xs, 2 * X_STRIDE, lane);
+        else head_gemm(c, fwd + (size_t)(4 * KS0 + (L - 1) * 4 * KS1 + mt4 * KS1) * 64, kq * (KS1 / 4), KS1 / 4, zin, 2 * Z_STRIDE, lane);
+        store_partial(c, part + kq * TILE * Z_STRIDE, Z_STRIDE, mt4, lane);
         __syncthreads();
-    }
-    // the last layer (L = 3) wrote z1.  Energies: warp w sums atoms 2w, 2w+1.
-    {
-        const float w0 = __ldg(hp + HP_WOUT + lane), w1 = __ldg(hp + HP_WOUT + 32 + lane), bo = __ldg(hp + HP_WOUT + HEAD_H);
+        // elementwise: bias, SiLU, residual; this thread owns neurons lane and lane + 32 of its atom
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
-            const int a = 2 * warp + q;
-            float e = w0 * z1[a * Z_STRIDE + lane] + w1 * z1[a * Z_STRIDE + 32 + lane];
-#pragma unroll
-            for (int o = 16; o; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
-            e += bo;
-            if (lane == 0 && a < count) {
-                k.e_atom[__ldg(k.center_order + first + a)] = e;
-                e_sum += (double)e;
+            const int nn = lane + 32 * q;
+            const float *pp = part + atom * Z_STRIDE + nn;
+            const float pre = ((pp[0] + pp[TILE * Z_STRIDE]) + (pp[2 * TILE * Z_STRIDE] + pp[3 * TILE * Z_STRIDE])) + __ldg(hp + HP_BIAS + L * HEAD_H + nn);
+            float d, y = silu_f(pre, d);
+            if (L > 0) { const float2 zi = *reinterpret_cast<const float2 *>(zin + atom * 2 * Z_STRIDE + 2 * nn); y += zi.x + zi.y; }
+            sD[(L * TILE + atom) * Z_STRIDE + nn] = d;
+            if (L < HEAD_L - 1) {
+                *reinterpret_cast<float2 *>(zout + atom * 2 * Z_STRIDE + 2 * nn) = split_pair(y);
+            } else {   // output layer and the start of the reverse pass: dE/dz = w_out
+                const float wo = __ldg(hp + HP_WOUT + nn);
+                e_i += wo * y;
+                dz[atom * Z_STRIDE + nn] = wo;
+                *reinterpret_cast<float2 *>(dp + atom * 2 * Z_STRIDE + 2 * nn) = split_pair(wo * d);
             }
         }
-    }
-    __syncthreads();
-    // reverse: dZ starts as w_out for every atom (written into z0), then layers 3, 2, 1 with their skip paths
-    for (int idx = threadIdx.x; idx < TILE * HEAD_H; idx += NW * 32)
-        z0[(idx >> 6) * Z_STRIDE + (idx & 63)] = __ldg(hp + HP_WOUT + (idx & 63));
-    __syncthreads();
-    int flip = 0;   // dZ currently in z0
-    for (int L = HEAD_L - 1; L >= 1; --L) {
-        const float *din = flip ? z1 : z0;
-        float *dout = flip ? z0 : z1;
-        const float *dact = sD + L * TILE * Z_STRIDE;
-        const float4 *rec = bwd + (size_t)((N_INV / 8) * 8 + (L - 1) * 64 + warp * 8) * 32;
-        float c[4];
-        head_gemm(c, rec, 8, lane, [&](int row, int col) { return din[row * Z_STRIDE + col] * dact[row * Z_STRIDE + col]; });
-        const int n0 = 8 * warp + 2 * t;
-        *reinterpret_cast<float2 *>(dout + g * Z_STRIDE + n0) = make_float2(c[0] + din[g * Z_STRIDE + n0], c[1] + din[g * Z_STRIDE + n0 + 1]);
-        *reinterpret_cast<float2 *>(dout + (g + 8) * Z_STRIDE + n0) =
-            make_float2(c[2] + din[(g + 8) * Z_STRIDE + n0], c[3] + din[(g + 8) * Z_STRIDE + n0 + 1]);
-        flip ^= 1;
         __syncthreads();
     }
-    {   // first layer: dE/dG [16 x 128], two n-tiles per warp, written over the invariants
-        const float *din = flip ? z1 : z0;
-        const float *dact = sD;
+#pragma unroll
+    for (int o = 16; o; o >>= 1) e_i += __shfl_xor_sync(0xffffffffu, e_i, o);
+    e_i += __ldg(hp + HP_WOUT + HEAD_H);
+    if (lane == 0 && atom < count) {
+        k.e_atom[__ldg(k.center_order + first + atom)] = e_i;
+        e_sum += (double)e_i;
+    }
+
+    // reverse through the hidden layers 3, 2, 1 (each with its skip path)
+    for (int L = HEAD_L - 1; L >= 1; --L) {
+        float c[2][4];
+        head_gemm(c, bwd + (size_t)((N_INV / 16) * 8 + (L - 1) * 32 + mt4 * 8) * 64, kq * 2, 2, dp, 2 * Z_STRIDE, lane);
+        store_partial(c, part + kq * TILE * Z_STRIDE, Z_STRIDE, mt4, lane);
+        __syncthreads();
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
-            const int nt = warp + 8 * q;
-            float c[4];
-            head_gemm(c, bwd + (size_t)(nt * 8) * 32, 8, lane, [&](int row, int col) { return din[row * Z_STRIDE + col] * dact[row * Z_STRIDE + col]; });
-            const int n0 = 8 * nt + 2 * t;
-            *reinterpret_cast<float2 *>(sh.sX + g * X_STRIDE + n0) = make_float2(c[0], c[1]);
-            *reinterpret_cast<float2 *>(sh.sX + (g + 8) * X_STRIDE + n0) = make_float2(c[2], c[3]);
+            const int nn = lane + 32 * q;
+            const float *pp = part + atom * Z_STRIDE + nn;
+            const float dzn = dz[atom * Z_STRIDE + nn] + ((pp[0] + pp[TILE * Z_STRIDE]) + (pp[2 * TILE * Z_STRIDE] + pp[3 * TILE * Z_STRIDE]));
+            dz[atom * Z_STRIDE + nn] = dzn;
+            *reinterpret_cast<float2 *>(dp + atom * 2 * Z_STRIDE + 2 * nn) = split_pair(dzn * sD[((L - 1) * TILE + atom) * Z_STRIDE + nn]);
         }
+        __syncthreads();
+    }
+    {   // first layer: dE/dG [128 x 16]: 8 m-tiles x 2 k-halves
+        const int mt8 = warp & 7, kh = warp >> 3;
+        float c[2][4];
+        head_gemm(c, bwd + (size_t)(mt8 * 8) * 64, kh * 4, 4, dp, 2 * Z_STRIDE, lane);
+        store_partial(c, part + kh * TILE * X_STRIDE, X_STRIDE, mt8, lane);
+        __syncthreads();
+        for (int f = lane; f < N_INV; f += 32)
+            sX[atom * X_STRIDE + f] = part[atom * X_STRIDE + f] + part[TILE * X_STRIDE + atom * X_STRIDE + f];
     }
     __syncthreads();
 }
 
-__global__ void __launch_bounds__(NW * 32, 2) k_mega(KernelArgs k) {
+template <bool TAB_SMEM>
+__global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words) {
     extern __shared__ __align__(16) float smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
-    Shared sh;
-    sh.sP = smem;
-    sh.sX = smem + SP_WORDS;
-    sh.head = sh.sX + SX_WORDS;
-    sh.warp = sh.head + warp * WARP_WORDS;
-    sh.ctl = reinterpret_cast<int *>(sh.head + NW * WARP_WORDS);
+    float *s_tab = smem;                         // [C][rows][TAB_STRIDE_SMEM] when TAB_SMEM
+    float *sX = smem + (TAB_SMEM ? tab_words : 0);
+    float *hb = sX + SX_WORDS;                   // head buffers = all per-warp buffers
+    float *wbuf = hb + warp * WARP_WORDS;
+    int *ctl = reinterpret_cast<int *>(hb + NW * WARP_WORDS);
+    const int rows = k.tab.knots + 3;
 
     // species-pure tiles: tiles of species s start at tile_first[s]
     int tile_first[MAX_SPECIES + 1];
     tile_first[0] = 0;
+#pragma unroll
     for (int s = 0; s < MAX_SPECIES; ++s) {
         int cnt = s < k.n_species ? __ldg(k.species_start + s + 1) - __ldg(k.species_start + s) : 0;
         tile_first[s + 1] = tile_first[s] + (cnt + TILE - 1) / TILE;
@@ -569,37 +596,48 @@ __global__ void __launch_bounds__(NW * 32, 2) k_mega(KernelArgs k) {
     double e_sum = 0.0;
     float vir[9] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     unsigned long long n_pairs = 0;
+    int loaded_species = -1;
+    TableView tv;
 
     while (true) {
         __syncthreads();
-        if (threadIdx.x == 0) sh.ctl[0] = atomicAdd(k.tile_counter, 1);
+        if (threadIdx.x == 0) ctl[0] = atomicAdd(k.tile_counter, 1);
         __syncthreads();
-        const int tile = sh.ctl[0];
+        const int tile = ctl[0];
         if (tile >= n_tiles) break;
         int species = 0;
-        while (tile >= tile_first[species + 1]) ++species;
+#pragma unroll
+        for (int s = 1; s < MAX_SPECIES; ++s) species += tile >= tile_first[s] ? 1 : 0;
         const int s_beg = __ldg(k.species_start + species), s_end = __ldg(k.species_start + species + 1);
         const int first = s_beg + (tile - tile_first[species]) * TILE;
         const int count = min(TILE, s_end - first);
 
-        // ---------------- Encoding + invariants ----------------
-#pragma unroll 1
-        for (int q = 0; q < 2; ++q) {
-            const int a = 2 * warp + q;
-            float *xrow = sh.sX + a * X_STRIDE;
-            if (a >= count) {   // empty slot of a ragged tile: feed zeros to the head
-                for (int c = lane; c < N_INV; c += 32) xrow[c] = 0.f;
-                continue;
+        if (species != loaded_species) {   // radial tables of this central species
+            if (TAB_SMEM) {
+                const float4 *src = reinterpret_cast<const float4 *>(k.tab.coef + (size_t)species * k.n_species * rows * K_RADIAL);
+                const int n4 = k.n_species * rows * (K_RADIAL / 4);
+                for (int idx = threadIdx.x; idx < n4; idx += NW * 32)
+                    *reinterpret_cast<float4 *>(s_tab + (idx >> 3) * TAB_STRIDE_SMEM + 4 * (idx & 7)) = __ldg(src + idx);
+                tv.base = s_tab; tv.row_stride = TAB_STRIDE_SMEM; tv.table_stride = rows * TAB_STRIDE_SMEM;
+            } else {
+                tv.base = k.tab.coef + (size_t)species * k.n_species * rows * K_RADIAL;
+                tv.row_stride = K_RADIAL; tv.table_stride = rows * K_RADIAL;
             }
-            const int i = __ldg(k.center_order + first + a);
-            const double4 pi = k.pos4[i];
-            float Pf[4][4];
-            n_pairs += encode_atom(k, pi, species, k.nbr_off[i], k.nbr_off[i + 1], sh.warp, lane, Pf);
-            float *prow = sh.sP + a * 16 * 32;
-#pragma unroll
-            for (int nt = 0; nt < 4; ++nt)
-#pragma unroll
-                for (int r = 0; r < 4; ++r) prow[(4 * nt + r) * 32 + lane] = Pf[nt][r];
+            loaded_species = species;
+            __syncthreads();
+        }
+
+        // ---------------- Encoding + invariants: warp = atom ----------------
+        const bool have = warp < count;
+        const int i = have ? __ldg(k.center_order + first + warp) : 0;
+        double4 pi = make_double4(0.0, 0.0, 0.0, 0.0);
+        int64_t beg = 0, end = 0;
+        float Pf[4][4];
+        float *xrow = sX + warp * X_STRIDE;
+        if (have) {
+            pi = k.pos4[i];
+            beg = k.nbr_off[i]; end = k.nbr_off[i + 1];
+            n_pairs += encode_atom(k, tv, pi, beg, end, wbuf, lane, Pf);
             // Eq. 5 (C_l = I): this lane holds rows a = g, g + 8 of channels 8t + j; sum squares over the rows of a block
             float part[4][8];
 #pragma unroll
@@ -623,21 +661,17 @@ __global__ void __launch_bounds__(NW * 32, 2) k_mega(KernelArgs k) {
                     *reinterpret_cast<float4 *>(xrow + 32 * l + 8 * t + 4) = make_float4(part[l][4], part[l][5], part[l][6], part[l][7]);
                 }
             }
+        } else {   // empty slot of a ragged tile: feed zeros to the head
+            for (int c = lane; c < N_INV; c += 32) xrow[c] = 0.f;
         }
         __syncthreads();
 
         // ---------------- Regression ----------------
-        head_tile(k, sh, species, count, first, warp, lane, e_sum);
+        head_tile(k, sX, hb, species, count, first, warp, lane, e_sum);
 
         // ---------------- Derivation ----------------
-#pragma unroll 1
-        for (int q = 0; q < 2; ++q) {
-            const int a = 2 * warp + q;
-            if (a >= count) continue;
-            const int i = __ldg(k.center_order + first + a);
-            const double4 pi = k.pos4[i];
+        if (have) {
             // W_i = dE_i/dP_i (Eq. 7), already in B-fragment order
-            const float *xrow = sh.sX + a * X_STRIDE, *prow = sh.sP + a * 16 * 32;
             const int la = g == 0 ? 0 : (g <= 3 ? 1 : 2), lb = g == 0 ? 2 : 3;
             float da[8], db[8];
             {
@@ -649,18 +683,16 @@ __global__ void __launch_bounds__(NW * 32, 2) k_mega(KernelArgs k) {
             uint32_t Wh[4][4], Wl[4][4];
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) {
-                const float p0 = prow[(4 * ks + 0) * 32 + lane], p1 = prow[(4 * ks + 1) * 32 + lane];
-                const float p2 = prow[(4 * ks + 2) * 32 + lane], p3 = prow[(4 * ks + 3) * 32 + lane];
-                const float w0 = g == 0 ? da[ks] : 2.f * da[ks] * p0;          // row a = g,     channel 8t + ks
-                const float w1 = g == 0 ? da[4 + ks] : 2.f * da[4 + ks] * p1;  // row a = g,     channel 8t + 4 + ks
-                const float w2 = 2.f * db[ks] * p2;                            // row a = g + 8, channel 8t + ks
-                const float w3 = 2.f * db[4 + ks] * p3;                        // row a = g + 8, channel 8t + 4 + ks
+                const float w0 = g == 0 ? da[ks] : 2.f * da[ks] * Pf[ks][0];          // row a = g,     channel 8t + ks
+                const float w1 = g == 0 ? da[4 + ks] : 2.f * da[4 + ks] * Pf[ks][1];  // row a = g,     channel 8t + 4 + ks
+                const float w2 = 2.f * db[ks] * Pf[ks][2];                            // row a = g + 8, channel 8t + ks
+                const float w3 = 2.f * db[4 + ks] * Pf[ks][3];                        // row a = g + 8, channel 8t + 4 + ks
                 split_tf32(w0, Wh[ks][0], Wl[ks][0]);
                 split_tf32(w1, Wh[ks][1], Wl[ks][1]);
                 split_tf32(w2, Wh[ks][2], Wl[ks][2]);
                 split_tf32(w3, Wh[ks][3], Wl[ks][3]);
             }
-            derive_atom(k, pi, i, species, k.nbr_off[i], k.nbr_off[i + 1], sh.warp, lane, Wh, Wl, vir);
+            derive_atom(k, tv, pi, i, beg, end, wbuf, lane, Wh, Wl, vir);
         }
     }
 
@@ -687,6 +719,9 @@ static inline void split_host(float x, float &hi, float &lo) {
     lo = x - hi;
 }
 
+int table_smem_words(const mlip_ctx *c) { return c->cfg.n_species * (c->cfg.table_knots + 3) * TAB_STRIDE_SMEM; }
+bool tables_fit_smem(const mlip_ctx *c) { return FIXED_WORDS + table_smem_words(c) <= SMEM_LIMIT_WORDS; }
+
 int upload_head(mlip_ctx *c, const double *w) {
     const int C = c->cfg.n_species;
     float *host = (float *)calloc((size_t)C * HP_TOTAL, sizeof(float));
@@ -698,28 +733,33 @@ int upload_head(mlip_ctx *c, const double *w) {
         int in = N_INV;
         for (int L = 0; L < HEAD_L; ++L) {
             const int nks = in / 8;
-            // forward: B[k][n] = W[n][k]; record (nt, ks), lane (g, t): b0 = W[8nt+g][8ks+t], b1 = W[8nt+g][8ks+t+4]
-            for (int nt = 0; nt < 8; ++nt)
+            // forward: A[m][k] = W[m][k]; record (mt, ks), lane (g, t):
+            //   a0 = W[16mt+g][8ks+t], a1 = W[16mt+g+8][8ks+t], a2 = W[16mt+g][8ks+t+4], a3 = W[16mt+g+8][8ks+t+4]
+            for (int mt = 0; mt < 4; ++mt)
                 for (int ks = 0; ks < nks; ++ks)
                     for (int lane = 0; lane < 32; ++lane) {
                         const int g = lane >> 2, t = lane & 3;
-                        float *rec = fwd + ((size_t)(nt * nks + ks) * 32 + lane) * 4;
-                        split_host((float)src[(8 * nt + g) * in + 8 * ks + t], rec[0], rec[2]);
-                        split_host((float)src[(8 * nt + g) * in + 8 * ks + t + 4], rec[1], rec[3]);
+                        float *rec = fwd + ((size_t)(mt * nks + ks) * 32 + lane) * 8;
+                        split_host((float)src[(16 * mt + g) * in + 8 * ks + t], rec[0], rec[4]);
+                        split_host((float)src[(16 * mt + g + 8) * in + 8 * ks + t], rec[1], rec[5]);
+                        split_host((float)src[(16 * mt + g) * in + 8 * ks + t + 4], rec[2], rec[6]);
+                        split_host((float)src[(16 * mt + g + 8) * in + 8 * ks + t + 4], rec[3], rec[7]);
                     }
-            // reverse: B[k][n] = W[k][n] (k = neuron, n = input); record (nt, ks): b0 = W[8ks+t][8nt+g], b1 = W[8ks+t+4][8nt+g]
-            for (int nt = 0; nt < in / 8; ++nt)
+            // reverse: A[m][k] = W[k][m] (m = input, k = neuron); record (mt, ks)
+            for (int mt = 0; mt < in / 16; ++mt)
                 for (int ks = 0; ks < 8; ++ks)
                     for (int lane = 0; lane < 32; ++lane) {
                         const int g = lane >> 2, t = lane & 3;
-                        float *rec = bwd + ((size_t)(nt * 8 + ks) * 32 + lane) * 4;
-                        split_host((float)src[(8 * ks + t) * in + 8 * nt + g], rec[0], rec[2]);
-                        split_host((float)src[(8 * ks + t + 4) * in + 8 * nt + g], rec[1], rec[3]);
+                        float *rec = bwd + ((size_t)(mt * 8 + ks) * 32 + lane) * 8;
+                        split_host((float)src[(8 * ks + t) * in + 16 * mt + g], rec[0], rec[4]);
+                        split_host((float)src[(8 * ks + t) * in + 16 * mt + g + 8], rec[1], rec[5]);
+                        split_host((float)src[(8 * ks + t + 4) * in + 16 * mt + g], rec[2], rec[6]);
+                        split_host((float)src[(8 * ks + t + 4) * in + 16 * mt + g + 8], rec[3], rec[7]);
                     }
             for (int o = 0; o < HEAD_H; ++o) hp[HP_BIAS + L * HEAD_H + o] = (float)src[in * HEAD_H + o];
             src += in * HEAD_H + HEAD_H;
-            fwd += (size_t)8 * nks * 128;
-            bwd += (size_t)(in / 8) * 8 * 128;
+            fwd += (size_t)4 * nks * 256;
+            bwd += (size_t)(in / 16) * 8 * 256;
             in = HEAD_H;
         }
         for (int o = 0; o < HEAD_H + 1; ++o) hp[HP_WOUT + o] = (float)src[o];
@@ -729,8 +769,6 @@ int upload_head(mlip_ctx *c, const double *w) {
     free(host);
     if (e != cudaSuccess) { c->err = cudaGetErrorString(e); return MLIP_ERR_CUDA; }
     c->resident += sizeof(float) * (size_t)C * HP_TOTAL;
-    e = cudaFuncSetAttribute(k_mega, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
-    if (e != cudaSuccess) { c->err = std::string("fused kernel shared memory: ") + cudaGetErrorString(e); return MLIP_ERR_CUDA; }
     return MLIP_OK;
 }
 
@@ -741,7 +779,16 @@ int launch_megakernel(mlip_ctx *c, cudaStream_t s) {
     MLIP_CUDA_TRY(c, cudaMemsetAsync(c->pair_counter, 0, sizeof(unsigned long long), s));
     MLIP_CUDA_TRY(c, cudaMemsetAsync(c->tile_counter, 0, sizeof(int), s));
     const int64_t tiles_max = (n + TILE - 1) / TILE + c->cfg.n_species;
-    const int blocks = (int)std::min<int64_t>(tiles_max, (int64_t)c->n_sm * 2);
+    const int blocks = (int)std::min<int64_t>(tiles_max, (int64_t)c->n_sm);
+    const bool in_smem = tables_fit_smem(c);
+    const int tab_words = in_smem ? table_smem_words(c) : 0;
+    const size_t smem_bytes = sizeof(float) * (size_t)(FIXED_WORDS + tab_words);
+    if (!c->kernel_ready) {
+        cudaError_t e = in_smem ? cudaFuncSetAttribute(k_mega<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes)
+                                : cudaFuncSetAttribute(k_mega<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+        if (e != cudaSuccess) { c->err = std::string("fused kernel shared memory: ") + cudaGetErrorString(e); return MLIP_ERR_CUDA; }
+        c->kernel_ready = true;
+    }
     KernelArgs k;
     k.n = n; k.n_species = c->cfg.n_species; k.grid = c->grid; k.rc2 = c->cfg.r_cut * c->cfg.r_cut; k.tab = c->tab;
     k.pos4 = c->pos4; k.center_order = c->center_order; k.species_start = c->species_start;
@@ -749,7 +796,8 @@ int launch_megakernel(mlip_ctx *c, cudaStream_t s) {
     k.acc = c->acc; k.pair_counter = c->pair_counter; k.status = c->status; k.tile_counter = c->tile_counter;
     const int slot = (int)(c->ev_count % mlip_ctx::EV_POOL);
     MLIP_CUDA_TRY(c, cudaEventRecord(c->ev[2 * slot], s));
-    k_mega<<<blocks, NW * 32, SMEM_BYTES, s>>>(k);
+    if (in_smem) k_mega<true><<<blocks, NW * 32, smem_bytes, s>>>(k, tab_words);
+    else k_mega<false><<<blocks, NW * 32, smem_bytes, s>>>(k, tab_words);
     MLIP_CUDA_TRY(c, cudaEventRecord(c->ev[2 * slot + 1], s));
     c->ev_count += 1;
     c->launches += 1;

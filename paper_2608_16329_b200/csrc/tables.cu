@@ -145,8 +145,11 @@ int build_tables(mlip_ctx *c, const double *enc_w_host, size_t n_enc) {
     MLIP_CUDA_TRY(c, cudaMalloc(&work, sizeof(double) * (size_t)n_nets * k * 2 * n_knot_pts));
     MLIP_CUDA_TRY(c, cudaMalloc(&stats, sizeof(unsigned long long) * 4));
     const size_t coef_bytes = sizeof(float) * (size_t)n_nets * (K + 3) * k;
+    if (c->table) { cudaFree(c->table); c->table = nullptr; c->resident -= c->table_bytes; }   // a retry with more knots
     MLIP_CUDA_TRY(c, cudaMalloc(&c->table, coef_bytes));
+    c->table_bytes = coef_bytes;
     c->resident += coef_bytes;
+    c->kernel_ready = false;
     MLIP_CUDA_TRY(c, cudaMemcpy(w, enc_w_host, sizeof(double) * n_enc, cudaMemcpyHostToDevice));
     MLIP_CUDA_TRY(c, cudaMemset(stats, 0, sizeof(unsigned long long) * 4));
 
