@@ -13,7 +13,7 @@ import os
 import numpy as np
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libmlip_b200.so")
+LIB_PATH = os.environ.get("MLIP_B200_LIB") or os.path.join(_PKG, "libmlip_b200.so")
 
 OK = 0
 ERRORS = {0: "MLIP_OK", 1: "MLIP_ERR_INVALID_ARG", 2: "MLIP_ERR_UNSUPPORTED", 3: "MLIP_ERR_BOX_TOO_SMALL",

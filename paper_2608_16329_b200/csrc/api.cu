@@ -189,7 +189,8 @@ int mlip_table_error(const mlip_ctx *c, double *err_value, double *err_deriv) {
 
 int mlip_build_neighbors(mlip_ctx *c, int64_t n, const double *pos, const int32_t *species, const double *box, void *stream) {
     if (!c) return MLIP_ERR_INVALID_ARG;
-    if (n < 1 || n > 2000000000LL || !pos || !species || !box) return fail(c, MLIP_ERR_INVALID_ARG, "bad arguments to mlip_build_neighbors");
+    if (n < 1 || !pos || !species || !box) return fail(c, MLIP_ERR_INVALID_ARG, "bad arguments to mlip_build_neighbors");
+    if (n > (1LL << 28)) return fail(c, MLIP_ERR_UNSUPPORTED, "more than 2^28 atoms per context (the pair queue packs index and species in 32 bits)");
     cudaStream_t s = (cudaStream_t)stream;
     c->last_stream = s;
     cudaSetDevice(c->cfg.device);
@@ -372,6 +373,13 @@ int mlip_kernel_time(mlip_ctx *c, int64_t *n_launches, double *total_ms, int res
     if (reset) c->ev_count = 0;
     return MLIP_OK;
 }
+
+#ifdef MLIP_PHASE_CLOCKS
+int mlip_debug_acc(mlip_ctx *c, double *out16) {   // profiling builds only
+    cudaDeviceSynchronize();
+    return cudaMemcpy(out16, c->acc, sizeof(double) * ACC_COUNT, cudaMemcpyDeviceToHost) == cudaSuccess ? MLIP_OK : MLIP_ERR_CUDA;
+}
+#endif
 
 size_t mlip_resident_bytes(const mlip_ctx *c) { return c ? c->resident : 0; }
 

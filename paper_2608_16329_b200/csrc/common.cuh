@@ -29,7 +29,7 @@ enum : int {
 };
 
 // accumulator slots (double)
-enum : int { ACC_ENERGY = 0, ACC_VIRIAL = 1, ACC_KINETIC = 10, ACC_COUNT = 16 };
+enum : int { ACC_ENERGY = 0, ACC_VIRIAL = 1, ACC_KINETIC = 10, ACC_COUNT = 32 };
 
 struct CellGrid {
     int n[3];          // cells per dimension

@@ -33,7 +33,8 @@ namespace mlip {
 
 constexpr int TILE = 16;      // atoms per tile = warps per CTA
 constexpr int NW = 16;
-constexpr int PB_CAP = 64;    // queued pairs per warp
+constexpr int PB_CAP = 160;   // queued pairs per warp: up to 31 left over + four list chunks of 32
+constexpr int J_BITS = 28;    // queue entries pack the neighbor index (low 28 bits) with its species
 constexpr int ST_STRIDE = 24; // encoding hand-over: 16 h, 4 b, table offset (bank-conflict-free for the fragment reads)
 constexpr int BS_STRIDE = 12; // derivation hand-over: 4 b, 4 b', table offset
 constexpr int VT_STRIDE = 40; // 16 v + 16 t per pair
@@ -41,8 +42,9 @@ constexpr int X_STRIDE = 132; // invariants / dE/dG per atom
 constexpr int Z_STRIDE = 68;  // head activations per atom
 constexpr int TAB_STRIDE_SMEM = 36;   // padded table row in shared memory
 
-constexpr int WARP_WORDS = 6 * PB_CAP + 32 * BS_STRIDE + 32 * VT_STRIDE;   // 384 + 384 + 1280 = 2048
-static_assert(32 * ST_STRIDE <= 32 * BS_STRIDE + 32 * VT_STRIDE, "encoding stage must fit the derivation buffers");
+constexpr int Q_WORDS = 4 * PB_CAP;                             // pair queue of a warp: kept from encoding to derivation
+constexpr int SCR_WORDS = 32 * BS_STRIDE + 32 * VT_STRIDE;      // scratch of a warp: 384 + 1280
+static_assert(32 * ST_STRIDE <= SCR_WORDS, "encoding stage must fit the derivation buffers");
 constexpr int SX_WORDS = TILE * X_STRIDE;
 // head buffers (alias of the per-warp buffers)
 constexpr int HB_XS = 0;                                   // split invariants  [16][2 * X_STRIDE]
@@ -53,8 +55,9 @@ constexpr int HB_DP = HB_DZ + TILE * Z_STRIDE;             // split dE/dpre     
 constexpr int HB_PART = HB_DP + TILE * 2 * Z_STRIDE;       // split-K partials  [4][16][Z_STRIDE] or [2][16][X_STRIDE]
 constexpr int HB_WORDS = HB_PART + 4 * TILE * Z_STRIDE;
 static_assert(2 * TILE * X_STRIDE <= 4 * TILE * Z_STRIDE, "partials of the last reverse layer");
-static_assert(HB_WORDS <= NW * WARP_WORDS, "head buffers alias the per-warp buffers");
-constexpr int FIXED_WORDS = SX_WORDS + NW * WARP_WORDS + 16;
+static_assert(HB_WORDS <= NW * SCR_WORDS, "head buffers alias the per-warp scratch");
+constexpr int HC_WORDS = HEAD_L * HEAD_H + HEAD_H + 16;         // biases, w_out, b_out of the current species
+constexpr int FIXED_WORDS = SX_WORDS + NW * (Q_WORDS + SCR_WORDS) + HC_WORDS + 16;
 constexpr int SMEM_LIMIT_WORDS = 227 * 1024 / 4 - 256;
 
 // Pre-packed head weights per species (floats).  A record holds the A operand of one
@@ -90,7 +93,7 @@ __device__ __forceinline__ float2 split_pair(float x) {
 }
 
 __device__ __forceinline__ void mma_tf32(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+    asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
@@ -190,6 +193,23 @@ __device__ __forceinline__ int spline_basis(float r, const TableDesc &tab, float
     return i;
 }
 
+// Optional per-phase cycle counters (profiling builds only: -DMLIP_PHASE_CLOCKS).  Slots 16.. of
+// the accumulator array receive the summed clock64 ticks of lane 0 of every warp.
+#ifdef MLIP_PHASE_CLOCKS
+struct PhaseClock {
+    long long t, acc[16];
+    __device__ __forceinline__ void start() { t = clock64(); for (int q = 0; q < 16; ++q) acc[q] = 0; }
+    __device__ __forceinline__ void mark(int slot) { const long long now = clock64(); acc[slot] += now - t; t = now; }
+    __device__ __forceinline__ void flush(double *a, int lane) { if (lane == 0) for (int q = 0; q < 16; ++q) atomicAdd(&a[16 + q], (double)acc[q]); }
+};
+#else
+struct PhaseClock {
+    __device__ __forceinline__ void start() {}
+    __device__ __forceinline__ void mark(int) {}
+    __device__ __forceinline__ void flush(double *, int) {}
+};
+#endif
+
 struct KernelArgs {
     int64_t n;
     int n_species;
@@ -218,74 +238,63 @@ struct TableView {
     int table_stride;   // floats per neighbor species
 };
 
-// Scan the list of atom i (lane = entry), append the pairs inside r_cut to the warp's queue and
-// hand every 32 queued pairs (and the remainder) to `batch(n)`, which consumes entries [0, n).
-template <typename Batch>
-__device__ __forceinline__ int scan_pairs(const KernelArgs &k, const double4 &pi, int64_t beg, int64_t end, float *pb, int lane, Batch batch) {
-    float *px = pb, *py = pb + PB_CAP, *pz = pb + 2 * PB_CAP, *pr = pb + 3 * PB_CAP;
-    int *pj = reinterpret_cast<int *>(pb + 4 * PB_CAP), *ps = reinterpret_cast<int *>(pb + 5 * PB_CAP);
-    int nq = 0, total = 0;
-    for (int64_t base = beg; base < end; base += 32) {
-        const int64_t e = base + lane;
-        bool valid = false;
-        float x = 0.f, y = 0.f, z = 0.f, r = 1.f;
-        int j = 0, sj = 0;
-        if (e < end) {
-            j = __ldg(k.nbr + e);
-            const double4 pj4 = k.pos4[j];
-            double dx = min_image(pj4.x - pi.x, k.grid.box[0], k.grid.half[0]);
-            double dy = min_image(pj4.y - pi.y, k.grid.box[1], k.grid.half[1]);
-            double dz = min_image(pj4.z - pi.z, k.grid.box[2], k.grid.half[2]);
-            double d2 = dx * dx + dy * dy + dz * dz;
-            valid = d2 < k.rc2;
-            x = (float)dx; y = (float)dy; z = (float)dz;
-            r = sqrtf((float)d2);
-            sj = (int)pj4.w;
+// Fill the warp's pair queue from list position `cur` on (lane = entry), four chunks at a time with
+// all index loads, then all position gathers, in flight together.  Pairs inside r_cut are queued as
+// {x, y, z, j | species << 28}.  Stops when the list ends or the next group might not fit; returns
+// the number of queued pairs and advances `cur`.
+__device__ __forceinline__ int collect_pairs(const KernelArgs &k, const double4 &pi, int64_t &cur, int64_t end, float4 *pq, int lane) {
+    int nq = 0;
+    while (cur < end && nq + (int)min((int64_t)128, end - cur) <= PB_CAP) {
+        int jj[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const int64_t e = cur + 32 * c + lane;
+            jj[c] = e < end ? __ldg(k.nbr + e) : -1;
         }
-        const unsigned m = __ballot_sync(0xffffffffu, valid);
-        if (valid) {
-            const int slot = nq + __popc(m & ((1u << lane) - 1u));
-            px[slot] = x; py[slot] = y; pz[slot] = z; pr[slot] = r; pj[slot] = j; ps[slot] = sj;
+        double4 pp[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) pp[c] = k.pos4[jj[c] < 0 ? 0 : jj[c]];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const double dx = min_image(pp[c].x - pi.x, k.grid.box[0], k.grid.half[0]);
+            const double dy = min_image(pp[c].y - pi.y, k.grid.box[1], k.grid.half[1]);
+            const double dz = min_image(pp[c].z - pi.z, k.grid.box[2], k.grid.half[2]);
+            const double d2 = dx * dx + dy * dy + dz * dz;
+            const bool valid = jj[c] >= 0 && d2 < k.rc2;
+            const unsigned m = __ballot_sync(0xffffffffu, valid);
+            if (valid)
+                pq[nq + __popc(m & ((1u << lane) - 1u))] =
+                    make_float4((float)dx, (float)dy, (float)dz, __int_as_float(jj[c] | ((int)pp[c].w << J_BITS)));
+            nq += __popc(m);
         }
-        nq += __popc(m);
-        __syncwarp();
-        if (nq >= 32) {
-            batch(32);
-            total += 32;
-            // move the tail of the queue to the front
-            float tx = 0.f, ty = 0.f, tz = 0.f, tr = 1.f; int tj = 0, ts = 0;
-            const bool mv = 32 + lane < nq;
-            if (mv) { tx = px[32 + lane]; ty = py[32 + lane]; tz = pz[32 + lane]; tr = pr[32 + lane]; tj = pj[32 + lane]; ts = ps[32 + lane]; }
-            __syncwarp();
-            if (mv) { px[lane] = tx; py[lane] = ty; pz[lane] = tz; pr[lane] = tr; pj[lane] = tj; ps[lane] = ts; }
-            nq -= 32;
-            __syncwarp();
-        }
+        cur += 128;
     }
-    if (nq > 0) { batch(nq); total += nq; }
-    return total;
+    __syncwarp();
+    return nq;
 }
 
 // ---------------- Encoding of one atom: returns the moment as accumulator fragments ----------------
+// `queued` returns the number of pairs left in the queue when the whole list fitted in one round
+// (the derivation then reuses them), or -1.
 __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView &tv, const double4 &pi, int64_t beg, int64_t end,
-                                           float *wbuf, int lane, float (&Pf)[4][4]) {
+                                           float4 *pq, float *stage, int lane, float (&Pf)[4][4], int &queued, PhaseClock &pc) {
     const int g = lane >> 2, t = lane & 3;
-    float *pb = wbuf, *stage = wbuf + 6 * PB_CAP;
     const int rs = tv.row_stride;
 #pragma unroll
     for (int a = 0; a < 4; ++a)
 #pragma unroll
         for (int b = 0; b < 4; ++b) Pf[a][b] = 0.f;
 
-    auto batch = [&](int n) {
+    auto batch = [&](int first, int n) {
         {   // lane = pair: harmonics (Eq. 3) and spline basis
             float h[D_ANG], b[4];
             int off = 0;
             if (lane < n) {
-                const float r = pb[3 * PB_CAP + lane], rinv = 1.0f / r;
-                harmonics(pb[lane] * rinv, pb[PB_CAP + lane] * rinv, pb[2 * PB_CAP + lane] * rinv, h);
+                const float4 e = pq[first + lane];
+                const float r = sqrtf(e.x * e.x + e.y * e.y + e.z * e.z), rinv = 1.0f / r;
+                harmonics(e.x * rinv, e.y * rinv, e.z * rinv, h);
                 const int iv = spline_basis<false>(r, k.tab, b, nullptr, k.status);
-                const int sj = reinterpret_cast<const int *>(pb)[5 * PB_CAP + lane];
+                const int sj = __float_as_int(e.w) >> J_BITS;
                 off = sj * tv.table_stride + iv * rs;
             } else {
 #pragma unroll
@@ -301,6 +310,7 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
             reinterpret_cast<int *>(stage)[lane * ST_STRIDE + 20] = off;
         }
         __syncwarp();
+        pc.mark(1);
         const int nks = (n + 7) >> 3;
         for (int ks = 0; ks < nks; ++ks) {
             // A = H^T (16 x 8 pairs): rows a = g, g + 8; columns pairs t, t + 4 of this k-step
@@ -327,38 +337,61 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
             gb[1] = bb.x * b0.y + bb.y * b1.y + bb.z * b2.y + bb.w * b3.y;
             gb[2] = bb.x * b0.z + bb.y * b1.z + bb.z * b2.z + bb.w * b3.z;
             gb[3] = bb.x * b0.w + bb.y * b1.w + bb.z * b2.w + bb.w * b3.w;
+            // Eq. 4 for eight pairs; the three terms of each n-tile are issued interleaved over the n-tiles
+            uint32_t bh[4][2], bl[4][2];
+            float c[4][4];
 #pragma unroll
             for (int nt = 0; nt < 4; ++nt) {
-                uint32_t bh0, bl0, bh1, bl1;
-                split_tf32(ga[nt], bh0, bl0);
-                split_tf32(gb[nt], bh1, bl1);
-                float c[4] = {0.f, 0.f, 0.f, 0.f};
-                mma3(c, ah, al, bh0, bh1, bl0, bl1);   // Eq. 4, eight pairs
-                Pf[nt][0] += c[0]; Pf[nt][1] += c[1]; Pf[nt][2] += c[2]; Pf[nt][3] += c[3];
+                split_tf32(ga[nt], bh[nt][0], bl[nt][0]);
+                split_tf32(gb[nt], bh[nt][1], bl[nt][1]);
+                c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
             }
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) mma_tf32(c[nt], al[0], al[1], al[2], al[3], bh[nt][0], bh[nt][1]);
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) mma_tf32(c[nt], ah[0], ah[1], ah[2], ah[3], bl[nt][0], bl[nt][1]);
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) mma_tf32(c[nt], ah[0], ah[1], ah[2], ah[3], bh[nt][0], bh[nt][1]);
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) { Pf[nt][0] += c[nt][0]; Pf[nt][1] += c[nt][1]; Pf[nt][2] += c[nt][2]; Pf[nt][3] += c[nt][3]; }
         }
         __syncwarp();
+        pc.mark(2);
     };
-    return scan_pairs(k, pi, beg, end, pb, lane, batch);
+    int total = 0, rounds = 0, n = 0;
+    int64_t cur = beg;
+    do {
+        n = collect_pairs(k, pi, cur, end, pq, lane);
+        pc.mark(0);
+        for (int q0 = 0; q0 < n; q0 += 32) batch(q0, min(32, n - q0));
+        total += n;
+        ++rounds;
+    } while (cur < end);
+    queued = rounds == 1 ? n : -1;
+    return total;
 }
 
 // ---------------- Derivation of one atom (Eq. 8-10) ----------------
 __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView &tv, const double4 &pi, int i, int64_t beg, int64_t end,
-                                            float *wbuf, int lane, const uint32_t (&Wh)[4][4], const uint32_t (&Wl)[4][4],
-                                            float (&vir)[9]) {
+                                            float4 *pq, float *scr, int queued, int lane, const uint32_t (&Wh)[4][4],
+                                            const uint32_t (&Wl)[4][4], float (&vir)[9], PhaseClock &pc) {
     const int g = lane >> 2, t = lane & 3;
-    float *pb = wbuf, *bs = wbuf + 6 * PB_CAP, *vt = bs + 32 * BS_STRIDE;
+    float *bs = scr, *vt = scr + 32 * BS_STRIDE;
     const int rs = tv.row_stride;
     float fx = 0.f, fy = 0.f, fz = 0.f;
 
-    auto batch = [&](int n) {
+    auto batch = [&](int first, int n) {
+        float4 ent = make_float4(1.f, 0.f, 0.f, 0.f);
+        float rinv = 1.f;
         {   // lane = pair: spline basis and its derivative
             float b[4] = {0.f, 0.f, 0.f, 0.f}, db[4] = {0.f, 0.f, 0.f, 0.f};
             int off = 0;
             if (lane < n) {
-                const int iv = spline_basis<true>(pb[3 * PB_CAP + lane], k.tab, b, db, k.status);
-                const int sj = reinterpret_cast<const int *>(pb)[5 * PB_CAP + lane];
-                off = sj * tv.table_stride + iv * rs;
+                ent = pq[first + lane];
+                const float r = sqrtf(ent.x * ent.x + ent.y * ent.y + ent.z * ent.z);
+                rinv = 1.0f / r;
+                const int iv = spline_basis<true>(r, k.tab, b, db, k.status);
+                off = (__float_as_int(ent.w) >> J_BITS) * tv.table_stride + iv * rs;
             }
             float4 *row = reinterpret_cast<float4 *>(bs + lane * BS_STRIDE);
             row[0] = make_float4(b[0], b[1], b[2], b[3]);
@@ -366,14 +399,17 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
             reinterpret_cast<int *>(bs)[lane * BS_STRIDE + 8] = off;
         }
         __syncwarp();
+        pc.mark(4);
         const int nmt = (n + 15) >> 4;
         for (int mt = 0; mt < nmt; ++mt) {
             // A = [G; G'] (16 pairs x 32 channels): rows pairs g, g + 8; this lane evaluates channels 8t .. 8t+7
-            float V[2][4], T[2][4], Vs[2][4], Ts[2][4];   // main (hi x hi) and small (cross) terms apart
+            // (one accumulator per output here: the truncating accumulation costs ~1e-6 relative on a
+            // 12-term chain, irrelevant for forces, and the registers are needed elsewhere)
+            float V[2][4], T[2][4];
 #pragma unroll
             for (int a = 0; a < 2; ++a)
 #pragma unroll
-                for (int b = 0; b < 4; ++b) { V[a][b] = 0.f; T[a][b] = 0.f; Vs[a][b] = 0.f; Ts[a][b] = 0.f; }
+                for (int b = 0; b < 4; ++b) { V[a][b] = 0.f; T[a][b] = 0.f; }
             float G[2][8], dG[2][8];
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
@@ -398,21 +434,32 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
                 split_tf32(G[0][4 + ks], ah[2], al[2]);  split_tf32(G[1][4 + ks], ah[3], al[3]);
                 split_tf32(dG[0][ks], dh[0], dl[0]);     split_tf32(dG[1][ks], dh[1], dl[1]);
                 split_tf32(dG[0][4 + ks], dh[2], dl[2]); split_tf32(dG[1][4 + ks], dh[3], dl[3]);
-                mma3s(V[0], Vs[0], ah, al, Wh[ks][0], Wh[ks][1], Wl[ks][0], Wl[ks][1]);   // Eq. 9: rows of V, a = 0..7
-                mma3s(V[1], Vs[1], ah, al, Wh[ks][2], Wh[ks][3], Wl[ks][2], Wl[ks][3]);   //                  a = 8..15
-                mma3s(T[0], Ts[0], dh, dl, Wh[ks][0], Wh[ks][1], Wl[ks][0], Wl[ks][1]);   // W g' (Eq. 8 re-associated)
-                mma3s(T[1], Ts[1], dh, dl, Wh[ks][2], Wh[ks][3], Wl[ks][2], Wl[ks][3]);
+                // Eq. 9 (rows of V: a = 0..7 and 8..15) and W g' (Eq. 8 re-associated); cross terms first, the
+                // four independent accumulators interleaved
+                mma_tf32(V[0], al[0], al[1], al[2], al[3], Wh[ks][0], Wh[ks][1]);
+                mma_tf32(V[1], al[0], al[1], al[2], al[3], Wh[ks][2], Wh[ks][3]);
+                mma_tf32(T[0], dl[0], dl[1], dl[2], dl[3], Wh[ks][0], Wh[ks][1]);
+                mma_tf32(T[1], dl[0], dl[1], dl[2], dl[3], Wh[ks][2], Wh[ks][3]);
+                mma_tf32(V[0], ah[0], ah[1], ah[2], ah[3], Wl[ks][0], Wl[ks][1]);
+                mma_tf32(V[1], ah[0], ah[1], ah[2], ah[3], Wl[ks][2], Wl[ks][3]);
+                mma_tf32(T[0], dh[0], dh[1], dh[2], dh[3], Wl[ks][0], Wl[ks][1]);
+                mma_tf32(T[1], dh[0], dh[1], dh[2], dh[3], Wl[ks][2], Wl[ks][3]);
+                mma_tf32(V[0], ah[0], ah[1], ah[2], ah[3], Wh[ks][0], Wh[ks][1]);
+                mma_tf32(V[1], ah[0], ah[1], ah[2], ah[3], Wh[ks][2], Wh[ks][3]);
+                mma_tf32(T[0], dh[0], dh[1], dh[2], dh[3], Wh[ks][0], Wh[ks][1]);
+                mma_tf32(T[1], dh[0], dh[1], dh[2], dh[3], Wh[ks][2], Wh[ks][3]);
             }
             float *va = vt + (16 * mt + g) * VT_STRIDE + 2 * t, *vb = va + 8 * VT_STRIDE;
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
-                *reinterpret_cast<float2 *>(va + 8 * q) = make_float2(V[q][0] + Vs[q][0], V[q][1] + Vs[q][1]);
-                *reinterpret_cast<float2 *>(vb + 8 * q) = make_float2(V[q][2] + Vs[q][2], V[q][3] + Vs[q][3]);
-                *reinterpret_cast<float2 *>(va + 16 + 8 * q) = make_float2(T[q][0] + Ts[q][0], T[q][1] + Ts[q][1]);
-                *reinterpret_cast<float2 *>(vb + 16 + 8 * q) = make_float2(T[q][2] + Ts[q][2], T[q][3] + Ts[q][3]);
+                *reinterpret_cast<float2 *>(va + 8 * q) = make_float2(V[q][0], V[q][1]);
+                *reinterpret_cast<float2 *>(vb + 8 * q) = make_float2(V[q][2], V[q][3]);
+                *reinterpret_cast<float2 *>(va + 16 + 8 * q) = make_float2(T[q][0], T[q][1]);
+                *reinterpret_cast<float2 *>(vb + 16 + 8 * q) = make_float2(T[q][2], T[q][3]);
             }
         }
         __syncwarp();
+        pc.mark(5);
         if (lane < n) {   // lane = pair: projection onto the pair vector (Eq. 10) and scatter
             float v[D_ANG], tt[D_ANG];
             const float4 *src = reinterpret_cast<const float4 *>(vt + lane * VT_STRIDE);
@@ -422,8 +469,8 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
                 v[4 * q] = a.x; v[4 * q + 1] = a.y; v[4 * q + 2] = a.z; v[4 * q + 3] = a.w;
                 tt[4 * q] = b.x; tt[4 * q + 1] = b.y; tt[4 * q + 2] = b.z; tt[4 * q + 3] = b.w;
             }
-            const float x = pb[lane], y = pb[PB_CAP + lane], z = pb[2 * PB_CAP + lane], rinv = 1.0f / pb[3 * PB_CAP + lane];
-            const int j = reinterpret_cast<const int *>(pb)[4 * PB_CAP + lane];
+            const float x = ent.x, y = ent.y, z = ent.z;
+            const int j = __float_as_int(ent.w) & ((1 << J_BITS) - 1);
             const float ux = x * rinv, uy = y * rinv, uz = z * rinv;
             float s, tx, ty, tz, tu;
             harmonics_project(ux, uy, uz, v, tt, s, tx, ty, tz, tu);
@@ -440,8 +487,18 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
             vir[6] -= z * qx; vir[7] -= z * qy; vir[8] -= z * qz;
         }
         __syncwarp();
+        pc.mark(6);
     };
-    scan_pairs(k, pi, beg, end, pb, lane, batch);
+    if (queued >= 0) {   // the encoding left every pair of this atom in the queue
+        for (int q0 = 0; q0 < queued; q0 += 32) batch(q0, min(32, queued - q0));
+    } else {
+        int64_t cur = beg;
+        do {
+            const int n = collect_pairs(k, pi, cur, end, pq, lane);
+            pc.mark(3);
+            for (int q0 = 0; q0 < n; q0 += 32) batch(q0, min(32, n - q0));
+        } while (cur < end);
+    }
 #pragma unroll
     for (int o = 16; o; o >>= 1) {
         fx += __shfl_xor_sync(0xffffffffu, fx, o);
@@ -455,29 +512,42 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
     }
 }
 
-// Head contraction on the tensor pipe: C^T[16 rows of W x 16 atoms] over k-steps [ks0, ks0 + nks).
-// A records come pre-split from global memory, B = activations (hi, lo interleaved) from shared
+// Head contraction on the tensor pipe: C^T[16 rows of W x 16 atoms] over NKS k-steps from ks0.
+// A records come pre-split from global memory (`head_load`, issued a pass ahead so that the L2
+// latency hides behind the previous epilogue), B = activations (hi, lo interleaved) from shared
 // memory with `bstride` floats per atom.  c[nt] covers atoms 8 nt .. 8 nt + 7.
-__device__ __forceinline__ void head_gemm(float (&c)[2][4], const float4 *__restrict__ rec, int ks0, int nks,
+template <int NKS>
+__device__ __forceinline__ void head_load(float4 (&wh)[4], float4 (&wl)[4], const float4 *__restrict__ rec, int ks0, int lane) {
+#pragma unroll
+    for (int q = 0; q < NKS; ++q) {
+        wh[q] = __ldg(rec + (size_t)(ks0 + q) * 64 + 2 * lane);
+        wl[q] = __ldg(rec + (size_t)(ks0 + q) * 64 + 2 * lane + 1);
+    }
+}
+template <int NKS>
+__device__ __forceinline__ void head_gemm(float (&c)[2][4], const float4 (&wh)[4], const float4 (&wl)[4], int ks0,
                                           const float *__restrict__ act, int bstride, int lane) {
     const int g = lane >> 2, t = lane & 3;
 #pragma unroll
     for (int a = 0; a < 2; ++a)
 #pragma unroll
         for (int b = 0; b < 4; ++b) c[a][b] = 0.f;
-#pragma unroll 2
-    for (int ks = ks0; ks < ks0 + nks; ++ks) {
-        const float4 ah4 = __ldg(rec + (size_t)ks * 64 + 2 * lane), al4 = __ldg(rec + (size_t)ks * 64 + 2 * lane + 1);
-        const uint32_t ah[4] = {__float_as_uint(ah4.x), __float_as_uint(ah4.y), __float_as_uint(ah4.z), __float_as_uint(ah4.w)};
-        const uint32_t al[4] = {__float_as_uint(al4.x), __float_as_uint(al4.y), __float_as_uint(al4.z), __float_as_uint(al4.w)};
 #pragma unroll
-        for (int nt = 0; nt < 2; ++nt) {
-            const float *row = act + (8 * nt + g) * bstride + 2 * (8 * ks + t);
-            const float2 b0 = *reinterpret_cast<const float2 *>(row), b1 = *reinterpret_cast<const float2 *>(row + 8);
-            float p[4] = {0.f, 0.f, 0.f, 0.f};
-            mma3(p, ah, al, __float_as_uint(b0.x), __float_as_uint(b1.x), __float_as_uint(b0.y), __float_as_uint(b1.y));
-            c[nt][0] += p[0]; c[nt][1] += p[1]; c[nt][2] += p[2]; c[nt][3] += p[3];
-        }
+    for (int q = 0; q < NKS; ++q) {
+        const uint32_t ah[4] = {__float_as_uint(wh[q].x), __float_as_uint(wh[q].y), __float_as_uint(wh[q].z), __float_as_uint(wh[q].w)};
+        const uint32_t al[4] = {__float_as_uint(wl[q].x), __float_as_uint(wl[q].y), __float_as_uint(wl[q].z), __float_as_uint(wl[q].w)};
+        const float *r0 = act + g * bstride + 2 * (8 * (ks0 + q) + t), *r1 = r0 + 8 * bstride;
+        const float2 x0 = *reinterpret_cast<const float2 *>(r0), x1 = *reinterpret_cast<const float2 *>(r0 + 8);
+        const float2 y0 = *reinterpret_cast<const float2 *>(r1), y1 = *reinterpret_cast<const float2 *>(r1 + 8);
+        float p[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        mma_tf32(p[0], al[0], al[1], al[2], al[3], __float_as_uint(x0.x), __float_as_uint(x1.x));
+        mma_tf32(p[1], al[0], al[1], al[2], al[3], __float_as_uint(y0.x), __float_as_uint(y1.x));
+        mma_tf32(p[0], ah[0], ah[1], ah[2], ah[3], __float_as_uint(x0.y), __float_as_uint(x1.y));
+        mma_tf32(p[1], ah[0], ah[1], ah[2], ah[3], __float_as_uint(y0.y), __float_as_uint(y1.y));
+        mma_tf32(p[0], ah[0], ah[1], ah[2], ah[3], __float_as_uint(x0.x), __float_as_uint(x1.x));
+        mma_tf32(p[1], ah[0], ah[1], ah[2], ah[3], __float_as_uint(y0.x), __float_as_uint(y1.x));
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) { c[nt][0] += p[nt][0]; c[nt][1] += p[nt][1]; c[nt][2] += p[nt][2]; c[nt][3] += p[nt][3]; }
     }
 }
 
@@ -493,61 +563,79 @@ __device__ __forceinline__ void store_partial(const float (&c)[2][4], float *par
 
 // ---------------- Regression (Eq. 6) forward and reverse for the tile ----------------
 // In: sX = invariants [atom][128].  Out: sX = dE/dG; per-atom energies written.
-__device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float *hb, int species, int count, int first,
-                                          int warp, int lane, double &e_sum) {
+// hc = biases [4][64], w_out [64], b_out of the species in shared memory.
+__device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float *hb, const float *hc, int species, int count, int first,
+                                          int warp, int lane, double &e_sum, PhaseClock &pc) {
     const float *hp = k.head_pack + (size_t)species * HP_TOTAL;
     const float4 *fwd = reinterpret_cast<const float4 *>(hp + HP_FWD), *bwd = reinterpret_cast<const float4 *>(hp + HP_BWD);
     float *xs = hb + HB_XS, *zs = hb + HB_ZS, *sD = hb + HB_SD, *dz = hb + HB_DZ, *dp = hb + HB_DP, *part = hb + HB_PART;
     const int mt4 = warp & 3, kq = warp >> 2;   // forward / reverse hidden layers: 4 m-tiles x 4 k-quarters
     const int atom = warp;                      // elementwise phases: warp = atom, lane = neuron (and neuron + 32)
+    float4 wh[4], wl[4];
 
+    head_load<KS0 / 4>(wh, wl, fwd + (size_t)(mt4 * KS0) * 64, kq * (KS0 / 4), lane);
     // split the invariants once
     for (int f = lane; f < N_INV; f += 32)
         *reinterpret_cast<float2 *>(xs + atom * 2 * X_STRIDE + 2 * f) = split_pair(sX[atom * X_STRIDE + f]);
+    pc.mark(3);
     __syncthreads();
+    pc.mark(14);
 
     float e_i = 0.f;
+#pragma unroll
     for (int L = 0; L < HEAD_L; ++L) {
         const float *zin = zs + ((L + 1) & 1) * TILE * 2 * Z_STRIDE;
         float *zout = zs + (L & 1) * TILE * 2 * Z_STRIDE;
         float c[2][4];
-        if (L == 0) head_gemm(c, fwd + (size_t)(mt4 * KS0) * 64, kq * (KS0 / 4), KS0 / 4, xs, 2 * X_STRIDE, lane);
-        else head_gemm(c, fwd + (size_t)(4 * KS0 + (L - 1) * 4 * KS1 + mt4 * KS1) * 64, kq * (KS1 / 4), KS1 / 4, zin, 2 * Z_STRIDE, lane);
+        if (L == 0) head_gemm<KS0 / 4>(c, wh, wl, kq * (KS0 / 4), xs, 2 * X_STRIDE, lane);
+        else head_gemm<KS1 / 4>(c, wh, wl, kq * (KS1 / 4), zin, 2 * Z_STRIDE, lane);
+        pc.mark(12);
         store_partial(c, part + kq * TILE * Z_STRIDE, Z_STRIDE, mt4, lane);
+        // weights of the next pass
+        if (L < HEAD_L - 1) head_load<KS1 / 4>(wh, wl, fwd + (size_t)(4 * KS0 + L * 4 * KS1 + mt4 * KS1) * 64, kq * (KS1 / 4), lane);
+        else head_load<2>(wh, wl, bwd + (size_t)((N_INV / 16) * 8 + (HEAD_L - 2) * 32 + mt4 * 8) * 64, kq * 2, lane);
+        pc.mark(13);
         __syncthreads();
+        pc.mark(14);
         // elementwise: bias, SiLU, residual; this thread owns neurons lane and lane + 32 of its atom
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
             const int nn = lane + 32 * q;
             const float *pp = part + atom * Z_STRIDE + nn;
-            const float pre = ((pp[0] + pp[TILE * Z_STRIDE]) + (pp[2 * TILE * Z_STRIDE] + pp[3 * TILE * Z_STRIDE])) + __ldg(hp + HP_BIAS + L * HEAD_H + nn);
+            const float pre = ((pp[0] + pp[TILE * Z_STRIDE]) + (pp[2 * TILE * Z_STRIDE] + pp[3 * TILE * Z_STRIDE])) + hc[L * HEAD_H + nn];
             float d, y = silu_f(pre, d);
             if (L > 0) { const float2 zi = *reinterpret_cast<const float2 *>(zin + atom * 2 * Z_STRIDE + 2 * nn); y += zi.x + zi.y; }
             sD[(L * TILE + atom) * Z_STRIDE + nn] = d;
             if (L < HEAD_L - 1) {
                 *reinterpret_cast<float2 *>(zout + atom * 2 * Z_STRIDE + 2 * nn) = split_pair(y);
             } else {   // output layer and the start of the reverse pass: dE/dz = w_out
-                const float wo = __ldg(hp + HP_WOUT + nn);
+                const float wo = hc[HEAD_L * HEAD_H + nn];
                 e_i += wo * y;
                 dz[atom * Z_STRIDE + nn] = wo;
                 *reinterpret_cast<float2 *>(dp + atom * 2 * Z_STRIDE + 2 * nn) = split_pair(wo * d);
             }
         }
+        pc.mark(15);
         __syncthreads();
+        pc.mark(14);
     }
 #pragma unroll
     for (int o = 16; o; o >>= 1) e_i += __shfl_xor_sync(0xffffffffu, e_i, o);
-    e_i += __ldg(hp + HP_WOUT + HEAD_H);
+    e_i += hc[HEAD_L * HEAD_H + HEAD_H];
     if (lane == 0 && atom < count) {
         k.e_atom[__ldg(k.center_order + first + atom)] = e_i;
         e_sum += (double)e_i;
     }
 
     // reverse through the hidden layers 3, 2, 1 (each with its skip path)
+    const int mt8 = warp & 7, kh = warp >> 3;   // first layer: 8 m-tiles x 2 k-halves
+#pragma unroll
     for (int L = HEAD_L - 1; L >= 1; --L) {
         float c[2][4];
-        head_gemm(c, bwd + (size_t)((N_INV / 16) * 8 + (L - 1) * 32 + mt4 * 8) * 64, kq * 2, 2, dp, 2 * Z_STRIDE, lane);
+        head_gemm<2>(c, wh, wl, kq * 2, dp, 2 * Z_STRIDE, lane);
         store_partial(c, part + kq * TILE * Z_STRIDE, Z_STRIDE, mt4, lane);
+        if (L > 1) head_load<2>(wh, wl, bwd + (size_t)((N_INV / 16) * 8 + (L - 2) * 32 + mt4 * 8) * 64, kq * 2, lane);
+        else head_load<4>(wh, wl, bwd + (size_t)(mt8 * 8) * 64, kh * 4, lane);
         __syncthreads();
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
@@ -559,10 +647,9 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
         }
         __syncthreads();
     }
-    {   // first layer: dE/dG [128 x 16]: 8 m-tiles x 2 k-halves
-        const int mt8 = warp & 7, kh = warp >> 3;
+    {   // first layer: dE/dG [128 x 16]
         float c[2][4];
-        head_gemm(c, bwd + (size_t)(mt8 * 8) * 64, kh * 4, 4, dp, 2 * Z_STRIDE, lane);
+        head_gemm<4>(c, wh, wl, kh * 4, dp, 2 * Z_STRIDE, lane);
         store_partial(c, part + kh * TILE * X_STRIDE, X_STRIDE, mt8, lane);
         __syncthreads();
         for (int f = lane; f < N_INV; f += 32)
@@ -578,9 +665,11 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
     const int g = lane >> 2, t = lane & 3;
     float *s_tab = smem;                         // [C][rows][TAB_STRIDE_SMEM] when TAB_SMEM
     float *sX = smem + (TAB_SMEM ? tab_words : 0);
-    float *hb = sX + SX_WORDS;                   // head buffers = all per-warp buffers
-    float *wbuf = hb + warp * WARP_WORDS;
-    int *ctl = reinterpret_cast<int *>(hb + NW * WARP_WORDS);
+    float *hb = sX + SX_WORDS;                   // head buffers = the scratch of all warps
+    float *scr = hb + warp * SCR_WORDS;
+    float4 *pq = reinterpret_cast<float4 *>(hb + NW * SCR_WORDS + warp * Q_WORDS);
+    float *hc = hb + NW * (SCR_WORDS + Q_WORDS);
+    int *ctl = reinterpret_cast<int *>(hc + HC_WORDS);
     const int rows = k.tab.knots + 3;
 
     // species-pure tiles: tiles of species s start at tile_first[s]
@@ -598,11 +687,14 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
     unsigned long long n_pairs = 0;
     int loaded_species = -1;
     TableView tv;
+    PhaseClock pc;
+    pc.start();
 
     while (true) {
         __syncthreads();
         if (threadIdx.x == 0) ctl[0] = atomicAdd(k.tile_counter, 1);
         __syncthreads();
+        pc.mark(11);
         const int tile = ctl[0];
         if (tile >= n_tiles) break;
         int species = 0;
@@ -623,6 +715,8 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
                 tv.base = k.tab.coef + (size_t)species * k.n_species * rows * K_RADIAL;
                 tv.row_stride = K_RADIAL; tv.table_stride = rows * K_RADIAL;
             }
+            for (int idx = threadIdx.x; idx < HEAD_L * HEAD_H + HEAD_H + 1; idx += NW * 32)
+                hc[idx] = __ldg(k.head_pack + (size_t)species * HP_TOTAL + HP_BIAS + idx);
             loaded_species = species;
             __syncthreads();
         }
@@ -633,11 +727,12 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
         double4 pi = make_double4(0.0, 0.0, 0.0, 0.0);
         int64_t beg = 0, end = 0;
         float Pf[4][4];
+        int queued = -1;
         float *xrow = sX + warp * X_STRIDE;
         if (have) {
             pi = k.pos4[i];
             beg = k.nbr_off[i]; end = k.nbr_off[i + 1];
-            n_pairs += encode_atom(k, tv, pi, beg, end, wbuf, lane, Pf);
+            n_pairs += encode_atom(k, tv, pi, beg, end, pq, scr, lane, Pf, queued, pc);
             // Eq. 5 (C_l = I): this lane holds rows a = g, g + 8 of channels 8t + j; sum squares over the rows of a block
             float part[4][8];
 #pragma unroll
@@ -664,10 +759,13 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
         } else {   // empty slot of a ragged tile: feed zeros to the head
             for (int c = lane; c < N_INV; c += 32) xrow[c] = 0.f;
         }
+        pc.mark(7);
         __syncthreads();
+        pc.mark(8);
 
         // ---------------- Regression ----------------
-        head_tile(k, sX, hb, species, count, first, warp, lane, e_sum);
+        head_tile(k, sX, hb, hc, species, count, first, warp, lane, e_sum, pc);
+        pc.mark(9);
 
         // ---------------- Derivation ----------------
         if (have) {
@@ -692,9 +790,11 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
                 split_tf32(w2, Wh[ks][2], Wl[ks][2]);
                 split_tf32(w3, Wh[ks][3], Wl[ks][3]);
             }
-            derive_atom(k, tv, pi, i, beg, end, wbuf, lane, Wh, Wl, vir);
+            derive_atom(k, tv, pi, i, beg, end, pq, scr, queued, lane, Wh, Wl, vir, pc);
         }
+        pc.mark(10);
     }
+    pc.flush(k.acc, lane);
 
     // per-warp totals -> global accumulators
 #pragma unroll
