@@ -112,6 +112,21 @@ class ClockSampler:
                 "power_w_max": float(max(power)), "samples": len(sm)}
 
 
+def max_over_ranks(x: float, device) -> float:
+    """Slowest rank's time: the number every rank reports against (no-op for a single process)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(atoms_per_rank: int, steps: int, seconds_max: float, world: int) -> float:
+    """Replicas: every rank advances its own atoms; aggregate = all ranks' atom-steps over the slowest rank's time."""
+    return world * atoms_per_rank * steps / seconds_max
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -217,11 +232,8 @@ def main():
     counters = mlip.mlip_get_counters(pot.ctx)
     k_launches, k_ms = mlip.mlip_kernel_time(pot.ctx, reset=True)
     e_final = pot.energies().cpu().numpy()
-    t = torch.tensor([ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_max = float(t.item())
-    value = world * n * args.steps / (ms_max * 1e-3)
+    ms_max = max_over_ranks(ms, dev)
+    value = whole_job_value(n, args.steps, ms_max * 1e-3, world)
 
     # ---- end to end: host buffers through mlip_compute_host, copies inside the timed region ----
     e2e = None
@@ -247,12 +259,9 @@ def main():
             mlip.mlip_compute_host(pot.ctx, p, species_h if rebuild else None, w.box if rebuild else None, rebuild,
                                    forces_h, virial_h)
         torch.cuda.synchronize()
-        dt = time.perf_counter() - t0
-        t = torch.tensor([dt], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dt = max_over_ranks(time.perf_counter() - t0, dev)
         n_rebuilds = (e2e_steps + REBUILD_EVERY - 1) // REBUILD_EVERY
-        e2e = {"value": world * n * e2e_steps / float(t.item()), "unit": UNIT,
+        e2e = {"value": whole_job_value(n, e2e_steps, dt, world), "unit": UNIT,
                "h2d_bytes_per_step": int(24 * n + 4 * n * n_rebuilds / e2e_steps),
                "d2h_bytes_per_step": int(12 * n + 80),
                "call": "mlip_compute_host (positions in, forces + energy + virial out, list rebuild every 10th call)"}
