@@ -111,6 +111,26 @@ int mlip_build_neighbors(mlip_ctx *ctx, int64_t n_atoms, const double *pos, cons
 int mlip_get_neighbors(mlip_ctx *ctx, int64_t *seg_ptr, int32_t *nbr, int64_t capacity,
                        int64_t *n_entries_host, void *stream);
 
+/*
+ * mlip_get_neighbors without any allocation (the paper has no counterpart: this is a
+ * deployment variant, not a step of its method).  Same arguments, same output, same status codes.
+ * mlip_get_neighbors takes two temporary device blocks with cudaMalloc on every call; some callers
+ * cannot afford that: an MD driver that has handed all device memory to its own pools, a plug-in
+ * that must not disturb its host's allocator, code running where an allocation would stall every
+ * stream.  This variant keeps those temporaries in a static device array of about 4 MiB that every
+ * GPU loading the library holds until the process exits, and calls no cudaMalloc, cudaFree or
+ * allocating library routine.
+ *   Limit: n_atoms * n_species <= 1,048,576; larger systems get MLIP_ERR_UNSUPPORTED.
+ *   The first call on a device looks up the array's device address (once per device, with that
+ *   device current); make that first call before starting any stream capture.
+ *   All calls share the array and it keeps the previous call's contents (every word that is read
+ *   is rewritten first, so nothing needs clearing); calls whose kernels overlap on one GPU race on
+ *   it - issue them one after another.
+ * Synchronises, like mlip_get_neighbors.
+ */
+int mlip_get_neighbors_noalloc(mlip_ctx *ctx, int64_t *seg_ptr, int32_t *nbr, int64_t capacity,
+                               int64_t *n_entries_host, void *stream);
+
 /* Replace positions (dev [N][3], caller's order) keeping the current lists. */
 int mlip_set_positions(mlip_ctx *ctx, const double *pos, void *stream);
 /* Set velocities (dev [N][3], Angstrom/fs, caller's order). */

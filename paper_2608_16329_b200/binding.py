@@ -22,7 +22,7 @@ ERRORS = {0: "MLIP_OK", 1: "MLIP_ERR_INVALID_ARG", 2: "MLIP_ERR_UNSUPPORTED", 3:
           11: "MLIP_ERR_TABLE_RANGE"}
 CODES = {v: k for k, v in ERRORS.items()}
 
-EXPORTS = ["mlip_create", "mlip_table_error", "mlip_build_neighbors", "mlip_get_neighbors", "mlip_set_positions",
+EXPORTS = ["mlip_create", "mlip_table_error", "mlip_build_neighbors", "mlip_get_neighbors", "mlip_get_neighbors_noalloc", "mlip_set_positions",
            "mlip_set_velocities", "mlip_compute", "mlip_compute_host", "mlip_step", "mlip_get_state",
            "mlip_get_energies", "mlip_sync_status", "mlip_get_counters", "mlip_kernel_time",
            "mlip_resident_bytes", "mlip_last_error", "mlip_destroy"]
@@ -117,6 +117,17 @@ def mlip_get_neighbors(ctx, seg_ptr, nbr, stream=None):
     n = ctypes.c_int64(0)
     cap = 0 if nbr is None else nbr.numel()
     rc = lib().mlip_get_neighbors(ctx, _dev(seg_ptr), _dev(nbr), ctypes.c_int64(cap), ctypes.byref(n), _stream(stream))
+    _check(ctx, rc, allow=(CODES["MLIP_ERR_NEIGHBOR_OVERFLOW"],))
+    return rc, n.value
+
+
+def mlip_get_neighbors_noalloc(ctx, seg_ptr, nbr, stream=None):
+    """mlip_get_neighbors for callers that must not allocate device memory: the export's temporaries
+    sit in a static device array inside the library (n_atoms * n_species <= 1,048,576).  Returns
+    (status, number of entries); an unsupported size raises MlipError."""
+    n = ctypes.c_int64(0)
+    cap = 0 if nbr is None else nbr.numel()
+    rc = lib().mlip_get_neighbors_noalloc(ctx, _dev(seg_ptr), _dev(nbr), ctypes.c_int64(cap), ctypes.byref(n), _stream(stream))
     _check(ctx, rc, allow=(CODES["MLIP_ERR_NEIGHBOR_OVERFLOW"],))
     return rc, n.value
 

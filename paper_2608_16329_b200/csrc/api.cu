@@ -217,6 +217,14 @@ int mlip_get_neighbors(mlip_ctx *c, int64_t *seg_ptr, int32_t *nbr, int64_t capa
     return launch_export(c, seg_ptr, nbr, capacity, n_entries_host, (cudaStream_t)stream);
 }
 
+int mlip_get_neighbors_noalloc(mlip_ctx *c, int64_t *seg_ptr, int32_t *nbr, int64_t capacity, int64_t *n_entries_host, void *stream) {
+    if (!c || !seg_ptr) return MLIP_ERR_INVALID_ARG;
+    if (!c->built) return fail(c, MLIP_ERR_NOT_BUILT, "no neighbor lists yet");
+    c->last_stream = (cudaStream_t)stream;
+    cudaSetDevice(c->cfg.device);
+    return launch_export_noalloc(c, seg_ptr, nbr, capacity, n_entries_host, (cudaStream_t)stream);
+}
+
 int mlip_set_positions(mlip_ctx *c, const double *pos, void *stream) {
     if (!c || !pos) return MLIP_ERR_INVALID_ARG;
     if (!c->built) return fail(c, MLIP_ERR_NOT_BUILT, "no neighbor lists yet");

@@ -132,6 +132,7 @@ namespace mlip {
 int launch_pack_source(mlip_ctx *c, const double *pos, const int32_t *species, cudaStream_t s);
 int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s);
 int launch_export(mlip_ctx *c, int64_t *seg_ptr, int32_t *nbr, int64_t capacity, int64_t *n_entries_host, cudaStream_t s);
+int launch_export_noalloc(mlip_ctx *c, int64_t *seg_ptr, int32_t *nbr, int64_t capacity, int64_t *n_entries_host, cudaStream_t s);
 // tables.cu
 int build_tables(mlip_ctx *c, const double *enc_w_host, size_t n_enc);
 // megakernel.cu

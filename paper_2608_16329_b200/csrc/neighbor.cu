@@ -279,3 +279,72 @@ int launch_export(mlip_ctx *c, int64_t *seg_ptr, int32_t *nbr, int64_t capacity,
 }
 
 }  // namespace mlip
+
+// ---- allocation-free variant of the canonical export ----
+//
+// For callers that must not allocate device memory while they run: code inside a region where
+// cudaMalloc would serialise or fail (a latency-critical MD loop that owns a fixed memory budget, a
+// plug-in running under a host application whose allocator it may not touch), or a process whose
+// device memory is already fully committed.  The two temporaries of the export (per-(atom, species)
+// counts and the partial sums of the prefix scan) live in a file-scope device array instead of
+// fresh cudaMalloc blocks.  Every GPU that loads the library holds the array until the process exits.
+namespace mlip {
+
+constexpr int64_t NOALLOC_MAX_SEGMENTS = 1 << 20;   // n_atoms * n_species accepted by the entry point
+constexpr size_t NOALLOC_COUNT_BYTES = ((sizeof(int32_t) * (NOALLOC_MAX_SEGMENTS + 1) + 255) / 256) * 256;
+constexpr size_t NOALLOC_SCAN_ITEMS = NOALLOC_MAX_SEGMENTS / SCAN_TILE + 3;
+constexpr size_t NOALLOC_BYTES = NOALLOC_COUNT_BYTES + sizeof(int64_t) * NOALLOC_SCAN_ITEMS;   // about 4 MiB
+
+static __device__ __align__(256) unsigned char g_export_scratch[NOALLOC_BYTES];
+
+// In host code `g_export_scratch` is only a handle for the runtime, not a device address; the
+// address a kernel may use comes from cudaGetSymbolAddress, asked once per device with that device
+// current.  Slot d caches device d's answer.
+static void *g_export_scratch_addr[64] = {nullptr};
+
+static int export_scratch_for_current_device(mlip_ctx *c, void **out) {
+    int dev = -1;
+    MLIP_CUDA_TRY(c, cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) { c->err = "device ordinal out of range for the static scratch table"; return MLIP_ERR_UNSUPPORTED; }
+    if (!g_export_scratch_addr[dev]) {
+        void *p = nullptr;
+        MLIP_CUDA_TRY(c, cudaGetSymbolAddress(&p, g_export_scratch));
+        g_export_scratch_addr[dev] = p;
+    }
+    *out = g_export_scratch_addr[dev];
+    return MLIP_OK;
+}
+
+// Same kernels and the same order as launch_export, with the temporaries taken from the static
+// array.  Every scratch word that is read (counts of all n * C segments, the scan's tile sums) is
+// written earlier in the same call, so nothing has to be cleared between calls; two calls whose
+// kernels overlap on the GPU (different streams or contexts on one device) would race on it.
+int launch_export_noalloc(mlip_ctx *c, int64_t *seg_ptr, int32_t *nbr, int64_t capacity, int64_t *n_entries_host, cudaStream_t s) {
+    const int64_t n = c->n;
+    const int C = c->cfg.n_species;
+    if (n * C > NOALLOC_MAX_SEGMENTS) {
+        c->err = "mlip_get_neighbors_noalloc: n_atoms * n_species exceeds 1048576 (the static scratch size); use mlip_get_neighbors";
+        return MLIP_ERR_UNSUPPORTED;
+    }
+    void *base = nullptr;
+    int rc = export_scratch_for_current_device(c, &base);
+    if (rc != MLIP_OK) return rc;
+    int32_t *seg_count = reinterpret_cast<int32_t *>(base);
+    int64_t *tmp = reinterpret_cast<int64_t *>(static_cast<unsigned char *>(base) + NOALLOC_COUNT_BYTES);
+    k_export_count<<<blocks_for(n * 32, 256), 256, 0, s>>>(n, C, c->nbr_off, c->nbr, c->pos4, c->user_of, seg_count);
+    exclusive_scan<int32_t, int64_t>(seg_count, seg_ptr, n * C, tmp, s);
+    MLIP_CUDA_TRY(c, cudaMemcpyAsync(c->total_host, seg_ptr + n * C, sizeof(int64_t), cudaMemcpyDeviceToHost, s));
+    MLIP_CUDA_TRY(c, cudaStreamSynchronize(s));
+    c->launches += 4;
+    if (n_entries_host) *n_entries_host = *c->total_host;
+    if (*c->total_host > capacity || !nbr) {
+        c->err = "neighbor export: capacity too small";
+        return MLIP_ERR_NEIGHBOR_OVERFLOW;
+    }
+    k_export_fill<<<blocks_for(n * 32, 256), 256, 0, s>>>(n, C, c->nbr_off, c->nbr, c->pos4, c->user_of, seg_ptr, nbr);
+    c->launches += 1;
+    MLIP_CUDA_TRY(c, cudaStreamSynchronize(s));
+    return MLIP_OK;
+}
+
+}  // namespace mlip
