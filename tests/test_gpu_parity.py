@@ -159,3 +159,49 @@ def test_table_tolerance_is_enforced():
     pot = mlip.Potential(6, 6.0, 1.0, enc, head, np.ones(6))
     ev, ed = mlip.mlip_table_error(pot.ctx)
     assert ev < 1e-6
+
+
+def test_full_size_benchmark_workload_sampled_against_oracle():
+    """8,001,504 atoms (the benchmark's launch configuration): sampled E_i and forces, global invariants."""
+    w, model, pot = make_pair(5, 126, 1.0)
+    pot.build_neighbors(w.pos, w.species, w.box)
+    out = pot.compute(want_e_atom=True)
+    pot.sync_status()
+    atoms = np.array([0, 1, 4_000_751, 8_001_503, 123_456, 6_543_210, 2_718_281, 3_141_592])
+    ref = oracle.sampled(model, w.pos, w.species, w.box, atoms)
+    f = out["forces"][atoms].cpu().numpy().astype(np.float64)
+    ea = out["e_atom"][atoms].cpu().numpy().astype(np.float64)
+    assert np.abs(f - ref["forces"]).max() <= F_ATOL
+    assert np.abs(ea - ref["e_atom"]).max() <= 2e-5 * max(1.0, np.abs(ref["e_atom"]).max())
+    # properties that hold at any size: energy is the sum of the per-atom energies, no net force
+    e = float(out["energy"].cpu())
+    e_sum = float(out["e_atom"].double().sum().cpu())
+    assert abs(e - e_sum) <= 1e-6 * abs(e)
+    net = out["forces"].double().sum(0).cpu().numpy()
+    assert np.abs(net).max() < 1e-3 * np.sqrt(w.n_atoms)
+    import paper_2608_16329_b200 as mlip
+    c = mlip.mlip_get_counters(pot.ctx)
+    assert 77.5 < c["pairs_in_cutoff"] / w.n_atoms < 78.5 and 133.0 < c["list_entries"] / w.n_atoms < 135.0
+
+
+# (workload 4 is far from equilibrium under random weights: its kinetic energy grows ~50 % in 8 steps and the light
+# species soon outruns skin/2 in a few steps, so it gets a short run with a rebuild every 3 steps)
+@pytest.mark.parametrize("cfg,n_cells,steps,every", [(3, 16, 30, 10), (4, 24, 12, 3)])
+def test_nve_with_rebuilds_conserves_energy_on_multicomponent_workloads(cfg, n_cells, steps, every):
+    w, model, pot = make_pair(cfg, n_cells, 1.0)
+    pot.build_neighbors(w.pos, w.species, w.box)
+    pot.set_velocities(w.vel)
+    pot.compute()
+    e0 = pot.energies().cpu().numpy()
+    pot.step(steps, 1.0, every)
+    assert pot.sync_status(raise_on_error=False) == 0
+    e1 = pot.energies().cpu().numpy()
+    exchanged = abs(e1[1] - e0[1])
+    assert exchanged > 0.05 * e0[1]                       # the system is really moving
+    assert abs(e1.sum() - e0.sum()) < 0.02 * exchanged + 2e-6 * abs(e0[0])
+    # the lists after in-step rebuilds are the lists of the current positions
+    pos, vel, step = pot.state()
+    seg, nbr = pot.neighbors()
+    p = pos.cpu().numpy()
+    nl = oracle.neighbors(p, w.species, w.n_species, w.box, w.r_cut + w.skin)
+    assert step == steps and canonical_equal(nl, seg, nbr)
