@@ -147,7 +147,7 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
         if ((rc = dev_alloc(c, &c->acc, (size_t)ACC_COUNT)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->pair_counter, 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->status, 1)) != MLIP_OK) break;
-        if ((rc = dev_alloc(c, &c->tile_counter, 1)) != MLIP_OK) break;
+        if ((rc = dev_alloc(c, &c->tile_counter, (size_t)MAX_SPECIES)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->species_start, (size_t)MAX_SPECIES + 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->stage_out, 10)) != MLIP_OK) break;
         if (cudaMallocHost((void **)&c->status_host, sizeof(int)) != cudaSuccess ||

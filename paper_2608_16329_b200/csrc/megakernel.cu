@@ -3,10 +3,12 @@
 // angular features are recomputed in the derivation stage instead of being kept).
 //
 // Work decomposition
-//   One persistent CTA of 16 warps per SM takes tiles of 16 central atoms of ONE species from a
-//   global counter; a warp owns one atom of the tile.  The radial tables of that central species
-//   (one per neighbor species) are staged in shared memory and stay there until the species of
-//   the CTA's tiles changes (tiles are handed out in species order).
+//   One persistent CTA of 16 warps per SM, organised as two independent groups of 8 warps.  The CTA
+//   walks through the central species in order; for each it stages that species' radial tables
+//   (one per neighbor species) and head constants in shared memory, then each group takes tiles of
+//   8 central atoms of that species from a global counter (warp = atom) and runs them on its own,
+//   synchronising only inside the group (named barriers), so that one group's latency-bound head
+//   overlaps the other group's pair loops.
 //   Encoding    The warp scans the atom's list (lane = entry), queues the pairs inside r_cut in
 //               shared memory, and every 32 queued pairs evaluates harmonics (Eq. 3) and the
 //               spline basis with lane = pair.  The moment P_i = H^T G (Eq. 4, 16 x n times
@@ -15,9 +17,9 @@
 //               radial values g being evaluated straight into the B fragments.  P_i stays in
 //               the accumulator registers until the derivation.
 //   Invariants  Eq. 5 from the accumulator fragments by three xor-shuffles.
-//   Regression  Eq. 6 forward and reverse for the 16 atoms at once as W X^T on the tensor pipe
-//               (weights pre-split and pre-packed in A-fragment order, 4-way split over the
-//               reduction dimension, elementwise epilogue over all threads).
+//   Regression  Eq. 6 forward and reverse for the 8 atoms of the tile at once as W X^T on the tensor
+//               pipe (weights pre-packed in A-fragment order, 2-way split over the reduction
+//               dimension across the group's warps, elementwise epilogue over the group's threads).
 //   Derivation  W_i (Eq. 7) is the accumulator fragment of P_i scaled in place: by construction
 //               of the channel permutation it already is the B fragment of the next contraction.
 //               [V; T] = [G; G'] W^T (Eq. 9 and the re-associated Eq. 8 term, U_i never formed)
@@ -31,8 +33,9 @@
 
 namespace mlip {
 
-constexpr int TILE = 16;      // atoms per tile = warps per CTA
-constexpr int NW = 16;
+constexpr int TILE = 8;       // atoms per tile = warps per group
+constexpr int NG = 2;         // groups per CTA
+constexpr int NW = NG * TILE; // warps per CTA
 constexpr int PB_CAP = 160;   // queued pairs per warp: up to 31 left over + four list chunks of 32
 constexpr int J_BITS = 28;    // queue entries pack the neighbor index (low 28 bits) with its species
 constexpr int ST_STRIDE = 24; // encoding hand-over: 16 h, 4 b, table offset (bank-conflict-free for the fragment reads)
@@ -40,28 +43,30 @@ constexpr int BS_STRIDE = 12; // derivation hand-over: 4 b, 4 b', table offset
 constexpr int VT_STRIDE = 40; // 16 v + 16 t per pair
 constexpr int X_STRIDE = 132; // invariants / dE/dG per atom
 constexpr int Z_STRIDE = 68;  // head activations per atom
-constexpr int TAB_STRIDE_SMEM = 36;   // padded table row in shared memory
+#ifndef MLIP_TAB_STRIDE
+#define MLIP_TAB_STRIDE 36
+#endif
+constexpr int TAB_STRIDE_SMEM = MLIP_TAB_STRIDE;   // padded table row in shared memory
 
 constexpr int Q_WORDS = 4 * PB_CAP;                             // pair queue of a warp: kept from encoding to derivation
 constexpr int SCR_WORDS = 32 * BS_STRIDE + 32 * VT_STRIDE;      // scratch of a warp: 384 + 1280
 static_assert(32 * ST_STRIDE <= SCR_WORDS, "encoding stage must fit the derivation buffers");
-constexpr int SX_WORDS = TILE * X_STRIDE;
-// head buffers (alias of the per-warp buffers)
-constexpr int HB_XS = 0;                                   // split invariants  [16][2 * X_STRIDE]
-constexpr int HB_ZS = HB_XS + TILE * 2 * X_STRIDE;         // split activations [2][16][2 * Z_STRIDE]
-constexpr int HB_SD = HB_ZS + 2 * TILE * 2 * Z_STRIDE;     // SiLU'             [4][16][Z_STRIDE]
-constexpr int HB_DZ = HB_SD + HEAD_L * TILE * Z_STRIDE;    // dE/dz             [16][Z_STRIDE]
-constexpr int HB_DP = HB_DZ + TILE * Z_STRIDE;             // split dE/dpre     [16][2 * Z_STRIDE]
-constexpr int HB_PART = HB_DP + TILE * 2 * Z_STRIDE;       // split-K partials  [4][16][Z_STRIDE] or [2][16][X_STRIDE]
-constexpr int HB_WORDS = HB_PART + 4 * TILE * Z_STRIDE;
-static_assert(2 * TILE * X_STRIDE <= 4 * TILE * Z_STRIDE, "partials of the last reverse layer");
-static_assert(HB_WORDS <= NW * SCR_WORDS, "head buffers alias the per-warp scratch");
+constexpr int SX_WORDS = TILE * X_STRIDE;                       // per group
+// head buffers of a group (alias of the scratch of the group's warps)
+constexpr int HB_XS = 0;                                   // split invariants  [8][2 * X_STRIDE]
+constexpr int HB_ZS = HB_XS + TILE * 2 * X_STRIDE;         // split activations [2][8][2 * Z_STRIDE]
+constexpr int HB_SD = HB_ZS + 2 * TILE * 2 * Z_STRIDE;     // SiLU'             [4][8][Z_STRIDE]
+constexpr int HB_DZ = HB_SD + HEAD_L * TILE * Z_STRIDE;    // dE/dz             [8][Z_STRIDE]
+constexpr int HB_DP = HB_DZ + TILE * Z_STRIDE;             // split dE/dpre     [8][2 * Z_STRIDE]
+constexpr int HB_PART = HB_DP + TILE * 2 * Z_STRIDE;       // split-K partials  [2][8][Z_STRIDE]
+constexpr int HB_WORDS = HB_PART + 2 * TILE * Z_STRIDE;
+static_assert(HB_WORDS <= TILE * SCR_WORDS, "head buffers alias the scratch of the group's warps");
 constexpr int HC_WORDS = HEAD_L * HEAD_H + HEAD_H + 16;         // biases, w_out, b_out of the current species
-constexpr int FIXED_WORDS = SX_WORDS + NW * (Q_WORDS + SCR_WORDS) + HC_WORDS + 16;
+constexpr int FIXED_WORDS = NG * SX_WORDS + NW * (Q_WORDS + SCR_WORDS) + HC_WORDS + 16;
 constexpr int SMEM_LIMIT_WORDS = 227 * 1024 / 4 - 256;
 
 // Pre-packed head weights per species (floats).  A record holds the A operand of one
-// (m-tile, k-step): per lane {a0..a3 hi, a0..a3 lo}, i.e. 256 floats.
+// (m-tile, k-step): per lane {a0, a1, a2, a3}, i.e. 128 floats (split into hi + lo in registers).
 //   forward  layer L: A[m][k] = W_L[m][k]   (m = neuron)    4 m-tiles, K_L / 8 k-steps
 //   reverse  layer L: A[m][k] = W_L[k][m]   (m = input)     K_L / 16 m-tiles, 8 k-steps
 // followed by biases [4][64], w_out[64], b_out, pad.
@@ -69,8 +74,8 @@ constexpr int KS0 = N_INV / 8, KS1 = HEAD_H / 8;
 constexpr int FWD_RECORDS = 4 * KS0 + (HEAD_L - 1) * 4 * KS1;
 constexpr int BWD_RECORDS = (N_INV / 16) * 8 + (HEAD_L - 1) * 4 * 8;
 constexpr int HP_FWD = 0;
-constexpr int HP_BWD = HP_FWD + FWD_RECORDS * 256;
-constexpr int HP_BIAS = HP_BWD + BWD_RECORDS * 256;
+constexpr int HP_BWD = HP_FWD + FWD_RECORDS * 128;
+constexpr int HP_BIAS = HP_BWD + BWD_RECORDS * 128;
 constexpr int HP_WOUT = HP_BIAS + HEAD_L * HEAD_H;
 constexpr int HP_TOTAL = HP_WOUT + HEAD_H + 4;
 
@@ -512,73 +517,64 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
     }
 }
 
-// Head contraction on the tensor pipe: C^T[16 rows of W x 16 atoms] over NKS k-steps from ks0.
-// A records come pre-split from global memory (`head_load`, issued a pass ahead so that the L2
-// latency hides behind the previous epilogue), B = activations (hi, lo interleaved) from shared
-// memory with `bstride` floats per atom.  c[nt] covers atoms 8 nt .. 8 nt + 7.
+// Barrier among the 256 threads of one group (hardware barrier 1 + group).
+__device__ __forceinline__ void group_sync(int group) {
+    asm volatile("bar.sync %0, %1;" ::"r"(group + 1), "r"(TILE * 32) : "memory");
+}
+
+// Head contraction on the tensor pipe: C^T[16 rows of W x 8 atoms] over NKS k-steps from ks0.
+// A records come from global memory (`head_load`, issued a pass ahead so that the L2 latency hides
+// behind the previous epilogue) and are split into hi + lo here; B = activations (hi, lo
+// interleaved) from shared memory with `bstride` floats per atom.
 template <int NKS>
-__device__ __forceinline__ void head_load(float4 (&wh)[4], float4 (&wl)[4], const float4 *__restrict__ rec, int ks0, int lane) {
+__device__ __forceinline__ void head_load(float4 (&w)[8], const float4 *__restrict__ rec, int ks0, int lane) {
 #pragma unroll
-    for (int q = 0; q < NKS; ++q) {
-        wh[q] = __ldg(rec + (size_t)(ks0 + q) * 64 + 2 * lane);
-        wl[q] = __ldg(rec + (size_t)(ks0 + q) * 64 + 2 * lane + 1);
-    }
+    for (int q = 0; q < NKS; ++q) w[q] = __ldg(rec + (size_t)(ks0 + q) * 32 + lane);
 }
 template <int NKS>
-__device__ __forceinline__ void head_gemm(float (&c)[2][4], const float4 (&wh)[4], const float4 (&wl)[4], int ks0,
-                                          const float *__restrict__ act, int bstride, int lane) {
+__device__ __forceinline__ void head_gemm(float (&c)[4], const float4 (&w)[8], int ks0, const float *__restrict__ act, int bstride, int lane) {
     const int g = lane >> 2, t = lane & 3;
-#pragma unroll
-    for (int a = 0; a < 2; ++a)
-#pragma unroll
-        for (int b = 0; b < 4; ++b) c[a][b] = 0.f;
+    c[0] = c[1] = c[2] = c[3] = 0.f;
 #pragma unroll
     for (int q = 0; q < NKS; ++q) {
-        const uint32_t ah[4] = {__float_as_uint(wh[q].x), __float_as_uint(wh[q].y), __float_as_uint(wh[q].z), __float_as_uint(wh[q].w)};
-        const uint32_t al[4] = {__float_as_uint(wl[q].x), __float_as_uint(wl[q].y), __float_as_uint(wl[q].z), __float_as_uint(wl[q].w)};
-        const float *r0 = act + g * bstride + 2 * (8 * (ks0 + q) + t), *r1 = r0 + 8 * bstride;
+        uint32_t ah[4], al[4];
+        split_tf32(w[q].x, ah[0], al[0]); split_tf32(w[q].y, ah[1], al[1]);
+        split_tf32(w[q].z, ah[2], al[2]); split_tf32(w[q].w, ah[3], al[3]);
+        const float *r0 = act + g * bstride + 2 * (8 * (ks0 + q) + t);
         const float2 x0 = *reinterpret_cast<const float2 *>(r0), x1 = *reinterpret_cast<const float2 *>(r0 + 8);
-        const float2 y0 = *reinterpret_cast<const float2 *>(r1), y1 = *reinterpret_cast<const float2 *>(r1 + 8);
-        float p[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-        mma_tf32(p[0], al[0], al[1], al[2], al[3], __float_as_uint(x0.x), __float_as_uint(x1.x));
-        mma_tf32(p[1], al[0], al[1], al[2], al[3], __float_as_uint(y0.x), __float_as_uint(y1.x));
-        mma_tf32(p[0], ah[0], ah[1], ah[2], ah[3], __float_as_uint(x0.y), __float_as_uint(x1.y));
-        mma_tf32(p[1], ah[0], ah[1], ah[2], ah[3], __float_as_uint(y0.y), __float_as_uint(y1.y));
-        mma_tf32(p[0], ah[0], ah[1], ah[2], ah[3], __float_as_uint(x0.x), __float_as_uint(x1.x));
-        mma_tf32(p[1], ah[0], ah[1], ah[2], ah[3], __float_as_uint(y0.x), __float_as_uint(y1.x));
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt) { c[nt][0] += p[nt][0]; c[nt][1] += p[nt][1]; c[nt][2] += p[nt][2]; c[nt][3] += p[nt][3]; }
+        float p[4] = {0.f, 0.f, 0.f, 0.f};
+        mma_tf32(p, al[0], al[1], al[2], al[3], __float_as_uint(x0.x), __float_as_uint(x1.x));
+        mma_tf32(p, ah[0], ah[1], ah[2], ah[3], __float_as_uint(x0.y), __float_as_uint(x1.y));
+        mma_tf32(p, ah[0], ah[1], ah[2], ah[3], __float_as_uint(x0.x), __float_as_uint(x1.x));
+        c[0] += p[0]; c[1] += p[1]; c[2] += p[2]; c[3] += p[3];
     }
 }
 
-// c fragments (rows = 16 m + g, g + 8; columns = atoms) -> part[atom][row] with `pstride` floats per atom
-__device__ __forceinline__ void store_partial(const float (&c)[2][4], float *part, int pstride, int m_tile, int lane) {
+// c fragment (rows = 16 m + g, g + 8; columns = atoms 2t, 2t + 1) -> part[atom][row] with `pstride` floats per atom
+__device__ __forceinline__ void store_partial(const float (&c)[4], float *part, int pstride, int m_tile, int lane) {
     const int g = lane >> 2, t = lane & 3;
-#pragma unroll
-    for (int nt = 0; nt < 2; ++nt) {
-        float *p = part + (8 * nt + 2 * t) * pstride + 16 * m_tile + g;
-        p[0] = c[nt][0]; p[pstride] = c[nt][1]; p[8] = c[nt][2]; p[pstride + 8] = c[nt][3];
-    }
+    float *p = part + 2 * t * pstride + 16 * m_tile + g;
+    p[0] = c[0]; p[pstride] = c[1]; p[8] = c[2]; p[pstride + 8] = c[3];
 }
 
-// ---------------- Regression (Eq. 6) forward and reverse for the tile ----------------
+// ---------------- Regression (Eq. 6) forward and reverse for the group's tile ----------------
 // In: sX = invariants [atom][128].  Out: sX = dE/dG; per-atom energies written.
-// hc = biases [4][64], w_out [64], b_out of the species in shared memory.
+// hc = biases [4][64], w_out [64], b_out of the species in shared memory.  wg = warp within the group.
 __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float *hb, const float *hc, int species, int count, int first,
-                                          int warp, int lane, double &e_sum, PhaseClock &pc) {
+                                          int group, int wg, int lane, double &e_sum, PhaseClock &pc) {
     const float *hp = k.head_pack + (size_t)species * HP_TOTAL;
     const float4 *fwd = reinterpret_cast<const float4 *>(hp + HP_FWD), *bwd = reinterpret_cast<const float4 *>(hp + HP_BWD);
     float *xs = hb + HB_XS, *zs = hb + HB_ZS, *sD = hb + HB_SD, *dz = hb + HB_DZ, *dp = hb + HB_DP, *part = hb + HB_PART;
-    const int mt4 = warp & 3, kq = warp >> 2;   // forward / reverse hidden layers: 4 m-tiles x 4 k-quarters
-    const int atom = warp;                      // elementwise phases: warp = atom, lane = neuron (and neuron + 32)
-    float4 wh[4], wl[4];
+    const int mt4 = wg & 3, kh = wg >> 2;   // forward / reverse hidden layers: 4 m-tiles x 2 k-halves
+    const int atom = wg;                    // elementwise phases: warp = atom, lane = neuron (and neuron + 32)
+    float4 w[8];
 
-    head_load<KS0 / 4>(wh, wl, fwd + (size_t)(mt4 * KS0) * 64, kq * (KS0 / 4), lane);
+    head_load<KS0 / 2>(w, fwd + (size_t)(mt4 * KS0) * 32, kh * (KS0 / 2), lane);
     // split the invariants once
     for (int f = lane; f < N_INV; f += 32)
         *reinterpret_cast<float2 *>(xs + atom * 2 * X_STRIDE + 2 * f) = split_pair(sX[atom * X_STRIDE + f]);
     pc.mark(3);
-    __syncthreads();
+    group_sync(group);
     pc.mark(14);
 
     float e_i = 0.f;
@@ -586,23 +582,23 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
     for (int L = 0; L < HEAD_L; ++L) {
         const float *zin = zs + ((L + 1) & 1) * TILE * 2 * Z_STRIDE;
         float *zout = zs + (L & 1) * TILE * 2 * Z_STRIDE;
-        float c[2][4];
-        if (L == 0) head_gemm<KS0 / 4>(c, wh, wl, kq * (KS0 / 4), xs, 2 * X_STRIDE, lane);
-        else head_gemm<KS1 / 4>(c, wh, wl, kq * (KS1 / 4), zin, 2 * Z_STRIDE, lane);
+        float c[4];
+        if (L == 0) head_gemm<KS0 / 2>(c, w, kh * (KS0 / 2), xs, 2 * X_STRIDE, lane);
+        else head_gemm<KS1 / 2>(c, w, kh * (KS1 / 2), zin, 2 * Z_STRIDE, lane);
         pc.mark(12);
-        store_partial(c, part + kq * TILE * Z_STRIDE, Z_STRIDE, mt4, lane);
+        store_partial(c, part + kh * TILE * Z_STRIDE, Z_STRIDE, mt4, lane);
         // weights of the next pass
-        if (L < HEAD_L - 1) head_load<KS1 / 4>(wh, wl, fwd + (size_t)(4 * KS0 + L * 4 * KS1 + mt4 * KS1) * 64, kq * (KS1 / 4), lane);
-        else head_load<2>(wh, wl, bwd + (size_t)((N_INV / 16) * 8 + (HEAD_L - 2) * 32 + mt4 * 8) * 64, kq * 2, lane);
+        if (L < HEAD_L - 1) head_load<KS1 / 2>(w, fwd + (size_t)(4 * KS0 + L * 4 * KS1 + mt4 * KS1) * 32, kh * (KS1 / 2), lane);
+        else head_load<4>(w, bwd + (size_t)((N_INV / 16) * 8 + (HEAD_L - 2) * 32 + mt4 * 8) * 32, kh * 4, lane);
         pc.mark(13);
-        __syncthreads();
+        group_sync(group);
         pc.mark(14);
         // elementwise: bias, SiLU, residual; this thread owns neurons lane and lane + 32 of its atom
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
             const int nn = lane + 32 * q;
             const float *pp = part + atom * Z_STRIDE + nn;
-            const float pre = ((pp[0] + pp[TILE * Z_STRIDE]) + (pp[2 * TILE * Z_STRIDE] + pp[3 * TILE * Z_STRIDE])) + hc[L * HEAD_H + nn];
+            const float pre = (pp[0] + pp[TILE * Z_STRIDE]) + hc[L * HEAD_H + nn];
             float d, y = silu_f(pre, d);
             if (L > 0) { const float2 zi = *reinterpret_cast<const float2 *>(zin + atom * 2 * Z_STRIDE + 2 * nn); y += zi.x + zi.y; }
             sD[(L * TILE + atom) * Z_STRIDE + nn] = d;
@@ -616,7 +612,7 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
             }
         }
         pc.mark(15);
-        __syncthreads();
+        group_sync(group);
         pc.mark(14);
     }
 #pragma unroll
@@ -628,171 +624,157 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
     }
 
     // reverse through the hidden layers 3, 2, 1 (each with its skip path)
-    const int mt8 = warp & 7, kh = warp >> 3;   // first layer: 8 m-tiles x 2 k-halves
 #pragma unroll
     for (int L = HEAD_L - 1; L >= 1; --L) {
-        float c[2][4];
-        head_gemm<2>(c, wh, wl, kq * 2, dp, 2 * Z_STRIDE, lane);
-        store_partial(c, part + kq * TILE * Z_STRIDE, Z_STRIDE, mt4, lane);
-        if (L > 1) head_load<2>(wh, wl, bwd + (size_t)((N_INV / 16) * 8 + (L - 2) * 32 + mt4 * 8) * 64, kq * 2, lane);
-        else head_load<4>(wh, wl, bwd + (size_t)(mt8 * 8) * 64, kh * 4, lane);
-        __syncthreads();
+        float c[4];
+        head_gemm<4>(c, w, kh * 4, dp, 2 * Z_STRIDE, lane);
+        store_partial(c, part + kh * TILE * Z_STRIDE, Z_STRIDE, mt4, lane);
+        if (L > 1) head_load<4>(w, bwd + (size_t)((N_INV / 16) * 8 + (L - 2) * 32 + mt4 * 8) * 32, kh * 4, lane);
+        else head_load<8>(w, bwd + (size_t)(wg * 8) * 32, 0, lane);   // first layer: warp = m-tile, all 8 k-steps
+        group_sync(group);
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
             const int nn = lane + 32 * q;
             const float *pp = part + atom * Z_STRIDE + nn;
-            const float dzn = dz[atom * Z_STRIDE + nn] + ((pp[0] + pp[TILE * Z_STRIDE]) + (pp[2 * TILE * Z_STRIDE] + pp[3 * TILE * Z_STRIDE]));
+            const float dzn = dz[atom * Z_STRIDE + nn] + (pp[0] + pp[TILE * Z_STRIDE]);
             dz[atom * Z_STRIDE + nn] = dzn;
             *reinterpret_cast<float2 *>(dp + atom * 2 * Z_STRIDE + 2 * nn) = split_pair(dzn * sD[((L - 1) * TILE + atom) * Z_STRIDE + nn]);
         }
-        __syncthreads();
+        group_sync(group);
     }
-    {   // first layer: dE/dG [128 x 16]
-        float c[2][4];
-        head_gemm<4>(c, wh, wl, kh * 4, dp, 2 * Z_STRIDE, lane);
-        store_partial(c, part + kh * TILE * X_STRIDE, X_STRIDE, mt8, lane);
-        __syncthreads();
-        for (int f = lane; f < N_INV; f += 32)
-            sX[atom * X_STRIDE + f] = part[atom * X_STRIDE + f] + part[TILE * X_STRIDE + atom * X_STRIDE + f];
+    {   // first layer: dE/dG [128 x 8], warp = m-tile (16 inputs), written over the invariants
+        float c[4];
+        head_gemm<8>(c, w, 0, dp, 2 * Z_STRIDE, lane);
+        store_partial(c, sX, X_STRIDE, wg, lane);
     }
-    __syncthreads();
+    group_sync(group);
 }
 
 template <bool TAB_SMEM>
 __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words) {
     extern __shared__ __align__(16) float smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int group = warp / TILE, wg = warp % TILE;
     const int g = lane >> 2, t = lane & 3;
-    float *s_tab = smem;                         // [C][rows][TAB_STRIDE_SMEM] when TAB_SMEM
-    float *sX = smem + (TAB_SMEM ? tab_words : 0);
-    float *hb = sX + SX_WORDS;                   // head buffers = the scratch of all warps
-    float *scr = hb + warp * SCR_WORDS;
-    float4 *pq = reinterpret_cast<float4 *>(hb + NW * SCR_WORDS + warp * Q_WORDS);
-    float *hc = hb + NW * (SCR_WORDS + Q_WORDS);
+    float *s_tab = smem;                                   // [C][rows][TAB_STRIDE_SMEM] when TAB_SMEM
+    float *sX = smem + (TAB_SMEM ? tab_words : 0) + group * SX_WORDS;
+    float *scr_all = smem + (TAB_SMEM ? tab_words : 0) + NG * SX_WORDS;
+    float *hb = scr_all + group * TILE * SCR_WORDS;        // head buffers = the scratch of the group's warps
+    float *scr = scr_all + warp * SCR_WORDS;
+    float4 *pq = reinterpret_cast<float4 *>(scr_all + NW * SCR_WORDS + warp * Q_WORDS);
+    float *hc = scr_all + NW * (SCR_WORDS + Q_WORDS);
     int *ctl = reinterpret_cast<int *>(hc + HC_WORDS);
     const int rows = k.tab.knots + 3;
-
-    // species-pure tiles: tiles of species s start at tile_first[s]
-    int tile_first[MAX_SPECIES + 1];
-    tile_first[0] = 0;
-#pragma unroll
-    for (int s = 0; s < MAX_SPECIES; ++s) {
-        int cnt = s < k.n_species ? __ldg(k.species_start + s + 1) - __ldg(k.species_start + s) : 0;
-        tile_first[s + 1] = tile_first[s] + (cnt + TILE - 1) / TILE;
-    }
-    const int n_tiles = tile_first[MAX_SPECIES];
 
     double e_sum = 0.0;
     float vir[9] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     unsigned long long n_pairs = 0;
-    int loaded_species = -1;
     TableView tv;
     PhaseClock pc;
     pc.start();
 
-    while (true) {
-        __syncthreads();
-        if (threadIdx.x == 0) ctl[0] = atomicAdd(k.tile_counter, 1);
-        __syncthreads();
-        pc.mark(11);
-        const int tile = ctl[0];
-        if (tile >= n_tiles) break;
-        int species = 0;
-#pragma unroll
-        for (int s = 1; s < MAX_SPECIES; ++s) species += tile >= tile_first[s] ? 1 : 0;
+    for (int species = 0; species < k.n_species; ++species) {
         const int s_beg = __ldg(k.species_start + species), s_end = __ldg(k.species_start + species + 1);
-        const int first = s_beg + (tile - tile_first[species]) * TILE;
-        const int count = min(TILE, s_end - first);
-
-        if (species != loaded_species) {   // radial tables of this central species
-            if (TAB_SMEM) {
-                const float4 *src = reinterpret_cast<const float4 *>(k.tab.coef + (size_t)species * k.n_species * rows * K_RADIAL);
-                const int n4 = k.n_species * rows * (K_RADIAL / 4);
-                for (int idx = threadIdx.x; idx < n4; idx += NW * 32)
-                    *reinterpret_cast<float4 *>(s_tab + (idx >> 3) * TAB_STRIDE_SMEM + 4 * (idx & 7)) = __ldg(src + idx);
-                tv.base = s_tab; tv.row_stride = TAB_STRIDE_SMEM; tv.table_stride = rows * TAB_STRIDE_SMEM;
-            } else {
-                tv.base = k.tab.coef + (size_t)species * k.n_species * rows * K_RADIAL;
-                tv.row_stride = K_RADIAL; tv.table_stride = rows * K_RADIAL;
-            }
-            for (int idx = threadIdx.x; idx < HEAD_L * HEAD_H + HEAD_H + 1; idx += NW * 32)
-                hc[idx] = __ldg(k.head_pack + (size_t)species * HP_TOTAL + HP_BIAS + idx);
-            loaded_species = species;
-            __syncthreads();
+        const int n_tiles = (s_end - s_beg + TILE - 1) / TILE;
+        if (n_tiles == 0) continue;
+        __syncthreads();   // both groups are done with the previous species' tables
+        if (TAB_SMEM) {
+            const float4 *src = reinterpret_cast<const float4 *>(k.tab.coef + (size_t)species * k.n_species * rows * K_RADIAL);
+            const int n4 = k.n_species * rows * (K_RADIAL / 4);
+            for (int idx = threadIdx.x; idx < n4; idx += NW * 32)
+                *reinterpret_cast<float4 *>(s_tab + (idx >> 3) * TAB_STRIDE_SMEM + 4 * (idx & 7)) = __ldg(src + idx);
+            tv.base = s_tab; tv.row_stride = TAB_STRIDE_SMEM; tv.table_stride = rows * TAB_STRIDE_SMEM;
+        } else {
+            tv.base = k.tab.coef + (size_t)species * k.n_species * rows * K_RADIAL;
+            tv.row_stride = K_RADIAL; tv.table_stride = rows * K_RADIAL;
         }
-
-        // ---------------- Encoding + invariants: warp = atom ----------------
-        const bool have = warp < count;
-        const int i = have ? __ldg(k.center_order + first + warp) : 0;
-        double4 pi = make_double4(0.0, 0.0, 0.0, 0.0);
-        int64_t beg = 0, end = 0;
-        float Pf[4][4];
-        int queued = -1;
-        float *xrow = sX + warp * X_STRIDE;
-        if (have) {
-            pi = k.pos4[i];
-            beg = k.nbr_off[i]; end = k.nbr_off[i + 1];
-            n_pairs += encode_atom(k, tv, pi, beg, end, pq, scr, lane, Pf, queued, pc);
-            // Eq. 5 (C_l = I): this lane holds rows a = g, g + 8 of channels 8t + j; sum squares over the rows of a block
-            float part[4][8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const float pa = Pf[j & 3][j >> 2], pb = Pf[j & 3][2 + (j >> 2)];
-                part[0][j] = g == 0 ? pa : 0.f;
-                part[1][j] = (g >= 1 && g <= 3) ? pa * pa : 0.f;
-                part[2][j] = (g >= 4 ? pa * pa : 0.f) + (g == 0 ? pb * pb : 0.f);
-                part[3][j] = g >= 1 ? pb * pb : 0.f;
-            }
-#pragma unroll
-            for (int o = 4; o < 32; o <<= 1)
-#pragma unroll
-                for (int l = 0; l < 4; ++l)
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) part[l][j] += __shfl_xor_sync(0xffffffffu, part[l][j], o);
-            if (g == 0) {
-#pragma unroll
-                for (int l = 0; l < 4; ++l) {
-                    *reinterpret_cast<float4 *>(xrow + 32 * l + 8 * t) = make_float4(part[l][0], part[l][1], part[l][2], part[l][3]);
-                    *reinterpret_cast<float4 *>(xrow + 32 * l + 8 * t + 4) = make_float4(part[l][4], part[l][5], part[l][6], part[l][7]);
-                }
-            }
-        } else {   // empty slot of a ragged tile: feed zeros to the head
-            for (int c = lane; c < N_INV; c += 32) xrow[c] = 0.f;
-        }
-        pc.mark(7);
+        for (int idx = threadIdx.x; idx < HEAD_L * HEAD_H + HEAD_H + 1; idx += NW * 32)
+            hc[idx] = __ldg(k.head_pack + (size_t)species * HP_TOTAL + HP_BIAS + idx);
         __syncthreads();
-        pc.mark(8);
 
-        // ---------------- Regression ----------------
-        head_tile(k, sX, hb, hc, species, count, first, warp, lane, e_sum, pc);
-        pc.mark(9);
+        while (true) {   // the group's tiles of this species
+            group_sync(group);
+            if (wg == 0 && lane == 0) ctl[group] = atomicAdd(k.tile_counter + species, 1);
+            group_sync(group);
+            pc.mark(11);
+            const int tile = ctl[group];
+            if (tile >= n_tiles) break;
+            const int first = s_beg + tile * TILE;
+            const int count = min(TILE, s_end - first);
 
-        // ---------------- Derivation ----------------
-        if (have) {
-            // W_i = dE_i/dP_i (Eq. 7), already in B-fragment order
-            const int la = g == 0 ? 0 : (g <= 3 ? 1 : 2), lb = g == 0 ? 2 : 3;
-            float da[8], db[8];
-            {
-                const float4 a0 = *reinterpret_cast<const float4 *>(xrow + 32 * la + 8 * t), a1 = *reinterpret_cast<const float4 *>(xrow + 32 * la + 8 * t + 4);
-                const float4 b0 = *reinterpret_cast<const float4 *>(xrow + 32 * lb + 8 * t), b1 = *reinterpret_cast<const float4 *>(xrow + 32 * lb + 8 * t + 4);
-                da[0] = a0.x; da[1] = a0.y; da[2] = a0.z; da[3] = a0.w; da[4] = a1.x; da[5] = a1.y; da[6] = a1.z; da[7] = a1.w;
-                db[0] = b0.x; db[1] = b0.y; db[2] = b0.z; db[3] = b0.w; db[4] = b1.x; db[5] = b1.y; db[6] = b1.z; db[7] = b1.w;
-            }
-            uint32_t Wh[4][4], Wl[4][4];
+            // ---------------- Encoding + invariants: warp = atom ----------------
+            const bool have = wg < count;
+            const int i = have ? __ldg(k.center_order + first + wg) : 0;
+            double4 pi = make_double4(0.0, 0.0, 0.0, 0.0);
+            int64_t beg = 0, end = 0;
+            float Pf[4][4];
+            int queued = -1;
+            float *xrow = sX + wg * X_STRIDE;
+            if (have) {
+                pi = k.pos4[i];
+                beg = k.nbr_off[i]; end = k.nbr_off[i + 1];
+                n_pairs += encode_atom(k, tv, pi, beg, end, pq, scr, lane, Pf, queued, pc);
+                // Eq. 5 (C_l = I): this lane holds rows a = g, g + 8 of channels 8t + j; sum squares over the rows of a block
+                float part[4][8];
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
-                const float w0 = g == 0 ? da[ks] : 2.f * da[ks] * Pf[ks][0];          // row a = g,     channel 8t + ks
-                const float w1 = g == 0 ? da[4 + ks] : 2.f * da[4 + ks] * Pf[ks][1];  // row a = g,     channel 8t + 4 + ks
-                const float w2 = 2.f * db[ks] * Pf[ks][2];                            // row a = g + 8, channel 8t + ks
-                const float w3 = 2.f * db[4 + ks] * Pf[ks][3];                        // row a = g + 8, channel 8t + 4 + ks
-                split_tf32(w0, Wh[ks][0], Wl[ks][0]);
-                split_tf32(w1, Wh[ks][1], Wl[ks][1]);
-                split_tf32(w2, Wh[ks][2], Wl[ks][2]);
-                split_tf32(w3, Wh[ks][3], Wl[ks][3]);
+                for (int j = 0; j < 8; ++j) {
+                    const float pa = Pf[j & 3][j >> 2], pb = Pf[j & 3][2 + (j >> 2)];
+                    part[0][j] = g == 0 ? pa : 0.f;
+                    part[1][j] = (g >= 1 && g <= 3) ? pa * pa : 0.f;
+                    part[2][j] = (g >= 4 ? pa * pa : 0.f) + (g == 0 ? pb * pb : 0.f);
+                    part[3][j] = g >= 1 ? pb * pb : 0.f;
+                }
+#pragma unroll
+                for (int o = 4; o < 32; o <<= 1)
+#pragma unroll
+                    for (int l = 0; l < 4; ++l)
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) part[l][j] += __shfl_xor_sync(0xffffffffu, part[l][j], o);
+                if (g == 0) {
+#pragma unroll
+                    for (int l = 0; l < 4; ++l) {
+                        *reinterpret_cast<float4 *>(xrow + 32 * l + 8 * t) = make_float4(part[l][0], part[l][1], part[l][2], part[l][3]);
+                        *reinterpret_cast<float4 *>(xrow + 32 * l + 8 * t + 4) = make_float4(part[l][4], part[l][5], part[l][6], part[l][7]);
+                    }
+                }
+            } else {   // empty slot of a ragged tile: feed zeros to the head
+                for (int c = lane; c < N_INV; c += 32) xrow[c] = 0.f;
             }
-            derive_atom(k, tv, pi, i, beg, end, pq, scr, queued, lane, Wh, Wl, vir, pc);
+            pc.mark(7);
+            group_sync(group);
+            pc.mark(8);
+
+            // ---------------- Regression ----------------
+            head_tile(k, sX, hb, hc, species, count, first, group, wg, lane, e_sum, pc);
+            pc.mark(9);
+
+            // ---------------- Derivation ----------------
+            if (have) {
+                // W_i = dE_i/dP_i (Eq. 7), already in B-fragment order
+                const int la = g == 0 ? 0 : (g <= 3 ? 1 : 2), lb = g == 0 ? 2 : 3;
+                float da[8], db[8];
+                {
+                    const float4 a0 = *reinterpret_cast<const float4 *>(xrow + 32 * la + 8 * t), a1 = *reinterpret_cast<const float4 *>(xrow + 32 * la + 8 * t + 4);
+                    const float4 b0 = *reinterpret_cast<const float4 *>(xrow + 32 * lb + 8 * t), b1 = *reinterpret_cast<const float4 *>(xrow + 32 * lb + 8 * t + 4);
+                    da[0] = a0.x; da[1] = a0.y; da[2] = a0.z; da[3] = a0.w; da[4] = a1.x; da[5] = a1.y; da[6] = a1.z; da[7] = a1.w;
+                    db[0] = b0.x; db[1] = b0.y; db[2] = b0.z; db[3] = b0.w; db[4] = b1.x; db[5] = b1.y; db[6] = b1.z; db[7] = b1.w;
+                }
+                uint32_t Wh[4][4], Wl[4][4];
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    const float w0 = g == 0 ? da[ks] : 2.f * da[ks] * Pf[ks][0];          // row a = g,     channel 8t + ks
+                    const float w1 = g == 0 ? da[4 + ks] : 2.f * da[4 + ks] * Pf[ks][1];  // row a = g,     channel 8t + 4 + ks
+                    const float w2 = 2.f * db[ks] * Pf[ks][2];                            // row a = g + 8, channel 8t + ks
+                    const float w3 = 2.f * db[4 + ks] * Pf[ks][3];                        // row a = g + 8, channel 8t + 4 + ks
+                    split_tf32(w0, Wh[ks][0], Wl[ks][0]);
+                    split_tf32(w1, Wh[ks][1], Wl[ks][1]);
+                    split_tf32(w2, Wh[ks][2], Wl[ks][2]);
+                    split_tf32(w3, Wh[ks][3], Wl[ks][3]);
+                }
+                derive_atom(k, tv, pi, i, beg, end, pq, scr, queued, lane, Wh, Wl, vir, pc);
+            }
+            pc.mark(10);
         }
-        pc.mark(10);
     }
     pc.flush(k.acc, lane);
 
@@ -811,14 +793,6 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
 }
 
 // ---------------- host side ----------------
-static inline void split_host(float x, float &hi, float &lo) {
-    uint32_t u;
-    memcpy(&u, &x, 4);
-    u = (u + 0x1000u) & 0xffffe000u;   // round to nearest (ties away) at 10 mantissa bits
-    memcpy(&hi, &u, 4);
-    lo = x - hi;
-}
-
 int table_smem_words(const mlip_ctx *c) { return c->cfg.n_species * (c->cfg.table_knots + 3) * TAB_STRIDE_SMEM; }
 bool tables_fit_smem(const mlip_ctx *c) { return FIXED_WORDS + table_smem_words(c) <= SMEM_LIMIT_WORDS; }
 
@@ -839,27 +813,27 @@ int upload_head(mlip_ctx *c, const double *w) {
                 for (int ks = 0; ks < nks; ++ks)
                     for (int lane = 0; lane < 32; ++lane) {
                         const int g = lane >> 2, t = lane & 3;
-                        float *rec = fwd + ((size_t)(mt * nks + ks) * 32 + lane) * 8;
-                        split_host((float)src[(16 * mt + g) * in + 8 * ks + t], rec[0], rec[4]);
-                        split_host((float)src[(16 * mt + g + 8) * in + 8 * ks + t], rec[1], rec[5]);
-                        split_host((float)src[(16 * mt + g) * in + 8 * ks + t + 4], rec[2], rec[6]);
-                        split_host((float)src[(16 * mt + g + 8) * in + 8 * ks + t + 4], rec[3], rec[7]);
+                        float *rec = fwd + ((size_t)(mt * nks + ks) * 32 + lane) * 4;
+                        rec[0] = (float)src[(16 * mt + g) * in + 8 * ks + t];
+                        rec[1] = (float)src[(16 * mt + g + 8) * in + 8 * ks + t];
+                        rec[2] = (float)src[(16 * mt + g) * in + 8 * ks + t + 4];
+                        rec[3] = (float)src[(16 * mt + g + 8) * in + 8 * ks + t + 4];
                     }
             // reverse: A[m][k] = W[k][m] (m = input, k = neuron); record (mt, ks)
             for (int mt = 0; mt < in / 16; ++mt)
                 for (int ks = 0; ks < 8; ++ks)
                     for (int lane = 0; lane < 32; ++lane) {
                         const int g = lane >> 2, t = lane & 3;
-                        float *rec = bwd + ((size_t)(mt * 8 + ks) * 32 + lane) * 8;
-                        split_host((float)src[(8 * ks + t) * in + 16 * mt + g], rec[0], rec[4]);
-                        split_host((float)src[(8 * ks + t) * in + 16 * mt + g + 8], rec[1], rec[5]);
-                        split_host((float)src[(8 * ks + t + 4) * in + 16 * mt + g], rec[2], rec[6]);
-                        split_host((float)src[(8 * ks + t + 4) * in + 16 * mt + g + 8], rec[3], rec[7]);
+                        float *rec = bwd + ((size_t)(mt * 8 + ks) * 32 + lane) * 4;
+                        rec[0] = (float)src[(8 * ks + t) * in + 16 * mt + g];
+                        rec[1] = (float)src[(8 * ks + t) * in + 16 * mt + g + 8];
+                        rec[2] = (float)src[(8 * ks + t + 4) * in + 16 * mt + g];
+                        rec[3] = (float)src[(8 * ks + t + 4) * in + 16 * mt + g + 8];
                     }
             for (int o = 0; o < HEAD_H; ++o) hp[HP_BIAS + L * HEAD_H + o] = (float)src[in * HEAD_H + o];
             src += in * HEAD_H + HEAD_H;
-            fwd += (size_t)4 * nks * 256;
-            bwd += (size_t)(in / 16) * 8 * 256;
+            fwd += (size_t)4 * nks * 128;
+            bwd += (size_t)(in / 16) * 8 * 128;
             in = HEAD_H;
         }
         for (int o = 0; o < HEAD_H + 1; ++o) hp[HP_WOUT + o] = (float)src[o];
@@ -877,7 +851,7 @@ int launch_megakernel(mlip_ctx *c, cudaStream_t s) {
     MLIP_CUDA_TRY(c, cudaMemsetAsync(c->force, 0, sizeof(float4) * n, s));
     MLIP_CUDA_TRY(c, cudaMemsetAsync(c->acc, 0, sizeof(double) * ACC_KINETIC, s));
     MLIP_CUDA_TRY(c, cudaMemsetAsync(c->pair_counter, 0, sizeof(unsigned long long), s));
-    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->tile_counter, 0, sizeof(int), s));
+    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->tile_counter, 0, sizeof(int) * MAX_SPECIES, s));
     const int64_t tiles_max = (n + TILE - 1) / TILE + c->cfg.n_species;
     const int blocks = (int)std::min<int64_t>(tiles_max, (int64_t)c->n_sm);
     const bool in_smem = tables_fit_smem(c);
