@@ -62,7 +62,9 @@ constexpr int HB_PART = HB_DP + TILE * 2 * Z_STRIDE;       // split-K partials  
 constexpr int HB_WORDS = HB_PART + 2 * TILE * Z_STRIDE;
 static_assert(HB_WORDS <= TILE * SCR_WORDS, "head buffers alias the scratch of the group's warps");
 constexpr int HC_WORDS = HEAD_L * HEAD_H + HEAD_H + 16;         // biases, w_out, b_out of the current species
-constexpr int FIXED_WORDS = NG * SX_WORDS + NW * (Q_WORDS + SCR_WORDS) + HC_WORDS + 16;
+constexpr int PF_IDX = 160;                                     // neighbor indices prefetched per warp for its next atom
+constexpr int PF_WORDS = PF_IDX + 4;                            // + {atom, list start (2 words), list length}
+constexpr int FIXED_WORDS = NG * SX_WORDS + NW * (Q_WORDS + SCR_WORDS + PF_WORDS) + HC_WORDS + 16;
 constexpr int SMEM_LIMIT_WORDS = 227 * 1024 / 4 - 256;
 
 // Pre-packed head weights per species (floats).  A record holds the A operand of one
@@ -103,23 +105,17 @@ __device__ __forceinline__ void mma_tf32(float (&c)[4], uint32_t a0, uint32_t a1
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// c += A B with both operands split: A_hi B_hi + A_lo B_hi + A_hi B_lo.  The tensor pipe truncates
-// when it adds into its fp32 accumulator, so callers keep accumulation chains short (a fresh
-// accumulator per k-step, folded into the running sum by a rounded fp32 add): a long chain of
-// same-sign terms otherwise drifts by ~1e-6 relative.
-__device__ __forceinline__ void mma3(float (&c)[4], const uint32_t (&ah)[4], const uint32_t (&al)[4], uint32_t bh0, uint32_t bh1,
-                                     uint32_t bl0, uint32_t bl1) {
-    mma_tf32(c, al[0], al[1], al[2], al[3], bh0, bh1);
-    mma_tf32(c, ah[0], ah[1], ah[2], ah[3], bl0, bl1);
-    mma_tf32(c, ah[0], ah[1], ah[2], ah[3], bh0, bh1);
+// d = A B (zero accumulator input: saves initialising the accumulator registers)
+__device__ __forceinline__ void mma_tf32_z(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
 }
-// Same product with the main and the small terms kept in separate accumulators.
-__device__ __forceinline__ void mma3s(float (&c)[4], float (&cs)[4], const uint32_t (&ah)[4], const uint32_t (&al)[4],
-                                      uint32_t bh0, uint32_t bh1, uint32_t bl0, uint32_t bl1) {
-    mma_tf32(cs, al[0], al[1], al[2], al[3], bh0, bh1);
-    mma_tf32(cs, ah[0], ah[1], ah[2], ah[3], bl0, bl1);
-    mma_tf32(c, ah[0], ah[1], ah[2], ah[3], bh0, bh1);
-}
+
+// Every product A B below has both operands split: A_hi B_hi + A_lo B_hi + A_hi B_lo.  The tensor
+// pipe truncates when it adds into its fp32 accumulator, so the energy path keeps accumulation
+// chains short (a fresh accumulator per k-step, folded into the running sum by a rounded fp32
+// add): a long chain of same-sign terms otherwise drifts by ~1e-6 relative.
 
 // Irreducible harmonic polynomials up to l = 3 of a unit vector (one valid solution of the
 // projection constraints of Section 3.3.1: harmonic, orthonormal under the multinomial metric).
@@ -235,6 +231,14 @@ struct KernelArgs {
     int *tile_counter;
 };
 
+// One 256-bit load per gathered atom (a 32-byte sector) instead of two 128-bit ones: halves the
+// number of L1 wavefronts of the uncoalesced position gathers.
+__device__ __forceinline__ double4 load_pos4(const double4 *p) {
+    double4 v;
+    asm volatile("ld.global.nc.v4.f64 {%0,%1,%2,%3}, [%4];" : "=d"(v.x), "=d"(v.y), "=d"(v.z), "=d"(v.w) : "l"(p));
+    return v;
+}
+
 // Where the radial tables of the current central species live: shared memory (rows padded to
 // TAB_STRIDE_SMEM, table index = neighbor species) or, when they do not fit, global memory.
 struct TableView {
@@ -243,24 +247,29 @@ struct TableView {
     int table_stride;   // floats per neighbor species
 };
 
-// Fill the warp's pair queue from list position `cur` on (lane = entry), four chunks at a time with
-// all index loads, then all position gathers, in flight together.  Pairs inside r_cut are queued as
-// {x, y, z, j | species << 28}.  Stops when the list ends or the next group might not fit; returns
-// the number of queued pairs and advances `cur`.
-__device__ __forceinline__ int collect_pairs(const KernelArgs &k, const double4 &pi, int64_t &cur, int64_t end, float4 *pq, int lane) {
+// Fill the warp's pair queue from list position `cur` on (lane = entry), up to five 32-entry chunks
+// at a time with all index loads, then all position gathers, in flight together (a typical list
+// of ~134 entries is one round trip).  Pairs inside r_cut are queued as {x, y, z, j | species << 28}.
+// Stops when the list ends or the next group might not fit; returns the number of queued pairs
+// and advances `cur`.  The first n_pref indices of the list may come from shared memory (sidx).
+constexpr int SCAN_CHUNKS = 5;
+static_assert(SCAN_CHUNKS * 32 <= PB_CAP, "a full group must fit an empty queue");
+__device__ __forceinline__ int collect_pairs(const KernelArgs &k, const double4 &pi, int64_t beg, int64_t &cur, int64_t end, float4 *pq, int lane,
+                                             const int *sidx, int n_pref) {
     int nq = 0;
-    while (cur < end && nq + (int)min((int64_t)128, end - cur) <= PB_CAP) {
-        int jj[4];
+    while (cur < end && nq + (int)min((int64_t)(SCAN_CHUNKS * 32), end - cur) <= PB_CAP) {
+        int jj[SCAN_CHUNKS];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < SCAN_CHUNKS; ++c) {
             const int64_t e = cur + 32 * c + lane;
-            jj[c] = e < end ? __ldg(k.nbr + e) : -1;
+            jj[c] = e < end ? (e - beg < n_pref ? sidx[e - beg] : __ldg(k.nbr + e)) : -1;
         }
-        double4 pp[4];
+        double4 pp[SCAN_CHUNKS];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) pp[c] = k.pos4[jj[c] < 0 ? 0 : jj[c]];
+        for (int c = 0; c < SCAN_CHUNKS; ++c) pp[c] = load_pos4(k.pos4 + (jj[c] < 0 ? 0 : jj[c]));
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < SCAN_CHUNKS; ++c) {
+            if (cur + 32 * c >= end) continue;   // warp-uniform: nothing in this chunk
             const double dx = min_image(pp[c].x - pi.x, k.grid.box[0], k.grid.half[0]);
             const double dy = min_image(pp[c].y - pi.y, k.grid.box[1], k.grid.half[1]);
             const double dz = min_image(pp[c].z - pi.z, k.grid.box[2], k.grid.half[2]);
@@ -272,7 +281,7 @@ __device__ __forceinline__ int collect_pairs(const KernelArgs &k, const double4 
                     make_float4((float)dx, (float)dy, (float)dz, __int_as_float(jj[c] | ((int)pp[c].w << J_BITS)));
             nq += __popc(m);
         }
-        cur += 128;
+        cur += SCAN_CHUNKS * 32;
     }
     __syncwarp();
     return nq;
@@ -282,7 +291,8 @@ __device__ __forceinline__ int collect_pairs(const KernelArgs &k, const double4 
 // `queued` returns the number of pairs left in the queue when the whole list fitted in one round
 // (the derivation then reuses them), or -1.
 __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView &tv, const double4 &pi, int64_t beg, int64_t end,
-                                           float4 *pq, float *stage, int lane, float (&Pf)[4][4], int &queued, PhaseClock &pc) {
+                                           float4 *pq, float *stage, int lane, float (&Pf)[4][4], int &queued, const int *sidx, int n_pref,
+                                           PhaseClock &pc) {
     const int g = lane >> 2, t = lane & 3;
     const int rs = tv.row_stride;
 #pragma unroll
@@ -349,10 +359,9 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
             for (int nt = 0; nt < 4; ++nt) {
                 split_tf32(ga[nt], bh[nt][0], bl[nt][0]);
                 split_tf32(gb[nt], bh[nt][1], bl[nt][1]);
-                c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
             }
 #pragma unroll
-            for (int nt = 0; nt < 4; ++nt) mma_tf32(c[nt], al[0], al[1], al[2], al[3], bh[nt][0], bh[nt][1]);
+            for (int nt = 0; nt < 4; ++nt) mma_tf32_z(c[nt], al[0], al[1], al[2], al[3], bh[nt][0], bh[nt][1]);
 #pragma unroll
             for (int nt = 0; nt < 4; ++nt) mma_tf32(c[nt], ah[0], ah[1], ah[2], ah[3], bl[nt][0], bl[nt][1]);
 #pragma unroll
@@ -366,7 +375,7 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
     int total = 0, rounds = 0, n = 0;
     int64_t cur = beg;
     do {
-        n = collect_pairs(k, pi, cur, end, pq, lane);
+        n = collect_pairs(k, pi, beg, cur, end, pq, lane, sidx, n_pref);
         pc.mark(0);
         for (int q0 = 0; q0 < n; q0 += 32) batch(q0, min(32, n - q0));
         total += n;
@@ -386,22 +395,36 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
     float fx = 0.f, fy = 0.f, fz = 0.f;
 
     auto batch = [&](int first, int n) {
-        float4 ent = make_float4(1.f, 0.f, 0.f, 0.f);
-        float rinv = 1.f;
         {   // lane = pair: spline basis and its derivative
+            float4 ent = make_float4(1.f, 0.f, 0.f, 0.f);
+            float rinv = 1.f;
             float b[4] = {0.f, 0.f, 0.f, 0.f}, db[4] = {0.f, 0.f, 0.f, 0.f};
-            int off = 0;
-            if (lane < n) {
+            int off = 0, row_index = 0;
+            const bool live = lane < n;
+            if (live) {
                 ent = pq[first + lane];
                 const float r = sqrtf(ent.x * ent.x + ent.y * ent.y + ent.z * ent.z);
                 rinv = 1.0f / r;
                 const int iv = spline_basis<true>(r, k.tab, b, db, k.status);
-                off = (__float_as_int(ent.w) >> J_BITS) * tv.table_stride + iv * rs;
+                row_index = (__float_as_int(ent.w) >> J_BITS) * (k.tab.knots + 3) + iv;
+                off = row_index * rs;
             }
-            float4 *row = reinterpret_cast<float4 *>(bs + lane * BS_STRIDE);
+            // Slot of this pair in the batch: pairs whose table rows have even index go to even slots, odd
+            // to odd (as far as the counts allow).  Neighboring fragment rows then read table rows of
+            // opposite parity, which the padded row stride maps to disjoint shared-memory banks.
+            const unsigned lt = (1u << lane) - 1u;
+            const unsigned ev = __ballot_sync(0xffffffffu, live && !(row_index & 1)), od = __ballot_sync(0xffffffffu, live && (row_index & 1));
+            const int ne = __popc(ev), no = __popc(od), ecap = (n + 1) >> 1, ocap = n >> 1;
+            const int re = __popc(ev & lt), ro = __popc(od & lt);
+            int slot = lane;
+            if (live) slot = (row_index & 1) ? (ro < ocap ? 2 * ro + 1 : 2 * (ne + ro - ocap)) : (re < ecap ? 2 * re : 2 * (no + re - ecap) + 1);
+            float4 *row = reinterpret_cast<float4 *>(bs + slot * BS_STRIDE);
             row[0] = make_float4(b[0], b[1], b[2], b[3]);
             row[1] = make_float4(db[0], db[1], db[2], db[3]);
-            reinterpret_cast<int *>(bs)[lane * BS_STRIDE + 8] = off;
+            reinterpret_cast<int *>(bs)[slot * BS_STRIDE + 8] = off;
+            // geometry for the projection, which runs with lane = slot (spare words of the V/T row)
+            *reinterpret_cast<float4 *>(vt + slot * VT_STRIDE + 32) = ent;
+            vt[slot * VT_STRIDE + 36] = rinv;
         }
         __syncwarp();
         pc.mark(4);
@@ -411,10 +434,6 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
             // (one accumulator per output here: the truncating accumulation costs ~1e-6 relative on a
             // 12-term chain, irrelevant for forces, and the registers are needed elsewhere)
             float V[2][4], T[2][4];
-#pragma unroll
-            for (int a = 0; a < 2; ++a)
-#pragma unroll
-                for (int b = 0; b < 4; ++b) { V[a][b] = 0.f; T[a][b] = 0.f; }
             float G[2][8], dG[2][8];
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
@@ -441,10 +460,17 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
                 split_tf32(dG[0][4 + ks], dh[2], dl[2]); split_tf32(dG[1][4 + ks], dh[3], dl[3]);
                 // Eq. 9 (rows of V: a = 0..7 and 8..15) and W g' (Eq. 8 re-associated); cross terms first, the
                 // four independent accumulators interleaved
-                mma_tf32(V[0], al[0], al[1], al[2], al[3], Wh[ks][0], Wh[ks][1]);
-                mma_tf32(V[1], al[0], al[1], al[2], al[3], Wh[ks][2], Wh[ks][3]);
-                mma_tf32(T[0], dl[0], dl[1], dl[2], dl[3], Wh[ks][0], Wh[ks][1]);
-                mma_tf32(T[1], dl[0], dl[1], dl[2], dl[3], Wh[ks][2], Wh[ks][3]);
+                if (ks == 0) {
+                    mma_tf32_z(V[0], al[0], al[1], al[2], al[3], Wh[ks][0], Wh[ks][1]);
+                    mma_tf32_z(V[1], al[0], al[1], al[2], al[3], Wh[ks][2], Wh[ks][3]);
+                    mma_tf32_z(T[0], dl[0], dl[1], dl[2], dl[3], Wh[ks][0], Wh[ks][1]);
+                    mma_tf32_z(T[1], dl[0], dl[1], dl[2], dl[3], Wh[ks][2], Wh[ks][3]);
+                } else {
+                    mma_tf32(V[0], al[0], al[1], al[2], al[3], Wh[ks][0], Wh[ks][1]);
+                    mma_tf32(V[1], al[0], al[1], al[2], al[3], Wh[ks][2], Wh[ks][3]);
+                    mma_tf32(T[0], dl[0], dl[1], dl[2], dl[3], Wh[ks][0], Wh[ks][1]);
+                    mma_tf32(T[1], dl[0], dl[1], dl[2], dl[3], Wh[ks][2], Wh[ks][3]);
+                }
                 mma_tf32(V[0], ah[0], ah[1], ah[2], ah[3], Wl[ks][0], Wl[ks][1]);
                 mma_tf32(V[1], ah[0], ah[1], ah[2], ah[3], Wl[ks][2], Wl[ks][3]);
                 mma_tf32(T[0], dh[0], dh[1], dh[2], dh[3], Wl[ks][0], Wl[ks][1]);
@@ -474,6 +500,8 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
                 v[4 * q] = a.x; v[4 * q + 1] = a.y; v[4 * q + 2] = a.z; v[4 * q + 3] = a.w;
                 tt[4 * q] = b.x; tt[4 * q + 1] = b.y; tt[4 * q + 2] = b.z; tt[4 * q + 3] = b.w;
             }
+            const float4 ent = *reinterpret_cast<const float4 *>(vt + lane * VT_STRIDE + 32);
+            const float rinv = vt[lane * VT_STRIDE + 36];
             const float x = ent.x, y = ent.y, z = ent.z;
             const int j = __float_as_int(ent.w) & ((1 << J_BITS) - 1);
             const float ux = x * rinv, uy = y * rinv, uz = z * rinv;
@@ -484,9 +512,7 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
             const float qy = s * uy + (ty - tu * uy) * rinv;
             const float qz = s * uz + (tz - tu * uz) * rinv;
             fx += qx; fy += qy; fz += qz;
-            atomicAdd(&k.force[j].x, -qx);
-            atomicAdd(&k.force[j].y, -qy);
-            atomicAdd(&k.force[j].z, -qz);
+            atomicAdd(&k.force[j], make_float4(-qx, -qy, -qz, 0.f));   // one 128-bit reduction per pair
             vir[0] -= x * qx; vir[1] -= x * qy; vir[2] -= x * qz;
             vir[3] -= y * qx; vir[4] -= y * qy; vir[5] -= y * qz;
             vir[6] -= z * qx; vir[7] -= z * qy; vir[8] -= z * qz;
@@ -499,7 +525,7 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
     } else {
         int64_t cur = beg;
         do {
-            const int n = collect_pairs(k, pi, cur, end, pq, lane);
+            const int n = collect_pairs(k, pi, beg, cur, end, pq, lane, nullptr, 0);
             pc.mark(3);
             for (int q0 = 0; q0 < n; q0 += 32) batch(q0, min(32, n - q0));
         } while (cur < end);
@@ -511,9 +537,7 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
         fz += __shfl_xor_sync(0xffffffffu, fz, o);
     }
     if (lane == 0) {
-        atomicAdd(&k.force[i].x, fx);
-        atomicAdd(&k.force[i].y, fy);
-        atomicAdd(&k.force[i].z, fz);
+        atomicAdd(&k.force[i], make_float4(fx, fy, fz, 0.f));
     }
 }
 
@@ -531,10 +555,11 @@ __device__ __forceinline__ void head_load(float4 (&w)[8], const float4 *__restri
 #pragma unroll
     for (int q = 0; q < NKS; ++q) w[q] = __ldg(rec + (size_t)(ks0 + q) * 32 + lane);
 }
-template <int NKS>
+// FRESH: every k-step gets its own accumulator, folded in by a rounded add (energy path);
+// otherwise one accumulation chain (reverse pass: feeds forces only).
+template <int NKS, bool FRESH>
 __device__ __forceinline__ void head_gemm(float (&c)[4], const float4 (&w)[8], int ks0, const float *__restrict__ act, int bstride, int lane) {
     const int g = lane >> 2, t = lane & 3;
-    c[0] = c[1] = c[2] = c[3] = 0.f;
 #pragma unroll
     for (int q = 0; q < NKS; ++q) {
         uint32_t ah[4], al[4];
@@ -542,11 +567,18 @@ __device__ __forceinline__ void head_gemm(float (&c)[4], const float4 (&w)[8], i
         split_tf32(w[q].z, ah[2], al[2]); split_tf32(w[q].w, ah[3], al[3]);
         const float *r0 = act + g * bstride + 2 * (8 * (ks0 + q) + t);
         const float2 x0 = *reinterpret_cast<const float2 *>(r0), x1 = *reinterpret_cast<const float2 *>(r0 + 8);
-        float p[4] = {0.f, 0.f, 0.f, 0.f};
-        mma_tf32(p, al[0], al[1], al[2], al[3], __float_as_uint(x0.x), __float_as_uint(x1.x));
-        mma_tf32(p, ah[0], ah[1], ah[2], ah[3], __float_as_uint(x0.y), __float_as_uint(x1.y));
-        mma_tf32(p, ah[0], ah[1], ah[2], ah[3], __float_as_uint(x0.x), __float_as_uint(x1.x));
-        c[0] += p[0]; c[1] += p[1]; c[2] += p[2]; c[3] += p[3];
+        if (FRESH || q == 0) {
+            float p[4];
+            mma_tf32_z(p, al[0], al[1], al[2], al[3], __float_as_uint(x0.x), __float_as_uint(x1.x));
+            mma_tf32(p, ah[0], ah[1], ah[2], ah[3], __float_as_uint(x0.y), __float_as_uint(x1.y));
+            mma_tf32(p, ah[0], ah[1], ah[2], ah[3], __float_as_uint(x0.x), __float_as_uint(x1.x));
+            if (q == 0) { c[0] = p[0]; c[1] = p[1]; c[2] = p[2]; c[3] = p[3]; }
+            else { c[0] += p[0]; c[1] += p[1]; c[2] += p[2]; c[3] += p[3]; }
+        } else {
+            mma_tf32(c, al[0], al[1], al[2], al[3], __float_as_uint(x0.x), __float_as_uint(x1.x));
+            mma_tf32(c, ah[0], ah[1], ah[2], ah[3], __float_as_uint(x0.y), __float_as_uint(x1.y));
+            mma_tf32(c, ah[0], ah[1], ah[2], ah[3], __float_as_uint(x0.x), __float_as_uint(x1.x));
+        }
     }
 }
 
@@ -557,11 +589,52 @@ __device__ __forceinline__ void store_partial(const float (&c)[4], float *part, 
     p[0] = c[0]; p[pstride] = c[1]; p[8] = c[2]; p[pstride + 8] = c[3];
 }
 
+// Prefetch of the warp's atom in the group's NEXT tile, spread over three points of the head so
+// that each dependent global load has a barrier's worth of time to arrive: centre index -> list
+// bounds -> the first PF_IDX neighbor indices (cp.async straight into shared memory).
+struct NextAtom {
+    const KernelArgs *k;
+    int *meta;        // shared: {atom, list start lo, list start hi, list length}
+    int *sidx;        // shared: neighbor indices
+    int slot;         // position in center_order, or -1
+    int i;
+    int64_t beg, end;
+    __device__ __forceinline__ void stage_a() { if (slot >= 0) i = __ldg(k->center_order + slot); }
+    __device__ __forceinline__ void stage_b() { if (slot >= 0) { beg = __ldg(k->nbr_off + i); end = __ldg(k->nbr_off + i + 1); } }
+    __device__ __forceinline__ void stage_c(int lane) {
+        if (slot < 0) return;
+        const int n = (int)min((int64_t)PF_IDX, end - beg);
+#pragma unroll
+        for (int c = 0; c < PF_IDX / 32; ++c) {
+            const int e = 32 * c + lane;
+            if (e < n) {
+                const unsigned dst = (unsigned)__cvta_generic_to_shared(sidx + e);
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(k->nbr + beg + e) : "memory");
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        if (lane == 0) { meta[0] = i; meta[1] = (int)(beg & 0xffffffff); meta[2] = (int)(beg >> 32); meta[3] = (int)(end - beg); }
+    }
+    // once the indices have landed: pull the neighbors' positions (and the atom's own) into L2
+    __device__ __forceinline__ void stage_d(int lane) {
+        if (slot < 0) return;
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncwarp();
+        const int n = (int)min((int64_t)PF_IDX, end - beg);
+#pragma unroll
+        for (int c = 0; c < PF_IDX / 32; ++c) {
+            const int e = 32 * c + lane;
+            if (e < n) asm volatile("prefetch.global.L2 [%0];" ::"l"(k->pos4 + sidx[e]));
+        }
+        if (lane == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(k->pos4 + i));
+    }
+};
+
 // ---------------- Regression (Eq. 6) forward and reverse for the group's tile ----------------
 // In: sX = invariants [atom][128].  Out: sX = dE/dG; per-atom energies written.
 // hc = biases [4][64], w_out [64], b_out of the species in shared memory.  wg = warp within the group.
 __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float *hb, const float *hc, int species, int count, int first,
-                                          int group, int wg, int lane, double &e_sum, PhaseClock &pc) {
+                                          int group, int wg, int lane, double &e_sum, NextAtom &nx, PhaseClock &pc) {
     const float *hp = k.head_pack + (size_t)species * HP_TOTAL;
     const float4 *fwd = reinterpret_cast<const float4 *>(hp + HP_FWD), *bwd = reinterpret_cast<const float4 *>(hp + HP_BWD);
     float *xs = hb + HB_XS, *zs = hb + HB_ZS, *sD = hb + HB_SD, *dz = hb + HB_DZ, *dp = hb + HB_DP, *part = hb + HB_PART;
@@ -573,6 +646,7 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
     // split the invariants once
     for (int f = lane; f < N_INV; f += 32)
         *reinterpret_cast<float2 *>(xs + atom * 2 * X_STRIDE + 2 * f) = split_pair(sX[atom * X_STRIDE + f]);
+    nx.stage_a();
     pc.mark(3);
     group_sync(group);
     pc.mark(14);
@@ -583,13 +657,16 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
         const float *zin = zs + ((L + 1) & 1) * TILE * 2 * Z_STRIDE;
         float *zout = zs + (L & 1) * TILE * 2 * Z_STRIDE;
         float c[4];
-        if (L == 0) head_gemm<KS0 / 2>(c, w, kh * (KS0 / 2), xs, 2 * X_STRIDE, lane);
-        else head_gemm<KS1 / 2>(c, w, kh * (KS1 / 2), zin, 2 * Z_STRIDE, lane);
+        if (L == 0) head_gemm<KS0 / 2, true>(c, w, kh * (KS0 / 2), xs, 2 * X_STRIDE, lane);
+        else head_gemm<KS1 / 2, true>(c, w, kh * (KS1 / 2), zin, 2 * Z_STRIDE, lane);
         pc.mark(12);
         store_partial(c, part + kh * TILE * Z_STRIDE, Z_STRIDE, mt4, lane);
         // weights of the next pass
         if (L < HEAD_L - 1) head_load<KS1 / 2>(w, fwd + (size_t)(4 * KS0 + L * 4 * KS1 + mt4 * KS1) * 32, kh * (KS1 / 2), lane);
         else head_load<4>(w, bwd + (size_t)((N_INV / 16) * 8 + (HEAD_L - 2) * 32 + mt4 * 8) * 32, kh * 4, lane);
+        if (L == 0) nx.stage_b();
+        if (L == 1) nx.stage_c(lane);
+        if (L == 3) nx.stage_d(lane);
         pc.mark(13);
         group_sync(group);
         pc.mark(14);
@@ -627,7 +704,7 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
 #pragma unroll
     for (int L = HEAD_L - 1; L >= 1; --L) {
         float c[4];
-        head_gemm<4>(c, w, kh * 4, dp, 2 * Z_STRIDE, lane);
+        head_gemm<4, false>(c, w, kh * 4, dp, 2 * Z_STRIDE, lane);
         store_partial(c, part + kh * TILE * Z_STRIDE, Z_STRIDE, mt4, lane);
         if (L > 1) head_load<4>(w, bwd + (size_t)((N_INV / 16) * 8 + (L - 2) * 32 + mt4 * 8) * 32, kh * 4, lane);
         else head_load<8>(w, bwd + (size_t)(wg * 8) * 32, 0, lane);   // first layer: warp = m-tile, all 8 k-steps
@@ -644,7 +721,7 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
     }
     {   // first layer: dE/dG [128 x 8], warp = m-tile (16 inputs), written over the invariants
         float c[4];
-        head_gemm<8>(c, w, 0, dp, 2 * Z_STRIDE, lane);
+        head_gemm<8, false>(c, w, 0, dp, 2 * Z_STRIDE, lane);
         store_partial(c, sX, X_STRIDE, wg, lane);
     }
     group_sync(group);
@@ -662,7 +739,8 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
     float *hb = scr_all + group * TILE * SCR_WORDS;        // head buffers = the scratch of the group's warps
     float *scr = scr_all + warp * SCR_WORDS;
     float4 *pq = reinterpret_cast<float4 *>(scr_all + NW * SCR_WORDS + warp * Q_WORDS);
-    float *hc = scr_all + NW * (SCR_WORDS + Q_WORDS);
+    int *pf = reinterpret_cast<int *>(scr_all + NW * (SCR_WORDS + Q_WORDS)) + warp * PF_WORDS;
+    float *hc = scr_all + NW * (SCR_WORDS + Q_WORDS + PF_WORDS);
     int *ctl = reinterpret_cast<int *>(hc + HC_WORDS);
     const int rows = k.tab.knots + 3;
 
@@ -692,28 +770,44 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
             hc[idx] = __ldg(k.head_pack + (size_t)species * HP_TOTAL + HP_BIAS + idx);
         __syncthreads();
 
-        while (true) {   // the group's tiles of this species
+        bool prefetched = false;   // this warp's atom of the coming tile sits in the prefetch buffer
+        int look_ahead = -1;       // (group leader) the tile after the current one
+        while (true) {   // the group's tiles of this species, claimed one ahead
             group_sync(group);
-            if (wg == 0 && lane == 0) ctl[group] = atomicAdd(k.tile_counter + species, 1);
+            if (wg == 0 && lane == 0) {
+                ctl[2 * group] = look_ahead >= 0 ? look_ahead : atomicAdd(k.tile_counter + species, 1);
+                look_ahead = atomicAdd(k.tile_counter + species, 1);
+                ctl[2 * group + 1] = look_ahead;
+            }
             group_sync(group);
             pc.mark(11);
-            const int tile = ctl[group];
+            const int tile = ctl[2 * group], tile_next = ctl[2 * group + 1];
             if (tile >= n_tiles) break;
             const int first = s_beg + tile * TILE;
             const int count = min(TILE, s_end - first);
 
             // ---------------- Encoding + invariants: warp = atom ----------------
             const bool have = wg < count;
-            const int i = have ? __ldg(k.center_order + first + wg) : 0;
+            int i = 0, n_pref = 0;
             double4 pi = make_double4(0.0, 0.0, 0.0, 0.0);
             int64_t beg = 0, end = 0;
             float Pf[4][4];
             int queued = -1;
             float *xrow = sX + wg * X_STRIDE;
             if (have) {
-                pi = k.pos4[i];
-                beg = k.nbr_off[i]; end = k.nbr_off[i + 1];
-                n_pairs += encode_atom(k, tv, pi, beg, end, pq, scr, lane, Pf, queued, pc);
+                if (prefetched) {
+                    asm volatile("cp.async.wait_group 0;" ::: "memory");
+                    __syncwarp();
+                    i = pf[PF_IDX];
+                    beg = ((int64_t)pf[PF_IDX + 2] << 32) | (unsigned)pf[PF_IDX + 1];
+                    end = beg + pf[PF_IDX + 3];
+                    n_pref = min(PF_IDX, pf[PF_IDX + 3]);
+                } else {
+                    i = __ldg(k.center_order + first + wg);
+                    beg = k.nbr_off[i]; end = k.nbr_off[i + 1];
+                }
+                pi = load_pos4(k.pos4 + i);
+                n_pairs += encode_atom(k, tv, pi, beg, end, pq, scr, lane, Pf, queued, pf, n_pref, pc);
                 // Eq. 5 (C_l = I): this lane holds rows a = g, g + 8 of channels 8t + j; sum squares over the rows of a block
                 float part[4][8];
 #pragma unroll
@@ -744,8 +838,13 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
             group_sync(group);
             pc.mark(8);
 
-            // ---------------- Regression ----------------
-            head_tile(k, sX, hb, hc, species, count, first, group, wg, lane, e_sum, pc);
+            // ---------------- Regression (and the prefetch for the next tile) ----------------
+            NextAtom nx;
+            nx.k = &k; nx.sidx = pf; nx.meta = pf + PF_IDX;
+            nx.slot = (tile_next < n_tiles && s_beg + tile_next * TILE + wg < s_end) ? s_beg + tile_next * TILE + wg : -1;
+            nx.i = 0; nx.beg = 0; nx.end = 0;
+            head_tile(k, sX, hb, hc, species, count, first, group, wg, lane, e_sum, nx, pc);
+            prefetched = nx.slot >= 0;
             pc.mark(9);
 
             // ---------------- Derivation ----------------
