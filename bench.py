@@ -42,8 +42,9 @@ FLOP_PER_ATOM = 88700.0        # invariants, W_i, head forward + reverse, SiLU
 FP32_LANES_PER_SM = 128
 
 # DRAM traffic of one fused-kernel launch from the committed ncu capture
-# (profiles/k_mega_hea6.md: dram__bytes_read.sum + dram__bytes_write.sum, bytes per atom, scaled by atoms).
-NCU_DRAM_BYTES_PER_ATOM = None
+# (profiles/k_mega_hea6_fcc50.md: dram__bytes_read.sum + dram__bytes_write.sum of a 500,000-atom launch, per atom;
+# the traffic is per-atom, so a launch of N atoms is reported as this figure times N).
+NCU_DRAM_BYTES_PER_ATOM = 761.0
 
 
 def parse_args():
@@ -56,6 +57,8 @@ def parse_args():
     ap.add_argument("--cpu-centers", type=int, default=49152, help="central atoms in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sweep", default="", help="comma-separated FCC cell counts: size sweep of the 6-species workload "
+                    "(inputs generated on the device), one JSON line per size; not the contract line")
     return ap.parse_args()
 
 
@@ -179,8 +182,74 @@ def run_reference(args, rank, world):
     print(json.dumps(line), flush=True)
 
 
+def run_sweep(args):
+    """Throughput and footprint versus system size up to what fits in HBM (the paper's Fig. 4(b) analogue).
+    Lattice, displacements, species and velocities are drawn on the device with a seeded torch generator."""
+    import torch
+    import paper_2608_16329_b200 as mlip
+    from paper_2608_16329_b200 import workloads as wl
+    dev = torch.device("cuda", 0)
+    enc, head = wl.workload_weights(CFG, 6)
+    masses = np.array(wl.MASSES[CFG])
+    for cells in [int(x) for x in args.sweep.split(",") if x]:
+        n = 4 * cells ** 3
+        line = {"sweep": True, "cells": cells, "atoms": n}
+        pot = None
+        try:
+            gen = torch.Generator(device=dev)
+            gen.manual_seed(wl.BASE_SEED + cells)
+            a = 3.6
+            idx = torch.arange(n, device=dev, dtype=torch.int64)
+            basis = torch.tensor(wl._FCC_BASIS, device=dev, dtype=torch.float64)[idx % 4]
+            cell = torch.div(idx, 4, rounding_mode="floor")
+            pos = torch.stack([torch.div(cell, cells * cells, rounding_mode="floor"), torch.div(cell, cells, rounding_mode="floor") % cells,
+                               cell % cells], dim=1).to(torch.float64)
+            del idx, cell
+            pos = (pos + basis) * a
+            del basis
+            pos += 0.05 * torch.randn(pos.shape, generator=gen, device=dev, dtype=torch.float64)
+            box = np.full(3, cells * a)
+            pos -= torch.floor(pos / (cells * a)) * (cells * a)
+            pos.clamp_(0.0, float(np.nextafter(cells * a, 0.0)))
+            species = torch.randint(0, 6, (n,), generator=gen, device=dev, dtype=torch.int32)
+            pot = mlip.Potential(6, 6.0, 1.0, enc, head, masses)
+            pot.n = n
+            mlip.mlip_build_neighbors(pot.ctx, pos, species, box)
+            sig = torch.sqrt(torch.tensor(wl.KB_EV_PER_K * 300.0 * wl.ACC_UNIT / masses, device=dev))[species.long()]
+            vel = torch.randn(pos.shape, generator=gen, device=dev, dtype=torch.float64) * sig[:, None]
+            mlip.mlip_set_velocities(pot.ctx, vel)
+            del pos, species, vel, sig
+            torch.cuda.empty_cache()
+            pot.step(args.warmup, DT_FS, REBUILD_EVERY)
+            torch.cuda.synchronize()
+            mlip.mlip_kernel_time(pot.ctx, reset=True)
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record()
+            pot.step(args.steps, DT_FS, REBUILD_EVERY)
+            ev1.record()
+            torch.cuda.synchronize()
+            ms = ev0.elapsed_time(ev1)
+            k_n, k_ms = mlip.mlip_kernel_time(pot.ctx)
+            status = pot.sync_status(raise_on_error=False)
+            line.update({"atom_steps_per_s": n * args.steps / (ms * 1e-3), "ms_per_step": ms / args.steps,
+                         "kernel_ms": k_ms / max(k_n, 1), "resident_GB": mlip.mlip_resident_bytes(pot.ctx) / 1e9,
+                         "resident_bytes_per_atom": mlip.mlip_resident_bytes(pot.ctx) / n,
+                         "status": mlip.binding.ERRORS.get(status, status)})
+        except Exception as exc:   # out of memory ends the sweep
+            line["error"] = str(exc)[:200]
+        print(json.dumps(line), flush=True)
+        if pot is not None:
+            pot.close()
+        torch.cuda.empty_cache()
+        if "error" in line:
+            break
+
+
 def main():
     args = parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
