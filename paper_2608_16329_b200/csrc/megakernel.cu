@@ -335,10 +335,15 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
             split_tf32(ra[g + 8], ah[1], al[1]);
             split_tf32(rb[g], ah[2], al[2]);
             split_tf32(rb[g + 8], ah[3], al[3]);
-            // B = G (8 pairs x 8 channels per n-tile): this lane evaluates channels 4g .. 4g+3 (one per n-tile)
-            const float4 ba = *reinterpret_cast<const float4 *>(ra + 16), bb = *reinterpret_cast<const float4 *>(rb + 16);
-            const float *ta = tv.base + reinterpret_cast<const int *>(ra)[20] + 4 * g;
-            const float *tb = tv.base + reinterpret_cast<const int *>(rb)[20] + 4 * g;
+            // B = G (8 pairs x 8 channels per n-tile).  Evaluation pattern: quarter-warp q reads the table
+            // rows of ONE pair (8 lanes x 16 bytes = a full row per access: no bank conflicts), i.e. lane
+            // (q, c) evaluates channels 4c .. 4c+3 of pairs q and q + 4 of this k-step; a fixed shuffle
+            // then hands the values to the lane that owns them in the B fragment (pair t, channels 4g .. 4g+3).
+            const int q = lane >> 3, cch = lane & 7;
+            const float *qa = stage + (8 * ks + q) * ST_STRIDE, *qb = qa + 4 * ST_STRIDE;
+            const float4 ba = *reinterpret_cast<const float4 *>(qa + 16), bb = *reinterpret_cast<const float4 *>(qb + 16);
+            const float *ta = tv.base + reinterpret_cast<const int *>(qa)[20] + 4 * cch;
+            const float *tb = tv.base + reinterpret_cast<const int *>(qb)[20] + 4 * cch;
             const float4 a0 = *reinterpret_cast<const float4 *>(ta), a1 = *reinterpret_cast<const float4 *>(ta + rs);
             const float4 a2 = *reinterpret_cast<const float4 *>(ta + 2 * rs), a3 = *reinterpret_cast<const float4 *>(ta + 3 * rs);
             const float4 b0 = *reinterpret_cast<const float4 *>(tb), b1 = *reinterpret_cast<const float4 *>(tb + rs);
@@ -352,6 +357,12 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
             gb[1] = bb.x * b0.y + bb.y * b1.y + bb.z * b2.y + bb.w * b3.y;
             gb[2] = bb.x * b0.z + bb.y * b1.z + bb.z * b2.z + bb.w * b3.z;
             gb[3] = bb.x * b0.w + bb.y * b1.w + bb.z * b2.w + bb.w * b3.w;
+            const int owner_src = 8 * t + g;   // lane (g, t) takes (pair t, chunk g) from lane (q = t, c = g)
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                ga[nt] = __shfl_sync(0xffffffffu, ga[nt], owner_src);
+                gb[nt] = __shfl_sync(0xffffffffu, gb[nt], owner_src);
+            }
             // Eq. 4 for eight pairs; the three terms of each n-tile are issued interleaved over the n-tiles
             uint32_t bh[4][2], bl[4][2];
             float c[4][4];
