@@ -48,8 +48,6 @@ struct TableDesc {
     float r_cut2;
 };
 
-struct Buffers;  // defined in api.cu
-
 }  // namespace mlip
 
 struct mlip_ctx {
@@ -58,10 +56,9 @@ struct mlip_ctx {
     int n_sm = 0;
 
     // model
-    float *head_w = nullptr;     // [C][HEAD_NET] fp32, layout see megakernel.cu
+    float *head_w = nullptr;     // per-species head weights packed in MMA fragment order (megakernel.cu)
     float *table = nullptr;      // spline coefficients
     double *mass = nullptr;      // [C] dev
-    float *inv_mass_acc = nullptr; // unused placeholder
     double table_err_value = 0, table_err_deriv = 0;
     mlip::TableDesc tab{};
 
@@ -76,7 +73,6 @@ struct mlip_ctx {
     float *e_atom = nullptr;       // E_i, internal order
     float *disp = nullptr;         // [N][3] displacement since the last build
     int32_t *center_order = nullptr;  // internal indices sorted by (species, cell)
-    int32_t species_start_host[mlip::MAX_SPECIES + 1] = {0};
     // second set used as the source of a rebuild
     double4 *pos4_src = nullptr;
     double *vel_src = nullptr;
@@ -97,7 +93,7 @@ struct mlip_ctx {
     double *acc = nullptr;         // [ACC_COUNT]
     unsigned long long *pair_counter = nullptr;
     int *status = nullptr;         // device status word
-    int *tile_counter = nullptr;   // dynamic tile scheduler
+    int *tile_counter = nullptr;   // [MAX_SPECIES] dynamic tile scheduler, one counter per central species
     int *status_host = nullptr;    // pinned
     int64_t *total_host = nullptr; // pinned
     double *stage_pos = nullptr;   // [N][3] staging for host entry point

@@ -205,3 +205,41 @@ def test_nve_with_rebuilds_conserves_energy_on_multicomponent_workloads(cfg, n_c
     p = pos.cpu().numpy()
     nl = oracle.neighbors(p, w.species, w.n_species, w.box, w.r_cut + w.skin)
     assert step == steps and canonical_equal(nl, seg, nbr)
+
+
+def test_tables_in_global_memory_path_matches_oracle():
+    """With 256 knots the six tables of a central species no longer fit in shared memory: the kernel's fallback
+    instantiation reads them from global memory."""
+    w, model, pot = make_pair(1, 4, 0.0, table_knots=256)
+    pot.build_neighbors(w.pos, w.species, w.box)
+    out = pot.compute()
+    pot.sync_status()
+    ref = oracle.evaluate(model, w.pos, w.species, w.box)
+    assert abs(float(out["energy"].cpu()) - ref["energy"]) <= E_RTOL * abs(ref["energy"])
+    assert np.abs(out["forces"].cpu().numpy() - ref["forces"]).max() <= F_ATOL
+
+
+def test_dense_system_beyond_the_pair_queue_matches_oracle():
+    """A compressed lattice with ~165 neighbors inside the cutoff: more than the 160-entry pair queue, so the
+    encoding runs in several rounds and the derivation re-scans the list."""
+    import paper_2608_16329_b200 as mlip
+    from paper_2608_16329_b200 import workloads as wl
+    rng = np.random.default_rng(21)
+    a, n = 2.8, 6
+    box = np.full(3, a * n)
+    pos = wl.lattice_sites((n, n, n), a, wl._FCC_BASIS) + rng.normal(0.0, 0.03, (4 * n ** 3, 3))
+    pos -= np.floor(pos / box) * box
+    species = rng.integers(0, 2, len(pos)).astype(np.int32)
+    enc, head = wl.make_weights(2, seed=77, enc_out_scale=0.05, head_out_scale=0.3)
+    model = oracle.Model(2, 6.0, enc, head)
+    pot = mlip.Potential(2, 6.0, 1.0, enc, head, np.array([50.0, 60.0]))
+    pot.build_neighbors(pos, species, box)
+    out = pot.compute(want_e_atom=True)
+    pot.sync_status()
+    c = mlip.mlip_get_counters(pot.ctx)
+    assert c["pairs_in_cutoff"] / len(pos) > 160
+    ref = oracle.evaluate(model, pos, species, box)
+    scale = max(1.0, float(np.sqrt((ref["forces"] ** 2).sum(1).mean())))
+    assert abs(float(out["energy"].cpu()) - ref["energy"]) <= E_RTOL * abs(ref["energy"])
+    assert np.abs(out["forces"].cpu().numpy() - ref["forces"]).max() <= F_ATOL * scale
+    assert np.abs(out["e_atom"].cpu().numpy() - ref["e_atom"]).max() <= 2e-5 * max(1.0, np.abs(ref["e_atom"]).max())
