@@ -681,22 +681,28 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
         pc.mark(13);
         group_sync(group);
         pc.mark(14);
-        // elementwise: bias, SiLU, residual; this thread owns neurons lane and lane + 32 of its atom
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {
-            const int nn = lane + 32 * q;
-            const float *pp = part + atom * Z_STRIDE + nn;
-            const float pre = (pp[0] + pp[TILE * Z_STRIDE]) + hc[L * HEAD_H + nn];
-            float d, y = silu_f(pre, d);
-            if (L > 0) { const float2 zi = *reinterpret_cast<const float2 *>(zin + atom * 2 * Z_STRIDE + 2 * nn); y += zi.x + zi.y; }
-            sD[(L * TILE + atom) * Z_STRIDE + nn] = d;
+        // elementwise: bias, SiLU, residual; this thread owns neurons 2 lane, 2 lane + 1 of its atom
+        {
+            const int n0 = 2 * lane;
+            const float2 p0 = *reinterpret_cast<const float2 *>(part + atom * Z_STRIDE + n0);
+            const float2 p1 = *reinterpret_cast<const float2 *>(part + (TILE + atom) * Z_STRIDE + n0);
+            const float2 bb = *reinterpret_cast<const float2 *>(hc + L * HEAD_H + n0);
+            float d0, d1;
+            float y0 = silu_f((p0.x + p1.x) + bb.x, d0), y1 = silu_f((p0.y + p1.y) + bb.y, d1);
+            if (L > 0) {
+                const float4 zi = *reinterpret_cast<const float4 *>(zin + atom * 2 * Z_STRIDE + 2 * n0);
+                y0 += zi.x + zi.y; y1 += zi.z + zi.w;
+            }
+            *reinterpret_cast<float2 *>(sD + (L * TILE + atom) * Z_STRIDE + n0) = make_float2(d0, d1);
             if (L < HEAD_L - 1) {
-                *reinterpret_cast<float2 *>(zout + atom * 2 * Z_STRIDE + 2 * nn) = split_pair(y);
+                const float2 s0 = split_pair(y0), s1 = split_pair(y1);
+                *reinterpret_cast<float4 *>(zout + atom * 2 * Z_STRIDE + 2 * n0) = make_float4(s0.x, s0.y, s1.x, s1.y);
             } else {   // output layer and the start of the reverse pass: dE/dz = w_out
-                const float wo = hc[HEAD_L * HEAD_H + nn];
-                e_i += wo * y;
-                dz[atom * Z_STRIDE + nn] = wo;
-                *reinterpret_cast<float2 *>(dp + atom * 2 * Z_STRIDE + 2 * nn) = split_pair(wo * d);
+                const float2 wo = *reinterpret_cast<const float2 *>(hc + HEAD_L * HEAD_H + n0);
+                e_i += wo.x * y0 + wo.y * y1;
+                *reinterpret_cast<float2 *>(dz + atom * Z_STRIDE + n0) = wo;
+                const float2 s0 = split_pair(wo.x * d0), s1 = split_pair(wo.y * d1);
+                *reinterpret_cast<float4 *>(dp + atom * 2 * Z_STRIDE + 2 * n0) = make_float4(s0.x, s0.y, s1.x, s1.y);
             }
         }
         pc.mark(15);
@@ -720,13 +726,16 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
         if (L > 1) head_load<4>(w, bwd + (size_t)((N_INV / 16) * 8 + (L - 2) * 32 + mt4 * 8) * 32, kh * 4, lane);
         else head_load<8>(w, bwd + (size_t)(wg * 8) * 32, 0, lane);   // first layer: warp = m-tile, all 8 k-steps
         group_sync(group);
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {
-            const int nn = lane + 32 * q;
-            const float *pp = part + atom * Z_STRIDE + nn;
-            const float dzn = dz[atom * Z_STRIDE + nn] + (pp[0] + pp[TILE * Z_STRIDE]);
-            dz[atom * Z_STRIDE + nn] = dzn;
-            *reinterpret_cast<float2 *>(dp + atom * 2 * Z_STRIDE + 2 * nn) = split_pair(dzn * sD[((L - 1) * TILE + atom) * Z_STRIDE + nn]);
+        {
+            const int n0 = 2 * lane;
+            const float2 p0 = *reinterpret_cast<const float2 *>(part + atom * Z_STRIDE + n0);
+            const float2 p1 = *reinterpret_cast<const float2 *>(part + (TILE + atom) * Z_STRIDE + n0);
+            float2 dzn = *reinterpret_cast<const float2 *>(dz + atom * Z_STRIDE + n0);
+            dzn.x += p0.x + p1.x; dzn.y += p0.y + p1.y;
+            *reinterpret_cast<float2 *>(dz + atom * Z_STRIDE + n0) = dzn;
+            const float2 da = *reinterpret_cast<const float2 *>(sD + ((L - 1) * TILE + atom) * Z_STRIDE + n0);
+            const float2 s0 = split_pair(dzn.x * da.x), s1 = split_pair(dzn.y * da.y);
+            *reinterpret_cast<float4 *>(dp + atom * 2 * Z_STRIDE + 2 * n0) = make_float4(s0.x, s0.y, s1.x, s1.y);
         }
         group_sync(group);
     }
