@@ -286,8 +286,12 @@ def main():
     barrier()
     mlip.mlip_kernel_time(pot.ctx, reset=True)
     launches0 = mlip.mlip_get_counters(pot.ctx)["launches"]
-    sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
-                           int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
+    gpu_index = local_rank
+    try:   # nvidia-smi numbers physical devices; honour a numeric CUDA_VISIBLE_DEVICES mapping
+        gpu_index = int(os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",")[local_rank])
+    except (ValueError, IndexError):
+        pass
+    sampler = ClockSampler(gpu_index)
     if rank == 0:
         sampler.start()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

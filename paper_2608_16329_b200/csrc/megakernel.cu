@@ -570,27 +570,38 @@ __device__ __forceinline__ void head_load(float4 (&w)[8], const float4 *__restri
 // otherwise one accumulation chain (reverse pass: feeds forces only).
 template <int NKS, bool FRESH>
 __device__ __forceinline__ void head_gemm(float (&c)[4], const float4 (&w)[8], int ks0, const float *__restrict__ act, int bstride, int lane) {
+    static_assert(NKS % 2 == 0, "k-steps are processed two at a time (two independent MMA chains in flight)");
     const int g = lane >> 2, t = lane & 3;
+    float ce[4], co[4];   // FRESH: per-k-step products; otherwise the even / odd accumulation chains
 #pragma unroll
-    for (int q = 0; q < NKS; ++q) {
-        uint32_t ah[4], al[4];
-        split_tf32(w[q].x, ah[0], al[0]); split_tf32(w[q].y, ah[1], al[1]);
-        split_tf32(w[q].z, ah[2], al[2]); split_tf32(w[q].w, ah[3], al[3]);
-        const float *r0 = act + g * bstride + 2 * (8 * (ks0 + q) + t);
-        const float2 x0 = *reinterpret_cast<const float2 *>(r0), x1 = *reinterpret_cast<const float2 *>(r0 + 8);
+    for (int q = 0; q < NKS; q += 2) {
+        uint32_t ah[2][4], al[2][4];
+        float2 x0[2], x1[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            split_tf32(w[q + u].x, ah[u][0], al[u][0]); split_tf32(w[q + u].y, ah[u][1], al[u][1]);
+            split_tf32(w[q + u].z, ah[u][2], al[u][2]); split_tf32(w[q + u].w, ah[u][3], al[u][3]);
+            const float *r0 = act + g * bstride + 2 * (8 * (ks0 + q + u) + t);
+            x0[u] = *reinterpret_cast<const float2 *>(r0);
+            x1[u] = *reinterpret_cast<const float2 *>(r0 + 8);
+        }
         if (FRESH || q == 0) {
-            float p[4];
-            mma_tf32_z(p, al[0], al[1], al[2], al[3], __float_as_uint(x0.x), __float_as_uint(x1.x));
-            mma_tf32(p, ah[0], ah[1], ah[2], ah[3], __float_as_uint(x0.y), __float_as_uint(x1.y));
-            mma_tf32(p, ah[0], ah[1], ah[2], ah[3], __float_as_uint(x0.x), __float_as_uint(x1.x));
-            if (q == 0) { c[0] = p[0]; c[1] = p[1]; c[2] = p[2]; c[3] = p[3]; }
-            else { c[0] += p[0]; c[1] += p[1]; c[2] += p[2]; c[3] += p[3]; }
+            mma_tf32_z(ce, al[0][0], al[0][1], al[0][2], al[0][3], __float_as_uint(x0[0].x), __float_as_uint(x1[0].x));
+            mma_tf32_z(co, al[1][0], al[1][1], al[1][2], al[1][3], __float_as_uint(x0[1].x), __float_as_uint(x1[1].x));
         } else {
-            mma_tf32(c, al[0], al[1], al[2], al[3], __float_as_uint(x0.x), __float_as_uint(x1.x));
-            mma_tf32(c, ah[0], ah[1], ah[2], ah[3], __float_as_uint(x0.y), __float_as_uint(x1.y));
-            mma_tf32(c, ah[0], ah[1], ah[2], ah[3], __float_as_uint(x0.x), __float_as_uint(x1.x));
+            mma_tf32(ce, al[0][0], al[0][1], al[0][2], al[0][3], __float_as_uint(x0[0].x), __float_as_uint(x1[0].x));
+            mma_tf32(co, al[1][0], al[1][1], al[1][2], al[1][3], __float_as_uint(x0[1].x), __float_as_uint(x1[1].x));
+        }
+        mma_tf32(ce, ah[0][0], ah[0][1], ah[0][2], ah[0][3], __float_as_uint(x0[0].y), __float_as_uint(x1[0].y));
+        mma_tf32(co, ah[1][0], ah[1][1], ah[1][2], ah[1][3], __float_as_uint(x0[1].y), __float_as_uint(x1[1].y));
+        mma_tf32(ce, ah[0][0], ah[0][1], ah[0][2], ah[0][3], __float_as_uint(x0[0].x), __float_as_uint(x1[0].x));
+        mma_tf32(co, ah[1][0], ah[1][1], ah[1][2], ah[1][3], __float_as_uint(x0[1].x), __float_as_uint(x1[1].x));
+        if (FRESH) {
+            if (q == 0) { c[0] = ce[0] + co[0]; c[1] = ce[1] + co[1]; c[2] = ce[2] + co[2]; c[3] = ce[3] + co[3]; }
+            else { c[0] += ce[0] + co[0]; c[1] += ce[1] + co[1]; c[2] += ce[2] + co[2]; c[3] += ce[3] + co[3]; }
         }
     }
+    if (!FRESH) { c[0] = ce[0] + co[0]; c[1] = ce[1] + co[1]; c[2] = ce[2] + co[2]; c[3] = ce[3] + co[3]; }
 }
 
 // c fragment (rows = 16 m + g, g + 8; columns = atoms 2t, 2t + 1) -> part[atom][row] with `pstride` floats per atom
@@ -796,12 +807,11 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
             group_sync(group);
             if (wg == 0 && lane == 0) {
                 ctl[2 * group] = look_ahead >= 0 ? look_ahead : atomicAdd(k.tile_counter + species, 1);
-                look_ahead = atomicAdd(k.tile_counter + species, 1);
-                ctl[2 * group + 1] = look_ahead;
+                look_ahead = atomicAdd(k.tile_counter + species, 1);   // consumed after the encoding: its latency is hidden
             }
             group_sync(group);
             pc.mark(11);
-            const int tile = ctl[2 * group], tile_next = ctl[2 * group + 1];
+            const int tile = ctl[2 * group];
             if (tile >= n_tiles) break;
             const int first = s_beg + tile * TILE;
             const int count = min(TILE, s_end - first);
@@ -854,9 +864,11 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
             } else {   // empty slot of a ragged tile: feed zeros to the head
                 for (int c = lane; c < N_INV; c += 32) xrow[c] = 0.f;
             }
+            if (wg == 0 && lane == 0) ctl[2 * group + 1] = look_ahead;
             pc.mark(7);
             group_sync(group);
             pc.mark(8);
+            const int tile_next = ctl[2 * group + 1];
 
             // ---------------- Regression (and the prefetch for the next tile) ----------------
             NextAtom nx;
