@@ -40,6 +40,7 @@ FLOP_PER_PAIR = 3960.0         # pair inside r_cut: both neighbor loops (geometr
 FLOP_PER_SKIN_ENTRY = 24.0     # list entry between r_cut and r_cut + skin: distance test in both loops
 FLOP_PER_ATOM = 88700.0        # invariants, W_i, head forward + reverse, SiLU
 FP32_LANES_PER_SM = 128
+FP64_LANES_PER_SM = 64         # fp64 path: DFMA lanes per SM
 
 # DRAM traffic of one fused-kernel launch from the committed ncu capture
 # (profiles/k_mega_hea6_fcc50.md: dram__bytes_read.sum + dram__bytes_write.sum of a 500,000-atom launch, per atom;
@@ -60,6 +61,8 @@ def parse_args():
     ap.add_argument("--cfg", type=int, default=CFG, choices=[2, 3, 4, 5],
                     help="workload: 5 = the 6-species alloy the metric is quoted on (default); 2, 3, 4 = the unary, "
                          "3-species alloy and ionic stand-ins at their full sizes (extra data points, not the contract line)")
+    ap.add_argument("--precision", default="f32", choices=["f32", "f64"],
+                    help="f64 runs the double-precision evaluation path instead (an extra data point, not the contract line)")
     ap.add_argument("--sweep", default="", help="comma-separated FCC cell counts: size sweep of the 6-species workload "
                     "(inputs generated on the device), one JSON line per size; not the contract line")
     return ap.parse_args()
@@ -280,7 +283,8 @@ def main():
     enc, head = wl.workload_weights(cfg, w.n_species)
     rebuild_every = REBUILD_EVERY if cfg != 4 else 3   # the ionic stand-in is far from equilibrium under random weights
     n = w.n_atoms
-    pot = mlip.Potential(w.n_species, w.r_cut, w.skin, enc, head, w.masses, device=local_rank)
+    f64 = args.precision == "f64"
+    pot = mlip.Potential(w.n_species, w.r_cut, w.skin, enc, head, w.masses, device=local_rank, precision=1 if f64 else 0)
     table_err = mlip.mlip_table_error(pot.ctx)
 
     # ---- device-resident run: inputs already in HBM when timing starts ----
@@ -349,26 +353,27 @@ def main():
         props = torch.cuda.get_device_properties(local_rank)
         n_sm = props.multi_processor_count
         sm_max = (clocks or {}).get("sm_max_mhz") or peaks.get("sm_max_mhz", 1965.0)
-        peak_tflops = n_sm * FP32_LANES_PER_SM * 2 * sm_max * 1e6 / 1e12
+        lanes = FP64_LANES_PER_SM if f64 else FP32_LANES_PER_SM
+        peak_tflops = n_sm * lanes * 2 * sm_max * 1e6 / 1e12
         pairs = counters["pairs_in_cutoff"]
         entries = counters["list_entries"]
         flop = FLOP_PER_PAIR * pairs + FLOP_PER_SKIN_ENTRY * max(entries - pairs, 0) + FLOP_PER_ATOM * n
         k_avg_ms = k_ms / max(k_launches, 1)
         achieved = flop / (k_avg_ms * 1e-3) / 1e12
-        roofline = {"bound": "alu", "kernel": "k_mega", "achieved": achieved, "peak": peak_tflops, "unit": "TFLOP/s",
+        roofline = {"bound": "alu", "kernel": "k_mega_f64" if f64 else "k_mega", "achieved": achieved, "peak": peak_tflops, "unit": "TFLOP/s",
                     "frac": achieved / peak_tflops,
-                    "peak_source": f"{n_sm} SMs x {FP32_LANES_PER_SM} fp32 lanes x 2 x {sm_max:.0f} MHz (max SM clock)",
+                    "peak_source": f"{n_sm} SMs x {lanes} fp{args.precision[1:]} lanes x 2 x {sm_max:.0f} MHz (max SM clock)",
                     "kernel_ms_avg": k_avg_ms, "kernel_launches_timed": k_launches,
                     "kernel_share_of_step": k_ms / ms if ms > 0 else None,
                     "flop_per_launch": flop, "pairs_in_cutoff_per_atom": pairs / n, "list_entries_per_atom": entries / n,
-                    "traffic": None if NCU_DRAM_BYTES_PER_ATOM is None else NCU_DRAM_BYTES_PER_ATOM * n,
+                    "traffic": None if NCU_DRAM_BYTES_PER_ATOM is None or f64 else NCU_DRAM_BYTES_PER_ATOM * n,
                     "hbm_peak_gbs": peaks["hbm_gbs"], "hbm_peak_kind": f"of {peak_kind}"}
         if clocks and clocks.get("sm_mhz"):
-            roofline["frac_at_sampled_clock"] = achieved / (n_sm * FP32_LANES_PER_SM * 2 * clocks["sm_mhz"] * 1e6 / 1e12)
+            roofline["frac_at_sampled_clock"] = achieved / (n_sm * lanes * 2 * clocks["sm_mhz"] * 1e6 / 1e12)
         resident = mlip.mlip_resident_bytes(pot.ctx)
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
                 "ms_per_step": ms_max / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-                "dtype": "f32", "data": "synthetic",
+                "dtype": args.precision, "data": "synthetic",
                 "config": {"workload": f"cfg{cfg} {w.name}: {n} atoms, {w.n_species} species, r_cut 6 A, skin 1 A, "
                                        f"NVE dt 1 fs, list rebuild every {rebuild_every} steps",
                            "atoms_per_gpu": n, "parallelism": "replicas" if world > 1 else "single",

@@ -65,8 +65,12 @@ typedef struct {
     int head_hidden, head_layers;  /* 64, 4 */
     int table_knots;      /* intervals of the radial table on [table_r_min, r_cut]; 0 = automatic: 64, doubled until table_tol holds */
     double table_r_min;   /* smallest tabulated distance; 0 = default (1.0) */
-    double table_tol;     /* accepted table error relative to max|g|; 0 = default (1e-6) */
+    double table_tol;     /* accepted table error relative to max|g|; 0 = default (1e-6; with precision 1: 1e-10, and 100 x that for g') */
     int device;           /* CUDA device ordinal */
+    int precision;        /* 0: fp32 with the contractions on the tensor pipe (split TF32), the production path;
+                             1: every step of Eq. 1-10 in fp64 (Section 4.2 evaluates in double precision by default):
+                                fp64 tables (automatic knots start at 512), fp64 forces kept for the integrator,
+                                +32 bytes per atom, several times slower */
 } mlip_config;
 
 /*
@@ -144,6 +148,14 @@ int mlip_set_velocities(mlip_ctx *ctx, const double *vel, void *stream);
  *   e_atom dev [N] float
  */
 int mlip_compute(mlip_ctx *ctx, double *energy, float *forces, double *virial, float *e_atom, void *stream);
+
+/*
+ * The same evaluation with fp64 per-atom outputs (forces dev [N][3] double,
+ * e_atom dev [N] double), for contexts created with precision = 1; returns
+ * MLIP_ERR_UNSUPPORTED on an fp32 context.  mlip_compute() on an fp64 context
+ * runs the fp64 kernel and rounds the per-atom outputs to float.
+ */
+int mlip_compute_f64(mlip_ctx *ctx, double *energy, double *forces, double *virial, double *e_atom, void *stream);
 
 /*
  * Same evaluation with HOST buffers: copies positions in (and species at a

@@ -23,7 +23,7 @@ ERRORS = {0: "MLIP_OK", 1: "MLIP_ERR_INVALID_ARG", 2: "MLIP_ERR_UNSUPPORTED", 3:
 CODES = {v: k for k, v in ERRORS.items()}
 
 EXPORTS = ["mlip_create", "mlip_table_error", "mlip_build_neighbors", "mlip_get_neighbors", "mlip_get_neighbors_noalloc", "mlip_set_positions",
-           "mlip_set_velocities", "mlip_compute", "mlip_compute_host", "mlip_step", "mlip_get_state",
+           "mlip_set_velocities", "mlip_compute", "mlip_compute_f64", "mlip_compute_host", "mlip_step", "mlip_get_state",
            "mlip_get_energies", "mlip_sync_status", "mlip_get_counters", "mlip_kernel_time",
            "mlip_resident_bytes", "mlip_last_error", "mlip_destroy"]
 
@@ -40,7 +40,7 @@ class Config(ctypes.Structure):
                 ("enc_hidden", ctypes.c_int), ("enc_layers", ctypes.c_int),
                 ("head_hidden", ctypes.c_int), ("head_layers", ctypes.c_int),
                 ("table_knots", ctypes.c_int), ("table_r_min", ctypes.c_double), ("table_tol", ctypes.c_double),
-                ("device", ctypes.c_int)]
+                ("device", ctypes.c_int), ("precision", ctypes.c_int)]
 
 
 _lib = None
@@ -144,6 +144,10 @@ def mlip_compute(ctx, energy=None, forces=None, virial=None, e_atom=None, stream
     _check(ctx, lib().mlip_compute(ctx, _dev(energy), _dev(forces), _dev(virial), _dev(e_atom), _stream(stream)))
 
 
+def mlip_compute_f64(ctx, energy=None, forces=None, virial=None, e_atom=None, stream=None):
+    _check(ctx, lib().mlip_compute_f64(ctx, _dev(energy), _dev(forces), _dev(virial), _dev(e_atom), _stream(stream)))
+
+
 def mlip_compute_host(ctx, pos, species, box, rebuild, forces_out, virial_out=None):
     e = ctypes.c_double(0)
     box = None if box is None else np.ascontiguousarray(box, dtype=np.float64)
@@ -205,13 +209,14 @@ class Potential:
     """Convenience owner of one context; allocates outputs as torch tensors."""
 
     def __init__(self, n_species, r_cut, skin, enc_w, head_w, masses, device=0, table_knots=0,
-                 table_r_min=0.0, table_tol=0.0, enc_hidden=128, enc_layers=3, allow_table_error=False):
+                 table_r_min=0.0, table_tol=0.0, enc_hidden=128, enc_layers=3, allow_table_error=False, precision=0):
         import torch
         self.torch = torch
         self.device = torch.device("cuda", device)
         self.n_species = n_species
         self.cfg = Config(n_species, r_cut, skin, 32, 3, enc_hidden, enc_layers, 64, 4, table_knots, table_r_min,
-                          table_tol, device)
+                          table_tol, device, precision)
+        self.precision = precision
         self.ctx = mlip_create(self.cfg, enc_w, head_w, masses, allow_table_error)
         self.n = 0
 
@@ -243,12 +248,15 @@ class Potential:
         return seg, nbr[:total]
 
     def compute(self, want_e_atom=False):
+        """Per-atom outputs are float32, or float64 on a context created with precision=1."""
         t = self.torch
+        real = t.float64 if self.precision == 1 else t.float32
         out = {"energy": t.zeros(1, dtype=t.float64, device=self.device),
-               "forces": t.empty((self.n, 3), dtype=t.float32, device=self.device),
+               "forces": t.empty((self.n, 3), dtype=real, device=self.device),
                "virial": t.zeros(9, dtype=t.float64, device=self.device),
-               "e_atom": t.empty(self.n, dtype=t.float32, device=self.device) if want_e_atom else None}
-        mlip_compute(self.ctx, out["energy"], out["forces"], out["virial"], out["e_atom"])
+               "e_atom": t.empty(self.n, dtype=real, device=self.device) if want_e_atom else None}
+        call = mlip_compute_f64 if self.precision == 1 else mlip_compute
+        call(self.ctx, out["energy"], out["forces"], out["virial"], out["e_atom"])
         return out
 
     def set_positions(self, pos):

@@ -47,6 +47,7 @@ static void free_atoms(mlip_ctx *c) {
     dev_free(c, &c->force, n); dev_free(c, &c->disp, 3 * n); dev_free(c, &c->e_atom, n);
     dev_free(c, &c->center_order, n); dev_free(c, &c->cell_of, n);
     dev_free(c, &c->nbr_count, n); dev_free(c, &c->nbr_off, n + 1);
+    if (c->cfg.precision == 1) { dev_free(c, &c->force_d, 3 * n); dev_free(c, &c->e_atom_d, n); }
     c->cap_atoms = 0;
 }
 
@@ -69,6 +70,7 @@ static int ensure_capacity(mlip_ctx *c, int64_t n, int64_t n_cells) {
         TRY_ALLOC(c->force, m); TRY_ALLOC(c->disp, 3 * m); TRY_ALLOC(c->e_atom, m);
         TRY_ALLOC(c->center_order, m); TRY_ALLOC(c->cell_of, m);
         TRY_ALLOC(c->nbr_count, m); TRY_ALLOC(c->nbr_off, m + 1);
+        if (c->cfg.precision == 1) { TRY_ALLOC(c->force_d, 3 * m); TRY_ALLOC(c->e_atom_d, m); }
         c->cap_atoms = n;
     }
     if (n_cells > c->cap_cells) {
@@ -122,14 +124,16 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
     if (n_head != (size_t)cfg->n_species * HEAD_NET) return fail(nullptr, MLIP_ERR_INVALID_ARG, "head weight count does not match the shape");
     for (int s = 0; s < cfg->n_species; ++s)
         if (!(mass[s] > 0.0)) return fail(nullptr, MLIP_ERR_INVALID_ARG, "mass must be positive");
+    if (cfg->precision != 0 && cfg->precision != 1) return fail(nullptr, MLIP_ERR_INVALID_ARG, "precision must be 0 (fp32) or 1 (fp64)");
 
     mlip_ctx *c = new (std::nothrow) mlip_ctx();
     if (!c) return fail(nullptr, MLIP_ERR_OOM, "host allocation failed");
     c->cfg = *cfg;
     const bool auto_knots = c->cfg.table_knots <= 0;
-    if (auto_knots) c->cfg.table_knots = 64;
+    const bool f64 = c->cfg.precision == 1;
+    if (auto_knots) c->cfg.table_knots = f64 ? 512 : 64;
     if (c->cfg.table_r_min <= 0.0) c->cfg.table_r_min = 1.0;
-    if (c->cfg.table_tol <= 0.0) c->cfg.table_tol = 1e-6;
+    if (c->cfg.table_tol <= 0.0) c->cfg.table_tol = f64 ? 1e-10 : 1e-6;
     if (c->cfg.table_knots > 8192 || c->cfg.table_r_min >= c->cfg.r_cut) { delete c; return fail(nullptr, MLIP_ERR_INVALID_ARG, "bad table parameters"); }
 
     int rc = MLIP_OK;
@@ -162,10 +166,10 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
             cudaMemset(c->status, 0, sizeof(int)) != cudaSuccess || cudaMemset(c->acc, 0, sizeof(double) * ACC_COUNT) != cudaSuccess) {
             rc = MLIP_ERR_CUDA; c->err = "initial upload failed"; break;
         }
-        if ((rc = upload_head(c, head_w)) != MLIP_OK) break;
+        if ((rc = f64 ? upload_head_f64(c, head_w) : upload_head(c, head_w)) != MLIP_OK) break;
         rc = build_tables(c, enc_w, n_enc);
         // automatic knot count: double until the spline meets the tolerance
-        while (auto_knots && rc == MLIP_ERR_TABLE_TOLERANCE && c->cfg.table_knots < 2048) {
+        while (auto_knots && rc == MLIP_ERR_TABLE_TOLERANCE && c->cfg.table_knots < (f64 ? 8192 : 2048)) {
             c->cfg.table_knots *= 2;
             rc = build_tables(c, enc_w, n_enc);
         }
@@ -240,12 +244,32 @@ int mlip_set_velocities(mlip_ctx *c, const double *vel, void *stream) {
     return launch_set_velocities(c, vel, (cudaStream_t)stream);
 }
 
+// The fused evaluation in the context's precision.
+static int evaluate(mlip_ctx *c, cudaStream_t s) {
+    return c->cfg.precision == 1 ? launch_megakernel_f64(c, s) : launch_megakernel(c, s);
+}
+
+int mlip_compute_f64(mlip_ctx *c, double *energy, double *forces, double *virial, double *e_atom, void *stream) {
+    if (!c) return MLIP_ERR_INVALID_ARG;
+    if (c->cfg.precision != 1) return fail(c, MLIP_ERR_UNSUPPORTED, "mlip_compute_f64 needs a context created with precision = 1");
+    if (!c->built) return fail(c, MLIP_ERR_NOT_BUILT, "no neighbor lists yet");
+    cudaStream_t s = (cudaStream_t)stream;
+    c->last_stream = s;
+    int rc = launch_megakernel_f64(c, s);
+    if (rc != MLIP_OK) return rc;
+    c->forces_current = true;
+    if (energy) MLIP_CUDA_TRY(c, cudaMemcpyAsync(energy, c->acc + ACC_ENERGY, sizeof(double), cudaMemcpyDeviceToDevice, s));
+    if (virial) MLIP_CUDA_TRY(c, cudaMemcpyAsync(virial, c->acc + ACC_VIRIAL, sizeof(double) * 9, cudaMemcpyDeviceToDevice, s));
+    if (forces || e_atom) rc = launch_scatter_forces_f64(c, forces, e_atom, s);
+    return rc;
+}
+
 int mlip_compute(mlip_ctx *c, double *energy, float *forces, double *virial, float *e_atom, void *stream) {
     if (!c) return MLIP_ERR_INVALID_ARG;
     if (!c->built) return fail(c, MLIP_ERR_NOT_BUILT, "no neighbor lists yet");
     cudaStream_t s = (cudaStream_t)stream;
     c->last_stream = s;
-    int rc = launch_megakernel(c, s);
+    int rc = evaluate(c, s);
     if (rc != MLIP_OK) return rc;
     c->forces_current = true;
     if (energy) MLIP_CUDA_TRY(c, cudaMemcpyAsync(energy, c->acc + ACC_ENERGY, sizeof(double), cudaMemcpyDeviceToDevice, s));
@@ -294,7 +318,7 @@ int mlip_step(mlip_ctx *c, int n_steps, double dt, int rebuild_every, void *stre
     c->last_stream = s;
     int rc;
     if (!c->forces_current) {
-        if ((rc = launch_megakernel(c, s)) != MLIP_OK) return rc;
+        if ((rc = evaluate(c, s)) != MLIP_OK) return rc;
         c->forces_current = true;
     }
     for (int it = 0; it < n_steps; ++it) {
@@ -306,7 +330,7 @@ int mlip_step(mlip_ctx *c, int n_steps, double dt, int rebuild_every, void *stre
             std::swap(c->user_of, c->user_src);
             if ((rc = launch_build(c, false, s)) != MLIP_OK) return rc;
         }
-        if ((rc = launch_megakernel(c, s)) != MLIP_OK) return rc;
+        if ((rc = evaluate(c, s)) != MLIP_OK) return rc;
         if ((rc = launch_kick(c, dt, s)) != MLIP_OK) return rc;
     }
     return MLIP_OK;
@@ -400,6 +424,7 @@ void mlip_destroy(mlip_ctx *c) {
     free_atoms(c);
     free_cells(c);
     cudaFree(c->nbr); cudaFree(c->scan_tmp); cudaFree(c->head_w); cudaFree(c->table); cudaFree(c->mass);
+    cudaFree(c->head_w_d); cudaFree(c->table_d);
     cudaFree(c->acc); cudaFree(c->pair_counter); cudaFree(c->status); cudaFree(c->tile_counter);
     cudaFree(c->species_start); cudaFree(c->stage_pos); cudaFree(c->stage_species); cudaFree(c->stage_force);
     cudaFree(c->stage_out);

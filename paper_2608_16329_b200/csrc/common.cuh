@@ -59,6 +59,11 @@ struct mlip_ctx {
     float *head_w = nullptr;     // per-species head weights packed in MMA fragment order (megakernel.cu)
     float *table = nullptr;      // spline coefficients
     double *mass = nullptr;      // [C] dev
+    // fp64 path (precision = 1) only
+    double *head_w_d = nullptr;  // per-species head weights, row-major and transposed (megakernel_f64.cu)
+    double *table_d = nullptr;   // spline coefficients in fp64
+    double *force_d = nullptr;   // [N][3]
+    double *e_atom_d = nullptr;  // [N]
     double table_err_value = 0, table_err_deriv = 0;
     mlip::TableDesc tab{};
 
@@ -134,11 +139,15 @@ int build_tables(mlip_ctx *c, const double *enc_w_host, size_t n_enc);
 // megakernel.cu
 int upload_head(mlip_ctx *c, const double *head_w_host);
 int launch_megakernel(mlip_ctx *c, cudaStream_t s);
+// megakernel_f64.cu
+int upload_head_f64(mlip_ctx *c, const double *head_w_host);
+int launch_megakernel_f64(mlip_ctx *c, cudaStream_t s);
 // integrate.cu
 int launch_kick_drift(mlip_ctx *c, double dt, cudaStream_t s);
 int launch_kick(mlip_ctx *c, double dt, cudaStream_t s);
 int launch_kinetic(mlip_ctx *c, cudaStream_t s);
 int launch_scatter_forces(mlip_ctx *c, float *forces, float *e_atom, cudaStream_t s);
+int launch_scatter_forces_f64(mlip_ctx *c, double *forces, double *e_atom, cudaStream_t s);
 int launch_set_positions(mlip_ctx *c, const double *pos, cudaStream_t s);
 int launch_set_velocities(mlip_ctx *c, const double *vel, cudaStream_t s);
 int launch_get_state(mlip_ctx *c, double *pos, double *vel, cudaStream_t s);

@@ -6,14 +6,21 @@
 
 namespace mlip {
 
+// Force on atom i: the fp64 array when the context evaluates in fp64, else the fp32 one.
+__device__ __forceinline__ double3 load_force(const float4 *__restrict__ force, const double *__restrict__ force_d, int64_t i) {
+    if (force_d) return make_double3(force_d[3 * i], force_d[3 * i + 1], force_d[3 * i + 2]);
+    const float4 f = force[i];
+    return make_double3(f.x, f.y, f.z);
+}
+
 // v += dt/2 a;  x += dt v;  wrap into [0, L);  track the displacement since the last list build.
 __global__ void k_kick_drift(int64_t n, double dt, CellGrid g, const double *__restrict__ mass, float skin_half2,
                              double4 *__restrict__ pos4, double *__restrict__ vel, const float4 *__restrict__ force,
-                             float *__restrict__ disp, int *status) {
+                             const double *__restrict__ force_d, float *__restrict__ disp, int *status) {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     double4 p = pos4[i];
-    const float4 f = force[i];
+    const double3 f = load_force(force, force_d, i);
     const double k = 0.5 * dt * ACC_UNIT / mass[(int)p.w];
     double v[3] = {vel[3 * i] + k * f.x, vel[3 * i + 1] + k * f.y, vel[3 * i + 2] + k * f.z};
     double x[3] = {p.x + dt * v[0], p.y + dt * v[1], p.z + dt * v[2]};
@@ -35,10 +42,10 @@ __global__ void k_kick_drift(int64_t n, double dt, CellGrid g, const double *__r
 
 // v += dt/2 a
 __global__ void k_kick(int64_t n, double dt, const double *__restrict__ mass, const double4 *__restrict__ pos4,
-                       double *__restrict__ vel, const float4 *__restrict__ force) {
+                       double *__restrict__ vel, const float4 *__restrict__ force, const double *__restrict__ force_d) {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
-    const float4 f = force[i];
+    const double3 f = load_force(force, force_d, i);
     const double k = 0.5 * dt * ACC_UNIT / mass[(int)pos4[i].w];
     vel[3 * i] += k * f.x; vel[3 * i + 1] += k * f.y; vel[3 * i + 2] += k * f.z;
 }
@@ -68,6 +75,15 @@ __global__ void k_scatter_forces(int64_t n, const int32_t *__restrict__ user_of,
     const float4 f = force[i];
     const int64_t u = user_of[i];
     if (forces_out) { forces_out[3 * u] = f.x; forces_out[3 * u + 1] = f.y; forces_out[3 * u + 2] = f.z; }
+    if (e_atom) e_atom[u] = e_in[i];
+}
+
+__global__ void k_scatter_forces_f64(int64_t n, const int32_t *__restrict__ user_of, const double *__restrict__ force,
+                                     const double *__restrict__ e_in, double *__restrict__ forces_out, double *__restrict__ e_atom) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int64_t u = user_of[i];
+    if (forces_out) { forces_out[3 * u] = force[3 * i]; forces_out[3 * u + 1] = force[3 * i + 1]; forces_out[3 * u + 2] = force[3 * i + 2]; }
     if (e_atom) e_atom[u] = e_in[i];
 }
 
@@ -114,13 +130,13 @@ static inline unsigned nb(int64_t n) { return (unsigned)((n + 255) / 256); }
 static inline float skin_half2(const mlip_ctx *c) { float h = 0.5f * (float)c->cfg.skin; return h * h; }
 
 int launch_kick_drift(mlip_ctx *c, double dt, cudaStream_t s) {
-    k_kick_drift<<<nb(c->n), 256, 0, s>>>(c->n, dt, c->grid, c->mass, skin_half2(c), c->pos4, c->vel, c->force, c->disp, c->status);
+    k_kick_drift<<<nb(c->n), 256, 0, s>>>(c->n, dt, c->grid, c->mass, skin_half2(c), c->pos4, c->vel, c->force, c->force_d, c->disp, c->status);
     c->launches += 1;
     MLIP_CUDA_TRY(c, cudaGetLastError());
     return MLIP_OK;
 }
 int launch_kick(mlip_ctx *c, double dt, cudaStream_t s) {
-    k_kick<<<nb(c->n), 256, 0, s>>>(c->n, dt, c->mass, c->pos4, c->vel, c->force);
+    k_kick<<<nb(c->n), 256, 0, s>>>(c->n, dt, c->mass, c->pos4, c->vel, c->force, c->force_d);
     c->launches += 1;
     MLIP_CUDA_TRY(c, cudaGetLastError());
     return MLIP_OK;
@@ -136,6 +152,12 @@ int launch_kinetic(mlip_ctx *c, cudaStream_t s) {
 }
 int launch_scatter_forces(mlip_ctx *c, float *forces, float *e_atom, cudaStream_t s) {
     k_scatter_forces<<<nb(c->n), 256, 0, s>>>(c->n, c->user_of, c->force, c->e_atom, forces, e_atom);
+    c->launches += 1;
+    MLIP_CUDA_TRY(c, cudaGetLastError());
+    return MLIP_OK;
+}
+int launch_scatter_forces_f64(mlip_ctx *c, double *forces, double *e_atom, cudaStream_t s) {
+    k_scatter_forces_f64<<<nb(c->n), 256, 0, s>>>(c->n, c->user_of, c->force_d, c->e_atom_d, forces, e_atom);
     c->launches += 1;
     MLIP_CUDA_TRY(c, cudaGetLastError());
     return MLIP_OK;

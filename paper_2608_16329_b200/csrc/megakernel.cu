@@ -30,6 +30,7 @@
 #include <algorithm>
 
 #include "common.cuh"
+#include "pair_math.cuh"
 
 namespace mlip {
 
@@ -116,83 +117,6 @@ __device__ __forceinline__ void mma_tf32_z(float (&d)[4], uint32_t a0, uint32_t 
 // pipe truncates when it adds into its fp32 accumulator, so the energy path keeps accumulation
 // chains short (a fresh accumulator per k-step, folded into the running sum by a rounded fp32
 // add): a long chain of same-sign terms otherwise drifts by ~1e-6 relative.
-
-// Irreducible harmonic polynomials up to l = 3 of a unit vector (one valid solution of the
-// projection constraints of Section 3.3.1: harmonic, orthonormal under the multinomial metric).
-__device__ __forceinline__ void harmonics(float x, float y, float z, float *h) {
-    const float s2 = 1.41421356237f, is2 = 0.70710678118f, is6 = 0.40824829046f;
-    const float s6 = 2.44948974278f, s15 = 1.22474487139f, is10 = 0.31622776601f;
-    float xx = x * x, yy = y * y, zz = z * z;
-    h[0] = 1.0f;
-    h[1] = x; h[2] = y; h[3] = z;
-    h[4] = s2 * x * y; h[5] = s2 * x * z; h[6] = s2 * y * z;
-    h[7] = is2 * (xx - yy);
-    h[8] = is6 * (2.0f * zz - xx - yy);
-    h[9] = s6 * x * y * z;
-    h[10] = s15 * z * (xx - yy);
-    h[11] = s15 * x * (yy - zz);
-    h[12] = s15 * y * (zz - xx);
-    h[13] = is10 * x * (2.0f * xx - 3.0f * yy - 3.0f * zz);
-    h[14] = is10 * y * (2.0f * yy - 3.0f * xx - 3.0f * zz);
-    h[15] = is10 * z * (2.0f * zz - 3.0f * xx - 3.0f * yy);
-}
-
-// s = sum_a h_a t_a,  (tx,ty,tz) = sum_a v_a grad h_a,  tu = sum_a l_a v_a h_a  (Euler: grad h_a . u = l_a h_a).
-__device__ __forceinline__ void harmonics_project(float x, float y, float z, const float *v, const float *t,
-                                                  float &s, float &tx, float &ty, float &tz, float &tu) {
-    const float s2 = 1.41421356237f, is2 = 0.70710678118f, is6 = 0.40824829046f;
-    const float s6 = 2.44948974278f, s15 = 1.22474487139f, is10 = 0.31622776601f;
-    float xx = x * x, yy = y * y, zz = z * z, h;
-    s = t[0]; tx = ty = tz = 0.f; tu = 0.f;
-    s += x * t[1] + y * t[2] + z * t[3];
-    tx += v[1]; ty += v[2]; tz += v[3];
-    tu += x * v[1] + y * v[2] + z * v[3];
-    float u2 = 0.f;
-    h = s2 * x * y; s += h * t[4]; u2 += h * v[4]; tx += s2 * y * v[4]; ty += s2 * x * v[4];
-    h = s2 * x * z; s += h * t[5]; u2 += h * v[5]; tx += s2 * z * v[5]; tz += s2 * x * v[5];
-    h = s2 * y * z; s += h * t[6]; u2 += h * v[6]; ty += s2 * z * v[6]; tz += s2 * y * v[6];
-    h = is2 * (xx - yy); s += h * t[7]; u2 += h * v[7]; tx += s2 * x * v[7]; ty -= s2 * y * v[7];
-    h = is6 * (2.f * zz - xx - yy); s += h * t[8]; u2 += h * v[8];
-    tx -= 2.f * is6 * x * v[8]; ty -= 2.f * is6 * y * v[8]; tz += 4.f * is6 * z * v[8];
-    float u3 = 0.f;
-    h = s6 * x * y * z; s += h * t[9]; u3 += h * v[9];
-    tx += s6 * y * z * v[9]; ty += s6 * x * z * v[9]; tz += s6 * x * y * v[9];
-    h = s15 * z * (xx - yy); s += h * t[10]; u3 += h * v[10];
-    tx += 2.f * s15 * x * z * v[10]; ty -= 2.f * s15 * y * z * v[10]; tz += s15 * (xx - yy) * v[10];
-    h = s15 * x * (yy - zz); s += h * t[11]; u3 += h * v[11];
-    tx += s15 * (yy - zz) * v[11]; ty += 2.f * s15 * x * y * v[11]; tz -= 2.f * s15 * x * z * v[11];
-    h = s15 * y * (zz - xx); s += h * t[12]; u3 += h * v[12];
-    tx -= 2.f * s15 * x * y * v[12]; ty += s15 * (zz - xx) * v[12]; tz += 2.f * s15 * y * z * v[12];
-    h = is10 * x * (2.f * xx - 3.f * yy - 3.f * zz); s += h * t[13]; u3 += h * v[13];
-    tx += is10 * (6.f * xx - 3.f * yy - 3.f * zz) * v[13]; ty -= 6.f * is10 * x * y * v[13]; tz -= 6.f * is10 * x * z * v[13];
-    h = is10 * y * (2.f * yy - 3.f * xx - 3.f * zz); s += h * t[14]; u3 += h * v[14];
-    tx -= 6.f * is10 * x * y * v[14]; ty += is10 * (6.f * yy - 3.f * xx - 3.f * zz) * v[14]; tz -= 6.f * is10 * y * z * v[14];
-    h = is10 * z * (2.f * zz - 3.f * xx - 3.f * yy); s += h * t[15]; u3 += h * v[15];
-    tx -= 6.f * is10 * x * z * v[15]; ty -= 6.f * is10 * y * z * v[15]; tz += is10 * (6.f * zz - 3.f * xx - 3.f * yy) * v[15];
-    tu += 2.f * u2 + 3.f * u3;
-}
-
-// Spline interval and cubic B-spline basis (and its r-derivative) at distance r.
-template <bool DERIV>
-__device__ __forceinline__ int spline_basis(float r, const TableDesc &tab, float *b, float *db, int *status) {
-    float xk = (r - tab.r_min) * tab.inv_h;
-    if (xk < 0.f) { atomicOr(status, FLAG_TABLE_RANGE); xk = 0.f; }
-    int i = (int)xk;
-    i = i > tab.knots - 1 ? tab.knots - 1 : i;
-    float u = xk - (float)i, u2 = u * u, u3 = u2 * u, w = 1.f - u;
-    const float sixth = 1.0f / 6.0f;
-    b[0] = w * w * w * sixth;
-    b[1] = (3.f * u3 - 6.f * u2 + 4.f) * sixth;
-    b[2] = (-3.f * u3 + 3.f * u2 + 3.f * u + 1.f) * sixth;
-    b[3] = u3 * sixth;
-    if (DERIV) {
-        db[0] = -0.5f * w * w * tab.inv_h;
-        db[1] = (1.5f * u2 - 2.f * u) * tab.inv_h;
-        db[2] = (-1.5f * u2 + u + 0.5f) * tab.inv_h;
-        db[3] = 0.5f * u2 * tab.inv_h;
-    }
-    return i;
-}
 
 // Optional per-phase cycle counters (profiling builds only: -DMLIP_PHASE_CLOCKS).  Slots 16.. of
 // the accumulator array receive the summed clock64 ticks of lane 0 of every warp.
@@ -308,7 +232,7 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
                 const float4 e = pq[first + lane];
                 const float r = sqrtf(e.x * e.x + e.y * e.y + e.z * e.z), rinv = 1.0f / r;
                 harmonics(e.x * rinv, e.y * rinv, e.z * rinv, h);
-                const int iv = spline_basis<false>(r, k.tab, b, nullptr, k.status);
+                const int iv = spline_basis<false, float>(r, k.tab.r_min, k.tab.inv_h, k.tab.knots, b, nullptr, k.status);
                 const int sj = __float_as_int(e.w) >> J_BITS;
                 off = sj * tv.table_stride + iv * rs;
             } else {
@@ -416,7 +340,7 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
                 ent = pq[first + lane];
                 const float r = sqrtf(ent.x * ent.x + ent.y * ent.y + ent.z * ent.z);
                 rinv = 1.0f / r;
-                const int iv = spline_basis<true>(r, k.tab, b, db, k.status);
+                const int iv = spline_basis<true, float>(r, k.tab.r_min, k.tab.inv_h, k.tab.knots, b, db, k.status);
                 row_index = (__float_as_int(ent.w) >> J_BITS) * (k.tab.knots + 3) + iv;
                 off = row_index * rs;
             }

@@ -70,8 +70,9 @@ __global__ void k_table_sample(const double *__restrict__ enc_w, size_t net_size
 // One thread per (net, channel): clamped cubic B-spline interpolation through the K + 1 knot values.
 // Unknown control points c_0 .. c_{K+2};  (c_i + 4 c_{i+1} + c_{i+2}) / 6 = f_i,  (c_2 - c_0) / 2h = f'_0,
 // (c_{K+2} - c_K) / 2h = f'_K.  Thomas algorithm on c_1 .. c_{K+1}; `work` holds 2 (K + 1) doubles per thread.
+template <typename CoefT>
 __global__ void k_table_solve(const double *__restrict__ val, const double *__restrict__ der, int n_nets, int knots, int k,
-                              double h, double *__restrict__ work, float *__restrict__ coef) {
+                              double h, double *__restrict__ work, CoefT *__restrict__ coef) {
     int t = blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= n_nets * k) return;
     const int net = t / k, c = t % k, n = knots + 1;
@@ -90,19 +91,20 @@ __global__ void k_table_solve(const double *__restrict__ val, const double *__re
         x[i] = (rhs - lower * x[i - 1]) / m;
     }
     for (int i = n - 2; i >= 0; --i) x[i] -= cp[i] * x[i + 1];
-    float *out = coef + (size_t)net * (knots + 3) * k + c;
-    out[0] = (float)(x[1] - 2.0 * h * fp[0]);                        // c_0 = c_2 - 2 h f'_0
-    for (int i = 0; i < n; ++i) out[(size_t)(i + 1) * k] = (float)x[i];
-    out[(size_t)(knots + 2) * k] = (float)(x[n - 2] + 2.0 * h * fp[(size_t)(n - 1) * k]);
+    CoefT *out = coef + (size_t)net * (knots + 3) * k + c;
+    out[0] = (CoefT)(x[1] - 2.0 * h * fp[0]);                        // c_0 = c_2 - 2 h f'_0
+    for (int i = 0; i < n; ++i) out[(size_t)(i + 1) * k] = (CoefT)x[i];
+    out[(size_t)(knots + 2) * k] = (CoefT)(x[n - 2] + 2.0 * h * fp[(size_t)(n - 1) * k]);
 }
 
 __device__ inline void atomic_max_pos(unsigned long long *addr, double v) {   // v >= 0: bit patterns are ordered
     atomicMax(addr, (unsigned long long)__double_as_longlong(v));
 }
 
-// Compare the fp32 spline (evaluated in fp64) with network samples taken between the knots.
+// Compare the stored spline (evaluated in fp64) with network samples taken between the knots.
 // out[0] = max |g|, out[1] = max |g'|, out[2] = max |spline - g|, out[3] = max |spline' - g'|
-__global__ void k_table_check(const double *__restrict__ val, const double *__restrict__ der, const float *__restrict__ coef,
+template <typename CoefT>
+__global__ void k_table_check(const double *__restrict__ val, const double *__restrict__ der, const CoefT *__restrict__ coef,
                               int n_nets, int n_points, int knots, int k, double r_min, double r0, double step, double h,
                               unsigned long long *out) {
     int t = blockIdx.x * blockDim.x + threadIdx.x;
@@ -117,7 +119,7 @@ __global__ void k_table_check(const double *__restrict__ val, const double *__re
     double db[4] = {-0.5 * v * v / h, (1.5 * u2 - 2.0 * u) / h, (-1.5 * u2 + u + 0.5) / h, 0.5 * u2 / h};
     double m[4] = {0, 0, 0, 0};
     for (int c = 0; c < k; ++c) {
-        const float *cf = coef + ((size_t)net * (knots + 3) + i) * k + c;
+        const CoefT *cf = coef + ((size_t)net * (knots + 3) + i) * k + c;
         double s = 0.0, ds = 0.0;
         for (int q = 0; q < 4; ++q) { s += b[q] * (double)cf[(size_t)q * k]; ds += db[q] * (double)cf[(size_t)q * k]; }
         double g = val[((size_t)net * n_points + p) * k + c], dg = der[((size_t)net * n_points + p) * k + c];
@@ -144,9 +146,15 @@ int build_tables(mlip_ctx *c, const double *enc_w_host, size_t n_enc) {
     MLIP_CUDA_TRY(c, cudaMalloc(&der, sizeof(double) * n_pts_max));
     MLIP_CUDA_TRY(c, cudaMalloc(&work, sizeof(double) * (size_t)n_nets * k * 2 * n_knot_pts));
     MLIP_CUDA_TRY(c, cudaMalloc(&stats, sizeof(unsigned long long) * 4));
-    const size_t coef_bytes = sizeof(float) * (size_t)n_nets * (K + 3) * k;
-    if (c->table) { cudaFree(c->table); c->table = nullptr; c->resident -= c->table_bytes; }   // a retry with more knots
-    MLIP_CUDA_TRY(c, cudaMalloc(&c->table, coef_bytes));
+    const bool f64 = cfg.precision == 1;
+    const size_t coef_bytes = (f64 ? sizeof(double) : sizeof(float)) * (size_t)n_nets * (K + 3) * k;
+    if (c->table || c->table_d) {   // a retry with more knots
+        cudaFree(c->table); cudaFree(c->table_d);
+        c->table = nullptr; c->table_d = nullptr;
+        c->resident -= c->table_bytes;
+    }
+    if (f64) MLIP_CUDA_TRY(c, cudaMalloc(&c->table_d, coef_bytes));
+    else MLIP_CUDA_TRY(c, cudaMalloc(&c->table, coef_bytes));
     c->table_bytes = coef_bytes;
     c->resident += coef_bytes;
     c->kernel_ready = false;
@@ -155,11 +163,13 @@ int build_tables(mlip_ctx *c, const double *enc_w_host, size_t n_enc) {
 
     int nt = n_nets * n_knot_pts;
     k_table_sample<<<(nt + 63) / 64, 64>>>(w, net_size, sh, n_nets, n_knot_pts, r_min, h, cfg.r_cut, val, der);
-    k_table_solve<<<(n_nets * k + 63) / 64, 64>>>(val, der, n_nets, K, k, h, work, c->table);
+    if (f64) k_table_solve<double><<<(n_nets * k + 63) / 64, 64>>>(val, der, n_nets, K, k, h, work, c->table_d);
+    else k_table_solve<float><<<(n_nets * k + 63) / 64, 64>>>(val, der, n_nets, K, k, h, work, c->table);
     nt = n_nets * n_chk;
     const double step = h / 4.0, r0 = r_min + 0.37 * step;
     k_table_sample<<<(nt + 63) / 64, 64>>>(w, net_size, sh, n_nets, n_chk, r0, step, r0 + (n_chk - 1) * step, val, der);
-    k_table_check<<<(nt + 63) / 64, 64>>>(val, der, c->table, n_nets, n_chk, K, k, r_min, r0, step, h, stats);
+    if (f64) k_table_check<double><<<(nt + 63) / 64, 64>>>(val, der, c->table_d, n_nets, n_chk, K, k, r_min, r0, step, h, stats);
+    else k_table_check<float><<<(nt + 63) / 64, 64>>>(val, der, c->table, n_nets, n_chk, K, k, r_min, r0, step, h, stats);
     c->launches += 4;
     unsigned long long host_stats[4];
     MLIP_CUDA_TRY(c, cudaMemcpy(host_stats, stats, sizeof host_stats, cudaMemcpyDeviceToHost));
@@ -174,9 +184,13 @@ int build_tables(mlip_ctx *c, const double *enc_w_host, size_t n_enc) {
     c->tab.r_min = (float)r_min;
     c->tab.inv_h = (float)(1.0 / h);
     c->tab.r_cut2 = (float)(cfg.r_cut * cfg.r_cut);
-    if (c->table_err_value > cfg.table_tol) {
-        char buf[160];
-        snprintf(buf, sizeof buf, "radial table error %.3g exceeds table_tol %.3g; raise table_knots", c->table_err_value, cfg.table_tol);
+    // the fp64 path also bounds the derivative (it carries the forces): one order in h worse than the value
+    const bool value_ok = c->table_err_value <= cfg.table_tol;
+    const bool deriv_ok = !f64 || c->table_err_deriv <= 100.0 * cfg.table_tol;
+    if (!value_ok || !deriv_ok) {
+        char buf[200];
+        snprintf(buf, sizeof buf, "radial table error %.3g (derivative %.3g) exceeds table_tol %.3g; raise table_knots",
+                 c->table_err_value, c->table_err_deriv, cfg.table_tol);
         c->err = buf;
         return MLIP_ERR_TABLE_TOLERANCE;
     }

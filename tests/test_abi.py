@@ -9,7 +9,7 @@ from conftest import ROOT
 def _declared():
     text = open(os.path.join(ROOT, "include", "mlip.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(mlip_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(mlip_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_library_exports_every_declared_symbol():
