@@ -240,13 +240,16 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
                 for (int a = 0; a < D_ANG; ++a) h[a] = 0.f;
                 b[0] = b[1] = b[2] = b[3] = 0.f;
             }
+            // 16-byte chunk c of row r is stored at chunk c ^ ((r >> 2) & 1): the eight rows of a store phase
+            // then fall into eight different bank groups (the row stride alone gives only four)
+            const int sw = (lane >> 2) & 1;
             float4 *row = reinterpret_cast<float4 *>(stage + lane * ST_STRIDE);
-            row[0] = make_float4(h[0], h[1], h[2], h[3]);
-            row[1] = make_float4(h[4], h[5], h[6], h[7]);
-            row[2] = make_float4(h[8], h[9], h[10], h[11]);
-            row[3] = make_float4(h[12], h[13], h[14], h[15]);
-            row[4] = make_float4(b[0], b[1], b[2], b[3]);
-            reinterpret_cast<int *>(stage)[lane * ST_STRIDE + 20] = off;
+            row[0 ^ sw] = make_float4(h[0], h[1], h[2], h[3]);
+            row[1 ^ sw] = make_float4(h[4], h[5], h[6], h[7]);
+            row[2 ^ sw] = make_float4(h[8], h[9], h[10], h[11]);
+            row[3 ^ sw] = make_float4(h[12], h[13], h[14], h[15]);
+            row[4 ^ sw] = make_float4(b[0], b[1], b[2], b[3]);
+            reinterpret_cast<int *>(stage)[lane * ST_STRIDE + 4 * (5 ^ sw)] = off;
         }
         __syncwarp();
         pc.mark(1);
@@ -257,17 +260,17 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
             uint32_t ah[4], al[4];
             split_tf32(ra[g], ah[0], al[0]);
             split_tf32(ra[g + 8], ah[1], al[1]);
-            split_tf32(rb[g], ah[2], al[2]);
-            split_tf32(rb[g + 8], ah[3], al[3]);
+            split_tf32(rb[g ^ 4], ah[2], al[2]);        // rows t + 4 are stored with their chunk pairs swapped
+            split_tf32(rb[(g ^ 4) + 8], ah[3], al[3]);
             // B = G (8 pairs x 8 channels per n-tile).  Evaluation pattern: quarter-warp q reads the table
             // rows of ONE pair (8 lanes x 16 bytes = a full row per access: no bank conflicts), i.e. lane
             // (q, c) evaluates channels 4c .. 4c+3 of pairs q and q + 4 of this k-step; a fixed shuffle
             // then hands the values to the lane that owns them in the B fragment (pair t, channels 4g .. 4g+3).
             const int q = lane >> 3, cch = lane & 7;
             const float *qa = stage + (8 * ks + q) * ST_STRIDE, *qb = qa + 4 * ST_STRIDE;
-            const float4 ba = *reinterpret_cast<const float4 *>(qa + 16), bb = *reinterpret_cast<const float4 *>(qb + 16);
+            const float4 ba = *reinterpret_cast<const float4 *>(qa + 16), bb = *reinterpret_cast<const float4 *>(qb + 20);
             const float *ta = tv.base + reinterpret_cast<const int *>(qa)[20] + 4 * cch;
-            const float *tb = tv.base + reinterpret_cast<const int *>(qb)[20] + 4 * cch;
+            const float *tb = tv.base + reinterpret_cast<const int *>(qb)[16] + 4 * cch;
             const float4 a0 = *reinterpret_cast<const float4 *>(ta), a1 = *reinterpret_cast<const float4 *>(ta + rs);
             const float4 a2 = *reinterpret_cast<const float4 *>(ta + 2 * rs), a3 = *reinterpret_cast<const float4 *>(ta + 3 * rs);
             const float4 b0 = *reinterpret_cast<const float4 *>(tb), b1 = *reinterpret_cast<const float4 *>(tb + rs);
@@ -332,14 +335,12 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
     auto batch = [&](int first, int n) {
         {   // lane = pair: spline basis and its derivative
             float4 ent = make_float4(1.f, 0.f, 0.f, 0.f);
-            float rinv = 1.f;
             float b[4] = {0.f, 0.f, 0.f, 0.f}, db[4] = {0.f, 0.f, 0.f, 0.f};
             int off = 0, row_index = 0;
             const bool live = lane < n;
             if (live) {
                 ent = pq[first + lane];
                 const float r = sqrtf(ent.x * ent.x + ent.y * ent.y + ent.z * ent.z);
-                rinv = 1.0f / r;
                 const int iv = spline_basis<true, float>(r, k.tab.r_min, k.tab.inv_h, k.tab.knots, b, db, k.status);
                 row_index = (__float_as_int(ent.w) >> J_BITS) * (k.tab.knots + 3) + iv;
                 off = row_index * rs;
@@ -357,9 +358,9 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
             row[0] = make_float4(b[0], b[1], b[2], b[3]);
             row[1] = make_float4(db[0], db[1], db[2], db[3]);
             reinterpret_cast<int *>(bs)[slot * BS_STRIDE + 8] = off;
-            // geometry for the projection, which runs with lane = slot (spare words of the V/T row)
-            *reinterpret_cast<float4 *>(vt + slot * VT_STRIDE + 32) = ent;
-            vt[slot * VT_STRIDE + 36] = rinv;
+            // geometry for the projection, which runs with lane = slot (spare chunk of the V/T row; the row's
+            // 16-byte chunks are stored at chunk ^ ((slot >> 2) & 1) so that lane = row reads hit eight bank groups)
+            *reinterpret_cast<float4 *>(vt + slot * VT_STRIDE + 32 + 4 * ((slot >> 2) & 1)) = ent;
         }
         __syncwarp();
         pc.mark(4);
@@ -415,7 +416,7 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
                 mma_tf32(T[0], dh[0], dh[1], dh[2], dh[3], Wh[ks][0], Wh[ks][1]);
                 mma_tf32(T[1], dh[0], dh[1], dh[2], dh[3], Wh[ks][2], Wh[ks][3]);
             }
-            float *va = vt + (16 * mt + g) * VT_STRIDE + 2 * t, *vb = va + 8 * VT_STRIDE;
+            float *va = vt + (16 * mt + g) * VT_STRIDE + ((2 * t) ^ (g & 4)), *vb = va + 8 * VT_STRIDE;   // chunk ^ ((row >> 2) & 1)
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 *reinterpret_cast<float2 *>(va + 8 * q) = make_float2(V[q][0], V[q][1]);
@@ -428,16 +429,17 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
         pc.mark(5);
         if (lane < n) {   // lane = pair: projection onto the pair vector (Eq. 10) and scatter
             float v[D_ANG], tt[D_ANG];
+            const int sw = (lane >> 2) & 1;
             const float4 *src = reinterpret_cast<const float4 *>(vt + lane * VT_STRIDE);
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                const float4 a = src[q], b = src[4 + q];
+                const float4 a = src[q ^ sw], b = src[(4 + q) ^ sw];
                 v[4 * q] = a.x; v[4 * q + 1] = a.y; v[4 * q + 2] = a.z; v[4 * q + 3] = a.w;
                 tt[4 * q] = b.x; tt[4 * q + 1] = b.y; tt[4 * q + 2] = b.z; tt[4 * q + 3] = b.w;
             }
-            const float4 ent = *reinterpret_cast<const float4 *>(vt + lane * VT_STRIDE + 32);
-            const float rinv = vt[lane * VT_STRIDE + 36];
+            const float4 ent = src[8 ^ sw];
             const float x = ent.x, y = ent.y, z = ent.z;
+            const float rinv = 1.0f / sqrtf(x * x + y * y + z * z);
             const int j = __float_as_int(ent.w) & ((1 << J_BITS) - 1);
             const float ux = x * rinv, uy = y * rinv, uz = z * rinv;
             float s, tx, ty, tz, tu;
