@@ -71,15 +71,19 @@ typedef struct {
                              1: every step of Eq. 1-10 in fp64 (Section 4.2 evaluates in double precision by default):
                                 fp64 tables (automatic knots start at 512), fp64 forces kept for the integrator,
                                 +32 bytes per atom, several times slower */
+    int enc_conditioning; /* species information given to the encoder (Section 3.2.2): 0 = the pair (s_i, s_j), C*C nets
+                             (the paper's choice); 1 = the neighbor species s_j, C nets; 2 = none, one net */
+    int head_conditioning;/* ... to the regression network: 0 = central species s_i, C nets; 1 = none, one net */
 } mlip_config;
 
 /*
  * Create a context: uploads the networks, tabulates every ordered-pair encoder
  * (Eq. 2: g = f_c(r) E(r; s_i, s_j), cosine envelope f_c) as a cubic B-spline
  * in fp64 on the device and checks it against the network.  Synchronises.
- *   enc_weights_host  [C*C] nets, net index s_i*C + s_j; each net is
+ *   enc_weights_host  [C*C] nets, net index s_i*C + s_j ([C] nets indexed s_j, or one net, with
+ *                     enc_conditioning 1 or 2); each net is
  *                     W1[h][1], b1[h], W2[h][h], b2[h], ..., Wout[k][h], bout[k], row-major [out][in]
- *   head_weights_host [C] nets; each W1[64][128], b1, W2[64][64], b2, ..., w_out[64], b_out
+ *   head_weights_host [C] nets (one with head_conditioning 1); each W1[64][128], b1, W2[64][64], b2, ..., w_out[64], b_out
  *   mass_amu_host     [C]
  * Errors: INVALID_ARG, UNSUPPORTED, OOM, CUDA, TABLE_TOLERANCE (context is still returned
  * for inspection through mlip_table_error when the tolerance fails, *out otherwise NULL).

@@ -38,7 +38,8 @@ class _CModel(ctypes.Structure):
                 ("enc_hidden", ctypes.c_int), ("enc_layers", ctypes.c_int),
                 ("head_hidden", ctypes.c_int), ("head_layers", ctypes.c_int),
                 ("r_cut", ctypes.c_double),
-                ("enc_w", ctypes.c_void_p), ("head_w", ctypes.c_void_p), ("q", ctypes.c_void_p)]
+                ("enc_w", ctypes.c_void_p), ("head_w", ctypes.c_void_p), ("q", ctypes.c_void_p),
+                ("chi_e", ctypes.c_int), ("chi_r", ctypes.c_int)]
 
 
 _lib = None
@@ -75,6 +76,8 @@ class Model:
     head_hidden: int = 64
     head_layers: int = 4
     q: np.ndarray | None = None   # override the projection matrices (tests)
+    chi_e: int = 0   # encoder conditioning (Section 3.2.2): 0 = species pair, C*C nets; 1 = neighbor species, C nets; 2 = none, 1 net
+    chi_r: int = 0   # regression-network conditioning: 0 = central species, C nets; 1 = none, 1 net
 
     def __post_init__(self):
         self.enc_w = np.ascontiguousarray(self.enc_w, dtype=np.float64)
@@ -84,7 +87,7 @@ class Model:
         self.q = np.ascontiguousarray(self.q, dtype=np.float64)
         self._c = _CModel(self.n_species, self.k, self.l_max, self.enc_hidden, self.enc_layers,
                           self.head_hidden, self.head_layers, float(self.r_cut),
-                          _p(self.enc_w), _p(self.head_w), _p(self.q))
+                          _p(self.enc_w), _p(self.head_w), _p(self.q), self.chi_e, self.chi_r)
 
     @property
     def d(self) -> int:
@@ -93,6 +96,14 @@ class Model:
     @property
     def n_inv(self) -> int:
         return (self.l_max + 1) * self.k
+
+    @property
+    def n_enc_nets(self) -> int:
+        return {0: self.n_species ** 2, 1: self.n_species, 2: 1}[self.chi_e]
+
+    @property
+    def n_head_nets(self) -> int:
+        return {0: self.n_species, 1: 1}[self.chi_r]
 
     def ref(self):
         return ctypes.byref(self._c)

@@ -51,10 +51,20 @@ typedef struct {
     int enc_hidden, enc_layers;
     int head_hidden, head_layers;
     double r_cut;
-    const double *enc_w;   /* [C*C] nets, index s_i*C + s_j */
-    const double *head_w;  /* [C] nets, index s_i */
+    const double *enc_w;   /* encoder nets, indexed by enc_net_index() */
+    const double *head_w;  /* head nets, indexed by head_net_index() */
     const double *q;       /* Q_0 .. Q_lmax, row-major, concatenated */
+    int chi_e;             /* species information given to the encoder (Section 3.2.2): 0 = pair (s_i, s_j), C*C nets;
+                              1 = neighbor species s_j, C nets; 2 = none, one net */
+    int chi_r;             /* ... to the regression network: 0 = central species s_i, C nets; 1 = none, one net */
 } oracle_model;
+
+static int enc_net_index(const oracle_model *m, int si, int sj) {
+    if (m->chi_e == 2) return 0;
+    if (m->chi_e == 1) return sj;
+    return si * m->n_species + sj;
+}
+static int head_net_index(const oracle_model *m, int si) { return m->chi_r == 1 ? 0 : si; }
 
 static int n_mono(int l) { return (l + 1) * (l + 2) / 2; }
 static int ang_dim(int l_max) { return (l_max + 1) * (l_max + 1); }
@@ -121,7 +131,7 @@ void oracle_angular(const oracle_model *m, const double u[3], double *h, double 
 /* ---- Eq. 2: encoder network of the ordered pair (s_i, s_j): y(r) and dy/dr ---- */
 void oracle_encoder(const oracle_model *m, int si, int sj, double r, double *y, double *dy) {
     const int H = m->enc_hidden, K = m->k;
-    const double *w = m->enc_w + (size_t)(si * m->n_species + sj) * enc_net_size(m);
+    const double *w = m->enc_w + (size_t)enc_net_index(m, si, sj) * enc_net_size(m);
     double a[H], da[H], pre[H], dpre[H];
     const double *W = w, *b = w + H;
     for (int o = 0; o < H; ++o) {
@@ -171,7 +181,7 @@ void oracle_radial(const oracle_model *m, int si, int sj, double r, double *g, d
 /* ---- Eq. 6: head of species s: E = R(G); optionally dE/dG ---- */
 double oracle_head(const oracle_model *m, int s, const double *G, double *dG /* may be NULL */) {
     const int H = m->head_hidden, L = m->head_layers, n_in = (m->l_max + 1) * m->k;
-    const double *w0 = m->head_w + (size_t)s * head_net_size(m);
+    const double *w0 = m->head_w + (size_t)head_net_index(m, s) * head_net_size(m);
     double pre[L][H], z[H];
     const double *w = w0;
     for (int o = 0; o < H; ++o) {

@@ -3,6 +3,7 @@
 #include <math.h>
 #include <new>
 #include <string.h>
+#include <vector>
 
 #include "common.cuh"
 #include "scan.cuh"
@@ -121,7 +122,35 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
     if (cfg->head_hidden != HEAD_H || cfg->head_layers != HEAD_L) return fail(nullptr, MLIP_ERR_UNSUPPORTED, "only a 4 x 64 head is compiled in");
     if (cfg->enc_hidden < 1 || cfg->enc_layers < 1) return fail(nullptr, MLIP_ERR_INVALID_ARG, "bad encoder shape");
     if (!(cfg->r_cut > 0.0) || !(cfg->skin >= 0.0)) return fail(nullptr, MLIP_ERR_INVALID_ARG, "bad r_cut or skin");
-    if (n_head != (size_t)cfg->n_species * HEAD_NET) return fail(nullptr, MLIP_ERR_INVALID_ARG, "head weight count does not match the shape");
+    if (cfg->enc_conditioning < 0 || cfg->enc_conditioning > 2 || cfg->head_conditioning < 0 || cfg->head_conditioning > 1)
+        return fail(nullptr, MLIP_ERR_INVALID_ARG, "bad enc_conditioning or head_conditioning");
+    // Species conditioning (Section 3.2.2): the kernels always index C*C encoder tables and C heads; the variants
+    // with fewer networks are expanded here by repeating the shared ones.
+    const int C = cfg->n_species;
+    const size_t enc_net = (size_t)2 * cfg->enc_hidden + (size_t)(cfg->enc_layers - 1) * ((size_t)cfg->enc_hidden * cfg->enc_hidden + cfg->enc_hidden) +
+                           (size_t)cfg->k * cfg->enc_hidden + cfg->k;
+    const size_t n_enc_nets = cfg->enc_conditioning == 0 ? (size_t)C * C : cfg->enc_conditioning == 1 ? (size_t)C : 1;
+    const size_t n_head_nets = cfg->head_conditioning == 0 ? (size_t)C : 1;
+    if (n_enc != n_enc_nets * enc_net) return fail(nullptr, MLIP_ERR_INVALID_ARG, "encoder weight count does not match shape and conditioning");
+    if (n_head != n_head_nets * HEAD_NET) return fail(nullptr, MLIP_ERR_INVALID_ARG, "head weight count does not match shape and conditioning");
+    std::vector<double> enc_full, head_full;
+    try {
+        if (cfg->enc_conditioning != 0) enc_full.resize((size_t)C * C * enc_net);
+        if (cfg->head_conditioning != 0) head_full.resize((size_t)C * HEAD_NET);
+    } catch (const std::bad_alloc &) {
+        return fail(nullptr, MLIP_ERR_OOM, "host allocation failed");
+    }
+    if (cfg->enc_conditioning != 0) {
+        for (int si = 0; si < C; ++si)
+            for (int sj = 0; sj < C; ++sj)
+                memcpy(&enc_full[((size_t)si * C + sj) * enc_net], enc_w + (cfg->enc_conditioning == 1 ? (size_t)sj : 0) * enc_net, sizeof(double) * enc_net);
+        enc_w = enc_full.data();
+        n_enc = enc_full.size();
+    }
+    if (cfg->head_conditioning != 0) {
+        for (int si = 0; si < C; ++si) memcpy(&head_full[(size_t)si * HEAD_NET], head_w, sizeof(double) * HEAD_NET);
+        head_w = head_full.data();
+    }
     for (int s = 0; s < cfg->n_species; ++s)
         if (!(mass[s] > 0.0)) return fail(nullptr, MLIP_ERR_INVALID_ARG, "mass must be positive");
     if (cfg->precision != 0 && cfg->precision != 1) return fail(nullptr, MLIP_ERR_INVALID_ARG, "precision must be 0 (fp32) or 1 (fp64)");

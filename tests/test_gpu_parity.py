@@ -243,3 +243,30 @@ def test_dense_system_beyond_the_pair_queue_matches_oracle():
     assert abs(float(out["energy"].cpu()) - ref["energy"]) <= E_RTOL * abs(ref["energy"])
     assert np.abs(out["forces"].cpu().numpy() - ref["forces"]).max() <= F_ATOL * scale
     assert np.abs(out["e_atom"].cpu().numpy() - ref["e_atom"]).max() <= 2e-5 * max(1.0, np.abs(ref["e_atom"]).max())
+
+
+@pytest.mark.parametrize("chi_e,chi_r,precision", [(1, 0, 0), (2, 1, 0), (0, 1, 0), (1, 1, 1)])
+def test_species_conditioning_variants_match_oracle(chi_e, chi_r, precision):
+    """Section 3.2.2: encoder conditioned on the neighbor species only or on nothing, universal regression network."""
+    import paper_2608_16329_b200 as mlip
+    from paper_2608_16329_b200 import workloads as wl
+    C = 3
+    w = wl.make_workload(3, n_cells=5)
+    enc, head = wl.workload_weights(3, C)
+    ne, nh = wl.enc_net_size(), wl.head_net_size(128)
+    enc_small = enc.reshape(C * C, ne)[:{0: C * C, 1: C, 2: 1}[chi_e]].ravel()
+    head_small = head.reshape(C, nh)[:{0: C, 1: 1}[chi_r]].ravel()
+    model = oracle.Model(C, w.r_cut, enc_small, head_small, chi_e=chi_e, chi_r=chi_r)
+    pot = mlip.Potential(C, w.r_cut, 1.0, enc_small, head_small, w.masses, precision=precision,
+                         enc_conditioning=chi_e, head_conditioning=chi_r)
+    pot.build_neighbors(w.pos, w.species, w.box)
+    out = pot.compute()
+    pot.sync_status()
+    ref = oracle.evaluate(model, w.pos, w.species, w.box)
+    e_tol, f_tol = (1e-10, 2e-9) if precision == 1 else (E_RTOL, F_ATOL)
+    assert abs(float(out["energy"].cpu()) - ref["energy"]) <= e_tol * abs(ref["energy"])
+    assert np.abs(out["forces"].cpu().numpy() - ref["forces"]).max() <= f_tol
+    # a weight blob of the wrong count for the conditioning is refused
+    with pytest.raises(mlip.MlipError) as err:
+        mlip.Potential(C, w.r_cut, 1.0, enc, head, w.masses, enc_conditioning=2 if chi_e != 2 else 1, head_conditioning=chi_r)
+    assert err.value.code == mlip.binding.CODES["MLIP_ERR_INVALID_ARG"]
