@@ -172,12 +172,21 @@ int mlip_compute_host(mlip_ctx *ctx, int64_t n_atoms, const double *pos_host, co
                       double *virial_host);
 
 /*
- * n_steps of velocity-Verlet NVE with time step dt_fs; lists are rebuilt every
- * `rebuild_every` steps of the context's running step counter (0 = never).
+ * n_steps of velocity-Verlet NVE with time step dt_fs.  List rebuilds:
+ *   rebuild_every > 0   every `rebuild_every` steps of the context's running step counter
+ *   rebuild_every = 0   never
+ *   rebuild_every < 0   displacement-triggered, the policy of the paper's MD runs (Section 4.2: the criterion is
+ *                       checked every five steps and the list rebuilt only when required): every -rebuild_every
+ *                       steps the host reads a device flag (one stream synchronisation) and rebuilds if some atom
+ *                       has moved more than 0.8 * skin/2 since the last build.  The hard limit skin/2 still raises
+ *                       MLIP_ERR_SKIN_EXCEEDED in mlip_sync_status().
  * Needs a prior mlip_build_neighbors; evaluates forces first if none are current.
- * Does not synchronise; device-side problems surface in mlip_sync_status().
+ * Does not synchronise unless rebuild_every < 0; device-side problems surface in mlip_sync_status().
  */
 int mlip_step(mlip_ctx *ctx, int n_steps, double dt_fs, int rebuild_every, void *stream);
+
+/* Number of list builds since mlip_create (initial builds, in-step rebuilds, host-entry rebuilds). */
+int mlip_get_rebuilds(const mlip_ctx *ctx, int64_t *n_builds_host);
 
 /* Positions / velocities in the caller's order (dev [N][3] double, may be NULL); step counter (host). */
 int mlip_get_state(mlip_ctx *ctx, double *pos, double *vel, int64_t *step_host, void *stream);

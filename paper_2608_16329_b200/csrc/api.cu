@@ -180,19 +180,20 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
         if ((rc = dev_alloc(c, &c->acc, (size_t)ACC_COUNT)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->pair_counter, 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->status, 1)) != MLIP_OK) break;
+        if ((rc = dev_alloc(c, &c->rebuild_flag, 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->tile_counter, (size_t)MAX_SPECIES)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->species_start, (size_t)MAX_SPECIES + 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->stage_out, 10)) != MLIP_OK) break;
         if (cudaMallocHost((void **)&c->status_host, sizeof(int)) != cudaSuccess ||
             cudaMallocHost((void **)&c->total_host, sizeof(int64_t)) != cudaSuccess ||
-            false) {
+            cudaMallocHost((void **)&c->rebuild_host, sizeof(int)) != cudaSuccess) {
             rc = MLIP_ERR_CUDA; c->err = "pinned host allocation failed"; break;
         }
         bool ev_ok = true;
         for (int q = 0; q < 2 * mlip_ctx::EV_POOL; ++q) ev_ok = ev_ok && cudaEventCreate(&c->ev[q]) == cudaSuccess;
         if (!ev_ok) { rc = MLIP_ERR_CUDA; c->err = "event creation failed"; break; }
         if (cudaMemcpy(c->mass, mass, sizeof(double) * cfg->n_species, cudaMemcpyHostToDevice) != cudaSuccess ||
-            cudaMemset(c->status, 0, sizeof(int)) != cudaSuccess || cudaMemset(c->acc, 0, sizeof(double) * ACC_COUNT) != cudaSuccess) {
+            cudaMemset(c->status, 0, sizeof(int)) != cudaSuccess || cudaMemset(c->rebuild_flag, 0, sizeof(int)) != cudaSuccess || cudaMemset(c->acc, 0, sizeof(double) * ACC_COUNT) != cudaSuccess) {
             rc = MLIP_ERR_CUDA; c->err = "initial upload failed"; break;
         }
         if ((rc = f64 ? upload_head_f64(c, head_w) : upload_head(c, head_w)) != MLIP_OK) break;
@@ -238,8 +239,10 @@ int mlip_build_neighbors(mlip_ctx *c, int64_t n, const double *pos, const int32_
     rc = launch_build(c, true, s);
     c->vel_src = keep;
     if (rc != MLIP_OK) return rc;
+    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->rebuild_flag, 0, sizeof(int), s));
     c->built = true;
     c->forces_current = false;
+    c->n_builds += 1;
     return MLIP_OK;
 }
 
@@ -341,7 +344,7 @@ int mlip_compute_host(mlip_ctx *c, int64_t n, const double *pos_host, const int3
 }
 
 int mlip_step(mlip_ctx *c, int n_steps, double dt, int rebuild_every, void *stream) {
-    if (!c || n_steps < 0 || !(dt > 0.0) || rebuild_every < 0) return MLIP_ERR_INVALID_ARG;
+    if (!c || n_steps < 0 || !(dt > 0.0)) return MLIP_ERR_INVALID_ARG;
     if (!c->built) return fail(c, MLIP_ERR_NOT_BUILT, "no neighbor lists yet");
     cudaStream_t s = (cudaStream_t)stream;
     c->last_stream = s;
@@ -353,7 +356,15 @@ int mlip_step(mlip_ctx *c, int n_steps, double dt, int rebuild_every, void *stre
     for (int it = 0; it < n_steps; ++it) {
         if ((rc = launch_kick_drift(c, dt, s)) != MLIP_OK) return rc;
         c->step += 1;
-        if (rebuild_every > 0 && c->step % rebuild_every == 0) {
+        bool rebuild = rebuild_every > 0 && c->step % rebuild_every == 0;
+        if (rebuild_every < 0 && c->step % -rebuild_every == 0) {   // displacement-triggered: ask the device
+            MLIP_CUDA_TRY(c, cudaMemcpyAsync(c->rebuild_host, c->rebuild_flag, sizeof(int), cudaMemcpyDeviceToHost, s));
+            MLIP_CUDA_TRY(c, cudaStreamSynchronize(s));
+            rebuild = *c->rebuild_host != 0;
+        }
+        if (rebuild) {
+            MLIP_CUDA_TRY(c, cudaMemsetAsync(c->rebuild_flag, 0, sizeof(int), s));
+            c->n_builds += 1;
             std::swap(c->pos4, c->pos4_src);
             std::swap(c->vel, c->vel_src);
             std::swap(c->user_of, c->user_src);
@@ -371,6 +382,12 @@ int mlip_get_state(mlip_ctx *c, double *pos, double *vel, int64_t *step_host, vo
     c->last_stream = (cudaStream_t)stream;
     if (step_host) *step_host = c->step;
     if (pos || vel) return launch_get_state(c, pos, vel, (cudaStream_t)stream);
+    return MLIP_OK;
+}
+
+int mlip_get_rebuilds(const mlip_ctx *c, int64_t *n_builds_host) {
+    if (!c || !n_builds_host) return MLIP_ERR_INVALID_ARG;
+    *n_builds_host = c->n_builds;
     return MLIP_OK;
 }
 
@@ -454,11 +471,12 @@ void mlip_destroy(mlip_ctx *c) {
     free_cells(c);
     cudaFree(c->nbr); cudaFree(c->scan_tmp); cudaFree(c->head_w); cudaFree(c->table); cudaFree(c->mass);
     cudaFree(c->head_w_d); cudaFree(c->table_d);
-    cudaFree(c->acc); cudaFree(c->pair_counter); cudaFree(c->status); cudaFree(c->tile_counter);
+    cudaFree(c->acc); cudaFree(c->pair_counter); cudaFree(c->status); cudaFree(c->rebuild_flag); cudaFree(c->tile_counter);
     cudaFree(c->species_start); cudaFree(c->stage_pos); cudaFree(c->stage_species); cudaFree(c->stage_force);
     cudaFree(c->stage_out);
     if (c->status_host) cudaFreeHost(c->status_host);
     if (c->total_host) cudaFreeHost(c->total_host);
+    if (c->rebuild_host) cudaFreeHost(c->rebuild_host);
     for (int q = 0; q < 2 * mlip_ctx::EV_POOL; ++q)
         if (c->ev[q]) cudaEventDestroy(c->ev[q]);
     delete c;

@@ -98,6 +98,9 @@ struct mlip_ctx {
     double *acc = nullptr;         // [ACC_COUNT]
     unsigned long long *pair_counter = nullptr;
     int *status = nullptr;         // device status word
+    int *rebuild_flag = nullptr;   // set when an atom has moved beyond the rebuild trigger; pinned copy in rebuild_host
+    int *rebuild_host = nullptr;
+    int64_t n_builds = 0;
     int *tile_counter = nullptr;   // [MAX_SPECIES] dynamic tile scheduler, one counter per central species
     int *status_host = nullptr;    // pinned
     int64_t *total_host = nullptr; // pinned

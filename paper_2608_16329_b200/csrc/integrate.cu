@@ -16,7 +16,8 @@ __device__ __forceinline__ double3 load_force(const float4 *__restrict__ force, 
 // v += dt/2 a;  x += dt v;  wrap into [0, L);  track the displacement since the last list build.
 __global__ void k_kick_drift(int64_t n, double dt, CellGrid g, const double *__restrict__ mass, float skin_half2,
                              double4 *__restrict__ pos4, double *__restrict__ vel, const float4 *__restrict__ force,
-                             const double *__restrict__ force_d, float *__restrict__ disp, int *status) {
+                             const double *__restrict__ force_d, float *__restrict__ disp, int *status, float trigger2,
+                             int *rebuild_flag) {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     double4 p = pos4[i];
@@ -37,6 +38,7 @@ __global__ void k_kick_drift(int64_t n, double dt, CellGrid g, const double *__r
         if (!(x[a] >= 0.0 && x[a] < L)) x[a] = 0.0;   // -eps + L rounds to L; NaN is reported below
     }
     if (!(d2 <= skin_half2)) atomicOr(status, d2 == d2 ? FLAG_SKIN_EXCEEDED : FLAG_NONFINITE);
+    if (d2 > trigger2) *rebuild_flag = 1;   // same value from every writer
     pos4[i] = make_double4(x[0], x[1], x[2], p.w);
 }
 
@@ -130,7 +132,8 @@ static inline unsigned nb(int64_t n) { return (unsigned)((n + 255) / 256); }
 static inline float skin_half2(const mlip_ctx *c) { float h = 0.5f * (float)c->cfg.skin; return h * h; }
 
 int launch_kick_drift(mlip_ctx *c, double dt, cudaStream_t s) {
-    k_kick_drift<<<nb(c->n), 256, 0, s>>>(c->n, dt, c->grid, c->mass, skin_half2(c), c->pos4, c->vel, c->force, c->force_d, c->disp, c->status);
+    k_kick_drift<<<nb(c->n), 256, 0, s>>>(c->n, dt, c->grid, c->mass, skin_half2(c), c->pos4, c->vel, c->force, c->force_d, c->disp, c->status,
+                                               0.64f * skin_half2(c), c->rebuild_flag);
     c->launches += 1;
     MLIP_CUDA_TRY(c, cudaGetLastError());
     return MLIP_OK;

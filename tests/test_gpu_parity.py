@@ -270,3 +270,30 @@ def test_species_conditioning_variants_match_oracle(chi_e, chi_r, precision):
     with pytest.raises(mlip.MlipError) as err:
         mlip.Potential(C, w.r_cut, 1.0, enc, head, w.masses, enc_conditioning=2 if chi_e != 2 else 1, head_conditioning=chi_r)
     assert err.value.code == mlip.binding.CODES["MLIP_ERR_INVALID_ARG"]
+
+
+def test_displacement_triggered_rebuilds_keep_the_lists_valid():
+    """The paper's MD policy (Section 4.2): check the criterion every few steps, rebuild only when an atom has moved far
+    enough.  The lists in use must at every moment hold all pairs inside r_cut."""
+    w, model, pot = make_pair(3, 8, 1.0)
+    pot.build_neighbors(w.pos, w.species, w.box)
+    pot.set_velocities(w.vel)
+    pot.compute()
+    e0 = pot.energies().cpu().numpy()
+    assert pot.rebuilds() == 1
+    pot.step(60, 1.0, -2)
+    assert pot.sync_status(raise_on_error=False) == 0
+    n_rebuilds = pot.rebuilds() - 1
+    assert 2 <= n_rebuilds < 20                      # triggered, but not at every check
+    pos, vel, step = pot.state()
+    e1 = pot.energies().cpu().numpy()
+    exchanged = abs(e1[1] - e0[1])
+    assert abs(e1.sum() - e0.sum()) < 0.02 * exchanged + 2e-6 * abs(e0[0])
+    seg, nbr = pot.neighbors()
+    seg, nbr = seg.cpu().numpy(), nbr.cpu().numpy().astype(np.int64)
+    n, C = w.n_atoms, w.n_species
+    have = (np.repeat(np.arange(n * C), np.diff(seg)) // C) * n + nbr
+    ref = oracle.neighbors(pos.cpu().numpy(), w.species, C, w.box, w.r_cut)
+    want = (np.repeat(np.arange(n * C), np.diff(ref.seg_ptr)) // C) * n + ref.nbr.astype(np.int64)
+    assert np.isin(want, have).all()
+    assert have.size > want.size                     # the lists carry the skin shell as well
