@@ -63,6 +63,8 @@ def parse_args():
                          "3-species alloy and ionic stand-ins at their full sizes (extra data points, not the contract line)")
     ap.add_argument("--precision", default="f32", choices=["f32", "f64"],
                     help="f64 runs the double-precision evaluation path instead (an extra data point, not the contract line)")
+    ap.add_argument("--k", type=int, default=32, choices=[16, 32, 64], help="radial channels (other than 32: --precision f64 only)")
+    ap.add_argument("--lmax", type=int, default=3, choices=[1, 2, 3], help="angular order (other than 3: --precision f64 only)")
     ap.add_argument("--sweep", default="", help="comma-separated FCC cell counts: size sweep of the 6-species workload "
                     "(inputs generated on the device), one JSON line per size; not the contract line")
     return ap.parse_args()
@@ -280,11 +282,17 @@ def main():
 
     cfg = args.cfg
     w = wl.make_workload(cfg, n_cells=args.cells if cfg == CFG else None, seed=wl.BASE_SEED + cfg + 17 * rank)
-    enc, head = wl.workload_weights(cfg, w.n_species)
+    default_shape = args.k == 32 and args.lmax == 3
+    if default_shape:
+        enc, head = wl.workload_weights(cfg, w.n_species)
+    else:   # descriptor-shape variants of the paper's ablations: same recipe, networks of that shape
+        enc, head = wl.make_weights(w.n_species, wl.BASE_SEED + cfg + 1000, wl.ENC_OUT_SCALE[cfg], wl.HEAD_OUT_SCALE[cfg],
+                                    k=args.k, l_max=args.lmax)
     rebuild_every = REBUILD_EVERY if cfg != 4 else 3   # the ionic stand-in is far from equilibrium under random weights
     n = w.n_atoms
     f64 = args.precision == "f64"
-    pot = mlip.Potential(w.n_species, w.r_cut, w.skin, enc, head, w.masses, device=local_rank, precision=1 if f64 else 0)
+    pot = mlip.Potential(w.n_species, w.r_cut, w.skin, enc, head, w.masses, device=local_rank, precision=1 if f64 else 0,
+                         k=args.k, l_max=args.lmax)
     table_err = mlip.mlip_table_error(pot.ctx)
 
     # ---- device-resident run: inputs already in HBM when timing starts ----
@@ -357,7 +365,12 @@ def main():
         peak_tflops = n_sm * lanes * 2 * sm_max * 1e6 / 1e12
         pairs = counters["pairs_in_cutoff"]
         entries = counters["list_entries"]
-        flop = FLOP_PER_PAIR * pairs + FLOP_PER_SKIN_ENTRY * max(entries - pairs, 0) + FLOP_PER_ATOM * n
+        flop_pair, flop_atom = FLOP_PER_PAIR, FLOP_PER_ATOM
+        if not default_shape:   # the same count written out in k and d = (l_max + 1)^2
+            d_ang, n_inv = (args.lmax + 1) ** 2, (args.lmax + 1) * args.k
+            flop_pair = 60 + 150 * d_ang / 16 + 512 * args.k / 32 + 6 * d_ang * args.k + 168 * d_ang / 16
+            flop_atom = 3 * d_ang * args.k + 4 * (n_inv * 64 + 3 * 64 * 64) + 256 + 5000
+        flop = flop_pair * pairs + FLOP_PER_SKIN_ENTRY * max(entries - pairs, 0) + flop_atom * n
         k_avg_ms = k_ms / max(k_launches, 1)
         achieved = flop / (k_avg_ms * 1e-3) / 1e12
         roofline = {"bound": "alu", "kernel": "k_mega_f64" if f64 else "k_mega", "achieved": achieved, "peak": peak_tflops, "unit": "TFLOP/s",
@@ -375,7 +388,8 @@ def main():
                 "ms_per_step": ms_max / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": args.precision, "data": "synthetic",
                 "config": {"workload": f"cfg{cfg} {w.name}: {n} atoms, {w.n_species} species, r_cut 6 A, skin 1 A, "
-                                       f"NVE dt 1 fs, list rebuild every {rebuild_every} steps",
+                                       f"NVE dt 1 fs, list rebuild every {rebuild_every} steps"
+                                       + ("" if default_shape else f", k = {args.k}, l_max = {args.lmax}"),
                            "atoms_per_gpu": n, "parallelism": "replicas" if world > 1 else "single",
                            "l2": "inputs larger than L2 (positions + lists = %.1f GB per GPU)" % ((32 * n + 4 * entries) / 1e9)},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": counters["launches"] - launches0,

@@ -22,7 +22,8 @@
  *     Calls enqueue work and return without synchronising unless stated.
  *   - Units: Angstrom, eV, amu, fs.  Atom order of every array argument is the
  *     caller's; the library keeps its own cell-sorted order internally.
- *   - Only k = 32 radial channels and l_max = 3 (d = 16) are compiled in; the
+ *   - The fp32 path is compiled for k = 32 radial channels and l_max = 3 (d = 16), the paper's production
+ *     shape; the fp64 path (precision = 1) also for k in {16, 32, 64} x l_max in {1, 2, 3}.  The
  *     encoder is 1 -> enc_hidden x enc_layers -> k, the head is
  *     (l_max+1) k -> head_hidden x head_layers -> 1 with head_hidden = 64,
  *     head_layers = 4 (Section 4.1.3), SiLU, identity skips around hidden
@@ -59,8 +60,8 @@ typedef struct {
     int n_species;        /* C, 1..8 */
     double r_cut;         /* Angstrom */
     double skin;          /* list radius = r_cut + skin */
-    int k;                /* 32 */
-    int l_max;            /* 3 */
+    int k;                /* 32 (precision 1: 16, 32 or 64) */
+    int l_max;            /* 3 (precision 1: 1, 2 or 3) */
     int enc_hidden, enc_layers;    /* e.g. 128, 3 */
     int head_hidden, head_layers;  /* 64, 4 */
     int table_knots;      /* intervals of the radial table on [table_r_min, r_cut]; 0 = automatic: 64, doubled until table_tol holds */

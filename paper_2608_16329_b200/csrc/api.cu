@@ -118,7 +118,12 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
     *out = nullptr;
     if (!cfg || !enc_w || !head_w || !mass) return fail(nullptr, MLIP_ERR_INVALID_ARG, "NULL argument");
     if (cfg->n_species < 1 || cfg->n_species > MAX_SPECIES) return fail(nullptr, MLIP_ERR_UNSUPPORTED, "n_species must be 1..8");
-    if (cfg->k != K_RADIAL || cfg->l_max != 3) return fail(nullptr, MLIP_ERR_UNSUPPORTED, "only k = 32, l_max = 3 are compiled in");
+    if (cfg->precision == 1) {
+        if (!f64_shape_supported(cfg->k, cfg->l_max))
+            return fail(nullptr, MLIP_ERR_UNSUPPORTED, "the fp64 path is compiled for k in {16, 32, 64} and l_max in {1, 2, 3}");
+    } else if (cfg->k != K_RADIAL || cfg->l_max != 3) {
+        return fail(nullptr, MLIP_ERR_UNSUPPORTED, "the fp32 path is compiled for k = 32, l_max = 3 only (other shapes: precision = 1)");
+    }
     if (cfg->head_hidden != HEAD_H || cfg->head_layers != HEAD_L) return fail(nullptr, MLIP_ERR_UNSUPPORTED, "only a 4 x 64 head is compiled in");
     if (cfg->enc_hidden < 1 || cfg->enc_layers < 1) return fail(nullptr, MLIP_ERR_INVALID_ARG, "bad encoder shape");
     if (!(cfg->r_cut > 0.0) || !(cfg->skin >= 0.0)) return fail(nullptr, MLIP_ERR_INVALID_ARG, "bad r_cut or skin");
@@ -132,11 +137,12 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
     const size_t n_enc_nets = cfg->enc_conditioning == 0 ? (size_t)C * C : cfg->enc_conditioning == 1 ? (size_t)C : 1;
     const size_t n_head_nets = cfg->head_conditioning == 0 ? (size_t)C : 1;
     if (n_enc != n_enc_nets * enc_net) return fail(nullptr, MLIP_ERR_INVALID_ARG, "encoder weight count does not match shape and conditioning");
-    if (n_head != n_head_nets * HEAD_NET) return fail(nullptr, MLIP_ERR_INVALID_ARG, "head weight count does not match shape and conditioning");
+    const size_t head_net = head_net_size((cfg->l_max + 1) * cfg->k);
+    if (n_head != n_head_nets * head_net) return fail(nullptr, MLIP_ERR_INVALID_ARG, "head weight count does not match shape and conditioning");
     std::vector<double> enc_full, head_full;
     try {
         if (cfg->enc_conditioning != 0) enc_full.resize((size_t)C * C * enc_net);
-        if (cfg->head_conditioning != 0) head_full.resize((size_t)C * HEAD_NET);
+        if (cfg->head_conditioning != 0) head_full.resize((size_t)C * head_net);
     } catch (const std::bad_alloc &) {
         return fail(nullptr, MLIP_ERR_OOM, "host allocation failed");
     }
@@ -148,7 +154,7 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
         n_enc = enc_full.size();
     }
     if (cfg->head_conditioning != 0) {
-        for (int si = 0; si < C; ++si) memcpy(&head_full[(size_t)si * HEAD_NET], head_w, sizeof(double) * HEAD_NET);
+        for (int si = 0; si < C; ++si) memcpy(&head_full[(size_t)si * head_net], head_w, sizeof(double) * head_net);
         head_w = head_full.data();
     }
     for (int s = 0; s < cfg->n_species; ++s)

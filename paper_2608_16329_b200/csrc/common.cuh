@@ -15,7 +15,11 @@ constexpr int N_INV = 128;     // (l_max + 1) * k invariants (Eq. 5)
 constexpr int HEAD_H = 64;     // head width (Section 4.1.3)
 constexpr int HEAD_L = 4;      // head hidden layers
 constexpr int MAX_SPECIES = 8;
-constexpr int HEAD_NET = N_INV * HEAD_H + HEAD_H + (HEAD_L - 1) * (HEAD_H * HEAD_H + HEAD_H) + HEAD_H + 1;
+constexpr int MAX_K = 64;      // widest radial feature vector of the fp64 path's shape variants
+constexpr size_t head_net_size(int n_inv) {   // doubles per regression network in the caller's layout
+    return (size_t)n_inv * HEAD_H + HEAD_H + (size_t)(HEAD_L - 1) * (HEAD_H * HEAD_H + HEAD_H) + HEAD_H + 1;
+}
+constexpr int HEAD_NET = (int)head_net_size(N_INV);
 
 // 1 eV/(Angstrom amu) in Angstrom/fs^2
 constexpr double ACC_UNIT = 1.602176634e-19 / 1.66053906660e-27 * 1e-10;
@@ -145,6 +149,7 @@ int launch_megakernel(mlip_ctx *c, cudaStream_t s);
 // megakernel_f64.cu
 int upload_head_f64(mlip_ctx *c, const double *head_w_host);
 int launch_megakernel_f64(mlip_ctx *c, cudaStream_t s);
+bool f64_shape_supported(int k, int l_max);
 // integrate.cu
 int launch_kick_drift(mlip_ctx *c, double dt, cudaStream_t s);
 int launch_kick(mlip_ctx *c, double dt, cudaStream_t s);

@@ -59,7 +59,7 @@ __global__ void k_table_sample(const double *__restrict__ enc_w, size_t net_size
     if (t >= n_nets * n_points) return;
     int net = t / n_points, p = t % n_points;
     double r = p == n_points - 1 ? r_last : r0 + p * step;
-    double g[K_RADIAL], dg[K_RADIAL];
+    double g[MAX_K], dg[MAX_K];
     eval_radial(enc_w + (size_t)net * net_size, sh, r, g, dg);
     for (int c = 0; c < sh.k; ++c) {
         val[((size_t)net * n_points + p) * sh.k + c] = g[c];

@@ -98,3 +98,36 @@ def test_fp64_dense_neighborhood_matches_oracle():
     ref = oracle.evaluate(model, pos, w.species, w.box)
     assert abs(float(out["energy"].cpu()) - ref["energy"]) <= E_RTOL_F64 * abs(ref["energy"])
     assert np.abs(out["forces"].cpu().numpy() - ref["forces"]).max() <= F_ATOL_F64
+
+
+@pytest.mark.parametrize("k,l_max", [(16, 3), (64, 3), (32, 1), (32, 2), (16, 2), (64, 1)])
+def test_fp64_descriptor_shape_variants_match_oracle(k, l_max):
+    """Radial width k and angular order l_max of the paper's ablations (Tables 6 and 7, Fig. 4(c)); the fp64 kernel is
+    compiled for each shape, the oracle is generic in both."""
+    import paper_2608_16329_b200 as mlip
+    from paper_2608_16329_b200 import workloads as wl
+    C = 3
+    w = wl.make_workload(3, n_cells=5)
+    enc, head = wl.make_weights(C, 77, wl.ENC_OUT_SCALE[3], wl.HEAD_OUT_SCALE[3], k=k, l_max=l_max)
+    model = oracle.Model(C, w.r_cut, enc, head, k=k, l_max=l_max)
+    pot = mlip.Potential(C, w.r_cut, 1.0, enc, head, w.masses, precision=1, k=k, l_max=l_max)
+    pot.build_neighbors(w.pos, w.species, w.box)
+    out = pot.compute(want_e_atom=True)
+    pot.sync_status()
+    ref = oracle.evaluate(model, w.pos, w.species, w.box)
+    e = float(out["energy"].cpu())
+    f = out["forces"].cpu().numpy()
+    print(f"k={k} l_max={l_max}: rel dE={abs(e - ref['energy']) / abs(ref['energy']):.2e} max|dF|={np.abs(f - ref['forces']).max():.2e}")
+    assert abs(e - ref["energy"]) <= E_RTOL_F64 * abs(ref["energy"])
+    assert np.abs(f - ref["forces"]).max() <= F_ATOL_F64
+    assert np.abs(out["e_atom"].cpu().numpy() - ref["e_atom"]).max() <= 1e-9 * max(1.0, np.abs(ref["e_atom"]).max())
+    assert np.abs(out["virial"].cpu().numpy().reshape(3, 3) - ref["virial"]).max() <= 1e-9 * np.abs(ref["virial"]).max()
+
+
+def test_other_shapes_are_refused_by_the_fp32_path():
+    import paper_2608_16329_b200 as mlip
+    from paper_2608_16329_b200 import workloads as wl
+    enc, head = wl.make_weights(1, 3, k=16, l_max=3)
+    with pytest.raises(mlip.MlipError) as err:
+        mlip.Potential(1, 6.0, 1.0, enc, head, np.array([50.0]), k=16, l_max=3)
+    assert err.value.code == mlip.binding.CODES["MLIP_ERR_UNSUPPORTED"]
