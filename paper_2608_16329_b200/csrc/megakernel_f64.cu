@@ -1,18 +1,20 @@
 // Double-precision evaluation path (`precision = 1`): the same fused pass as megakernel.cu --
 // encoding (Eq. 1-5), regression (Eq. 6) and derivation (Eq. 7-10) of an atom back to back with
-// nothing per pair or per atom written to device memory except forces and E_i -- in plain fp64
-// arithmetic.  Section 4.2 evaluates the potential in double precision by default; this path is
-// for validation and for runs that want that accuracy.  The tensor pipe has no fp64 mode worth
-// the operand shuffling at these shapes, so every contraction here is DFMA work:
+// nothing per pair or per atom written to device memory except forces and E_i -- in fp64.
+// Section 4.2 evaluates the potential in double precision by default; this path is for validation
+// and for runs that want that accuracy.
 //
-//   one warp = one atom at a time (atoms in (species, cell) order, static stride over warps)
-//   encoding    lane = list entry for geometry, harmonics and spline basis; then lane = channel
-//               for g (Eq. 2) and the moment P (Eq. 4), the pair's h / basis handed over in
-//               shared memory
-//   regression  lane = neuron (and neuron + 32); weights read from L2 (a transposed copy for the
-//               forward pass keeps both directions coalesced)
-//   derivation  lane = pair, after compacting the pairs inside r_cut: v = W g, t = W g' against
-//               W_i in shared memory, projection onto the pair vector, fp64 atomics for f_j
+//   CTA = 8 warps = a tile of 8 atoms of one central species (atoms in (species, cell) order)
+//   encoding    one warp per atom: lane = list entry for geometry, harmonics and spline basis; then
+//               lane = channel for g (Eq. 2) and the moment P (Eq. 4), the pair's h / basis handed
+//               over in shared memory; plain DFMA
+//   regression  the whole CTA on the tile: every layer is W [64 x in] times the tile's activations
+//               [in x 8 atoms] on the fp64 tensor pipe (mma.sync m8n8k4, IEEE fp64 FMA chains), warp =
+//               8 rows of W, so each weight is read from L2 once per tile instead of once per atom;
+//               the reverse pass uses the same row-major weights as the transposed operand
+//   derivation  one warp per atom, lane = pair after compacting the pairs inside r_cut: v = W g,
+//               t = W g' against W_i in shared memory, projection onto the pair vector, fp64
+//               atomics for f_j; table rows are read a 32-byte sector at a time
 //
 // The radial tables are the same clamped cubic B-splines as in the fp32 path but with fp64
 // coefficients and enough knots for ~1e-11 relative error; they stay in global memory (L2).
@@ -28,18 +30,17 @@
 
 namespace mlip {
 
-constexpr int F64_WARPS = 8;
+constexpr int F64_TILE = 8;         // atoms per tile = warps per CTA = columns of the tensor-pipe tile
 constexpr int F64_ST = 22;          // hand-over row: 16 h, 4 b, table offset, pad
+constexpr int F64_YS = HEAD_H + 4;  // activation row stride: 4 mod 16 keeps the B-fragment reads conflict-free
 
-// per-species head block (doubles) for n_inv inputs
+// per-species head block (doubles) for n_inv inputs: the caller's row-major matrices, then biases and output layer
 struct Head64 {
-    int w0, w0t, wl, wlt, bias, wout, total;
+    int w0, wl, bias, wout, total;
     __host__ __device__ constexpr explicit Head64(int n_inv)
-        : w0(0),                                            // [64][n_inv]  row-major, reverse pass
-          w0t(HEAD_H * n_inv),                              // [n_inv][64]  transposed, forward pass
-          wl(2 * HEAD_H * n_inv),                           // 3 x [64][64]
-          wlt(wl + (HEAD_L - 1) * HEAD_H * HEAD_H),
-          bias(wlt + (HEAD_L - 1) * HEAD_H * HEAD_H),       // [4][64]
+        : w0(0),                                            // [64][n_inv]
+          wl(HEAD_H * n_inv),                               // 3 x [64][64]
+          bias(wl + (HEAD_L - 1) * HEAD_H * HEAD_H),        // [4][64]
           wout(bias + HEAD_L * HEAD_H),                     // [64] + b_out
           total(wout + HEAD_H + 8) {}
 };
@@ -47,17 +48,19 @@ struct Head64 {
 __host__ __device__ constexpr int l_of(int a) { return a == 0 ? 0 : (a < 4 ? 1 : (a < 9 ? 2 : 3)); }
 
 template <int K, int LMAX>
-struct WarpScratch {
+struct TileSmem {
     static constexpr int D = (LMAX + 1) * (LMAX + 1);
     static constexpr int NINV = (LMAX + 1) * K;
-    static constexpr int NINV_PAD = (NINV + 31) / 32 * 32;
-    double x[NINV_PAD];           // invariants, then dE/dG
-    double y[HEAD_H];             // running activation
-    double sd[HEAD_L][HEAD_H];    // SiLU'(pre-activation) per layer
-    double dp[HEAD_H];            // dE/dpre of the current layer
-    double w[D * K];              // W_i = dE_i/dP_i (Eq. 7)
-    double st[32][F64_ST];
-    int q[64];                    // compacted neighbor indices
+    static constexpr int XS = (NINV + 31) / 32 * 32 + 4;
+    double x[F64_TILE][XS];                 // invariants, then dE/dG
+    double y[2][F64_TILE][F64_YS];          // activations of the previous / current layer
+    double sd[HEAD_L][F64_TILE][F64_YS];    // SiLU'(pre-activation) per layer
+    double dp[2][F64_TILE][F64_YS];         // dE/dpre of the layer being propagated
+    union {
+        double st[32][F64_ST];              // encoding hand-over
+        double w[D * K];                    // W_i = dE_i/dP_i (Eq. 7), derivation
+    } pw[F64_TILE];
+    int q[F64_TILE][64];                    // compacted neighbor indices
 };
 
 struct F64Args {
@@ -70,6 +73,7 @@ struct F64Args {
     double r_min, inv_h;
     const double4 *pos4;
     const int32_t *center_order;
+    const int32_t *species_start;
     const int64_t *nbr_off;
     const int32_t *nbr;
     const double *head;
@@ -86,39 +90,48 @@ __device__ __forceinline__ double silu_d(double x, double &dsilu) {
     return x * s;
 }
 
-// One hidden layer forward for this warp's atom: pre = W in + b for neurons lane, lane + 32.
-template <int IN>
-__device__ __forceinline__ void layer_forward(const double *__restrict__ wt, const double *__restrict__ bias, const double *in, int lane,
-                                              double &p0, double &p1) {
-    p0 = bias[lane]; p1 = bias[lane + 32];
-#pragma unroll 8
-    for (int i = 0; i < IN; ++i) {
-        const double a = in[i];
-        p0 = fma(wt[i * HEAD_H + lane], a, p0);
-        p1 = fma(wt[i * HEAD_H + 32 + lane], a, p1);
-    }
+// C[8 x 8] += A[8 x 4] B[4 x 8] in fp64: lane (g = lane / 4, t = lane % 4) holds A[g][t], B[t][g], C[g][2t], C[g][2t + 1]
+__device__ __forceinline__ void dmma(double &c0, double &c1, double a, double b) {
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};" : "+d"(c0), "+d"(c1) : "d"(a), "d"(b));
 }
 
 template <int K, int LMAX>
-__global__ void __launch_bounds__(F64_WARPS * 32, K <= 32 ? 2 : 1) k_mega_f64(F64Args k) {
-    using WS = WarpScratch<K, LMAX>;
-    constexpr int D = WS::D, NINV = WS::NINV, NQ = WS::NINV_PAD / 32;
+__global__ void __launch_bounds__(F64_TILE * 32, K <= 32 ? 2 : 1) k_mega_f64(F64Args k) {
+    using SM = TileSmem<K, LMAX>;
+    constexpr int D = SM::D, NINV = SM::NINV;
     constexpr int CPL = (K + 31) / 32;   // channels per lane
     constexpr Head64 H(NINV);
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    SM &sm = *reinterpret_cast<SM *>(smem_raw);
+    __shared__ int s_start[MAX_SPECIES + 1];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    WS &ws = reinterpret_cast<WS *>(smem_raw)[wid];
+    const int g = lane >> 2, t = lane & 3;
     const int C = k.n_species;
-    const int64_t n_warps = (int64_t)gridDim.x * F64_WARPS;
+    if (threadIdx.x <= C) s_start[threadIdx.x] = k.species_start[threadIdx.x];
+    __syncthreads();
+    int total_tiles = 0;
+    for (int s = 0; s < C; ++s) total_tiles += (s_start[s + 1] - s_start[s] + F64_TILE - 1) / F64_TILE;
     double e_sum = 0.0, vir[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
     unsigned long long n_pairs = 0;
 
-    for (int64_t slot = (int64_t)blockIdx.x * F64_WARPS + wid; slot < k.n; slot += n_warps) {
-        const int i = k.center_order[slot];
-        const double4 pi = k.pos4[i];
-        const int si = (int)pi.w;
-        const int64_t beg = k.nbr_off[i], end = k.nbr_off[i + 1];
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        int si = 0, tl = tile;
+        for (;;) {   // tiles are numbered species by species
+            const int nt = (s_start[si + 1] - s_start[si] + F64_TILE - 1) / F64_TILE;
+            if (tl < nt) break;
+            tl -= nt; ++si;
+        }
+        const int slot = s_start[si] + F64_TILE * tl + wid;
+        const bool have = slot < s_start[si + 1];
         const double *hd = k.head + (size_t)si * H.total;
+        int i = 0;
+        double4 pi = make_double4(0.0, 0.0, 0.0, 0.0);
+        int64_t beg = 0, end = 0;
+        if (have) {
+            i = k.center_order[slot];
+            pi = k.pos4[i];
+            beg = k.nbr_off[i]; end = k.nbr_off[i + 1];
+        }
 
         // ---------------- Encoding: P = H^T G (Eq. 4), lane = channel ----------------
         double P[D][CPL];
@@ -142,12 +155,13 @@ __global__ void __launch_bounds__(F64_WARPS * 32, K <= 32 ? 2 : 1) k_mega_f64(F6
                     double h[D_ANG], b[4];
                     harmonics(dx * rinv, dy * rinv, dz * rinv, h);
                     const int iv = spline_basis<false, double>(r, k.r_min, k.inv_h, k.knots, b, nullptr, k.status);
+                    double *row = sm.pw[wid].st[lane];
 #pragma unroll
-                    for (int a = 0; a < D; ++a) ws.st[lane][a] = h[a];
+                    for (int a = 0; a < D; ++a) row[a] = h[a];
 #pragma unroll
-                    for (int m = 0; m < 4; ++m) ws.st[lane][16 + m] = b[m];
+                    for (int m = 0; m < 4; ++m) row[16 + m] = b[m];
                     const long long off = ((long long)(si * C + (int)pj.w) * (k.knots + 3) + iv) * K;
-                    ws.st[lane][20] = __longlong_as_double(off);
+                    row[20] = __longlong_as_double(off);
                 }
             }
             unsigned mask = __ballot_sync(0xffffffffu, valid);
@@ -156,113 +170,122 @@ __global__ void __launch_bounds__(F64_WARPS * 32, K <= 32 ? 2 : 1) k_mega_f64(F6
             while (mask) {
                 const int p = __ffs(mask) - 1;
                 mask &= mask - 1;
-                const double *row = ws.st[p];
+                const double *row = sm.pw[wid].st[p];
                 const double *cf = k.coef + __double_as_longlong(row[20]);
 #pragma unroll
                 for (int q = 0; q < CPL; ++q) {
                     const int c = lane + 32 * q;
-                    double g = 0.0;
+                    double gq = 0.0;
                     if (c < K) {
-                        g = row[16] * cf[c];
-                        g = fma(row[17], cf[K + c], g);
-                        g = fma(row[18], cf[2 * K + c], g);
-                        g = fma(row[19], cf[3 * K + c], g);
+                        gq = row[16] * cf[c];
+                        gq = fma(row[17], cf[K + c], gq);
+                        gq = fma(row[18], cf[2 * K + c], gq);
+                        gq = fma(row[19], cf[3 * K + c], gq);
                     }
 #pragma unroll
-                    for (int a = 0; a < D; ++a) P[a][q] = fma(row[a], g, P[a][q]);
+                    for (int a = 0; a < D; ++a) P[a][q] = fma(row[a], gq, P[a][q]);
                 }
             }
             __syncwarp();
         }
 
-        // ---------------- Invariants (Eq. 5, C_l = I) ----------------
+        // ---------------- Invariants (Eq. 5, C_l = I); an empty slot of a ragged tile feeds zeros ----------------
 #pragma unroll
         for (int q = 0; q < CPL; ++q) {
             const int c = lane + 32 * q;
             if (c < K) {
-                ws.x[c] = P[0][q];
+                sm.x[wid][c] = P[0][q];
 #pragma unroll
                 for (int l = 1; l <= LMAX; ++l) {
                     double s = 0.0;
 #pragma unroll
                     for (int a = l * l; a < (l + 1) * (l + 1); ++a) s = fma(P[a][q], P[a][q], s);
-                    ws.x[l * K + c] = s;
+                    sm.x[wid][l * K + c] = s;
                 }
+            }
+        }
+        __syncthreads();
+
+        // ---------------- Regression (Eq. 6) and its reverse pass: the CTA on the tile ----------------
+        {
+            const int n = 8 * wid + g;   // this lane's row of W (forward: neuron; reverse: input of the layer)
+            double y0, y1, d0, d1;
+            {   // layer 0: pre[64 x 8] = W0 [64 x NINV] X^T
+                double c0 = hd[H.bias + n], c1 = c0;
+                const double *wrow = hd + H.w0 + (size_t)n * NINV + t;
+                const double *xb = &sm.x[g][t];
+#pragma unroll 8
+                for (int ks = 0; ks < NINV / 4; ++ks) dmma(c0, c1, wrow[4 * ks], xb[4 * ks]);
+                y0 = silu_d(c0, d0); y1 = silu_d(c1, d1);
+                sm.y[0][2 * t][n] = y0; sm.y[0][2 * t + 1][n] = y1;
+                sm.sd[0][2 * t][n] = d0; sm.sd[0][2 * t + 1][n] = d1;
+            }
+            __syncthreads();
+#pragma unroll 1
+            for (int L = 1; L < HEAD_L; ++L) {
+                double c0 = hd[H.bias + L * HEAD_H + n], c1 = c0;
+                const double *wrow = hd + H.wl + (L - 1) * HEAD_H * HEAD_H + n * HEAD_H + t;
+                const double *xb = &sm.y[(L - 1) & 1][g][t];
+#pragma unroll
+                for (int ks = 0; ks < HEAD_H / 4; ++ks) dmma(c0, c1, wrow[4 * ks], xb[4 * ks]);
+                y0 += silu_d(c0, d0); y1 += silu_d(c1, d1);
+                sm.y[L & 1][2 * t][n] = y0; sm.y[L & 1][2 * t + 1][n] = y1;
+                sm.sd[L][2 * t][n] = d0; sm.sd[L][2 * t + 1][n] = d1;
+                __syncthreads();
+            }
+            {   // output layer: warp = atom
+                const double *yf = sm.y[(HEAD_L - 1) & 1][wid];
+                double e_i = hd[H.wout + lane] * yf[lane] + hd[H.wout + 32 + lane] * yf[lane + 32];
+#pragma unroll
+                for (int o = 16; o; o >>= 1) e_i += __shfl_xor_sync(0xffffffffu, e_i, o);
+                e_i += hd[H.wout + HEAD_H];
+                if (lane == 0 && have) { k.e_atom[i] = e_i; e_sum += e_i; }
+            }
+            // reverse: this lane keeps dE/dy[n] of atoms 2t, 2t + 1; each hidden layer adds W^T (dE/dy . SiLU') through its skip
+            double g0 = hd[H.wout + n], g1 = g0;
+            sm.dp[(HEAD_L - 1) & 1][2 * t][n] = g0 * sm.sd[HEAD_L - 1][2 * t][n];
+            sm.dp[(HEAD_L - 1) & 1][2 * t + 1][n] = g1 * sm.sd[HEAD_L - 1][2 * t + 1][n];
+            __syncthreads();
+#pragma unroll 1
+            for (int L = HEAD_L - 1; L >= 1; --L) {
+                const double *wcol = hd + H.wl + (L - 1) * HEAD_H * HEAD_H + t * HEAD_H + n;   // A[n][o] = W[o][n]
+                const double *xb = &sm.dp[L & 1][g][t];
+#pragma unroll
+                for (int ks = 0; ks < HEAD_H / 4; ++ks) dmma(g0, g1, wcol[4 * ks * HEAD_H], xb[4 * ks]);
+                sm.dp[(L - 1) & 1][2 * t][n] = g0 * sm.sd[L - 1][2 * t][n];
+                sm.dp[(L - 1) & 1][2 * t + 1][n] = g1 * sm.sd[L - 1][2 * t + 1][n];
+                __syncthreads();
+            }
+            // layer 0: dE/dG [NINV x 8] = W0^T dp, written over the invariants; warp = every 8th block of 8 inputs
+#pragma unroll 1
+            for (int m = wid; m < NINV / 8; m += F64_TILE) {
+                double c0 = 0.0, c1 = 0.0;
+                const double *wcol = hd + H.w0 + (size_t)t * NINV + 8 * m + g;
+                const double *xb = &sm.dp[0][g][t];
+#pragma unroll
+                for (int ks = 0; ks < HEAD_H / 4; ++ks) dmma(c0, c1, wcol[(size_t)4 * ks * NINV], xb[4 * ks]);
+                sm.x[2 * t][8 * m + g] = c0; sm.x[2 * t + 1][8 * m + g] = c1;
+            }
+            __syncthreads();
+        }
+
+        // W_i = dE_i/dP_i (Eq. 7)
+        double *wi = sm.pw[wid].w;
+#pragma unroll
+        for (int q = 0; q < CPL; ++q) {
+            const int c = lane + 32 * q;
+            if (c < K) {
+                wi[c] = sm.x[wid][c];
+#pragma unroll
+                for (int a = 1; a < D; ++a) wi[a * K + c] = 2.0 * sm.x[wid][l_of(a) * K + c] * P[a][q];
             }
         }
         __syncwarp();
 
-        // ---------------- Regression (Eq. 6) and its reverse pass ----------------
-        {
-            double p0, p1, d0, d1;
-            layer_forward<NINV>(hd + H.w0t, hd + H.bias, ws.x, lane, p0, p1);
-            double y0 = silu_d(p0, d0), y1 = silu_d(p1, d1);
-            ws.sd[0][lane] = d0; ws.sd[0][lane + 32] = d1;
-            ws.y[lane] = y0; ws.y[lane + 32] = y1;
-            __syncwarp();
-#pragma unroll 1
-            for (int L = 1; L < HEAD_L; ++L) {
-                layer_forward<HEAD_H>(hd + H.wlt + (L - 1) * HEAD_H * HEAD_H, hd + H.bias + L * HEAD_H, ws.y, lane, p0, p1);
-                y0 += silu_d(p0, d0); y1 += silu_d(p1, d1);
-                __syncwarp();
-                ws.sd[L][lane] = d0; ws.sd[L][lane + 32] = d1;
-                ws.y[lane] = y0; ws.y[lane + 32] = y1;
-                __syncwarp();
-            }
-            const double wo0 = hd[H.wout + lane], wo1 = hd[H.wout + 32 + lane];
-            double e_i = wo0 * y0 + wo1 * y1;
-#pragma unroll
-            for (int o = 16; o; o >>= 1) e_i += __shfl_xor_sync(0xffffffffu, e_i, o);
-            e_i += hd[H.wout + HEAD_H];
-            if (lane == 0) { k.e_atom[i] = e_i; e_sum += e_i; }
-
-            // dE/dy of the last layer is w_out; each hidden layer adds W^T (dE/dy . SiLU') through its skip
-            double g0 = wo0, g1 = wo1;
-#pragma unroll 1
-            for (int L = HEAD_L - 1; L >= 1; --L) {
-                ws.dp[lane] = g0 * ws.sd[L][lane]; ws.dp[lane + 32] = g1 * ws.sd[L][lane + 32];
-                __syncwarp();
-                const double *w = hd + H.wl + (L - 1) * HEAD_H * HEAD_H;
-#pragma unroll 8
-                for (int o = 0; o < HEAD_H; ++o) {
-                    const double d = ws.dp[o];
-                    g0 = fma(w[o * HEAD_H + lane], d, g0);
-                    g1 = fma(w[o * HEAD_H + 32 + lane], d, g1);
-                }
-                __syncwarp();
-            }
-            ws.dp[lane] = g0 * ws.sd[0][lane]; ws.dp[lane + 32] = g1 * ws.sd[0][lane + 32];
-            __syncwarp();
-            double dx[NQ];   // dE/dG of invariants lane + 32 q
-#pragma unroll
-            for (int q = 0; q < NQ; ++q) dx[q] = 0.0;
-            const double *w0 = hd + H.w0;
-#pragma unroll 4
-            for (int o = 0; o < HEAD_H; ++o) {
-                const double d = ws.dp[o];
-#pragma unroll
-                for (int q = 0; q < NQ; ++q)
-                    if (lane + 32 * q < NINV) dx[q] = fma(w0[o * NINV + 32 * q + lane], d, dx[q]);
-            }
-#pragma unroll
-            for (int q = 0; q < NQ; ++q) ws.x[lane + 32 * q] = dx[q];
-            __syncwarp();
-            // W_i = dE_i/dP_i (Eq. 7)
-#pragma unroll
-            for (int q = 0; q < CPL; ++q) {
-                const int c = lane + 32 * q;
-                if (c < K) {
-                    ws.w[c] = ws.x[c];
-#pragma unroll
-                    for (int a = 1; a < D; ++a) ws.w[a * K + c] = 2.0 * ws.x[l_of(a) * K + c] * P[a][q];
-                }
-            }
-            __syncwarp();
-        }
-
         // ---------------- Derivation (Eq. 8-10), lane = pair ----------------
         double fx = 0.0, fy = 0.0, fz = 0.0;
         int nq = 0;
+        int *queue = sm.q[wid];
         for (int64_t base = beg; base < end || nq > 0; base += 32) {
             if (base < end) {   // compact the entries inside r_cut into the warp's queue
                 const int64_t e = base + lane;
@@ -277,14 +300,14 @@ __global__ void __launch_bounds__(F64_WARPS * 32, K <= 32 ? 2 : 1) k_mega_f64(F6
                     valid = dx * dx + dy * dy + dz * dz < k.rc2;
                 }
                 const unsigned m = __ballot_sync(0xffffffffu, valid);
-                if (valid) ws.q[nq + __popc(m & ((1u << lane) - 1u))] = j;
+                if (valid) queue[nq + __popc(m & ((1u << lane) - 1u))] = j;
                 nq += __popc(m);
                 __syncwarp();
                 if (nq < 32 && base + 32 < end) continue;
             }
             const int nb = min(nq, 32);
             if (lane < nb) {
-                const int j = ws.q[lane];
+                const int j = queue[lane];
                 const double4 pj = k.pos4[j];
                 const double x = min_image(pj.x - pi.x, k.grid.box[0], k.grid.half[0]);
                 const double y = min_image(pj.y - pi.y, k.grid.box[1], k.grid.half[1]);
@@ -294,27 +317,30 @@ __global__ void __launch_bounds__(F64_WARPS * 32, K <= 32 ? 2 : 1) k_mega_f64(F6
                 double b[4], db[4];
                 const int iv = spline_basis<true, double>(r, k.r_min, k.inv_h, k.knots, b, db, k.status);
                 const double *cf = k.coef + ((size_t)(si * C + (int)pj.w) * (k.knots + 3) + iv) * K;
-                double v[D_ANG], t[D_ANG];   // components beyond d stay zero and drop out of the projection
+                double v[D_ANG], tt[D_ANG];   // components beyond d stay zero and drop out of the projection
 #pragma unroll
-                for (int a = 0; a < D_ANG; ++a) { v[a] = 0.0; t[a] = 0.0; }
+                for (int a = 0; a < D_ANG; ++a) { v[a] = 0.0; tt[a] = 0.0; }
 #pragma unroll 1
-                for (int c = 0; c < K; c += 2) {
-                    double g0 = 0.0, g1 = 0.0, dg0 = 0.0, dg1 = 0.0;
+                for (int c = 0; c < K; c += 4) {   // four channels = one 32-byte sector per table row
+                    double gv[4] = {0.0, 0.0, 0.0, 0.0}, dg[4] = {0.0, 0.0, 0.0, 0.0};
 #pragma unroll
                     for (int m = 0; m < 4; ++m) {
-                        const double2 cc = *reinterpret_cast<const double2 *>(cf + m * K + c);
-                        g0 = fma(b[m], cc.x, g0); g1 = fma(b[m], cc.y, g1);
-                        dg0 = fma(db[m], cc.x, dg0); dg1 = fma(db[m], cc.y, dg1);
+                        double cc[4];
+                        asm volatile("ld.global.nc.v4.f64 {%0,%1,%2,%3}, [%4];"
+                                     : "=d"(cc[0]), "=d"(cc[1]), "=d"(cc[2]), "=d"(cc[3]) : "l"(cf + m * K + c));
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) { gv[u] = fma(b[m], cc[u], gv[u]); dg[u] = fma(db[m], cc[u], dg[u]); }
                     }
 #pragma unroll
                     for (int a = 0; a < D; ++a) {
-                        const double2 w = *reinterpret_cast<const double2 *>(&ws.w[a * K + c]);
-                        v[a] = fma(w.x, g0, fma(w.y, g1, v[a]));
-                        t[a] = fma(w.x, dg0, fma(w.y, dg1, t[a]));
+                        const double2 w0 = *reinterpret_cast<const double2 *>(&wi[a * K + c]);
+                        const double2 w1 = *reinterpret_cast<const double2 *>(&wi[a * K + c + 2]);
+                        v[a] = fma(w0.x, gv[0], fma(w0.y, gv[1], fma(w1.x, gv[2], fma(w1.y, gv[3], v[a]))));
+                        tt[a] = fma(w0.x, dg[0], fma(w0.y, dg[1], fma(w1.x, dg[2], fma(w1.y, dg[3], tt[a]))));
                     }
                 }
                 double s, tx, ty, tz, tu;
-                harmonics_project(ux, uy, uz, v, t, s, tx, ty, tz, tu);
+                harmonics_project(ux, uy, uz, v, tt, s, tx, ty, tz, tu);
                 // f_ij = (g' . u_ij) r^ + J_ang^T v_ij,  J_ang = (grad_u h)(I - u u^T) / r
                 const double qx = s * ux + (tx - tu * ux) * rinv;
                 const double qy = s * uy + (ty - tu * uy) * rinv;
@@ -330,9 +356,9 @@ __global__ void __launch_bounds__(F64_WARPS * 32, K <= 32 ? 2 : 1) k_mega_f64(F6
             __syncwarp();
             // move what is left of the queue to its front
             const int rest = nq - nb;
-            const int keep = lane < rest ? ws.q[nb + lane] : 0;
+            const int keep = lane < rest ? queue[nb + lane] : 0;
             __syncwarp();
-            if (lane < rest) ws.q[lane] = keep;
+            if (lane < rest) queue[lane] = keep;
             nq = rest;
             __syncwarp();
         }
@@ -342,11 +368,12 @@ __global__ void __launch_bounds__(F64_WARPS * 32, K <= 32 ? 2 : 1) k_mega_f64(F6
             fy += __shfl_xor_sync(0xffffffffu, fy, o);
             fz += __shfl_xor_sync(0xffffffffu, fz, o);
         }
-        if (lane == 0) {
+        if (lane == 0 && have) {
             atomicAdd(&k.force[3 * (size_t)i], fx);
             atomicAdd(&k.force[3 * (size_t)i + 1], fy);
             atomicAdd(&k.force[3 * (size_t)i + 2], fz);
         }
+        __syncthreads();   // the next tile's encoding reuses the hand-over rows that alias W_i, and x
     }
 
 #pragma unroll
@@ -383,17 +410,12 @@ int upload_head_f64(mlip_ctx *c, const double *w) {
         int in = n_inv;
         for (int L = 0; L < HEAD_L; ++L) {
             double *row = L == 0 ? hp + H.w0 : hp + H.wl + (L - 1) * HEAD_H * HEAD_H;
-            double *tr = L == 0 ? hp + H.w0t : hp + H.wlt + (L - 1) * HEAD_H * HEAD_H;
-            for (int o = 0; o < HEAD_H; ++o)
-                for (int q = 0; q < in; ++q) {
-                    row[o * in + q] = src[o * in + q];
-                    tr[q * HEAD_H + o] = src[o * in + q];
-                }
-            for (int o = 0; o < HEAD_H; ++o) hp[H.bias + L * HEAD_H + o] = src[in * HEAD_H + o];
+            memcpy(row, src, sizeof(double) * HEAD_H * in);
+            memcpy(hp + H.bias + L * HEAD_H, src + in * HEAD_H, sizeof(double) * HEAD_H);
             src += in * HEAD_H + HEAD_H;
             in = HEAD_H;
         }
-        for (int o = 0; o < HEAD_H + 1; ++o) hp[H.wout + o] = src[o];
+        memcpy(hp + H.wout, src, sizeof(double) * (HEAD_H + 1));
     }
     const size_t bytes = sizeof(double) * (size_t)C * H.total;
     cudaError_t e = cudaMalloc(&c->head_w_d, bytes);
@@ -406,16 +428,17 @@ int upload_head_f64(mlip_ctx *c, const double *w) {
 
 template <int K, int LMAX>
 static cudaError_t launch_shape(mlip_ctx *c, const F64Args &k, cudaStream_t s, cudaEvent_t start, cudaEvent_t stop) {
-    const size_t smem_bytes = sizeof(WarpScratch<K, LMAX>) * F64_WARPS;
+    const size_t smem_bytes = sizeof(TileSmem<K, LMAX>);
     if (!c->kernel_ready) {
         cudaError_t e = cudaFuncSetAttribute(k_mega_f64<K, LMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
         if (e != cudaSuccess) return e;
         c->kernel_ready = true;
     }
     const int per_sm = K <= 32 ? 2 : 1;
-    const int blocks = (int)std::min<int64_t>((k.n + F64_WARPS - 1) / F64_WARPS, (int64_t)per_sm * c->n_sm);
+    const int64_t tiles_max = (k.n + F64_TILE - 1) / F64_TILE + k.n_species;
+    const int blocks = (int)std::min<int64_t>(tiles_max, (int64_t)per_sm * c->n_sm);
     cudaEventRecord(start, s);
-    k_mega_f64<K, LMAX><<<blocks, F64_WARPS * 32, smem_bytes, s>>>(k);
+    k_mega_f64<K, LMAX><<<blocks, F64_TILE * 32, smem_bytes, s>>>(k);
     cudaEventRecord(stop, s);
     return cudaGetLastError();
 }
@@ -431,7 +454,8 @@ int launch_megakernel_f64(mlip_ctx *c, cudaStream_t s) {
     k.n = n; k.n_species = c->cfg.n_species; k.grid = c->grid; k.rc2 = c->cfg.r_cut * c->cfg.r_cut;
     k.coef = c->table_d; k.knots = c->cfg.table_knots; k.r_min = c->cfg.table_r_min;
     k.inv_h = c->cfg.table_knots / (c->cfg.r_cut - c->cfg.table_r_min);
-    k.pos4 = c->pos4; k.center_order = c->center_order; k.nbr_off = c->nbr_off; k.nbr = c->nbr;
+    k.pos4 = c->pos4; k.center_order = c->center_order; k.species_start = c->species_start;
+    k.nbr_off = c->nbr_off; k.nbr = c->nbr;
     k.head = c->head_w_d; k.force = c->force_d; k.e_atom = c->e_atom_d; k.acc = c->acc;
     k.pair_counter = c->pair_counter; k.status = c->status;
     const int slot = (int)(c->ev_count % mlip_ctx::EV_POOL);
