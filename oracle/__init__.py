@@ -242,3 +242,85 @@ def nve(model: Model, pos, vel, species, masses, box, n_steps, dt_fs, r_list, re
         e_pot.append(out["energy"])
         e_kin.append(kinetic_energy(vel, species, masses))
     return {"pos": pos, "vel": vel, "e_pot": np.array(e_pot), "e_kin": np.array(e_kin), "forces": out["forces"]}
+
+
+def nhc_masses(n_f, kT, t_damp_fs, chain=3):
+    """Thermostat masses of a Nose-Hoover chain: Q_1 = N_f kT tau^2, Q_k = kT tau^2 (eV fs^2)."""
+    q = np.full(chain, kT * t_damp_fs ** 2)
+    q[0] *= n_f
+    return q
+
+
+def nhc_half_step(ke2, v_eta, eta, q, n_f, kT, dt_fs):
+    """Advance a Nose-Hoover chain by dt/2 at fixed particle positions and return the factor by which the
+    particle velocities are scaled (Martyna, Tuckerman, Tobias and Klein 1996: one Suzuki-Yoshida term, one
+    sub-cycle).  ke2 = sum m v^2 (twice the kinetic energy, eV); v_eta, eta are updated in place.
+
+    Equations of motion: dv_i/dt = -v_eta1 v_i;  dv_eta_k/dt = G_k - v_eta_{k+1} v_eta_k,
+    G_1 = (sum m v^2 - N_f kT) / Q_1,  G_k = (Q_{k-1} v_eta_{k-1}^2 - kT) / Q_k;  d eta_k/dt = v_eta_k.
+    """
+    M = len(q)
+    d = 0.5 * dt_fs
+    G = np.empty(M)
+    G[0] = (ke2 - n_f * kT) / q[0]
+    for k in range(1, M):
+        G[k] = (q[k - 1] * v_eta[k - 1] ** 2 - kT) / q[k]
+    v_eta[M - 1] += 0.5 * d * G[M - 1]
+    for k in range(M - 2, -1, -1):
+        a = np.exp(-0.25 * d * v_eta[k + 1])
+        v_eta[k] = (v_eta[k] * a + 0.5 * d * G[k]) * a
+    scale = np.exp(-d * v_eta[0])
+    ke2 = ke2 * scale * scale
+    eta += d * v_eta
+    G[0] = (ke2 - n_f * kT) / q[0]
+    for k in range(M - 1):
+        a = np.exp(-0.25 * d * v_eta[k + 1])
+        v_eta[k] = (v_eta[k] * a + 0.5 * d * G[k]) * a
+        G[k + 1] = (q[k] * v_eta[k] ** 2 - kT) / q[k + 1]
+    v_eta[M - 1] += 0.5 * d * G[M - 1]
+    return scale
+
+
+def nhc_energy(v_eta, eta, q, n_f, kT):
+    """Thermostat part of the conserved quantity of Nose-Hoover-chain dynamics."""
+    return float(0.5 * np.sum(q * v_eta ** 2) + n_f * kT * eta[0] + kT * np.sum(eta[1:]))
+
+
+def nvt(model: Model, pos, vel, species, masses, box, n_steps, dt_fs, r_list, t_target, t_damp_fs, rebuild_every=1,
+        chain=3, n_f=None):
+    """Nose-Hoover-chain NVT: thermostat half step, velocity-Verlet step, thermostat half step.
+
+    Section 4.2 runs NVT at 300 K through LAMMPS without naming the thermostat; this is the reading taken (the
+    chain thermostat of LAMMPS's own NVT integrator, chain length 3).  N_f defaults to 3 N - 3.
+    Returns positions, velocities, per-step energies and the conserved quantity (index 0 = initial state).
+    """
+    pos = np.array(pos, dtype=np.float64)
+    vel = np.array(vel, dtype=np.float64)
+    box = np.asarray(box, dtype=np.float64)
+    n = pos.shape[0]
+    n_f = 3 * n - 3 if n_f is None else n_f
+    kT = KB_EV_PER_K * t_target
+    q = nhc_masses(n_f, kT, t_damp_fs, chain)
+    v_eta, eta = np.zeros(chain), np.zeros(chain)
+    inv_m = (ACC_UNIT / np.asarray(masses, dtype=np.float64))[species][:, None]
+    nl = neighbors(pos, species, model.n_species, box, r_list)
+    out = compute(model, pos, species, box, nl)
+    ke = kinetic_energy(vel, species, masses)
+    e_pot, e_kin = [out["energy"]], [ke]
+    conserved = [out["energy"] + ke + nhc_energy(v_eta, eta, q, n_f, kT)]
+    for step in range(1, n_steps + 1):
+        vel *= nhc_half_step(2.0 * kinetic_energy(vel, species, masses), v_eta, eta, q, n_f, kT, dt_fs)
+        vel += 0.5 * dt_fs * out["forces"] * inv_m
+        pos += dt_fs * vel
+        pos -= np.floor(pos / box) * box
+        if rebuild_every > 0 and step % rebuild_every == 0:
+            nl = neighbors(pos, species, model.n_species, box, r_list)
+        out = compute(model, pos, species, box, nl)
+        vel += 0.5 * dt_fs * out["forces"] * inv_m
+        vel *= nhc_half_step(2.0 * kinetic_energy(vel, species, masses), v_eta, eta, q, n_f, kT, dt_fs)
+        ke = kinetic_energy(vel, species, masses)
+        e_pot.append(out["energy"])
+        e_kin.append(ke)
+        conserved.append(out["energy"] + ke + nhc_energy(v_eta, eta, q, n_f, kT))
+    return {"pos": pos, "vel": vel, "e_pot": np.array(e_pot), "e_kin": np.array(e_kin), "conserved": np.array(conserved),
+            "v_eta": v_eta, "eta": eta, "forces": out["forces"]}
