@@ -63,6 +63,8 @@ def parse_args():
                          "3-species alloy and ionic stand-ins at their full sizes (extra data points, not the contract line)")
     ap.add_argument("--precision", default="f32", choices=["f32", "f64"],
                     help="f64 runs the double-precision evaluation path instead (an extra data point, not the contract line)")
+    ap.add_argument("--ensemble", default="nve", choices=["nve", "nvt"],
+                    help="nvt adds the Nose-Hoover-chain thermostat (the paper's ensemble) to every step: an extra data point")
     ap.add_argument("--k", type=int, default=32, choices=[16, 32, 64], help="radial channels (other than 32: --precision f64 only)")
     ap.add_argument("--lmax", type=int, default=3, choices=[1, 2, 3], help="angular order (other than 3: --precision f64 only)")
     ap.add_argument("--sweep", default="", help="comma-separated FCC cell counts: size sweep of the 6-species workload "
@@ -298,7 +300,13 @@ def main():
     # ---- device-resident run: inputs already in HBM when timing starts ----
     pot.build_neighbors(w.pos, w.species, w.box)
     pot.set_velocities(w.vel)
-    pot.step(args.warmup, DT_FS, rebuild_every)
+    def advance(n_steps):
+        if args.ensemble == "nvt":
+            pot.step_nvt(n_steps, DT_FS, rebuild_every, w.temperature, 100.0)
+        else:
+            pot.step(n_steps, DT_FS, rebuild_every)
+
+    advance(args.warmup)
     pot.sync_status()
     barrier()
     mlip.mlip_kernel_time(pot.ctx, reset=True)
@@ -313,7 +321,7 @@ def main():
         sampler.start()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
-    pot.step(args.steps, DT_FS, rebuild_every)
+    advance(args.steps)
     ev1.record()
     barrier()
     ms = ev0.elapsed_time(ev1)
@@ -388,7 +396,7 @@ def main():
                 "ms_per_step": ms_max / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": args.precision, "data": "synthetic",
                 "config": {"workload": f"cfg{cfg} {w.name}: {n} atoms, {w.n_species} species, r_cut 6 A, skin 1 A, "
-                                       f"NVE dt 1 fs, list rebuild every {rebuild_every} steps"
+                                       f"{args.ensemble.upper()} dt 1 fs, list rebuild every {rebuild_every} steps"
                                        + ("" if default_shape else f", k = {args.k}, l_max = {args.lmax}"),
                            "atoms_per_gpu": n, "parallelism": "replicas" if world > 1 else "single",
                            "l2": "inputs larger than L2 (positions + lists = %.1f GB per GPU)" % ((32 * n + 4 * entries) / 1e9)},

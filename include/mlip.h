@@ -186,6 +186,24 @@ int mlip_compute_host(mlip_ctx *ctx, int64_t n_atoms, const double *pos_host, co
  */
 int mlip_step(mlip_ctx *ctx, int n_steps, double dt_fs, int rebuild_every, void *stream);
 
+/*
+ * n_steps of NVT dynamics at t_target_K: a Nose-Hoover chain of three thermostats (damping time t_damp_fs, N_f = 3N - 3,
+ * Martyna-Tuckerman-Tobias-Klein integration: thermostat half step, velocity-Verlet step, thermostat half step) around
+ * the same force evaluation.  Section 4.2 runs its MD in the NVT ensemble at 300 K without naming the thermostat; the
+ * chain thermostat is the reading taken.  rebuild_every as in mlip_step.  The thermostat state lives in the context
+ * (zero at creation) and carries over between calls.  Per step it adds a kinetic-energy reduction, two one-thread
+ * kernels and one velocity scaling to the NVE step.
+ */
+int mlip_step_nvt(mlip_ctx *ctx, int n_steps, double dt_fs, int rebuild_every, double t_target_K, double t_damp_fs,
+                  void *stream);
+/*
+ * Thermostat velocities and positions (host [3] each) and the thermostat's part of the conserved quantity
+ * (sum Q_k v_eta_k^2 / 2 + N_f kT eta_1 + kT (eta_2 + eta_3), eV, with the parameters of the last mlip_step_nvt).
+ * Synchronises.  mlip_reset_thermostat zeroes the state.
+ */
+int mlip_get_thermostat(mlip_ctx *ctx, double *v_eta_host, double *eta_host, double *energy_host);
+int mlip_reset_thermostat(mlip_ctx *ctx);
+
 /* Number of list builds since mlip_create (initial builds, in-step rebuilds, host-entry rebuilds). */
 int mlip_get_rebuilds(const mlip_ctx *ctx, int64_t *n_builds_host);
 

@@ -23,7 +23,7 @@ ERRORS = {0: "MLIP_OK", 1: "MLIP_ERR_INVALID_ARG", 2: "MLIP_ERR_UNSUPPORTED", 3:
 CODES = {v: k for k, v in ERRORS.items()}
 
 EXPORTS = ["mlip_create", "mlip_table_error", "mlip_build_neighbors", "mlip_get_neighbors", "mlip_get_neighbors_noalloc", "mlip_set_positions",
-           "mlip_set_velocities", "mlip_compute", "mlip_compute_f64", "mlip_compute_host", "mlip_step", "mlip_get_rebuilds", "mlip_get_state",
+           "mlip_set_velocities", "mlip_compute", "mlip_compute_f64", "mlip_compute_host", "mlip_step", "mlip_step_nvt", "mlip_get_thermostat", "mlip_reset_thermostat", "mlip_get_rebuilds", "mlip_get_state",
            "mlip_get_energies", "mlip_sync_status", "mlip_get_counters", "mlip_kernel_time",
            "mlip_resident_bytes", "mlip_last_error", "mlip_destroy"]
 
@@ -161,6 +161,22 @@ def mlip_step(ctx, n_steps, dt_fs, rebuild_every, stream=None):
     _check(ctx, lib().mlip_step(ctx, ctypes.c_int(n_steps), ctypes.c_double(dt_fs), ctypes.c_int(rebuild_every), _stream(stream)))
 
 
+def mlip_step_nvt(ctx, n_steps, dt_fs, rebuild_every, t_target_K, t_damp_fs, stream=None):
+    _check(ctx, lib().mlip_step_nvt(ctx, ctypes.c_int(n_steps), ctypes.c_double(dt_fs), ctypes.c_int(rebuild_every),
+                                    ctypes.c_double(t_target_K), ctypes.c_double(t_damp_fs), _stream(stream)))
+
+
+def mlip_get_thermostat(ctx):
+    """(v_eta [3], eta [3], thermostat energy in eV)."""
+    v, e, en = (ctypes.c_double * 3)(), (ctypes.c_double * 3)(), ctypes.c_double(0)
+    _check(ctx, lib().mlip_get_thermostat(ctx, v, e, ctypes.byref(en)))
+    return np.array(v[:]), np.array(e[:]), en.value
+
+
+def mlip_reset_thermostat(ctx):
+    _check(ctx, lib().mlip_reset_thermostat(ctx))
+
+
 def mlip_get_rebuilds(ctx) -> int:
     n = ctypes.c_int64(0)
     _check(ctx, lib().mlip_get_rebuilds(ctx, ctypes.byref(n)))
@@ -280,6 +296,12 @@ class Potential:
     def step(self, n_steps, dt_fs, rebuild_every):
         """rebuild_every > 0: fixed interval; 0: never; < 0: displacement-triggered, checked every -rebuild_every steps."""
         mlip_step(self.ctx, n_steps, dt_fs, rebuild_every)
+
+    def step_nvt(self, n_steps, dt_fs, rebuild_every, t_target_K, t_damp_fs=100.0):
+        mlip_step_nvt(self.ctx, n_steps, dt_fs, rebuild_every, t_target_K, t_damp_fs)
+
+    def thermostat(self):
+        return mlip_get_thermostat(self.ctx)
 
     def rebuilds(self) -> int:
         return mlip_get_rebuilds(self.ctx)

@@ -187,6 +187,7 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
         if ((rc = dev_alloc(c, &c->pair_counter, 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->status, 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->rebuild_flag, 1)) != MLIP_OK) break;
+        if ((rc = dev_alloc(c, &c->nhc, 8)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->tile_counter, (size_t)MAX_SPECIES)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->species_start, (size_t)MAX_SPECIES + 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->stage_out, 10)) != MLIP_OK) break;
@@ -199,7 +200,8 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
         for (int q = 0; q < 2 * mlip_ctx::EV_POOL; ++q) ev_ok = ev_ok && cudaEventCreate(&c->ev[q]) == cudaSuccess;
         if (!ev_ok) { rc = MLIP_ERR_CUDA; c->err = "event creation failed"; break; }
         if (cudaMemcpy(c->mass, mass, sizeof(double) * cfg->n_species, cudaMemcpyHostToDevice) != cudaSuccess ||
-            cudaMemset(c->status, 0, sizeof(int)) != cudaSuccess || cudaMemset(c->rebuild_flag, 0, sizeof(int)) != cudaSuccess || cudaMemset(c->acc, 0, sizeof(double) * ACC_COUNT) != cudaSuccess) {
+            cudaMemset(c->status, 0, sizeof(int)) != cudaSuccess || cudaMemset(c->rebuild_flag, 0, sizeof(int)) != cudaSuccess ||
+            cudaMemset(c->nhc, 0, sizeof(double) * 8) != cudaSuccess || cudaMemset(c->acc, 0, sizeof(double) * ACC_COUNT) != cudaSuccess) {
             rc = MLIP_ERR_CUDA; c->err = "initial upload failed"; break;
         }
         if ((rc = f64 ? upload_head_f64(c, head_w) : upload_head(c, head_w)) != MLIP_OK) break;
@@ -349,6 +351,23 @@ int mlip_compute_host(mlip_ctx *c, int64_t n, const double *pos_host, const int3
     return MLIP_OK;
 }
 
+// After a drift: rebuild the lists if the policy asks for it (fixed interval, or displacement-triggered).
+static int rebuild_if_due(mlip_ctx *c, int rebuild_every, cudaStream_t s) {
+    bool rebuild = rebuild_every > 0 && c->step % rebuild_every == 0;
+    if (rebuild_every < 0 && c->step % -rebuild_every == 0) {   // displacement-triggered: ask the device
+        MLIP_CUDA_TRY(c, cudaMemcpyAsync(c->rebuild_host, c->rebuild_flag, sizeof(int), cudaMemcpyDeviceToHost, s));
+        MLIP_CUDA_TRY(c, cudaStreamSynchronize(s));
+        rebuild = *c->rebuild_host != 0;
+    }
+    if (!rebuild) return MLIP_OK;
+    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->rebuild_flag, 0, sizeof(int), s));
+    c->n_builds += 1;
+    std::swap(c->pos4, c->pos4_src);
+    std::swap(c->vel, c->vel_src);
+    std::swap(c->user_of, c->user_src);
+    return launch_build(c, false, s);
+}
+
 int mlip_step(mlip_ctx *c, int n_steps, double dt, int rebuild_every, void *stream) {
     if (!c || n_steps < 0 || !(dt > 0.0)) return MLIP_ERR_INVALID_ARG;
     if (!c->built) return fail(c, MLIP_ERR_NOT_BUILT, "no neighbor lists yet");
@@ -362,23 +381,61 @@ int mlip_step(mlip_ctx *c, int n_steps, double dt, int rebuild_every, void *stre
     for (int it = 0; it < n_steps; ++it) {
         if ((rc = launch_kick_drift(c, dt, s)) != MLIP_OK) return rc;
         c->step += 1;
-        bool rebuild = rebuild_every > 0 && c->step % rebuild_every == 0;
-        if (rebuild_every < 0 && c->step % -rebuild_every == 0) {   // displacement-triggered: ask the device
-            MLIP_CUDA_TRY(c, cudaMemcpyAsync(c->rebuild_host, c->rebuild_flag, sizeof(int), cudaMemcpyDeviceToHost, s));
-            MLIP_CUDA_TRY(c, cudaStreamSynchronize(s));
-            rebuild = *c->rebuild_host != 0;
-        }
-        if (rebuild) {
-            MLIP_CUDA_TRY(c, cudaMemsetAsync(c->rebuild_flag, 0, sizeof(int), s));
-            c->n_builds += 1;
-            std::swap(c->pos4, c->pos4_src);
-            std::swap(c->vel, c->vel_src);
-            std::swap(c->user_of, c->user_src);
-            if ((rc = launch_build(c, false, s)) != MLIP_OK) return rc;
-        }
+        if ((rc = rebuild_if_due(c, rebuild_every, s)) != MLIP_OK) return rc;
         if ((rc = evaluate(c, s)) != MLIP_OK) return rc;
         if ((rc = launch_kick(c, dt, s)) != MLIP_OK) return rc;
     }
+    return MLIP_OK;
+}
+
+int mlip_step_nvt(mlip_ctx *c, int n_steps, double dt, int rebuild_every, double t_target, double t_damp, void *stream) {
+    if (!c || n_steps < 0 || !(dt > 0.0) || !(t_target > 0.0) || !(t_damp > 0.0)) return MLIP_ERR_INVALID_ARG;
+    if (!c->built) return fail(c, MLIP_ERR_NOT_BUILT, "no neighbor lists yet");
+    if (c->n < 2) return fail(c, MLIP_ERR_INVALID_ARG, "the thermostat needs at least two atoms");
+    cudaStream_t s = (cudaStream_t)stream;
+    c->last_stream = s;
+    const double kB = 8.617333262e-5;   // eV/K
+    c->nhc_nf = 3.0 * (double)c->n - 3.0;
+    c->nhc_kT = kB * t_target;
+    c->nhc_qk = c->nhc_kT * t_damp * t_damp;
+    c->nhc_q1 = c->nhc_nf * c->nhc_qk;
+    int rc;
+    if (!c->forces_current) {
+        if ((rc = evaluate(c, s)) != MLIP_OK) return rc;
+        c->forces_current = true;
+    }
+    if ((rc = launch_kinetic(c, s)) != MLIP_OK) return rc;
+    for (int it = 0; it < n_steps; ++it) {
+        // thermostat half step; its velocity factor is applied inside the kick-drift kernel
+        if ((rc = launch_nhc_half(c, c->nhc_nf, c->nhc_kT, c->nhc_q1, c->nhc_qk, dt, s)) != MLIP_OK) return rc;
+        if ((rc = launch_kick_drift(c, dt, s, c->nhc + 6)) != MLIP_OK) return rc;
+        c->step += 1;
+        if ((rc = rebuild_if_due(c, rebuild_every, s)) != MLIP_OK) return rc;
+        if ((rc = evaluate(c, s)) != MLIP_OK) return rc;
+        if ((rc = launch_kick(c, dt, s)) != MLIP_OK) return rc;
+        if ((rc = launch_kinetic(c, s)) != MLIP_OK) return rc;
+        if ((rc = launch_nhc_half(c, c->nhc_nf, c->nhc_kT, c->nhc_q1, c->nhc_qk, dt, s)) != MLIP_OK) return rc;
+        if ((rc = launch_scale_velocities(c, s)) != MLIP_OK) return rc;
+    }
+    return MLIP_OK;
+}
+
+int mlip_get_thermostat(mlip_ctx *c, double *v_eta_host, double *eta_host, double *energy_host) {
+    if (!c) return MLIP_ERR_INVALID_ARG;
+    double st[8];
+    MLIP_CUDA_TRY(c, cudaStreamSynchronize(c->last_stream));
+    MLIP_CUDA_TRY(c, cudaMemcpy(st, c->nhc, sizeof st, cudaMemcpyDeviceToHost));
+    if (v_eta_host) memcpy(v_eta_host, st, sizeof(double) * 3);
+    if (eta_host) memcpy(eta_host, st + 3, sizeof(double) * 3);
+    if (energy_host)
+        *energy_host = 0.5 * (c->nhc_q1 * st[0] * st[0] + c->nhc_qk * (st[1] * st[1] + st[2] * st[2])) +
+                       c->nhc_nf * c->nhc_kT * st[3] + c->nhc_kT * (st[4] + st[5]);
+    return MLIP_OK;
+}
+
+int mlip_reset_thermostat(mlip_ctx *c) {
+    if (!c) return MLIP_ERR_INVALID_ARG;
+    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->nhc, 0, sizeof(double) * 8, c->last_stream));
     return MLIP_OK;
 }
 
@@ -477,7 +534,7 @@ void mlip_destroy(mlip_ctx *c) {
     free_cells(c);
     cudaFree(c->nbr); cudaFree(c->scan_tmp); cudaFree(c->head_w); cudaFree(c->table); cudaFree(c->mass);
     cudaFree(c->head_w_d); cudaFree(c->table_d);
-    cudaFree(c->acc); cudaFree(c->pair_counter); cudaFree(c->status); cudaFree(c->rebuild_flag); cudaFree(c->tile_counter);
+    cudaFree(c->acc); cudaFree(c->pair_counter); cudaFree(c->status); cudaFree(c->rebuild_flag); cudaFree(c->nhc); cudaFree(c->tile_counter);
     cudaFree(c->species_start); cudaFree(c->stage_pos); cudaFree(c->stage_species); cudaFree(c->stage_force);
     cudaFree(c->stage_out);
     if (c->status_host) cudaFreeHost(c->status_host);

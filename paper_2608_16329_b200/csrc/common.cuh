@@ -63,6 +63,8 @@ struct mlip_ctx {
     float *head_w = nullptr;     // per-species head weights packed in MMA fragment order (megakernel.cu)
     float *table = nullptr;      // spline coefficients
     double *mass = nullptr;      // [C] dev
+    double *nhc = nullptr;       // thermostat state {v_eta[3], eta[3], scale, -} (integrate.cu)
+    double nhc_nf = 0, nhc_kT = 0, nhc_q1 = 0, nhc_qk = 0;   // parameters of the last NVT call
     // fp64 path (precision = 1) only
     double *head_w_d = nullptr;  // per-species head weights, row-major and transposed (megakernel_f64.cu)
     double *table_d = nullptr;   // spline coefficients in fp64
@@ -151,7 +153,9 @@ int upload_head_f64(mlip_ctx *c, const double *head_w_host);
 int launch_megakernel_f64(mlip_ctx *c, cudaStream_t s);
 bool f64_shape_supported(int k, int l_max);
 // integrate.cu
-int launch_kick_drift(mlip_ctx *c, double dt, cudaStream_t s);
+int launch_kick_drift(mlip_ctx *c, double dt, cudaStream_t s, const double *vscale = nullptr);
+int launch_nhc_half(mlip_ctx *c, double n_f, double kT, double q1, double qk, double dt, cudaStream_t s);
+int launch_scale_velocities(mlip_ctx *c, cudaStream_t s);
 int launch_kick(mlip_ctx *c, double dt, cudaStream_t s);
 int launch_kinetic(mlip_ctx *c, cudaStream_t s);
 int launch_scatter_forces(mlip_ctx *c, float *forces, float *e_atom, cudaStream_t s);

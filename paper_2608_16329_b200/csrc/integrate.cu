@@ -17,13 +17,14 @@ __device__ __forceinline__ double3 load_force(const float4 *__restrict__ force, 
 __global__ void k_kick_drift(int64_t n, double dt, CellGrid g, const double *__restrict__ mass, float skin_half2,
                              double4 *__restrict__ pos4, double *__restrict__ vel, const float4 *__restrict__ force,
                              const double *__restrict__ force_d, float *__restrict__ disp, int *status, float trigger2,
-                             int *rebuild_flag) {
+                             int *rebuild_flag, const double *__restrict__ vscale) {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     double4 p = pos4[i];
     const double3 f = load_force(force, force_d, i);
     const double k = 0.5 * dt * ACC_UNIT / mass[(int)p.w];
-    double v[3] = {vel[3 * i] + k * f.x, vel[3 * i + 1] + k * f.y, vel[3 * i + 2] + k * f.z};
+    const double sc = vscale ? *vscale : 1.0;   // thermostat factor applied ahead of the kick (NVT)
+    double v[3] = {vel[3 * i] * sc + k * f.x, vel[3 * i + 1] * sc + k * f.y, vel[3 * i + 2] * sc + k * f.z};
     double x[3] = {p.x + dt * v[0], p.y + dt * v[1], p.z + dt * v[2]};
     float d2 = 0.f;
 #pragma unroll
@@ -50,6 +51,44 @@ __global__ void k_kick(int64_t n, double dt, const double *__restrict__ mass, co
     const double3 f = load_force(force, force_d, i);
     const double k = 0.5 * dt * ACC_UNIT / mass[(int)pos4[i].w];
     vel[3 * i] += k * f.x; vel[3 * i + 1] += k * f.y; vel[3 * i + 2] += k * f.z;
+}
+
+// Half-step (dt/2) of a Nose-Hoover chain of three thermostats coupled to the kinetic energy in acc[ACC_KINETIC]
+// (Martyna-Tuckerman-Tobias-Klein factorisation, one Suzuki-Yoshida term).  One thread.  state = {v_eta[3], eta[3], scale}:
+//   dv_eta_k/dt = G_k - v_eta_{k+1} v_eta_k,  G_1 = (2 KE - N_f kT) / Q_1,  G_k = (Q_{k-1} v_eta_{k-1}^2 - kT) / Q_k,
+//   particle velocities scale by exp(-v_eta_1 dt/2); the stored kinetic energy is scaled with them.
+__global__ void k_nhc_half(double *state, double *acc, double n_f, double kT, double q1, double qk, double dt) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    constexpr int M = 3;
+    double v[M] = {state[0], state[1], state[2]};
+    const double q[M] = {q1, qk, qk}, d = 0.5 * dt;
+    double ke2 = 2.0 * acc[ACC_KINETIC];
+    double G[M];
+    G[0] = (ke2 - n_f * kT) / q[0];
+    for (int c = 1; c < M; ++c) G[c] = (q[c - 1] * v[c - 1] * v[c - 1] - kT) / q[c];
+    v[M - 1] += 0.5 * d * G[M - 1];
+    for (int c = M - 2; c >= 0; --c) {
+        const double a = exp(-0.25 * d * v[c + 1]);
+        v[c] = (v[c] * a + 0.5 * d * G[c]) * a;
+    }
+    const double scale = exp(-d * v[0]);
+    ke2 *= scale * scale;
+    for (int c = 0; c < M; ++c) state[3 + c] += d * v[c];
+    G[0] = (ke2 - n_f * kT) / q[0];
+    for (int c = 0; c < M - 1; ++c) {
+        const double a = exp(-0.25 * d * v[c + 1]);
+        v[c] = (v[c] * a + 0.5 * d * G[c]) * a;
+        G[c + 1] = (q[c] * v[c] * v[c] - kT) / q[c + 1];
+    }
+    v[M - 1] += 0.5 * d * G[M - 1];
+    for (int c = 0; c < M; ++c) state[c] = v[c];
+    state[6] = scale;
+    acc[ACC_KINETIC] = 0.5 * ke2;
+}
+
+__global__ void k_scale_velocities(int64_t n3, double *__restrict__ vel, const double *__restrict__ scale) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n3) vel[i] *= *scale;
 }
 
 __global__ void k_kinetic(int64_t n, const double *__restrict__ mass, const double4 *__restrict__ pos4,
@@ -131,15 +170,27 @@ __global__ void k_get_state(int64_t n, const int32_t *__restrict__ user_of, cons
 static inline unsigned nb(int64_t n) { return (unsigned)((n + 255) / 256); }
 static inline float skin_half2(const mlip_ctx *c) { float h = 0.5f * (float)c->cfg.skin; return h * h; }
 
-int launch_kick_drift(mlip_ctx *c, double dt, cudaStream_t s) {
+int launch_kick_drift(mlip_ctx *c, double dt, cudaStream_t s, const double *vscale) {
     k_kick_drift<<<nb(c->n), 256, 0, s>>>(c->n, dt, c->grid, c->mass, skin_half2(c), c->pos4, c->vel, c->force, c->force_d, c->disp, c->status,
-                                               0.64f * skin_half2(c), c->rebuild_flag);
+                                               0.64f * skin_half2(c), c->rebuild_flag, vscale);
     c->launches += 1;
     MLIP_CUDA_TRY(c, cudaGetLastError());
     return MLIP_OK;
 }
 int launch_kick(mlip_ctx *c, double dt, cudaStream_t s) {
     k_kick<<<nb(c->n), 256, 0, s>>>(c->n, dt, c->mass, c->pos4, c->vel, c->force, c->force_d);
+    c->launches += 1;
+    MLIP_CUDA_TRY(c, cudaGetLastError());
+    return MLIP_OK;
+}
+int launch_nhc_half(mlip_ctx *c, double n_f, double kT, double q1, double qk, double dt, cudaStream_t s) {
+    k_nhc_half<<<1, 32, 0, s>>>(c->nhc, c->acc, n_f, kT, q1, qk, dt);
+    c->launches += 1;
+    MLIP_CUDA_TRY(c, cudaGetLastError());
+    return MLIP_OK;
+}
+int launch_scale_velocities(mlip_ctx *c, cudaStream_t s) {
+    k_scale_velocities<<<nb(3 * c->n), 256, 0, s>>>(3 * c->n, c->vel, c->nhc + 6);
     c->launches += 1;
     MLIP_CUDA_TRY(c, cudaGetLastError());
     return MLIP_OK;
