@@ -297,3 +297,54 @@ def test_displacement_triggered_rebuilds_keep_the_lists_valid():
     want = (np.repeat(np.arange(n * C), np.diff(ref.seg_ptr)) // C) * n + ref.nbr.astype(np.int64)
     assert np.isin(want, have).all()
     assert have.size > want.size                     # the lists carry the skin shell as well
+
+
+@pytest.mark.parametrize("precision", [0, 1])
+def test_dilute_system_with_isolated_atoms_ragged_tiles_and_an_absent_species(precision):
+    """Degenerate inputs: atoms with no neighbor inside r_cut (E_i = head(0), no force), lists that hold skin-shell entries
+    only, species counts that are not multiples of the tile size, and a declared species that no atom has."""
+    import paper_2608_16329_b200 as mlip
+    from paper_2608_16329_b200 import workloads as wl
+    rng = np.random.default_rng(11)
+    C, a, m = 4, 5.0, 7
+    grid = np.stack(np.meshgrid(*[np.arange(m)] * 3, indexing="ij"), -1).reshape(-1, 3).astype(np.float64)
+    keep = rng.random(len(grid)) < 0.3
+    pos = (grid[keep] + 0.5) * a + rng.uniform(-0.8, 0.8, (keep.sum(), 3))
+    box = np.array([m * a] * 3)
+    species = rng.choice([0, 1, 3], size=len(pos)).astype(np.int32)           # species 2 is absent
+    enc, head = wl.make_weights(C, 5, wl.ENC_OUT_SCALE[1], wl.HEAD_OUT_SCALE[1])
+    masses = np.array([20.0, 30.0, 40.0, 50.0])
+    model = oracle.Model(C, 6.0, enc, head)
+    pot = mlip.Potential(C, 6.0, 1.0, enc, head, masses, precision=precision)
+    pot.build_neighbors(pos, species, box)
+    out = pot.compute(want_e_atom=True)
+    pot.sync_status()
+    ref = oracle.evaluate(model, pos, species, box)
+    nl = oracle.neighbors(pos, species, C, box, 6.0)
+    counts = np.diff(nl.seg_ptr).reshape(-1, C).sum(1)
+    assert (counts == 0).sum() >= 5 and len(pos) % 8 != 0                      # the case really is degenerate
+    f = out["forces"].cpu().numpy().astype(np.float64)
+    ea = out["e_atom"].cpu().numpy().astype(np.float64)
+    e_tol, f_tol, ea_tol = (1e-10, 2e-9, 1e-9) if precision == 1 else (E_RTOL, F_ATOL, 2e-5)
+    assert abs(float(out["energy"].cpu()) - ref["energy"]) <= e_tol * abs(ref["energy"])
+    assert np.abs(f - ref["forces"]).max() <= f_tol
+    assert np.abs(ea - ref["e_atom"]).max() <= ea_tol * max(1.0, np.abs(ref["e_atom"]).max())
+    assert np.abs(f[counts == 0]).max() == 0.0                                 # isolated atoms feel nothing
+
+
+@pytest.mark.parametrize("precision", [0, 1])
+def test_single_atom(precision):
+    import paper_2608_16329_b200 as mlip
+    from paper_2608_16329_b200 import workloads as wl
+    enc, head = wl.make_weights(2, 9)
+    model = oracle.Model(2, 6.0, enc, head)
+    pos, species, box = np.array([[3.0, 4.0, 5.0]]), np.array([1], dtype=np.int32), np.array([20.0, 20.0, 20.0])
+    pot = mlip.Potential(2, 6.0, 1.0, enc, head, np.array([10.0, 12.0]), precision=precision)
+    pot.build_neighbors(pos, species, box)
+    out = pot.compute()
+    pot.step(2, 1.0, 1)
+    pot.sync_status()
+    ref = oracle.evaluate(model, pos, species, box)
+    assert abs(float(out["energy"].cpu()) - ref["energy"]) <= 1e-6 * abs(ref["energy"])
+    assert np.abs(out["forces"].cpu().numpy()).max() == 0.0
+    assert np.abs(out["virial"].cpu().numpy()).max() == 0.0
