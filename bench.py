@@ -35,7 +35,10 @@ DEFAULT_CELLS = 126            # 4 * 126^3 = 8,001,504 atoms: the size the targe
 REBUILD_EVERY = 10
 DT_FS = 1.0
 
-# Algorithmic work (fp32 operations, FMA = 2) of the fused kernel, per unit.  Derivation in the design doc.
+# Algorithmic work (fp32 operations, FMA = 2) of the fused kernel, per unit, with d = 16, k = 32:
+#   pair: geometry 60 + harmonics 150 + spline value 192 and value + derivative 320 + Eq. 4 (2 d k = 1,024)
+#         + Eq. 8-9 (4 d k = 2,048) + projection 168
+#   atom: invariants and Eq. 7 (3 d k = 1,536) + head forward and reverse (82,176) + SiLU (~5,000)
 FLOP_PER_PAIR = 3960.0         # pair inside r_cut: both neighbor loops (geometry, harmonics, spline, 6 d k contraction)
 FLOP_PER_SKIN_ENTRY = 24.0     # list entry between r_cut and r_cut + skin: distance test in both loops
 FLOP_PER_ATOM = 88700.0        # invariants, W_i, head forward + reverse, SiLU
