@@ -39,7 +39,7 @@ class _CModel(ctypes.Structure):
                 ("head_hidden", ctypes.c_int), ("head_layers", ctypes.c_int),
                 ("r_cut", ctypes.c_double),
                 ("enc_w", ctypes.c_void_p), ("head_w", ctypes.c_void_p), ("q", ctypes.c_void_p),
-                ("chi_e", ctypes.c_int), ("chi_r", ctypes.c_int)]
+                ("chi_e", ctypes.c_int), ("chi_r", ctypes.c_int), ("envelope", ctypes.c_int)]
 
 
 _lib = None
@@ -78,6 +78,7 @@ class Model:
     q: np.ndarray | None = None   # override the projection matrices (tests)
     chi_e: int = 0   # encoder conditioning (Section 3.2.2): 0 = species pair, C*C nets; 1 = neighbor species, C nets; 2 = none, 1 net
     chi_r: int = 0   # regression-network conditioning: 0 = central species, C nets; 1 = none, 1 net
+    envelope: int = 0   # smooth cutoff: 0 = cosine, 1 = quintic polynomial 1 - 10 x^3 + 15 x^4 - 6 x^5
 
     def __post_init__(self):
         self.enc_w = np.ascontiguousarray(self.enc_w, dtype=np.float64)
@@ -87,7 +88,7 @@ class Model:
         self.q = np.ascontiguousarray(self.q, dtype=np.float64)
         self._c = _CModel(self.n_species, self.k, self.l_max, self.enc_hidden, self.enc_layers,
                           self.head_hidden, self.head_layers, float(self.r_cut),
-                          _p(self.enc_w), _p(self.head_w), _p(self.q), self.chi_e, self.chi_r)
+                          _p(self.enc_w), _p(self.head_w), _p(self.q), self.chi_e, self.chi_r, self.envelope)
 
     @property
     def d(self) -> int:

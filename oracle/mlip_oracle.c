@@ -57,6 +57,7 @@ typedef struct {
     int chi_e;             /* species information given to the encoder (Section 3.2.2): 0 = pair (s_i, s_j), C*C nets;
                               1 = neighbor species s_j, C nets; 2 = none, one net */
     int chi_r;             /* ... to the regression network: 0 = central species s_i, C nets; 1 = none, one net */
+    int envelope;          /* smooth cutoff (the paper names none): 0 = (1 + cos(pi x)) / 2, 1 = 1 - 10 x^3 + 15 x^4 - 6 x^5, x = r / r_c */
 } oracle_model;
 
 static int enc_net_index(const oracle_model *m, int si, int sj) {
@@ -161,20 +162,25 @@ void oracle_encoder(const oracle_model *m, int si, int sj, double r, double *y, 
     }
 }
 
-/* cosine envelope and its derivative */
-static void envelope(double r, double r_cut, double *fc, double *dfc) {
-    if (r < r_cut) {
+/* smooth cutoff and its derivative: cosine, or the quintic that also has a vanishing second derivative at both ends */
+static void envelope(int kind, double r, double r_cut, double *fc, double *dfc) {
+    if (r >= r_cut) { *fc = 0.0; *dfc = 0.0; return; }
+    if (kind == 1) {
+        double x = r / r_cut;
+        *fc = 1.0 - 10.0 * x * x * x + 15.0 * x * x * x * x - 6.0 * x * x * x * x * x;
+        *dfc = (-30.0 * x * x + 60.0 * x * x * x - 30.0 * x * x * x * x) / r_cut;
+    } else {
         double x = M_PI * r / r_cut;
         *fc = 0.5 * (1.0 + cos(x));
         *dfc = -0.5 * (M_PI / r_cut) * sin(x);
-    } else { *fc = 0.0; *dfc = 0.0; }
+    }
 }
 
 /* radial feature g = f_c(r) E(r) and dg/dr */
 void oracle_radial(const oracle_model *m, int si, int sj, double r, double *g, double *dg) {
     double y[m->k], dy[m->k], fc, dfc;
     oracle_encoder(m, si, sj, r, y, dy);
-    envelope(r, m->r_cut, &fc, &dfc);
+    envelope(m->envelope, r, m->r_cut, &fc, &dfc);
     for (int c = 0; c < m->k; ++c) { g[c] = fc * y[c]; dg[c] = dfc * y[c] + fc * dy[c]; }
 }
 

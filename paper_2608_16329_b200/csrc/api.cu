@@ -129,6 +129,7 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
     if (!(cfg->r_cut > 0.0) || !(cfg->skin >= 0.0)) return fail(nullptr, MLIP_ERR_INVALID_ARG, "bad r_cut or skin");
     if (cfg->enc_conditioning < 0 || cfg->enc_conditioning > 2 || cfg->head_conditioning < 0 || cfg->head_conditioning > 1)
         return fail(nullptr, MLIP_ERR_INVALID_ARG, "bad enc_conditioning or head_conditioning");
+    if (cfg->envelope < 0 || cfg->envelope > 1) return fail(nullptr, MLIP_ERR_INVALID_ARG, "envelope must be 0 (cosine) or 1 (quintic)");
     // Species conditioning (Section 3.2.2): the kernels always index C*C encoder tables and C heads; the variants
     // with fewer networks are expanded here by repeating the shared ones.
     const int C = cfg->n_species;

@@ -10,11 +10,11 @@ namespace mlip {
 
 constexpr int MAX_ENC_H = 256;
 
-struct EncShape { int hidden, layers, k, n_species; double r_cut; };
+struct EncShape { int hidden, layers, k, n_species; double r_cut; int envelope; };
 
 __device__ inline double d_sigmoid(double x) { return 1.0 / (1.0 + exp(-x)); }
 
-// Encoder value and derivative (forward mode) times the cosine envelope.
+// Encoder value and derivative (forward mode) times the smooth cutoff.
 __device__ void eval_radial(const double *__restrict__ w, EncShape sh, double r, double *g, double *dg) {
     const int H = sh.hidden;
     double a[MAX_ENC_H], da[MAX_ENC_H], pre[MAX_ENC_H], dpre[MAX_ENC_H];
@@ -39,9 +39,18 @@ __device__ void eval_radial(const double *__restrict__ w, EncShape sh, double r,
         }
         w += (size_t)H * H + H;
     }
-    const double x = M_PI * r / sh.r_cut;
-    const double fc = r < sh.r_cut ? 0.5 * (1.0 + cos(x)) : 0.0;
-    const double dfc = r < sh.r_cut ? -0.5 * (M_PI / sh.r_cut) * sin(x) : 0.0;
+    double fc = 0.0, dfc = 0.0;   // smooth cutoff: cosine or quintic polynomial
+    if (r < sh.r_cut) {
+        if (sh.envelope == 1) {
+            const double x = r / sh.r_cut, x2 = x * x;
+            fc = 1.0 + x2 * x * (-10.0 + x * (15.0 - 6.0 * x));
+            dfc = x2 * (-30.0 + x * (60.0 - 30.0 * x)) / sh.r_cut;
+        } else {
+            const double x = M_PI * r / sh.r_cut;
+            fc = 0.5 * (1.0 + cos(x));
+            dfc = -0.5 * (M_PI / sh.r_cut) * sin(x);
+        }
+    }
     const double *b = w + (size_t)sh.k * H;
     for (int c = 0; c < sh.k; ++c) {
         double y = b[c], dy = 0.0;
@@ -136,7 +145,7 @@ int build_tables(mlip_ctx *c, const double *enc_w_host, size_t n_enc) {
     if (n_enc != net_size * n_nets) { c->err = "encoder weight count does not match the configured shape"; return MLIP_ERR_INVALID_ARG; }
     if (H > MAX_ENC_H) { c->err = "enc_hidden above 256 is not compiled in"; return MLIP_ERR_UNSUPPORTED; }
     const double r_min = cfg.table_r_min, h = (cfg.r_cut - r_min) / K;
-    const EncShape sh{H, cfg.enc_layers, k, C, cfg.r_cut};
+    const EncShape sh{H, cfg.enc_layers, k, C, cfg.r_cut, cfg.envelope};
     const int n_knot_pts = K + 1, n_chk = 4 * K;     // check at 4 points per interval, offset from the knots
     double *w = nullptr, *val = nullptr, *der = nullptr, *work = nullptr;
     unsigned long long *stats = nullptr;

@@ -138,3 +138,32 @@ def test_species_conditioning_equals_the_pair_conditioned_model_with_tied_networ
     # and the conditioning matters: the fully conditioned model gives something else
     full = oracle.compute(oracle.Model(C, w.r_cut, enc, head), w.pos, w.species, w.box, nl)
     assert abs(full["energy"] - a["energy"]) > 1e-6 * abs(full["energy"])
+
+
+def test_quintic_envelope_closed_form_values_and_contact_order():
+    """f_c = 1 - 10 x^3 + 15 x^4 - 6 x^5: f_c(r_c / 2) = 1/2, f_c and its first two derivatives vanish at r_c, and
+    f_c = 1 - O(x^3) near the origin.  Checked through g = f_c y on a random encoder."""
+    enc, head = wl.make_weights(1, seed=9)
+    m = oracle.Model(1, 6.0, enc, head, envelope=1)
+    cosine = oracle.Model(1, 6.0, enc, head)
+
+    def fc(r, eps=0.0):
+        y, _ = oracle.encoder(m, 0, 0, r + eps)
+        g, _ = oracle.radial(m, 0, 0, r + eps)
+        return (g / y)[0]
+
+    assert abs(fc(3.0) - 0.5) < 1e-15
+    assert abs(fc(1.5) - (1 - 10 / 64 + 15 / 256 - 6 / 1024)) < 1e-15
+    assert abs(fc(0.06) - 1.0) < 1.1e-5                        # 10 x^3 with x = 0.01
+    # contact of third order at the cutoff: f_c(r_c - e) = 10 (e / r_c)^3 + O(e^4)
+    for e in (0.06, 0.03):
+        assert abs(fc(6.0 - e) / (10 * (e / 6.0) ** 3) - 1.0) < 3 * e / 6.0
+    g, dg = oracle.radial(m, 0, 0, 6.2)
+    assert not g.any() and not dg.any()
+    # analytic derivative against a central difference, and the two envelopes really differ
+    g0, dg0 = oracle.radial(m, 0, 0, 4.3)
+    gp, _ = oracle.radial(m, 0, 0, 4.3 + 1e-6)
+    gm, _ = oracle.radial(m, 0, 0, 4.3 - 1e-6)
+    assert np.abs((gp - gm) / 2e-6 - dg0).max() < 1e-8 * max(1.0, np.abs(dg0).max())
+    gc, _ = oracle.radial(cosine, 0, 0, 4.3)
+    assert np.abs(gc - g0).max() > 1e-3 * np.abs(g0).max()
