@@ -312,7 +312,7 @@ def main():
     advance(args.warmup)
     pot.sync_status()
     barrier()
-    mlip.mlip_kernel_time(pot.ctx, reset=True)
+    mlip.mlip_get_timings(pot.ctx, reset=True)
     launches0 = mlip.mlip_get_counters(pot.ctx)["launches"]
     gpu_index = local_rank
     try:   # nvidia-smi numbers physical devices; honour a numeric CUDA_VISIBLE_DEVICES mapping
@@ -331,6 +331,7 @@ def main():
     clocks = sampler.stop() if rank == 0 else None
     status = pot.sync_status(raise_on_error=False)
     counters = mlip.mlip_get_counters(pot.ctx)
+    t_build, t_kernel, t_integrate = mlip.mlip_get_timings(pot.ctx)
     k_launches, k_ms = mlip.mlip_kernel_time(pot.ctx, reset=True)
     e_final = pot.energies().cpu().numpy()
     ms_max = max_over_ranks(ms, dev)
@@ -405,6 +406,8 @@ def main():
                            "l2": "inputs larger than L2 (positions + lists = %.1f GB per GPU)" % ((32 * n + 4 * entries) / 1e9)},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": counters["launches"] - launches0,
                 "roofline": roofline,
+                "device_ms_per_step": {"list_build": t_build / args.steps, "fused_kernel": t_kernel / args.steps,
+                                       "integrator": t_integrate / args.steps},
                 "resident_bytes_per_atom": resident / n,
                 "max_atoms_in_180GB_extrapolated": int(180e9 / (resident / n)),
                 "table_error": {"value": table_err[0], "deriv": table_err[1]},

@@ -226,6 +226,14 @@ int mlip_get_counters(mlip_ctx *ctx, int64_t *n_list_entries, int64_t *n_pairs_i
  */
 int mlip_kernel_time(mlip_ctx *ctx, int64_t *n_launches, double *total_ms, int reset);
 
+/*
+ * Device time (CUDA events on the launching streams, ms) of the three parts of the path since the last reset:
+ * list builds (binning + count + fill), fused-kernel launches, integrator kernels (kicks, drift, thermostat).
+ * Each part keeps its last 256 records.  Waits for the recorded events; reset != 0 clears all three (and the
+ * record of mlip_kernel_time).  Any pointer may be NULL.
+ */
+int mlip_get_timings(mlip_ctx *ctx, double *ms_build_host, double *ms_kernel_host, double *ms_integrate_host, int reset);
+
 size_t mlip_resident_bytes(const mlip_ctx *ctx);   /* device bytes the context holds */
 const char *mlip_last_error(const mlip_ctx *ctx);  /* text of the last failure (ctx may be NULL) */
 void mlip_destroy(mlip_ctx *ctx);

@@ -24,7 +24,7 @@ CODES = {v: k for k, v in ERRORS.items()}
 
 EXPORTS = ["mlip_create", "mlip_table_error", "mlip_build_neighbors", "mlip_get_neighbors", "mlip_get_neighbors_noalloc", "mlip_set_positions",
            "mlip_set_velocities", "mlip_compute", "mlip_compute_f64", "mlip_compute_host", "mlip_step", "mlip_step_nvt", "mlip_get_thermostat", "mlip_reset_thermostat", "mlip_get_rebuilds", "mlip_get_state",
-           "mlip_get_energies", "mlip_sync_status", "mlip_get_counters", "mlip_kernel_time",
+           "mlip_get_energies", "mlip_sync_status", "mlip_get_counters", "mlip_kernel_time", "mlip_get_timings",
            "mlip_resident_bytes", "mlip_last_error", "mlip_destroy"]
 
 
@@ -175,6 +175,13 @@ def mlip_get_thermostat(ctx):
 
 def mlip_reset_thermostat(ctx):
     _check(ctx, lib().mlip_reset_thermostat(ctx))
+
+
+def mlip_get_timings(ctx, reset=False):
+    """Device ms spent in (list builds, fused kernel, integrator kernels) since the last reset."""
+    b, k, i = ctypes.c_double(0), ctypes.c_double(0), ctypes.c_double(0)
+    _check(ctx, lib().mlip_get_timings(ctx, ctypes.byref(b), ctypes.byref(k), ctypes.byref(i), ctypes.c_int(int(reset))))
+    return b.value, k.value, i.value
 
 
 def mlip_get_rebuilds(ctx) -> int:

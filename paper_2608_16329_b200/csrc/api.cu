@@ -198,7 +198,9 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
             rc = MLIP_ERR_CUDA; c->err = "pinned host allocation failed"; break;
         }
         bool ev_ok = true;
-        for (int q = 0; q < 2 * mlip_ctx::EV_POOL; ++q) ev_ok = ev_ok && cudaEventCreate(&c->ev[q]) == cudaSuccess;
+        for (int q = 0; q < 2 * mlip_ctx::EV_POOL; ++q)
+            ev_ok = ev_ok && cudaEventCreate(&c->ev[q]) == cudaSuccess && cudaEventCreate(&c->ev_build[q]) == cudaSuccess &&
+                    cudaEventCreate(&c->ev_integrate[q]) == cudaSuccess;
         if (!ev_ok) { rc = MLIP_ERR_CUDA; c->err = "event creation failed"; break; }
         if (cudaMemcpy(c->mass, mass, sizeof(double) * cfg->n_species, cudaMemcpyHostToDevice) != cudaSuccess ||
             cudaMemset(c->status, 0, sizeof(int)) != cudaSuccess || cudaMemset(c->rebuild_flag, 0, sizeof(int)) != cudaSuccess ||
@@ -516,6 +518,35 @@ int mlip_kernel_time(mlip_ctx *c, int64_t *n_launches, double *total_ms, int res
     return MLIP_OK;
 }
 
+// Sum of the last min(count, EV_POOL) event pairs of a pool, in ms.
+static int pool_total(mlip_ctx *c, cudaEvent_t *pool, int64_t count, double *total_ms) {
+    const int64_t kept = count < mlip_ctx::EV_POOL ? count : mlip_ctx::EV_POOL;
+    double total = 0.0;
+    for (int64_t q = 0; q < kept; ++q) {
+        const int slot = (int)((count - 1 - q) % mlip_ctx::EV_POOL);
+        float ms = 0.f;
+        MLIP_CUDA_TRY(c, cudaEventSynchronize(pool[2 * slot + 1]));
+        MLIP_CUDA_TRY(c, cudaEventElapsedTime(&ms, pool[2 * slot], pool[2 * slot + 1]));
+        total += ms;
+    }
+    *total_ms = total;
+    return MLIP_OK;
+}
+
+int mlip_get_timings(mlip_ctx *c, double *ms_build, double *ms_kernel, double *ms_integrate, int reset) {
+    if (!c) return MLIP_ERR_INVALID_ARG;
+    double b = 0.0, k = 0.0, i = 0.0;
+    int rc;
+    if ((rc = pool_total(c, c->ev_build, c->build_count, &b)) != MLIP_OK) return rc;
+    if ((rc = pool_total(c, c->ev, c->ev_count, &k)) != MLIP_OK) return rc;
+    if ((rc = pool_total(c, c->ev_integrate, c->integrate_count, &i)) != MLIP_OK) return rc;
+    if (ms_build) *ms_build = b;
+    if (ms_kernel) *ms_kernel = k;
+    if (ms_integrate) *ms_integrate = i;
+    if (reset) { c->build_count = 0; c->ev_count = 0; c->integrate_count = 0; }
+    return MLIP_OK;
+}
+
 #ifdef MLIP_PHASE_CLOCKS
 int mlip_debug_acc(mlip_ctx *c, double *out16) {   // profiling builds only
     cudaDeviceSynchronize();
@@ -541,8 +572,11 @@ void mlip_destroy(mlip_ctx *c) {
     if (c->status_host) cudaFreeHost(c->status_host);
     if (c->total_host) cudaFreeHost(c->total_host);
     if (c->rebuild_host) cudaFreeHost(c->rebuild_host);
-    for (int q = 0; q < 2 * mlip_ctx::EV_POOL; ++q)
+    for (int q = 0; q < 2 * mlip_ctx::EV_POOL; ++q) {
         if (c->ev[q]) cudaEventDestroy(c->ev[q]);
+        if (c->ev_build[q]) cudaEventDestroy(c->ev_build[q]);
+        if (c->ev_integrate[q]) cudaEventDestroy(c->ev_integrate[q]);
+    }
     delete c;
 }
 

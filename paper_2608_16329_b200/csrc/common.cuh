@@ -125,6 +125,9 @@ struct mlip_ctx {
     static constexpr int EV_POOL = 256;
     cudaEvent_t ev[2 * EV_POOL] = {nullptr};
     int64_t ev_count = 0;          // launches timed since the last reset
+    // event pairs around list builds and around the integrator's kernels (mlip_get_timings)
+    cudaEvent_t ev_build[2 * EV_POOL] = {nullptr}, ev_integrate[2 * EV_POOL] = {nullptr};
+    int64_t build_count = 0, integrate_count = 0;
 };
 
 namespace mlip {
@@ -137,6 +140,10 @@ namespace mlip {
             return e_ == cudaErrorMemoryAllocation ? MLIP_ERR_OOM : MLIP_ERR_CUDA;        \
         }                                                                                 \
     } while (0)
+
+// Record the start / stop event of the next slot of a timing pool on stream s.
+inline void timing_begin(cudaEvent_t *pool, int64_t count, cudaStream_t s) { cudaEventRecord(pool[2 * (count % mlip_ctx::EV_POOL)], s); }
+inline void timing_end(cudaEvent_t *pool, int64_t &count, cudaStream_t s) { cudaEventRecord(pool[2 * (count % mlip_ctx::EV_POOL) + 1], s); count += 1; }
 
 // neighbor.cu
 int launch_pack_source(mlip_ctx *c, const double *pos, const int32_t *species, cudaStream_t s);

@@ -171,26 +171,34 @@ static inline unsigned nb(int64_t n) { return (unsigned)((n + 255) / 256); }
 static inline float skin_half2(const mlip_ctx *c) { float h = 0.5f * (float)c->cfg.skin; return h * h; }
 
 int launch_kick_drift(mlip_ctx *c, double dt, cudaStream_t s, const double *vscale) {
+    timing_begin(c->ev_integrate, c->integrate_count, s);
     k_kick_drift<<<nb(c->n), 256, 0, s>>>(c->n, dt, c->grid, c->mass, skin_half2(c), c->pos4, c->vel, c->force, c->force_d, c->disp, c->status,
                                                0.64f * skin_half2(c), c->rebuild_flag, vscale);
+    timing_end(c->ev_integrate, c->integrate_count, s);
     c->launches += 1;
     MLIP_CUDA_TRY(c, cudaGetLastError());
     return MLIP_OK;
 }
 int launch_kick(mlip_ctx *c, double dt, cudaStream_t s) {
+    timing_begin(c->ev_integrate, c->integrate_count, s);
     k_kick<<<nb(c->n), 256, 0, s>>>(c->n, dt, c->mass, c->pos4, c->vel, c->force, c->force_d);
+    timing_end(c->ev_integrate, c->integrate_count, s);
     c->launches += 1;
     MLIP_CUDA_TRY(c, cudaGetLastError());
     return MLIP_OK;
 }
 int launch_nhc_half(mlip_ctx *c, double n_f, double kT, double q1, double qk, double dt, cudaStream_t s) {
+    timing_begin(c->ev_integrate, c->integrate_count, s);
     k_nhc_half<<<1, 32, 0, s>>>(c->nhc, c->acc, n_f, kT, q1, qk, dt);
+    timing_end(c->ev_integrate, c->integrate_count, s);
     c->launches += 1;
     MLIP_CUDA_TRY(c, cudaGetLastError());
     return MLIP_OK;
 }
 int launch_scale_velocities(mlip_ctx *c, cudaStream_t s) {
+    timing_begin(c->ev_integrate, c->integrate_count, s);
     k_scale_velocities<<<nb(3 * c->n), 256, 0, s>>>(3 * c->n, c->vel, c->nhc + 6);
+    timing_end(c->ev_integrate, c->integrate_count, s);
     c->launches += 1;
     MLIP_CUDA_TRY(c, cudaGetLastError());
     return MLIP_OK;

@@ -211,6 +211,7 @@ int launch_pack_source(mlip_ctx *c, const double *pos, const int32_t *species, c
 
 // Sort (pos4_src, vel_src, user_src) into cell order and build the lists.
 int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
+    timing_begin(c->ev_build, c->build_count, s);
     const int64_t n = c->n;
     const CellGrid &g = c->grid;
     const int C = c->cfg.n_species;
@@ -245,6 +246,7 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
     }
     k_neighbors<true><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, c->cell_start, c->nbr_count, c->nbr_off, c->nbr, c->nbr_cap, c->status);
     c->launches += 1;
+    timing_end(c->ev_build, c->build_count, s);
     MLIP_CUDA_TRY(c, cudaGetLastError());
     return MLIP_OK;
 }

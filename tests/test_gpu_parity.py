@@ -367,3 +367,25 @@ def test_quintic_envelope_matches_oracle(precision):
     e_tol, f_tol = (1e-10, 5e-9) if precision == 1 else (E_RTOL, F_ATOL)
     assert abs(float(out["energy"].cpu()) - ref["energy"]) <= e_tol * abs(ref["energy"])
     assert np.abs(out["forces"].cpu().numpy() - ref["forces"]).max() <= f_tol
+
+
+def test_timings_cover_the_three_parts_of_a_step():
+    import time
+    import paper_2608_16329_b200 as mlip
+    w, model, pot = make_pair(3, 16, 1.0)
+    pot.build_neighbors(w.pos, w.species, w.box)
+    pot.set_velocities(w.vel)
+    pot.step(2, 1.0, 0)
+    pot.sync_status()
+    mlip.mlip_get_timings(pot.ctx, reset=True)
+    t0 = time.perf_counter()
+    pot.step(10, 1.0, 5)
+    pot.sync_status()
+    wall_ms = (time.perf_counter() - t0) * 1e3
+    build, kernel, integrate = mlip.mlip_get_timings(pot.ctx)
+    n, k_ms = mlip.mlip_kernel_time(pot.ctx)
+    assert n == 10 and abs(k_ms - kernel) < 1e-9
+    assert build > 0 and integrate > 0 and kernel > build / 10
+    assert build + kernel + integrate <= wall_ms
+    assert mlip.mlip_get_timings(pot.ctx, reset=True)[1] == kernel
+    assert mlip.mlip_get_timings(pot.ctx) == (0.0, 0.0, 0.0)
