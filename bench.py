@@ -66,6 +66,8 @@ def parse_args():
                          "3-species alloy and ionic stand-ins at their full sizes (extra data points, not the contract line)")
     ap.add_argument("--precision", default="f32", choices=["f32", "f64"],
                     help="f64 runs the double-precision evaluation path instead (an extra data point, not the contract line)")
+    ap.add_argument("--deterministic", action="store_true",
+                    help="force_mode = 1: integer accumulation of forces, energy and virial (bit-reproducible): an extra data point")
     ap.add_argument("--ensemble", default="nve", choices=["nve", "nvt"],
                     help="nvt adds the Nose-Hoover-chain thermostat (the paper's ensemble) to every step: an extra data point")
     ap.add_argument("--k", type=int, default=32, choices=[16, 32, 64], help="radial channels (other than 32: --precision f64 only)")
@@ -292,12 +294,12 @@ def main():
         enc, head = wl.workload_weights(cfg, w.n_species)
     else:   # descriptor-shape variants of the paper's ablations: same recipe, networks of that shape
         enc, head = wl.make_weights(w.n_species, wl.BASE_SEED + cfg + 1000, wl.ENC_OUT_SCALE[cfg], wl.HEAD_OUT_SCALE[cfg],
-                                    k=args.k, l_max=args.lmax)
+                                    k=args.k, l_max=args.lmax, force_mode=1 if args.deterministic else 0)
     rebuild_every = REBUILD_EVERY if cfg != 4 else 3   # the ionic stand-in is far from equilibrium under random weights
     n = w.n_atoms
     f64 = args.precision == "f64"
     pot = mlip.Potential(w.n_species, w.r_cut, w.skin, enc, head, w.masses, device=local_rank, precision=1 if f64 else 0,
-                         k=args.k, l_max=args.lmax)
+                         k=args.k, l_max=args.lmax, force_mode=1 if args.deterministic else 0)
     table_err = mlip.mlip_table_error(pot.ctx)
 
     # ---- device-resident run: inputs already in HBM when timing starts ----
@@ -401,7 +403,8 @@ def main():
                 "dtype": args.precision, "data": "synthetic",
                 "config": {"workload": f"cfg{cfg} {w.name}: {n} atoms, {w.n_species} species, r_cut 6 A, skin 1 A, "
                                        f"{args.ensemble.upper()} dt 1 fs, list rebuild every {rebuild_every} steps"
-                                       + ("" if default_shape else f", k = {args.k}, l_max = {args.lmax}"),
+                                       + ("" if default_shape else f", k = {args.k}, l_max = {args.lmax}")
+                                       + (", deterministic force mode" if args.deterministic else ""),
                            "atoms_per_gpu": n, "parallelism": "replicas" if world > 1 else "single",
                            "l2": "inputs larger than L2 (positions + lists = %.1f GB per GPU)" % ((32 * n + 4 * entries) / 1e9)},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": counters["launches"] - launches0,

@@ -75,6 +75,10 @@ typedef struct {
     int enc_conditioning; /* species information given to the encoder (Section 3.2.2): 0 = the pair (s_i, s_j), C*C nets
                              (the paper's choice); 1 = the neighbor species s_j, C nets; 2 = none, one net */
     int head_conditioning;/* ... to the regression network: 0 = central species s_i, C nets; 1 = none, one net */
+    int force_mode;       /* 0: floating-point atomics for the force scatter and the energy / virial totals (results vary in
+                             the last bits from run to run); 1: deterministic -- those sums are taken in integer arithmetic
+                             (forces in units of 2^-32 eV/Angstrom), so equal inputs give bit-identical outputs and
+                             trajectories; +24 bytes per atom, fp32 path only */
     int envelope;         /* smooth cutoff f_c multiplying the encoder output (the paper names none): 0 = (1 + cos(pi r / r_c)) / 2,
                              1 = 1 - 10 x^3 + 15 x^4 - 6 x^5 with x = r / r_c (second derivative also vanishes at r_c) */
 } mlip_config;

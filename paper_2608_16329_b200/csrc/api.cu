@@ -49,6 +49,7 @@ static void free_atoms(mlip_ctx *c) {
     dev_free(c, &c->center_order, n); dev_free(c, &c->cell_of, n);
     dev_free(c, &c->nbr_count, n); dev_free(c, &c->nbr_off, n + 1);
     if (c->cfg.precision == 1) { dev_free(c, &c->force_d, 3 * n); dev_free(c, &c->e_atom_d, n); }
+    if (c->cfg.force_mode == 1) dev_free(c, &c->force_fx, 3 * n);
     c->cap_atoms = 0;
 }
 
@@ -72,6 +73,7 @@ static int ensure_capacity(mlip_ctx *c, int64_t n, int64_t n_cells) {
         TRY_ALLOC(c->center_order, m); TRY_ALLOC(c->cell_of, m);
         TRY_ALLOC(c->nbr_count, m); TRY_ALLOC(c->nbr_off, m + 1);
         if (c->cfg.precision == 1) { TRY_ALLOC(c->force_d, 3 * m); TRY_ALLOC(c->e_atom_d, m); }
+        if (c->cfg.force_mode == 1) TRY_ALLOC(c->force_fx, 3 * m);
         c->cap_atoms = n;
     }
     if (n_cells > c->cap_cells) {
@@ -129,6 +131,8 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
     if (!(cfg->r_cut > 0.0) || !(cfg->skin >= 0.0)) return fail(nullptr, MLIP_ERR_INVALID_ARG, "bad r_cut or skin");
     if (cfg->enc_conditioning < 0 || cfg->enc_conditioning > 2 || cfg->head_conditioning < 0 || cfg->head_conditioning > 1)
         return fail(nullptr, MLIP_ERR_INVALID_ARG, "bad enc_conditioning or head_conditioning");
+    if (cfg->force_mode < 0 || cfg->force_mode > 1) return fail(nullptr, MLIP_ERR_INVALID_ARG, "force_mode must be 0 (atomics) or 1 (deterministic)");
+    if (cfg->force_mode == 1 && cfg->precision == 1) return fail(nullptr, MLIP_ERR_UNSUPPORTED, "the deterministic force mode is compiled for the fp32 path only");
     if (cfg->envelope < 0 || cfg->envelope > 1) return fail(nullptr, MLIP_ERR_INVALID_ARG, "envelope must be 0 (cosine) or 1 (quintic)");
     // Species conditioning (Section 3.2.2): the kernels always index C*C encoder tables and C heads; the variants
     // with fewer networks are expanded here by repeating the shared ones.
@@ -189,6 +193,7 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
         if ((rc = dev_alloc(c, &c->status, 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->rebuild_flag, 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->nhc, 8)) != MLIP_OK) break;
+        if ((rc = dev_alloc(c, &c->acc_fx, 10)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->tile_counter, (size_t)MAX_SPECIES)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->species_start, (size_t)MAX_SPECIES + 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->stage_out, 10)) != MLIP_OK) break;
@@ -566,7 +571,7 @@ void mlip_destroy(mlip_ctx *c) {
     free_cells(c);
     cudaFree(c->nbr); cudaFree(c->scan_tmp); cudaFree(c->head_w); cudaFree(c->table); cudaFree(c->mass);
     cudaFree(c->head_w_d); cudaFree(c->table_d);
-    cudaFree(c->acc); cudaFree(c->pair_counter); cudaFree(c->status); cudaFree(c->rebuild_flag); cudaFree(c->nhc); cudaFree(c->tile_counter);
+    cudaFree(c->acc); cudaFree(c->pair_counter); cudaFree(c->status); cudaFree(c->rebuild_flag); cudaFree(c->nhc); cudaFree(c->acc_fx); cudaFree(c->tile_counter);
     cudaFree(c->species_start); cudaFree(c->stage_pos); cudaFree(c->stage_species); cudaFree(c->stage_force);
     cudaFree(c->stage_out);
     if (c->status_host) cudaFreeHost(c->status_host);

@@ -81,6 +81,8 @@ struct mlip_ctx {
     double *vel = nullptr;         // [N][3]
     int32_t *user_of = nullptr;    // internal -> caller index
     float4 *force = nullptr;       // fx, fy, fz, unused
+    long long *force_fx = nullptr; // [N][3] fixed-point forces, deterministic mode only
+    long long *acc_fx = nullptr;   // [10] fixed-point energy and virial, deterministic mode only
     float *e_atom = nullptr;       // E_i, internal order
     float *disp = nullptr;         // [N][3] displacement since the last build
     int32_t *center_order = nullptr;  // internal indices sorted by (species, cell)

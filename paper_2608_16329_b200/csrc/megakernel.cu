@@ -118,6 +118,18 @@ __device__ __forceinline__ void mma_tf32_z(float (&d)[4], uint32_t a0, uint32_t 
 // chains short (a fresh accumulator per k-step, folded into the running sum by a rounded fp32
 // add): a long chain of same-sign terms otherwise drifts by ~1e-6 relative.
 
+// Deterministic mode (force_mode = 1): every sum whose order depends on scheduling -- the force scatter across
+// warps, the energy and virial totals -- is taken in integer arithmetic, which is associative, so two runs on the
+// same input agree bit for bit.  Per-atom and per-pair terms are computed in a fixed order in either mode.
+constexpr float FORCE_FX = 4294967296.f;        // 2^32 per eV/Angstrom
+constexpr double ENERGY_FX = 4294967296.0;      // 2^32 per eV
+constexpr double VIRIAL_FX = 268435456.0;       // 2^28 per eV
+__device__ __forceinline__ void fixed_add3(long long *p, float x, float y, float z) {
+    atomicAdd(reinterpret_cast<unsigned long long *>(p), (unsigned long long)__float2ll_rn(x * FORCE_FX));
+    atomicAdd(reinterpret_cast<unsigned long long *>(p + 1), (unsigned long long)__float2ll_rn(y * FORCE_FX));
+    atomicAdd(reinterpret_cast<unsigned long long *>(p + 2), (unsigned long long)__float2ll_rn(z * FORCE_FX));
+}
+
 // Optional per-phase cycle counters (profiling builds only: -DMLIP_PHASE_CLOCKS).  Slots 16.. of
 // the accumulator array receive the summed clock64 ticks of lane 0 of every warp.
 #ifdef MLIP_PHASE_CLOCKS
@@ -148,6 +160,8 @@ struct KernelArgs {
     const int32_t *nbr;
     const float *head_pack;
     float4 *force;
+    long long *force_fx;   // deterministic mode: forces as 2^-32 eV/Angstrom integers [N][3]
+    long long *acc_fx;     // deterministic mode: energy (2^-32 eV) and virial (2^-28 eV) integers [10]
     float *e_atom;
     double *acc;
     unsigned long long *pair_counter;
@@ -324,6 +338,7 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
 }
 
 // ---------------- Derivation of one atom (Eq. 8-10) ----------------
+template <bool DET>
 __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView &tv, const double4 &pi, int i, int64_t beg, int64_t end,
                                             float4 *pq, float *scr, int queued, int lane, const uint32_t (&Wh)[4][4],
                                             const uint32_t (&Wl)[4][4], float (&vir)[9], PhaseClock &pc) {
@@ -449,7 +464,8 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
             const float qy = s * uy + (ty - tu * uy) * rinv;
             const float qz = s * uz + (tz - tu * uz) * rinv;
             fx += qx; fy += qy; fz += qz;
-            atomicAdd(&k.force[j], make_float4(-qx, -qy, -qz, 0.f));   // one 128-bit reduction per pair
+            if (DET) fixed_add3(k.force_fx + 3 * (size_t)j, -qx, -qy, -qz);
+            else atomicAdd(&k.force[j], make_float4(-qx, -qy, -qz, 0.f));   // one 128-bit reduction per pair
             vir[0] -= x * qx; vir[1] -= x * qy; vir[2] -= x * qz;
             vir[3] -= y * qx; vir[4] -= y * qy; vir[5] -= y * qz;
             vir[6] -= z * qx; vir[7] -= z * qy; vir[8] -= z * qz;
@@ -474,7 +490,8 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
         fz += __shfl_xor_sync(0xffffffffu, fz, o);
     }
     if (lane == 0) {
-        atomicAdd(&k.force[i], make_float4(fx, fy, fz, 0.f));
+        if (DET) fixed_add3(k.force_fx + 3 * (size_t)i, fx, fy, fz);
+        else atomicAdd(&k.force[i], make_float4(fx, fy, fz, 0.f));
     }
 }
 
@@ -581,6 +598,7 @@ struct NextAtom {
 // ---------------- Regression (Eq. 6) forward and reverse for the group's tile ----------------
 // In: sX = invariants [atom][128].  Out: sX = dE/dG; per-atom energies written.
 // hc = biases [4][64], w_out [64], b_out of the species in shared memory.  wg = warp within the group.
+template <bool DET>
 __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float *hb, const float *hc, int species, int count, int first,
                                           int group, int wg, int lane, double &e_sum, NextAtom &nx, PhaseClock &pc) {
     const float *hp = k.head_pack + (size_t)species * HP_TOTAL;
@@ -651,7 +669,7 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
     e_i += hc[HEAD_L * HEAD_H + HEAD_H];
     if (lane == 0 && atom < count) {
         k.e_atom[__ldg(k.center_order + first + atom)] = e_i;
-        e_sum += (double)e_i;
+        e_sum += DET ? rint((double)e_i * ENERGY_FX) : (double)e_i;   // DET: exact integer sums
     }
 
     // reverse through the hidden layers 3, 2, 1 (each with its skip path)
@@ -684,7 +702,7 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
     group_sync(group);
 }
 
-template <bool TAB_SMEM>
+template <bool TAB_SMEM, bool DET>
 __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words) {
     extern __shared__ __align__(16) float smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -703,6 +721,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
 
     double e_sum = 0.0;
     float vir[9] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    double vir_fx = 0.0;   // DET: lane q < 9 keeps component q as an exact integer-valued sum
     unsigned long long n_pairs = 0;
     TableView tv;
     PhaseClock pc;
@@ -801,7 +820,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
             nx.k = &k; nx.sidx = pf; nx.meta = pf + PF_IDX;
             nx.slot = (tile_next < n_tiles && s_beg + tile_next * TILE + wg < s_end) ? s_beg + tile_next * TILE + wg : -1;
             nx.i = 0; nx.beg = 0; nx.end = 0;
-            head_tile(k, sX, hb, hc, species, count, first, group, wg, lane, e_sum, nx, pc);
+            head_tile<DET>(k, sX, hb, hc, species, count, first, group, wg, lane, e_sum, nx, pc);
             prefetched = nx.slot >= 0;
             pc.mark(9);
 
@@ -828,7 +847,17 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
                     split_tf32(w2, Wh[ks][2], Wl[ks][2]);
                     split_tf32(w3, Wh[ks][3], Wl[ks][3]);
                 }
-                derive_atom(k, tv, pi, i, beg, end, pq, scr, queued, lane, Wh, Wl, vir, pc);
+                derive_atom<DET>(k, tv, pi, i, beg, end, pq, scr, queued, lane, Wh, Wl, vir, pc);
+                if (DET) {   // fold this atom's virial in now: lane sums in a fixed order, then integers
+#pragma unroll
+                    for (int q = 0; q < 9; ++q) {
+                        float x = vir[q];
+#pragma unroll
+                        for (int o = 16; o; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+                        if (lane == q) vir_fx += rint((double)x * VIRIAL_FX);
+                        vir[q] = 0.f;
+                    }
+                }
             }
             pc.mark(10);
         }
@@ -836,17 +865,20 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
     pc.flush(k.acc, lane);
 
     // per-warp totals -> global accumulators
+    if (DET) {
+        if (lane < 9) atomicAdd(reinterpret_cast<unsigned long long *>(k.acc_fx + 1 + lane), (unsigned long long)(long long)vir_fx);
+        if (lane == 0) atomicAdd(reinterpret_cast<unsigned long long *>(k.acc_fx), (unsigned long long)(long long)e_sum);
+    } else {
 #pragma unroll
-    for (int q = 0; q < 9; ++q) {
-        float x = vir[q];
+        for (int q = 0; q < 9; ++q) {
+            float x = vir[q];
 #pragma unroll
-        for (int o = 16; o; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
-        if (lane == 0) atomicAdd(&k.acc[ACC_VIRIAL + q], (double)x);
+            for (int o = 16; o; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+            if (lane == 0) atomicAdd(&k.acc[ACC_VIRIAL + q], (double)x);
+        }
+        if (lane == 0) atomicAdd(&k.acc[ACC_ENERGY], e_sum);
     }
-    if (lane == 0) {
-        atomicAdd(&k.acc[ACC_ENERGY], e_sum);
-        atomicAdd(k.pair_counter, n_pairs);
-    }
+    if (lane == 0) atomicAdd(k.pair_counter, n_pairs);
 }
 
 // ---------------- host side ----------------
@@ -903,8 +935,28 @@ int upload_head(mlip_ctx *c, const double *w) {
     return MLIP_OK;
 }
 
+// Deterministic mode: integer sums -> the float / double outputs the rest of the library reads.
+__global__ void k_fixed_finish(int64_t n, const long long *__restrict__ force_fx, const long long *__restrict__ acc_fx,
+                               float4 *__restrict__ force, double *__restrict__ acc) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) {
+        const double inv = 1.0 / (double)FORCE_FX;
+        force[i] = make_float4((float)((double)force_fx[3 * i] * inv), (float)((double)force_fx[3 * i + 1] * inv),
+                               (float)((double)force_fx[3 * i + 2] * inv), 0.f);
+    }
+    if (i == 0) {
+        acc[ACC_ENERGY] = (double)acc_fx[0] / ENERGY_FX;
+        for (int q = 0; q < 9; ++q) acc[ACC_VIRIAL + q] = (double)acc_fx[1 + q] / VIRIAL_FX;
+    }
+}
+
 int launch_megakernel(mlip_ctx *c, cudaStream_t s) {
     const int64_t n = c->n;
+    const bool det = c->cfg.force_mode == 1;
+    if (det) {
+        MLIP_CUDA_TRY(c, cudaMemsetAsync(c->force_fx, 0, sizeof(long long) * 3 * n, s));
+        MLIP_CUDA_TRY(c, cudaMemsetAsync(c->acc_fx, 0, sizeof(long long) * 10, s));
+    }
     MLIP_CUDA_TRY(c, cudaMemsetAsync(c->force, 0, sizeof(float4) * n, s));
     MLIP_CUDA_TRY(c, cudaMemsetAsync(c->acc, 0, sizeof(double) * ACC_KINETIC, s));
     MLIP_CUDA_TRY(c, cudaMemsetAsync(c->pair_counter, 0, sizeof(unsigned long long), s));
@@ -915,8 +967,9 @@ int launch_megakernel(mlip_ctx *c, cudaStream_t s) {
     const int tab_words = in_smem ? table_smem_words(c) : 0;
     const size_t smem_bytes = sizeof(float) * (size_t)(FIXED_WORDS + tab_words);
     if (!c->kernel_ready) {
-        cudaError_t e = in_smem ? cudaFuncSetAttribute(k_mega<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes)
-                                : cudaFuncSetAttribute(k_mega<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+        const void *fn = in_smem ? (det ? (const void *)k_mega<true, true> : (const void *)k_mega<true, false>)
+                                 : (det ? (const void *)k_mega<false, true> : (const void *)k_mega<false, false>);
+        cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
         if (e != cudaSuccess) { c->err = std::string("fused kernel shared memory: ") + cudaGetErrorString(e); return MLIP_ERR_CUDA; }
         c->kernel_ready = true;
     }
@@ -924,11 +977,18 @@ int launch_megakernel(mlip_ctx *c, cudaStream_t s) {
     k.n = n; k.n_species = c->cfg.n_species; k.grid = c->grid; k.rc2 = c->cfg.r_cut * c->cfg.r_cut; k.tab = c->tab;
     k.pos4 = c->pos4; k.center_order = c->center_order; k.species_start = c->species_start;
     k.nbr_off = c->nbr_off; k.nbr = c->nbr; k.head_pack = c->head_w; k.force = c->force; k.e_atom = c->e_atom;
+    k.force_fx = c->force_fx; k.acc_fx = c->acc_fx;
     k.acc = c->acc; k.pair_counter = c->pair_counter; k.status = c->status; k.tile_counter = c->tile_counter;
     const int slot = (int)(c->ev_count % mlip_ctx::EV_POOL);
     MLIP_CUDA_TRY(c, cudaEventRecord(c->ev[2 * slot], s));
-    if (in_smem) k_mega<true><<<blocks, NW * 32, smem_bytes, s>>>(k, tab_words);
-    else k_mega<false><<<blocks, NW * 32, smem_bytes, s>>>(k, tab_words);
+    if (in_smem && det) k_mega<true, true><<<blocks, NW * 32, smem_bytes, s>>>(k, tab_words);
+    else if (in_smem) k_mega<true, false><<<blocks, NW * 32, smem_bytes, s>>>(k, tab_words);
+    else if (det) k_mega<false, true><<<blocks, NW * 32, smem_bytes, s>>>(k, tab_words);
+    else k_mega<false, false><<<blocks, NW * 32, smem_bytes, s>>>(k, tab_words);
+    if (det) {
+        k_fixed_finish<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(n, c->force_fx, c->acc_fx, c->force, c->acc);
+        c->launches += 1;
+    }
     MLIP_CUDA_TRY(c, cudaEventRecord(c->ev[2 * slot + 1], s));
     c->ev_count += 1;
     c->launches += 1;

@@ -389,3 +389,43 @@ def test_timings_cover_the_three_parts_of_a_step():
     assert build + kernel + integrate <= wall_ms
     assert mlip.mlip_get_timings(pot.ctx, reset=True)[1] == kernel
     assert mlip.mlip_get_timings(pot.ctx) == (0.0, 0.0, 0.0)
+
+
+def test_deterministic_force_mode_is_bit_reproducible_and_matches_oracle():
+    """force_mode = 1 takes every scheduling-dependent sum in integer arithmetic: two contexts fed the same input give
+    bit-identical energies, forces, virial and trajectories (the default mode agrees only to rounding)."""
+    import paper_2608_16329_b200 as mlip
+    from paper_2608_16329_b200 import workloads as wl
+    w = wl.make_workload(5, n_cells=12)                    # 6,912 atoms: thousands of tiles over all SMs
+    enc, head = wl.workload_weights(5, 6)
+    runs = []
+    for _ in range(2):
+        pot = mlip.Potential(6, w.r_cut, 1.0, enc, head, w.masses, force_mode=1)
+        pot.build_neighbors(w.pos, w.species, w.box)
+        pot.set_velocities(w.vel)
+        first = pot.compute(want_e_atom=True)
+        again = pot.compute(want_e_atom=True)
+        for key in ("energy", "forces", "virial", "e_atom"):
+            assert pot.torch.equal(first[key], again[key]), key
+        pot.step(12, 1.0, 5)
+        pot.sync_status()
+        pos, vel, _ = pot.state()
+        runs.append((first, pos.cpu().numpy(), vel.cpu().numpy(), pot.energies().cpu().numpy()))
+        pot.close()
+    a, b = runs
+    for key in ("energy", "forces", "virial", "e_atom"):
+        assert a[0][key].cpu().numpy().tobytes() == b[0][key].cpu().numpy().tobytes(), key
+    assert a[1].tobytes() == b[1].tobytes() and a[2].tobytes() == b[2].tobytes()
+    assert a[3][0] == b[3][0]
+    model = oracle.Model(6, w.r_cut, enc, head)
+    rows = np.arange(0, w.n_atoms, 16)
+    ref = oracle.sampled(model, w.pos, w.species, w.box, rows)
+    f = a[0]["forces"].cpu().numpy().astype(np.float64)
+    assert np.abs(f[rows] - ref["forces"]).max() <= F_ATOL
+    assert np.abs(a[0]["e_atom"].cpu().numpy()[rows] - ref["e_atom"]).max() <= 2e-5 * np.abs(ref["e_atom"]).max()
+    full = oracle.evaluate(model, w.pos, w.species, w.box)
+    assert abs(float(a[0]["energy"].cpu()) - full["energy"]) <= E_RTOL * abs(full["energy"])
+    assert np.abs(a[0]["virial"].cpu().numpy().reshape(3, 3) - full["virial"]).max() <= 1e-5 * np.abs(full["virial"]).max()
+    with pytest.raises(mlip.MlipError) as err:
+        mlip.Potential(6, w.r_cut, 1.0, enc, head, w.masses, force_mode=1, precision=1)
+    assert err.value.code == mlip.binding.CODES["MLIP_ERR_UNSUPPORTED"]
