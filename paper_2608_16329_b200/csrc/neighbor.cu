@@ -107,6 +107,9 @@ __global__ void k_center_order(int n_cells, int n_species, const int32_t *__rest
 }
 
 // Warp per atom over the surrounding cells.  FILL = false counts, FILL = true writes the list.
+// Lanes 0..26 fetch the atom ranges of the (up to) 27 cells in one round trip; the cells are then visited
+// in a fixed order (x, y, z offsets ascending: the order of the list) with the positions of the next
+// cell requested before the current one is tested, so that an atom costs a few load latencies instead of 54.
 template <bool FILL>
 __global__ void __launch_bounds__(256) k_neighbors(int64_t n, CellGrid g, double rl2, const double4 *__restrict__ pos4,
                                                    const int32_t *__restrict__ cell_start, int32_t *__restrict__ nbr_count,
@@ -116,21 +119,31 @@ __global__ void __launch_bounds__(256) k_neighbors(int64_t n, CellGrid g, double
     int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (i >= n) return;
     const double4 pi = pos4[i];
-    int c0[3] = {cell_coord(pi.x, g.inv_edge[0], g.n[0]), cell_coord(pi.y, g.inv_edge[1], g.n[1]),
-                 cell_coord(pi.z, g.inv_edge[2], g.n[2])};
-    int lst[3][3], nl[3];
+    // this lane's cell: offsets (ox, oy, oz) = (lane / 9, lane / 3 % 3, lane % 3); dimensions with fewer than
+    // three cells list each cell once
+    int cb = 0, ce = 0;
+    {
+        const int o[3] = {lane / 9, (lane / 3) % 3, lane % 3};
+        const double p[3] = {pi.x, pi.y, pi.z};
+        int cc[3];
+        bool ok = lane < 27;
 #pragma unroll
-    for (int a = 0; a < 3; ++a) {   // distinct periodic cells among c-1, c, c+1
-        int na = g.n[a];
-        nl[a] = na < 3 ? na : 3;
-        for (int o = 0; o < 3; ++o) {
-            int c = c0[a] + o - 1;
+        for (int a = 0; a < 3; ++a) {
+            const int na = g.n[a];
+            const int c0 = cell_coord(p[a], g.inv_edge[a], na);
+            int c = c0 + o[a] - 1;
             c = c < 0 ? c + na : (c >= na ? c - na : c);
-            lst[a][o] = c;
+            if (na < 3) { c = o[a]; ok = ok && o[a] < na; }
+            cc[a] = c;
         }
-        if (na == 2) { lst[a][0] = 0; lst[a][1] = 1; }
-        if (na == 1) lst[a][0] = 0;
+        if (ok) {
+            const int c = (cc[0] * g.n[1] + cc[1]) * g.n[2] + cc[2];
+            cb = cell_start[c]; ce = cell_start[c + 1];
+        }
     }
+    const float boxf[3] = {(float)g.box[0], (float)g.box[1], (float)g.box[2]};
+    const float halff[3] = {(float)g.half[0], (float)g.half[1], (float)g.half[2]};
+    const float rl2_lo = (float)(rl2 * (1.0 - 1e-5)), rl2_hi = (float)(rl2 * (1.0 + 1e-5));
     int64_t off = 0;
     bool writable = true;
     if (FILL) {
@@ -139,27 +152,44 @@ __global__ void __launch_bounds__(256) k_neighbors(int64_t n, CellGrid g, double
         if (!writable && lane == 0) atomicOr(status, FLAG_NEIGHBOR_OVERFLOW);
     }
     int cnt = 0;
-    for (int x = 0; x < nl[0]; ++x)
-        for (int y = 0; y < nl[1]; ++y)
-            for (int z = 0; z < nl[2]; ++z) {
-                int c = (lst[0][x] * g.n[1] + lst[1][y]) * g.n[2] + lst[2][z];
-                int beg = cell_start[c], end = cell_start[c + 1];
-                for (int base = beg; base < end; base += 32) {
-                    int j = base + lane;
-                    bool hit = false;
-                    if (j < end && j != i) {
-                        double4 pj = pos4[j];
-                        double dx = min_image(__dsub_rn(pj.x, pi.x), g.box[0], g.half[0]);
-                        double dy = min_image(__dsub_rn(pj.y, pi.y), g.box[1], g.half[1]);
-                        double dz = min_image(__dsub_rn(pj.z, pi.z), g.box[2], g.half[2]);
-                        double d2 = __dadd_rn(__dadd_rn(__dmul_rn(dx, dx), __dmul_rn(dy, dy)), __dmul_rn(dz, dz));
-                        hit = d2 < rl2;
-                    }
-                    unsigned m = __ballot_sync(0xffffffffu, hit);
-                    if (FILL && hit && writable) nbr[off + cnt + __popc(m & ((1u << lane) - 1u))] = j;
-                    cnt += __popc(m);
+    int beg = __shfl_sync(0xffffffffu, cb, 0), end = __shfl_sync(0xffffffffu, ce, 0);
+    double4 pj_next = make_double4(0.0, 0.0, 0.0, 0.0);
+    if (beg + lane < end) pj_next = pos4[beg + lane];
+    for (int it = 0; it < 27; ++it) {
+        const int cur_beg = beg, cur_end = end;
+        double4 pj = pj_next;
+        if (it + 1 < 27) {   // request the first chunk of the next cell
+            beg = __shfl_sync(0xffffffffu, cb, it + 1);
+            end = __shfl_sync(0xffffffffu, ce, it + 1);
+            if (beg + lane < end) pj_next = pos4[beg + lane];
+        }
+        for (int base = cur_beg; base < cur_end; base += 32) {
+            const int j = base + lane;
+            if (base != cur_beg && j < cur_end) pj = pos4[j];
+            bool hit = false;
+            if (j < cur_end && j != i) {
+                const double ex = __dsub_rn(pj.x, pi.x), ey = __dsub_rn(pj.y, pi.y), ez = __dsub_rn(pj.z, pi.z);
+                // fp32 screen: the squared distance to ~1e-6 relative decides every candidate that is not within
+                // 1e-5 of the list radius; only those few take the exact, individually rounded fp64 predicate
+                float fx = fabsf((float)ex), fy = fabsf((float)ey), fz = fabsf((float)ez);
+                fx = fx > halff[0] ? boxf[0] - fx : fx;
+                fy = fy > halff[1] ? boxf[1] - fy : fy;
+                fz = fz > halff[2] ? boxf[2] - fz : fz;
+                const float d2f = fx * fx + fy * fy + fz * fz;
+                if (d2f < rl2_lo) hit = true;
+                else if (d2f <= rl2_hi) {
+                    const double dx = min_image(ex, g.box[0], g.half[0]);
+                    const double dy = min_image(ey, g.box[1], g.half[1]);
+                    const double dz = min_image(ez, g.box[2], g.half[2]);
+                    const double d2 = __dadd_rn(__dadd_rn(__dmul_rn(dx, dx), __dmul_rn(dy, dy)), __dmul_rn(dz, dz));
+                    hit = d2 < rl2;
                 }
             }
+            const unsigned m = __ballot_sync(0xffffffffu, hit);
+            if (FILL && hit && writable) nbr[off + cnt + __popc(m & ((1u << lane) - 1u))] = j;
+            cnt += __popc(m);
+        }
+    }
     if (!FILL && lane == 0) nbr_count[i] = cnt;
 }
 
