@@ -193,6 +193,101 @@ __global__ void __launch_bounds__(256) k_neighbors(int64_t n, CellGrid g, double
     if (!FILL && lane == 0) nbr_count[i] = cnt;
 }
 
+// Positions relative to the lower corner of the atom's own cell, in fp32 (|x_rel| < cell edge, so the rounding is ~5e-7
+// Angstrom whatever the box size).  Lives in the force array, which is idle during a build.
+__global__ void k_rel_pos(int64_t n, CellGrid g, const double4 *__restrict__ pos4, float4 *__restrict__ rel) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const double4 p = pos4[i];
+    const double x[3] = {p.x, p.y, p.z};
+    float r[3];
+#pragma unroll
+    for (int a = 0; a < 3; ++a) {
+        const int c = cell_coord(x[a], g.inv_edge[a], g.n[a]);
+        r[a] = (float)(x[a] - (double)c * (g.box[a] / g.n[a]));
+    }
+    rel[i] = make_float4(r[0], r[1], r[2], 0.f);
+}
+
+// The same traversal for grids with at least three cells per dimension, on the cell-relative fp32 positions: the
+// separation is x_rel(j) - x_rel(i) + (cell offset) * edge -- the cell offset already names the periodic image, so no
+// minimum-image step and no fp64 arithmetic per candidate.  Candidates within 1e-5 of the list radius (the fp32 distance is
+// good to ~1e-6) are decided by the exact fp64 predicate on the full positions, so the lists are the same bit for bit.
+template <bool FILL>
+__global__ void __launch_bounds__(256) k_neighbors_rel(int64_t n, CellGrid g, double rl2, const double4 *__restrict__ pos4,
+                                                       const float4 *__restrict__ rel, const int32_t *__restrict__ cell_start,
+                                                       int32_t *__restrict__ nbr_count, const int64_t *__restrict__ nbr_off,
+                                                       int32_t *__restrict__ nbr, int64_t nbr_cap, int *status) {
+    const int lane = threadIdx.x & 31;
+    int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (i >= n) return;
+    const double4 pi = pos4[i];
+    const float4 ri = rel[i];
+    int cb = 0, ce = 0;
+    if (lane < 27) {
+        const int o[3] = {lane / 9, (lane / 3) % 3, lane % 3};
+        const double p[3] = {pi.x, pi.y, pi.z};
+        int cc[3];
+#pragma unroll
+        for (int a = 0; a < 3; ++a) {
+            const int na = g.n[a];
+            int c = cell_coord(p[a], g.inv_edge[a], na) + o[a] - 1;
+            cc[a] = c < 0 ? c + na : (c >= na ? c - na : c);
+        }
+        const int c = (cc[0] * g.n[1] + cc[1]) * g.n[2] + cc[2];
+        cb = cell_start[c]; ce = cell_start[c + 1];
+    }
+    const float edge[3] = {(float)(g.box[0] / g.n[0]), (float)(g.box[1] / g.n[1]), (float)(g.box[2] / g.n[2])};
+    const float rl2_lo = (float)(rl2 * (1.0 - 1e-5)), rl2_hi = (float)(rl2 * (1.0 + 1e-5));
+    int64_t off = 0;
+    bool writable = true;
+    if (FILL) {
+        off = nbr_off[i];
+        writable = nbr_off[i + 1] <= nbr_cap;
+        if (!writable && lane == 0) atomicOr(status, FLAG_NEIGHBOR_OVERFLOW);
+    }
+    int cnt = 0;
+    int beg = __shfl_sync(0xffffffffu, cb, 0), end = __shfl_sync(0xffffffffu, ce, 0);
+    float4 rj_next = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (beg + lane < end) rj_next = rel[beg + lane];
+#pragma unroll
+    for (int it = 0; it < 27; ++it) {
+        const int cur_beg = beg, cur_end = end;
+        float4 rj = rj_next;
+        if (it + 1 < 27) {   // request the first chunk of the next cell
+            beg = __shfl_sync(0xffffffffu, cb, it + 1);
+            end = __shfl_sync(0xffffffffu, ce, it + 1);
+            if (beg + lane < end) rj_next = rel[beg + lane];
+        }
+        // separation = x_rel(j) + shift, shift = (cell offset) * edge - x_rel(i)
+        const float sx = (float)(it / 9 - 1) * edge[0] - ri.x;
+        const float sy = (float)((it / 3) % 3 - 1) * edge[1] - ri.y;
+        const float sz = (float)(it % 3 - 1) * edge[2] - ri.z;
+        for (int base = cur_beg; base < cur_end; base += 32) {
+            const int j = base + lane;
+            if (base != cur_beg && j < cur_end) rj = rel[j];
+            bool hit = false;
+            if (j < cur_end && j != i) {
+                const float dx = rj.x + sx, dy = rj.y + sy, dz = rj.z + sz;
+                const float d2f = dx * dx + dy * dy + dz * dz;
+                if (d2f < rl2_lo) hit = true;
+                else if (d2f <= rl2_hi) {
+                    const double4 pj = pos4[j];
+                    const double ex = min_image(__dsub_rn(pj.x, pi.x), g.box[0], g.half[0]);
+                    const double ey = min_image(__dsub_rn(pj.y, pi.y), g.box[1], g.half[1]);
+                    const double ez = min_image(__dsub_rn(pj.z, pi.z), g.box[2], g.half[2]);
+                    const double d2 = __dadd_rn(__dadd_rn(__dmul_rn(ex, ex), __dmul_rn(ey, ey)), __dmul_rn(ez, ez));
+                    hit = d2 < rl2;
+                }
+            }
+            const unsigned m = __ballot_sync(0xffffffffu, hit);
+            if (FILL && hit && writable) nbr[off + cnt + __popc(m & ((1u << lane) - 1u))] = j;
+            cnt += __popc(m);
+        }
+    }
+    if (!FILL && lane == 0) nbr_count[i] = cnt;
+}
+
 // ---- canonical export: caller's indices, species-segmented, ascending ----
 __global__ void k_export_count(int64_t n, int n_species, const int64_t *__restrict__ nbr_off, const int32_t *__restrict__ nbr,
                                const double4 *__restrict__ pos4, const int32_t *__restrict__ user_of,
@@ -258,7 +353,15 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
     exclusive_scan<int32_t, int32_t>(c->bin_count, c->bin_start, (int64_t)C * g.n_cells, c->scan_tmp, s);
     int nthreads_co = g.n_cells > C + 1 ? g.n_cells : C + 1;
     k_center_order<<<blocks_for(nthreads_co, 128), 128, 0, s>>>(g.n_cells, C, c->cell_start, c->pos4, c->bin_start, c->center_order, c->species_start);
-    k_neighbors<false><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, c->cell_start, c->nbr_count, nullptr, nullptr, 0, c->status);
+    // grids of at least 3 x 3 x 3 cells take the fp32 cell-relative traversal (positions staged in the idle force array)
+    const bool rel = g.n[0] >= 3 && g.n[1] >= 3 && g.n[2] >= 3;
+    float4 *relpos = c->force;
+    if (rel) {
+        k_rel_pos<<<blocks_for(n, 256), 256, 0, s>>>(n, g, c->pos4, relpos);
+        k_neighbors_rel<false><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_count, nullptr, nullptr, 0, c->status);
+        c->launches += 1;
+    } else
+        k_neighbors<false><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, c->cell_start, c->nbr_count, nullptr, nullptr, 0, c->status);
     exclusive_scan<int32_t, int64_t>(c->nbr_count, c->nbr_off, n, c->scan_tmp, s);
     c->launches += 7 + 9;
     MLIP_CUDA_TRY(c, cudaGetLastError());
@@ -274,7 +377,10 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
             c->resident += sizeof(int32_t) * want;
         }
     }
-    k_neighbors<true><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, c->cell_start, c->nbr_count, c->nbr_off, c->nbr, c->nbr_cap, c->status);
+    if (rel)
+        k_neighbors_rel<true><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_count, c->nbr_off, c->nbr, c->nbr_cap, c->status);
+    else
+        k_neighbors<true><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, c->cell_start, c->nbr_count, c->nbr_off, c->nbr, c->nbr_cap, c->status);
     c->launches += 1;
     timing_end(c->ev_build, c->build_count, s);
     MLIP_CUDA_TRY(c, cudaGetLastError());
