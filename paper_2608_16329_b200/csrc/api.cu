@@ -50,6 +50,7 @@ static void free_atoms(mlip_ctx *c) {
     dev_free(c, &c->nbr_count, n); dev_free(c, &c->nbr_off, n + 1);
     if (c->cfg.precision == 1) { dev_free(c, &c->force_d, 3 * n); dev_free(c, &c->e_atom_d, n); }
     if (c->cfg.force_mode == 1) dev_free(c, &c->force_fx, 3 * n);
+    dev_free(c, &c->tile_state, n / 64 + 2);
     c->cap_atoms = 0;
 }
 
@@ -74,6 +75,7 @@ static int ensure_capacity(mlip_ctx *c, int64_t n, int64_t n_cells) {
         TRY_ALLOC(c->nbr_count, m); TRY_ALLOC(c->nbr_off, m + 1);
         if (c->cfg.precision == 1) { TRY_ALLOC(c->force_d, 3 * m); TRY_ALLOC(c->e_atom_d, m); }
         if (c->cfg.force_mode == 1) TRY_ALLOC(c->force_fx, 3 * m);
+        TRY_ALLOC(c->tile_state, m / 64 + 2);
         c->cap_atoms = n;
     }
     if (n_cells > c->cap_cells) {
@@ -194,6 +196,7 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
         if ((rc = dev_alloc(c, &c->rebuild_flag, 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->nhc, 8)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->acc_fx, 10)) != MLIP_OK) break;
+        if ((rc = dev_alloc(c, &c->tile_ticket, 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->tile_counter, (size_t)MAX_SPECIES)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->species_start, (size_t)MAX_SPECIES + 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->stage_out, 10)) != MLIP_OK) break;
@@ -571,7 +574,7 @@ void mlip_destroy(mlip_ctx *c) {
     free_cells(c);
     cudaFree(c->nbr); cudaFree(c->scan_tmp); cudaFree(c->head_w); cudaFree(c->table); cudaFree(c->mass);
     cudaFree(c->head_w_d); cudaFree(c->table_d);
-    cudaFree(c->acc); cudaFree(c->pair_counter); cudaFree(c->status); cudaFree(c->rebuild_flag); cudaFree(c->nhc); cudaFree(c->acc_fx); cudaFree(c->tile_counter);
+    cudaFree(c->acc); cudaFree(c->pair_counter); cudaFree(c->status); cudaFree(c->rebuild_flag); cudaFree(c->nhc); cudaFree(c->acc_fx); cudaFree(c->tile_ticket); cudaFree(c->tile_counter);
     cudaFree(c->species_start); cudaFree(c->stage_pos); cudaFree(c->stage_species); cudaFree(c->stage_force);
     cudaFree(c->stage_out);
     if (c->status_host) cudaFreeHost(c->status_host);

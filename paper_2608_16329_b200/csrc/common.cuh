@@ -99,6 +99,8 @@ struct mlip_ctx {
     int32_t *nbr_count = nullptr;  // [N]
     int64_t *nbr_off = nullptr;    // [N + 1]
     int32_t *nbr = nullptr;
+    unsigned long long *tile_state = nullptr;   // [ceil(N / 64) + 1] look-back words of the one-pass rebuild
+    int *tile_ticket = nullptr;
     int64_t nbr_cap = 0, n_entries = 0;
     // scratch
     int64_t *scan_tmp = nullptr;   // block sums for the scans

@@ -288,6 +288,198 @@ __global__ void __launch_bounds__(256) k_neighbors_rel(int64_t n, CellGrid g, do
     if (!FILL && lane == 0) nbr_count[i] = cnt;
 }
 
+// ---- one-pass variant for in-step rebuilds ----
+// Count and fill in a single traversal: a CTA takes a tile of 64 consecutive atoms (8 per warp), keeps the hit masks of
+// every 32-candidate chunk in shared memory while it counts, obtains the tile's list offset from a decoupled look-back
+// scan over the tiles before it (tile aggregate / inclusive prefix published in one 64-bit word, tiles handed out by a
+// ticket so that every predecessor belongs to a CTA that is already running), and then replays the masks to write the
+// lists.  Offsets are the same exclusive prefix sums the two-pass build produces, so the lists are identical.
+// Every wait is bounded: after OP_SPIN polls the tile raises FLAG_NEIGHBOR_OVERFLOW, publishes what it has and goes on.
+constexpr int OP_PER_WARP = 8;
+constexpr int OP_TILE = 8 * OP_PER_WARP;
+static_assert(OP_TILE == 64, "the in-tile scan handles two counts per lane of one warp");
+constexpr int OP_MAXCH = 64;                     // chunk masks kept per atom; chunks beyond are re-tested in the replay
+constexpr int OP_SPIN = 1 << 18;
+
+__device__ __forceinline__ bool rel_hit(const float4 &rj, float sx, float sy, float sz, float rl2_lo, float rl2_hi, double rl2,
+                                        const double4 &pi, const double4 *__restrict__ pos4, int j, const CellGrid &g) {
+    const float dx = rj.x + sx, dy = rj.y + sy, dz = rj.z + sz;
+    const float d2f = dx * dx + dy * dy + dz * dz;
+    if (d2f < rl2_lo) return true;
+    if (d2f > rl2_hi) return false;
+    const double4 pj = pos4[j];
+    const double ex = min_image(__dsub_rn(pj.x, pi.x), g.box[0], g.half[0]);
+    const double ey = min_image(__dsub_rn(pj.y, pi.y), g.box[1], g.half[1]);
+    const double ez = min_image(__dsub_rn(pj.z, pi.z), g.box[2], g.half[2]);
+    return __dadd_rn(__dadd_rn(__dmul_rn(ex, ex), __dmul_rn(ey, ey)), __dmul_rn(ez, ez)) < rl2;
+}
+
+// atom ranges of the 27 cells around position p, one cell per lane (lanes 27.. get an empty range)
+__device__ __forceinline__ void cell_ranges(const double4 &p4, const CellGrid &g, const int32_t *__restrict__ cell_start, int lane,
+                                            int &cb, int &ce) {
+    cb = 0; ce = 0;
+    if (lane < 27) {
+        const int o[3] = {lane / 9, (lane / 3) % 3, lane % 3};
+        const double p[3] = {p4.x, p4.y, p4.z};
+        int cc[3];
+#pragma unroll
+        for (int a = 0; a < 3; ++a) {
+            const int na = g.n[a];
+            int c = cell_coord(p[a], g.inv_edge[a], na) + o[a] - 1;
+            cc[a] = c < 0 ? c + na : (c >= na ? c - na : c);
+        }
+        const int c = (cc[0] * g.n[1] + cc[1]) * g.n[2] + cc[2];
+        cb = cell_start[c]; ce = cell_start[c + 1];
+    }
+}
+
+__global__ void __launch_bounds__(256) k_neighbors_onepass(int64_t n, CellGrid g, double rl2, const double4 *__restrict__ pos4,
+                                                           const float4 *__restrict__ rel, const int32_t *__restrict__ cell_start,
+                                                           int64_t *__restrict__ nbr_off, int32_t *__restrict__ nbr, int64_t nbr_cap,
+                                                           int *status, unsigned long long *tile_state, int *ticket) {
+    // look-back word: flag in the top two bits (0 empty, 1 tile aggregate, 2 inclusive prefix), value below
+    constexpr unsigned long long OP_AGG = 1ull << 62, OP_INC = 2ull << 62, OP_VAL = (1ull << 62) - 1;
+    __shared__ unsigned s_mask[OP_TILE][OP_MAXCH];
+    __shared__ int s_cnt[OP_TILE];
+    __shared__ long long s_off[OP_TILE];
+    __shared__ long long s_prefix, s_total;
+    __shared__ int s_tile;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) s_tile = atomicAdd(ticket, 1);
+    __syncthreads();
+    const int64_t tile = s_tile, first = tile * OP_TILE;
+    const float edge[3] = {(float)(g.box[0] / g.n[0]), (float)(g.box[1] / g.n[1]), (float)(g.box[2] / g.n[2])};
+    const float rl2_lo = (float)(rl2 * (1.0 - 1e-5)), rl2_hi = (float)(rl2 * (1.0 + 1e-5));
+
+    // ---- traversal: count, keep the masks ----
+    for (int a = 0; a < OP_PER_WARP; ++a) {
+        const int slot = warp * OP_PER_WARP + a;
+        const int64_t i = first + slot;
+        int cnt = 0;
+        if (i < n) {
+            const double4 pi = pos4[i];
+            const float4 ri = rel[i];
+            int cb, ce;
+            cell_ranges(pi, g, cell_start, lane, cb, ce);
+            int ch = 0;
+            int beg = __shfl_sync(0xffffffffu, cb, 0), end = __shfl_sync(0xffffffffu, ce, 0);
+            float4 rj_next = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (beg + lane < end) rj_next = rel[beg + lane];
+#pragma unroll
+            for (int it = 0; it < 27; ++it) {
+                const int cur_beg = beg, cur_end = end;
+                float4 rj = rj_next;
+                if (it + 1 < 27) {
+                    beg = __shfl_sync(0xffffffffu, cb, it + 1);
+                    end = __shfl_sync(0xffffffffu, ce, it + 1);
+                    if (beg + lane < end) rj_next = rel[beg + lane];
+                }
+                const float sx = (float)(it / 9 - 1) * edge[0] - ri.x;
+                const float sy = (float)((it / 3) % 3 - 1) * edge[1] - ri.y;
+                const float sz = (float)(it % 3 - 1) * edge[2] - ri.z;
+                for (int base = cur_beg; base < cur_end; base += 32) {
+                    const int j = base + lane;
+                    if (base != cur_beg && j < cur_end) rj = rel[j];
+                    const bool hit = j < cur_end && j != i && rel_hit(rj, sx, sy, sz, rl2_lo, rl2_hi, rl2, pi, pos4, j, g);
+                    const unsigned m = __ballot_sync(0xffffffffu, hit);
+                    if (ch < OP_MAXCH && lane == 0) s_mask[slot][ch] = m;
+                    ++ch;
+                    cnt += __popc(m);
+                }
+            }
+        }
+        if (lane == 0) s_cnt[slot] = cnt;
+    }
+    __syncthreads();
+
+    // ---- offsets: scan inside the tile, look back over the tiles before it ----
+    if (warp == 0) {
+        const int c0 = s_cnt[2 * lane], c1 = s_cnt[2 * lane + 1];
+        long long incl = c0 + c1;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const long long v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        s_off[2 * lane] = incl - c0 - c1;
+        s_off[2 * lane + 1] = incl - c1;
+        const long long aggregate = __shfl_sync(0xffffffffu, incl, 31);
+        volatile unsigned long long *state = tile_state;
+        long long prefix = 0;
+        if (tile > 0) {
+            if (lane == 0) state[tile] = OP_AGG | (unsigned long long)aggregate;
+            int64_t hi = tile - 1;
+            int spins = 0;
+            for (;;) {   // windows of 32 predecessors, nearest first
+                const int64_t p = hi - lane;
+                unsigned long long v = OP_INC;
+                if (p >= 0) v = state[p];
+                const unsigned flag = (unsigned)(v >> 62);
+                const unsigned inc = __ballot_sync(0xffffffffu, flag == 2), empty = __ballot_sync(0xffffffffu, flag == 0);
+                const int first_inc = inc ? __ffs(inc) - 1 : 32;
+                const unsigned need = first_inc >= 31 ? 0xffffffffu : ((2u << first_inc) - 1u);
+                if (empty & need) {   // a tile in the window has not published yet
+                    if (++spins > OP_SPIN) { if (lane == 0) atomicOr(status, FLAG_NEIGHBOR_OVERFLOW); break; }
+                    __nanosleep(200);
+                    continue;
+                }
+                long long val = (lane <= first_inc && p >= 0) ? (long long)(v & OP_VAL) : 0;
+#pragma unroll
+                for (int o = 16; o; o >>= 1) val += __shfl_xor_sync(0xffffffffu, val, o);
+                prefix += val;
+                if (first_inc < 32) break;
+                hi -= 32;
+            }
+        }
+        if (lane == 0) {
+            state[tile] = OP_INC | (unsigned long long)(prefix + aggregate);
+            s_prefix = prefix;
+            s_total = prefix + aggregate;
+        }
+    }
+    __syncthreads();
+    const long long tile_off = s_prefix;
+    if (first + OP_TILE >= n && threadIdx.x == 0) nbr_off[n] = s_total;   // the last tile closes the offsets
+
+    // ---- replay: write the lists from the masks ----
+    for (int a = 0; a < OP_PER_WARP; ++a) {
+        const int slot = warp * OP_PER_WARP + a;
+        const int64_t i = first + slot;
+        if (i >= n) break;
+        const long long off = tile_off + s_off[slot];
+        if (lane == 0) nbr_off[i] = off;
+        if (off + s_cnt[slot] > nbr_cap) {
+            if (lane == 0) atomicOr(status, FLAG_NEIGHBOR_OVERFLOW);
+            continue;
+        }
+        const double4 pi = pos4[i];
+        const float4 ri = rel[i];
+        int cb, ce;
+        cell_ranges(pi, g, cell_start, lane, cb, ce);
+        int ch = 0, run = 0;
+        for (int it = 0; it < 27; ++it) {
+            const int cur_beg = __shfl_sync(0xffffffffu, cb, it), cur_end = __shfl_sync(0xffffffffu, ce, it);
+            for (int base = cur_beg; base < cur_end; base += 32) {
+                const int j = base + lane;
+                unsigned m;
+                if (ch < OP_MAXCH) m = s_mask[slot][ch];
+                else {   // beyond the kept masks: test again
+                    const float sx = (float)(it / 9 - 1) * edge[0] - ri.x;
+                    const float sy = (float)((it / 3) % 3 - 1) * edge[1] - ri.y;
+                    const float sz = (float)(it % 3 - 1) * edge[2] - ri.z;
+                    float4 rj = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (j < cur_end) rj = rel[j];
+                    const bool hit = j < cur_end && j != i && rel_hit(rj, sx, sy, sz, rl2_lo, rl2_hi, rl2, pi, pos4, j, g);
+                    m = __ballot_sync(0xffffffffu, hit);
+                }
+                if ((m >> lane) & 1u) nbr[off + run + __popc(m & ((1u << lane) - 1u))] = j;
+                run += __popc(m);
+                ++ch;
+            }
+        }
+    }
+}
+
 // ---- canonical export: caller's indices, species-segmented, ascending ----
 __global__ void k_export_count(int64_t n, int n_species, const int64_t *__restrict__ nbr_off, const int32_t *__restrict__ nbr,
                                const double4 *__restrict__ pos4, const int32_t *__restrict__ user_of,
@@ -356,6 +548,18 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
     // grids of at least 3 x 3 x 3 cells take the fp32 cell-relative traversal (positions staged in the idle force array)
     const bool rel = g.n[0] >= 3 && g.n[1] >= 3 && g.n[2] >= 3;
     float4 *relpos = c->force;
+    if (rel && !allow_sync_grow && c->tile_state) {   // in-step rebuild: single traversal, capacity as it stands
+        const int64_t n_tiles = (n + OP_TILE - 1) / OP_TILE;
+        MLIP_CUDA_TRY(c, cudaMemsetAsync(c->tile_state, 0, sizeof(unsigned long long) * (n_tiles + 1), s));
+        MLIP_CUDA_TRY(c, cudaMemsetAsync(c->tile_ticket, 0, sizeof(int), s));
+        k_rel_pos<<<blocks_for(n, 256), 256, 0, s>>>(n, g, c->pos4, relpos);
+        k_neighbors_onepass<<<(unsigned)n_tiles, 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_off, c->nbr, c->nbr_cap,
+                                                               c->status, c->tile_state, c->tile_ticket);
+        c->launches += 7 + 6 + 2;
+        timing_end(c->ev_build, c->build_count, s);
+        MLIP_CUDA_TRY(c, cudaGetLastError());
+        return MLIP_OK;
+    }
     if (rel) {
         k_rel_pos<<<blocks_for(n, 256), 256, 0, s>>>(n, g, c->pos4, relpos);
         k_neighbors_rel<false><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_count, nullptr, nullptr, 0, c->status);
