@@ -365,7 +365,7 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
 
 // ---------------- Derivation of one atom (Eq. 8-10) ----------------
 template <bool DET>
-__device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView &tv, const double4 &pi, int i, int64_t beg, int64_t end,
+__device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView &tv, int i,
                                             float4 *pq, float *scr, int queued, int lane, const uint32_t (&Wh)[4][4],
                                             const uint32_t (&Wl)[4][4], float (&vir)[9], PhaseClock &pc) {
     const int g = lane >> 2, t = lane & 3;
@@ -508,7 +508,10 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
     };
     if (queued >= 0) {   // the encoding left every pair of this atom in the queue
         for (int q0 = 0; q0 < queued; q0 += 32) batch(q0, min(32, queued - q0));
-    } else {
+    } else {   // rare: the list did not fit the queue; position and list bounds are fetched again rather than kept
+               // in registers through the head
+        const double4 pi = load_pos4(k.pos4 + i);
+        const int64_t beg = k.nbr_off[i], end = k.nbr_off[i + 1];
         int64_t cur = beg;
         do {
             const int n = collect_pairs(k, pi, beg, cur, end, pq, lane, nullptr, 0);
@@ -880,7 +883,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
                     split_tf32(w2, Wh[ks][2], Wl[ks][2]);
                     split_tf32(w3, Wh[ks][3], Wl[ks][3]);
                 }
-                derive_atom<DET>(k, tv, pi, i, beg, end, pq, scr, queued, lane, Wh, Wl, vir, pc);
+                derive_atom<DET>(k, tv, i, pq, scr, queued, lane, Wh, Wl, vir, pc);
                 if (DET) {   // fold this atom's virial in now: lane sums in a fixed order, then integers
 #pragma unroll
                     for (int q = 0; q < 9; ++q) {
