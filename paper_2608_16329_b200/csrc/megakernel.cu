@@ -257,7 +257,7 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
             int off = 0;
             if (lane < n) {
                 const float4 e = pq[first + lane];
-                const float r = sqrtf(e.x * e.x + e.y * e.y + e.z * e.z), rinv = 1.0f / r;
+                const float d2 = e.x * e.x + e.y * e.y + e.z * e.z, rinv = rsqrtf(d2), r = d2 * rinv;
                 harmonics(e.x * rinv, e.y * rinv, e.z * rinv, h);
                 const int iv = spline_basis<false, float>(r, k.tab.r_min, k.tab.inv_h, k.tab.knots, b, nullptr, k.status);
                 const int sj = __float_as_int(e.w) >> J_BITS;
@@ -281,6 +281,7 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
         __syncwarp();
         pc.mark(1);
         const int nks = (n + 7) >> 3;
+#pragma unroll 2
         for (int ks = 0; ks < nks; ++ks) {
             // A = H^T (16 x 8 pairs): rows a = g, g + 8; columns pairs t, t + 4 of this k-step
             const float *ra = stage + (8 * ks + t) * ST_STRIDE, *rb = ra + 4 * ST_STRIDE;
@@ -381,7 +382,7 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
             const bool live = lane < n;
             if (live) {
                 ent = pq[first + lane];
-                const float r = sqrtf(ent.x * ent.x + ent.y * ent.y + ent.z * ent.z);
+                const float d2 = ent.x * ent.x + ent.y * ent.y + ent.z * ent.z, r = d2 * rsqrtf(d2);
                 const int iv = spline_basis<true, float>(r, k.tab.r_min, k.tab.inv_h, k.tab.knots, b, db, k.status);
                 row_index = (__float_as_int(ent.w) >> J_BITS) * (k.tab.knots + 3) + iv;
                 off = row_index * rs;
@@ -487,7 +488,7 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
             }
             const float4 ent = src[8 ^ sw];
             const float x = ent.x, y = ent.y, z = ent.z;
-            const float rinv = 1.0f / sqrtf(x * x + y * y + z * z);
+            const float rinv = rsqrtf(x * x + y * y + z * z);
             const int j = __float_as_int(ent.w) & ((1 << J_BITS) - 1);
             const float ux = x * rinv, uy = y * rinv, uz = z * rinv;
             float s, tx, ty, tz, tu;
