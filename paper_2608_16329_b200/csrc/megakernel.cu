@@ -785,16 +785,15 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
 
         bool prefetched = false;   // this warp's atom of the coming tile sits in the prefetch buffer
         int look_ahead = -1;       // (group leader) the tile after the current one
-        while (true) {   // the group's tiles of this species, claimed one ahead
-            group_sync(group);
-            if (wg == 0 && lane == 0) {
-                ctl[2 * group] = look_ahead >= 0 ? look_ahead : atomicAdd(k.tile_counter + species, 1);
-                look_ahead = atomicAdd(k.tile_counter + species, 1);   // consumed after the encoding: its latency is hidden
-            }
-            group_sync(group);
+        // the group's tiles of this species, claimed one ahead: the first is broadcast here, every later one travels with
+        // the barrier between encoding and head
+        group_sync(group);
+        if (wg == 0 && lane == 0) ctl[2 * group] = atomicAdd(k.tile_counter + species, 1);
+        group_sync(group);
+        int tile = ctl[2 * group];
+        while (tile < n_tiles) {
+            if (wg == 0 && lane == 0) look_ahead = atomicAdd(k.tile_counter + species, 1);   // consumed after the encoding
             pc.mark(11);
-            const int tile = ctl[2 * group];
-            if (tile >= n_tiles) break;
             const int first = s_beg + tile * TILE;
             const int count = min(TILE, s_end - first);
 
@@ -897,6 +896,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
                 }
             }
             pc.mark(10);
+            tile = tile_next;
         }
     }
     pc.flush(k.acc, lane);
