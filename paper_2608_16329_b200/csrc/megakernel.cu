@@ -832,7 +832,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
 #pragma unroll
                 for (int o = 4; o < 32; o <<= 1)
 #pragma unroll
-                    for (int l = 0; l < 4; ++l)
+                    for (int l = 1; l < 4; ++l)   // l = 0 is a single row: the lane that stores it (g == 0) already holds it
 #pragma unroll
                         for (int j = 0; j < 8; ++j) part[l][j] += __shfl_xor_sync(0xffffffffu, part[l][j], o);
                 if (g == 0) {
