@@ -550,38 +550,42 @@ __device__ __forceinline__ void head_load(float4 (&w)[8], const float4 *__restri
 // otherwise one accumulation chain (reverse pass: feeds forces only).
 template <int NKS, bool FRESH>
 __device__ __forceinline__ void head_gemm(float (&c)[4], const float4 (&w)[8], int ks0, const float *__restrict__ act, int bstride, int lane) {
-    static_assert(NKS % 2 == 0, "k-steps are processed two at a time (two independent MMA chains in flight)");
+    static_assert(NKS % 4 == 0, "k-steps are processed four at a time (four independent MMA chains in flight)");
     const int g = lane >> 2, t = lane & 3;
-    float ce[4], co[4];   // FRESH: per-k-step products; otherwise the even / odd accumulation chains
+    float acc[4][4];   // FRESH: per-k-step products; otherwise four accumulation chains
 #pragma unroll
-    for (int q = 0; q < NKS; q += 2) {
-        uint32_t ah[2][4], al[2][4];
-        float2 x0[2], x1[2];
+    for (int q = 0; q < NKS; q += 4) {
+        uint32_t ah[4][4], al[4][4];
+        float2 x0[4], x1[4];
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
+        for (int u = 0; u < 4; ++u) {
             split_tf32(w[q + u].x, ah[u][0], al[u][0]); split_tf32(w[q + u].y, ah[u][1], al[u][1]);
             split_tf32(w[q + u].z, ah[u][2], al[u][2]); split_tf32(w[q + u].w, ah[u][3], al[u][3]);
             const float *r0 = act + g * bstride + 2 * (8 * (ks0 + q + u) + t);
             x0[u] = *reinterpret_cast<const float2 *>(r0);
             x1[u] = *reinterpret_cast<const float2 *>(r0 + 8);
         }
-        if (FRESH || q == 0) {
-            mma_tf32_z(ce, al[0][0], al[0][1], al[0][2], al[0][3], __float_as_uint(x0[0].x), __float_as_uint(x1[0].x));
-            mma_tf32_z(co, al[1][0], al[1][1], al[1][2], al[1][3], __float_as_uint(x0[1].x), __float_as_uint(x1[1].x));
-        } else {
-            mma_tf32(ce, al[0][0], al[0][1], al[0][2], al[0][3], __float_as_uint(x0[0].x), __float_as_uint(x1[0].x));
-            mma_tf32(co, al[1][0], al[1][1], al[1][2], al[1][3], __float_as_uint(x0[1].x), __float_as_uint(x1[1].x));
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (FRESH || q == 0) mma_tf32_z(acc[u], al[u][0], al[u][1], al[u][2], al[u][3], __float_as_uint(x0[u].x), __float_as_uint(x1[u].x));
+            else mma_tf32(acc[u], al[u][0], al[u][1], al[u][2], al[u][3], __float_as_uint(x0[u].x), __float_as_uint(x1[u].x));
         }
-        mma_tf32(ce, ah[0][0], ah[0][1], ah[0][2], ah[0][3], __float_as_uint(x0[0].y), __float_as_uint(x1[0].y));
-        mma_tf32(co, ah[1][0], ah[1][1], ah[1][2], ah[1][3], __float_as_uint(x0[1].y), __float_as_uint(x1[1].y));
-        mma_tf32(ce, ah[0][0], ah[0][1], ah[0][2], ah[0][3], __float_as_uint(x0[0].x), __float_as_uint(x1[0].x));
-        mma_tf32(co, ah[1][0], ah[1][1], ah[1][2], ah[1][3], __float_as_uint(x0[1].x), __float_as_uint(x1[1].x));
+#pragma unroll
+        for (int u = 0; u < 4; ++u) mma_tf32(acc[u], ah[u][0], ah[u][1], ah[u][2], ah[u][3], __float_as_uint(x0[u].y), __float_as_uint(x1[u].y));
+#pragma unroll
+        for (int u = 0; u < 4; ++u) mma_tf32(acc[u], ah[u][0], ah[u][1], ah[u][2], ah[u][3], __float_as_uint(x0[u].x), __float_as_uint(x1[u].x));
         if (FRESH) {
-            if (q == 0) { c[0] = ce[0] + co[0]; c[1] = ce[1] + co[1]; c[2] = ce[2] + co[2]; c[3] = ce[3] + co[3]; }
-            else { c[0] += ce[0] + co[0]; c[1] += ce[1] + co[1]; c[2] += ce[2] + co[2]; c[3] += ce[3] + co[3]; }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float s4 = (acc[0][e] + acc[1][e]) + (acc[2][e] + acc[3][e]);
+                c[e] = q == 0 ? s4 : c[e] + s4;
+            }
         }
     }
-    if (!FRESH) { c[0] = ce[0] + co[0]; c[1] = ce[1] + co[1]; c[2] = ce[2] + co[2]; c[3] = ce[3] + co[3]; }
+    if (!FRESH) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) c[e] = (acc[0][e] + acc[1][e]) + (acc[2][e] + acc[3][e]);
+    }
 }
 
 // c fragment (rows = 16 m + g, g + 8; columns = atoms 2t, 2t + 1) -> part[atom][row] with `pstride` floats per atom
