@@ -555,7 +555,7 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
         k_rel_pos<<<blocks_for(n, 256), 256, 0, s>>>(n, g, c->pos4, relpos);
         k_neighbors_onepass<<<(unsigned)n_tiles, 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_off, c->nbr, c->nbr_cap,
                                                                c->status, c->tile_state, c->tile_ticket);
-        c->launches += 7 + 6 + 2;
+        c->launches += 5 + 2 * 3 + 2;   // cell id, place, sort, gather, centre order; two scans; relative positions, lists
         timing_end(c->ev_build, c->build_count, s);
         MLIP_CUDA_TRY(c, cudaGetLastError());
         return MLIP_OK;
@@ -567,7 +567,7 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
     } else
         k_neighbors<false><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, c->cell_start, c->nbr_count, nullptr, nullptr, 0, c->status);
     exclusive_scan<int32_t, int64_t>(c->nbr_count, c->nbr_off, n, c->scan_tmp, s);
-    c->launches += 7 + 9;
+    c->launches += 5 + 1 + 3 * 3;   // cell id, place, sort, gather, centre order; count; three scans
     MLIP_CUDA_TRY(c, cudaGetLastError());
     if (allow_sync_grow) {
         MLIP_CUDA_TRY(c, cudaMemcpyAsync(c->total_host, c->nbr_off + n, sizeof(int64_t), cudaMemcpyDeviceToHost, s));
