@@ -387,15 +387,7 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
                 row_index = (__float_as_int(ent.w) >> J_BITS) * (k.tab.knots + 3) + iv;
                 off = row_index * rs;
             }
-            // Slot of this pair in the batch: pairs whose table rows have even index go to even slots, odd
-            // to odd (as far as the counts allow).  Neighboring fragment rows then read table rows of
-            // opposite parity, which the padded row stride maps to disjoint shared-memory banks.
-            const unsigned lt = (1u << lane) - 1u;
-            const unsigned ev = __ballot_sync(0xffffffffu, live && !(row_index & 1)), od = __ballot_sync(0xffffffffu, live && (row_index & 1));
-            const int ne = __popc(ev), no = __popc(od), ecap = (n + 1) >> 1, ocap = n >> 1;
-            const int re = __popc(ev & lt), ro = __popc(od & lt);
-            int slot = lane;
-            if (live) slot = (row_index & 1) ? (ro < ocap ? 2 * ro + 1 : 2 * (ne + ro - ocap)) : (re < ecap ? 2 * re : 2 * (no + re - ecap) + 1);
+            const int slot = lane;
             float4 *row = reinterpret_cast<float4 *>(bs + slot * BS_STRIDE);
             row[0] = make_float4(b[0], b[1], b[2], b[3]);
             row[1] = make_float4(db[0], db[1], db[2], db[3]);
