@@ -589,7 +589,8 @@ __device__ __forceinline__ void store_partial(const float (&c)[4], float *part, 
 
 // Prefetch of the warp's atom in the group's NEXT tile, spread over three points of the head so
 // that each dependent global load has a barrier's worth of time to arrive: centre index -> list
-// bounds -> the first PF_IDX neighbor indices (cp.async straight into shared memory).
+// bounds -> the first PF_IDX neighbor indices (cp.async straight into shared memory).  (Pulling the
+// neighbors' positions into L2 as a fourth step cost more issue slots than it saved latency.)
 struct NextAtom {
     const KernelArgs *k;
     int *meta;        // shared: {atom, list start lo, list start hi, list length}
@@ -612,19 +613,6 @@ struct NextAtom {
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
         if (lane == 0) { meta[0] = i; meta[1] = (int)(beg & 0xffffffff); meta[2] = (int)(beg >> 32); meta[3] = (int)(end - beg); }
-    }
-    // once the indices have landed: pull the neighbors' positions (and the atom's own) into L2
-    __device__ __forceinline__ void stage_d(int lane) {
-        if (slot < 0) return;
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
-        __syncwarp();
-        const int n = (int)min((int64_t)PF_IDX, end - beg);
-#pragma unroll
-        for (int c = 0; c < PF_IDX / 32; ++c) {
-            const int e = 32 * c + lane;
-            if (e < n) asm volatile("prefetch.global.L2 [%0];" ::"l"(k->pos4 + sidx[e]));
-        }
-        if (lane == 0) asm volatile("prefetch.global.L2 [%0];" ::"l"(k->pos4 + i));
     }
 };
 
@@ -665,7 +653,6 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
         else head_load<4>(w, bwd + (size_t)((N_INV / 16) * 8 + (HEAD_L - 2) * 32 + mt4 * 8) * 32, kh * 4, lane);
         if (L == 0) nx.stage_b();
         if (L == 1) nx.stage_c(lane);
-        if (L == 3) nx.stage_d(lane);
         pc.mark(13);
         group_sync(group);
         pc.mark(14);
