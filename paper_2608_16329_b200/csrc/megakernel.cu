@@ -624,7 +624,7 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
                                           int group, int wg, int lane, double &e_sum, NextAtom &nx, PhaseClock &pc) {
     const float *hp = k.head_pack + (size_t)species * HP_TOTAL;
     const float4 *fwd = reinterpret_cast<const float4 *>(hp + HP_FWD), *bwd = reinterpret_cast<const float4 *>(hp + HP_BWD);
-    float *xs = hb + HB_XS, *zs = hb + HB_ZS, *sD = hb + HB_SD, *dp = hb + HB_DP, *part = hb + HB_PART;
+    float *xs = hb + HB_XS, *zs = hb + HB_ZS, *dp = hb + HB_DP, *part = hb + HB_PART;
     const int mt4 = wg & 3, kh = wg >> 2;   // forward / reverse hidden layers: 4 m-tiles x 2 k-halves
     const int atom = wg;                    // elementwise phases: warp = atom, lane = neuron (and neuron + 32)
     float4 w[8];
@@ -641,6 +641,7 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
     float e_i = 0.f;
     float ya = 0.f, yb = 0.f;   // running activations of this thread's two neurons (the skip path)
     float2 dzn = make_float2(0.f, 0.f);   // dE/dy of the same two neurons in the reverse pass
+    float2 sdr[HEAD_L];                    // SiLU' of their pre-activations, layer by layer
 #pragma unroll
     for (int L = 0; L < HEAD_L; ++L) {
         const float *zin = zs + ((L + 1) & 1) * TILE * 2 * Z_STRIDE;
@@ -668,7 +669,7 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
             ya += silu_f((p0.x + p1.x) + bb.x, d0);
             yb += silu_f((p0.y + p1.y) + bb.y, d1);
             const float y0 = ya, y1 = yb;
-            *reinterpret_cast<float2 *>(sD + (L * TILE + atom) * Z_STRIDE + n0) = make_float2(d0, d1);
+            sdr[L] = make_float2(d0, d1);
             if (L < HEAD_L - 1) {
                 const float2 s0 = split_pair(y0), s1 = split_pair(y1);
                 *reinterpret_cast<float4 *>(zout + atom * 2 * Z_STRIDE + 2 * n0) = make_float4(s0.x, s0.y, s1.x, s1.y);
@@ -706,7 +707,7 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
             const float2 p0 = *reinterpret_cast<const float2 *>(part + atom * Z_STRIDE + n0);
             const float2 p1 = *reinterpret_cast<const float2 *>(part + (TILE + atom) * Z_STRIDE + n0);
             dzn.x += p0.x + p1.x; dzn.y += p0.y + p1.y;
-            const float2 da = *reinterpret_cast<const float2 *>(sD + ((L - 1) * TILE + atom) * Z_STRIDE + n0);
+            const float2 da = sdr[L - 1];
             const float2 s0 = split_pair(dzn.x * da.x), s1 = split_pair(dzn.y * da.y);
             *reinterpret_cast<float4 *>(dp + atom * 2 * Z_STRIDE + 2 * n0) = make_float4(s0.x, s0.y, s1.x, s1.y);
         }
