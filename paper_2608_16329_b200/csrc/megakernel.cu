@@ -56,9 +56,7 @@ constexpr int SX_WORDS = TILE * X_STRIDE;                       // per group
 // head buffers of a group (alias of the scratch of the group's warps)
 constexpr int HB_XS = 0;                                   // split invariants  [8][2 * X_STRIDE]
 constexpr int HB_ZS = HB_XS + TILE * 2 * X_STRIDE;         // split activations [2][8][2 * Z_STRIDE]
-constexpr int HB_SD = HB_ZS + 2 * TILE * 2 * Z_STRIDE;     // SiLU'             [4][8][Z_STRIDE]
-constexpr int HB_DZ = HB_SD + HEAD_L * TILE * Z_STRIDE;    // dE/dz             [8][Z_STRIDE]
-constexpr int HB_DP = HB_DZ + TILE * Z_STRIDE;             // split dE/dpre     [8][2 * Z_STRIDE]
+constexpr int HB_DP = HB_ZS + 2 * TILE * 2 * Z_STRIDE;     // split dE/dpre     [8][2 * Z_STRIDE]
 constexpr int HB_PART = HB_DP + TILE * 2 * Z_STRIDE;       // split-K partials  [2][8][Z_STRIDE]
 constexpr int HB_WORDS = HB_PART + 2 * TILE * Z_STRIDE;
 static_assert(HB_WORDS <= TILE * SCR_WORDS, "head buffers alias the scratch of the group's warps");
