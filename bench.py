@@ -48,7 +48,7 @@ FP64_LANES_PER_SM = 64         # fp64 path: DFMA lanes per SM
 # DRAM traffic of one fused-kernel launch from the committed ncu capture
 # (profiles/k_mega_hea6_fcc50.md: dram__bytes_read.sum + dram__bytes_write.sum of a 500,000-atom launch, per atom;
 # the traffic is per-atom, so a launch of N atoms is reported as this figure times N).
-NCU_DRAM_BYTES_PER_ATOM = 751.0
+NCU_DRAM_BYTES_PER_ATOM = 746.0
 
 
 def parse_args():
