@@ -289,16 +289,14 @@ __global__ void __launch_bounds__(256) k_neighbors_rel(int64_t n, CellGrid g, do
 }
 
 // ---- one-pass variant for in-step rebuilds ----
-// Count and fill in a single traversal: a CTA takes a tile of 64 consecutive atoms (8 per warp), keeps the hit masks of
-// every 32-candidate chunk in shared memory while it counts, obtains the tile's list offset from a decoupled look-back
-// scan over the tiles before it (tile aggregate / inclusive prefix published in one 64-bit word, tiles handed out by a
-// ticket so that every predecessor belongs to a CTA that is already running), and then replays the masks to write the
-// lists.  Offsets are the same exclusive prefix sums the two-pass build produces, so the lists are identical.
+// Count and fill in a single traversal: a CTA takes a tile of 64 consecutive atoms (8 per warp), collects each atom's hits
+// in shared memory while it counts, obtains the tile's list offset from a decoupled look-back scan over the tiles before
+// it (tile aggregate / inclusive prefix published in one 64-bit word, tiles handed out by a ticket so that every
+// predecessor belongs to a CTA that is already running), and then copies the lists out in full rows.  Offsets are the same exclusive prefix sums the two-pass build produces, so the lists are identical.
 // Every wait is bounded: after OP_SPIN polls the tile raises FLAG_NEIGHBOR_OVERFLOW, publishes what it has and goes on.
 constexpr int OP_PER_WARP = 8;
 constexpr int OP_TILE = 8 * OP_PER_WARP;
 static_assert(OP_TILE == 64, "the in-tile scan handles two counts per lane of one warp");
-constexpr int OP_MAXCH = 64;                     // chunk masks kept per atom; chunks beyond are re-tested in the replay
 constexpr int OP_SPIN = 1 << 18;
 
 __device__ __forceinline__ bool rel_hit(const float4 &rj, float sx, float sy, float sz, float rl2_lo, float rl2_hi, double rl2,
@@ -333,13 +331,53 @@ __device__ __forceinline__ void cell_ranges(const double4 &p4, const CellGrid &g
     }
 }
 
+// One atom's traversal for the one-pass build: hits go to `out` (shared memory: the first `cap` of them; or global memory
+// with cap = INT_MAX); returns the number of hits.
+__device__ __forceinline__ int onepass_traverse(int64_t i, const CellGrid &g, double rl2, const float (&edge)[3], float rl2_lo, float rl2_hi,
+                                                const double4 *__restrict__ pos4, const float4 *__restrict__ rel,
+                                                const int32_t *__restrict__ cell_start, int lane, int32_t *out, int cap) {
+    const double4 pi = pos4[i];
+    const float4 ri = rel[i];
+    int cb, ce;
+    cell_ranges(pi, g, cell_start, lane, cb, ce);
+    int cnt = 0;
+    int beg = __shfl_sync(0xffffffffu, cb, 0), end = __shfl_sync(0xffffffffu, ce, 0);
+    float4 rj_next = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (beg + lane < end) rj_next = rel[beg + lane];
+#pragma unroll
+    for (int it = 0; it < 27; ++it) {
+        const int cur_beg = beg, cur_end = end;
+        float4 rj = rj_next;
+        if (it + 1 < 27) {
+            beg = __shfl_sync(0xffffffffu, cb, it + 1);
+            end = __shfl_sync(0xffffffffu, ce, it + 1);
+            if (beg + lane < end) rj_next = rel[beg + lane];
+        }
+        const float sx = (float)(it / 9 - 1) * edge[0] - ri.x;
+        const float sy = (float)((it / 3) % 3 - 1) * edge[1] - ri.y;
+        const float sz = (float)(it % 3 - 1) * edge[2] - ri.z;
+        for (int base = cur_beg; base < cur_end; base += 32) {
+            const int j = base + lane;
+            if (base != cur_beg && j < cur_end) rj = rel[j];
+            const bool hit = j < cur_end && j != i && rel_hit(rj, sx, sy, sz, rl2_lo, rl2_hi, rl2, pi, pos4, j, g);
+            const unsigned m = __ballot_sync(0xffffffffu, hit);
+            const int slot = cnt + __popc(m & ((1u << lane) - 1u));
+            if (hit && slot < cap) out[slot] = j;
+            cnt += __popc(m);
+        }
+    }
+    return cnt;
+}
+
+constexpr int OP_BUF = 160;   // hits kept per atom in shared memory; a longer list is traversed again straight into global memory
+
 __global__ void __launch_bounds__(256) k_neighbors_onepass(int64_t n, CellGrid g, double rl2, const double4 *__restrict__ pos4,
                                                            const float4 *__restrict__ rel, const int32_t *__restrict__ cell_start,
                                                            int64_t *__restrict__ nbr_off, int32_t *__restrict__ nbr, int64_t nbr_cap,
                                                            int *status, unsigned long long *tile_state, int *ticket) {
     // look-back word: flag in the top two bits (0 empty, 1 tile aggregate, 2 inclusive prefix), value below
     constexpr unsigned long long OP_AGG = 1ull << 62, OP_INC = 2ull << 62, OP_VAL = (1ull << 62) - 1;
-    __shared__ unsigned s_mask[OP_TILE][OP_MAXCH];
+    extern __shared__ int32_t s_hits[];   // [OP_TILE][OP_BUF]
     __shared__ int s_cnt[OP_TILE];
     __shared__ long long s_off[OP_TILE];
     __shared__ long long s_prefix, s_total;
@@ -351,43 +389,12 @@ __global__ void __launch_bounds__(256) k_neighbors_onepass(int64_t n, CellGrid g
     const float edge[3] = {(float)(g.box[0] / g.n[0]), (float)(g.box[1] / g.n[1]), (float)(g.box[2] / g.n[2])};
     const float rl2_lo = (float)(rl2 * (1.0 - 1e-5)), rl2_hi = (float)(rl2 * (1.0 + 1e-5));
 
-    // ---- traversal: count, keep the masks ----
+    // ---- traversal: count, keep the hits ----
     for (int a = 0; a < OP_PER_WARP; ++a) {
         const int slot = warp * OP_PER_WARP + a;
         const int64_t i = first + slot;
         int cnt = 0;
-        if (i < n) {
-            const double4 pi = pos4[i];
-            const float4 ri = rel[i];
-            int cb, ce;
-            cell_ranges(pi, g, cell_start, lane, cb, ce);
-            int ch = 0;
-            int beg = __shfl_sync(0xffffffffu, cb, 0), end = __shfl_sync(0xffffffffu, ce, 0);
-            float4 rj_next = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (beg + lane < end) rj_next = rel[beg + lane];
-#pragma unroll
-            for (int it = 0; it < 27; ++it) {
-                const int cur_beg = beg, cur_end = end;
-                float4 rj = rj_next;
-                if (it + 1 < 27) {
-                    beg = __shfl_sync(0xffffffffu, cb, it + 1);
-                    end = __shfl_sync(0xffffffffu, ce, it + 1);
-                    if (beg + lane < end) rj_next = rel[beg + lane];
-                }
-                const float sx = (float)(it / 9 - 1) * edge[0] - ri.x;
-                const float sy = (float)((it / 3) % 3 - 1) * edge[1] - ri.y;
-                const float sz = (float)(it % 3 - 1) * edge[2] - ri.z;
-                for (int base = cur_beg; base < cur_end; base += 32) {
-                    const int j = base + lane;
-                    if (base != cur_beg && j < cur_end) rj = rel[j];
-                    const bool hit = j < cur_end && j != i && rel_hit(rj, sx, sy, sz, rl2_lo, rl2_hi, rl2, pi, pos4, j, g);
-                    const unsigned m = __ballot_sync(0xffffffffu, hit);
-                    if (ch < OP_MAXCH && lane == 0) s_mask[slot][ch] = m;
-                    ++ch;
-                    cnt += __popc(m);
-                }
-            }
-        }
+        if (i < n) cnt = onepass_traverse(i, g, rl2, edge, rl2_lo, rl2_hi, pos4, rel, cell_start, lane, s_hits + slot * OP_BUF, OP_BUF);
         if (lane == 0) s_cnt[slot] = cnt;
     }
     __syncthreads();
@@ -441,41 +448,23 @@ __global__ void __launch_bounds__(256) k_neighbors_onepass(int64_t n, CellGrid g
     const long long tile_off = s_prefix;
     if (first + OP_TILE >= n && threadIdx.x == 0) nbr_off[n] = s_total;   // the last tile closes the offsets
 
-    // ---- replay: write the lists from the masks ----
+    // ---- write the lists: full rows from shared memory ----
     for (int a = 0; a < OP_PER_WARP; ++a) {
         const int slot = warp * OP_PER_WARP + a;
         const int64_t i = first + slot;
         if (i >= n) break;
         const long long off = tile_off + s_off[slot];
+        const int cnt = s_cnt[slot];
         if (lane == 0) nbr_off[i] = off;
-        if (off + s_cnt[slot] > nbr_cap) {
+        if (off + cnt > nbr_cap) {
             if (lane == 0) atomicOr(status, FLAG_NEIGHBOR_OVERFLOW);
             continue;
         }
-        const double4 pi = pos4[i];
-        const float4 ri = rel[i];
-        int cb, ce;
-        cell_ranges(pi, g, cell_start, lane, cb, ce);
-        int ch = 0, run = 0;
-        for (int it = 0; it < 27; ++it) {
-            const int cur_beg = __shfl_sync(0xffffffffu, cb, it), cur_end = __shfl_sync(0xffffffffu, ce, it);
-            for (int base = cur_beg; base < cur_end; base += 32) {
-                const int j = base + lane;
-                unsigned m;
-                if (ch < OP_MAXCH) m = s_mask[slot][ch];
-                else {   // beyond the kept masks: test again
-                    const float sx = (float)(it / 9 - 1) * edge[0] - ri.x;
-                    const float sy = (float)((it / 3) % 3 - 1) * edge[1] - ri.y;
-                    const float sz = (float)(it % 3 - 1) * edge[2] - ri.z;
-                    float4 rj = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (j < cur_end) rj = rel[j];
-                    const bool hit = j < cur_end && j != i && rel_hit(rj, sx, sy, sz, rl2_lo, rl2_hi, rl2, pi, pos4, j, g);
-                    m = __ballot_sync(0xffffffffu, hit);
-                }
-                if ((m >> lane) & 1u) nbr[off + run + __popc(m & ((1u << lane) - 1u))] = j;
-                run += __popc(m);
-                ++ch;
-            }
+        if (cnt <= OP_BUF) {
+            const int32_t *src = s_hits + slot * OP_BUF;
+            for (int e = lane; e < cnt; e += 32) nbr[off + e] = src[e];
+        } else {
+            onepass_traverse(i, g, rl2, edge, rl2_lo, rl2_hi, pos4, rel, cell_start, lane, nbr + off, 0x7fffffff);
         }
     }
 }
@@ -553,7 +542,7 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
         MLIP_CUDA_TRY(c, cudaMemsetAsync(c->tile_state, 0, sizeof(unsigned long long) * (n_tiles + 1), s));
         MLIP_CUDA_TRY(c, cudaMemsetAsync(c->tile_ticket, 0, sizeof(int), s));
         k_rel_pos<<<blocks_for(n, 256), 256, 0, s>>>(n, g, c->pos4, relpos);
-        k_neighbors_onepass<<<(unsigned)n_tiles, 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_off, c->nbr, c->nbr_cap,
+        k_neighbors_onepass<<<(unsigned)n_tiles, 256, sizeof(int32_t) * OP_TILE * OP_BUF, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_off, c->nbr, c->nbr_cap,
                                                                c->status, c->tile_state, c->tile_ticket);
         c->launches += 5 + 2 * 3 + 2;   // cell id, place, sort, gather, centre order; two scans; relative positions, lists
         timing_end(c->ev_build, c->build_count, s);

@@ -429,3 +429,18 @@ def test_deterministic_force_mode_is_bit_reproducible_and_matches_oracle():
     with pytest.raises(mlip.MlipError) as err:
         mlip.Potential(6, w.r_cut, 1.0, enc, head, w.masses, force_mode=1, precision=1)
     assert err.value.code == mlip.binding.CODES["MLIP_ERR_UNSUPPORTED"]
+
+
+def test_in_step_rebuild_with_lists_longer_than_the_hit_buffer():
+    """A wide skin gives ~220 entries per atom: the one-pass rebuild then takes its second-traversal path for every atom."""
+    w, model, pot = make_pair(1, 8, 2.5)
+    pot.build_neighbors(w.pos, w.species, w.box)
+    pot.set_velocities(w.vel)
+    pot.step(4, 1.0, 2)
+    assert pot.sync_status(raise_on_error=False) == 0
+    assert pot.rebuilds() == 3
+    pos, vel, step = pot.state()
+    seg, nbr = pot.neighbors()
+    nl = oracle.neighbors(pos.cpu().numpy(), w.species, w.n_species, w.box, w.r_cut + 2.5)
+    assert nl.nbr.size / w.n_atoms > 200
+    assert canonical_equal(nl, seg, nbr)
