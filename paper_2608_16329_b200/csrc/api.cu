@@ -196,7 +196,7 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
         if ((rc = dev_alloc(c, &c->rebuild_flag, 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->nhc, 8)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->acc_fx, 10)) != MLIP_OK) break;
-        if ((rc = dev_alloc(c, &c->tile_ticket, 1)) != MLIP_OK) break;
+        if ((rc = dev_alloc(c, &c->tile_ticket, 2)) != MLIP_OK) break;   // ticket, private overflow flag
         if ((rc = dev_alloc(c, &c->tile_counter, (size_t)MAX_SPECIES)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->species_start, (size_t)MAX_SPECIES + 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->stage_out, 10)) != MLIP_OK) break;

@@ -537,20 +537,36 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
     // grids of at least 3 x 3 x 3 cells take the fp32 cell-relative traversal (positions staged in the idle force array)
     const bool rel = g.n[0] >= 3 && g.n[1] >= 3 && g.n[2] >= 3;
     float4 *relpos = c->force;
-    if (rel && !allow_sync_grow && c->tile_state) {   // in-step rebuild: single traversal, capacity as it stands
+    // Single traversal whenever a list array exists: always for in-step rebuilds (capacity as it stands, overflow -> status
+    // bit), and for a synchronising build as a first try whose overflow flag is private and sends it to the two-pass path.
+    bool rel_ready = false;
+    if (rel && c->tile_state && c->nbr_cap > 0) {
         const int64_t n_tiles = (n + OP_TILE - 1) / OP_TILE;
         MLIP_CUDA_TRY(c, cudaMemsetAsync(c->tile_state, 0, sizeof(unsigned long long) * (n_tiles + 1), s));
-        MLIP_CUDA_TRY(c, cudaMemsetAsync(c->tile_ticket, 0, sizeof(int), s));
+        MLIP_CUDA_TRY(c, cudaMemsetAsync(c->tile_ticket, 0, 2 * sizeof(int), s));
         k_rel_pos<<<blocks_for(n, 256), 256, 0, s>>>(n, g, c->pos4, relpos);
+        rel_ready = true;
+        int *flag = allow_sync_grow ? c->tile_ticket + 1 : c->status;
         k_neighbors_onepass<<<(unsigned)n_tiles, 256, sizeof(int32_t) * OP_TILE * OP_BUF, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_off, c->nbr, c->nbr_cap,
-                                                               c->status, c->tile_state, c->tile_ticket);
+                                                               flag, c->tile_state, c->tile_ticket);
         c->launches += 5 + 2 * 3 + 2;   // cell id, place, sort, gather, centre order; two scans; relative positions, lists
-        timing_end(c->ev_build, c->build_count, s);
         MLIP_CUDA_TRY(c, cudaGetLastError());
-        return MLIP_OK;
+        bool done = true;
+        if (allow_sync_grow) {
+            int overflow = 0;
+            MLIP_CUDA_TRY(c, cudaMemcpyAsync(c->total_host, c->nbr_off + n, sizeof(int64_t), cudaMemcpyDeviceToHost, s));
+            MLIP_CUDA_TRY(c, cudaMemcpyAsync(&overflow, c->tile_ticket + 1, sizeof(int), cudaMemcpyDeviceToHost, s));
+            MLIP_CUDA_TRY(c, cudaStreamSynchronize(s));
+            done = overflow == 0 && *c->total_host <= c->nbr_cap;
+            if (done) c->n_entries = *c->total_host;
+        }
+        if (done) {
+            timing_end(c->ev_build, c->build_count, s);
+            return MLIP_OK;
+        }
     }
     if (rel) {
-        k_rel_pos<<<blocks_for(n, 256), 256, 0, s>>>(n, g, c->pos4, relpos);
+        if (!rel_ready) k_rel_pos<<<blocks_for(n, 256), 256, 0, s>>>(n, g, c->pos4, relpos);
         k_neighbors_rel<false><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_count, nullptr, nullptr, 0, c->status);
         c->launches += 1;
     } else
