@@ -173,7 +173,7 @@ def run_reference(args, rank, world):
     """CPU oracle arm: each step evaluates a bounded sample of central atoms of the same workload."""
     if rank != 0:
         return
-    from paper_2608_16329_b200 import workloads as wl
+    import workloads as wl
     w = wl.make_workload(CFG, n_cells=args.cells)
     enc, head = wl.workload_weights(CFG, w.n_species)
     n_centers = min(args.cpu_centers, 2048)
@@ -202,7 +202,7 @@ def run_sweep(args):
     Lattice, displacements, species and velocities are drawn on the device with a seeded torch generator."""
     import torch
     import paper_2608_16329_b200 as mlip
-    from paper_2608_16329_b200 import workloads as wl
+    import workloads as wl
     dev = torch.device("cuda", 0)
     enc, head = wl.workload_weights(CFG, 6)
     masses = np.array(wl.MASSES[CFG])
@@ -275,7 +275,7 @@ def main():
     import torch
     import torch.distributed as dist
     import paper_2608_16329_b200 as mlip
-    from paper_2608_16329_b200 import workloads as wl
+    import workloads as wl
 
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)

@@ -3,13 +3,13 @@
 Run `python -m oracle.calibrate_workloads` from the repository root.  For each
 workload (a small instance of it) it prints the RMS of the invariants and of
 the force magnitude with the scales currently stored in
-`paper_2608_16329_b200/workloads.py`, and the head scale that would bring the
+`workloads/__init__.py`, and the head scale that would bring the
 RMS force to 1 eV/Angstrom.  Calls only the oracle.
 """
 import numpy as np
 
 import oracle
-from paper_2608_16329_b200 import workloads as wl
+import workloads as wl
 
 SMALL = {1: 4, 2: 6, 3: 4, 4: 8, 5: 4}
 

@@ -105,7 +105,7 @@ def test_fp64_descriptor_shape_variants_match_oracle(k, l_max):
     """Radial width k and angular order l_max of the paper's ablations (Tables 6 and 7, Fig. 4(c)); the fp64 kernel is
     compiled for each shape, the oracle is generic in both."""
     import paper_2608_16329_b200 as mlip
-    from paper_2608_16329_b200 import workloads as wl
+    import workloads as wl
     C = 3
     w = wl.make_workload(3, n_cells=5)
     enc, head = wl.make_weights(C, 77, wl.ENC_OUT_SCALE[3], wl.HEAD_OUT_SCALE[3], k=k, l_max=l_max)
@@ -126,7 +126,7 @@ def test_fp64_descriptor_shape_variants_match_oracle(k, l_max):
 
 def test_other_shapes_are_refused_by_the_fp32_path():
     import paper_2608_16329_b200 as mlip
-    from paper_2608_16329_b200 import workloads as wl
+    import workloads as wl
     enc, head = wl.make_weights(1, 3, k=16, l_max=3)
     with pytest.raises(mlip.MlipError) as err:
         mlip.Potential(1, 6.0, 1.0, enc, head, np.array([50.0]), k=16, l_max=3)

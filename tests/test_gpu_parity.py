@@ -23,7 +23,7 @@ def test_neighbor_lists_bit_exact(cfg, n_cells, skin):
 
 def test_neighbor_lists_non_cubic_random_gas():
     import paper_2608_16329_b200 as mlip
-    from paper_2608_16329_b200 import workloads as wl
+    import workloads as wl
     rng = np.random.default_rng(3)
     box = np.array([15.0, 21.5, 29.0])
     pos = rng.uniform(0, 1, (3000, 3)) * box
@@ -151,7 +151,7 @@ def test_device_side_problems_become_status_codes():
 
 def test_table_tolerance_is_enforced():
     import paper_2608_16329_b200 as mlip
-    from paper_2608_16329_b200 import workloads as wl
+    import workloads as wl
     enc, head = wl.workload_weights(5, 6)
     with pytest.raises(mlip.MlipError) as err:
         mlip.Potential(6, 6.0, 1.0, enc, head, np.ones(6), table_knots=8)
@@ -223,7 +223,7 @@ def test_dense_system_beyond_the_pair_queue_matches_oracle():
     """A compressed lattice with ~165 neighbors inside the cutoff: more than the 160-entry pair queue, so the
     encoding runs in several rounds and the derivation re-scans the list."""
     import paper_2608_16329_b200 as mlip
-    from paper_2608_16329_b200 import workloads as wl
+    import workloads as wl
     rng = np.random.default_rng(21)
     a, n = 2.8, 6
     box = np.full(3, a * n)
@@ -249,7 +249,7 @@ def test_dense_system_beyond_the_pair_queue_matches_oracle():
 def test_species_conditioning_variants_match_oracle(chi_e, chi_r, precision):
     """Section 3.2.2: encoder conditioned on the neighbor species only or on nothing, universal regression network."""
     import paper_2608_16329_b200 as mlip
-    from paper_2608_16329_b200 import workloads as wl
+    import workloads as wl
     C = 3
     w = wl.make_workload(3, n_cells=5)
     enc, head = wl.workload_weights(3, C)
@@ -304,7 +304,7 @@ def test_dilute_system_with_isolated_atoms_ragged_tiles_and_an_absent_species(pr
     """Degenerate inputs: atoms with no neighbor inside r_cut (E_i = head(0), no force), lists that hold skin-shell entries
     only, species counts that are not multiples of the tile size, and a declared species that no atom has."""
     import paper_2608_16329_b200 as mlip
-    from paper_2608_16329_b200 import workloads as wl
+    import workloads as wl
     rng = np.random.default_rng(11)
     C, a, m = 4, 5.0, 7
     grid = np.stack(np.meshgrid(*[np.arange(m)] * 3, indexing="ij"), -1).reshape(-1, 3).astype(np.float64)
@@ -335,7 +335,7 @@ def test_dilute_system_with_isolated_atoms_ragged_tiles_and_an_absent_species(pr
 @pytest.mark.parametrize("precision", [0, 1])
 def test_single_atom(precision):
     import paper_2608_16329_b200 as mlip
-    from paper_2608_16329_b200 import workloads as wl
+    import workloads as wl
     enc, head = wl.make_weights(2, 9)
     model = oracle.Model(2, 6.0, enc, head)
     pos, species, box = np.array([[3.0, 4.0, 5.0]]), np.array([1], dtype=np.int32), np.array([20.0, 20.0, 20.0])
@@ -353,7 +353,7 @@ def test_single_atom(precision):
 @pytest.mark.parametrize("precision", [0, 1])
 def test_quintic_envelope_matches_oracle(precision):
     import paper_2608_16329_b200 as mlip
-    from paper_2608_16329_b200 import workloads as wl
+    import workloads as wl
     w = wl.make_workload(3, n_cells=5)
     enc, head = wl.workload_weights(3, 3)
     model = oracle.Model(3, w.r_cut, enc, head, envelope=1)
@@ -395,7 +395,7 @@ def test_deterministic_force_mode_is_bit_reproducible_and_matches_oracle():
     """force_mode = 1 takes every scheduling-dependent sum in integer arithmetic: two contexts fed the same input give
     bit-identical energies, forces, virial and trajectories (the default mode agrees only to rounding)."""
     import paper_2608_16329_b200 as mlip
-    from paper_2608_16329_b200 import workloads as wl
+    import workloads as wl
     w = wl.make_workload(5, n_cells=12)                    # 6,912 atoms: thousands of tiles over all SMs
     enc, head = wl.workload_weights(5, 6)
     runs = []

@@ -122,7 +122,7 @@ def test_derivative_matches_finite_difference():
 
 def test_invariants_do_not_depend_on_the_choice_of_q():
     """Q_l is fixed only up to an orthogonal mixing of rows; energies must not notice."""
-    from paper_2608_16329_b200 import workloads as wl
+    import workloads as wl
     w = wl.make_workload(1, n_cells=4)
     enc, head = wl.workload_weights(1, 6)
     base = oracle.Model(6, 6.0, enc, head)

@@ -6,7 +6,7 @@ from scipy.special import eval_legendre
 from scipy.stats import special_ortho_group
 
 import oracle
-from paper_2608_16329_b200 import workloads as wl
+import workloads as wl
 
 BIG = np.array([60.0, 60.0, 60.0])
 

@@ -3,7 +3,7 @@ import numpy as np
 import pytest
 
 import oracle
-from paper_2608_16329_b200 import workloads as wl
+import workloads as wl
 
 # textbook coordination shells: (squared distance in units of a^2, multiplicity)
 FCC_SHELLS = [(0.5, 12), (1.0, 6), (1.5, 24), (2.0, 12), (2.5, 24), (3.0, 8), (3.5, 48), (4.0, 6)]

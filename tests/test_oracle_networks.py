@@ -6,7 +6,7 @@ import pytest
 from scipy.special import expit
 
 import oracle
-from paper_2608_16329_b200 import workloads as wl
+import workloads as wl
 from conftest import golden_lines
 
 LN3 = math.log(3.0)

@@ -2,7 +2,7 @@
 import numpy as np
 
 import oracle
-from paper_2608_16329_b200 import workloads as wl
+import workloads as wl
 
 
 def _setup():

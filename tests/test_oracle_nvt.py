@@ -3,7 +3,7 @@ import numpy as np
 from scipy.integrate import solve_ivp
 
 import oracle
-from paper_2608_16329_b200 import workloads as wl
+import workloads as wl
 
 
 def _setup():
