@@ -45,10 +45,33 @@ FLOP_PER_ATOM = 88700.0        # invariants, W_i, head forward + reverse, SiLU
 FP32_LANES_PER_SM = 128
 FP64_LANES_PER_SM = 64         # fp64 path: DFMA lanes per SM
 
-# DRAM traffic of one fused-kernel launch from the committed ncu capture
-# (profiles/k_mega_hea6_fcc50.md: dram__bytes_read.sum + dram__bytes_write.sum of a 500,000-atom launch, per atom;
-# the traffic is per-atom, so a launch of N atoms is reported as this figure times N).
-NCU_DRAM_BYTES_PER_ATOM = 746.0
+# DRAM traffic of one fused-kernel launch comes from the committed ncu capture of a 500,000-atom launch
+# (dram__bytes_read.sum + dram__bytes_write.sum per atom; the traffic is per-atom, so a launch of N atoms is reported as
+# that figure times N).  The record names the kernel sources it was captured from; a different kernel prints no traffic.
+TRAFFIC_RECORD = os.path.join(ROOT, "profiles", "k_mega_hea6_fcc50.traffic.txt")
+KERNEL_SOURCES = ["megakernel.cu", "pair_math.cuh", "common.cuh"]
+
+
+def kernel_revision() -> str:
+    """Hash of the fused kernel's sources: ties a profiler record to the code it was taken from."""
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2608_16329_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic():
+    """(bytes per atom, note) from the ncu record, or (None, why) when it does not belong to the kernel as built."""
+    try:
+        rec = dict(line.split(":", 1) for line in open(TRAFFIC_RECORD) if ":" in line and not line.startswith("#"))
+        rev, per_atom = rec["kernel_revision"].strip(), float(rec["dram_bytes_per_atom"])
+    except (OSError, KeyError, ValueError):
+        return None, "no ncu record"
+    if rev != kernel_revision():
+        return None, f"ncu record is of kernel revision {rev}, this kernel is {kernel_revision()}"
+    return per_atom, f"ncu capture of a 500,000-atom launch scaled per atom (kernel revision {rev})"
 
 
 def parse_args():
@@ -153,20 +176,71 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "sm_max_mhz": 1965.0}, "fallback"
 
 
-def cpu_oracle_sample(w, enc, head, n_centers, repeats=1):
-    """Time the oracle (neighbor search + full evaluation) on evenly spread central atoms."""
+LATTICES = {2: ((32, 32, 32), 2, 3.3), 3: ((64, 64, 64), 4, 4.05), 4: ((125, 125, 128), 1, 20.0 ** (1.0 / 3.0))}
+
+
+def sample_blocks(cells, n_basis, a, r_cut, n_centers, seed=0):
+    """Central atoms for the CPU leg: rectangular blocks of unit cells spread over the box (caller indices; lattice
+    sites are numbered (ix, iy, iz, basis)).  Returns (all block atoms, those far enough inside a block that every atom
+    within r_cut of them is in the block too -- the atoms whose complete force the block's evaluation gives)."""
+    size = tuple(min(c, s) for c, s in zip(cells, (8, 8, 24)))
+    per_block = size[0] * size[1] * size[2] * n_basis
+    n_blocks = max(1, n_centers // per_block)
+    margin = int(np.ceil((r_cut + 0.75) / a))
+    rng = np.random.default_rng(seed)
+    origins = [(0, 0, 0), tuple(c - s for c, s in zip(cells, size))]
+    while len(origins) < n_blocks:
+        origins.append(tuple(int(rng.integers(0, c - s + 1)) for c, s in zip(cells, size)))
+    all_atoms, inner = [], []
+    for o in origins[:n_blocks]:
+        ix, iy, iz, b = np.meshgrid(*[o[d] + np.arange(size[d]) for d in range(3)], np.arange(n_basis), indexing="ij")
+        idx = (((ix * cells[1] + iy) * cells[2] + iz) * n_basis + b)
+        all_atoms.append(idx.ravel())
+        if min(size) > 2 * margin:
+            inner.append(idx[margin:size[0] - margin, margin:size[1] - margin, margin:size[2] - margin].ravel())
+    all_atoms = np.unique(np.concatenate(all_atoms)).astype(np.int64)
+    inner = np.unique(np.concatenate(inner)).astype(np.int64) if inner else np.empty(0, np.int64)
+    return all_atoms, inner
+
+
+def cpu_oracle_sample(w, enc, head, n_centers, repeats=1, rows=None, pos=None, k=32, l_max=3):
+    """Time the oracle (neighbor search + full evaluation) on `rows` (default: evenly spread central atoms).
+    Returns (rows, seconds, threads, the oracle's outputs)."""
     import oracle
-    model = oracle.Model(w.n_species, w.r_cut, enc, head)
-    rows = np.linspace(0, w.n_atoms - 1, n_centers).astype(np.int64)
-    rows = np.unique(rows)
-    best = None
+    model = oracle.Model(w.n_species, w.r_cut, enc, head, k=k, l_max=l_max)
+    if rows is None:
+        rows = np.unique(np.linspace(0, w.n_atoms - 1, n_centers).astype(np.int64))
+    pos = w.pos if pos is None else pos
+    best, out = None, None
     for _ in range(repeats):
         t0 = time.perf_counter()
-        nl = oracle.neighbors(w.pos, w.species, w.n_species, w.box, w.r_cut + w.skin, rows=rows)
-        oracle.compute(model, w.pos, w.species, w.box, nl)
+        nl = oracle.neighbors(pos, w.species, w.n_species, w.box, w.r_cut + w.skin, rows=rows)
+        out = oracle.compute(model, pos, w.species, w.box, nl)
         dt = time.perf_counter() - t0
         best = dt if best is None else min(best, dt)
-    return rows.size, best, oracle.num_threads()
+    return rows, best, oracle.num_threads(), out
+
+
+def problem_setup(args, rank=0):
+    """Workload, weights and the algorithmic work per unit for the flags given (no GPU needed)."""
+    import workloads as wl
+    cfg = args.cfg
+    w = wl.make_workload(cfg, n_cells=args.cells if cfg == CFG else None, seed=wl.BASE_SEED + cfg + 17 * rank)
+    default_shape = args.k == 32 and args.lmax == 3
+    if default_shape:
+        enc, head = wl.workload_weights(cfg, w.n_species)
+    else:   # descriptor-shape variants of the paper's ablations: same recipe, networks of that shape
+        enc, head = wl.make_weights(w.n_species, wl.BASE_SEED + cfg + 1000, wl.ENC_OUT_SCALE[cfg], wl.HEAD_OUT_SCALE[cfg],
+                                    k=args.k, l_max=args.lmax)
+    flop_pair, flop_atom = FLOP_PER_PAIR, FLOP_PER_ATOM
+    if not default_shape:   # the same count written out in k and d = (l_max + 1)^2
+        d_ang, n_inv = (args.lmax + 1) ** 2, (args.lmax + 1) * args.k
+        flop_pair = 60 + 150 * d_ang / 16 + 512 * args.k / 32 + 6 * d_ang * args.k + 168 * d_ang / 16
+        flop_atom = 3 * d_ang * args.k + 4 * (n_inv * 64 + 3 * 64 * 64) + 256 + 5000
+    lattice = ((args.cells,) * 3, 4, 3.6) if cfg == CFG else LATTICES[cfg]
+    return {"w": w, "enc": enc, "head": head, "default_shape": default_shape, "flop_pair": flop_pair, "flop_atom": flop_atom,
+            "rebuild_every": REBUILD_EVERY if cfg != 4 else 3,   # the ionic stand-in is far from equilibrium under random weights
+            "lattice": lattice, "f64": args.precision == "f64"}
 
 
 def run_reference(args, rank, world):
@@ -182,8 +256,8 @@ def run_reference(args, rank, world):
     t0 = time.perf_counter()
     done, cores = 0, 1
     for _ in range(args.steps):
-        n, _, cores = cpu_oracle_sample(w, enc, head, n_centers)
-        done += n
+        rows, _, cores, _ = cpu_oracle_sample(w, enc, head, n_centers)
+        done += rows.size
     dt = time.perf_counter() - t0
     value = done / dt
     sample = (f"{n_centers} central atoms spread evenly over the {w.n_atoms}-atom workload per step: cell-list "
@@ -288,16 +362,9 @@ def main():
         torch.cuda.synchronize()
 
     cfg = args.cfg
-    w = wl.make_workload(cfg, n_cells=args.cells if cfg == CFG else None, seed=wl.BASE_SEED + cfg + 17 * rank)
-    default_shape = args.k == 32 and args.lmax == 3
-    if default_shape:
-        enc, head = wl.workload_weights(cfg, w.n_species)
-    else:   # descriptor-shape variants of the paper's ablations: same recipe, networks of that shape
-        enc, head = wl.make_weights(w.n_species, wl.BASE_SEED + cfg + 1000, wl.ENC_OUT_SCALE[cfg], wl.HEAD_OUT_SCALE[cfg],
-                                    k=args.k, l_max=args.lmax, force_mode=1 if args.deterministic else 0)
-    rebuild_every = REBUILD_EVERY if cfg != 4 else 3   # the ionic stand-in is far from equilibrium under random weights
+    prob = problem_setup(args, rank)
+    w, enc, head, default_shape, rebuild_every, f64 = (prob[q] for q in ("w", "enc", "head", "default_shape", "rebuild_every", "f64"))
     n = w.n_atoms
-    f64 = args.precision == "f64"
     pot = mlip.Potential(w.n_species, w.r_cut, w.skin, enc, head, w.masses, device=local_rank, precision=1 if f64 else 0,
                          k=args.k, l_max=args.lmax, force_mode=1 if args.deterministic else 0)
     table_err = mlip.mlip_table_error(pot.ctx)
@@ -379,11 +446,7 @@ def main():
         peak_tflops = n_sm * lanes * 2 * sm_max * 1e6 / 1e12
         pairs = counters["pairs_in_cutoff"]
         entries = counters["list_entries"]
-        flop_pair, flop_atom = FLOP_PER_PAIR, FLOP_PER_ATOM
-        if not default_shape:   # the same count written out in k and d = (l_max + 1)^2
-            d_ang, n_inv = (args.lmax + 1) ** 2, (args.lmax + 1) * args.k
-            flop_pair = 60 + 150 * d_ang / 16 + 512 * args.k / 32 + 6 * d_ang * args.k + 168 * d_ang / 16
-            flop_atom = 3 * d_ang * args.k + 4 * (n_inv * 64 + 3 * 64 * 64) + 256 + 5000
+        flop_pair, flop_atom = prob["flop_pair"], prob["flop_atom"]
         flop = flop_pair * pairs + FLOP_PER_SKIN_ENTRY * max(entries - pairs, 0) + flop_atom * n
         k_avg_ms = k_ms / max(k_launches, 1)
         achieved = flop / (k_avg_ms * 1e-3) / 1e12
@@ -393,10 +456,16 @@ def main():
                     "kernel_ms_avg": k_avg_ms, "kernel_launches_timed": k_launches,
                     "kernel_share_of_step": k_ms / ms if ms > 0 else None,
                     "flop_per_launch": flop, "pairs_in_cutoff_per_atom": pairs / n, "list_entries_per_atom": entries / n,
-                    "traffic": None if NCU_DRAM_BYTES_PER_ATOM is None or f64 else NCU_DRAM_BYTES_PER_ATOM * n,
                     "hbm_peak_gbs": peaks["hbm_gbs"], "hbm_peak_kind": f"of {peak_kind}"}
+        per_atom, traffic_note = recorded_traffic() if (default_shape and not f64 and cfg == CFG) else (None, "no ncu record for this variant")
+        roofline["traffic"] = None if per_atom is None else per_atom * n
+        roofline["traffic_source"] = traffic_note
         if clocks and clocks.get("sm_mhz"):
             roofline["frac_at_sampled_clock"] = achieved / (n_sm * lanes * 2 * clocks["sm_mhz"] * 1e6 / 1e12)
+        if not f64:   # the same fraction against an FMA-saturating kernel timed in this process
+            ffma = mlip.mlip_measure_fp32_peak(local_rank)
+            roofline["peak_measured_ffma"] = ffma
+            roofline["frac_of_measured_ffma"] = achieved / ffma
         resident = mlip.mlip_resident_bytes(pot.ctx)
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
                 "ms_per_step": ms_max / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -417,10 +486,27 @@ def main():
                 "status": mlip.binding.ERRORS.get(status, status),
                 "energy_final_eV": {"potential": float(e_final[0]), "kinetic": float(e_final[1])}}
         if not args.no_cpu_baseline and world == 1:
-            nc, sec, cores = cpu_oracle_sample(w, enc, head, args.cpu_centers)
-            line["cpu_baseline"] = {"value": nc / sec, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                    "sample": f"{nc} central atoms spread evenly over the {n}-atom workload, one energy/"
-                                              f"force/virial evaluation incl. their neighbor search ({sec:.1f} s)"}
+            # The oracle on blocks of central atoms at the positions the run ended on; its outputs are then compared
+            # with the GPU's evaluation of the same state: E_i of every sampled atom, the force of the blocks' interior
+            # atoms (those whose whole r_cut neighborhood was evaluated).
+            cells, n_basis, a_lat = prob["lattice"]
+            rows, inner = sample_blocks(cells, n_basis, a_lat, w.r_cut, args.cpu_centers)
+            pos_t, _, _ = pot.state()
+            gpu = pot.compute(want_e_atom=True)
+            pot.sync_status(raise_on_error=False)
+            pos_now = pos_t.cpu().numpy()
+            rows, sec, cores, ref = cpu_oracle_sample(w, enc, head, rows.size, rows=rows, pos=pos_now, k=args.k, l_max=args.lmax)
+            line["cpu_baseline"] = {"value": rows.size / sec, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                    "sample": f"{rows.size} central atoms in blocks of cells spread over the {n}-atom workload, one "
+                                              f"energy/force/virial evaluation incl. their neighbor search ({sec:.1f} s)"}
+            rows_t, inner_t = torch.as_tensor(rows, device=dev), torch.as_tensor(inner, device=dev)
+            d_e = np.abs(gpu["e_atom"][rows_t].double().cpu().numpy() - ref["e_atom"][rows])
+            d_f = np.abs(gpu["forces"][inner_t].double().cpu().numpy() - ref["forces"][inner]) if inner.size else np.zeros(1)
+            e_tol, f_tol = (1e-9, 2e-9) if f64 else (2e-5, 1e-4)
+            line["parity"] = {"against": "oracle, same state (positions after the timed steps)", "n_atoms_e": int(rows.size),
+                              "max_dE_i": float(d_e.max()), "n_atoms_f": int(inner.size), "max_dF": float(d_f.max()),
+                              "tolerance": {"dE_i": e_tol * max(1.0, float(np.abs(ref["e_atom"][rows]).max())), "dF": f_tol},
+                              "ok": bool(d_e.max() <= e_tol * max(1.0, float(np.abs(ref["e_atom"][rows]).max())) and d_f.max() <= f_tol)}
         print(json.dumps(line), flush=True)
     pot.close()
     if world > 1:

@@ -46,9 +46,10 @@ enum {
     MLIP_ERR_INVALID_ARG = 1,
     MLIP_ERR_UNSUPPORTED = 2,      /* k, l_max, network shape, species count not compiled in */
     MLIP_ERR_BOX_TOO_SMALL = 3,    /* an edge is shorter than 2 (r_cut + skin) */
-    MLIP_ERR_NEIGHBOR_OVERFLOW = 4,/* list capacity exceeded during an in-step rebuild */
+    MLIP_ERR_NEIGHBOR_OVERFLOW = 4,/* list capacity exceeded during an in-step rebuild (the fused kernel then skips its
+                                      evaluations until the lists are rebuilt by mlip_build_neighbors) */
     MLIP_ERR_SKIN_EXCEEDED = 5,    /* an atom moved more than skin/2 since the last build */
-    MLIP_ERR_NONFINITE = 6,        /* NaN/Inf or out-of-box position */
+    MLIP_ERR_NONFINITE = 6,        /* NaN/Inf or out-of-box position, species out of range, over-full cell */
     MLIP_ERR_TABLE_TOLERANCE = 7,  /* radial table misses the encoder by more than table_tol */
     MLIP_ERR_NOT_BUILT = 8,        /* compute/step before build_neighbors */
     MLIP_ERR_OOM = 9,
@@ -78,7 +79,8 @@ typedef struct {
     int force_mode;       /* 0: floating-point atomics for the force scatter and the energy / virial totals (results vary in
                              the last bits from run to run); 1: deterministic -- those sums are taken in integer arithmetic
                              (forces in units of 2^-32 eV/Angstrom), so equal inputs give bit-identical outputs and
-                             trajectories; +24 bytes per atom, fp32 path only */
+                             trajectories, NVE and NVT alike (the thermostat's kinetic energy is summed in a fixed order in
+                             either mode); +24 bytes per atom, fp32 path only */
     int envelope;         /* smooth cutoff f_c multiplying the encoder output (the paper names none): 0 = (1 + cos(pi r / r_c)) / 2,
                              1 = 1 - 10 x^3 + 15 x^4 - 6 x^5 with x = r / r_c (second derivative also vanishes at r_c) */
 } mlip_config;
@@ -110,7 +112,11 @@ int mlip_table_error(const mlip_ctx *ctx, double *err_value, double *err_deriv);
  * velocities are reset to zero.  Positions must lie in [0, L).  May reallocate
  * and synchronises once (to size the list).
  *   pos      dev [N][3] double      species  dev [N] int32 in [0, C)
- *   box      host [3] edge lengths (orthorhombic); each >= 2 (r_cut + skin)
+ *   box      host [9]: the three cell vectors, row-major (a_x a_y a_z  b_x b_y b_z  c_x c_y c_z).  Only orthorhombic
+ *            cells aligned with the axes are compiled in: a non-zero off-diagonal entry gives MLIP_ERR_UNSUPPORTED;
+ *            each edge (the diagonal) must be >= 2 (r_cut + skin), else MLIP_ERR_BOX_TOO_SMALL.
+ * A non-finite or out-of-box position, a species outside [0, C) or more than 1,024 atoms in one cell is reported at once
+ * as MLIP_ERR_NONFINITE (no lists are built).
  */
 int mlip_build_neighbors(mlip_ctx *ctx, int64_t n_atoms, const double *pos, const int32_t *species,
                          const double *box, void *stream);
@@ -121,7 +127,8 @@ int mlip_build_neighbors(mlip_ctx *ctx, int64_t n_atoms, const double *pos, cons
  * nbr[seg_ptr[i*C+s] .. seg_ptr[i*C+s+1]).  Synchronises.
  *   seg_ptr dev [N*C+1] int64, nbr dev [capacity] int32, n_entries_host out.
  * If capacity is too small only seg_ptr and *n_entries_host are valid and
- * MLIP_ERR_NEIGHBOR_OVERFLOW is returned.
+ * MLIP_ERR_NEIGHBOR_OVERFLOW is returned.  While the status word holds a list overflow or a broken configuration from
+ * an in-step rebuild (see mlip_sync_status) the lists are incomplete and the call returns that error without exporting.
  */
 int mlip_get_neighbors(mlip_ctx *ctx, int64_t *seg_ptr, int32_t *nbr, int64_t capacity,
                        int64_t *n_entries_host, void *stream);
@@ -172,7 +179,7 @@ int mlip_compute_f64(mlip_ctx *ctx, double *energy, double *forces, double *viri
  * Same evaluation with HOST buffers: copies positions in (and species at a
  * rebuild), rebuilds the lists when `rebuild` != 0 or none exist, evaluates,
  * copies results out and synchronises.  This is the call a host-side MD code
- * makes once per time step.
+ * makes once per time step.  box_host as in mlip_build_neighbors ([9], row-major cell vectors).
  */
 int mlip_compute_host(mlip_ctx *ctx, int64_t n_atoms, const double *pos_host, const int32_t *species_host,
                       const double *box_host, int rebuild, double *energy_host, float *forces_host,
@@ -197,7 +204,7 @@ int mlip_step(mlip_ctx *ctx, int n_steps, double dt_fs, int rebuild_every, void 
  * Martyna-Tuckerman-Tobias-Klein integration: thermostat half step, velocity-Verlet step, thermostat half step) around
  * the same force evaluation.  Section 4.2 runs its MD in the NVT ensemble at 300 K without naming the thermostat; the
  * chain thermostat is the reading taken.  rebuild_every as in mlip_step.  The thermostat state lives in the context
- * (zero at creation) and carries over between calls.  Per step it adds a kinetic-energy reduction, two one-thread
+ * (zero at creation) and carries over between calls.  Per step it adds two kinetic-energy reductions, two one-thread
  * kernels and one velocity scaling to the NVE step.
  */
 int mlip_step_nvt(mlip_ctx *ctx, int n_steps, double dt_fs, int rebuild_every, double t_target_K, double t_damp_fs,
@@ -215,6 +222,18 @@ int mlip_get_rebuilds(const mlip_ctx *ctx, int64_t *n_builds_host);
 
 /* Positions / velocities in the caller's order (dev [N][3] double, may be NULL); step counter (host). */
 int mlip_get_state(mlip_ctx *ctx, double *pos, double *vel, int64_t *step_host, void *stream);
+/*
+ * The inverse of mlip_get_state + mlip_get_thermostat, for checkpoint / resume: positions (as mlip_set_positions: the
+ * lists are kept), velocities (dev [N][3] double, caller's order; either may be NULL = unchanged), the running step
+ * counter (it decides when fixed-interval rebuilds fall), and the thermostat state (host [3] each, NULL = unchanged).
+ * To resume on a fresh context: mlip_create, mlip_build_neighbors with the saved positions, then mlip_set_state with
+ * pos = NULL.  With force_mode = 1 the continued trajectory is bit-identical to the uninterrupted one provided the
+ * state was saved right after a step on which the lists were rebuilt (the resumed context builds its lists from the
+ * saved positions; between rebuilds the original run's lists were built from earlier positions, hold the pairs in
+ * another order, and the fp32 per-atom sums then round differently).
+ */
+int mlip_set_state(mlip_ctx *ctx, const double *pos, const double *vel, int64_t step, const double *v_eta_host,
+                   const double *eta_host, void *stream);
 /* Potential energy of the last evaluation and kinetic energy now (dev [1] each, may be NULL). */
 int mlip_get_energies(mlip_ctx *ctx, double *e_pot, double *e_kin, void *stream);
 
@@ -237,6 +256,23 @@ int mlip_kernel_time(mlip_ctx *ctx, int64_t *n_launches, double *total_ms, int r
  * record of mlip_kernel_time).  Any pointer may be NULL.
  */
 int mlip_get_timings(mlip_ctx *ctx, double *ms_build_host, double *ms_kernel_host, double *ms_integrate_host, int reset);
+
+/*
+ * Diagnostic: rebuild the lists at the current positions the way an in-step rebuild does (single traversal, no
+ * synchronisation, capacity as it stands) with the look-back wait of the offset scan limited to `spin_limit` polls and,
+ * if unpublished_tile >= 0, with that 64-atom tile withholding its look-back word.  Its successor's wait then runs out:
+ * the kernel must still finish, raise MLIP_ERR_NEIGHBOR_OVERFLOW in the status word and leave every list range inside
+ * the array.  The lists are unusable afterwards until the next mlip_build_neighbors.  For tests of the failure path only.
+ */
+int mlip_debug_rebuild(mlip_ctx *ctx, int spin_limit, int64_t unpublished_tile, void *stream);
+
+/*
+ * Measured fp32 fused-multiply-add rate of `device` in TFLOP/s (FMA = 2): a kernel of independent FMA chains on every SM,
+ * best of four timed launches (CUDA events, default stream; about 10 ms in all).  The fused kernel is bound by the fp32
+ * pipes (Section 3.4 discusses compute throughput, not bandwidth, as its limit), so reports quote its achieved rate
+ * against this number taken in the same process, next to the nominal lanes x clock figure.  Synchronises.
+ */
+int mlip_measure_fp32_peak(int device, double *tflops_host);
 
 size_t mlip_resident_bytes(const mlip_ctx *ctx);   /* device bytes the context holds */
 const char *mlip_last_error(const mlip_ctx *ctx);  /* text of the last failure (ctx may be NULL) */

@@ -23,8 +23,8 @@ ERRORS = {0: "MLIP_OK", 1: "MLIP_ERR_INVALID_ARG", 2: "MLIP_ERR_UNSUPPORTED", 3:
 CODES = {v: k for k, v in ERRORS.items()}
 
 EXPORTS = ["mlip_create", "mlip_table_error", "mlip_build_neighbors", "mlip_get_neighbors", "mlip_get_neighbors_noalloc", "mlip_set_positions",
-           "mlip_set_velocities", "mlip_compute", "mlip_compute_f64", "mlip_compute_host", "mlip_step", "mlip_step_nvt", "mlip_get_thermostat", "mlip_reset_thermostat", "mlip_get_rebuilds", "mlip_get_state",
-           "mlip_get_energies", "mlip_sync_status", "mlip_get_counters", "mlip_kernel_time", "mlip_get_timings",
+           "mlip_set_velocities", "mlip_compute", "mlip_compute_f64", "mlip_compute_host", "mlip_step", "mlip_step_nvt", "mlip_get_thermostat", "mlip_reset_thermostat", "mlip_get_rebuilds", "mlip_get_state", "mlip_set_state", "mlip_debug_rebuild",
+           "mlip_get_energies", "mlip_sync_status", "mlip_get_counters", "mlip_kernel_time", "mlip_get_timings", "mlip_measure_fp32_peak",
            "mlip_resident_bytes", "mlip_last_error", "mlip_destroy"]
 
 
@@ -110,8 +110,17 @@ def mlip_table_error(ctx):
     return a.value, b.value
 
 
+def _cell(box):
+    """Row-major cell vectors [9] from three edge lengths, nine numbers or a 3 x 3 matrix."""
+    box = np.asarray(box, dtype=np.float64)
+    if box.size == 3:
+        box = np.diag(box.ravel())
+    assert box.size == 9, "box: three edge lengths or the 3 x 3 cell vectors"
+    return np.ascontiguousarray(box.ravel())
+
+
 def mlip_build_neighbors(ctx, pos, species, box, stream=None):
-    box = np.ascontiguousarray(box, dtype=np.float64)
+    box = _cell(box)
     _check(ctx, lib().mlip_build_neighbors(ctx, ctypes.c_int64(pos.shape[0]), _dev(pos), _dev(species), _host(box), _stream(stream)))
 
 
@@ -152,7 +161,7 @@ def mlip_compute_f64(ctx, energy=None, forces=None, virial=None, e_atom=None, st
 
 def mlip_compute_host(ctx, pos, species, box, rebuild, forces_out, virial_out=None):
     e = ctypes.c_double(0)
-    box = None if box is None else np.ascontiguousarray(box, dtype=np.float64)
+    box = None if box is None else _cell(box)
     _check(ctx, lib().mlip_compute_host(ctx, ctypes.c_int64(pos.shape[0]), _host(pos), _host(species), _host(box),
                                         ctypes.c_int(int(rebuild)), ctypes.byref(e), _host(forces_out), _host(virial_out)))
     return e.value
@@ -197,6 +206,16 @@ def mlip_get_state(ctx, pos=None, vel=None, stream=None):
     return step.value
 
 
+def mlip_set_state(ctx, pos=None, vel=None, step=0, v_eta=None, eta=None, stream=None):
+    v_eta = None if v_eta is None else np.ascontiguousarray(v_eta, dtype=np.float64)
+    eta = None if eta is None else np.ascontiguousarray(eta, dtype=np.float64)
+    _check(ctx, lib().mlip_set_state(ctx, _dev(pos), _dev(vel), ctypes.c_int64(step), _host(v_eta), _host(eta), _stream(stream)))
+
+
+def mlip_debug_rebuild(ctx, spin_limit, unpublished_tile=-1, stream=None):
+    _check(ctx, lib().mlip_debug_rebuild(ctx, ctypes.c_int(spin_limit), ctypes.c_int64(unpublished_tile), _stream(stream)))
+
+
 def mlip_get_energies(ctx, e_pot=None, e_kin=None, stream=None):
     _check(ctx, lib().mlip_get_energies(ctx, _dev(e_pot), _dev(e_kin), _stream(stream)))
 
@@ -219,6 +238,15 @@ def mlip_kernel_time(ctx, reset=False):
     n, ms = ctypes.c_int64(0), ctypes.c_double(0)
     _check(ctx, lib().mlip_kernel_time(ctx, ctypes.byref(n), ctypes.byref(ms), ctypes.c_int(int(reset))))
     return n.value, ms.value
+
+
+def mlip_measure_fp32_peak(device=0) -> float:
+    """Measured fp32 FMA rate of the device in TFLOP/s."""
+    v = ctypes.c_double(0)
+    rc = lib().mlip_measure_fp32_peak(ctypes.c_int(device), ctypes.byref(v))
+    if rc != OK:
+        raise MlipError(rc, "fp32 peak measurement failed")
+    return v.value
 
 
 def mlip_resident_bytes(ctx):
@@ -320,6 +348,14 @@ class Potential:
         vel = t.empty((self.n, 3), dtype=t.float64, device=self.device)
         step = mlip_get_state(self.ctx, pos, vel)
         return pos, vel, step
+
+    def set_state(self, pos=None, vel=None, step=0, v_eta=None, eta=None):
+        t = self.torch
+        if pos is not None:
+            self._pos = t.as_tensor(pos, dtype=t.float64, device=self.device).contiguous()
+        if vel is not None:
+            self._vel = t.as_tensor(vel, dtype=t.float64, device=self.device).contiguous()
+        mlip_set_state(self.ctx, self._pos if pos is not None else None, self._vel if vel is not None else None, step, v_eta, eta)
 
     def energies(self):
         t = self.torch

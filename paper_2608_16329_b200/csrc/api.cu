@@ -95,6 +95,15 @@ static int ensure_capacity(mlip_ctx *c, int64_t n, int64_t n_cells) {
     return MLIP_OK;
 }
 
+// Row-major cell vectors -> edge lengths; only orthorhombic cells aligned with the axes are compiled in.
+static int box_edges(mlip_ctx *c, const double *cell, double *edges) {
+    for (int a = 0; a < 3; ++a)
+        for (int b = 0; b < 3; ++b)
+            if (a != b && cell[3 * a + b] != 0.0) return fail(c, MLIP_ERR_UNSUPPORTED, "triclinic cells are not supported: off-diagonal cell-vector components must be zero");
+    for (int a = 0; a < 3; ++a) edges[a] = cell[3 * a + a];
+    return MLIP_OK;
+}
+
 static int set_grid(mlip_ctx *c, const double *box) {
     const double rl = c->cfg.r_cut + c->cfg.skin;
     CellGrid g;
@@ -200,6 +209,7 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
         if ((rc = dev_alloc(c, &c->tile_counter, (size_t)MAX_SPECIES)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->species_start, (size_t)MAX_SPECIES + 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->stage_out, 10)) != MLIP_OK) break;
+        if ((rc = dev_alloc(c, &c->kin_part, 1184)) != MLIP_OK) break;
         if (cudaMallocHost((void **)&c->status_host, sizeof(int)) != cudaSuccess ||
             cudaMallocHost((void **)&c->total_host, sizeof(int64_t)) != cudaSuccess ||
             cudaMallocHost((void **)&c->rebuild_host, sizeof(int)) != cudaSuccess) {
@@ -247,8 +257,10 @@ int mlip_build_neighbors(mlip_ctx *c, int64_t n, const double *pos, const int32_
     cudaStream_t s = (cudaStream_t)stream;
     c->last_stream = s;
     cudaSetDevice(c->cfg.device);
-    int rc = set_grid(c, box);
+    double edges[3];
+    int rc = box_edges(c, box, edges);
     if (rc != MLIP_OK) return rc;
+    if ((rc = set_grid(c, edges)) != MLIP_OK) return rc;
     c->built = false;
     if ((rc = ensure_capacity(c, n, c->grid.n_cells)) != MLIP_OK) return rc;
     c->n = n;
@@ -269,6 +281,7 @@ int mlip_get_neighbors(mlip_ctx *c, int64_t *seg_ptr, int32_t *nbr, int64_t capa
     if (!c || !seg_ptr) return MLIP_ERR_INVALID_ARG;
     if (!c->built) return fail(c, MLIP_ERR_NOT_BUILT, "no neighbor lists yet");
     c->last_stream = (cudaStream_t)stream;
+    cudaSetDevice(c->cfg.device);
     return launch_export(c, seg_ptr, nbr, capacity, n_entries_host, (cudaStream_t)stream);
 }
 
@@ -415,9 +428,11 @@ int mlip_step_nvt(mlip_ctx *c, int n_steps, double dt, int rebuild_every, double
         if ((rc = evaluate(c, s)) != MLIP_OK) return rc;
         c->forces_current = true;
     }
-    if ((rc = launch_kinetic(c, s)) != MLIP_OK) return rc;
     for (int it = 0; it < n_steps; ++it) {
-        // thermostat half step; its velocity factor is applied inside the kick-drift kernel
+        // kinetic energy of the velocities as they stand (not the previous half step's rescaled value, so that a run does
+        // not depend on how it is split into calls), then the thermostat half step; its velocity factor is applied
+        // inside the kick-drift kernel
+        if ((rc = launch_kinetic(c, s)) != MLIP_OK) return rc;
         if ((rc = launch_nhc_half(c, c->nhc_nf, c->nhc_kT, c->nhc_q1, c->nhc_qk, dt, s)) != MLIP_OK) return rc;
         if ((rc = launch_kick_drift(c, dt, s, c->nhc + 6)) != MLIP_OK) return rc;
         c->step += 1;
@@ -457,6 +472,48 @@ int mlip_get_state(mlip_ctx *c, double *pos, double *vel, int64_t *step_host, vo
     if (step_host) *step_host = c->step;
     if (pos || vel) return launch_get_state(c, pos, vel, (cudaStream_t)stream);
     return MLIP_OK;
+}
+
+int mlip_set_state(mlip_ctx *c, const double *pos, const double *vel, int64_t step, const double *v_eta_host,
+                   const double *eta_host, void *stream) {
+    if (!c || step < 0) return MLIP_ERR_INVALID_ARG;
+    if (!c->built) return fail(c, MLIP_ERR_NOT_BUILT, "no atoms yet: build the lists from the saved positions first");
+    cudaStream_t s = (cudaStream_t)stream;
+    c->last_stream = s;
+    int rc;
+    if (pos) {
+        c->forces_current = false;
+        if ((rc = launch_set_positions(c, pos, s)) != MLIP_OK) return rc;
+    }
+    if (vel && (rc = launch_set_velocities(c, vel, s)) != MLIP_OK) return rc;
+    c->step = step;
+    if (v_eta_host || eta_host) {   // thermostat state {v_eta[3], eta[3]}
+        double st[6];
+        MLIP_CUDA_TRY(c, cudaStreamSynchronize(s));
+        MLIP_CUDA_TRY(c, cudaMemcpy(st, c->nhc, sizeof st, cudaMemcpyDeviceToHost));
+        if (v_eta_host) memcpy(st, v_eta_host, sizeof(double) * 3);
+        if (eta_host) memcpy(st + 3, eta_host, sizeof(double) * 3);
+        MLIP_CUDA_TRY(c, cudaMemcpy(c->nhc, st, sizeof st, cudaMemcpyHostToDevice));
+    }
+    return MLIP_OK;
+}
+
+int mlip_debug_rebuild(mlip_ctx *c, int spin_limit, int64_t unpublished_tile, void *stream) {
+    if (!c || spin_limit < 1) return MLIP_ERR_INVALID_ARG;
+    if (!c->built) return fail(c, MLIP_ERR_NOT_BUILT, "no neighbor lists yet");
+    cudaStream_t s = (cudaStream_t)stream;
+    c->last_stream = s;
+    c->lookback_spin_limit = spin_limit;
+    c->lookback_unpublished_tile = unpublished_tile;
+    std::swap(c->pos4, c->pos4_src);
+    std::swap(c->vel, c->vel_src);
+    std::swap(c->user_of, c->user_src);
+    int rc = launch_build(c, false, s);
+    c->lookback_spin_limit = 0;
+    c->lookback_unpublished_tile = -1;
+    c->n_builds += 1;
+    c->forces_current = false;
+    return rc;
 }
 
 int mlip_get_rebuilds(const mlip_ctx *c, int64_t *n_builds_host) {
@@ -576,7 +633,7 @@ void mlip_destroy(mlip_ctx *c) {
     cudaFree(c->head_w_d); cudaFree(c->table_d);
     cudaFree(c->acc); cudaFree(c->pair_counter); cudaFree(c->status); cudaFree(c->rebuild_flag); cudaFree(c->nhc); cudaFree(c->acc_fx); cudaFree(c->tile_ticket); cudaFree(c->tile_counter);
     cudaFree(c->species_start); cudaFree(c->stage_pos); cudaFree(c->stage_species); cudaFree(c->stage_force);
-    cudaFree(c->stage_out);
+    cudaFree(c->stage_out); cudaFree(c->kin_part);
     if (c->status_host) cudaFreeHost(c->status_host);
     if (c->total_host) cudaFreeHost(c->total_host);
     if (c->rebuild_host) cudaFreeHost(c->rebuild_host);

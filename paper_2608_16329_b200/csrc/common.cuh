@@ -106,11 +106,14 @@ struct mlip_ctx {
     int64_t *scan_tmp = nullptr;   // block sums for the scans
     int64_t scan_tmp_cap = 0;
     double *acc = nullptr;         // [ACC_COUNT]
+    double *kin_part = nullptr;    // [1184] per-block kinetic-energy sums (integrate.cu)
     unsigned long long *pair_counter = nullptr;
     int *status = nullptr;         // device status word
     int *rebuild_flag = nullptr;   // set when an atom has moved beyond the rebuild trigger; pinned copy in rebuild_host
     int *rebuild_host = nullptr;
     int64_t n_builds = 0;
+    int lookback_spin_limit = 0;              // polls before a look-back wait of the one-pass list build gives up (0 = default)
+    long long lookback_unpublished_tile = -1; // diagnostic list builds only (mlip_debug_rebuild)
     int *tile_counter = nullptr;   // [MAX_SPECIES] dynamic tile scheduler, one counter per central species
     int *status_host = nullptr;    // pinned
     int64_t *total_host = nullptr; // pinned

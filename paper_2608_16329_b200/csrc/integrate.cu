@@ -91,8 +91,11 @@ __global__ void k_scale_velocities(int64_t n3, double *__restrict__ vel, const d
     if (i < n3) vel[i] *= *scale;
 }
 
+// Kinetic energy in two steps with a fixed summation order (grid-stride partial sums per block, then one warp adds the
+// block sums in index order), so that the thermostat -- and with it an NVT trajectory -- is bit-reproducible.
+constexpr int KIN_BLOCKS = 1184;
 __global__ void k_kinetic(int64_t n, const double *__restrict__ mass, const double4 *__restrict__ pos4,
-                          const double *__restrict__ vel, double *acc) {
+                          const double *__restrict__ vel, double *__restrict__ block_sum) {
     __shared__ double part[32];
     double e = 0.0;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
@@ -105,8 +108,14 @@ __global__ void k_kinetic(int64_t n, const double *__restrict__ mass, const doub
     if (threadIdx.x < 32) {
         e = threadIdx.x < (blockDim.x >> 5) ? part[threadIdx.x] : 0.0;
         for (int o = 16; o; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
-        if (threadIdx.x == 0) atomicAdd(&acc[ACC_KINETIC], e / ACC_UNIT);
+        if (threadIdx.x == 0) block_sum[blockIdx.x] = e;
     }
+}
+__global__ void k_kinetic_finish(int n_blocks, const double *__restrict__ block_sum, double *acc) {
+    double e = 0.0;
+    for (int b = threadIdx.x; b < n_blocks; b += 32) e += block_sum[b];
+    for (int o = 16; o; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
+    if (threadIdx.x == 0) acc[ACC_KINETIC] = e / ACC_UNIT;
 }
 
 __global__ void k_scatter_forces(int64_t n, const int32_t *__restrict__ user_of, const float4 *__restrict__ force,
@@ -204,11 +213,11 @@ int launch_scale_velocities(mlip_ctx *c, cudaStream_t s) {
     return MLIP_OK;
 }
 int launch_kinetic(mlip_ctx *c, cudaStream_t s) {
-    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->acc + ACC_KINETIC, 0, sizeof(double), s));
     int64_t blocks = nb(c->n);
-    if (blocks > 1184) blocks = 1184;
-    k_kinetic<<<(unsigned)blocks, 256, 0, s>>>(c->n, c->mass, c->pos4, c->vel, c->acc);
-    c->launches += 1;
+    if (blocks > KIN_BLOCKS) blocks = KIN_BLOCKS;
+    k_kinetic<<<(unsigned)blocks, 256, 0, s>>>(c->n, c->mass, c->pos4, c->vel, c->kin_part);
+    k_kinetic_finish<<<1, 32, 0, s>>>((int)blocks, c->kin_part, c->acc);
+    c->launches += 2;
     MLIP_CUDA_TRY(c, cudaGetLastError());
     return MLIP_OK;
 }

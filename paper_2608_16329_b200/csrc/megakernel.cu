@@ -735,6 +735,10 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
     float *hc = scr_all + NW * (SCR_WORDS + Q_WORDS + PF_WORDS);
     int *ctl = reinterpret_cast<int *>(hc + HC_WORDS);
     const int rows = k.tab.knots + 3;
+    // lists that an in-step rebuild could not complete (capacity, broken configuration) are not evaluated: the outputs
+    // stay at their cleared values and the status word tells the caller why (nothing in this kernel raises these bits,
+    // so every CTA takes the same decision)
+    if (*k.status & (FLAG_NEIGHBOR_OVERFLOW | FLAG_NONFINITE)) return;
 
     double e_sum = 0.0;
     float vir[9] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};

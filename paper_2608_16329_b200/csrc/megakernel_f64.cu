@@ -107,6 +107,9 @@ __global__ void __launch_bounds__(F64_TILE * 32, K <= 32 ? 2 : 1) k_mega_f64(F64
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
     const int C = k.n_species;
+    // lists that an in-step rebuild could not complete (capacity, broken configuration) are not evaluated: the outputs
+    // stay at their cleared values and the status word tells the caller why
+    if (*k.status & (FLAG_NEIGHBOR_OVERFLOW | FLAG_NONFINITE)) return;
     if (threadIdx.x <= C) s_start[threadIdx.x] = k.species_start[threadIdx.x];
     __syncthreads();
     int total_tiles = 0;

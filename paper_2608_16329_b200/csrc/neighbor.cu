@@ -50,13 +50,23 @@ __global__ void k_place(const int32_t *__restrict__ cell_of, int64_t n, const in
 }
 
 // One thread per cell: order the cell's atoms by (species, caller index) and count them per species.
+// A cell holding more than MAX_CELL_ATOMS atoms (a collapsed or diverged configuration: thousands of atoms in a cube of
+// one list radius) is not sorted -- the insertion sort is quadratic in one thread -- and raises FLAG_NONFINITE, which
+// makes the list kernels and the fused kernels that follow return at once.
+constexpr int MAX_CELL_ATOMS = 1024;
 __global__ void k_sort_cells(int n_cells, int n_species, const int32_t *__restrict__ cell_start,
                              int32_t *__restrict__ slot_src, const double4 *__restrict__ pos4_src,
-                             const int32_t *__restrict__ user_src, int32_t *__restrict__ bin_count) {
+                             const int32_t *__restrict__ user_src, int32_t *__restrict__ bin_count, int *status) {
     int c = blockIdx.x * blockDim.x + threadIdx.x;
     if (c >= n_cells) return;
     int beg = cell_start[c], end = cell_start[c + 1];
     int cnt[MAX_SPECIES] = {0};
+    if (end - beg > MAX_CELL_ATOMS) {
+        atomicOr(status, FLAG_NONFINITE);
+        for (int a = beg; a < end; ++a) cnt[(int)pos4_src[slot_src[a]].w]++;
+        for (int s = 0; s < n_species; ++s) bin_count[(int64_t)s * n_cells + c] = cnt[s];
+        return;
+    }
     for (int a = beg; a < end; ++a) {
         int src = slot_src[a];
         int sa = (int)pos4_src[src].w;
@@ -117,7 +127,7 @@ __global__ void __launch_bounds__(256) k_neighbors(int64_t n, CellGrid g, double
                                                    int64_t nbr_cap, int *status) {
     const int lane = threadIdx.x & 31;
     int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (i >= n) return;
+    if (i >= n || (*status & FLAG_NONFINITE)) return;   // a broken configuration is not traversed (see k_sort_cells)
     const double4 pi = pos4[i];
     // this lane's cell: offsets (ox, oy, oz) = (lane / 9, lane / 3 % 3, lane % 3); dimensions with fewer than
     // three cells list each cell once
@@ -220,7 +230,7 @@ __global__ void __launch_bounds__(256) k_neighbors_rel(int64_t n, CellGrid g, do
                                                        int32_t *__restrict__ nbr, int64_t nbr_cap, int *status) {
     const int lane = threadIdx.x & 31;
     int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (i >= n) return;
+    if (i >= n || (*status & FLAG_NONFINITE)) return;
     const double4 pi = pos4[i];
     const float4 ri = rel[i];
     int cb = 0, ce = 0;
@@ -293,7 +303,9 @@ __global__ void __launch_bounds__(256) k_neighbors_rel(int64_t n, CellGrid g, do
 // in shared memory while it counts, obtains the tile's list offset from a decoupled look-back scan over the tiles before
 // it (tile aggregate / inclusive prefix published in one 64-bit word, tiles handed out by a ticket so that every
 // predecessor belongs to a CTA that is already running), and then copies the lists out in full rows.  Offsets are the same exclusive prefix sums the two-pass build produces, so the lists are identical.
-// Every wait is bounded: after OP_SPIN polls the tile raises FLAG_NEIGHBOR_OVERFLOW, publishes what it has and goes on.
+// Every wait is bounded: after `spin_limit` polls (OP_SPIN in production) the tile raises FLAG_NEIGHBOR_OVERFLOW, publishes
+// what it has and goes on.  Offsets are clamped to the capacity and a list that crosses it is cut short, so whatever the
+// outcome every [nbr_off[i], nbr_off[i+1]) lies inside the array and holds atom indices.
 constexpr int OP_PER_WARP = 8;
 constexpr int OP_TILE = 8 * OP_PER_WARP;
 static_assert(OP_TILE == 64, "the in-tile scan handles two counts per lane of one warp");
@@ -374,7 +386,11 @@ constexpr int OP_BUF = 160;   // hits kept per atom in shared memory; a longer l
 __global__ void __launch_bounds__(256) k_neighbors_onepass(int64_t n, CellGrid g, double rl2, const double4 *__restrict__ pos4,
                                                            const float4 *__restrict__ rel, const int32_t *__restrict__ cell_start,
                                                            int64_t *__restrict__ nbr_off, int32_t *__restrict__ nbr, int64_t nbr_cap,
-                                                           int *status, unsigned long long *tile_state, int *ticket) {
+                                                           int *status, unsigned long long *tile_state, int *ticket,
+                                                           const int *global_status, int spin_limit, long long unpublished_tile) {
+    // `unpublished_tile` >= 0 (diagnostic builds of the lists only) names a tile that never publishes its look-back word,
+    // so that its successor's bounded wait can be seen to run out; -1 in production.
+    if (*global_status & FLAG_NONFINITE) return;   // a broken configuration is not traversed (see k_sort_cells)
     // look-back word: flag in the top two bits (0 empty, 1 tile aggregate, 2 inclusive prefix), value below
     constexpr unsigned long long OP_AGG = 1ull << 62, OP_INC = 2ull << 62, OP_VAL = (1ull << 62) - 1;
     extern __shared__ int32_t s_hits[];   // [OP_TILE][OP_BUF]
@@ -414,7 +430,7 @@ __global__ void __launch_bounds__(256) k_neighbors_onepass(int64_t n, CellGrid g
         volatile unsigned long long *state = tile_state;
         long long prefix = 0;
         if (tile > 0) {
-            if (lane == 0) state[tile] = OP_AGG | (unsigned long long)aggregate;
+            if (lane == 0 && tile != unpublished_tile) state[tile] = OP_AGG | (unsigned long long)aggregate;
             int64_t hi = tile - 1;
             int spins = 0;
             for (;;) {   // windows of 32 predecessors, nearest first
@@ -426,7 +442,7 @@ __global__ void __launch_bounds__(256) k_neighbors_onepass(int64_t n, CellGrid g
                 const int first_inc = inc ? __ffs(inc) - 1 : 32;
                 const unsigned need = first_inc >= 31 ? 0xffffffffu : ((2u << first_inc) - 1u);
                 if (empty & need) {   // a tile in the window has not published yet
-                    if (++spins > OP_SPIN) { if (lane == 0) atomicOr(status, FLAG_NEIGHBOR_OVERFLOW); break; }
+                    if (++spins > spin_limit) { if (lane == 0) atomicOr(status, FLAG_NEIGHBOR_OVERFLOW); break; }
                     __nanosleep(200);
                     continue;
                 }
@@ -439,14 +455,14 @@ __global__ void __launch_bounds__(256) k_neighbors_onepass(int64_t n, CellGrid g
             }
         }
         if (lane == 0) {
-            state[tile] = OP_INC | (unsigned long long)(prefix + aggregate);
+            if (tile != unpublished_tile) state[tile] = OP_INC | (unsigned long long)(prefix + aggregate);
             s_prefix = prefix;
             s_total = prefix + aggregate;
         }
     }
     __syncthreads();
     const long long tile_off = s_prefix;
-    if (first + OP_TILE >= n && threadIdx.x == 0) nbr_off[n] = s_total;   // the last tile closes the offsets
+    if (first + OP_TILE >= n && threadIdx.x == 0) nbr_off[n] = s_total < nbr_cap ? s_total : nbr_cap;   // the last tile closes the offsets
 
     // ---- write the lists: full rows from shared memory ----
     for (int a = 0; a < OP_PER_WARP; ++a) {
@@ -455,16 +471,18 @@ __global__ void __launch_bounds__(256) k_neighbors_onepass(int64_t n, CellGrid g
         if (i >= n) break;
         const long long off = tile_off + s_off[slot];
         const int cnt = s_cnt[slot];
-        if (lane == 0) nbr_off[i] = off;
+        int fit = cnt;   // entries of this list that the array still holds
         if (off + cnt > nbr_cap) {
             if (lane == 0) atomicOr(status, FLAG_NEIGHBOR_OVERFLOW);
-            continue;
+            fit = off < nbr_cap ? (int)(nbr_cap - off) : 0;
         }
+        if (lane == 0) nbr_off[i] = off < nbr_cap ? off : nbr_cap;
+        if (fit == 0) continue;
         if (cnt <= OP_BUF) {
             const int32_t *src = s_hits + slot * OP_BUF;
-            for (int e = lane; e < cnt; e += 32) nbr[off + e] = src[e];
+            for (int e = lane; e < fit; e += 32) nbr[off + e] = src[e];
         } else {
-            onepass_traverse(i, g, rl2, edge, rl2_lo, rl2_hi, pos4, rel, cell_start, lane, nbr + off, 0x7fffffff);
+            onepass_traverse(i, g, rl2, edge, rl2_lo, rl2_hi, pos4, rel, cell_start, lane, nbr + off, fit);
         }
     }
 }
@@ -515,6 +533,15 @@ int launch_pack_source(mlip_ctx *c, const double *pos, const int32_t *species, c
     return MLIP_OK;
 }
 
+// A synchronising build that met a non-finite or out-of-box position, a species out of range or an over-full cell: the
+// list kernels have not run, so there is nothing to size a list from.  Reports it now and clears the flag.
+static int refuse_broken_input(mlip_ctx *c, cudaStream_t s) {
+    timing_end(c->ev_build, c->build_count, s);
+    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->status, 0, sizeof(int), s));
+    c->err = "non-finite or out-of-box position, species out of range, or more than 1024 atoms in one cell";
+    return MLIP_ERR_NONFINITE;
+}
+
 // Sort (pos4_src, vel_src, user_src) into cell order and build the lists.
 int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
     timing_begin(c->ev_build, c->build_count, s);
@@ -529,7 +556,7 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
     // nbr_count doubles as the slot -> source map until the lists are counted
     int32_t *slot_src = c->nbr_count;
     k_place<<<blocks_for(n, 256), 256, 0, s>>>(c->cell_of, n, c->cell_start, c->cell_fill, slot_src);
-    k_sort_cells<<<blocks_for(g.n_cells, 128), 128, 0, s>>>(g.n_cells, C, c->cell_start, slot_src, c->pos4_src, c->user_src, c->bin_count);
+    k_sort_cells<<<blocks_for(g.n_cells, 128), 128, 0, s>>>(g.n_cells, C, c->cell_start, slot_src, c->pos4_src, c->user_src, c->bin_count, c->status);
     k_gather<<<blocks_for(n, 256), 256, 0, s>>>(n, slot_src, c->pos4_src, c->vel_src, c->user_src, c->pos4, c->vel, c->user_of, c->disp);
     exclusive_scan<int32_t, int32_t>(c->bin_count, c->bin_start, (int64_t)C * g.n_cells, c->scan_tmp, s);
     int nthreads_co = g.n_cells > C + 1 ? g.n_cells : C + 1;
@@ -548,7 +575,8 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
         rel_ready = true;
         int *flag = allow_sync_grow ? c->tile_ticket + 1 : c->status;
         k_neighbors_onepass<<<(unsigned)n_tiles, 256, sizeof(int32_t) * OP_TILE * OP_BUF, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_off, c->nbr, c->nbr_cap,
-                                                               flag, c->tile_state, c->tile_ticket);
+                                                               flag, c->tile_state, c->tile_ticket, c->status,
+                                                               c->lookback_spin_limit > 0 ? c->lookback_spin_limit : OP_SPIN, c->lookback_unpublished_tile);
         c->launches += 5 + 2 * 3 + 2;   // cell id, place, sort, gather, centre order; two scans; relative positions, lists
         MLIP_CUDA_TRY(c, cudaGetLastError());
         bool done = true;
@@ -556,8 +584,10 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
             int overflow = 0;
             MLIP_CUDA_TRY(c, cudaMemcpyAsync(c->total_host, c->nbr_off + n, sizeof(int64_t), cudaMemcpyDeviceToHost, s));
             MLIP_CUDA_TRY(c, cudaMemcpyAsync(&overflow, c->tile_ticket + 1, sizeof(int), cudaMemcpyDeviceToHost, s));
+            MLIP_CUDA_TRY(c, cudaMemcpyAsync(c->status_host, c->status, sizeof(int), cudaMemcpyDeviceToHost, s));
             MLIP_CUDA_TRY(c, cudaStreamSynchronize(s));
-            done = overflow == 0 && *c->total_host <= c->nbr_cap;
+            if (*c->status_host & FLAG_NONFINITE) return refuse_broken_input(c, s);
+            done = overflow == 0 && *c->total_host < c->nbr_cap;   // the kernel clamps the total to the capacity
             if (done) c->n_entries = *c->total_host;
         }
         if (done) {
@@ -576,7 +606,9 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
     MLIP_CUDA_TRY(c, cudaGetLastError());
     if (allow_sync_grow) {
         MLIP_CUDA_TRY(c, cudaMemcpyAsync(c->total_host, c->nbr_off + n, sizeof(int64_t), cudaMemcpyDeviceToHost, s));
+        MLIP_CUDA_TRY(c, cudaMemcpyAsync(c->status_host, c->status, sizeof(int), cudaMemcpyDeviceToHost, s));
         MLIP_CUDA_TRY(c, cudaStreamSynchronize(s));
+        if (*c->status_host & FLAG_NONFINITE) return refuse_broken_input(c, s);
         c->n_entries = *c->total_host;
         if (c->n_entries > c->nbr_cap) {
             int64_t want = c->n_entries + c->n_entries / 8 + 1024;
@@ -596,14 +628,29 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
     return MLIP_OK;
 }
 
+// The lists cannot be exported while the status word says that the last in-step rebuild did not complete them.
+static int lists_whole(mlip_ctx *c, cudaStream_t s) {
+    MLIP_CUDA_TRY(c, cudaMemcpyAsync(c->status_host, c->status, sizeof(int), cudaMemcpyDeviceToHost, s));
+    MLIP_CUDA_TRY(c, cudaStreamSynchronize(s));
+    if (*c->status_host & FLAG_NONFINITE) { c->err = "neighbor export: the configuration is broken (see mlip_sync_status)"; return MLIP_ERR_NONFINITE; }
+    if (*c->status_host & FLAG_NEIGHBOR_OVERFLOW) { c->err = "neighbor export: the last rebuild overflowed the list (see mlip_sync_status)"; return MLIP_ERR_NEIGHBOR_OVERFLOW; }
+    return MLIP_OK;
+}
+
 int launch_export(mlip_ctx *c, int64_t *seg_ptr, int32_t *nbr, int64_t capacity, int64_t *n_entries_host, cudaStream_t s) {
     const int64_t n = c->n;
     const int C = c->cfg.n_species;
-    // seg counts live temporarily in the bin_count-sized scratch? They need N*C ints: use a fresh buffer.
+    int whole = lists_whole(c, s);
+    if (whole != MLIP_OK) return whole;
     int32_t *seg_count = nullptr;
     MLIP_CUDA_TRY(c, cudaMalloc(&seg_count, sizeof(int32_t) * (size_t)(n * C + 1)));
     int64_t *tmp = nullptr;
-    MLIP_CUDA_TRY(c, cudaMalloc(&tmp, sizeof(int64_t) * (size_t)scan_tmp_items(n * C)));
+    if (cudaMalloc(&tmp, sizeof(int64_t) * (size_t)scan_tmp_items(n * C)) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(seg_count);
+        c->err = "neighbor export: cudaMalloc of the scan scratch failed";
+        return MLIP_ERR_OOM;
+    }
     k_export_count<<<blocks_for(n * 32, 256), 256, 0, s>>>(n, C, c->nbr_off, c->nbr, c->pos4, c->user_of, seg_count);
     exclusive_scan<int32_t, int64_t>(seg_count, seg_ptr, n * C, tmp, s);
     int rc = MLIP_OK;
@@ -646,7 +693,8 @@ static __device__ __align__(256) unsigned char g_export_scratch[NOALLOC_BYTES];
 
 // In host code `g_export_scratch` is only a handle for the runtime, not a device address; the
 // address a kernel may use comes from cudaGetSymbolAddress, asked once per device with that device
-// current.  Slot d caches device d's answer.
+// current.  Slot d caches device d's answer.  The cache is plain host state: fill it from one host thread at a time,
+// and a cudaDeviceReset() of that device invalidates the cached address (the library is not meant to outlive one).
 static void *g_export_scratch_addr[64] = {nullptr};
 
 static int export_scratch_for_current_device(mlip_ctx *c, void **out) {
@@ -674,8 +722,9 @@ int launch_export_noalloc(mlip_ctx *c, int64_t *seg_ptr, int32_t *nbr, int64_t c
         return MLIP_ERR_UNSUPPORTED;
     }
     void *base = nullptr;
-    int rc = export_scratch_for_current_device(c, &base);
+    int rc = lists_whole(c, s);
     if (rc != MLIP_OK) return rc;
+    if ((rc = export_scratch_for_current_device(c, &base)) != MLIP_OK) return rc;
     int32_t *seg_count = reinterpret_cast<int32_t *>(base);
     int64_t *tmp = reinterpret_cast<int64_t *>(static_cast<unsigned char *>(base) + NOALLOC_COUNT_BYTES);
     k_export_count<<<blocks_for(n * 32, 256), 256, 0, s>>>(n, C, c->nbr_off, c->nbr, c->pos4, c->user_of, seg_count);

@@ -60,3 +60,63 @@ def test_reference_arm_prints_one_json_line_with_the_contract_keys():
                 "dtype", "data", "config", "cpu_baseline", "e2e"):
         assert key in line
     assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle" and line["value"] > 0
+
+
+def _args(*flags):
+    import sys
+    import bench
+    old = sys.argv
+    sys.argv = ["bench.py"] + list(flags)
+    try:
+        return bench.parse_args()
+    finally:
+        sys.argv = old
+
+
+def test_every_flag_combination_sets_up_its_problem_without_a_gpu():
+    """Workload, weights (of the shape the flags ask for) and the work per unit for each mode the benchmark offers."""
+    import bench
+    import workloads as wl
+    for precision in ("f32", "f64"):
+        for k, lmax in [(32, 3), (16, 3), (64, 3), (32, 1), (32, 2)]:
+            for extra in ([], ["--deterministic"], ["--ensemble", "nvt"]):
+                args = _args("--cells", "4", "--precision", precision, "--k", str(k), "--lmax", str(lmax), *extra)
+                prob = bench.problem_setup(args)
+                w = prob["w"]
+                assert w.n_atoms == 256 and prob["enc"].size == 36 * wl.enc_net_size(k)
+                assert prob["head"].size == 6 * wl.head_net_size((lmax + 1) * k)
+                assert prob["flop_pair"] > 0 and prob["flop_atom"] > 0
+                if (k, lmax) == (32, 3):
+                    assert prob["flop_pair"] == bench.FLOP_PER_PAIR and prob["flop_atom"] == bench.FLOP_PER_ATOM
+    # the general count reduces to the default one at the default shape
+    d, n_inv = 16, 128
+    assert abs((60 + 150 + 512 + 6 * d * 32 + 168) - bench.FLOP_PER_PAIR) < 5
+    assert abs((3 * d * 32 + 4 * (n_inv * 64 + 3 * 64 * 64) + 256 + 5000) - bench.FLOP_PER_ATOM) < 1e-3 * bench.FLOP_PER_ATOM
+
+
+def test_sample_blocks_interior_atoms_have_their_whole_neighborhood_in_the_sample():
+    import numpy as np
+    import bench
+    import oracle
+    import workloads as wl
+    w = wl.make_workload(5, n_cells=12)
+    rows, inner = bench.sample_blocks((12, 12, 12), 4, 3.6, w.r_cut, 4 * 8 * 8 * 12)
+    assert rows.size == 4 * 8 * 8 * 12 and 0 < inner.size < rows.size and np.isin(inner, rows).all()
+    nl = oracle.neighbors(w.pos, w.species, w.n_species, w.box, w.r_cut, rows=inner)
+    assert np.isin(nl.nbr, rows).all()
+    # other lattices of the workload table
+    for cfg, (cells, n_basis, a) in bench.LATTICES.items():
+        r, i = bench.sample_blocks(cells, n_basis, a, 6.0, 49152)
+        assert r.max() < np.prod(cells) * n_basis and r.size <= 49152 + 8 * 8 * 24 * n_basis
+
+
+def test_traffic_record_is_tied_to_the_kernel_sources(tmp_path, monkeypatch):
+    import bench
+    rec = tmp_path / "t.txt"
+    monkeypatch.setattr(bench, "TRAFFIC_RECORD", str(rec))
+    assert bench.recorded_traffic()[0] is None
+    rec.write_text(f"# comment\nkernel_revision: {bench.kernel_revision()}\ndram_bytes_per_atom: 700.5\n")
+    assert bench.recorded_traffic()[0] == 700.5
+    rec.write_text("kernel_revision: 0123456789abcdef\ndram_bytes_per_atom: 700.5\n")
+    value, why = bench.recorded_traffic()
+    assert value is None and "revision" in why

@@ -136,8 +136,17 @@ def test_device_side_problems_become_status_codes():
         pot.build_neighbors(w.pos, w.species, np.array([10.0, 30.0, 30.0]))
     assert err.value.code == C["MLIP_ERR_BOX_TOO_SMALL"]
     bad = w.pos.copy(); bad[5, 1] = np.nan
-    pot.build_neighbors(bad, w.species, w.box)
-    assert pot.sync_status(raise_on_error=False) == C["MLIP_ERR_NONFINITE"]
+    with pytest.raises(mlip.MlipError) as err:          # a synchronising build reports broken input at once
+        pot.build_neighbors(bad, w.species, w.box)
+    assert err.value.code == C["MLIP_ERR_NONFINITE"]
+    assert pot.sync_status(raise_on_error=False) == C["MLIP_OK"]
+    with pytest.raises(mlip.MlipError) as err:
+        pot.compute()
+    assert err.value.code == C["MLIP_ERR_NOT_BUILT"]
+    outside = w.pos.copy(); outside[9, 2] = w.box[2] + 0.5
+    with pytest.raises(mlip.MlipError) as err:
+        pot.build_neighbors(outside, w.species, w.box)
+    assert err.value.code == C["MLIP_ERR_NONFINITE"]
     pot.build_neighbors(w.pos, w.species, w.box)
     assert pot.sync_status(raise_on_error=False) == C["MLIP_OK"]
     moved = w.pos.copy(); moved[7] += 0.9; moved -= np.floor(moved / w.box) * w.box
