@@ -111,6 +111,37 @@ __device__ __forceinline__ float2 split_pair(float x) {
     return make_float2(__uint_as_float(hi), __uint_as_float(lo));
 }
 
+// Two-at-a-time variant for operands that feed forces only.  The tensor pipe reads the upper 19 bits of a TF32 operand
+// and ignores the rest, so the fp32 value itself serves as "hi" (= its truncation) and lo = x - trunc(x), taken for two
+// values by one packed subtract: 1.5 instructions per value instead of 2, at one bit less in the lo term.
+__device__ __forceinline__ float2 sub2(float2 a, float2 b) {
+    unsigned long long ra, rb, rd;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(rd) : "l"(ra), "l"(rb));
+    float2 d;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
+    return d;
+}
+__device__ __forceinline__ float2 add2(float2 a, float2 b) {
+    unsigned long long ra, rb, rd;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(rd) : "l"(ra), "l"(rb));
+    float2 d;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
+    return d;
+}
+__device__ __forceinline__ void split2_force(float x, float y, uint32_t &xh, uint32_t &yh, uint32_t &xl, uint32_t &yl) {
+#ifdef MLIP_SPLIT_TRUNC
+    xh = __float_as_uint(x); yh = __float_as_uint(y);
+    const float2 lo = sub2(make_float2(x, y), make_float2(__uint_as_float(xh & 0xffffe000u), __uint_as_float(yh & 0xffffe000u)));
+    xl = __float_as_uint(lo.x); yl = __float_as_uint(lo.y);
+#else
+    split_tf32(x, xh, xl); split_tf32(y, yh, yl);
+#endif
+}
+
 __device__ __forceinline__ void mma_tf32(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
     asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
@@ -344,7 +375,15 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
 #pragma unroll
             for (int nt = 0; nt < 4; ++nt) mma_tf32(c[nt], ah[0], ah[1], ah[2], ah[3], bh[nt][0], bh[nt][1]);
 #pragma unroll
-            for (int nt = 0; nt < 4; ++nt) { Pf[nt][0] += c[nt][0]; Pf[nt][1] += c[nt][1]; Pf[nt][2] += c[nt][2]; Pf[nt][3] += c[nt][3]; }
+            for (int nt = 0; nt < 4; ++nt) {
+#ifdef MLIP_PACKED_ADD
+                const float2 s01 = add2(make_float2(Pf[nt][0], Pf[nt][1]), make_float2(c[nt][0], c[nt][1]));
+                const float2 s23 = add2(make_float2(Pf[nt][2], Pf[nt][3]), make_float2(c[nt][2], c[nt][3]));
+                Pf[nt][0] = s01.x; Pf[nt][1] = s01.y; Pf[nt][2] = s23.x; Pf[nt][3] = s23.y;
+#else
+                Pf[nt][0] += c[nt][0]; Pf[nt][1] += c[nt][1]; Pf[nt][2] += c[nt][2]; Pf[nt][3] += c[nt][3];
+#endif
+            }
         }
         __syncwarp();
         pc.mark(2);
@@ -429,10 +468,10 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) {
                 uint32_t ah[4], al[4], dh[4], dl[4];
-                split_tf32(G[0][ks], ah[0], al[0]);      split_tf32(G[1][ks], ah[1], al[1]);
-                split_tf32(G[0][4 + ks], ah[2], al[2]);  split_tf32(G[1][4 + ks], ah[3], al[3]);
-                split_tf32(dG[0][ks], dh[0], dl[0]);     split_tf32(dG[1][ks], dh[1], dl[1]);
-                split_tf32(dG[0][4 + ks], dh[2], dl[2]); split_tf32(dG[1][4 + ks], dh[3], dl[3]);
+                split2_force(G[0][ks], G[1][ks], ah[0], ah[1], al[0], al[1]);
+                split2_force(G[0][4 + ks], G[1][4 + ks], ah[2], ah[3], al[2], al[3]);
+                split2_force(dG[0][ks], dG[1][ks], dh[0], dh[1], dl[0], dl[1]);
+                split2_force(dG[0][4 + ks], dG[1][4 + ks], dh[2], dh[3], dl[2], dl[3]);
                 // Eq. 9 (rows of V: a = 0..7 and 8..15) and W g' (Eq. 8 re-associated); cross terms first, the
                 // four independent accumulators interleaved
                 if (ks == 0) {
@@ -549,8 +588,13 @@ __device__ __forceinline__ void head_gemm(float (&c)[4], const float4 (&w)[8], i
         float2 x0[4], x1[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            split_tf32(w[q + u].x, ah[u][0], al[u][0]); split_tf32(w[q + u].y, ah[u][1], al[u][1]);
-            split_tf32(w[q + u].z, ah[u][2], al[u][2]); split_tf32(w[q + u].w, ah[u][3], al[u][3]);
+            if (FRESH) {
+                split_tf32(w[q + u].x, ah[u][0], al[u][0]); split_tf32(w[q + u].y, ah[u][1], al[u][1]);
+                split_tf32(w[q + u].z, ah[u][2], al[u][2]); split_tf32(w[q + u].w, ah[u][3], al[u][3]);
+            } else {
+                split2_force(w[q + u].x, w[q + u].y, ah[u][0], ah[u][1], al[u][0], al[u][1]);
+                split2_force(w[q + u].z, w[q + u].w, ah[u][2], ah[u][3], al[u][2], al[u][3]);
+            }
             const float *r0 = act + g * bstride + 2 * (8 * (ks0 + q + u) + t);
             x0[u] = *reinterpret_cast<const float2 *>(r0);
             x1[u] = *reinterpret_cast<const float2 *>(r0 + 8);
