@@ -47,7 +47,7 @@ static void free_atoms(mlip_ctx *c) {
     dev_free(c, &c->user_of, n); dev_free(c, &c->user_src, n);
     dev_free(c, &c->force, n); dev_free(c, &c->disp, 3 * n); dev_free(c, &c->e_atom, n);
     dev_free(c, &c->center_order, n); dev_free(c, &c->cell_of, n);
-    dev_free(c, &c->nbr_count, n); dev_free(c, &c->nbr_off, n + 1);
+    dev_free(c, &c->nbr_count, n); dev_free(c, &c->nbr_near, n); dev_free(c, &c->nbr_off, n + 1);
     if (c->cfg.precision == 1) { dev_free(c, &c->force_d, 3 * n); dev_free(c, &c->e_atom_d, n); }
     if (c->cfg.force_mode == 1) dev_free(c, &c->force_fx, 3 * n);
     dev_free(c, &c->tile_state, n / 64 + 2);
@@ -72,7 +72,7 @@ static int ensure_capacity(mlip_ctx *c, int64_t n, int64_t n_cells) {
         TRY_ALLOC(c->user_of, m); TRY_ALLOC(c->user_src, m);
         TRY_ALLOC(c->force, m); TRY_ALLOC(c->disp, 3 * m); TRY_ALLOC(c->e_atom, m);
         TRY_ALLOC(c->center_order, m); TRY_ALLOC(c->cell_of, m);
-        TRY_ALLOC(c->nbr_count, m); TRY_ALLOC(c->nbr_off, m + 1);
+        TRY_ALLOC(c->nbr_count, m); TRY_ALLOC(c->nbr_near, m); TRY_ALLOC(c->nbr_off, m + 1);
         if (c->cfg.precision == 1) { TRY_ALLOC(c->force_d, 3 * m); TRY_ALLOC(c->e_atom_d, m); }
         if (c->cfg.force_mode == 1) TRY_ALLOC(c->force_fx, 3 * m);
         TRY_ALLOC(c->tile_state, m / 64 + 2);
@@ -203,6 +203,7 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
         if ((rc = dev_alloc(c, &c->pair_counter, 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->status, 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->rebuild_flag, 1)) != MLIP_OK) break;
+        if ((rc = dev_alloc(c, &c->far_flag, 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->nhc, 8)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->acc_fx, 10)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->tile_ticket, 2)) != MLIP_OK) break;   // ticket, private overflow flag
@@ -631,7 +632,7 @@ void mlip_destroy(mlip_ctx *c) {
     free_cells(c);
     cudaFree(c->nbr); cudaFree(c->scan_tmp); cudaFree(c->head_w); cudaFree(c->table); cudaFree(c->mass);
     cudaFree(c->head_w_d); cudaFree(c->table_d);
-    cudaFree(c->acc); cudaFree(c->pair_counter); cudaFree(c->status); cudaFree(c->rebuild_flag); cudaFree(c->nhc); cudaFree(c->acc_fx); cudaFree(c->tile_ticket); cudaFree(c->tile_counter);
+    cudaFree(c->acc); cudaFree(c->pair_counter); cudaFree(c->status); cudaFree(c->rebuild_flag); cudaFree(c->far_flag); cudaFree(c->nhc); cudaFree(c->acc_fx); cudaFree(c->tile_ticket); cudaFree(c->tile_counter);
     cudaFree(c->species_start); cudaFree(c->stage_pos); cudaFree(c->stage_species); cudaFree(c->stage_force);
     cudaFree(c->stage_out); cudaFree(c->kin_part);
     if (c->status_host) cudaFreeHost(c->status_host);

@@ -97,6 +97,8 @@ struct mlip_ctx {
     int32_t *species_start = nullptr;  // dev [C + 1]
     // lists
     int32_t *nbr_count = nullptr;  // [N]
+    int32_t *nbr_near = nullptr;   // [N] leading entries of each list that were within r_cut + skin / 2 at build time
+    int *far_flag = nullptr;       // raised once an atom has moved skin / 4 since the build: the far entries count again
     int64_t *nbr_off = nullptr;    // [N + 1]
     int32_t *nbr = nullptr;
     unsigned long long *tile_state = nullptr;   // [ceil(N / 64) + 1] look-back words of the one-pass rebuild

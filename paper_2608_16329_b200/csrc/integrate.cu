@@ -17,7 +17,7 @@ __device__ __forceinline__ double3 load_force(const float4 *__restrict__ force, 
 __global__ void k_kick_drift(int64_t n, double dt, CellGrid g, const double *__restrict__ mass, float skin_half2,
                              double4 *__restrict__ pos4, double *__restrict__ vel, const float4 *__restrict__ force,
                              const double *__restrict__ force_d, float *__restrict__ disp, int *status, float trigger2,
-                             int *rebuild_flag, const double *__restrict__ vscale) {
+                             int *rebuild_flag, const double *__restrict__ vscale, float far2, int *far_flag) {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     double4 p = pos4[i];
@@ -40,6 +40,7 @@ __global__ void k_kick_drift(int64_t n, double dt, CellGrid g, const double *__r
     }
     if (!(d2 <= skin_half2)) atomicOr(status, d2 == d2 ? FLAG_SKIN_EXCEEDED : FLAG_NONFINITE);
     if (d2 > trigger2) *rebuild_flag = 1;   // same value from every writer
+    if (!(d2 <= far2)) *far_flag = 1;       // from now on the lists' far entries may come inside r_cut
     pos4[i] = make_double4(x[0], x[1], x[2], p.w);
 }
 
@@ -138,7 +139,8 @@ __global__ void k_scatter_forces_f64(int64_t n, const int32_t *__restrict__ user
 }
 
 __global__ void k_set_positions(int64_t n, const int32_t *__restrict__ user_of, const double *__restrict__ pos,
-                                CellGrid g, float skin_half2, double4 *__restrict__ pos4, float *__restrict__ disp, int *status) {
+                                CellGrid g, float skin_half2, double4 *__restrict__ pos4, float *__restrict__ disp, int *status,
+                                float far2, int *far_flag) {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     const int64_t u = user_of[i];
@@ -156,6 +158,7 @@ __global__ void k_set_positions(int64_t n, const int32_t *__restrict__ user_of, 
     }
     if (!ok) atomicOr(status, FLAG_NONFINITE);
     else if (!(d2 <= skin_half2)) atomicOr(status, FLAG_SKIN_EXCEEDED);
+    if (!(d2 <= far2)) *far_flag = 1;
     pos4[i] = make_double4(x[0], x[1], x[2], p.w);
 }
 
@@ -178,11 +181,14 @@ __global__ void k_get_state(int64_t n, const int32_t *__restrict__ user_of, cons
 
 static inline unsigned nb(int64_t n) { return (unsigned)((n + 255) / 256); }
 static inline float skin_half2(const mlip_ctx *c) { float h = 0.5f * (float)c->cfg.skin; return h * h; }
+// Far entries lie beyond r_cut + skin / 2 at build time; a pair closes by at most twice the largest displacement, so they
+// stay outside r_cut while every atom has moved less than skin / 4 (0.245: room for the fp32 bookkeeping).
+static inline float far_trigger2(const mlip_ctx *c) { float h = 0.245f * (float)c->cfg.skin; return h * h; }
 
 int launch_kick_drift(mlip_ctx *c, double dt, cudaStream_t s, const double *vscale) {
     timing_begin(c->ev_integrate, c->integrate_count, s);
     k_kick_drift<<<nb(c->n), 256, 0, s>>>(c->n, dt, c->grid, c->mass, skin_half2(c), c->pos4, c->vel, c->force, c->force_d, c->disp, c->status,
-                                               0.64f * skin_half2(c), c->rebuild_flag, vscale);
+                                               0.64f * skin_half2(c), c->rebuild_flag, vscale, far_trigger2(c), c->far_flag);
     timing_end(c->ev_integrate, c->integrate_count, s);
     c->launches += 1;
     MLIP_CUDA_TRY(c, cudaGetLastError());
@@ -234,7 +240,7 @@ int launch_scatter_forces_f64(mlip_ctx *c, double *forces, double *e_atom, cudaS
     return MLIP_OK;
 }
 int launch_set_positions(mlip_ctx *c, const double *pos, cudaStream_t s) {
-    k_set_positions<<<nb(c->n), 256, 0, s>>>(c->n, c->user_of, pos, c->grid, skin_half2(c), c->pos4, c->disp, c->status);
+    k_set_positions<<<nb(c->n), 256, 0, s>>>(c->n, c->user_of, pos, c->grid, skin_half2(c), c->pos4, c->disp, c->status, far_trigger2(c), c->far_flag);
     c->launches += 1;
     MLIP_CUDA_TRY(c, cudaGetLastError());
     return MLIP_OK;

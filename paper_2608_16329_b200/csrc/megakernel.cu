@@ -133,13 +133,9 @@ __device__ __forceinline__ float2 add2(float2 a, float2 b) {
     return d;
 }
 __device__ __forceinline__ void split2_force(float x, float y, uint32_t &xh, uint32_t &yh, uint32_t &xl, uint32_t &yl) {
-#ifdef MLIP_SPLIT_TRUNC
     xh = __float_as_uint(x); yh = __float_as_uint(y);
     const float2 lo = sub2(make_float2(x, y), make_float2(__uint_as_float(xh & 0xffffe000u), __uint_as_float(yh & 0xffffe000u)));
     xl = __float_as_uint(lo.x); yl = __float_as_uint(lo.y);
-#else
-    split_tf32(x, xh, xl); split_tf32(y, yh, yl);
-#endif
 }
 
 __device__ __forceinline__ void mma_tf32(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
@@ -199,6 +195,8 @@ struct KernelArgs {
     const int32_t *center_order;
     const int32_t *species_start;
     const int64_t *nbr_off;
+    const int32_t *nbr_near;   // leading entries of each list that can be inside r_cut while far_flag is down
+    const int *far_flag;
     const int32_t *nbr;
     const float *head_pack;
     float4 *force;
@@ -234,8 +232,9 @@ struct TableView {
 // and advances `cur`.  The first n_pref indices of the list may come from shared memory (sidx).
 constexpr int SCAN_CHUNKS = 5;
 static_assert(SCAN_CHUNKS * 32 <= PB_CAP, "a full group must fit an empty queue");
-__device__ __forceinline__ int collect_pairs(const KernelArgs &k, const double4 &pi, int64_t beg, int64_t &cur, int64_t end, float4 *pq, int lane,
-                                             const int *sidx, int n_pref) {
+template <int SCAN_CHUNKS>
+__device__ __forceinline__ int collect_pairs_n(const KernelArgs &k, const double4 &pi, int64_t beg, int64_t &cur, int64_t end, float4 *pq, int lane,
+                                               const int *sidx, int n_pref) {
     int nq = 0;
     while (cur < end && nq + (int)min((int64_t)(SCAN_CHUNKS * 32), end - cur) <= PB_CAP) {
         int jj[SCAN_CHUNKS];
@@ -266,15 +265,23 @@ __device__ __forceinline__ int collect_pairs(const KernelArgs &k, const double4 
     __syncwarp();
     return nq;
 }
+// Short lists (the usual case while the far entries are skipped) take the three-chunk form: fewer loads in flight,
+// fewer registers.
+__device__ __forceinline__ int collect_pairs(const KernelArgs &k, const double4 &pi, int64_t beg, int64_t &cur, int64_t end, float4 *pq, int lane,
+                                             const int *sidx, int n_pref) {
+    if (end - beg <= 96) return collect_pairs_n<3>(k, pi, beg, cur, end, pq, lane, sidx, n_pref);
+    return collect_pairs_n<5>(k, pi, beg, cur, end, pq, lane, sidx, n_pref);
+}
 
 // ---------------- Encoding of one atom: returns the moment as accumulator fragments ----------------
 // `queued` returns the number of pairs left in the queue when the whole list fitted in one round
 // (the derivation then reuses them), or -1.
+template <bool TAB_SMEM>
 __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView &tv, const double4 &pi, int64_t beg, int64_t end,
                                            float4 *pq, float *stage, int lane, float (&Pf)[4][4], int &queued, const int *sidx, int n_pref,
                                            PhaseClock &pc) {
     const int g = lane >> 2, t = lane & 3;
-    const int rs = tv.row_stride;
+    constexpr int rs = TAB_SMEM ? TAB_STRIDE_SMEM : K_RADIAL;   // = tv.row_stride, known here so that row offsets fold into the loads
 #pragma unroll
     for (int a = 0; a < 4; ++a)
 #pragma unroll
@@ -376,13 +383,9 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
             for (int nt = 0; nt < 4; ++nt) mma_tf32(c[nt], ah[0], ah[1], ah[2], ah[3], bh[nt][0], bh[nt][1]);
 #pragma unroll
             for (int nt = 0; nt < 4; ++nt) {
-#ifdef MLIP_PACKED_ADD
                 const float2 s01 = add2(make_float2(Pf[nt][0], Pf[nt][1]), make_float2(c[nt][0], c[nt][1]));
                 const float2 s23 = add2(make_float2(Pf[nt][2], Pf[nt][3]), make_float2(c[nt][2], c[nt][3]));
                 Pf[nt][0] = s01.x; Pf[nt][1] = s01.y; Pf[nt][2] = s23.x; Pf[nt][3] = s23.y;
-#else
-                Pf[nt][0] += c[nt][0]; Pf[nt][1] += c[nt][1]; Pf[nt][2] += c[nt][2]; Pf[nt][3] += c[nt][3];
-#endif
             }
         }
         __syncwarp();
@@ -402,13 +405,13 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
 }
 
 // ---------------- Derivation of one atom (Eq. 8-10) ----------------
-template <bool DET>
+template <bool TAB_SMEM, bool DET>
 __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView &tv, int i,
                                             float4 *pq, float *scr, int queued, int lane, const uint32_t (&Wh)[4][4],
                                             const uint32_t (&Wl)[4][4], float (&vir)[9], PhaseClock &pc) {
     const int g = lane >> 2, t = lane & 3;
     float *bs = scr, *vt = scr + 32 * BS_STRIDE;
-    const int rs = tv.row_stride;
+    constexpr int rs = TAB_SMEM ? TAB_STRIDE_SMEM : K_RADIAL;
     float fx = 0.f, fy = 0.f, fz = 0.f;
 
     auto batch = [&](int first, int n) {
@@ -541,7 +544,7 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
     } else {   // rare: the list did not fit the queue; position and list bounds are fetched again rather than kept
                // in registers through the head
         const double4 pi = load_pos4(k.pos4 + i);
-        const int64_t beg = k.nbr_off[i], end = k.nbr_off[i + 1];
+        const int64_t beg = k.nbr_off[i], end = *k.far_flag ? k.nbr_off[i + 1] : beg + k.nbr_near[i];
         int64_t cur = beg;
         do {
             const int n = collect_pairs(k, pi, beg, cur, end, pq, lane, nullptr, 0);
@@ -561,25 +564,90 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
     }
 }
 
+// ---------------- Tensor memory (TMEM) as the home of the regression network's weights ----------------
+// The SM's 256 KB of tensor memory (128 lanes x 512 columns of 32 bits) is otherwise idle in this kernel (the
+// contractions are per-atom products too small for tcgen05.mma), and it is the one on-chip store large enough for a
+// species' head: 41 k weights in MMA-fragment order for the forward and the reverse pass, 27 k of them with their hi/lo
+// split already taken.  A warp reaches the 32 lanes of quarter (warp % 4); a "record" is one A fragment = 4 consecutive
+// columns (a0..a3 of each lane).  The four warps of a quarter are the two roles (m-tile = quarter, k-half 0 / 1) of
+// the two groups, so each role's region is written once per species (by group 0) and read by both groups.
+//   region of role kh: columns 256 kh + ...
+//     [  0,  32)  forward, first layer: 8 records as they are (split on the fly)
+//     [ 32, 128)  forward, hidden layers 2-4: per layer 4 records hi, then 4 records lo (rounded split: energy path)
+//     [128, 224)  reverse, hidden layers: per layer 4 records as they are, then 4 records lo of the truncating split
+//     [224, 256)  reverse, first layer: 8 records as they are
+// tcgen05.ld / st move 4, 16 or 32 consecutive columns between a thread's registers and its lane; they bypass the
+// L1/shared-memory data pipe, which is this kernel's busiest unit.
+constexpr uint32_t TM_COLS = 512;
+constexpr int TM_ROLE = 256, TM_FWD0 = 0, TM_FWD = 32, TM_BWD = 128, TM_BWD0 = 224;
+
+__device__ __forceinline__ void tmem_st4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&r)[32]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+                   "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+                   "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+                   "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// One warp of group 0 writes its role's region (wg = m-tile + 4 k-half) for the species whose packed weights start at hp.
+__device__ __forceinline__ void tmem_fill_role(uint32_t region, const float *__restrict__ hp, int wg, int lane) {
+    const float4 *fwd = reinterpret_cast<const float4 *>(hp + HP_FWD), *bwd = reinterpret_cast<const float4 *>(hp + HP_BWD);
+    const int mt4 = wg & 3, kh = wg >> 2;
+    auto as_is = [&](uint32_t col, const float4 *rec) {
+        const float4 v = __ldg(rec + lane);
+        tmem_st4(region + col, __float_as_uint(v.x), __float_as_uint(v.y), __float_as_uint(v.z), __float_as_uint(v.w));
+    };
+#pragma unroll 1
+    for (int q = 0; q < 8; ++q) {
+        as_is(TM_FWD0 + 4 * q, fwd + (size_t)(mt4 * KS0 + kh * 8 + q) * 32);
+        as_is(TM_BWD0 + 4 * q, bwd + (size_t)(wg * 8 + q) * 32);
+    }
+#pragma unroll 1
+    for (int b = 0; b < HEAD_L - 1; ++b)
+#pragma unroll 1
+        for (int q = 0; q < 4; ++q) {
+            {   // forward: hi, lo of the rounded split
+                const float4 v = __ldg(fwd + (size_t)(4 * KS0 + b * 4 * KS1 + mt4 * KS1 + kh * 4 + q) * 32 + lane);
+                uint32_t h[4], l[4];
+                split_tf32(v.x, h[0], l[0]); split_tf32(v.y, h[1], l[1]); split_tf32(v.z, h[2], l[2]); split_tf32(v.w, h[3], l[3]);
+                tmem_st4(region + TM_FWD + 32 * b + 4 * q, h[0], h[1], h[2], h[3]);
+                tmem_st4(region + TM_FWD + 32 * b + 16 + 4 * q, l[0], l[1], l[2], l[3]);
+            }
+            {   // reverse: the value itself (the tensor pipe truncates it), lo of the truncating split
+                const float4 v = __ldg(bwd + (size_t)((N_INV / 16) * 8 + b * 32 + mt4 * 8 + kh * 4 + q) * 32 + lane);
+                uint32_t h[4], l[4];
+                split2_force(v.x, v.y, h[0], h[1], l[0], l[1]);
+                split2_force(v.z, v.w, h[2], h[3], l[2], l[3]);
+                tmem_st4(region + TM_BWD + 32 * b + 4 * q, h[0], h[1], h[2], h[3]);
+                tmem_st4(region + TM_BWD + 32 * b + 16 + 4 * q, l[0], l[1], l[2], l[3]);
+            }
+        }
+    tmem_wait_st();
+}
+
 // Barrier among the 256 threads of one group (hardware barrier 1 + group).
 __device__ __forceinline__ void group_sync(int group) {
     asm volatile("bar.sync %0, %1;" ::"r"(group + 1), "r"(TILE * 32) : "memory");
 }
 
 // Head contraction on the tensor pipe: C^T[16 rows of W x 8 atoms] over NKS k-steps from ks0.
-// A records come from global memory (`head_load`, issued a pass ahead so that the L2 latency hides
-// behind the previous epilogue) and are split into hi + lo here; B = activations (hi, lo
-// interleaved) from shared memory with `bstride` floats per atom.
-template <int NKS>
-__device__ __forceinline__ void head_load(float4 (&w)[8], const float4 *__restrict__ rec, int ks0, int lane) {
-#pragma unroll
-    for (int q = 0; q < NKS; ++q) w[q] = __ldg(rec + (size_t)(ks0 + q) * 32 + lane);
-}
+// A records come from tensor memory (32 columns = 8 records as stored, or 4 records hi + 4 records lo when PRE);
+// B = activations (hi, lo interleaved) from shared memory with `bstride` floats per atom.
 // FRESH: every k-step gets its own accumulator, folded in by a rounded add (energy path);
 // otherwise one accumulation chain (reverse pass: feeds forces only).
-template <int NKS, bool FRESH>
-__device__ __forceinline__ void head_gemm(float (&c)[4], const float4 (&w)[8], int ks0, const float *__restrict__ act, int bstride, int lane) {
+template <int NKS, bool FRESH, bool PRE>
+__device__ __forceinline__ void head_gemm(float (&c)[4], const uint32_t (&wr)[32], int ks0, const float *__restrict__ act, int bstride, int lane) {
     static_assert(NKS % 4 == 0, "k-steps are processed four at a time (four independent MMA chains in flight)");
+    static_assert(!PRE || NKS == 4, "a pre-split load holds four records");
     const int g = lane >> 2, t = lane & 3;
     float acc[4][4];   // FRESH: per-k-step products; otherwise four accumulation chains
 #pragma unroll
@@ -588,16 +656,23 @@ __device__ __forceinline__ void head_gemm(float (&c)[4], const float4 (&w)[8], i
         float2 x0[4], x1[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            if (FRESH) {
-                split_tf32(w[q + u].x, ah[u][0], al[u][0]); split_tf32(w[q + u].y, ah[u][1], al[u][1]);
-                split_tf32(w[q + u].z, ah[u][2], al[u][2]); split_tf32(w[q + u].w, ah[u][3], al[u][3]);
-            } else {
-                split2_force(w[q + u].x, w[q + u].y, ah[u][0], ah[u][1], al[u][0], al[u][1]);
-                split2_force(w[q + u].z, w[q + u].w, ah[u][2], ah[u][3], al[u][2], al[u][3]);
-            }
             const float *r0 = act + g * bstride + 2 * (8 * (ks0 + q + u) + t);
             x0[u] = *reinterpret_cast<const float2 *>(r0);
             x1[u] = *reinterpret_cast<const float2 *>(r0 + 8);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int o = 4 * (q + u);
+            if (PRE) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) { ah[u][e] = wr[o + e]; al[u][e] = wr[16 + o + e]; }
+            } else if (FRESH) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) split_tf32(__uint_as_float(wr[o + e]), ah[u][e], al[u][e]);
+            } else {
+                split2_force(__uint_as_float(wr[o]), __uint_as_float(wr[o + 1]), ah[u][0], ah[u][1], al[u][0], al[u][1]);
+                split2_force(__uint_as_float(wr[o + 2]), __uint_as_float(wr[o + 3]), ah[u][2], ah[u][3], al[u][2], al[u][3]);
+            }
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
@@ -639,9 +714,12 @@ struct NextAtom {
     int *sidx;        // shared: neighbor indices
     int slot;         // position in center_order, or -1
     int i;
+    bool use_far;     // the lists' far entries have to be scanned as well
     int64_t beg, end;
     __device__ __forceinline__ void stage_a() { if (slot >= 0) i = __ldg(k->center_order + slot); }
-    __device__ __forceinline__ void stage_b() { if (slot >= 0) { beg = __ldg(k->nbr_off + i); end = __ldg(k->nbr_off + i + 1); } }
+    __device__ __forceinline__ void stage_b() {
+        if (slot >= 0) { beg = __ldg(k->nbr_off + i); end = use_far ? __ldg(k->nbr_off + i + 1) : beg + __ldg(k->nbr_near + i); }
+    }
     __device__ __forceinline__ void stage_c(int lane) {
         if (slot < 0) return;
         const int n = (int)min((int64_t)PF_IDX, end - beg);
@@ -662,16 +740,13 @@ struct NextAtom {
 // In: sX = invariants [atom][128].  Out: sX = dE/dG; per-atom energies written.
 // hc = biases [4][64], w_out [64], b_out of the species in shared memory.  wg = warp within the group.
 template <bool DET>
-__device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float *hb, const float *hc, int species, int count, int first,
+__device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float *hb, const float *hc, uint32_t tm_role, int count, int first,
                                           int group, int wg, int lane, double &e_sum, NextAtom &nx, PhaseClock &pc) {
-    const float *hp = k.head_pack + (size_t)species * HP_TOTAL;
-    const float4 *fwd = reinterpret_cast<const float4 *>(hp + HP_FWD), *bwd = reinterpret_cast<const float4 *>(hp + HP_BWD);
     float *xs = hb + HB_XS, *zs = hb + HB_ZS, *dp = hb + HB_DP, *part = hb + HB_PART;
     const int mt4 = wg & 3, kh = wg >> 2;   // forward / reverse hidden layers: 4 m-tiles x 2 k-halves
     const int atom = wg;                    // elementwise phases: warp = atom, lane = neuron (and neuron + 32)
-    float4 w[8];
+    uint32_t w[32];   // A records of the coming contraction, fetched from tensor memory just before it
 
-    head_load<KS0 / 2>(w, fwd + (size_t)(mt4 * KS0) * 32, kh * (KS0 / 2), lane);
     // split the invariants once
     for (int f = lane; f < N_INV; f += 32)
         *reinterpret_cast<float2 *>(xs + atom * 2 * X_STRIDE + 2 * f) = split_pair(sX[atom * X_STRIDE + f]);
@@ -689,13 +764,12 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
         const float *zin = zs + ((L + 1) & 1) * TILE * 2 * Z_STRIDE;
         float *zout = zs + (L & 1) * TILE * 2 * Z_STRIDE;
         float c[4];
-        if (L == 0) head_gemm<KS0 / 2, true>(c, w, kh * (KS0 / 2), xs, 2 * X_STRIDE, lane);
-        else head_gemm<KS1 / 2, true>(c, w, kh * (KS1 / 2), zin, 2 * Z_STRIDE, lane);
+        tmem_ld32(tm_role + (L == 0 ? TM_FWD0 : TM_FWD + 32 * (L - 1)), w);
+        tmem_wait_ld();
+        if (L == 0) head_gemm<KS0 / 2, true, false>(c, w, kh * (KS0 / 2), xs, 2 * X_STRIDE, lane);
+        else head_gemm<KS1 / 2, true, true>(c, w, kh * (KS1 / 2), zin, 2 * Z_STRIDE, lane);
         pc.mark(12);
         store_partial(c, part + kh * TILE * Z_STRIDE, Z_STRIDE, mt4, lane);
-        // weights of the next pass
-        if (L < HEAD_L - 1) head_load<KS1 / 2>(w, fwd + (size_t)(4 * KS0 + L * 4 * KS1 + mt4 * KS1) * 32, kh * (KS1 / 2), lane);
-        else head_load<4>(w, bwd + (size_t)((N_INV / 16) * 8 + (HEAD_L - 2) * 32 + mt4 * 8) * 32, kh * 4, lane);
         if (L == 0) nx.stage_b();
         if (L == 1) nx.stage_c(lane);
         pc.mark(13);
@@ -739,10 +813,10 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
 #pragma unroll
     for (int L = HEAD_L - 1; L >= 1; --L) {
         float c[4];
-        head_gemm<4, false>(c, w, kh * 4, dp, 2 * Z_STRIDE, lane);
+        tmem_ld32(tm_role + TM_BWD + 32 * (L - 1), w);
+        tmem_wait_ld();
+        head_gemm<4, false, true>(c, w, kh * 4, dp, 2 * Z_STRIDE, lane);
         store_partial(c, part + kh * TILE * Z_STRIDE, Z_STRIDE, mt4, lane);
-        if (L > 1) head_load<4>(w, bwd + (size_t)((N_INV / 16) * 8 + (L - 2) * 32 + mt4 * 8) * 32, kh * 4, lane);
-        else head_load<8>(w, bwd + (size_t)(wg * 8) * 32, 0, lane);   // first layer: warp = m-tile, all 8 k-steps
         group_sync(group);
         {
             const int n0 = 2 * lane;
@@ -757,7 +831,9 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
     }
     {   // first layer: dE/dG [128 x 8], warp = m-tile (16 inputs), written over the invariants
         float c[4];
-        head_gemm<8, false>(c, w, 0, dp, 2 * Z_STRIDE, lane);
+        tmem_ld32(tm_role + TM_BWD0, w);   // warp = m-tile, all 8 k-steps
+        tmem_wait_ld();
+        head_gemm<8, false, false>(c, w, 0, dp, 2 * Z_STRIDE, lane);
         store_partial(c, sX, X_STRIDE, wg, lane);
     }
     group_sync(group);
@@ -783,6 +859,18 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
     // stay at their cleared values and the status word tells the caller why (nothing in this kernel raises these bits,
     // so every CTA takes the same decision)
     if (*k.status & (FLAG_NEIGHBOR_OVERFLOW | FLAG_NONFINITE)) return;
+    const bool use_far = *k.far_flag != 0;   // an atom has moved skin / 4 since the build: every list entry counts
+
+    // all of tensor memory (this is the only CTA on the SM) for the head's weights
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(ctl + 4)), "r"(TM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tmem_fence_before_sync();
+    __syncthreads();
+    tmem_fence_after_sync();
+    const uint32_t tm_base = *reinterpret_cast<volatile uint32_t *>(ctl + 4);
+    const uint32_t tm_role = tm_base + ((uint32_t)(32 * (wg & 3)) << 16) + TM_ROLE * (wg >> 2);
 
     double e_sum = 0.0;
     float vir[9] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -809,7 +897,10 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
         }
         for (int idx = threadIdx.x; idx < HEAD_L * HEAD_H + HEAD_H + 1; idx += NW * 32)
             hc[idx] = __ldg(k.head_pack + (size_t)species * HP_TOTAL + HP_BIAS + idx);
+        if (group == 0) tmem_fill_role(tm_role, k.head_pack + (size_t)species * HP_TOTAL, wg, lane);
+        tmem_fence_before_sync();
         __syncthreads();
+        tmem_fence_after_sync();
 
         bool prefetched = false;   // this warp's atom of the coming tile sits in the prefetch buffer
         int look_ahead = -1;       // (group leader) the tile after the current one
@@ -843,10 +934,10 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
                     n_pref = min(PF_IDX, pf[PF_IDX + 3]);
                 } else {
                     i = __ldg(k.center_order + first + wg);
-                    beg = k.nbr_off[i]; end = k.nbr_off[i + 1];
+                    beg = k.nbr_off[i]; end = use_far ? k.nbr_off[i + 1] : beg + k.nbr_near[i];
                 }
                 pi = load_pos4(k.pos4 + i);
-                n_pairs += encode_atom(k, tv, pi, beg, end, pq, scr, lane, Pf, queued, pf, n_pref, pc);
+                n_pairs += encode_atom<TAB_SMEM>(k, tv, pi, beg, end, pq, scr, lane, Pf, queued, pf, n_pref, pc);
                 // Eq. 5 (C_l = I): this lane holds rows a = g, g + 8 of channels 8t + j; sum squares over the rows of a block
                 float part[4][8];
 #pragma unroll
@@ -883,8 +974,8 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
             NextAtom nx;
             nx.k = &k; nx.sidx = pf; nx.meta = pf + PF_IDX;
             nx.slot = (tile_next < n_tiles && s_beg + tile_next * TILE + wg < s_end) ? s_beg + tile_next * TILE + wg : -1;
-            nx.i = 0; nx.beg = 0; nx.end = 0;
-            head_tile<DET>(k, sX, hb, hc, species, count, first, group, wg, lane, e_sum, nx, pc);
+            nx.i = 0; nx.beg = 0; nx.end = 0; nx.use_far = use_far;
+            head_tile<DET>(k, sX, hb, hc, tm_role, count, first, group, wg, lane, e_sum, nx, pc);
             prefetched = nx.slot >= 0;
             pc.mark(9);
 
@@ -911,7 +1002,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
                     split_tf32(w2, Wh[ks][2], Wl[ks][2]);
                     split_tf32(w3, Wh[ks][3], Wl[ks][3]);
                 }
-                derive_atom<DET>(k, tv, i, pq, scr, queued, lane, Wh, Wl, vir, pc);
+                derive_atom<TAB_SMEM, DET>(k, tv, i, pq, scr, queued, lane, Wh, Wl, vir, pc);
                 if (DET) {   // fold this atom's virial in now: lane sums in a fixed order, then integers
 #pragma unroll
                     for (int q = 0; q < 9; ++q) {
@@ -944,6 +1035,9 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
         if (lane == 0) atomicAdd(&k.acc[ACC_ENERGY], e_sum);
     }
     if (lane == 0) atomicAdd(k.pair_counter, n_pairs);
+    tmem_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tm_base), "r"(TM_COLS) : "memory");
 }
 
 // ---------------- host side ----------------
@@ -1041,7 +1135,7 @@ int launch_megakernel(mlip_ctx *c, cudaStream_t s) {
     KernelArgs k;
     k.n = n; k.n_species = c->cfg.n_species; k.grid = c->grid; k.rc2 = c->cfg.r_cut * c->cfg.r_cut; k.tab = c->tab;
     k.pos4 = c->pos4; k.center_order = c->center_order; k.species_start = c->species_start;
-    k.nbr_off = c->nbr_off; k.nbr = c->nbr; k.head_pack = c->head_w; k.force = c->force; k.e_atom = c->e_atom;
+    k.nbr_off = c->nbr_off; k.nbr_near = c->nbr_near; k.far_flag = c->far_flag; k.nbr = c->nbr; k.head_pack = c->head_w; k.force = c->force; k.e_atom = c->e_atom;
     k.force_fx = c->force_fx; k.acc_fx = c->acc_fx;
     k.acc = c->acc; k.pair_counter = c->pair_counter; k.status = c->status; k.tile_counter = c->tile_counter;
     const int slot = (int)(c->ev_count % mlip_ctx::EV_POOL);

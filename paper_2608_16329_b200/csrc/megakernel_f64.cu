@@ -75,6 +75,8 @@ struct F64Args {
     const int32_t *center_order;
     const int32_t *species_start;
     const int64_t *nbr_off;
+    const int32_t *nbr_near;   // leading entries of each list that can be inside r_cut while far_flag is down
+    const int *far_flag;
     const int32_t *nbr;
     const double *head;
     double *force;      // [N][3]
@@ -110,6 +112,7 @@ __global__ void __launch_bounds__(F64_TILE * 32, K <= 32 ? 2 : 1) k_mega_f64(F64
     // lists that an in-step rebuild could not complete (capacity, broken configuration) are not evaluated: the outputs
     // stay at their cleared values and the status word tells the caller why
     if (*k.status & (FLAG_NEIGHBOR_OVERFLOW | FLAG_NONFINITE)) return;
+    const bool use_far = *k.far_flag != 0;   // an atom has moved skin / 4 since the build: every list entry counts
     if (threadIdx.x <= C) s_start[threadIdx.x] = k.species_start[threadIdx.x];
     __syncthreads();
     int total_tiles = 0;
@@ -133,7 +136,7 @@ __global__ void __launch_bounds__(F64_TILE * 32, K <= 32 ? 2 : 1) k_mega_f64(F64
         if (have) {
             i = k.center_order[slot];
             pi = k.pos4[i];
-            beg = k.nbr_off[i]; end = k.nbr_off[i + 1];
+            beg = k.nbr_off[i]; end = use_far ? k.nbr_off[i + 1] : beg + k.nbr_near[i];
         }
 
         // ---------------- Encoding: P = H^T G (Eq. 4), lane = channel ----------------
@@ -458,7 +461,7 @@ int launch_megakernel_f64(mlip_ctx *c, cudaStream_t s) {
     k.coef = c->table_d; k.knots = c->cfg.table_knots; k.r_min = c->cfg.table_r_min;
     k.inv_h = c->cfg.table_knots / (c->cfg.r_cut - c->cfg.table_r_min);
     k.pos4 = c->pos4; k.center_order = c->center_order; k.species_start = c->species_start;
-    k.nbr_off = c->nbr_off; k.nbr = c->nbr;
+    k.nbr_off = c->nbr_off; k.nbr_near = c->nbr_near; k.far_flag = c->far_flag; k.nbr = c->nbr;
     k.head = c->head_w_d; k.force = c->force_d; k.e_atom = c->e_atom_d; k.acc = c->acc;
     k.pair_counter = c->pair_counter; k.status = c->status;
     const int slot = (int)(c->ev_count % mlip_ctx::EV_POOL);

@@ -124,7 +124,7 @@ template <bool FILL>
 __global__ void __launch_bounds__(256) k_neighbors(int64_t n, CellGrid g, double rl2, const double4 *__restrict__ pos4,
                                                    const int32_t *__restrict__ cell_start, int32_t *__restrict__ nbr_count,
                                                    const int64_t *__restrict__ nbr_off, int32_t *__restrict__ nbr,
-                                                   int64_t nbr_cap, int *status) {
+                                                   int64_t nbr_cap, int *status, float near2, int32_t *__restrict__ nbr_near) {
     const int lane = threadIdx.x & 31;
     int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (i >= n || (*status & FLAG_NONFINITE)) return;   // a broken configuration is not traversed (see k_sort_cells)
@@ -156,12 +156,14 @@ __global__ void __launch_bounds__(256) k_neighbors(int64_t n, CellGrid g, double
     const float rl2_lo = (float)(rl2 * (1.0 - 1e-5)), rl2_hi = (float)(rl2 * (1.0 + 1e-5));
     int64_t off = 0;
     bool writable = true;
+    int total = 0;
     if (FILL) {
         off = nbr_off[i];
+        total = (int)(nbr_off[i + 1] - off);
         writable = nbr_off[i + 1] <= nbr_cap;
         if (!writable && lane == 0) atomicOr(status, FLAG_NEIGHBOR_OVERFLOW);
     }
-    int cnt = 0;
+    int cnt = 0, cn = 0;   // hits so far, near hits so far (near hits fill the list from the front, far hits from the back)
     int beg = __shfl_sync(0xffffffffu, cb, 0), end = __shfl_sync(0xffffffffu, ce, 0);
     double4 pj_next = make_double4(0.0, 0.0, 0.0, 0.0);
     if (beg + lane < end) pj_next = pos4[beg + lane];
@@ -177,6 +179,7 @@ __global__ void __launch_bounds__(256) k_neighbors(int64_t n, CellGrid g, double
             const int j = base + lane;
             if (base != cur_beg && j < cur_end) pj = pos4[j];
             bool hit = false;
+            float d2f = 0.f;
             if (j < cur_end && j != i) {
                 const double ex = __dsub_rn(pj.x, pi.x), ey = __dsub_rn(pj.y, pi.y), ez = __dsub_rn(pj.z, pi.z);
                 // fp32 screen: the squared distance to ~1e-6 relative decides every candidate that is not within
@@ -185,7 +188,7 @@ __global__ void __launch_bounds__(256) k_neighbors(int64_t n, CellGrid g, double
                 fx = fx > halff[0] ? boxf[0] - fx : fx;
                 fy = fy > halff[1] ? boxf[1] - fy : fy;
                 fz = fz > halff[2] ? boxf[2] - fz : fz;
-                const float d2f = fx * fx + fy * fy + fz * fz;
+                d2f = fx * fx + fy * fy + fz * fz;
                 if (d2f < rl2_lo) hit = true;
                 else if (d2f <= rl2_hi) {
                     const double dx = min_image(ex, g.box[0], g.half[0]);
@@ -195,12 +198,15 @@ __global__ void __launch_bounds__(256) k_neighbors(int64_t n, CellGrid g, double
                     hit = d2 < rl2;
                 }
             }
-            const unsigned m = __ballot_sync(0xffffffffu, hit);
-            if (FILL && hit && writable) nbr[off + cnt + __popc(m & ((1u << lane) - 1u))] = j;
+            const bool near = hit && d2f < near2;
+            const unsigned m = __ballot_sync(0xffffffffu, hit), mn = __ballot_sync(0xffffffffu, near), below = (1u << lane) - 1u;
+            if (FILL && hit && writable)
+                nbr[off + (near ? cn + __popc(mn & below) : total - 1 - (cnt - cn + __popc(m & ~mn & below)))] = j;
             cnt += __popc(m);
+            cn += __popc(mn);
         }
     }
-    if (!FILL && lane == 0) nbr_count[i] = cnt;
+    if (!FILL && lane == 0) { nbr_count[i] = cnt; nbr_near[i] = cn; }
 }
 
 // Positions relative to the lower corner of the atom's own cell, in fp32 (|x_rel| < cell edge, so the rounding is ~5e-7
@@ -227,7 +233,8 @@ template <bool FILL>
 __global__ void __launch_bounds__(256) k_neighbors_rel(int64_t n, CellGrid g, double rl2, const double4 *__restrict__ pos4,
                                                        const float4 *__restrict__ rel, const int32_t *__restrict__ cell_start,
                                                        int32_t *__restrict__ nbr_count, const int64_t *__restrict__ nbr_off,
-                                                       int32_t *__restrict__ nbr, int64_t nbr_cap, int *status) {
+                                                       int32_t *__restrict__ nbr, int64_t nbr_cap, int *status, float near2,
+                                                       int32_t *__restrict__ nbr_near) {
     const int lane = threadIdx.x & 31;
     int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (i >= n || (*status & FLAG_NONFINITE)) return;
@@ -251,12 +258,14 @@ __global__ void __launch_bounds__(256) k_neighbors_rel(int64_t n, CellGrid g, do
     const float rl2_lo = (float)(rl2 * (1.0 - 1e-5)), rl2_hi = (float)(rl2 * (1.0 + 1e-5));
     int64_t off = 0;
     bool writable = true;
+    int total = 0;
     if (FILL) {
         off = nbr_off[i];
+        total = (int)(nbr_off[i + 1] - off);
         writable = nbr_off[i + 1] <= nbr_cap;
         if (!writable && lane == 0) atomicOr(status, FLAG_NEIGHBOR_OVERFLOW);
     }
-    int cnt = 0;
+    int cnt = 0, cn = 0;
     int beg = __shfl_sync(0xffffffffu, cb, 0), end = __shfl_sync(0xffffffffu, ce, 0);
     float4 rj_next = make_float4(0.f, 0.f, 0.f, 0.f);
     if (beg + lane < end) rj_next = rel[beg + lane];
@@ -277,9 +286,10 @@ __global__ void __launch_bounds__(256) k_neighbors_rel(int64_t n, CellGrid g, do
             const int j = base + lane;
             if (base != cur_beg && j < cur_end) rj = rel[j];
             bool hit = false;
+            float d2f = 0.f;
             if (j < cur_end && j != i) {
                 const float dx = rj.x + sx, dy = rj.y + sy, dz = rj.z + sz;
-                const float d2f = dx * dx + dy * dy + dz * dz;
+                d2f = dx * dx + dy * dy + dz * dz;
                 if (d2f < rl2_lo) hit = true;
                 else if (d2f <= rl2_hi) {
                     const double4 pj = pos4[j];
@@ -290,12 +300,15 @@ __global__ void __launch_bounds__(256) k_neighbors_rel(int64_t n, CellGrid g, do
                     hit = d2 < rl2;
                 }
             }
-            const unsigned m = __ballot_sync(0xffffffffu, hit);
-            if (FILL && hit && writable) nbr[off + cnt + __popc(m & ((1u << lane) - 1u))] = j;
+            const bool near = hit && d2f < near2;
+            const unsigned m = __ballot_sync(0xffffffffu, hit), mn = __ballot_sync(0xffffffffu, near), below = (1u << lane) - 1u;
+            if (FILL && hit && writable)
+                nbr[off + (near ? cn + __popc(mn & below) : total - 1 - (cnt - cn + __popc(m & ~mn & below)))] = j;
             cnt += __popc(m);
+            cn += __popc(mn);
         }
     }
-    if (!FILL && lane == 0) nbr_count[i] = cnt;
+    if (!FILL && lane == 0) { nbr_count[i] = cnt; nbr_near[i] = cn; }
 }
 
 // ---- one-pass variant for in-step rebuilds ----
@@ -312,9 +325,9 @@ static_assert(OP_TILE == 64, "the in-tile scan handles two counts per lane of on
 constexpr int OP_SPIN = 1 << 18;
 
 __device__ __forceinline__ bool rel_hit(const float4 &rj, float sx, float sy, float sz, float rl2_lo, float rl2_hi, double rl2,
-                                        const double4 &pi, const double4 *__restrict__ pos4, int j, const CellGrid &g) {
+                                        const double4 &pi, const double4 *__restrict__ pos4, int j, const CellGrid &g, float &d2f) {
     const float dx = rj.x + sx, dy = rj.y + sy, dz = rj.z + sz;
-    const float d2f = dx * dx + dy * dy + dz * dz;
+    d2f = dx * dx + dy * dy + dz * dz;
     if (d2f < rl2_lo) return true;
     if (d2f > rl2_hi) return false;
     const double4 pj = pos4[j];
@@ -343,16 +356,19 @@ __device__ __forceinline__ void cell_ranges(const double4 &p4, const CellGrid &g
     }
 }
 
-// One atom's traversal for the one-pass build: hits go to `out` (shared memory: the first `cap` of them; or global memory
-// with cap = INT_MAX); returns the number of hits.
+// One atom's traversal for the one-pass build.  Near hits (inside near2) go to out[0], out[1], ..., far hits to out[top],
+// out[top - 1], ...; only positions below `limit` are written.  Shared-memory pass: top = capacity - 1 (if the list is
+// longer than the buffer the two ends collide and the list is traversed again); global pass: top = list length - 1.
+// Returns the number of hits, and the number of near hits in `n_near`.
 __device__ __forceinline__ int onepass_traverse(int64_t i, const CellGrid &g, double rl2, const float (&edge)[3], float rl2_lo, float rl2_hi,
                                                 const double4 *__restrict__ pos4, const float4 *__restrict__ rel,
-                                                const int32_t *__restrict__ cell_start, int lane, int32_t *out, int cap) {
+                                                const int32_t *__restrict__ cell_start, int lane, int32_t *out, int top, int limit,
+                                                float near2, int &n_near) {
     const double4 pi = pos4[i];
     const float4 ri = rel[i];
     int cb, ce;
     cell_ranges(pi, g, cell_start, lane, cb, ce);
-    int cnt = 0;
+    int cnt = 0, cn = 0;
     int beg = __shfl_sync(0xffffffffu, cb, 0), end = __shfl_sync(0xffffffffu, ce, 0);
     float4 rj_next = make_float4(0.f, 0.f, 0.f, 0.f);
     if (beg + lane < end) rj_next = rel[beg + lane];
@@ -371,13 +387,17 @@ __device__ __forceinline__ int onepass_traverse(int64_t i, const CellGrid &g, do
         for (int base = cur_beg; base < cur_end; base += 32) {
             const int j = base + lane;
             if (base != cur_beg && j < cur_end) rj = rel[j];
-            const bool hit = j < cur_end && j != i && rel_hit(rj, sx, sy, sz, rl2_lo, rl2_hi, rl2, pi, pos4, j, g);
-            const unsigned m = __ballot_sync(0xffffffffu, hit);
-            const int slot = cnt + __popc(m & ((1u << lane) - 1u));
-            if (hit && slot < cap) out[slot] = j;
+            float d2f = 0.f;
+            const bool hit = j < cur_end && j != i && rel_hit(rj, sx, sy, sz, rl2_lo, rl2_hi, rl2, pi, pos4, j, g, d2f);
+            const bool near = hit && d2f < near2;
+            const unsigned m = __ballot_sync(0xffffffffu, hit), mn = __ballot_sync(0xffffffffu, near), below = (1u << lane) - 1u;
+            const int slot = near ? cn + __popc(mn & below) : top - (cnt - cn + __popc(m & ~mn & below));
+            if (hit && slot >= 0 && slot < limit) out[slot] = j;
             cnt += __popc(m);
+            cn += __popc(mn);
         }
     }
+    n_near = cn;
     return cnt;
 }
 
@@ -387,14 +407,15 @@ __global__ void __launch_bounds__(256) k_neighbors_onepass(int64_t n, CellGrid g
                                                            const float4 *__restrict__ rel, const int32_t *__restrict__ cell_start,
                                                            int64_t *__restrict__ nbr_off, int32_t *__restrict__ nbr, int64_t nbr_cap,
                                                            int *status, unsigned long long *tile_state, int *ticket,
-                                                           const int *global_status, int spin_limit, long long unpublished_tile) {
+                                                           const int *global_status, int spin_limit, long long unpublished_tile,
+                                                           float near2, int32_t *__restrict__ nbr_near) {
     // `unpublished_tile` >= 0 (diagnostic builds of the lists only) names a tile that never publishes its look-back word,
     // so that its successor's bounded wait can be seen to run out; -1 in production.
     if (*global_status & FLAG_NONFINITE) return;   // a broken configuration is not traversed (see k_sort_cells)
     // look-back word: flag in the top two bits (0 empty, 1 tile aggregate, 2 inclusive prefix), value below
     constexpr unsigned long long OP_AGG = 1ull << 62, OP_INC = 2ull << 62, OP_VAL = (1ull << 62) - 1;
     extern __shared__ int32_t s_hits[];   // [OP_TILE][OP_BUF]
-    __shared__ int s_cnt[OP_TILE];
+    __shared__ int s_cnt[OP_TILE], s_near[OP_TILE];
     __shared__ long long s_off[OP_TILE];
     __shared__ long long s_prefix, s_total;
     __shared__ int s_tile;
@@ -409,9 +430,9 @@ __global__ void __launch_bounds__(256) k_neighbors_onepass(int64_t n, CellGrid g
     for (int a = 0; a < OP_PER_WARP; ++a) {
         const int slot = warp * OP_PER_WARP + a;
         const int64_t i = first + slot;
-        int cnt = 0;
-        if (i < n) cnt = onepass_traverse(i, g, rl2, edge, rl2_lo, rl2_hi, pos4, rel, cell_start, lane, s_hits + slot * OP_BUF, OP_BUF);
-        if (lane == 0) s_cnt[slot] = cnt;
+        int cnt = 0, cn = 0;
+        if (i < n) cnt = onepass_traverse(i, g, rl2, edge, rl2_lo, rl2_hi, pos4, rel, cell_start, lane, s_hits + slot * OP_BUF, OP_BUF - 1, OP_BUF, near2, cn);
+        if (lane == 0) { s_cnt[slot] = cnt; s_near[slot] = cn; }
     }
     __syncthreads();
 
@@ -476,13 +497,15 @@ __global__ void __launch_bounds__(256) k_neighbors_onepass(int64_t n, CellGrid g
             if (lane == 0) atomicOr(status, FLAG_NEIGHBOR_OVERFLOW);
             fit = off < nbr_cap ? (int)(nbr_cap - off) : 0;
         }
-        if (lane == 0) nbr_off[i] = off < nbr_cap ? off : nbr_cap;
+        const int near = s_near[slot];
+        if (lane == 0) { nbr_off[i] = off < nbr_cap ? off : nbr_cap; nbr_near[i] = near < fit ? near : fit; }
         if (fit == 0) continue;
-        if (cnt <= OP_BUF) {
+        if (cnt <= OP_BUF) {   // near hits sit at the front of the buffer, far hits at its back
             const int32_t *src = s_hits + slot * OP_BUF;
-            for (int e = lane; e < fit; e += 32) nbr[off + e] = src[e];
+            for (int e = lane; e < fit; e += 32) nbr[off + e] = src[e < near ? e : e + (OP_BUF - cnt)];
         } else {
-            onepass_traverse(i, g, rl2, edge, rl2_lo, rl2_hi, pos4, rel, cell_start, lane, nbr + off, fit);
+            int cn;
+            onepass_traverse(i, g, rl2, edge, rl2_lo, rl2_hi, pos4, rel, cell_start, lane, nbr + off, cnt - 1, fit, near2, cn);
         }
     }
 }
@@ -549,6 +572,11 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
     const CellGrid &g = c->grid;
     const int C = c->cfg.n_species;
     const double rl = c->cfg.r_cut + c->cfg.skin;
+    // entries farther than r_cut + skin / 2 at build time form the back part of each list: they cannot come inside r_cut
+    // before some atom has moved skin / 4, and the fused kernels skip them until then (far_flag, raised by the integrator)
+    const double rn = c->cfg.r_cut + 0.5 * c->cfg.skin;
+    const float near2 = c->cfg.skin > 0.0 ? (float)(rn * rn * (1.0 + 1e-5)) : 3.0e38f;
+    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->far_flag, 0, sizeof(int), s));
     MLIP_CUDA_TRY(c, cudaMemsetAsync(c->cell_count, 0, sizeof(int32_t) * (g.n_cells + 1), s));
     MLIP_CUDA_TRY(c, cudaMemsetAsync(c->cell_fill, 0, sizeof(int32_t) * (g.n_cells + 1), s));
     k_cell_id<<<blocks_for(n, 256), 256, 0, s>>>(c->pos4_src, n, g, c->cell_of, c->cell_count, c->status);
@@ -576,7 +604,8 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
         int *flag = allow_sync_grow ? c->tile_ticket + 1 : c->status;
         k_neighbors_onepass<<<(unsigned)n_tiles, 256, sizeof(int32_t) * OP_TILE * OP_BUF, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_off, c->nbr, c->nbr_cap,
                                                                flag, c->tile_state, c->tile_ticket, c->status,
-                                                               c->lookback_spin_limit > 0 ? c->lookback_spin_limit : OP_SPIN, c->lookback_unpublished_tile);
+                                                               c->lookback_spin_limit > 0 ? c->lookback_spin_limit : OP_SPIN, c->lookback_unpublished_tile,
+                                                               near2, c->nbr_near);
         c->launches += 5 + 2 * 3 + 2;   // cell id, place, sort, gather, centre order; two scans; relative positions, lists
         MLIP_CUDA_TRY(c, cudaGetLastError());
         bool done = true;
@@ -597,10 +626,10 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
     }
     if (rel) {
         if (!rel_ready) k_rel_pos<<<blocks_for(n, 256), 256, 0, s>>>(n, g, c->pos4, relpos);
-        k_neighbors_rel<false><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_count, nullptr, nullptr, 0, c->status);
+        k_neighbors_rel<false><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_count, nullptr, nullptr, 0, c->status, near2, c->nbr_near);
         c->launches += 1;
     } else
-        k_neighbors<false><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, c->cell_start, c->nbr_count, nullptr, nullptr, 0, c->status);
+        k_neighbors<false><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, c->cell_start, c->nbr_count, nullptr, nullptr, 0, c->status, near2, c->nbr_near);
     exclusive_scan<int32_t, int64_t>(c->nbr_count, c->nbr_off, n, c->scan_tmp, s);
     c->launches += 5 + 1 + 3 * 3;   // cell id, place, sort, gather, centre order; count; three scans
     MLIP_CUDA_TRY(c, cudaGetLastError());
@@ -619,9 +648,9 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
         }
     }
     if (rel)
-        k_neighbors_rel<true><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_count, c->nbr_off, c->nbr, c->nbr_cap, c->status);
+        k_neighbors_rel<true><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_count, c->nbr_off, c->nbr, c->nbr_cap, c->status, near2, c->nbr_near);
     else
-        k_neighbors<true><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, c->cell_start, c->nbr_count, c->nbr_off, c->nbr, c->nbr_cap, c->status);
+        k_neighbors<true><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, c->cell_start, c->nbr_count, c->nbr_off, c->nbr, c->nbr_cap, c->status, near2, c->nbr_near);
     c->launches += 1;
     timing_end(c->ev_build, c->build_count, s);
     MLIP_CUDA_TRY(c, cudaGetLastError());

@@ -27,39 +27,40 @@ __device__ __forceinline__ void harmonics(T x, T y, T z, T *h) {
     h[15] = is10 * z * (T(2) * zz - T(3) * xx - T(3) * yy);
 }
 
-// s = sum_a h_a t_a,  (tx,ty,tz) = sum_a v_a grad h_a,  tu = sum_a l_a v_a h_a  (Euler: grad h_a . u = l_a h_a).
+// s = sum_a h_a t_a,  (tx,ty,tz) = sum_a v_a grad h_a,  tu = sum_a l_a v_a h_a.
+// The gradient is taken of the polynomial Phi(u) = sum_a v_a h_a(u): its quadratic and cubic parts are written out in
+// monomial coefficients (a fixed linear map of v), which costs fewer operations than seven separate gradients, and
+// tu = u . grad Phi by Euler's theorem for homogeneous polynomials (grad h_a . u = l_a h_a).  (x, y, z) is a unit vector;
+// the values h_a in s use x^2 + y^2 + z^2 = 1 where that shortens them.
 template <typename T>
 __device__ __forceinline__ void harmonics_project(T x, T y, T z, const T *v, const T *t, T &s, T &tx, T &ty, T &tz, T &tu) {
     const T s2 = T(1.4142135623730951), is2 = T(0.7071067811865476), is6 = T(0.4082482904638631);
     const T s6 = T(2.449489742783178), s15 = T(1.224744871391589), is10 = T(0.31622776601683794);
-    T xx = x * x, yy = y * y, zz = z * z, h;
-    s = t[0]; tx = ty = tz = T(0); tu = T(0);
-    s += x * t[1] + y * t[2] + z * t[3];
-    tx += v[1]; ty += v[2]; tz += v[3];
-    tu += x * v[1] + y * v[2] + z * v[3];
-    T u2 = T(0);
-    h = s2 * x * y; s += h * t[4]; u2 += h * v[4]; tx += s2 * y * v[4]; ty += s2 * x * v[4];
-    h = s2 * x * z; s += h * t[5]; u2 += h * v[5]; tx += s2 * z * v[5]; tz += s2 * x * v[5];
-    h = s2 * y * z; s += h * t[6]; u2 += h * v[6]; ty += s2 * z * v[6]; tz += s2 * y * v[6];
-    h = is2 * (xx - yy); s += h * t[7]; u2 += h * v[7]; tx += s2 * x * v[7]; ty -= s2 * y * v[7];
-    h = is6 * (T(2) * zz - xx - yy); s += h * t[8]; u2 += h * v[8];
-    tx -= T(2) * is6 * x * v[8]; ty -= T(2) * is6 * y * v[8]; tz += T(4) * is6 * z * v[8];
-    T u3 = T(0);
-    h = s6 * x * y * z; s += h * t[9]; u3 += h * v[9];
-    tx += s6 * y * z * v[9]; ty += s6 * x * z * v[9]; tz += s6 * x * y * v[9];
-    h = s15 * z * (xx - yy); s += h * t[10]; u3 += h * v[10];
-    tx += T(2) * s15 * x * z * v[10]; ty -= T(2) * s15 * y * z * v[10]; tz += s15 * (xx - yy) * v[10];
-    h = s15 * x * (yy - zz); s += h * t[11]; u3 += h * v[11];
-    tx += s15 * (yy - zz) * v[11]; ty += T(2) * s15 * x * y * v[11]; tz -= T(2) * s15 * x * z * v[11];
-    h = s15 * y * (zz - xx); s += h * t[12]; u3 += h * v[12];
-    tx -= T(2) * s15 * x * y * v[12]; ty += s15 * (zz - xx) * v[12]; tz += T(2) * s15 * y * z * v[12];
-    h = is10 * x * (T(2) * xx - T(3) * yy - T(3) * zz); s += h * t[13]; u3 += h * v[13];
-    tx += is10 * (T(6) * xx - T(3) * yy - T(3) * zz) * v[13]; ty -= T(6) * is10 * x * y * v[13]; tz -= T(6) * is10 * x * z * v[13];
-    h = is10 * y * (T(2) * yy - T(3) * xx - T(3) * zz); s += h * t[14]; u3 += h * v[14];
-    tx -= T(6) * is10 * x * y * v[14]; ty += is10 * (T(6) * yy - T(3) * xx - T(3) * zz) * v[14]; tz -= T(6) * is10 * y * z * v[14];
-    h = is10 * z * (T(2) * zz - T(3) * xx - T(3) * yy); s += h * t[15]; u3 += h * v[15];
-    tx -= T(6) * is10 * x * z * v[15]; ty -= T(6) * is10 * y * z * v[15]; tz += is10 * (T(6) * zz - T(3) * xx - T(3) * yy) * v[15];
-    tu += T(2) * u2 + T(3) * u3;
+    const T xx = x * x, yy = y * y, zz = z * z, xy = x * y, xz = x * z, yz = y * z;
+    // ---- s: the harmonics' values against t
+    const T dxy = xx - yy, dyz = yy - zz, dzx = zz - xx;
+    T acc = t[0] + x * t[1] + y * t[2] + z * t[3];
+    acc += s2 * (xy * t[4] + xz * t[5] + yz * t[6]) + is2 * (dxy * t[7]) + is6 * ((T(3) * zz - T(1)) * t[8]);
+    acc += s6 * (xy * (z * t[9])) + s15 * (z * dxy * t[10] + x * dyz * t[11] + y * dzx * t[12]);
+    acc += is10 * (x * (T(5) * xx - T(3)) * t[13] + y * (T(5) * yy - T(3)) * t[14] + z * (T(5) * zz - T(3)) * t[15]);
+    s = acc;
+    // ---- quadratic part: Phi_2 = (Bxx x^2 + Byy y^2 + Bzz z^2) / 2 + Axy xy + Axz xz + Ayz yz
+    const T axy = s2 * v[4], axz = s2 * v[5], ayz = s2 * v[6], w7 = s2 * v[7], w8 = (T(2) * is6) * v[8];
+    const T bxx = w7 - w8, byy = -w7 - w8, bzz = T(2) * w8;
+    T gx = v[1] + bxx * x + axy * y + axz * z;
+    T gy = v[2] + axy * x + byy * y + ayz * z;
+    T gz = v[3] + axz * x + ayz * y + bzz * z;
+    // ---- cubic part: Phi_3 = (2/3)(p13 x^3 + p14 y^3 + p15 z^3) + x (cxyy y^2 + cxzz z^2) + y (cyxx x^2 + cyzz z^2)
+    //                          + z (czxx x^2 + czyy y^2) + cxyz xyz,   p = 3 v / sqrt(10), q = sqrt(3/2) v
+    const T p13 = (T(3) * is10) * v[13], p14 = (T(3) * is10) * v[14], p15 = (T(3) * is10) * v[15];
+    const T q10 = s15 * v[10], q11 = s15 * v[11], q12 = s15 * v[12], cxyz = s6 * v[9];
+    const T cxyy = q11 - p13, cxzz = -q11 - p13, cyxx = -q12 - p14, cyzz = q12 - p14, czxx = q10 - p15, czyy = -q10 - p15;
+    const T x2 = x + x, y2 = y + y, z2 = z + z;
+    gx += p13 * (xx + xx) + cxyy * yy + cxzz * zz + x2 * (cyxx * y + czxx * z) + cxyz * yz;
+    gy += p14 * (yy + yy) + cyxx * xx + cyzz * zz + y2 * (cxyy * x + czyy * z) + cxyz * xz;
+    gz += p15 * (zz + zz) + czxx * xx + czyy * yy + z2 * (cxzz * x + cyzz * y) + cxyz * xy;
+    tx = gx; ty = gy; tz = gz;
+    tu = x * gx + y * gy + z * gz;
 }
 
 // Spline interval and cubic B-spline basis (and its r-derivative) at distance r for a table of
