@@ -132,6 +132,19 @@ __device__ __forceinline__ float2 add2(float2 a, float2 b) {
     asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
     return d;
 }
+// Rounded hi/lo split of two values in four packed fp32 operations (Veltkamp's splitting with the constant 2^13 + 1:
+// hi keeps 11 significant bits, rounded to nearest, so it is exact in TF32; lo = x - hi exactly).  Same result as
+// split_tf32 up to ties, but on the FMA pipe and two values at a time -- the conversion instruction expands into integer
+// operations on the half-rate pipe.  For the energy path, where the truncating split's bias would show.
+// The product is written as an explicit fused multiply-add with a zero addend: given a separate packed multiply, the
+// assembler contracts it with the subtraction that follows (even with .rn on both), which turns the split into hi = x.
+__device__ __forceinline__ void split2_rn(float x, float y, uint32_t &xh, uint32_t &yh, uint32_t &xl, uint32_t &yl) {
+    const float2 v = make_float2(x, y);
+    const float2 c = ffma2(v, make_float2(8193.f, 8193.f), make_float2(0.f, 0.f));
+    const float2 hi = sub2(c, sub2(c, v));
+    const float2 lo = sub2(v, hi);
+    xh = __float_as_uint(hi.x); yh = __float_as_uint(hi.y); xl = __float_as_uint(lo.x); yl = __float_as_uint(lo.y);
+}
 __device__ __forceinline__ void split2_force(float x, float y, uint32_t &xh, uint32_t &yh, uint32_t &xl, uint32_t &yl) {
     xh = __float_as_uint(x); yh = __float_as_uint(y);
     const float2 lo = sub2(make_float2(x, y), make_float2(__uint_as_float(xh & 0xffffe000u), __uint_as_float(yh & 0xffffe000u)));
@@ -317,15 +330,17 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
         __syncwarp();
         pc.mark(1);
         const int nks = (n + 7) >> 3;
-#pragma unroll 2
+#ifndef MLIP_KSTEP_UNROLL
+#define MLIP_KSTEP_UNROLL 4
+#endif
+        constexpr int kstep_unroll = MLIP_KSTEP_UNROLL;
+#pragma unroll kstep_unroll
         for (int ks = 0; ks < nks; ++ks) {
             // A = H^T (16 x 8 pairs): rows a = g, g + 8; columns pairs t, t + 4 of this k-step
             const float *ra = stage + (8 * ks + t) * ST_STRIDE, *rb = ra + 4 * ST_STRIDE;
             uint32_t ah[4], al[4];
-            split_tf32(ra[g], ah[0], al[0]);
-            split_tf32(ra[g + 8], ah[1], al[1]);
-            split_tf32(rb[g ^ 4], ah[2], al[2]);        // rows t + 4 are stored with their chunk pairs swapped
-            split_tf32(rb[(g ^ 4) + 8], ah[3], al[3]);
+            split2_rn(ra[g], ra[g + 8], ah[0], ah[1], al[0], al[1]);
+            split2_rn(rb[g ^ 4], rb[(g ^ 4) + 8], ah[2], ah[3], al[2], al[3]);   // rows t + 4 are stored with their chunk pairs swapped
             // B = G (8 pairs x 8 channels per n-tile).  Evaluation pattern: quarter-warp q reads the table
             // rows of ONE pair (8 lanes x 16 bytes = a full row per access: no bank conflicts), i.e. lane
             // (q, c) evaluates channels 4c .. 4c+3 of pairs q and q + 4 of this k-step; a fixed shuffle
@@ -371,10 +386,7 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
             uint32_t bh[4][2], bl[4][2];
             float c[4][4];
 #pragma unroll
-            for (int nt = 0; nt < 4; ++nt) {
-                split_tf32(ga[nt], bh[nt][0], bl[nt][0]);
-                split_tf32(gb[nt], bh[nt][1], bl[nt][1]);
-            }
+            for (int nt = 0; nt < 4; ++nt) split2_rn(ga[nt], gb[nt], bh[nt][0], bh[nt][1], bl[nt][0], bl[nt][1]);
 #pragma unroll
             for (int nt = 0; nt < 4; ++nt) mma_tf32_z(c[nt], al[0], al[1], al[2], al[3], bh[nt][0], bh[nt][1]);
 #pragma unroll
@@ -439,6 +451,11 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
         __syncwarp();
         pc.mark(4);
         const int nmt = (n + 15) >> 4;
+#ifndef MLIP_MTILE_UNROLL
+#define MLIP_MTILE_UNROLL 1
+#endif
+        constexpr int mtile_unroll = MLIP_MTILE_UNROLL;
+#pragma unroll mtile_unroll
         for (int mt = 0; mt < nmt; ++mt) {
             // A = [G; G'] (16 pairs x 32 channels): rows pairs g, g + 8; this lane evaluates channels 8t .. 8t+7
             // (one accumulator per output here: the truncating accumulation costs ~1e-6 relative on a
@@ -667,8 +684,8 @@ __device__ __forceinline__ void head_gemm(float (&c)[4], const uint32_t (&wr)[32
 #pragma unroll
                 for (int e = 0; e < 4; ++e) { ah[u][e] = wr[o + e]; al[u][e] = wr[16 + o + e]; }
             } else if (FRESH) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) split_tf32(__uint_as_float(wr[o + e]), ah[u][e], al[u][e]);
+                split2_rn(__uint_as_float(wr[o]), __uint_as_float(wr[o + 1]), ah[u][0], ah[u][1], al[u][0], al[u][1]);
+                split2_rn(__uint_as_float(wr[o + 2]), __uint_as_float(wr[o + 3]), ah[u][2], ah[u][3], al[u][2], al[u][3]);
             } else {
                 split2_force(__uint_as_float(wr[o]), __uint_as_float(wr[o + 1]), ah[u][0], ah[u][1], al[u][0], al[u][1]);
                 split2_force(__uint_as_float(wr[o + 2]), __uint_as_float(wr[o + 3]), ah[u][2], ah[u][3], al[u][2], al[u][3]);
@@ -748,8 +765,13 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
     uint32_t w[32];   // A records of the coming contraction, fetched from tensor memory just before it
 
     // split the invariants once
-    for (int f = lane; f < N_INV; f += 32)
-        *reinterpret_cast<float2 *>(xs + atom * 2 * X_STRIDE + 2 * f) = split_pair(sX[atom * X_STRIDE + f]);
+#pragma unroll
+    for (int f = lane; f < N_INV; f += 64) {
+        uint32_t h0, h1, l0, l1;
+        split2_rn(sX[atom * X_STRIDE + f], sX[atom * X_STRIDE + f + 32], h0, h1, l0, l1);
+        *reinterpret_cast<float2 *>(xs + atom * 2 * X_STRIDE + 2 * f) = make_float2(__uint_as_float(h0), __uint_as_float(l0));
+        *reinterpret_cast<float2 *>(xs + atom * 2 * X_STRIDE + 2 * (f + 32)) = make_float2(__uint_as_float(h1), __uint_as_float(l1));
+    }
     nx.stage_a();
     pc.mark(3);
     group_sync(group);
@@ -787,14 +809,16 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
             const float y0 = ya, y1 = yb;
             sdr[L] = make_float2(d0, d1);
             if (L < HEAD_L - 1) {
-                const float2 s0 = split_pair(y0), s1 = split_pair(y1);
-                *reinterpret_cast<float4 *>(zout + atom * 2 * Z_STRIDE + 2 * n0) = make_float4(s0.x, s0.y, s1.x, s1.y);
+                uint32_t h0, h1, l0, l1;
+                split2_rn(y0, y1, h0, h1, l0, l1);
+                *reinterpret_cast<uint4 *>(zout + atom * 2 * Z_STRIDE + 2 * n0) = make_uint4(h0, l0, h1, l1);
             } else {   // output layer and the start of the reverse pass: dE/dz = w_out
                 const float2 wo = *reinterpret_cast<const float2 *>(hc + HEAD_L * HEAD_H + n0);
                 e_i += wo.x * y0 + wo.y * y1;
                 dzn = wo;
-                const float2 s0 = split_pair(wo.x * d0), s1 = split_pair(wo.y * d1);
-                *reinterpret_cast<float4 *>(dp + atom * 2 * Z_STRIDE + 2 * n0) = make_float4(s0.x, s0.y, s1.x, s1.y);
+                uint32_t h0, h1, l0, l1;
+                split2_rn(wo.x * d0, wo.y * d1, h0, h1, l0, l1);
+                *reinterpret_cast<uint4 *>(dp + atom * 2 * Z_STRIDE + 2 * n0) = make_uint4(h0, l0, h1, l1);
             }
         }
         pc.mark(15);
@@ -824,8 +848,9 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
             const float2 p1 = *reinterpret_cast<const float2 *>(part + (TILE + atom) * Z_STRIDE + n0);
             dzn.x += p0.x + p1.x; dzn.y += p0.y + p1.y;
             const float2 da = sdr[L - 1];
-            const float2 s0 = split_pair(dzn.x * da.x), s1 = split_pair(dzn.y * da.y);
-            *reinterpret_cast<float4 *>(dp + atom * 2 * Z_STRIDE + 2 * n0) = make_float4(s0.x, s0.y, s1.x, s1.y);
+            uint32_t h0, h1, l0, l1;
+            split2_rn(dzn.x * da.x, dzn.y * da.y, h0, h1, l0, l1);
+            *reinterpret_cast<uint4 *>(dp + atom * 2 * Z_STRIDE + 2 * n0) = make_uint4(h0, l0, h1, l1);
         }
         group_sync(group);
     }
@@ -938,22 +963,25 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
                 }
                 pi = load_pos4(k.pos4 + i);
                 n_pairs += encode_atom<TAB_SMEM>(k, tv, pi, beg, end, pq, scr, lane, Pf, queued, pf, n_pref, pc);
-                // Eq. 5 (C_l = I): this lane holds rows a = g, g + 8 of channels 8t + j; sum squares over the rows of a block
+                // Eq. 5 (C_l = I): this lane holds rows a = g, g + 8 of channels 8t + j; sum squares over the rows of a block.
+                // Rows 1..3 (l = 1) and 4..7 (l = 2) differ in the top bit of g, so one two-step butterfly over the lower
+                // bits sums both; l = 2 then takes row 8 (held by g = 0) and the upper half's sum, l = 3 is rows 9..15.
                 float part[4][8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     const float pa = Pf[j & 3][j >> 2], pb = Pf[j & 3][2 + (j >> 2)];
-                    part[0][j] = g == 0 ? pa : 0.f;
-                    part[1][j] = (g >= 1 && g <= 3) ? pa * pa : 0.f;
-                    part[2][j] = (g >= 4 ? pa * pa : 0.f) + (g == 0 ? pb * pb : 0.f);
-                    part[3][j] = g >= 1 ? pb * pb : 0.f;
+                    float qa = g >= 1 ? pa * pa : 0.f, qb = g >= 1 ? pb * pb : 0.f;
+                    qa += __shfl_xor_sync(0xffffffffu, qa, 4);
+                    qb += __shfl_xor_sync(0xffffffffu, qb, 4);
+                    qa += __shfl_xor_sync(0xffffffffu, qa, 8);
+                    qb += __shfl_xor_sync(0xffffffffu, qb, 8);
+                    const float upper = __shfl_xor_sync(0xffffffffu, qa, 16);   // g = 0 receives the sum over g = 4..7
+                    qb += __shfl_xor_sync(0xffffffffu, qb, 16);
+                    part[0][j] = pa;                  // (the values below are those of the storing lanes, g = 0)
+                    part[1][j] = qa;
+                    part[2][j] = upper + pb * pb;
+                    part[3][j] = qb;
                 }
-#pragma unroll
-                for (int o = 4; o < 32; o <<= 1)
-#pragma unroll
-                    for (int l = 1; l < 4; ++l)   // l = 0 is a single row: the lane that stores it (g == 0) already holds it
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) part[l][j] += __shfl_xor_sync(0xffffffffu, part[l][j], o);
                 if (g == 0) {
 #pragma unroll
                     for (int l = 0; l < 4; ++l) {
@@ -997,10 +1025,8 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
                     const float w1 = g == 0 ? da[4 + ks] : 2.f * da[4 + ks] * Pf[ks][1];  // row a = g,     channel 8t + 4 + ks
                     const float w2 = 2.f * db[ks] * Pf[ks][2];                            // row a = g + 8, channel 8t + ks
                     const float w3 = 2.f * db[4 + ks] * Pf[ks][3];                        // row a = g + 8, channel 8t + 4 + ks
-                    split_tf32(w0, Wh[ks][0], Wl[ks][0]);
-                    split_tf32(w1, Wh[ks][1], Wl[ks][1]);
-                    split_tf32(w2, Wh[ks][2], Wl[ks][2]);
-                    split_tf32(w3, Wh[ks][3], Wl[ks][3]);
+                    split2_rn(w0, w1, Wh[ks][0], Wh[ks][1], Wl[ks][0], Wl[ks][1]);   // once per atom: the rounded split
+                    split2_rn(w2, w3, Wh[ks][2], Wh[ks][3], Wl[ks][2], Wl[ks][3]);
                 }
                 derive_atom<TAB_SMEM, DET>(k, tv, i, pq, scr, queued, lane, Wh, Wl, vir, pc);
                 if (DET) {   // fold this atom's virial in now: lane sums in a fixed order, then integers
