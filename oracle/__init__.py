@@ -39,7 +39,8 @@ class _CModel(ctypes.Structure):
                 ("head_hidden", ctypes.c_int), ("head_layers", ctypes.c_int),
                 ("r_cut", ctypes.c_double),
                 ("enc_w", ctypes.c_void_p), ("head_w", ctypes.c_void_p), ("q", ctypes.c_void_p),
-                ("chi_e", ctypes.c_int), ("chi_r", ctypes.c_int), ("envelope", ctypes.c_int)]
+                ("chi_e", ctypes.c_int), ("chi_r", ctypes.c_int), ("envelope", ctypes.c_int),
+                ("basis", ctypes.c_int), ("metric", ctypes.c_void_p)]
 
 
 _lib = None
@@ -79,20 +80,23 @@ class Model:
     chi_e: int = 0   # encoder conditioning (Section 3.2.2): 0 = species pair, C*C nets; 1 = neighbor species, C nets; 2 = none, 1 net
     chi_r: int = 0   # regression-network conditioning: 0 = central species, C nets; 1 = none, 1 net
     envelope: int = 0   # smooth cutoff: 0 = cosine, 1 = quintic polynomial 1 - 10 x^3 + 15 x^4 - 6 x^5
+    basis: int = 0      # angular basis (Section 3.3): 0 = irreducible harmonics (C_l = I), 1 = canonical monomials (C_l = multiplicities)
 
     def __post_init__(self):
         self.enc_w = np.ascontiguousarray(self.enc_w, dtype=np.float64)
         self.head_w = np.ascontiguousarray(self.head_w, dtype=np.float64)
         if self.q is None:
-            self.q = harmonic_projection.q_table(self.l_max)
+            self.q = harmonic_projection.canonical_table(self.l_max) if self.basis == 1 else harmonic_projection.q_table(self.l_max)
         self.q = np.ascontiguousarray(self.q, dtype=np.float64)
+        self.metric = np.ascontiguousarray(harmonic_projection.metric_diagonal(self.l_max, self.basis), dtype=np.float64)
         self._c = _CModel(self.n_species, self.k, self.l_max, self.enc_hidden, self.enc_layers,
                           self.head_hidden, self.head_layers, float(self.r_cut),
-                          _p(self.enc_w), _p(self.head_w), _p(self.q), self.chi_e, self.chi_r, self.envelope)
+                          _p(self.enc_w), _p(self.head_w), _p(self.q), self.chi_e, self.chi_r, self.envelope,
+                          self.basis, _p(self.metric))
 
     @property
     def d(self) -> int:
-        return (self.l_max + 1) ** 2
+        return harmonic_projection.reducible_dim(self.l_max) if self.basis == 1 else (self.l_max + 1) ** 2
 
     @property
     def n_inv(self) -> int:

@@ -79,3 +79,16 @@ def q_matrix(l: int) -> np.ndarray:
 def q_table(l_max: int) -> np.ndarray:
     """Q_0 .. Q_lmax flattened row-major and concatenated (the C core's input)."""
     return np.concatenate([q_matrix(l).ravel() for l in range(l_max + 1)])
+
+
+def canonical_table(l_max: int) -> np.ndarray:
+    """Identity blocks in place of Q_l: the canonical (reducible) basis keeps every degree-l monomial (Section 3.3)."""
+    return np.concatenate([np.eye(n_monomials(l)).ravel() for l in range(l_max + 1)])
+
+
+def metric_diagonal(l_max: int, basis: int) -> np.ndarray:
+    """Diagonal of C_0 .. C_lmax of Eq. 5: ones for the irreducible basis, the multinomial multiplicities
+    l! / (ax! ay! az!) for the canonical one."""
+    if basis == 0:
+        return np.ones(reduced_dim(l_max))
+    return np.concatenate([multinomial_metric(l) for l in range(l_max + 1)])

@@ -16,7 +16,8 @@
  *   angular feature h = Omega_lmax(r^)    Eq. 3, Sec. 3.3.1 (Q_l applied to the
  *                                          degree-l monomials) -> oracle_angular
  *   moment P_i = sum_j h (x) g            Eq. 4        -> oracle_center
- *   invariants G_i                        Eq. 5 (C_l = I, irreducible basis)
+ *   invariants G_i                        Eq. 5 (C_l = I for the irreducible basis; the canonical monomial basis of
+ *                                          Section 3.3, Eq. 11, with C_l = the multinomial multiplicities)
  *   energy E_i = R(G_i; s_i)              Eq. 6, Sec. 4.1.3 (4 hidden layers of
  *                                          64, SiLU, residual) -> oracle_head
  *   W_i, U_i, V_i                         Eq. 7-9
@@ -58,6 +59,10 @@ typedef struct {
                               1 = neighbor species s_j, C nets; 2 = none, one net */
     int chi_r;             /* ... to the regression network: 0 = central species s_i, C nets; 1 = none, one net */
     int envelope;          /* smooth cutoff (the paper names none): 0 = (1 + cos(pi x)) / 2, 1 = 1 - 10 x^3 + 15 x^4 - 6 x^5, x = r / r_c */
+    int basis;             /* angular basis (Section 3.3): 0 = irreducible, block l has 2l+1 rows Q_l m_l(u), C_l = I;
+                              1 = canonical, block l holds all C(l+2,2) monomials of degree l (q = identity blocks),
+                              C_l = diag(l! / (ax! ay! az!)), the "Cartesian multiplicities" of Eq. 5 */
+    const double *metric;  /* diagonal of C_0 .. C_lmax, one entry per row of the angular feature vector */
 } oracle_model;
 
 static int enc_net_index(const oracle_model *m, int si, int sj) {
@@ -68,7 +73,12 @@ static int enc_net_index(const oracle_model *m, int si, int sj) {
 static int head_net_index(const oracle_model *m, int si) { return m->chi_r == 1 ? 0 : si; }
 
 static int n_mono(int l) { return (l + 1) * (l + 2) / 2; }
-static int ang_dim(int l_max) { return (l_max + 1) * (l_max + 1); }
+static int blk_rows(const oracle_model *m, int l) { return m->basis == 1 ? n_mono(l) : 2 * l + 1; }
+static int ang_dim(const oracle_model *m) {
+    int d = 0;
+    for (int l = 0; l <= m->l_max; ++l) d += blk_rows(m, l);
+    return d;
+}
 
 static double ipow(double x, int n) { double p = 1.0; for (int i = 0; i < n; ++i) p *= x; return p; }
 
@@ -110,7 +120,7 @@ void oracle_angular(const oracle_model *m, const double u[3], double *h, double 
                 dmono[col][2] = az ? az * ipow(u[0], ax) * ipow(u[1], ay) * ipow(u[2], az - 1) : 0.0;
                 ++col;
             }
-        for (int r = 0; r < 2 * l + 1; ++r) {
+        for (int r = 0; r < blk_rows(m, l); ++r) {
             double s = 0.0, d0 = 0.0, d1 = 0.0, d2 = 0.0;
             for (int c = 0; c < nm; ++c) {
                 double qrc = q[r * nm + c];
@@ -124,8 +134,8 @@ void oracle_angular(const oracle_model *m, const double u[3], double *h, double 
             dh[(row0 + r) * 3 + 1] = d1;
             dh[(row0 + r) * 3 + 2] = d2;
         }
-        q += (2 * l + 1) * nm;
-        row0 += 2 * l + 1;
+        q += blk_rows(m, l) * nm;
+        row0 += blk_rows(m, l);
     }
 }
 
@@ -253,7 +263,7 @@ static double pair_geometry(const double *pos, const double *box, int64_t i, int
 static double oracle_center(const oracle_model *m, int64_t i, const double *pos, const int32_t *species,
                             const double *box, const int32_t *list, int64_t n_list,
                             double *G_out, double *f_out, double *rij_out) {
-    const int K = m->k, D = ang_dim(m->l_max), NG = (m->l_max + 1) * K;
+    const int K = m->k, D = ang_dim(m), NG = (m->l_max + 1) * K;
     const int si = species[i];
     const double rc2 = m->r_cut * m->r_cut;
     double P[D][K], G[NG], dG[NG], W[D][K];
@@ -271,11 +281,11 @@ static double oracle_center(const oracle_model *m, int64_t i, const double *pos,
             for (int c = 0; c < K; ++c) P[a][c] += h[a] * g[c];          /* Eq. 4 */
     }
     for (int c = 0; c < K; ++c) G[c] = P[0][c];                           /* Eq. 5, l = 0 */
-    for (int l = 1, row = 1; l <= m->l_max; row += 2 * l + 1, ++l)
+    for (int l = 1, row = 1; l <= m->l_max; row += blk_rows(m, l), ++l)
         for (int c = 0; c < K; ++c) {
             double s = 0.0;
-            for (int a = row; a < row + 2 * l + 1; ++a) s += P[a][c] * P[a][c];
-            G[l * K + c] = s;                                             /* Eq. 5, C_l = I */
+            for (int a = row; a < row + blk_rows(m, l); ++a) s += m->metric[a] * P[a][c] * P[a][c];
+            G[l * K + c] = s;                                             /* Eq. 5: p^T C_l p */
         }
     if (G_out) memcpy(G_out, G, sizeof G);
 
@@ -285,9 +295,9 @@ static double oracle_center(const oracle_model *m, int64_t i, const double *pos,
 
     /* Derivation: W = dE/dP (Eq. 7) */
     for (int c = 0; c < K; ++c) W[0][c] = dG[c];
-    for (int l = 1, row = 1; l <= m->l_max; row += 2 * l + 1, ++l)
-        for (int a = row; a < row + 2 * l + 1; ++a)
-            for (int c = 0; c < K; ++c) W[a][c] = 2.0 * dG[l * K + c] * P[a][c];
+    for (int l = 1, row = 1; l <= m->l_max; row += blk_rows(m, l), ++l)
+        for (int a = row; a < row + blk_rows(m, l); ++a)
+            for (int c = 0; c < K; ++c) W[a][c] = 2.0 * dG[l * K + c] * m->metric[a] * P[a][c];
 
     for (int64_t n = 0; n < n_list; ++n) {
         double d[3], d2 = pair_geometry(pos, box, i, list[n], d);

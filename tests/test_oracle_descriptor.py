@@ -206,3 +206,74 @@ def test_sampled_evaluation_equals_full_evaluation():
     s = oracle.sampled(m, w.pos, w.species, w.box, atoms)
     assert np.abs(s["e_atom"] - full["e_atom"][atoms]).max() < 1e-12
     assert np.abs(s["forces"] - full["forces"][atoms]).max() < 1e-11
+
+
+# ---- canonical (reducible) angular basis: all monomials of each degree, C_l = multinomial multiplicities (Section 3.3, Eq. 5)
+
+def test_canonical_basis_has_the_dimensions_of_eq_11_and_its_metric_is_the_multinomial_count():
+    from oracle import harmonic_projection as hp
+    enc, head = wl.make_weights(1, seed=2)
+    for l_max, d in [(0, 1), (1, 4), (2, 10), (3, 20), (4, 35), (5, 56)]:
+        assert hp.reducible_dim(l_max) == d
+        assert hp.metric_diagonal(l_max, 1).size == d
+    # (x + y + z)^l expands with exactly these multiplicities
+    for l in range(6):
+        assert hp.multinomial_metric(l).sum() == 3 ** l
+    m = oracle.Model(1, 6.0, enc, head, basis=1)
+    assert m.d == 20
+    h, dh = oracle.angular(m, np.array([0.6, 0.0, 0.8]))
+    # degree-2 block in the order x^2, xy, xz, y^2, yz, z^2 (the paper's example)
+    assert np.allclose(h[4:10], [0.36, 0.0, 0.48, 0.0, 0.0, 0.64])
+
+
+def test_canonical_invariants_are_sums_of_powers_of_the_cosine():
+    """With C_l = multiplicities, p^T C_l p = sum_jj' g_jk g_j'k (u_j . u_j')^l by the multinomial theorem."""
+    rng = np.random.default_rng(10)
+    enc, head = wl.make_weights(3, seed=3)
+    m = oracle.Model(3, 6.0, enc, head, basis=1)
+    pos, sp = _cluster(rng, 9, 3)
+    out = _all(m, pos, sp)
+    for i in range(9):
+        others = [j for j in range(9) if j != i and np.linalg.norm(pos[j] - pos[i]) < 6.0]
+        g = np.array([oracle.radial(m, sp[i], sp[j], np.linalg.norm(pos[j] - pos[i]))[0] for j in others])
+        u = np.array([(pos[j] - pos[i]) / np.linalg.norm(pos[j] - pos[i]) for j in others])
+        cos = u @ u.T
+        for l in range(4):
+            want = np.einsum("jk,jm,mk->k", g, cos ** l, g) if l else g.sum(0)
+            got = out["G"][i, l * 32:(l + 1) * 32]
+            assert np.abs(got - want).max() < 1e-11 * max(1.0, np.abs(want).max())
+
+
+def test_canonical_and_irreducible_invariants_differ_by_lower_orders():
+    """cos^2 = (cos^2 - 1/3) + 1/3 and cos^3 = (cos^3 - 3/5 cos) + 3/5 cos: the canonical order-2 invariant repeats the
+    scalar one (squared), the order-3 invariant repeats order 1 -- the redundancy the irreducible projection removes."""
+    rng = np.random.default_rng(11)
+    enc, head = wl.make_weights(2, seed=8)
+    pos, sp = _cluster(rng, 10, 2)
+    irr = _all(oracle.Model(2, 6.0, enc, head), pos, sp)["G"]
+    can = _all(oracle.Model(2, 6.0, enc, head, basis=1), pos, sp)["G"]
+    k = 32
+    assert np.allclose(can[:, :2 * k], irr[:, :2 * k], rtol=1e-12, atol=1e-12)
+    assert np.allclose(can[:, 2 * k:3 * k], irr[:, 2 * k:3 * k] + irr[:, :k] ** 2 / 3.0, rtol=1e-11, atol=1e-11)
+    assert np.allclose(can[:, 3 * k:], irr[:, 3 * k:] + 0.6 * irr[:, k:2 * k], rtol=1e-11, atol=1e-11)
+    assert np.abs(can[:, 2 * k:] - irr[:, 2 * k:]).max() > 1e-3          # the two descriptors really differ
+
+
+def test_canonical_forces_match_central_differences_and_energy_is_rotation_invariant():
+    rng = np.random.default_rng(12)
+    enc, head = wl.make_weights(2, seed=9, enc_out_scale=0.3)
+    m = oracle.Model(2, 6.0, enc, head, basis=1)
+    pos, sp = _cluster(rng, 7, 2)
+    out = _all(m, pos, sp)
+    eps = 1e-5
+    for a in (0, 3, 6):
+        for b in range(3):
+            p1, p2 = pos.copy(), pos.copy()
+            p1[a, b] += eps
+            p2[a, b] -= eps
+            fd = -(_all(m, p1, sp)["energy"] - _all(m, p2, sp)["energy"]) / (2 * eps)
+            assert abs(fd - out["forces"][a, b]) < 1e-7 * max(1.0, np.abs(out["forces"]).max())
+    assert np.abs(out["forces"].sum(0)).max() < 1e-10 * max(1.0, np.abs(out["forces"]).max())
+    rot = special_ortho_group.rvs(3, random_state=5)
+    turned = 30.0 + (pos - 30.0) @ rot.T
+    assert abs(_all(m, turned, sp)["energy"] - out["energy"]) < 1e-10 * abs(out["energy"])
