@@ -122,6 +122,24 @@ int mlip_build_neighbors(mlip_ctx *ctx, int64_t n_atoms, const double *pos, cons
                          const double *box, void *stream);
 
 /*
+ * The same build for one sub-domain of a spatial decomposition (Section 3.5 couples the potential to an MD code that
+ * decomposes space and exchanges ghost atoms over MPI; Section 4.4 scales it that way).  The first n_owned atoms are this
+ * domain's own: they are the central atoms i of Eq. 4-10.  The n_ghost atoms after them are copies of other domains'
+ * atoms within r_cut + skin of the domain: they appear as neighbors j only -- no list, no E_i of their own.
+ *   pos / species   dev [n_owned + n_ghost], owned atoms first
+ *   box             as above.  In a dimension that is split, give the sub-domain's extent including its halos plus at
+ *                   least r_cut + skin of empty space, with coordinates shifted into [0, L): the periodic image across
+ *                   the padding is then out of reach and the dimension behaves as open.
+ * mlip_compute then returns, in the caller's order, the forces its central atoms exert: on owned atoms the part of
+ * F_a that comes from this domain's E_i, on the ghosts (entries n_owned ..) the reaction forces -dE_i/dr_a that the
+ * caller must send back to the ghosts' owners and add there.  Energy and virial are this domain's central atoms' sums;
+ * e_atom of a ghost is 0.  Summed over domains the results equal the single-domain evaluation.  New ghost positions
+ * arrive through mlip_set_positions; mlip_step and mlip_step_nvt return MLIP_ERR_UNSUPPORTED on such a context.
+ */
+int mlip_build_neighbors_ghost(mlip_ctx *ctx, int64_t n_owned, int64_t n_ghost, const double *pos, const int32_t *species,
+                               const double *box, void *stream);
+
+/*
  * Export the lists in canonical form: caller's atom indices; for atom i and
  * species s the neighbors of species s in ascending index order occupy
  * nbr[seg_ptr[i*C+s] .. seg_ptr[i*C+s+1]).  Synchronises.

@@ -22,7 +22,7 @@ ERRORS = {0: "MLIP_OK", 1: "MLIP_ERR_INVALID_ARG", 2: "MLIP_ERR_UNSUPPORTED", 3:
           11: "MLIP_ERR_TABLE_RANGE"}
 CODES = {v: k for k, v in ERRORS.items()}
 
-EXPORTS = ["mlip_create", "mlip_table_error", "mlip_build_neighbors", "mlip_get_neighbors", "mlip_get_neighbors_noalloc", "mlip_set_positions",
+EXPORTS = ["mlip_create", "mlip_table_error", "mlip_build_neighbors", "mlip_build_neighbors_ghost", "mlip_get_neighbors", "mlip_get_neighbors_noalloc", "mlip_set_positions",
            "mlip_set_velocities", "mlip_compute", "mlip_compute_f64", "mlip_compute_host", "mlip_step", "mlip_step_nvt", "mlip_get_thermostat", "mlip_reset_thermostat", "mlip_get_rebuilds", "mlip_get_state", "mlip_set_state", "mlip_debug_rebuild",
            "mlip_get_energies", "mlip_sync_status", "mlip_get_counters", "mlip_kernel_time", "mlip_get_timings", "mlip_measure_fp32_peak",
            "mlip_resident_bytes", "mlip_last_error", "mlip_destroy"]
@@ -122,6 +122,14 @@ def _cell(box):
 def mlip_build_neighbors(ctx, pos, species, box, stream=None):
     box = _cell(box)
     _check(ctx, lib().mlip_build_neighbors(ctx, ctypes.c_int64(pos.shape[0]), _dev(pos), _dev(species), _host(box), _stream(stream)))
+
+
+def mlip_build_neighbors_ghost(ctx, n_owned, pos, species, box, stream=None):
+    """Owned atoms first (pos[:n_owned] are the central atoms), ghosts after them."""
+    box = _cell(box)
+    n = pos.shape[0]
+    _check(ctx, lib().mlip_build_neighbors_ghost(ctx, ctypes.c_int64(n_owned), ctypes.c_int64(n - n_owned), _dev(pos), _dev(species),
+                                                 _host(box), _stream(stream)))
 
 
 def mlip_get_neighbors(ctx, seg_ptr, nbr, stream=None):
@@ -289,12 +297,16 @@ class Potential:
         except Exception:
             pass
 
-    def build_neighbors(self, pos, species, box):
+    def build_neighbors(self, pos, species, box, n_owned=None):
+        """n_owned: the leading atoms that are this domain's own; the rest are ghosts (default: all owned)."""
         t = self.torch
         self._pos = t.as_tensor(pos, dtype=t.float64, device=self.device).contiguous()
         self._species = t.as_tensor(species, dtype=t.int32, device=self.device).contiguous()
         self.n = self._pos.shape[0]
-        mlip_build_neighbors(self.ctx, self._pos, self._species, box)
+        if n_owned is None or n_owned == self.n:
+            mlip_build_neighbors(self.ctx, self._pos, self._species, box)
+        else:
+            mlip_build_neighbors_ghost(self.ctx, n_owned, self._pos, self._species, box)
 
     def neighbors(self):
         """Canonical lists as (seg_ptr int64 [N*C+1], nbr int32) on the device."""

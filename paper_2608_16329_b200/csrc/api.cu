@@ -252,8 +252,14 @@ int mlip_table_error(const mlip_ctx *c, double *err_value, double *err_deriv) {
 }
 
 int mlip_build_neighbors(mlip_ctx *c, int64_t n, const double *pos, const int32_t *species, const double *box, void *stream) {
+    return mlip_build_neighbors_ghost(c, n, 0, pos, species, box, stream);
+}
+
+int mlip_build_neighbors_ghost(mlip_ctx *c, int64_t n_owned, int64_t n_ghost, const double *pos, const int32_t *species,
+                               const double *box, void *stream) {
     if (!c) return MLIP_ERR_INVALID_ARG;
-    if (n < 1 || !pos || !species || !box) return fail(c, MLIP_ERR_INVALID_ARG, "bad arguments to mlip_build_neighbors");
+    const int64_t n = n_owned + n_ghost;
+    if (n_owned < 1 || n_ghost < 0 || !pos || !species || !box) return fail(c, MLIP_ERR_INVALID_ARG, "bad arguments to mlip_build_neighbors");
     if (n > (1LL << 28)) return fail(c, MLIP_ERR_UNSUPPORTED, "more than 2^28 atoms per context (the pair queue packs index and species in 32 bits)");
     cudaStream_t s = (cudaStream_t)stream;
     c->last_stream = s;
@@ -265,6 +271,9 @@ int mlip_build_neighbors(mlip_ctx *c, int64_t n, const double *pos, const int32_
     c->built = false;
     if ((rc = ensure_capacity(c, n, c->grid.n_cells)) != MLIP_OK) return rc;
     c->n = n;
+    c->n_owned = n_owned;
+    if (n_ghost > 0) MLIP_CUDA_TRY(c, cudaMemsetAsync(c->e_atom, 0, sizeof(float) * n, s));   // ghosts have no E_i
+    if (n_ghost > 0 && c->cfg.precision == 1) MLIP_CUDA_TRY(c, cudaMemsetAsync(c->e_atom_d, 0, sizeof(double) * n, s));
     if ((rc = launch_pack_source(c, pos, species, s)) != MLIP_OK) return rc;
     double *keep = c->vel_src;   // a NULL source makes the gather reset velocities to zero
     c->vel_src = nullptr;
@@ -396,6 +405,7 @@ static int rebuild_if_due(mlip_ctx *c, int rebuild_every, cudaStream_t s) {
 int mlip_step(mlip_ctx *c, int n_steps, double dt, int rebuild_every, void *stream) {
     if (!c || n_steps < 0 || !(dt > 0.0)) return MLIP_ERR_INVALID_ARG;
     if (!c->built) return fail(c, MLIP_ERR_NOT_BUILT, "no neighbor lists yet");
+    if (c->n_owned != c->n) return fail(c, MLIP_ERR_UNSUPPORTED, "a context with ghost atoms evaluates only: the owner of the ghosts integrates them");
     cudaStream_t s = (cudaStream_t)stream;
     c->last_stream = s;
     int rc;
@@ -417,6 +427,7 @@ int mlip_step_nvt(mlip_ctx *c, int n_steps, double dt, int rebuild_every, double
     if (!c || n_steps < 0 || !(dt > 0.0) || !(t_target > 0.0) || !(t_damp > 0.0)) return MLIP_ERR_INVALID_ARG;
     if (!c->built) return fail(c, MLIP_ERR_NOT_BUILT, "no neighbor lists yet");
     if (c->n < 2) return fail(c, MLIP_ERR_INVALID_ARG, "the thermostat needs at least two atoms");
+    if (c->n_owned != c->n) return fail(c, MLIP_ERR_UNSUPPORTED, "a context with ghost atoms evaluates only: the owner of the ghosts integrates them");
     cudaStream_t s = (cudaStream_t)stream;
     c->last_stream = s;
     const double kB = 8.617333262e-5;   // eV/K

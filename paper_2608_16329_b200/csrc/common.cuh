@@ -75,6 +75,7 @@ struct mlip_ctx {
 
     // system (internal order: by cell, then species, then caller index)
     int64_t n = 0, cap_atoms = 0;
+    int64_t n_owned = 0;           // atoms that are central atoms (caller indices below it); the rest are ghosts
     mlip::CellGrid grid{};
     int64_t cap_cells = 0;
     double4 *pos4 = nullptr;       // x, y, z, species stored as a double

@@ -20,6 +20,9 @@
 //   Regression  Eq. 6 forward and reverse for the 8 atoms of the tile at once as W X^T on the tensor
 //               pipe (weights pre-packed in A-fragment order, 2-way split over the reduction
 //               dimension across the group's warps, elementwise epilogue over the group's threads).
+//               The current species' weights live in tensor memory (tcgen05.alloc / st / ld): a warp
+//               fetches the 32 registers of its next contraction in one instruction, off the
+//               L1/shared-memory pipe; the hidden layers are stored already split into hi + lo.
 //   Derivation  W_i (Eq. 7) is the accumulator fragment of P_i scaled in place: by construction
 //               of the channel permutation it already is the B fragment of the next contraction.
 //               [V; T] = [G; G'] W^T (Eq. 9 and the re-associated Eq. 8 term, U_i never formed)
@@ -27,6 +30,11 @@
 //               memory to lane = pair for the projection of Eq. 10 and the scatter.
 // Everything that is not a contraction (geometry, harmonics, splines, projection) stays on the
 // fp32 pipe; positions are differenced in fp64.
+// Lists come in two parts (neighbor.cu): entries that were within r_cut + skin / 2 at build time first, the rest
+// behind them; the far part cannot reach r_cut before some atom has moved skin / 4, and is skipped until the
+// integrator raises far_flag.
+// Operand splits for the three-term TF32 products are packed fp32 arithmetic (two values per instruction): a
+// Veltkamp split where the result feeds energies, a truncating split where it feeds forces only.
 #include <algorithm>
 
 #include "common.cuh"

@@ -56,14 +56,15 @@ __global__ void k_place(const int32_t *__restrict__ cell_of, int64_t n, const in
 constexpr int MAX_CELL_ATOMS = 1024;
 __global__ void k_sort_cells(int n_cells, int n_species, const int32_t *__restrict__ cell_start,
                              int32_t *__restrict__ slot_src, const double4 *__restrict__ pos4_src,
-                             const int32_t *__restrict__ user_src, int32_t *__restrict__ bin_count, int *status) {
+                             const int32_t *__restrict__ user_src, int32_t *__restrict__ bin_count, int *status, int32_t n_owned) {
+    // (bin_count counts the atoms that will be central atoms: caller indices below n_owned; the others are ghosts)
     int c = blockIdx.x * blockDim.x + threadIdx.x;
     if (c >= n_cells) return;
     int beg = cell_start[c], end = cell_start[c + 1];
     int cnt[MAX_SPECIES] = {0};
     if (end - beg > MAX_CELL_ATOMS) {
         atomicOr(status, FLAG_NONFINITE);
-        for (int a = beg; a < end; ++a) cnt[(int)pos4_src[slot_src[a]].w]++;
+        for (int a = beg; a < end; ++a) { const int src = slot_src[a]; cnt[(int)pos4_src[src].w] += user_src[src] < n_owned; }
         for (int s = 0; s < n_species; ++s) bin_count[(int64_t)s * n_cells + c] = cnt[s];
         return;
     }
@@ -71,7 +72,7 @@ __global__ void k_sort_cells(int n_cells, int n_species, const int32_t *__restri
         int src = slot_src[a];
         int sa = (int)pos4_src[src].w;
         long long key = ((long long)sa << 32) | (unsigned)user_src[src];
-        cnt[sa]++;
+        cnt[sa] += user_src[src] < n_owned;
         int b = a - 1;
         while (b >= beg) {
             int sb_src = slot_src[b];
@@ -103,7 +104,8 @@ __global__ void k_gather(int64_t n, const int32_t *__restrict__ slot_src, const 
 // One thread per cell: the cell's atoms (already species-ordered) go to their (species, cell) bins.
 __global__ void k_center_order(int n_cells, int n_species, const int32_t *__restrict__ cell_start,
                                const double4 *__restrict__ pos4, const int32_t *__restrict__ bin_start,
-                               int32_t *__restrict__ center_order, int32_t *__restrict__ species_start) {
+                               int32_t *__restrict__ center_order, int32_t *__restrict__ species_start,
+                               const int32_t *__restrict__ user_of, int32_t n_owned) {
     int c = blockIdx.x * blockDim.x + threadIdx.x;
     if (c <= n_species) species_start[c] = c < n_species ? bin_start[(int64_t)c * n_cells] : bin_start[(int64_t)n_species * n_cells];
     if (c >= n_cells) return;
@@ -112,7 +114,7 @@ __global__ void k_center_order(int n_cells, int n_species, const int32_t *__rest
     for (int a = beg; a < end; ++a) {
         int s = (int)pos4[a].w;
         if (s != prev) { prev = s; r = 0; }
-        center_order[bin_start[(int64_t)s * n_cells + c] + r++] = a;
+        if (user_of[a] < n_owned) center_order[bin_start[(int64_t)s * n_cells + c] + r++] = a;   // ghosts are never central atoms
     }
 }
 
@@ -124,10 +126,15 @@ template <bool FILL>
 __global__ void __launch_bounds__(256) k_neighbors(int64_t n, CellGrid g, double rl2, const double4 *__restrict__ pos4,
                                                    const int32_t *__restrict__ cell_start, int32_t *__restrict__ nbr_count,
                                                    const int64_t *__restrict__ nbr_off, int32_t *__restrict__ nbr,
-                                                   int64_t nbr_cap, int *status, float near2, int32_t *__restrict__ nbr_near) {
+                                                   int64_t nbr_cap, int *status, float near2, int32_t *__restrict__ nbr_near,
+                                                   const int32_t *__restrict__ user_of, int32_t n_owned) {
     const int lane = threadIdx.x & 31;
     int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (i >= n || (*status & FLAG_NONFINITE)) return;   // a broken configuration is not traversed (see k_sort_cells)
+    if (user_of[i] >= n_owned) {   // a ghost is listed by others but has no list of its own
+        if (!FILL && lane == 0) { nbr_count[i] = 0; nbr_near[i] = 0; }
+        return;
+    }
     const double4 pi = pos4[i];
     // this lane's cell: offsets (ox, oy, oz) = (lane / 9, lane / 3 % 3, lane % 3); dimensions with fewer than
     // three cells list each cell once
@@ -234,10 +241,14 @@ __global__ void __launch_bounds__(256) k_neighbors_rel(int64_t n, CellGrid g, do
                                                        const float4 *__restrict__ rel, const int32_t *__restrict__ cell_start,
                                                        int32_t *__restrict__ nbr_count, const int64_t *__restrict__ nbr_off,
                                                        int32_t *__restrict__ nbr, int64_t nbr_cap, int *status, float near2,
-                                                       int32_t *__restrict__ nbr_near) {
+                                                       int32_t *__restrict__ nbr_near, const int32_t *__restrict__ user_of, int32_t n_owned) {
     const int lane = threadIdx.x & 31;
     int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (i >= n || (*status & FLAG_NONFINITE)) return;
+    if (user_of[i] >= n_owned) {
+        if (!FILL && lane == 0) { nbr_count[i] = 0; nbr_near[i] = 0; }
+        return;
+    }
     const double4 pi = pos4[i];
     const float4 ri = rel[i];
     int cb = 0, ce = 0;
@@ -408,7 +419,8 @@ __global__ void __launch_bounds__(256) k_neighbors_onepass(int64_t n, CellGrid g
                                                            int64_t *__restrict__ nbr_off, int32_t *__restrict__ nbr, int64_t nbr_cap,
                                                            int *status, unsigned long long *tile_state, int *ticket,
                                                            const int *global_status, int spin_limit, long long unpublished_tile,
-                                                           float near2, int32_t *__restrict__ nbr_near) {
+                                                           float near2, int32_t *__restrict__ nbr_near,
+                                                           const int32_t *__restrict__ user_of, int32_t n_owned) {
     // `unpublished_tile` >= 0 (diagnostic builds of the lists only) names a tile that never publishes its look-back word,
     // so that its successor's bounded wait can be seen to run out; -1 in production.
     if (*global_status & FLAG_NONFINITE) return;   // a broken configuration is not traversed (see k_sort_cells)
@@ -431,7 +443,8 @@ __global__ void __launch_bounds__(256) k_neighbors_onepass(int64_t n, CellGrid g
         const int slot = warp * OP_PER_WARP + a;
         const int64_t i = first + slot;
         int cnt = 0, cn = 0;
-        if (i < n) cnt = onepass_traverse(i, g, rl2, edge, rl2_lo, rl2_hi, pos4, rel, cell_start, lane, s_hits + slot * OP_BUF, OP_BUF - 1, OP_BUF, near2, cn);
+        if (i < n && user_of[i] < n_owned)   // (a ghost has no list of its own)
+            cnt = onepass_traverse(i, g, rl2, edge, rl2_lo, rl2_hi, pos4, rel, cell_start, lane, s_hits + slot * OP_BUF, OP_BUF - 1, OP_BUF, near2, cn);
         if (lane == 0) { s_cnt[slot] = cnt; s_near[slot] = cn; }
     }
     __syncthreads();
@@ -584,11 +597,11 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
     // nbr_count doubles as the slot -> source map until the lists are counted
     int32_t *slot_src = c->nbr_count;
     k_place<<<blocks_for(n, 256), 256, 0, s>>>(c->cell_of, n, c->cell_start, c->cell_fill, slot_src);
-    k_sort_cells<<<blocks_for(g.n_cells, 128), 128, 0, s>>>(g.n_cells, C, c->cell_start, slot_src, c->pos4_src, c->user_src, c->bin_count, c->status);
+    k_sort_cells<<<blocks_for(g.n_cells, 128), 128, 0, s>>>(g.n_cells, C, c->cell_start, slot_src, c->pos4_src, c->user_src, c->bin_count, c->status, (int32_t)c->n_owned);
     k_gather<<<blocks_for(n, 256), 256, 0, s>>>(n, slot_src, c->pos4_src, c->vel_src, c->user_src, c->pos4, c->vel, c->user_of, c->disp);
     exclusive_scan<int32_t, int32_t>(c->bin_count, c->bin_start, (int64_t)C * g.n_cells, c->scan_tmp, s);
     int nthreads_co = g.n_cells > C + 1 ? g.n_cells : C + 1;
-    k_center_order<<<blocks_for(nthreads_co, 128), 128, 0, s>>>(g.n_cells, C, c->cell_start, c->pos4, c->bin_start, c->center_order, c->species_start);
+    k_center_order<<<blocks_for(nthreads_co, 128), 128, 0, s>>>(g.n_cells, C, c->cell_start, c->pos4, c->bin_start, c->center_order, c->species_start, c->user_of, (int32_t)c->n_owned);
     // grids of at least 3 x 3 x 3 cells take the fp32 cell-relative traversal (positions staged in the idle force array)
     const bool rel = g.n[0] >= 3 && g.n[1] >= 3 && g.n[2] >= 3;
     float4 *relpos = c->force;
@@ -605,7 +618,7 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
         k_neighbors_onepass<<<(unsigned)n_tiles, 256, sizeof(int32_t) * OP_TILE * OP_BUF, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_off, c->nbr, c->nbr_cap,
                                                                flag, c->tile_state, c->tile_ticket, c->status,
                                                                c->lookback_spin_limit > 0 ? c->lookback_spin_limit : OP_SPIN, c->lookback_unpublished_tile,
-                                                               near2, c->nbr_near);
+                                                               near2, c->nbr_near, c->user_of, (int32_t)c->n_owned);
         c->launches += 5 + 2 * 3 + 2;   // cell id, place, sort, gather, centre order; two scans; relative positions, lists
         MLIP_CUDA_TRY(c, cudaGetLastError());
         bool done = true;
@@ -626,10 +639,10 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
     }
     if (rel) {
         if (!rel_ready) k_rel_pos<<<blocks_for(n, 256), 256, 0, s>>>(n, g, c->pos4, relpos);
-        k_neighbors_rel<false><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_count, nullptr, nullptr, 0, c->status, near2, c->nbr_near);
+        k_neighbors_rel<false><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_count, nullptr, nullptr, 0, c->status, near2, c->nbr_near, c->user_of, (int32_t)c->n_owned);
         c->launches += 1;
     } else
-        k_neighbors<false><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, c->cell_start, c->nbr_count, nullptr, nullptr, 0, c->status, near2, c->nbr_near);
+        k_neighbors<false><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, c->cell_start, c->nbr_count, nullptr, nullptr, 0, c->status, near2, c->nbr_near, c->user_of, (int32_t)c->n_owned);
     exclusive_scan<int32_t, int64_t>(c->nbr_count, c->nbr_off, n, c->scan_tmp, s);
     c->launches += 5 + 1 + 3 * 3;   // cell id, place, sort, gather, centre order; count; three scans
     MLIP_CUDA_TRY(c, cudaGetLastError());
@@ -648,9 +661,9 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
         }
     }
     if (rel)
-        k_neighbors_rel<true><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_count, c->nbr_off, c->nbr, c->nbr_cap, c->status, near2, c->nbr_near);
+        k_neighbors_rel<true><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_count, c->nbr_off, c->nbr, c->nbr_cap, c->status, near2, c->nbr_near, c->user_of, (int32_t)c->n_owned);
     else
-        k_neighbors<true><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, c->cell_start, c->nbr_count, c->nbr_off, c->nbr, c->nbr_cap, c->status, near2, c->nbr_near);
+        k_neighbors<true><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, c->cell_start, c->nbr_count, c->nbr_off, c->nbr, c->nbr_cap, c->status, near2, c->nbr_near, c->user_of, (int32_t)c->n_owned);
     c->launches += 1;
     timing_end(c->ev_build, c->build_count, s);
     MLIP_CUDA_TRY(c, cudaGetLastError());
