@@ -94,7 +94,10 @@ def parse_args():
     ap.add_argument("--ensemble", default="nve", choices=["nve", "nvt"],
                     help="nvt adds the Nose-Hoover-chain thermostat (the paper's ensemble) to every step: an extra data point")
     ap.add_argument("--k", type=int, default=32, choices=[16, 32, 64], help="radial channels (other than 32: --precision f64 only)")
-    ap.add_argument("--lmax", type=int, default=3, choices=[1, 2, 3], help="angular order (other than 3: --precision f64 only)")
+    ap.add_argument("--lmax", type=int, default=3, choices=[1, 2, 3, 4, 5], help="angular order (other than 3: --precision f64 only; 4, 5: k = 32)")
+    ap.add_argument("--basis", default="irreducible", choices=["irreducible", "canonical"],
+                    help="canonical = all Cartesian monomials with the multiplicity metric, the descriptor before the "
+                         "irreducible reduction (d = 20 at l_max = 3): --precision f64 only")
     ap.add_argument("--sweep", default="", help="comma-separated FCC cell counts: size sweep of the 6-species workload "
                     "(inputs generated on the device), one JSON line per size; not the contract line")
     return ap.parse_args()
@@ -203,11 +206,11 @@ def sample_blocks(cells, n_basis, a, r_cut, n_centers, seed=0):
     return all_atoms, inner
 
 
-def cpu_oracle_sample(w, enc, head, n_centers, repeats=1, rows=None, pos=None, k=32, l_max=3):
+def cpu_oracle_sample(w, enc, head, n_centers, repeats=1, rows=None, pos=None, k=32, l_max=3, basis=0):
     """Time the oracle (neighbor search + full evaluation) on `rows` (default: evenly spread central atoms).
     Returns (rows, seconds, threads, the oracle's outputs)."""
     import oracle
-    model = oracle.Model(w.n_species, w.r_cut, enc, head, k=k, l_max=l_max)
+    model = oracle.Model(w.n_species, w.r_cut, enc, head, k=k, l_max=l_max, basis=basis)
     if rows is None:
         rows = np.unique(np.linspace(0, w.n_atoms - 1, n_centers).astype(np.int64))
     pos = w.pos if pos is None else pos
@@ -226,7 +229,8 @@ def problem_setup(args, rank=0):
     import workloads as wl
     cfg = args.cfg
     w = wl.make_workload(cfg, n_cells=args.cells if cfg == CFG else None, seed=wl.BASE_SEED + cfg + 17 * rank)
-    default_shape = args.k == 32 and args.lmax == 3
+    canonical = args.basis == "canonical"
+    default_shape = args.k == 32 and args.lmax == 3 and not canonical
     if default_shape:
         enc, head = wl.workload_weights(cfg, w.n_species)
     else:   # descriptor-shape variants of the paper's ablations: same recipe, networks of that shape
@@ -234,13 +238,14 @@ def problem_setup(args, rank=0):
                                     k=args.k, l_max=args.lmax)
     flop_pair, flop_atom = FLOP_PER_PAIR, FLOP_PER_ATOM
     if not default_shape:   # the same count written out in k and d = (l_max + 1)^2
-        d_ang, n_inv = (args.lmax + 1) ** 2, (args.lmax + 1) * args.k
+        d_ang = (args.lmax + 1) * (args.lmax + 2) * (args.lmax + 3) // 6 if canonical else (args.lmax + 1) ** 2
+        n_inv = (args.lmax + 1) * args.k
         flop_pair = 60 + 150 * d_ang / 16 + 512 * args.k / 32 + 6 * d_ang * args.k + 168 * d_ang / 16
         flop_atom = 3 * d_ang * args.k + 4 * (n_inv * 64 + 3 * 64 * 64) + 256 + 5000
     lattice = ((args.cells,) * 3, 4, 3.6) if cfg == CFG else LATTICES[cfg]
     return {"w": w, "enc": enc, "head": head, "default_shape": default_shape, "flop_pair": flop_pair, "flop_atom": flop_atom,
             "rebuild_every": REBUILD_EVERY if cfg != 4 else 3,   # the ionic stand-in is far from equilibrium under random weights
-            "lattice": lattice, "f64": args.precision == "f64"}
+            "lattice": lattice, "f64": args.precision == "f64", "basis": 1 if canonical else 0}
 
 
 def run_reference(args, rank, world):
@@ -366,7 +371,7 @@ def main():
     w, enc, head, default_shape, rebuild_every, f64 = (prob[q] for q in ("w", "enc", "head", "default_shape", "rebuild_every", "f64"))
     n = w.n_atoms
     pot = mlip.Potential(w.n_species, w.r_cut, w.skin, enc, head, w.masses, device=local_rank, precision=1 if f64 else 0,
-                         k=args.k, l_max=args.lmax, force_mode=1 if args.deterministic else 0)
+                         k=args.k, l_max=args.lmax, force_mode=1 if args.deterministic else 0, basis=prob["basis"])
     table_err = mlip.mlip_table_error(pot.ctx)
 
     # ---- device-resident run: inputs already in HBM when timing starts ----
@@ -472,7 +477,7 @@ def main():
                 "dtype": args.precision, "data": "synthetic",
                 "config": {"workload": f"cfg{cfg} {w.name}: {n} atoms, {w.n_species} species, r_cut 6 A, skin 1 A, "
                                        f"{args.ensemble.upper()} dt 1 fs, list rebuild every {rebuild_every} steps"
-                                       + ("" if default_shape else f", k = {args.k}, l_max = {args.lmax}")
+                                       + ("" if default_shape else f", k = {args.k}, l_max = {args.lmax}, {args.basis} basis")
                                        + (", deterministic force mode" if args.deterministic else ""),
                            "atoms_per_gpu": n, "parallelism": "replicas" if world > 1 else "single",
                            "l2": "inputs larger than L2 (positions + lists = %.1f GB per GPU)" % ((32 * n + 4 * entries) / 1e9)},
@@ -495,7 +500,7 @@ def main():
             gpu = pot.compute(want_e_atom=True)
             pot.sync_status(raise_on_error=False)
             pos_now = pos_t.cpu().numpy()
-            rows, sec, cores, ref = cpu_oracle_sample(w, enc, head, rows.size, rows=rows, pos=pos_now, k=args.k, l_max=args.lmax)
+            rows, sec, cores, ref = cpu_oracle_sample(w, enc, head, rows.size, rows=rows, pos=pos_now, k=args.k, l_max=args.lmax, basis=prob["basis"])
             line["cpu_baseline"] = {"value": rows.size / sec, "unit": UNIT, "cores": cores, "kind": "oracle",
                                     "sample": f"{rows.size} central atoms in blocks of cells spread over the {n}-atom workload, one "
                                               f"energy/force/virial evaluation incl. their neighbor search ({sec:.1f} s)"}
@@ -503,10 +508,13 @@ def main():
             d_e = np.abs(gpu["e_atom"][rows_t].double().cpu().numpy() - ref["e_atom"][rows])
             d_f = np.abs(gpu["forces"][inner_t].double().cpu().numpy() - ref["forces"][inner]) if inner.size else np.zeros(1)
             e_tol, f_tol = (1e-9, 2e-9) if f64 else (2e-5, 1e-4)
-            line["parity"] = {"against": "oracle, same state (positions after the timed steps)", "n_atoms_e": int(rows.size),
+            e_tol *= max(1.0, float(np.abs(ref["e_atom"][rows]).max()))
+            if not default_shape and inner.size:   # networks of other shapes are not calibrated to forces of order 1 eV/Angstrom
+                f_tol *= max(1.0, float(np.abs(ref["forces"][inner]).max()))
+            line["parity"] = {"against": "oracle, same state (the positions the context held after the timed runs)", "n_atoms_e": int(rows.size),
                               "max_dE_i": float(d_e.max()), "n_atoms_f": int(inner.size), "max_dF": float(d_f.max()),
-                              "tolerance": {"dE_i": e_tol * max(1.0, float(np.abs(ref["e_atom"][rows]).max())), "dF": f_tol},
-                              "ok": bool(d_e.max() <= e_tol * max(1.0, float(np.abs(ref["e_atom"][rows]).max())) and d_f.max() <= f_tol)}
+                              "tolerance": {"dE_i": e_tol, "dF": f_tol},
+                              "ok": bool(d_e.max() <= e_tol and d_f.max() <= f_tol)}
         print(json.dumps(line), flush=True)
     pot.close()
     if world > 1:

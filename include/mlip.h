@@ -23,7 +23,8 @@
  *   - Units: Angstrom, eV, amu, fs.  Atom order of every array argument is the
  *     caller's; the library keeps its own cell-sorted order internally.
  *   - The fp32 path is compiled for k = 32 radial channels and l_max = 3 (d = 16), the paper's production
- *     shape; the fp64 path (precision = 1) also for k in {16, 32, 64} x l_max in {1, 2, 3}.  The
+ *     shape; the fp64 path (precision = 1) also for k in {16, 32, 64} x l_max in {1, 2, 3}, for k = 32 with
+ *     l_max = 4, 5 (d = 25, 36), and for the canonical angular basis (config.basis = 1) with k in {32, 64}.  The
  *     encoder is 1 -> enc_hidden x enc_layers -> k, the head is
  *     (l_max+1) k -> head_hidden x head_layers -> 1 with head_hidden = 64,
  *     head_layers = 4 (Section 4.1.3), SiLU, identity skips around hidden
@@ -62,7 +63,7 @@ typedef struct {
     double r_cut;         /* Angstrom */
     double skin;          /* list radius = r_cut + skin */
     int k;                /* 32 (precision 1: 16, 32 or 64) */
-    int l_max;            /* 3 (precision 1: 1, 2 or 3) */
+    int l_max;            /* 3 (precision 1: 1 .. 5, see above) */
     int enc_hidden, enc_layers;    /* e.g. 128, 3 */
     int head_hidden, head_layers;  /* 64, 4 */
     int table_knots;      /* intervals of the radial table on [table_r_min, r_cut]; 0 = automatic: 64, doubled until table_tol holds */
@@ -83,6 +84,10 @@ typedef struct {
                              either mode); +24 bytes per atom, fp32 path only */
     int envelope;         /* smooth cutoff f_c multiplying the encoder output (the paper names none): 0 = (1 + cos(pi r / r_c)) / 2,
                              1 = 1 - 10 x^3 + 15 x^4 - 6 x^5 with x = r / r_c (second derivative also vanishes at r_c) */
+    int basis;            /* angular basis (Section 3.3): 0 = irreducible harmonics, d = (l_max + 1)^2, C_l = I (the paper's
+                             choice); 1 = canonical: every Cartesian monomial of the unit vector up to degree l_max,
+                             d = 4, 10, 20 for l_max = 1, 2, 3 (Eq. 11), with C_l = the multinomial multiplicities in Eq. 5
+                             -- the descriptor "before reduction" of Table 7; precision 1 only */
 } mlip_config;
 
 /*

@@ -131,11 +131,13 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
     *out = nullptr;
     if (!cfg || !enc_w || !head_w || !mass) return fail(nullptr, MLIP_ERR_INVALID_ARG, "NULL argument");
     if (cfg->n_species < 1 || cfg->n_species > MAX_SPECIES) return fail(nullptr, MLIP_ERR_UNSUPPORTED, "n_species must be 1..8");
+    if (cfg->basis < 0 || cfg->basis > 1) return fail(nullptr, MLIP_ERR_INVALID_ARG, "basis must be 0 (irreducible) or 1 (canonical)");
     if (cfg->precision == 1) {
-        if (!f64_shape_supported(cfg->k, cfg->l_max))
-            return fail(nullptr, MLIP_ERR_UNSUPPORTED, "the fp64 path is compiled for k in {16, 32, 64} and l_max in {1, 2, 3}");
-    } else if (cfg->k != K_RADIAL || cfg->l_max != 3) {
-        return fail(nullptr, MLIP_ERR_UNSUPPORTED, "the fp32 path is compiled for k = 32, l_max = 3 only (other shapes: precision = 1)");
+        if (!f64_shape_supported(cfg->k, cfg->l_max, cfg->basis))
+            return fail(nullptr, MLIP_ERR_UNSUPPORTED, "the fp64 path is compiled for the irreducible basis with k in {16, 32, 64} x l_max in {1, 2, 3} and "
+                                                       "k = 32 x l_max in {4, 5}, and for the canonical basis with k in {32, 64} x l_max in {1, 2, 3}");
+    } else if (cfg->k != K_RADIAL || cfg->l_max != 3 || cfg->basis != 0) {
+        return fail(nullptr, MLIP_ERR_UNSUPPORTED, "the fp32 path is compiled for k = 32, l_max = 3, irreducible basis only (other shapes: precision = 1)");
     }
     if (cfg->head_hidden != HEAD_H || cfg->head_layers != HEAD_L) return fail(nullptr, MLIP_ERR_UNSUPPORTED, "only a 4 x 64 head is compiled in");
     if (cfg->enc_hidden < 1 || cfg->enc_layers < 1) return fail(nullptr, MLIP_ERR_INVALID_ARG, "bad encoder shape");

@@ -168,7 +168,7 @@ int launch_megakernel(mlip_ctx *c, cudaStream_t s);
 // megakernel_f64.cu
 int upload_head_f64(mlip_ctx *c, const double *head_w_host);
 int launch_megakernel_f64(mlip_ctx *c, cudaStream_t s);
-bool f64_shape_supported(int k, int l_max);
+bool f64_shape_supported(int k, int l_max, int basis);
 // integrate.cu
 int launch_kick_drift(mlip_ctx *c, double dt, cudaStream_t s, const double *vscale = nullptr);
 int launch_nhc_half(mlip_ctx *c, double n_f, double kT, double q1, double qk, double dt, cudaStream_t s);

@@ -19,19 +19,22 @@
 // The radial tables are the same clamped cubic B-splines as in the fp32 path but with fp64
 // coefficients and enough knots for ~1e-11 relative error; they stay in global memory (L2).
 //
-// The kernel is a template over the descriptor shape: k in {16, 32, 64} radial channels and
-// l_max in {1, 2, 3} (d = 4, 9, 16), the throughput side of the paper's ablations (Tables 6, 7 and
+// The kernel is a template over the descriptor shape: k in {16, 32, 64} radial channels,
+// l_max in {1, 2, 3} (d = 4, 9, 16) with closed-form harmonics, plus (angular.cuh) l_max = 4, 5
+// (d = 25, 36) through projection matrices and the canonical monomial basis (d = 4, 10, 20) with
+// the metric C_l of Eq. 5 -- the throughput side of the paper's ablations (Tables 6, 7 and
 // Fig. 4(c)).  With k = 16 the upper half-warp idles in the lane = channel phases; with k = 64
 // a lane owns channels lane and lane + 32.
 #include <algorithm>
+#include <type_traits>
 
+#include "angular.cuh"
 #include "common.cuh"
 #include "pair_math.cuh"
 
 namespace mlip {
 
 constexpr int F64_TILE = 8;         // atoms per tile = warps per CTA = columns of the tensor-pipe tile
-constexpr int F64_ST = 22;          // hand-over row: 16 h, 4 b, table offset, pad
 constexpr int F64_YS = HEAD_H + 4;  // activation row stride: 4 mod 16 keeps the B-fragment reads conflict-free
 
 // per-species head block (doubles) for n_inv inputs: the caller's row-major matrices, then biases and output layer
@@ -45,11 +48,11 @@ struct Head64 {
           total(wout + HEAD_H + 8) {}
 };
 
-__host__ __device__ constexpr int l_of(int a) { return a == 0 ? 0 : (a < 4 ? 1 : (a < 9 ? 2 : 3)); }
-
-template <int K, int LMAX>
+template <int K, int LMAX, int BASIS>
 struct TileSmem {
-    static constexpr int D = (LMAX + 1) * (LMAX + 1);
+    using Shape = AngShape<LMAX, BASIS>;
+    static constexpr int D = Shape::D;
+    static constexpr int ST = (D + 6) & ~1;   // hand-over row: D angular values, 4 spline weights, table offset, pad
     static constexpr int NINV = (LMAX + 1) * K;
     static constexpr int XS = (NINV + 31) / 32 * 32 + 4;
     double x[F64_TILE][XS];                 // invariants, then dE/dG
@@ -57,7 +60,7 @@ struct TileSmem {
     double sd[HEAD_L][F64_TILE][F64_YS];    // SiLU'(pre-activation) per layer
     double dp[2][F64_TILE][F64_YS];         // dE/dpre of the layer being propagated
     union {
-        double st[32][F64_ST];              // encoding hand-over
+        double st[32][ST];                  // encoding hand-over
         double w[D * K];                    // W_i = dE_i/dP_i (Eq. 7), derivation
     } pw[F64_TILE];
     int q[F64_TILE][64];                    // compacted neighbor indices
@@ -97,10 +100,12 @@ __device__ __forceinline__ void dmma(double &c0, double &c1, double a, double b)
     asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};" : "+d"(c0), "+d"(c1) : "d"(a), "d"(b));
 }
 
-template <int K, int LMAX>
-__global__ void __launch_bounds__(F64_TILE * 32, K <= 32 ? 2 : 1) k_mega_f64(F64Args k) {
-    using SM = TileSmem<K, LMAX>;
+template <int K, int LMAX, int BASIS>
+__global__ void __launch_bounds__(F64_TILE * 32, (K <= 32 && AngShape<LMAX, BASIS>::D <= 20) ? 2 : 1) k_mega_f64(F64Args k) {
+    using SM = TileSmem<K, LMAX, BASIS>;
+    using Shape = AngShape<LMAX, BASIS>;
     constexpr int D = SM::D, NINV = SM::NINV;
+    constexpr bool CLOSED = BASIS == 0 && LMAX <= 3;   // the default basis up to l = 3 has hand-written harmonics
     constexpr int CPL = (K + 31) / 32;   // channels per lane
     constexpr Head64 H(NINV);
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -158,16 +163,17 @@ __global__ void __launch_bounds__(F64_TILE * 32, K <= 32 ? 2 : 1) k_mega_f64(F64
                 valid = d2 < k.rc2;
                 if (valid) {
                     const double r = sqrt(d2), rinv = 1.0 / r;
-                    double h[D_ANG], b[4];
-                    harmonics(dx * rinv, dy * rinv, dz * rinv, h);
+                    double h[CLOSED ? D_ANG : D], b[4];
+                    if (CLOSED) harmonics(dx * rinv, dy * rinv, dz * rinv, h);
+                    else angular_values<LMAX, BASIS>(dx * rinv, dy * rinv, dz * rinv, h);
                     const int iv = spline_basis<false, double>(r, k.r_min, k.inv_h, k.knots, b, nullptr, k.status);
                     double *row = sm.pw[wid].st[lane];
 #pragma unroll
                     for (int a = 0; a < D; ++a) row[a] = h[a];
 #pragma unroll
-                    for (int m = 0; m < 4; ++m) row[16 + m] = b[m];
+                    for (int m = 0; m < 4; ++m) row[D + m] = b[m];
                     const long long off = ((long long)(si * C + (int)pj.w) * (k.knots + 3) + iv) * K;
-                    row[20] = __longlong_as_double(off);
+                    row[D + 4] = __longlong_as_double(off);
                 }
             }
             unsigned mask = __ballot_sync(0xffffffffu, valid);
@@ -177,16 +183,16 @@ __global__ void __launch_bounds__(F64_TILE * 32, K <= 32 ? 2 : 1) k_mega_f64(F64
                 const int p = __ffs(mask) - 1;
                 mask &= mask - 1;
                 const double *row = sm.pw[wid].st[p];
-                const double *cf = k.coef + __double_as_longlong(row[20]);
+                const double *cf = k.coef + __double_as_longlong(row[D + 4]);
 #pragma unroll
                 for (int q = 0; q < CPL; ++q) {
                     const int c = lane + 32 * q;
                     double gq = 0.0;
                     if (c < K) {
-                        gq = row[16] * cf[c];
-                        gq = fma(row[17], cf[K + c], gq);
-                        gq = fma(row[18], cf[2 * K + c], gq);
-                        gq = fma(row[19], cf[3 * K + c], gq);
+                        gq = row[D] * cf[c];
+                        gq = fma(row[D + 1], cf[K + c], gq);
+                        gq = fma(row[D + 2], cf[2 * K + c], gq);
+                        gq = fma(row[D + 3], cf[3 * K + c], gq);
                     }
 #pragma unroll
                     for (int a = 0; a < D; ++a) P[a][q] = fma(row[a], gq, P[a][q]);
@@ -195,7 +201,7 @@ __global__ void __launch_bounds__(F64_TILE * 32, K <= 32 ? 2 : 1) k_mega_f64(F64
             __syncwarp();
         }
 
-        // ---------------- Invariants (Eq. 5, C_l = I); an empty slot of a ragged tile feeds zeros ----------------
+        // ---------------- Invariants (Eq. 5: p^T C_l p); an empty slot of a ragged tile feeds zeros ----------------
 #pragma unroll
         for (int q = 0; q < CPL; ++q) {
             const int c = lane + 32 * q;
@@ -205,7 +211,7 @@ __global__ void __launch_bounds__(F64_TILE * 32, K <= 32 ? 2 : 1) k_mega_f64(F64
                 for (int l = 1; l <= LMAX; ++l) {
                     double s = 0.0;
 #pragma unroll
-                    for (int a = l * l; a < (l + 1) * (l + 1); ++a) s = fma(P[a][q], P[a][q], s);
+                    for (int a = Shape::begin(l); a < Shape::begin(l + 1); ++a) s = fma(Shape::metric(a) * P[a][q], P[a][q], s);
                     sm.x[wid][l * K + c] = s;
                 }
             }
@@ -283,7 +289,7 @@ __global__ void __launch_bounds__(F64_TILE * 32, K <= 32 ? 2 : 1) k_mega_f64(F64
             if (c < K) {
                 wi[c] = sm.x[wid][c];
 #pragma unroll
-                for (int a = 1; a < D; ++a) wi[a * K + c] = 2.0 * sm.x[wid][l_of(a) * K + c] * P[a][q];
+                for (int a = 1; a < D; ++a) wi[a * K + c] = (2.0 * Shape::metric(a)) * sm.x[wid][Shape::l_of(a) * K + c] * P[a][q];
             }
         }
         __syncwarp();
@@ -323,30 +329,46 @@ __global__ void __launch_bounds__(F64_TILE * 32, K <= 32 ? 2 : 1) k_mega_f64(F64
                 double b[4], db[4];
                 const int iv = spline_basis<true, double>(r, k.r_min, k.inv_h, k.knots, b, db, k.status);
                 const double *cf = k.coef + ((size_t)(si * C + (int)pj.w) * (k.knots + 3) + iv) * K;
-                double v[D_ANG], tt[D_ANG];   // components beyond d stay zero and drop out of the projection
+                // v = W g and t = W g' (Eq. 9 and the re-associated Eq. 8 term) for the rows of the angular degrees L0 .. L1,
+                // projected at once; wide bases go through in two degree ranges so that v and t stay in registers
+                double s = 0.0, tx = 0.0, ty = 0.0, tz = 0.0, tu = 0.0;
+                auto rows_of = [&](auto l0c, auto l1c) {
+                    constexpr int L0 = decltype(l0c)::value, L1 = decltype(l1c)::value;
+                    constexpr int A0 = CLOSED ? 0 : Shape::begin(L0), A1 = CLOSED ? D : Shape::begin(L1 + 1);
+                    constexpr int DV = CLOSED ? D_ANG : A1 - A0;
+                    double v[DV], tt[DV];   // (closed forms: components beyond d stay zero and drop out of the projection)
 #pragma unroll
-                for (int a = 0; a < D_ANG; ++a) { v[a] = 0.0; tt[a] = 0.0; }
+                    for (int a = 0; a < DV; ++a) { v[a] = 0.0; tt[a] = 0.0; }
 #pragma unroll 1
-                for (int c = 0; c < K; c += 4) {   // four channels = one 32-byte sector per table row
-                    double gv[4] = {0.0, 0.0, 0.0, 0.0}, dg[4] = {0.0, 0.0, 0.0, 0.0};
+                    for (int c = 0; c < K; c += 4) {   // four channels = one 32-byte sector per table row
+                        double gv[4] = {0.0, 0.0, 0.0, 0.0}, dg[4] = {0.0, 0.0, 0.0, 0.0};
 #pragma unroll
-                    for (int m = 0; m < 4; ++m) {
-                        double cc[4];
-                        asm volatile("ld.global.nc.v4.f64 {%0,%1,%2,%3}, [%4];"
-                                     : "=d"(cc[0]), "=d"(cc[1]), "=d"(cc[2]), "=d"(cc[3]) : "l"(cf + m * K + c));
+                        for (int m = 0; m < 4; ++m) {
+                            double cc[4];
+                            asm volatile("ld.global.nc.v4.f64 {%0,%1,%2,%3}, [%4];"
+                                         : "=d"(cc[0]), "=d"(cc[1]), "=d"(cc[2]), "=d"(cc[3]) : "l"(cf + m * K + c));
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) { gv[u] = fma(b[m], cc[u], gv[u]); dg[u] = fma(db[m], cc[u], dg[u]); }
+                            for (int u = 0; u < 4; ++u) { gv[u] = fma(b[m], cc[u], gv[u]); dg[u] = fma(db[m], cc[u], dg[u]); }
+                        }
+#pragma unroll
+                        for (int a = A0; a < A1; ++a) {
+                            const double2 w0 = *reinterpret_cast<const double2 *>(&wi[a * K + c]);
+                            const double2 w1 = *reinterpret_cast<const double2 *>(&wi[a * K + c + 2]);
+                            v[a - A0] = fma(w0.x, gv[0], fma(w0.y, gv[1], fma(w1.x, gv[2], fma(w1.y, gv[3], v[a - A0]))));
+                            tt[a - A0] = fma(w0.x, dg[0], fma(w0.y, dg[1], fma(w1.x, dg[2], fma(w1.y, dg[3], tt[a - A0]))));
+                        }
                     }
-#pragma unroll
-                    for (int a = 0; a < D; ++a) {
-                        const double2 w0 = *reinterpret_cast<const double2 *>(&wi[a * K + c]);
-                        const double2 w1 = *reinterpret_cast<const double2 *>(&wi[a * K + c + 2]);
-                        v[a] = fma(w0.x, gv[0], fma(w0.y, gv[1], fma(w1.x, gv[2], fma(w1.y, gv[3], v[a]))));
-                        tt[a] = fma(w0.x, dg[0], fma(w0.y, dg[1], fma(w1.x, dg[2], fma(w1.y, dg[3], tt[a]))));
-                    }
+                    double ps, px, py, pz, pu;
+                    if (CLOSED) harmonics_project(ux, uy, uz, v, tt, ps, px, py, pz, pu);
+                    else angular_project<LMAX, BASIS, L0, L1>(ux, uy, uz, v, tt, ps, px, py, pz, pu);
+                    s += ps; tx += px; ty += py; tz += pz; tu += pu;
+                };
+                if constexpr (!CLOSED && D > 25) {
+                    rows_of(std::integral_constant<int, 0>{}, std::integral_constant<int, 3>{});
+                    rows_of(std::integral_constant<int, 4>{}, std::integral_constant<int, LMAX>{});
+                } else {
+                    rows_of(std::integral_constant<int, 0>{}, std::integral_constant<int, LMAX>{});
                 }
-                double s, tx, ty, tz, tu;
-                harmonics_project(ux, uy, uz, v, tt, s, tx, ty, tz, tu);
                 // f_ij = (g' . u_ij) r^ + J_ang^T v_ij,  J_ang = (grad_u h)(I - u u^T) / r
                 const double qx = s * ux + (tx - tu * ux) * rinv;
                 const double qy = s * uy + (ty - tu * uy) * rinv;
@@ -432,24 +454,35 @@ int upload_head_f64(mlip_ctx *c, const double *w) {
     return MLIP_OK;
 }
 
-template <int K, int LMAX>
+template <int K, int LMAX, int BASIS>
 static cudaError_t launch_shape(mlip_ctx *c, const F64Args &k, cudaStream_t s, cudaEvent_t start, cudaEvent_t stop) {
-    const size_t smem_bytes = sizeof(TileSmem<K, LMAX>);
+    const size_t smem_bytes = sizeof(TileSmem<K, LMAX, BASIS>);
     if (!c->kernel_ready) {
-        cudaError_t e = cudaFuncSetAttribute(k_mega_f64<K, LMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+        cudaError_t e = cudaFuncSetAttribute(k_mega_f64<K, LMAX, BASIS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
         if (e != cudaSuccess) return e;
+        if (!(BASIS == 0 && LMAX <= 3)) {   // projection matrices for the general angular routines
+            double q[Q_TOTAL];
+            build_q_tables(q);
+            e = cudaMemcpyToSymbol(c_ang_q, q, sizeof q);
+            if (e != cudaSuccess) return e;
+        }
         c->kernel_ready = true;
     }
-    const int per_sm = K <= 32 ? 2 : 1;
+    const int per_sm = (K <= 32 && AngShape<LMAX, BASIS>::D <= 20) ? 2 : 1;
     const int64_t tiles_max = (k.n + F64_TILE - 1) / F64_TILE + k.n_species;
     const int blocks = (int)std::min<int64_t>(tiles_max, (int64_t)per_sm * c->n_sm);
     cudaEventRecord(start, s);
-    k_mega_f64<K, LMAX><<<blocks, F64_TILE * 32, smem_bytes, s>>>(k);
+    k_mega_f64<K, LMAX, BASIS><<<blocks, F64_TILE * 32, smem_bytes, s>>>(k);
     cudaEventRecord(stop, s);
     return cudaGetLastError();
 }
 
-bool f64_shape_supported(int k, int l_max) { return (k == 16 || k == 32 || k == 64) && l_max >= 1 && l_max <= 3; }
+bool f64_shape_supported(int k, int l_max, int basis) {
+    if (basis == 0 && (k == 16 || k == 32 || k == 64) && l_max >= 1 && l_max <= 3) return true;
+    if (basis == 0 && k == 32 && (l_max == 4 || l_max == 5)) return true;
+    if (basis == 1 && (k == 32 || k == 64) && l_max >= 1 && l_max <= 3) return true;
+    return false;
+}
 
 int launch_megakernel_f64(mlip_ctx *c, cudaStream_t s) {
     const int64_t n = c->n;
@@ -467,11 +500,14 @@ int launch_megakernel_f64(mlip_ctx *c, cudaStream_t s) {
     const int slot = (int)(c->ev_count % mlip_ctx::EV_POOL);
     cudaEvent_t e0 = c->ev[2 * slot], e1 = c->ev[2 * slot + 1];
     cudaError_t e = cudaErrorInvalidValue;
-    switch (c->cfg.k * 10 + c->cfg.l_max) {
-#define MLIP_F64_CASE(K, L) case K * 10 + L: e = launch_shape<K, L>(c, k, s, e0, e1); break;
-        MLIP_F64_CASE(16, 1) MLIP_F64_CASE(16, 2) MLIP_F64_CASE(16, 3)
-        MLIP_F64_CASE(32, 1) MLIP_F64_CASE(32, 2) MLIP_F64_CASE(32, 3)
-        MLIP_F64_CASE(64, 1) MLIP_F64_CASE(64, 2) MLIP_F64_CASE(64, 3)
+    switch (c->cfg.basis * 1000 + c->cfg.k * 10 + c->cfg.l_max) {
+#define MLIP_F64_CASE(K, L, B) case B * 1000 + K * 10 + L: e = launch_shape<K, L, B>(c, k, s, e0, e1); break;
+        MLIP_F64_CASE(16, 1, 0) MLIP_F64_CASE(16, 2, 0) MLIP_F64_CASE(16, 3, 0)
+        MLIP_F64_CASE(32, 1, 0) MLIP_F64_CASE(32, 2, 0) MLIP_F64_CASE(32, 3, 0)
+        MLIP_F64_CASE(64, 1, 0) MLIP_F64_CASE(64, 2, 0) MLIP_F64_CASE(64, 3, 0)
+        MLIP_F64_CASE(32, 4, 0) MLIP_F64_CASE(32, 5, 0)
+        MLIP_F64_CASE(32, 1, 1) MLIP_F64_CASE(32, 2, 1) MLIP_F64_CASE(32, 3, 1)
+        MLIP_F64_CASE(64, 1, 1) MLIP_F64_CASE(64, 2, 1) MLIP_F64_CASE(64, 3, 1)
 #undef MLIP_F64_CASE
     }
     MLIP_CUDA_TRY(c, e);

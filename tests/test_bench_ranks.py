@@ -88,6 +88,12 @@ def test_every_flag_combination_sets_up_its_problem_without_a_gpu():
                 assert prob["flop_pair"] > 0 and prob["flop_atom"] > 0
                 if (k, lmax) == (32, 3):
                     assert prob["flop_pair"] == bench.FLOP_PER_PAIR and prob["flop_atom"] == bench.FLOP_PER_ATOM
+    # the angular ablation's shapes: canonical basis and the higher orders
+    can = bench.problem_setup(_args("--cells", "4", "--precision", "f64", "--basis", "canonical"))
+    irr = bench.problem_setup(_args("--cells", "4", "--precision", "f64"))
+    assert can["basis"] == 1 and can["flop_pair"] > irr["flop_pair"] and can["head"].size == irr["head"].size
+    l5 = bench.problem_setup(_args("--cells", "4", "--precision", "f64", "--lmax", "5"))
+    assert l5["head"].size == 6 * wl.head_net_size(6 * 32) and l5["flop_pair"] > can["flop_pair"]
     # the general count reduces to the default one at the default shape
     d, n_inv = 16, 128
     assert abs((60 + 150 + 512 + 6 * d * 32 + 168) - bench.FLOP_PER_PAIR) < 5

@@ -124,6 +124,42 @@ def test_fp64_descriptor_shape_variants_match_oracle(k, l_max):
     assert np.abs(out["virial"].cpu().numpy().reshape(3, 3) - ref["virial"]).max() <= 1e-9 * np.abs(ref["virial"]).max()
 
 
+@pytest.mark.parametrize("k,l_max,basis", [(32, 4, 0), (32, 5, 0), (32, 1, 1), (32, 2, 1), (32, 3, 1), (64, 3, 1)])
+def test_fp64_higher_orders_and_the_canonical_basis_match_oracle(k, l_max, basis):
+    """l_max = 4, 5 (d = 25, 36: Table 4, Fig. 4(c)) through projection matrices built on the host, and the canonical
+    monomial basis (d = 4, 10, 20) with the multiplicity metric of Eq. 5 -- the descriptor before the irreducible reduction
+    (Table 7).  The library's Q_l differ from the oracle's by a rotation of their rows; the invariants do not."""
+    import paper_2608_16329_b200 as mlip
+    import workloads as wl
+    C = 3
+    w = wl.make_workload(3, n_cells=5)
+    enc, head = wl.make_weights(C, 78, wl.ENC_OUT_SCALE[3], wl.HEAD_OUT_SCALE[3], k=k, l_max=l_max)
+    model = oracle.Model(C, w.r_cut, enc, head, k=k, l_max=l_max, basis=basis)
+    pot = mlip.Potential(C, w.r_cut, 1.0, enc, head, w.masses, precision=1, k=k, l_max=l_max, basis=basis)
+    pot.build_neighbors(w.pos, w.species, w.box)
+    out = pot.compute(want_e_atom=True)
+    pot.sync_status()
+    ref = oracle.evaluate(model, w.pos, w.species, w.box)
+    e = float(out["energy"].cpu())
+    f = out["forces"].cpu().numpy()
+    print(f"k={k} l_max={l_max} basis={basis}: rel dE={abs(e - ref['energy']) / abs(ref['energy']):.2e} max|dF|={np.abs(f - ref['forces']).max():.2e}")
+    scale = max(1.0, float(np.abs(ref["forces"]).max()))
+    assert abs(e - ref["energy"]) <= E_RTOL_F64 * abs(ref["energy"])
+    assert np.abs(f - ref["forces"]).max() <= F_ATOL_F64 * scale
+    assert np.abs(out["e_atom"].cpu().numpy() - ref["e_atom"]).max() <= 1e-9 * max(1.0, np.abs(ref["e_atom"]).max())
+    assert np.abs(out["virial"].cpu().numpy().reshape(3, 3) - ref["virial"]).max() <= 1e-9 * np.abs(ref["virial"]).max()
+
+
+def test_shapes_outside_the_compiled_set_are_refused():
+    import paper_2608_16329_b200 as mlip
+    import workloads as wl
+    for k, l_max, basis, precision in [(32, 3, 1, 0), (16, 3, 1, 1), (64, 5, 0, 1), (32, 4, 1, 1)]:
+        enc, head = wl.make_weights(1, 3, k=k, l_max=l_max)
+        with pytest.raises(mlip.MlipError) as err:
+            mlip.Potential(1, 6.0, 1.0, enc, head, np.array([50.0]), k=k, l_max=l_max, basis=basis, precision=precision)
+        assert err.value.code == mlip.binding.CODES["MLIP_ERR_UNSUPPORTED"]
+
+
 def test_other_shapes_are_refused_by_the_fp32_path():
     import paper_2608_16329_b200 as mlip
     import workloads as wl
