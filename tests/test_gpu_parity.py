@@ -453,3 +453,32 @@ def test_in_step_rebuild_with_lists_longer_than_the_hit_buffer():
     nl = oracle.neighbors(pos.cpu().numpy(), w.species, w.n_species, w.box, w.r_cut + 2.5)
     assert nl.nbr.size / w.n_atoms > 200
     assert canonical_equal(nl, seg, nbr)
+
+
+def test_saturated_head_activations_match_oracle():
+    """First-layer pre-activations of the regression network of order 25 (some beyond 60): SiLU runs on the fast
+    exponential, whose error grows with |x| while the sigmoid saturates; E_i and forces must still agree."""
+    import paper_2608_16329_b200 as mlip
+    import workloads as wl
+    w = wl.make_workload(1)
+    enc, head = wl.workload_weights(1, w.n_species)
+    nets = head.reshape(w.n_species, wl.head_net_size(128)).copy()
+    nets[:, :64 * 128 + 64] *= 25.0                                   # W1 and b1 of every species' network
+    head_big = nets.ravel()
+    model = oracle.Model(w.n_species, w.r_cut, enc, head_big)
+    nl = oracle.neighbors(w.pos, w.species, w.n_species, w.box, w.r_cut)
+    G = oracle.compute(model, w.pos, w.species, w.box, nl, want_G=True)["G"]
+    pre = np.array([nets[s, :64 * 128].reshape(64, 128) @ G[i] + nets[s, 64 * 128:64 * 128 + 64] for i, s in enumerate(w.species)])
+    assert 10 < np.abs(pre).mean() < 60 and np.abs(pre).max() > 60
+    pot = mlip.Potential(w.n_species, w.r_cut, 0.0, enc, head_big, w.masses)
+    pot.build_neighbors(w.pos, w.species, w.box)
+    out = pot.compute(want_e_atom=True)
+    pot.sync_status()
+    ref = oracle.evaluate(model, w.pos, w.species, w.box)
+    f_scale = max(1.0, float(np.sqrt((ref["forces"] ** 2).sum(1).mean())))
+    e_scale = max(1.0, float(np.abs(ref["e_atom"]).max()))
+    print(f"saturated head: mean|pre|={np.abs(pre).mean():.1f} max={np.abs(pre).max():.0f} rms|F|={f_scale:.1f} "
+          f"max|dF|={np.abs(out['forces'].cpu().numpy() - ref['forces']).max():.2e} max|dE_i|={np.abs(out['e_atom'].cpu().numpy() - ref['e_atom']).max():.2e}")
+    assert abs(float(out["energy"].cpu()) - ref["energy"]) <= E_RTOL * np.abs(ref["e_atom"]).sum()
+    assert np.abs(out["e_atom"].cpu().numpy() - ref["e_atom"]).max() <= 2e-5 * e_scale
+    assert np.abs(out["forces"].cpu().numpy() - ref["forces"]).max() <= F_ATOL * f_scale
