@@ -23,7 +23,8 @@
  *   - Units: Angstrom, eV, amu, fs.  Atom order of every array argument is the
  *     caller's; the library keeps its own cell-sorted order internally.
  *   - The fp32 path is compiled for k = 32 radial channels and l_max = 3 (d = 16), the paper's production
- *     shape; the fp64 path (precision = 1) also for k in {16, 32, 64} x l_max in {1, 2, 3}, for k = 32 with
+ *     shape; models with k < 32 or l_max < 3 run in it unchanged in value (their missing channels and orders are
+ *     zero-filled at create time) but at the full shape's cost; the fp64 path (precision = 1) also for k in {16, 32, 64} x l_max in {1, 2, 3}, for k = 32 with
  *     l_max = 4, 5 (d = 25, 36), and for the canonical angular basis (config.basis = 1) with k in {32, 64}.  The
  *     encoder is 1 -> enc_hidden x enc_layers -> k, the head is
  *     (l_max+1) k -> head_hidden x head_layers -> 1 with head_hidden = 64,
@@ -62,8 +63,8 @@ typedef struct {
     int n_species;        /* C, 1..8 */
     double r_cut;         /* Angstrom */
     double skin;          /* list radius = r_cut + skin */
-    int k;                /* 32 (precision 1: 16, 32 or 64) */
-    int l_max;            /* 3 (precision 1: 1 .. 5, see above) */
+    int k;                /* 1 .. 32 (precision 1: 16, 32 or 64) */
+    int l_max;            /* 0 .. 3 (precision 1: 1 .. 5, see above) */
     int enc_hidden, enc_layers;    /* e.g. 128, 3 */
     int head_hidden, head_layers;  /* 64, 4 */
     int table_knots;      /* intervals of the radial table on [table_r_min, r_cut]; 0 = automatic: 64, doubled until table_tol holds */

@@ -136,8 +136,9 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
         if (!f64_shape_supported(cfg->k, cfg->l_max, cfg->basis))
             return fail(nullptr, MLIP_ERR_UNSUPPORTED, "the fp64 path is compiled for the irreducible basis with k in {16, 32, 64} x l_max in {1, 2, 3} and "
                                                        "k = 32 x l_max in {4, 5}, and for the canonical basis with k in {32, 64} x l_max in {1, 2, 3}");
-    } else if (cfg->k != K_RADIAL || cfg->l_max != 3 || cfg->basis != 0) {
-        return fail(nullptr, MLIP_ERR_UNSUPPORTED, "the fp32 path is compiled for k = 32, l_max = 3, irreducible basis only (other shapes: precision = 1)");
+    } else if (cfg->k < 1 || cfg->k > K_RADIAL || cfg->l_max < 0 || cfg->l_max > 3 || cfg->basis != 0) {
+        return fail(nullptr, MLIP_ERR_UNSUPPORTED, "the fp32 path is compiled for k = 32, l_max = 3, irreducible basis (smaller k and l_max run in that "
+                                                   "shape with the missing channels and orders zero); other shapes: precision = 1");
     }
     if (cfg->head_hidden != HEAD_H || cfg->head_layers != HEAD_L) return fail(nullptr, MLIP_ERR_UNSUPPORTED, "only a 4 x 64 head is compiled in");
     if (cfg->enc_hidden < 1 || cfg->enc_layers < 1) return fail(nullptr, MLIP_ERR_INVALID_ARG, "bad encoder shape");
@@ -178,10 +179,45 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
     for (int s = 0; s < cfg->n_species; ++s)
         if (!(mass[s] > 0.0)) return fail(nullptr, MLIP_ERR_INVALID_ARG, "mass must be positive");
     if (cfg->precision != 0 && cfg->precision != 1) return fail(nullptr, MLIP_ERR_INVALID_ARG, "precision must be 0 (fp32) or 1 (fp64)");
+    // fp32 path, descriptor smaller than the compiled shape (k < 32 or l_max < 3): the fused kernel runs its own shape with
+    // the extra radial channels identically zero (zero output rows of every encoder) and the extra invariants unused
+    // (zero columns in the regression networks' first layer).  Same function, no saving in time: the throughput side of
+    // the k and l_max ablations is measured on the fp64 kernel, which is compiled per shape.
+    std::vector<double> enc_pad, head_pad;
+    mlip_config padded = *cfg;
+    if (cfg->precision == 0 && (cfg->k < K_RADIAL || cfg->l_max < 3)) {
+        const int k = cfg->k, H = cfg->enc_hidden;
+        const size_t trunk = enc_net - ((size_t)k * H + k), enc_net32 = trunk + (size_t)K_RADIAL * H + K_RADIAL;
+        const size_t head_tail = head_net - (size_t)HEAD_H * (cfg->l_max + 1) * k, head_net128 = head_tail + (size_t)HEAD_H * N_INV;
+        try {
+            enc_pad.assign((size_t)C * C * enc_net32, 0.0);
+            head_pad.assign((size_t)C * head_net128, 0.0);
+        } catch (const std::bad_alloc &) {
+            return fail(nullptr, MLIP_ERR_OOM, "host allocation failed");
+        }
+        for (int n = 0; n < C * C; ++n) {
+            const double *src = enc_w + (size_t)n * enc_net;
+            double *dst = &enc_pad[(size_t)n * enc_net32];
+            memcpy(dst, src, sizeof(double) * trunk);
+            memcpy(dst + trunk, src + trunk, sizeof(double) * (size_t)k * H);                               // W_out rows 0 .. k-1
+            memcpy(dst + trunk + (size_t)K_RADIAL * H, src + trunk + (size_t)k * H, sizeof(double) * k);    // b_out
+        }
+        for (int n = 0; n < C; ++n) {
+            const double *src = head_w + (size_t)n * head_net;
+            double *dst = &head_pad[(size_t)n * head_net128];
+            for (int o = 0; o < HEAD_H; ++o)
+                for (int l = 0; l <= cfg->l_max; ++l)
+                    memcpy(dst + (size_t)o * N_INV + (size_t)l * K_RADIAL, src + (size_t)o * (cfg->l_max + 1) * k + (size_t)l * k, sizeof(double) * k);
+            memcpy(dst + (size_t)HEAD_H * N_INV, src + (size_t)HEAD_H * (cfg->l_max + 1) * k, sizeof(double) * head_tail);
+        }
+        enc_w = enc_pad.data(); n_enc = enc_pad.size();
+        head_w = head_pad.data();
+        padded.k = K_RADIAL; padded.l_max = 3;
+    }
 
     mlip_ctx *c = new (std::nothrow) mlip_ctx();
     if (!c) return fail(nullptr, MLIP_ERR_OOM, "host allocation failed");
-    c->cfg = *cfg;
+    c->cfg = padded;
     const bool auto_knots = c->cfg.table_knots <= 0;
     const bool f64 = c->cfg.precision == 1;
     if (auto_knots) c->cfg.table_knots = f64 ? 512 : 64;

@@ -100,8 +100,14 @@ __device__ __forceinline__ void dmma(double &c0, double &c1, double a, double b)
     asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};" : "+d"(c0), "+d"(c1) : "d"(a), "d"(b));
 }
 
+#ifndef MLIP_F64_TWO_PER_SM_MAX_D
+#define MLIP_F64_TWO_PER_SM_MAX_D 20
+#endif
 template <int K, int LMAX, int BASIS>
-__global__ void __launch_bounds__(F64_TILE * 32, (K <= 32 && AngShape<LMAX, BASIS>::D <= 20) ? 2 : 1) k_mega_f64(F64Args k) {
+constexpr int f64_ctas_per_sm() { return (K <= 32 && AngShape<LMAX, BASIS>::D <= MLIP_F64_TWO_PER_SM_MAX_D) ? 2 : 1; }
+
+template <int K, int LMAX, int BASIS>
+__global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>()) k_mega_f64(F64Args k) {
     using SM = TileSmem<K, LMAX, BASIS>;
     using Shape = AngShape<LMAX, BASIS>;
     constexpr int D = SM::D, NINV = SM::NINV;
@@ -468,7 +474,7 @@ static cudaError_t launch_shape(mlip_ctx *c, const F64Args &k, cudaStream_t s, c
         }
         c->kernel_ready = true;
     }
-    const int per_sm = (K <= 32 && AngShape<LMAX, BASIS>::D <= 20) ? 2 : 1;
+    const int per_sm = f64_ctas_per_sm<K, LMAX, BASIS>();
     const int64_t tiles_max = (k.n + F64_TILE - 1) / F64_TILE + k.n_species;
     const int blocks = (int)std::min<int64_t>(tiles_max, (int64_t)per_sm * c->n_sm);
     cudaEventRecord(start, s);

@@ -33,11 +33,11 @@ def test_argument_checks_need_no_device():
     lib = mlip.binding.lib()
     assert lib.mlip_create(None, None, None, 0, None, 0, None) == mlip.binding.CODES["MLIP_ERR_INVALID_ARG"]
     assert lib.mlip_compute(None, None, None, None, None, None) == mlip.binding.CODES["MLIP_ERR_INVALID_ARG"]
-    cfg = mlip.binding.Config(6, 6.0, 1.0, 16, 3, 128, 3, 64, 4, 0, 0.0, 0.0, 0)
+    cfg = mlip.binding.Config(6, 6.0, 1.0, 64, 3, 128, 3, 64, 4, 0, 0.0, 0.0, 0)
     import numpy as np
     ctx = ctypes.c_void_p(0)
     w = np.zeros(8)
     rc = lib.mlip_create(ctypes.byref(ctx), ctypes.byref(cfg), w.ctypes.data_as(ctypes.c_void_p), ctypes.c_size_t(8),
                          w.ctypes.data_as(ctypes.c_void_p), ctypes.c_size_t(8), w.ctypes.data_as(ctypes.c_void_p))
-    assert rc == mlip.binding.CODES["MLIP_ERR_UNSUPPORTED"] and not ctx.value     # k = 16 is not compiled in
+    assert rc == mlip.binding.CODES["MLIP_ERR_UNSUPPORTED"] and not ctx.value     # k = 64 is not compiled into the fp32 path
     assert b"k = 32" in lib.mlip_last_error(None)

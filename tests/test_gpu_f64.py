@@ -163,7 +163,7 @@ def test_shapes_outside_the_compiled_set_are_refused():
 def test_other_shapes_are_refused_by_the_fp32_path():
     import paper_2608_16329_b200 as mlip
     import workloads as wl
-    enc, head = wl.make_weights(1, 3, k=16, l_max=3)
+    enc, head = wl.make_weights(1, 3, k=64, l_max=3)
     with pytest.raises(mlip.MlipError) as err:
-        mlip.Potential(1, 6.0, 1.0, enc, head, np.array([50.0]), k=16, l_max=3)
+        mlip.Potential(1, 6.0, 1.0, enc, head, np.array([50.0]), k=64, l_max=3)
     assert err.value.code == mlip.binding.CODES["MLIP_ERR_UNSUPPORTED"]

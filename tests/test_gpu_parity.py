@@ -482,3 +482,24 @@ def test_saturated_head_activations_match_oracle():
     assert abs(float(out["energy"].cpu()) - ref["energy"]) <= E_RTOL * np.abs(ref["e_atom"]).sum()
     assert np.abs(out["e_atom"].cpu().numpy() - ref["e_atom"]).max() <= 2e-5 * e_scale
     assert np.abs(out["forces"].cpu().numpy() - ref["forces"]).max() <= F_ATOL * f_scale
+
+
+@pytest.mark.parametrize("k,l_max", [(16, 3), (32, 1), (32, 2), (16, 2), (8, 0)])
+def test_smaller_descriptor_shapes_run_in_the_fp32_kernel(k, l_max):
+    """Models with fewer radial channels or a lower angular order than the compiled shape (k = 32, l_max = 3) are
+    zero-filled at create time; the result is that of the smaller model."""
+    import paper_2608_16329_b200 as mlip
+    import workloads as wl
+    C = 3
+    w = wl.make_workload(3, n_cells=5)
+    enc, head = wl.make_weights(C, 91, wl.ENC_OUT_SCALE[3], wl.HEAD_OUT_SCALE[3], k=k, l_max=l_max)
+    model = oracle.Model(C, w.r_cut, enc, head, k=k, l_max=l_max)
+    pot = mlip.Potential(C, w.r_cut, 1.0, enc, head, w.masses, k=k, l_max=l_max)
+    pot.build_neighbors(w.pos, w.species, w.box)
+    out = pot.compute(want_e_atom=True)
+    pot.sync_status()
+    ref = oracle.evaluate(model, w.pos, w.species, w.box)
+    f_scale = max(1.0, float(np.abs(ref["forces"]).max()))
+    assert abs(float(out["energy"].cpu()) - ref["energy"]) <= E_RTOL * abs(ref["energy"])
+    assert np.abs(out["forces"].cpu().numpy() - ref["forces"]).max() <= F_ATOL * f_scale
+    assert np.abs(out["e_atom"].cpu().numpy() - ref["e_atom"]).max() <= 2e-5 * max(1.0, np.abs(ref["e_atom"]).max())
