@@ -596,6 +596,7 @@ int mlip_sync_status(mlip_ctx *c) {
     if (f & FLAG_NONFINITE) return fail(c, MLIP_ERR_NONFINITE, "non-finite or out-of-box position, or species out of range");
     if (f & FLAG_NEIGHBOR_OVERFLOW) return fail(c, MLIP_ERR_NEIGHBOR_OVERFLOW, "neighbor list capacity exceeded during a rebuild");
     if (f & FLAG_SKIN_EXCEEDED) return fail(c, MLIP_ERR_SKIN_EXCEEDED, "an atom moved more than skin/2 since the last list build");
+    if (f & FLAG_BOUNDS) return fail(c, MLIP_ERR_CUDA, "range-checked build: an index left its array");
     if (f & FLAG_TABLE_RANGE) return fail(c, MLIP_ERR_TABLE_RANGE, "a pair came closer than table_r_min");
     return MLIP_OK;
 }

@@ -30,7 +30,17 @@ enum : int {
     FLAG_SKIN_EXCEEDED = 1 << 1,
     FLAG_NONFINITE = 1 << 2,
     FLAG_TABLE_RANGE = 1 << 3,
+    FLAG_BOUNDS = 1 << 4,   // raised only by builds with -DMLIP_DEBUG_BOUNDS: an index left its array
 };
+
+// Range-checked build (-DMLIP_DEBUG_BOUNDS): every index that the fused kernels and the export take from a list or an
+// order array is compared with its array's size before it is used; an index out of range raises FLAG_BOUNDS and is
+// replaced by 0, so the access still happens inside the array.  Stands in for a memory checker on the kernels' gathers.
+#ifdef MLIP_DEBUG_BOUNDS
+#define MLIP_CHECK_INDEX(idx, size, status) (((unsigned long long)(idx) < (unsigned long long)(size)) ? (idx) : (atomicOr((status), FLAG_BOUNDS), 0))
+#else
+#define MLIP_CHECK_INDEX(idx, size, status) (idx)
+#endif
 
 // accumulator slots (double)
 enum : int { ACC_ENERGY = 0, ACC_VIRIAL = 1, ACC_KINETIC = 10, ACC_COUNT = 32 };

@@ -219,6 +219,7 @@ struct KernelArgs {
     const int32_t *nbr_near;   // leading entries of each list that can be inside r_cut while far_flag is down
     const int *far_flag;
     const int32_t *nbr;
+    int64_t nbr_cap;           // entries the list array holds (range-checked builds)
     const float *head_pack;
     float4 *force;
     long long *force_fx;   // deterministic mode: forces as 2^-32 eV/Angstrom integers [N][3]
@@ -262,7 +263,8 @@ __device__ __forceinline__ int collect_pairs_n(const KernelArgs &k, const double
 #pragma unroll
         for (int c = 0; c < SCAN_CHUNKS; ++c) {
             const int64_t e = cur + 32 * c + lane;
-            jj[c] = e < end ? (e - beg < n_pref ? sidx[e - beg] : __ldg(k.nbr + e)) : -1;
+            jj[c] = e < end ? (e - beg < n_pref ? sidx[e - beg] : __ldg(k.nbr + MLIP_CHECK_INDEX(e, k.nbr_cap, k.status))) : -1;
+            if (jj[c] >= 0) jj[c] = (int)MLIP_CHECK_INDEX(jj[c], k.n, k.status);
         }
         double4 pp[SCAN_CHUNKS];
 #pragma unroll
@@ -966,7 +968,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
                     end = beg + pf[PF_IDX + 3];
                     n_pref = min(PF_IDX, pf[PF_IDX + 3]);
                 } else {
-                    i = __ldg(k.center_order + first + wg);
+                    i = (int)MLIP_CHECK_INDEX(__ldg(k.center_order + first + wg), k.n, k.status);
                     beg = k.nbr_off[i]; end = use_far ? k.nbr_off[i + 1] : beg + k.nbr_near[i];
                 }
                 pi = load_pos4(k.pos4 + i);
@@ -1169,7 +1171,7 @@ int launch_megakernel(mlip_ctx *c, cudaStream_t s) {
     KernelArgs k;
     k.n = n; k.n_species = c->cfg.n_species; k.grid = c->grid; k.rc2 = c->cfg.r_cut * c->cfg.r_cut; k.tab = c->tab;
     k.pos4 = c->pos4; k.center_order = c->center_order; k.species_start = c->species_start;
-    k.nbr_off = c->nbr_off; k.nbr_near = c->nbr_near; k.far_flag = c->far_flag; k.nbr = c->nbr; k.head_pack = c->head_w; k.force = c->force; k.e_atom = c->e_atom;
+    k.nbr_off = c->nbr_off; k.nbr_near = c->nbr_near; k.far_flag = c->far_flag; k.nbr = c->nbr; k.nbr_cap = c->nbr_cap; k.head_pack = c->head_w; k.force = c->force; k.e_atom = c->e_atom;
     k.force_fx = c->force_fx; k.acc_fx = c->acc_fx;
     k.acc = c->acc; k.pair_counter = c->pair_counter; k.status = c->status; k.tile_counter = c->tile_counter;
     const int slot = (int)(c->ev_count % mlip_ctx::EV_POOL);

@@ -81,6 +81,7 @@ struct F64Args {
     const int32_t *nbr_near;   // leading entries of each list that can be inside r_cut while far_flag is down
     const int *far_flag;
     const int32_t *nbr;
+    int64_t nbr_cap;           // entries the list array holds (range-checked builds)
     const double *head;
     double *force;      // [N][3]
     double *e_atom;
@@ -145,7 +146,7 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
         double4 pi = make_double4(0.0, 0.0, 0.0, 0.0);
         int64_t beg = 0, end = 0;
         if (have) {
-            i = k.center_order[slot];
+            i = (int)MLIP_CHECK_INDEX(k.center_order[slot], k.n, k.status);
             pi = k.pos4[i];
             beg = k.nbr_off[i]; end = use_far ? k.nbr_off[i + 1] : beg + k.nbr_near[i];
         }
@@ -160,7 +161,7 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
             const int64_t e = base + lane;
             bool valid = false;
             if (e < end) {
-                const int j = k.nbr[e];
+                const int j = (int)MLIP_CHECK_INDEX(k.nbr[MLIP_CHECK_INDEX(e, k.nbr_cap, k.status)], k.n, k.status);
                 const double4 pj = k.pos4[j];
                 const double dx = min_image(pj.x - pi.x, k.grid.box[0], k.grid.half[0]);
                 const double dy = min_image(pj.y - pi.y, k.grid.box[1], k.grid.half[1]);
@@ -310,7 +311,7 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                 bool valid = false;
                 int j = 0;
                 if (e < end) {
-                    j = k.nbr[e];
+                    j = (int)MLIP_CHECK_INDEX(k.nbr[MLIP_CHECK_INDEX(e, k.nbr_cap, k.status)], k.n, k.status);
                     const double4 pj = k.pos4[j];
                     const double dx = min_image(pj.x - pi.x, k.grid.box[0], k.grid.half[0]);
                     const double dy = min_image(pj.y - pi.y, k.grid.box[1], k.grid.half[1]);
@@ -500,7 +501,7 @@ int launch_megakernel_f64(mlip_ctx *c, cudaStream_t s) {
     k.coef = c->table_d; k.knots = c->cfg.table_knots; k.r_min = c->cfg.table_r_min;
     k.inv_h = c->cfg.table_knots / (c->cfg.r_cut - c->cfg.table_r_min);
     k.pos4 = c->pos4; k.center_order = c->center_order; k.species_start = c->species_start;
-    k.nbr_off = c->nbr_off; k.nbr_near = c->nbr_near; k.far_flag = c->far_flag; k.nbr = c->nbr;
+    k.nbr_off = c->nbr_off; k.nbr_near = c->nbr_near; k.far_flag = c->far_flag; k.nbr = c->nbr; k.nbr_cap = c->nbr_cap;
     k.head = c->head_w_d; k.force = c->force_d; k.e_atom = c->e_atom_d; k.acc = c->acc;
     k.pair_counter = c->pair_counter; k.status = c->status;
     const int slot = (int)(c->ev_count % mlip_ctx::EV_POOL);
