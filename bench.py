@@ -98,6 +98,8 @@ def parse_args():
     ap.add_argument("--basis", default="irreducible", choices=["irreducible", "canonical"],
                     help="canonical = all Cartesian monomials with the multiplicity metric, the descriptor before the "
                          "irreducible reduction (d = 20 at l_max = 3): --precision f64 only")
+    ap.add_argument("--list16", action="store_true",
+                    help="list_format = 1: neighbor lists as 16-bit cell-relative codes (half the list bytes): an extra data point")
     ap.add_argument("--sweep", default="", help="comma-separated FCC cell counts: size sweep of the 6-species workload "
                     "(inputs generated on the device), one JSON line per size; not the contract line")
     return ap.parse_args()
@@ -306,7 +308,7 @@ def run_sweep(args):
             pos -= torch.floor(pos / (cells * a)) * (cells * a)
             pos.clamp_(0.0, float(np.nextafter(cells * a, 0.0)))
             species = torch.randint(0, 6, (n,), generator=gen, device=dev, dtype=torch.int32)
-            pot = mlip.Potential(6, 6.0, 1.0, enc, head, masses)
+            pot = mlip.Potential(6, 6.0, 1.0, enc, head, masses, list_format=1 if args.list16 else 0)
             pot.n = n
             mlip.mlip_build_neighbors(pot.ctx, pos, species, box)
             sig = torch.sqrt(torch.tensor(wl.KB_EV_PER_K * 300.0 * wl.ACC_UNIT / masses, device=dev))[species.long()]
@@ -371,7 +373,8 @@ def main():
     w, enc, head, default_shape, rebuild_every, f64 = (prob[q] for q in ("w", "enc", "head", "default_shape", "rebuild_every", "f64"))
     n = w.n_atoms
     pot = mlip.Potential(w.n_species, w.r_cut, w.skin, enc, head, w.masses, device=local_rank, precision=1 if f64 else 0,
-                         k=args.k, l_max=args.lmax, force_mode=1 if args.deterministic else 0, basis=prob["basis"])
+                         k=args.k, l_max=args.lmax, force_mode=1 if args.deterministic else 0, basis=prob["basis"],
+                         list_format=1 if args.list16 else 0)
     table_err = mlip.mlip_table_error(pot.ctx)
 
     # ---- device-resident run: inputs already in HBM when timing starts ----
@@ -462,7 +465,7 @@ def main():
                     "kernel_share_of_step": k_ms / ms if ms > 0 else None,
                     "flop_per_launch": flop, "pairs_in_cutoff_per_atom": pairs / n, "list_entries_per_atom": entries / n,
                     "hbm_peak_gbs": peaks["hbm_gbs"], "hbm_peak_kind": f"of {peak_kind}"}
-        per_atom, traffic_note = recorded_traffic() if (default_shape and not f64 and cfg == CFG) else (None, "no ncu record for this variant")
+        per_atom, traffic_note = recorded_traffic() if (default_shape and not f64 and cfg == CFG and not args.list16) else (None, "no ncu record for this variant")
         roofline["traffic"] = None if per_atom is None else per_atom * n
         roofline["traffic_source"] = traffic_note
         if clocks and clocks.get("sm_mhz"):
@@ -478,7 +481,8 @@ def main():
                 "config": {"workload": f"cfg{cfg} {w.name}: {n} atoms, {w.n_species} species, r_cut 6 A, skin 1 A, "
                                        f"{args.ensemble.upper()} dt 1 fs, list rebuild every {rebuild_every} steps"
                                        + ("" if default_shape else f", k = {args.k}, l_max = {args.lmax}, {args.basis} basis")
-                                       + (", deterministic force mode" if args.deterministic else ""),
+                                       + (", deterministic force mode" if args.deterministic else "")
+                                       + (", 16-bit neighbor codes" if args.list16 else ""),
                            "atoms_per_gpu": n, "parallelism": "replicas" if world > 1 else "single",
                            "l2": "inputs larger than L2 (positions + lists = %.1f GB per GPU)" % ((32 * n + 4 * entries) / 1e9)},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": counters["launches"] - launches0,

@@ -89,6 +89,11 @@ typedef struct {
                              choice); 1 = canonical: every Cartesian monomial of the unit vector up to degree l_max,
                              d = 4, 10, 20 for l_max = 1, 2, 3 (Eq. 11), with C_l = the multinomial multiplicities in Eq. 5
                              -- the descriptor "before reduction" of Table 7; precision 1 only */
+    int list_format;      /* storage of the neighbor lists, the bulk of the footprint (Section 1 and Fig. 4(b): atoms per GPU
+                             are bounded by memory): 0 = int32 indices, 4 bytes per entry; 1 = 16-bit codes (which of the 27
+                             cells around the atom's own cell, position inside it), 2 bytes per entry + 4 per atom, decoded
+                             inside the kernels; same lists, same results.  Falls back to format 0 on grids with fewer
+                             than three cells along an edge */
 } mlip_config;
 
 /*

@@ -42,7 +42,7 @@ class Config(ctypes.Structure):
                 ("table_knots", ctypes.c_int), ("table_r_min", ctypes.c_double), ("table_tol", ctypes.c_double),
                 ("device", ctypes.c_int), ("precision", ctypes.c_int),
                 ("enc_conditioning", ctypes.c_int), ("head_conditioning", ctypes.c_int), ("force_mode", ctypes.c_int),
-                ("envelope", ctypes.c_int), ("basis", ctypes.c_int)]
+                ("envelope", ctypes.c_int), ("basis", ctypes.c_int), ("list_format", ctypes.c_int)]
 
 
 _lib = None
@@ -277,13 +277,13 @@ class Potential:
 
     def __init__(self, n_species, r_cut, skin, enc_w, head_w, masses, device=0, table_knots=0,
                  table_r_min=0.0, table_tol=0.0, enc_hidden=128, enc_layers=3, allow_table_error=False, precision=0,
-                 enc_conditioning=0, head_conditioning=0, k=32, l_max=3, envelope=0, force_mode=0, basis=0):
+                 enc_conditioning=0, head_conditioning=0, k=32, l_max=3, envelope=0, force_mode=0, basis=0, list_format=0):
         import torch
         self.torch = torch
         self.device = torch.device("cuda", device)
         self.n_species = n_species
         self.cfg = Config(n_species, r_cut, skin, k, l_max, enc_hidden, enc_layers, 64, 4, table_knots, table_r_min,
-                          table_tol, device, precision, enc_conditioning, head_conditioning, force_mode, envelope, basis)
+                          table_tol, device, precision, enc_conditioning, head_conditioning, force_mode, envelope, basis, list_format)
         self.precision = precision
         self.ctx = mlip_create(self.cfg, enc_w, head_w, masses, allow_table_error)
         self.n = 0

@@ -51,6 +51,7 @@ static void free_atoms(mlip_ctx *c) {
     if (c->cfg.precision == 1) { dev_free(c, &c->force_d, 3 * n); dev_free(c, &c->e_atom_d, n); }
     if (c->cfg.force_mode == 1) dev_free(c, &c->force_fx, 3 * n);
     dev_free(c, &c->tile_state, n / 64 + 2);
+    if (c->cfg.list_format == 1) dev_free(c, &c->cell_id, n);
     c->cap_atoms = 0;
 }
 
@@ -76,6 +77,7 @@ static int ensure_capacity(mlip_ctx *c, int64_t n, int64_t n_cells) {
         if (c->cfg.precision == 1) { TRY_ALLOC(c->force_d, 3 * m); TRY_ALLOC(c->e_atom_d, m); }
         if (c->cfg.force_mode == 1) TRY_ALLOC(c->force_fx, 3 * m);
         TRY_ALLOC(c->tile_state, m / 64 + 2);
+        if (c->cfg.list_format == 1) TRY_ALLOC(c->cell_id, m);
         c->cap_atoms = n;
     }
     if (n_cells > c->cap_cells) {
@@ -148,6 +150,7 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
     if (cfg->force_mode < 0 || cfg->force_mode > 1) return fail(nullptr, MLIP_ERR_INVALID_ARG, "force_mode must be 0 (atomics) or 1 (deterministic)");
     if (cfg->force_mode == 1 && cfg->precision == 1) return fail(nullptr, MLIP_ERR_UNSUPPORTED, "the deterministic force mode is compiled for the fp32 path only");
     if (cfg->envelope < 0 || cfg->envelope > 1) return fail(nullptr, MLIP_ERR_INVALID_ARG, "envelope must be 0 (cosine) or 1 (quintic)");
+    if (cfg->list_format < 0 || cfg->list_format > 1) return fail(nullptr, MLIP_ERR_INVALID_ARG, "list_format must be 0 (int32 indices) or 1 (16-bit cell-relative codes)");
     // Species conditioning (Section 3.2.2): the kernels always index C*C encoder tables and C heads; the variants
     // with fewer networks are expanded here by repeating the shared ones.
     const int C = cfg->n_species;

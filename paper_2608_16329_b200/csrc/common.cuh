@@ -111,7 +111,9 @@ struct mlip_ctx {
     int32_t *nbr_near = nullptr;   // [N] leading entries of each list that were within r_cut + skin / 2 at build time
     int *far_flag = nullptr;       // raised once an atom has moved skin / 4 since the build: the far entries count again
     int64_t *nbr_off = nullptr;    // [N + 1]
-    int32_t *nbr = nullptr;
+    int32_t *nbr = nullptr;        // list entries: int32 indices, or uint16 cell-relative codes when list16
+    bool list16 = false;           // format of the current lists (mlip_config.list_format = 1 on a grid of >= 3 cells per edge)
+    int32_t *cell_id = nullptr;    // [N] build-time cell of each atom, internal order (allocated for list_format = 1)
     unsigned long long *tile_state = nullptr;   // [ceil(N / 64) + 1] look-back words of the one-pass rebuild
     int *tile_ticket = nullptr;
     int64_t nbr_cap = 0, n_entries = 0;
@@ -190,6 +192,17 @@ int launch_scatter_forces_f64(mlip_ctx *c, double *forces, double *e_atom, cudaS
 int launch_set_positions(mlip_ctx *c, const double *pos, cudaStream_t s);
 int launch_set_velocities(mlip_ctx *c, const double *vel, cudaStream_t s);
 int launch_get_state(mlip_ctx *c, double *pos, double *vel, cudaStream_t s);
+
+// Compact list entries (neighbor.cu): cell number in the 27-cell traversal order << L16_SHIFT | position inside that cell.
+constexpr int L16_SHIFT = 11, L16_MASK = (1 << L16_SHIFT) - 1;
+__host__ __device__ inline int neighbor_cell(const CellGrid &g, int cid, int it) {
+    const int cz = cid % g.n[2], cy = (cid / g.n[2]) % g.n[1], cx = cid / (g.n[2] * g.n[1]);
+    int x = cx + it / 9 - 1, y = cy + (it / 3) % 3 - 1, z = cz + it % 3 - 1;
+    x = x < 0 ? x + g.n[0] : (x >= g.n[0] ? x - g.n[0] : x);
+    y = y < 0 ? y + g.n[1] : (y >= g.n[1] ? y - g.n[1] : y);
+    z = z < 0 ? z + g.n[2] : (z >= g.n[2] ? z - g.n[2] : z);
+    return (x * g.n[1] + y) * g.n[2] + z;
+}
 
 // Exact minimum-image squared distance in fp64, every operation rounded on its own
 // (no fused multiply-add), identical on host and device.

@@ -70,6 +70,8 @@ constexpr int HB_WORDS = HB_PART + 2 * TILE * Z_STRIDE;
 static_assert(HB_WORDS <= TILE * SCR_WORDS, "head buffers alias the scratch of the group's warps");
 constexpr int HC_WORDS = HEAD_L * HEAD_H + HEAD_H + 16;         // biases, w_out, b_out of the current species
 constexpr int PF_IDX = 160;                                     // neighbor indices prefetched per warp for its next atom
+constexpr int PF_CS = 96;                                       // compact lists: the codes take 81 words at most, the 27 cell bases sit here
+static_assert(PF_IDX / 2 + 1 <= PF_CS && PF_CS + 27 <= PF_IDX, "prefetch buffer layout for compact lists");
 constexpr int PF_WORDS = PF_IDX + 4;                            // + {atom, list start (2 words), list length}
 constexpr int FIXED_WORDS = NG * SX_WORDS + NW * (Q_WORDS + SCR_WORDS + PF_WORDS) + HC_WORDS + 16;
 constexpr int SMEM_LIMIT_WORDS = 227 * 1024 / 4 - 256;
@@ -219,6 +221,9 @@ struct KernelArgs {
     const int32_t *nbr_near;   // leading entries of each list that can be inside r_cut while far_flag is down
     const int *far_flag;
     const int32_t *nbr;
+    const uint16_t *nbr16;     // the same array when the lists hold 16-bit cell-relative codes (L16 instantiations)
+    const int32_t *cell_id;    // build-time cell of each atom (L16)
+    const int32_t *cell_start; // first atom of each cell (L16)
     int64_t nbr_cap;           // entries the list array holds (range-checked builds)
     const float *head_pack;
     float4 *force;
@@ -254,16 +259,28 @@ struct TableView {
 // and advances `cur`.  The first n_pref indices of the list may come from shared memory (sidx).
 constexpr int SCAN_CHUNKS = 5;
 static_assert(SCAN_CHUNKS * 32 <= PB_CAP, "a full group must fit an empty queue");
-template <int SCAN_CHUNKS>
+// Compact lists: lane q < 27 holds the first atom of the q-th cell around atom i's build-time cell; an entry's index is
+// that base (one shuffle) plus the position coded in its low bits.
+__device__ __forceinline__ int cell_base_of_lane(const KernelArgs &k, int i, int lane) {
+    return lane < 27 ? __ldg(k.cell_start + neighbor_cell(k.grid, __ldg(k.cell_id + i), lane)) : 0;
+}
+template <int SCAN_CHUNKS, bool L16>
 __device__ __forceinline__ int collect_pairs_n(const KernelArgs &k, const double4 &pi, int64_t beg, int64_t &cur, int64_t end, float4 *pq, int lane,
-                                               const int *sidx, int n_pref) {
+                                               const int *sidx, int n_pref, int cs) {
     int nq = 0;
     while (cur < end && nq + (int)min((int64_t)(SCAN_CHUNKS * 32), end - cur) <= PB_CAP) {
         int jj[SCAN_CHUNKS];
 #pragma unroll
         for (int c = 0; c < SCAN_CHUNKS; ++c) {
             const int64_t e = cur + 32 * c + lane;
-            jj[c] = e < end ? (e - beg < n_pref ? sidx[e - beg] : __ldg(k.nbr + MLIP_CHECK_INDEX(e, k.nbr_cap, k.status))) : -1;
+            if (L16) {   // (the prefetch copied whole 32-bit words starting at the even entry at or before `beg`)
+                const int code = e < end ? (e - beg < n_pref ? reinterpret_cast<const uint16_t *>(sidx)[(e - beg) + (beg & 1)]
+                                                             : __ldg(k.nbr16 + MLIP_CHECK_INDEX(e, k.nbr_cap, k.status))) : 0;
+                const int base = __shfl_sync(0xffffffffu, cs, code >> L16_SHIFT);
+                jj[c] = e < end ? base + (code & L16_MASK) : -1;
+            } else {
+                jj[c] = e < end ? (e - beg < n_pref ? sidx[e - beg] : __ldg(k.nbr + MLIP_CHECK_INDEX(e, k.nbr_cap, k.status))) : -1;
+            }
             if (jj[c] >= 0) jj[c] = (int)MLIP_CHECK_INDEX(jj[c], k.n, k.status);
         }
         double4 pp[SCAN_CHUNKS];
@@ -290,19 +307,20 @@ __device__ __forceinline__ int collect_pairs_n(const KernelArgs &k, const double
 }
 // Short lists (the usual case while the far entries are skipped) take the three-chunk form: fewer loads in flight,
 // fewer registers.
+template <bool L16>
 __device__ __forceinline__ int collect_pairs(const KernelArgs &k, const double4 &pi, int64_t beg, int64_t &cur, int64_t end, float4 *pq, int lane,
-                                             const int *sidx, int n_pref) {
-    if (end - beg <= 96) return collect_pairs_n<3>(k, pi, beg, cur, end, pq, lane, sidx, n_pref);
-    return collect_pairs_n<5>(k, pi, beg, cur, end, pq, lane, sidx, n_pref);
+                                             const int *sidx, int n_pref, int cs) {
+    if (end - beg <= 96) return collect_pairs_n<3, L16>(k, pi, beg, cur, end, pq, lane, sidx, n_pref, cs);
+    return collect_pairs_n<5, L16>(k, pi, beg, cur, end, pq, lane, sidx, n_pref, cs);
 }
 
 // ---------------- Encoding of one atom: returns the moment as accumulator fragments ----------------
 // `queued` returns the number of pairs left in the queue when the whole list fitted in one round
 // (the derivation then reuses them), or -1.
-template <bool TAB_SMEM>
+template <bool TAB_SMEM, bool L16>
 __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView &tv, const double4 &pi, int64_t beg, int64_t end,
                                            float4 *pq, float *stage, int lane, float (&Pf)[4][4], int &queued, const int *sidx, int n_pref,
-                                           PhaseClock &pc) {
+                                           int cs, PhaseClock &pc) {
     const int g = lane >> 2, t = lane & 3;
     constexpr int rs = TAB_SMEM ? TAB_STRIDE_SMEM : K_RADIAL;   // = tv.row_stride, known here so that row offsets fold into the loads
 #pragma unroll
@@ -416,7 +434,7 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
     int total = 0, rounds = 0, n = 0;
     int64_t cur = beg;
     do {
-        n = collect_pairs(k, pi, beg, cur, end, pq, lane, sidx, n_pref);
+        n = collect_pairs<L16>(k, pi, beg, cur, end, pq, lane, sidx, n_pref, cs);
         pc.mark(0);
         for (int q0 = 0; q0 < n; q0 += 32) batch(q0, min(32, n - q0));
         total += n;
@@ -427,7 +445,7 @@ __device__ __forceinline__ int encode_atom(const KernelArgs &k, const TableView 
 }
 
 // ---------------- Derivation of one atom (Eq. 8-10) ----------------
-template <bool TAB_SMEM, bool DET>
+template <bool TAB_SMEM, bool DET, bool L16>
 __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView &tv, int i,
                                             float4 *pq, float *scr, int queued, int lane, const uint32_t (&Wh)[4][4],
                                             const uint32_t (&Wl)[4][4], float (&vir)[9], PhaseClock &pc) {
@@ -573,8 +591,9 @@ __device__ __forceinline__ void derive_atom(const KernelArgs &k, const TableView
         const double4 pi = load_pos4(k.pos4 + i);
         const int64_t beg = k.nbr_off[i], end = *k.far_flag ? k.nbr_off[i + 1] : beg + k.nbr_near[i];
         int64_t cur = beg;
+        const int cs = L16 ? cell_base_of_lane(k, i, lane) : 0;
         do {
-            const int n = collect_pairs(k, pi, beg, cur, end, pq, lane, nullptr, 0);
+            const int n = collect_pairs<L16>(k, pi, beg, cur, end, pq, lane, nullptr, 0, cs);
             pc.mark(3);
             for (int q0 = 0; q0 < n; q0 += 32) batch(q0, min(32, n - q0));
         } while (cur < end);
@@ -743,19 +762,42 @@ struct NextAtom {
     int i;
     bool use_far;     // the lists' far entries have to be scanned as well
     int64_t beg, end;
+    int cid;          // compact lists: the atom's build-time cell
     __device__ __forceinline__ void stage_a() { if (slot >= 0) i = __ldg(k->center_order + slot); }
+    template <bool L16>
     __device__ __forceinline__ void stage_b() {
-        if (slot >= 0) { beg = __ldg(k->nbr_off + i); end = use_far ? __ldg(k->nbr_off + i + 1) : beg + __ldg(k->nbr_near + i); }
+        if (slot >= 0) {
+            beg = __ldg(k->nbr_off + i); end = use_far ? __ldg(k->nbr_off + i + 1) : beg + __ldg(k->nbr_near + i);
+            if (L16) cid = __ldg(k->cell_id + i);
+        }
     }
+    template <bool L16>
     __device__ __forceinline__ void stage_c(int lane) {
         if (slot < 0) return;
         const int n = (int)min((int64_t)PF_IDX, end - beg);
+        if (L16) {   // codes travel as whole 32-bit words from the even entry at or before `beg`; the 27 cell bases follow them
+            const int odd = (int)(beg & 1), words = (odd + n + 1) >> 1;
+            const int *src = reinterpret_cast<const int *>(k->nbr16 + (beg - odd));
 #pragma unroll
-        for (int c = 0; c < PF_IDX / 32; ++c) {
-            const int e = 32 * c + lane;
-            if (e < n) {
-                const unsigned dst = (unsigned)__cvta_generic_to_shared(sidx + e);
-                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(k->nbr + beg + e) : "memory");
+            for (int c = 0; c < (PF_IDX / 2 + 1 + 31) / 32; ++c) {
+                const int e = 32 * c + lane;
+                if (e < words) {
+                    const unsigned dst = (unsigned)__cvta_generic_to_shared(sidx + e);
+                    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src + e) : "memory");
+                }
+            }
+            if (lane < 27) {
+                const unsigned dst = (unsigned)__cvta_generic_to_shared(sidx + PF_CS + lane);
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(k->cell_start + neighbor_cell(k->grid, cid, lane)) : "memory");
+            }
+        } else {
+#pragma unroll
+            for (int c = 0; c < PF_IDX / 32; ++c) {
+                const int e = 32 * c + lane;
+                if (e < n) {
+                    const unsigned dst = (unsigned)__cvta_generic_to_shared(sidx + e);
+                    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(k->nbr + beg + e) : "memory");
+                }
             }
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
@@ -766,7 +808,7 @@ struct NextAtom {
 // ---------------- Regression (Eq. 6) forward and reverse for the group's tile ----------------
 // In: sX = invariants [atom][128].  Out: sX = dE/dG; per-atom energies written.
 // hc = biases [4][64], w_out [64], b_out of the species in shared memory.  wg = warp within the group.
-template <bool DET>
+template <bool DET, bool L16>
 __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float *hb, const float *hc, uint32_t tm_role, int count, int first,
                                           int group, int wg, int lane, double &e_sum, NextAtom &nx, PhaseClock &pc) {
     float *xs = hb + HB_XS, *zs = hb + HB_ZS, *dp = hb + HB_DP, *part = hb + HB_PART;
@@ -802,8 +844,8 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
         else head_gemm<KS1 / 2, true, true>(c, w, kh * (KS1 / 2), zin, 2 * Z_STRIDE, lane);
         pc.mark(12);
         store_partial(c, part + kh * TILE * Z_STRIDE, Z_STRIDE, mt4, lane);
-        if (L == 0) nx.stage_b();
-        if (L == 1) nx.stage_c(lane);
+        if (L == 0) nx.template stage_b<L16>();
+        if (L == 1) nx.template stage_c<L16>(lane);
         pc.mark(13);
         group_sync(group);
         pc.mark(14);
@@ -874,7 +916,7 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
     group_sync(group);
 }
 
-template <bool TAB_SMEM, bool DET>
+template <bool TAB_SMEM, bool DET, bool L16>
 __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words) {
     extern __shared__ __align__(16) float smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -953,7 +995,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
 
             // ---------------- Encoding + invariants: warp = atom ----------------
             const bool have = wg < count;
-            int i = 0, n_pref = 0;
+            int i = 0, n_pref = 0, cs = 0;
             double4 pi = make_double4(0.0, 0.0, 0.0, 0.0);
             int64_t beg = 0, end = 0;
             float Pf[4][4];
@@ -967,12 +1009,14 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
                     beg = ((int64_t)pf[PF_IDX + 2] << 32) | (unsigned)pf[PF_IDX + 1];
                     end = beg + pf[PF_IDX + 3];
                     n_pref = min(PF_IDX, pf[PF_IDX + 3]);
+                    if (L16) cs = lane < 27 ? pf[PF_CS + lane] : 0;
                 } else {
                     i = (int)MLIP_CHECK_INDEX(__ldg(k.center_order + first + wg), k.n, k.status);
                     beg = k.nbr_off[i]; end = use_far ? k.nbr_off[i + 1] : beg + k.nbr_near[i];
+                    if (L16) cs = cell_base_of_lane(k, i, lane);
                 }
                 pi = load_pos4(k.pos4 + i);
-                n_pairs += encode_atom<TAB_SMEM>(k, tv, pi, beg, end, pq, scr, lane, Pf, queued, pf, n_pref, pc);
+                n_pairs += encode_atom<TAB_SMEM, L16>(k, tv, pi, beg, end, pq, scr, lane, Pf, queued, pf, n_pref, cs, pc);
                 // Eq. 5 (C_l = I): this lane holds rows a = g, g + 8 of channels 8t + j; sum squares over the rows of a block.
                 // Rows 1..3 (l = 1) and 4..7 (l = 2) differ in the top bit of g, so one two-step butterfly over the lower
                 // bits sums both; l = 2 then takes row 8 (held by g = 0) and the upper half's sum, l = 3 is rows 9..15.
@@ -1012,8 +1056,8 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
             NextAtom nx;
             nx.k = &k; nx.sidx = pf; nx.meta = pf + PF_IDX;
             nx.slot = (tile_next < n_tiles && s_beg + tile_next * TILE + wg < s_end) ? s_beg + tile_next * TILE + wg : -1;
-            nx.i = 0; nx.beg = 0; nx.end = 0; nx.use_far = use_far;
-            head_tile<DET>(k, sX, hb, hc, tm_role, count, first, group, wg, lane, e_sum, nx, pc);
+            nx.i = 0; nx.beg = 0; nx.end = 0; nx.use_far = use_far; nx.cid = 0;
+            head_tile<DET, L16>(k, sX, hb, hc, tm_role, count, first, group, wg, lane, e_sum, nx, pc);
             prefetched = nx.slot >= 0;
             pc.mark(9);
 
@@ -1038,7 +1082,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
                     split2_rn(w0, w1, Wh[ks][0], Wh[ks][1], Wl[ks][0], Wl[ks][1]);   // once per atom: the rounded split
                     split2_rn(w2, w3, Wh[ks][2], Wh[ks][3], Wl[ks][2], Wl[ks][3]);
                 }
-                derive_atom<TAB_SMEM, DET>(k, tv, i, pq, scr, queued, lane, Wh, Wl, vir, pc);
+                derive_atom<TAB_SMEM, DET, L16>(k, tv, i, pq, scr, queued, lane, Wh, Wl, vir, pc);
                 if (DET) {   // fold this atom's virial in now: lane sums in a fixed order, then integers
 #pragma unroll
                     for (int q = 0; q < 9; ++q) {
@@ -1161,25 +1205,28 @@ int launch_megakernel(mlip_ctx *c, cudaStream_t s) {
     const bool in_smem = tables_fit_smem(c);
     const int tab_words = in_smem ? table_smem_words(c) : 0;
     const size_t smem_bytes = sizeof(float) * (size_t)(FIXED_WORDS + tab_words);
+    // instantiations: tables in shared / global memory x floating-point / integer scatter x int32 / 16-bit lists
+    using Kernel = void (*)(KernelArgs, int);
+    static const Kernel kernels[8] = {k_mega<false, false, false>, k_mega<false, false, true>, k_mega<false, true, false>, k_mega<false, true, true>,
+                                      k_mega<true, false, false>,  k_mega<true, false, true>,  k_mega<true, true, false>,  k_mega<true, true, true>};
     if (!c->kernel_ready) {
-        const void *fn = in_smem ? (det ? (const void *)k_mega<true, true> : (const void *)k_mega<true, false>)
-                                 : (det ? (const void *)k_mega<false, true> : (const void *)k_mega<false, false>);
-        cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
-        if (e != cudaSuccess) { c->err = std::string("fused kernel shared memory: ") + cudaGetErrorString(e); return MLIP_ERR_CUDA; }
+        for (int q = 0; q < 8; ++q) {
+            const size_t bytes = sizeof(float) * (size_t)(FIXED_WORDS + (q >= 4 ? tab_words : 0));
+            cudaError_t e = cudaFuncSetAttribute((const void *)kernels[q], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+            if (e != cudaSuccess) { c->err = std::string("fused kernel shared memory: ") + cudaGetErrorString(e); return MLIP_ERR_CUDA; }
+        }
         c->kernel_ready = true;
     }
     KernelArgs k;
     k.n = n; k.n_species = c->cfg.n_species; k.grid = c->grid; k.rc2 = c->cfg.r_cut * c->cfg.r_cut; k.tab = c->tab;
     k.pos4 = c->pos4; k.center_order = c->center_order; k.species_start = c->species_start;
-    k.nbr_off = c->nbr_off; k.nbr_near = c->nbr_near; k.far_flag = c->far_flag; k.nbr = c->nbr; k.nbr_cap = c->nbr_cap; k.head_pack = c->head_w; k.force = c->force; k.e_atom = c->e_atom;
+    k.nbr_off = c->nbr_off; k.nbr_near = c->nbr_near; k.far_flag = c->far_flag; k.nbr = c->nbr; k.nbr16 = reinterpret_cast<const uint16_t *>(c->nbr); k.cell_id = c->cell_id; k.cell_start = c->cell_start;
+    k.nbr_cap = c->nbr_cap; k.head_pack = c->head_w; k.force = c->force; k.e_atom = c->e_atom;
     k.force_fx = c->force_fx; k.acc_fx = c->acc_fx;
     k.acc = c->acc; k.pair_counter = c->pair_counter; k.status = c->status; k.tile_counter = c->tile_counter;
     const int slot = (int)(c->ev_count % mlip_ctx::EV_POOL);
     MLIP_CUDA_TRY(c, cudaEventRecord(c->ev[2 * slot], s));
-    if (in_smem && det) k_mega<true, true><<<blocks, NW * 32, smem_bytes, s>>>(k, tab_words);
-    else if (in_smem) k_mega<true, false><<<blocks, NW * 32, smem_bytes, s>>>(k, tab_words);
-    else if (det) k_mega<false, true><<<blocks, NW * 32, smem_bytes, s>>>(k, tab_words);
-    else k_mega<false, false><<<blocks, NW * 32, smem_bytes, s>>>(k, tab_words);
+    kernels[(in_smem ? 4 : 0) + (det ? 2 : 0) + (c->list16 ? 1 : 0)]<<<blocks, NW * 32, smem_bytes, s>>>(k, tab_words);
     if (det) {
         k_fixed_finish<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(n, c->force_fx, c->acc_fx, c->force, c->acc);
         c->launches += 1;

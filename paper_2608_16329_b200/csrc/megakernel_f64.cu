@@ -81,6 +81,8 @@ struct F64Args {
     const int32_t *nbr_near;   // leading entries of each list that can be inside r_cut while far_flag is down
     const int *far_flag;
     const int32_t *nbr;
+    const uint16_t *nbr16;     // non-null: the lists hold 16-bit cell-relative codes (decoded with cell_id / cell_start)
+    const int32_t *cell_id, *cell_start;
     int64_t nbr_cap;           // entries the list array holds (range-checked builds)
     const double *head;
     double *force;      // [N][3]
@@ -150,6 +152,14 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
             pi = k.pos4[i];
             beg = k.nbr_off[i]; end = use_far ? k.nbr_off[i + 1] : beg + k.nbr_near[i];
         }
+        // compact lists: lane q < 27 holds the first atom of the q-th cell around the atom's build-time cell
+        const int cs = (k.nbr16 && have && lane < 27) ? k.cell_start[neighbor_cell(k.grid, k.cell_id[i], lane)] : 0;
+        auto entry = [&](int64_t e, bool live) {   // index of list entry e (every lane of the warp calls this together)
+            if (!k.nbr16) return live ? (int)MLIP_CHECK_INDEX(k.nbr[MLIP_CHECK_INDEX(e, k.nbr_cap, k.status)], k.n, k.status) : 0;
+            const int code = live ? k.nbr16[MLIP_CHECK_INDEX(e, k.nbr_cap, k.status)] : 0;
+            const int base = __shfl_sync(0xffffffffu, cs, code >> L16_SHIFT);
+            return live ? (int)MLIP_CHECK_INDEX(base + (code & L16_MASK), k.n, k.status) : 0;
+        };
 
         // ---------------- Encoding: P = H^T G (Eq. 4), lane = channel ----------------
         double P[D][CPL];
@@ -160,8 +170,9 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
         for (int64_t base = beg; base < end; base += 32) {
             const int64_t e = base + lane;
             bool valid = false;
+            const int j_e = entry(e, e < end);
             if (e < end) {
-                const int j = (int)MLIP_CHECK_INDEX(k.nbr[MLIP_CHECK_INDEX(e, k.nbr_cap, k.status)], k.n, k.status);
+                const int j = j_e;
                 const double4 pj = k.pos4[j];
                 const double dx = min_image(pj.x - pi.x, k.grid.box[0], k.grid.half[0]);
                 const double dy = min_image(pj.y - pi.y, k.grid.box[1], k.grid.half[1]);
@@ -309,9 +320,8 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
             if (base < end) {   // compact the entries inside r_cut into the warp's queue
                 const int64_t e = base + lane;
                 bool valid = false;
-                int j = 0;
+                int j = entry(e, e < end);
                 if (e < end) {
-                    j = (int)MLIP_CHECK_INDEX(k.nbr[MLIP_CHECK_INDEX(e, k.nbr_cap, k.status)], k.n, k.status);
                     const double4 pj = k.pos4[j];
                     const double dx = min_image(pj.x - pi.x, k.grid.box[0], k.grid.half[0]);
                     const double dy = min_image(pj.y - pi.y, k.grid.box[1], k.grid.half[1]);
@@ -501,7 +511,8 @@ int launch_megakernel_f64(mlip_ctx *c, cudaStream_t s) {
     k.coef = c->table_d; k.knots = c->cfg.table_knots; k.r_min = c->cfg.table_r_min;
     k.inv_h = c->cfg.table_knots / (c->cfg.r_cut - c->cfg.table_r_min);
     k.pos4 = c->pos4; k.center_order = c->center_order; k.species_start = c->species_start;
-    k.nbr_off = c->nbr_off; k.nbr_near = c->nbr_near; k.far_flag = c->far_flag; k.nbr = c->nbr; k.nbr_cap = c->nbr_cap;
+    k.nbr_off = c->nbr_off; k.nbr_near = c->nbr_near; k.far_flag = c->far_flag; k.nbr = c->nbr; k.nbr16 = c->list16 ? reinterpret_cast<const uint16_t *>(c->nbr) : nullptr; k.cell_id = c->cell_id; k.cell_start = c->cell_start;
+    k.nbr_cap = c->nbr_cap;
     k.head = c->head_w_d; k.force = c->force_d; k.e_atom = c->e_atom_d; k.acc = c->acc;
     k.pair_counter = c->pair_counter; k.status = c->status;
     const int slot = (int)(c->ev_count % mlip_ctx::EV_POOL);

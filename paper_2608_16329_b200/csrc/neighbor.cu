@@ -16,6 +16,19 @@ __device__ __forceinline__ int cell_coord(double x, double inv_edge, int n) {
     return c < 0 ? 0 : (c >= n ? n - 1 : c);
 }
 
+// ---- compact list format ----
+// With atoms stored in cell order a neighbor j of atom i lies in one of the 27 cells around i's cell, so an entry can
+// be coded in 16 bits: the cell's number in the traversal order (0..26: x, y, z offsets ascending) in the top 5 bits, j's
+// position inside that cell in the low 11 (a cell holds at most MAX_CELL_ATOMS = 1,024 atoms).  Decoding needs the build-time
+// cell of i (cell_id) and the cell starts.  Half the bytes of the int32 list, the bulk of the resident footprint.
+// Used when mlip_config.list_format = 1 and every dimension has at least three cells.
+// One list entry in the format of the output array: the index itself, or its 16-bit code.
+template <typename OUT>
+__device__ __forceinline__ OUT list_entry(int j, int it, int cell_beg) {
+    if (sizeof(OUT) == 2) return (OUT)((it << L16_SHIFT) | (j - cell_beg));
+    return (OUT)j;
+}
+
 __global__ void k_pack_source(const double *__restrict__ pos, const int32_t *__restrict__ species, int64_t n,
                               int n_species, double4 *__restrict__ pos4, int32_t *__restrict__ user, int *status) {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -89,10 +102,11 @@ __global__ void k_sort_cells(int n_cells, int n_species, const int32_t *__restri
 __global__ void k_gather(int64_t n, const int32_t *__restrict__ slot_src, const double4 *__restrict__ pos4_src,
                          const double *__restrict__ vel_src, const int32_t *__restrict__ user_src,
                          double4 *__restrict__ pos4, double *__restrict__ vel, int32_t *__restrict__ user_of,
-                         float *__restrict__ disp) {
+                         float *__restrict__ disp, const int32_t *__restrict__ cell_of, int32_t *__restrict__ cell_id) {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     int src = slot_src[i];
+    if (cell_id) cell_id[i] = cell_of[src];   // build-time cell of the atom in the internal order (compact lists)
     pos4[i] = pos4_src[src];
     user_of[i] = user_src[src];
     for (int a = 0; a < 3; ++a) {
@@ -236,11 +250,11 @@ __global__ void k_rel_pos(int64_t n, CellGrid g, const double4 *__restrict__ pos
 // separation is x_rel(j) - x_rel(i) + (cell offset) * edge -- the cell offset already names the periodic image, so no
 // minimum-image step and no fp64 arithmetic per candidate.  Candidates within 1e-5 of the list radius (the fp32 distance is
 // good to ~1e-6) are decided by the exact fp64 predicate on the full positions, so the lists are the same bit for bit.
-template <bool FILL>
+template <bool FILL, typename OUT>
 __global__ void __launch_bounds__(256) k_neighbors_rel(int64_t n, CellGrid g, double rl2, const double4 *__restrict__ pos4,
                                                        const float4 *__restrict__ rel, const int32_t *__restrict__ cell_start,
                                                        int32_t *__restrict__ nbr_count, const int64_t *__restrict__ nbr_off,
-                                                       int32_t *__restrict__ nbr, int64_t nbr_cap, int *status, float near2,
+                                                       OUT *__restrict__ nbr, int64_t nbr_cap, int *status, float near2,
                                                        int32_t *__restrict__ nbr_near, const int32_t *__restrict__ user_of, int32_t n_owned) {
     const int lane = threadIdx.x & 31;
     int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -314,7 +328,7 @@ __global__ void __launch_bounds__(256) k_neighbors_rel(int64_t n, CellGrid g, do
             const bool near = hit && d2f < near2;
             const unsigned m = __ballot_sync(0xffffffffu, hit), mn = __ballot_sync(0xffffffffu, near), below = (1u << lane) - 1u;
             if (FILL && hit && writable)
-                nbr[off + (near ? cn + __popc(mn & below) : total - 1 - (cnt - cn + __popc(m & ~mn & below)))] = j;
+                nbr[off + (near ? cn + __popc(mn & below) : total - 1 - (cnt - cn + __popc(m & ~mn & below)))] = list_entry<OUT>(j, it, cur_beg);
             cnt += __popc(m);
             cn += __popc(mn);
         }
@@ -371,10 +385,12 @@ __device__ __forceinline__ void cell_ranges(const double4 &p4, const CellGrid &g
 // out[top - 1], ...; only positions below `limit` are written.  Shared-memory pass: top = capacity - 1 (if the list is
 // longer than the buffer the two ends collide and the list is traversed again); global pass: top = list length - 1.
 // Returns the number of hits, and the number of near hits in `n_near`.
+template <typename OUT, typename ENTRY>
 __device__ __forceinline__ int onepass_traverse(int64_t i, const CellGrid &g, double rl2, const float (&edge)[3], float rl2_lo, float rl2_hi,
                                                 const double4 *__restrict__ pos4, const float4 *__restrict__ rel,
-                                                const int32_t *__restrict__ cell_start, int lane, int32_t *out, int top, int limit,
+                                                const int32_t *__restrict__ cell_start, int lane, OUT *out, int top, int limit,
                                                 float near2, int &n_near) {
+    // OUT = type of the buffer written here (int32 in shared memory), ENTRY = format of the list (int32 or uint16)
     const double4 pi = pos4[i];
     const float4 ri = rel[i];
     int cb, ce;
@@ -403,7 +419,7 @@ __device__ __forceinline__ int onepass_traverse(int64_t i, const CellGrid &g, do
             const bool near = hit && d2f < near2;
             const unsigned m = __ballot_sync(0xffffffffu, hit), mn = __ballot_sync(0xffffffffu, near), below = (1u << lane) - 1u;
             const int slot = near ? cn + __popc(mn & below) : top - (cnt - cn + __popc(m & ~mn & below));
-            if (hit && slot >= 0 && slot < limit) out[slot] = j;
+            if (hit && slot >= 0 && slot < limit) out[slot] = (OUT)list_entry<ENTRY>(j, it, cur_beg);
             cnt += __popc(m);
             cn += __popc(mn);
         }
@@ -414,9 +430,10 @@ __device__ __forceinline__ int onepass_traverse(int64_t i, const CellGrid &g, do
 
 constexpr int OP_BUF = 160;   // hits kept per atom in shared memory; a longer list is traversed again straight into global memory
 
+template <typename ENTRY>
 __global__ void __launch_bounds__(256) k_neighbors_onepass(int64_t n, CellGrid g, double rl2, const double4 *__restrict__ pos4,
                                                            const float4 *__restrict__ rel, const int32_t *__restrict__ cell_start,
-                                                           int64_t *__restrict__ nbr_off, int32_t *__restrict__ nbr, int64_t nbr_cap,
+                                                           int64_t *__restrict__ nbr_off, ENTRY *__restrict__ nbr, int64_t nbr_cap,
                                                            int *status, unsigned long long *tile_state, int *ticket,
                                                            const int *global_status, int spin_limit, long long unpublished_tile,
                                                            float near2, int32_t *__restrict__ nbr_near,
@@ -444,7 +461,7 @@ __global__ void __launch_bounds__(256) k_neighbors_onepass(int64_t n, CellGrid g
         const int64_t i = first + slot;
         int cnt = 0, cn = 0;
         if (i < n && user_of[i] < n_owned)   // (a ghost has no list of its own)
-            cnt = onepass_traverse(i, g, rl2, edge, rl2_lo, rl2_hi, pos4, rel, cell_start, lane, s_hits + slot * OP_BUF, OP_BUF - 1, OP_BUF, near2, cn);
+            cnt = onepass_traverse<int32_t, ENTRY>(i, g, rl2, edge, rl2_lo, rl2_hi, pos4, rel, cell_start, lane, s_hits + slot * OP_BUF, OP_BUF - 1, OP_BUF, near2, cn);
         if (lane == 0) { s_cnt[slot] = cnt; s_near[slot] = cn; }
     }
     __syncthreads();
@@ -515,23 +532,36 @@ __global__ void __launch_bounds__(256) k_neighbors_onepass(int64_t n, CellGrid g
         if (fit == 0) continue;
         if (cnt <= OP_BUF) {   // near hits sit at the front of the buffer, far hits at its back
             const int32_t *src = s_hits + slot * OP_BUF;
-            for (int e = lane; e < fit; e += 32) nbr[off + e] = src[e < near ? e : e + (OP_BUF - cnt)];
+            for (int e = lane; e < fit; e += 32) nbr[off + e] = (ENTRY)src[e < near ? e : e + (OP_BUF - cnt)];
         } else {
             int cn;
-            onepass_traverse(i, g, rl2, edge, rl2_lo, rl2_hi, pos4, rel, cell_start, lane, nbr + off, cnt - 1, fit, near2, cn);
+            onepass_traverse<ENTRY, ENTRY>(i, g, rl2, edge, rl2_lo, rl2_hi, pos4, rel, cell_start, lane, nbr + off, cnt - 1, fit, near2, cn);
         }
     }
 }
 
 // ---- canonical export: caller's indices, species-segmented, ascending ----
-__global__ void k_export_count(int64_t n, int n_species, const int64_t *__restrict__ nbr_off, const int32_t *__restrict__ nbr,
+// Entry e of atom i's list as an internal index, whatever the list format (cell_id = nullptr: plain indices).
+struct ListView {
+    const int32_t *nbr;
+    const uint16_t *nbr16;
+    const int32_t *cell_id, *cell_start;
+    CellGrid grid;
+    __device__ __forceinline__ int at(int64_t i, int64_t e) const {
+        if (!nbr16) return nbr[e];
+        const int code = nbr16[e];
+        return cell_start[neighbor_cell(grid, cell_id[i], code >> L16_SHIFT)] + (code & L16_MASK);
+    }
+};
+
+__global__ void k_export_count(int64_t n, int n_species, const int64_t *__restrict__ nbr_off, ListView lv,
                                const double4 *__restrict__ pos4, const int32_t *__restrict__ user_of,
                                int32_t *__restrict__ seg_count) {
     const int lane = threadIdx.x & 31;
     int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (i >= n) return;
     int cnt[MAX_SPECIES] = {0};
-    for (int64_t e = nbr_off[i] + lane; e < nbr_off[i + 1]; e += 32) cnt[(int)pos4[nbr[e]].w]++;
+    for (int64_t e = nbr_off[i] + lane; e < nbr_off[i + 1]; e += 32) cnt[(int)pos4[lv.at(i, e)].w]++;
     int64_t row = (int64_t)user_of[i] * n_species;
     for (int s = 0; s < n_species; ++s) {
         int v = cnt[s];
@@ -540,7 +570,7 @@ __global__ void k_export_count(int64_t n, int n_species, const int64_t *__restri
     }
 }
 
-__global__ void k_export_fill(int64_t n, int n_species, const int64_t *__restrict__ nbr_off, const int32_t *__restrict__ nbr,
+__global__ void k_export_fill(int64_t n, int n_species, const int64_t *__restrict__ nbr_off, ListView lv,
                               const double4 *__restrict__ pos4, const int32_t *__restrict__ user_of,
                               const int64_t *__restrict__ seg_ptr, int32_t *__restrict__ out) {
     const int lane = threadIdx.x & 31;
@@ -549,11 +579,11 @@ __global__ void k_export_fill(int64_t n, int n_species, const int64_t *__restric
     const int64_t beg = nbr_off[i], end = nbr_off[i + 1];
     const int64_t row = (int64_t)user_of[i] * n_species;
     for (int64_t e = beg + lane; e < end; e += 32) {
-        int j = nbr[e];
+        int j = lv.at(i, e);
         int sj = (int)pos4[j].w, uj = user_of[j];
         int rank = 0;   // entries of the same species with a smaller caller index
         for (int64_t f = beg; f < end; ++f) {
-            int jf = nbr[f];
+            int jf = lv.at(i, f);
             rank += ((int)pos4[jf].w == sj) && (user_of[jf] < uj);
         }
         out[seg_ptr[row + sj] + rank] = uj;
@@ -561,6 +591,14 @@ __global__ void k_export_fill(int64_t n, int n_species, const int64_t *__restric
 }
 
 static inline unsigned blocks_for(int64_t n, int per_block) { return (unsigned)((n + per_block - 1) / per_block); }
+
+static ListView list_view(const mlip_ctx *c) {
+    ListView lv;
+    lv.nbr = c->nbr;
+    lv.nbr16 = c->list16 ? reinterpret_cast<const uint16_t *>(c->nbr) : nullptr;
+    lv.cell_id = c->cell_id; lv.cell_start = c->cell_start; lv.grid = c->grid;
+    return lv;
+}
 
 int launch_pack_source(mlip_ctx *c, const double *pos, const int32_t *species, cudaStream_t s) {
     k_pack_source<<<blocks_for(c->n, 256), 256, 0, s>>>(pos, species, c->n, c->cfg.n_species, c->pos4_src, c->user_src, c->status);
@@ -598,13 +636,24 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
     int32_t *slot_src = c->nbr_count;
     k_place<<<blocks_for(n, 256), 256, 0, s>>>(c->cell_of, n, c->cell_start, c->cell_fill, slot_src);
     k_sort_cells<<<blocks_for(g.n_cells, 128), 128, 0, s>>>(g.n_cells, C, c->cell_start, slot_src, c->pos4_src, c->user_src, c->bin_count, c->status, (int32_t)c->n_owned);
-    k_gather<<<blocks_for(n, 256), 256, 0, s>>>(n, slot_src, c->pos4_src, c->vel_src, c->user_src, c->pos4, c->vel, c->user_of, c->disp);
+    k_gather<<<blocks_for(n, 256), 256, 0, s>>>(n, slot_src, c->pos4_src, c->vel_src, c->user_src, c->pos4, c->vel, c->user_of, c->disp, c->cell_of, c->cell_id);
     exclusive_scan<int32_t, int32_t>(c->bin_count, c->bin_start, (int64_t)C * g.n_cells, c->scan_tmp, s);
     int nthreads_co = g.n_cells > C + 1 ? g.n_cells : C + 1;
     k_center_order<<<blocks_for(nthreads_co, 128), 128, 0, s>>>(g.n_cells, C, c->cell_start, c->pos4, c->bin_start, c->center_order, c->species_start, c->user_of, (int32_t)c->n_owned);
     // grids of at least 3 x 3 x 3 cells take the fp32 cell-relative traversal (positions staged in the idle force array)
     const bool rel = g.n[0] >= 3 && g.n[1] >= 3 && g.n[2] >= 3;
     float4 *relpos = c->force;
+    // entry format of this build: 16-bit cell-relative codes if asked for and the grid has 27 distinct cells around every
+    // cell, else plain indices.  A change of format gives up the old array (its capacity is counted in entries).
+    const bool list16 = c->cfg.list_format == 1 && rel;
+    if (list16 != c->list16 && c->nbr) {
+        cudaFree(c->nbr);
+        c->resident -= (c->list16 ? sizeof(uint16_t) : sizeof(int32_t)) * c->nbr_cap;
+        c->nbr = nullptr; c->nbr_cap = 0;
+    }
+    c->list16 = list16;
+    const size_t entry_bytes = list16 ? sizeof(uint16_t) : sizeof(int32_t);
+    uint16_t *nbr16 = reinterpret_cast<uint16_t *>(c->nbr);
     // Single traversal whenever a list array exists: always for in-step rebuilds (capacity as it stands, overflow -> status
     // bit), and for a synchronising build as a first try whose overflow flag is private and sends it to the two-pass path.
     bool rel_ready = false;
@@ -615,10 +664,15 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
         k_rel_pos<<<blocks_for(n, 256), 256, 0, s>>>(n, g, c->pos4, relpos);
         rel_ready = true;
         int *flag = allow_sync_grow ? c->tile_ticket + 1 : c->status;
-        k_neighbors_onepass<<<(unsigned)n_tiles, 256, sizeof(int32_t) * OP_TILE * OP_BUF, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_off, c->nbr, c->nbr_cap,
-                                                               flag, c->tile_state, c->tile_ticket, c->status,
-                                                               c->lookback_spin_limit > 0 ? c->lookback_spin_limit : OP_SPIN, c->lookback_unpublished_tile,
-                                                               near2, c->nbr_near, c->user_of, (int32_t)c->n_owned);
+        const int spin = c->lookback_spin_limit > 0 ? c->lookback_spin_limit : OP_SPIN;
+        if (list16)
+            k_neighbors_onepass<uint16_t><<<(unsigned)n_tiles, 256, sizeof(int32_t) * OP_TILE * OP_BUF, s>>>(
+                n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_off, nbr16, c->nbr_cap, flag, c->tile_state, c->tile_ticket, c->status, spin,
+                c->lookback_unpublished_tile, near2, c->nbr_near, c->user_of, (int32_t)c->n_owned);
+        else
+            k_neighbors_onepass<int32_t><<<(unsigned)n_tiles, 256, sizeof(int32_t) * OP_TILE * OP_BUF, s>>>(
+                n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_off, c->nbr, c->nbr_cap, flag, c->tile_state, c->tile_ticket, c->status, spin,
+                c->lookback_unpublished_tile, near2, c->nbr_near, c->user_of, (int32_t)c->n_owned);
         c->launches += 5 + 2 * 3 + 2;   // cell id, place, sort, gather, centre order; two scans; relative positions, lists
         MLIP_CUDA_TRY(c, cudaGetLastError());
         bool done = true;
@@ -639,7 +693,7 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
     }
     if (rel) {
         if (!rel_ready) k_rel_pos<<<blocks_for(n, 256), 256, 0, s>>>(n, g, c->pos4, relpos);
-        k_neighbors_rel<false><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_count, nullptr, nullptr, 0, c->status, near2, c->nbr_near, c->user_of, (int32_t)c->n_owned);
+        k_neighbors_rel<false, int32_t><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_count, nullptr, nullptr, 0, c->status, near2, c->nbr_near, c->user_of, (int32_t)c->n_owned);
         c->launches += 1;
     } else
         k_neighbors<false><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, c->cell_start, c->nbr_count, nullptr, nullptr, 0, c->status, near2, c->nbr_near, c->user_of, (int32_t)c->n_owned);
@@ -654,14 +708,17 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
         c->n_entries = *c->total_host;
         if (c->n_entries > c->nbr_cap) {
             int64_t want = c->n_entries + c->n_entries / 8 + 1024;
-            if (c->nbr) { cudaFree(c->nbr); c->resident -= sizeof(int32_t) * c->nbr_cap; c->nbr = nullptr; c->nbr_cap = 0; }
-            MLIP_CUDA_TRY(c, cudaMalloc(&c->nbr, sizeof(int32_t) * want));
+            if (c->nbr) { cudaFree(c->nbr); c->resident -= entry_bytes * c->nbr_cap; c->nbr = nullptr; c->nbr_cap = 0; }
+            MLIP_CUDA_TRY(c, cudaMalloc(&c->nbr, entry_bytes * want));
             c->nbr_cap = want;
-            c->resident += sizeof(int32_t) * want;
+            c->resident += entry_bytes * want;
+            nbr16 = reinterpret_cast<uint16_t *>(c->nbr);
         }
     }
-    if (rel)
-        k_neighbors_rel<true><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_count, c->nbr_off, c->nbr, c->nbr_cap, c->status, near2, c->nbr_near, c->user_of, (int32_t)c->n_owned);
+    if (rel && list16)
+        k_neighbors_rel<true, uint16_t><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_count, c->nbr_off, nbr16, c->nbr_cap, c->status, near2, c->nbr_near, c->user_of, (int32_t)c->n_owned);
+    else if (rel)
+        k_neighbors_rel<true, int32_t><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, relpos, c->cell_start, c->nbr_count, c->nbr_off, c->nbr, c->nbr_cap, c->status, near2, c->nbr_near, c->user_of, (int32_t)c->n_owned);
     else
         k_neighbors<true><<<blocks_for(n * 32, 256), 256, 0, s>>>(n, g, rl * rl, c->pos4, c->cell_start, c->nbr_count, c->nbr_off, c->nbr, c->nbr_cap, c->status, near2, c->nbr_near, c->user_of, (int32_t)c->n_owned);
     c->launches += 1;
@@ -693,7 +750,7 @@ int launch_export(mlip_ctx *c, int64_t *seg_ptr, int32_t *nbr, int64_t capacity,
         c->err = "neighbor export: cudaMalloc of the scan scratch failed";
         return MLIP_ERR_OOM;
     }
-    k_export_count<<<blocks_for(n * 32, 256), 256, 0, s>>>(n, C, c->nbr_off, c->nbr, c->pos4, c->user_of, seg_count);
+    k_export_count<<<blocks_for(n * 32, 256), 256, 0, s>>>(n, C, c->nbr_off, list_view(c), c->pos4, c->user_of, seg_count);
     exclusive_scan<int32_t, int64_t>(seg_count, seg_ptr, n * C, tmp, s);
     int rc = MLIP_OK;
     cudaError_t e = cudaMemcpyAsync(c->total_host, seg_ptr + n * C, sizeof(int64_t), cudaMemcpyDeviceToHost, s);
@@ -702,7 +759,7 @@ int launch_export(mlip_ctx *c, int64_t *seg_ptr, int32_t *nbr, int64_t capacity,
         if (n_entries_host) *n_entries_host = *c->total_host;
         if (*c->total_host > capacity || !nbr) rc = MLIP_ERR_NEIGHBOR_OVERFLOW;
         else {
-            k_export_fill<<<blocks_for(n * 32, 256), 256, 0, s>>>(n, C, c->nbr_off, c->nbr, c->pos4, c->user_of, seg_ptr, nbr);
+            k_export_fill<<<blocks_for(n * 32, 256), 256, 0, s>>>(n, C, c->nbr_off, list_view(c), c->pos4, c->user_of, seg_ptr, nbr);
             e = cudaStreamSynchronize(s);
         }
     }
@@ -769,7 +826,7 @@ int launch_export_noalloc(mlip_ctx *c, int64_t *seg_ptr, int32_t *nbr, int64_t c
     if ((rc = export_scratch_for_current_device(c, &base)) != MLIP_OK) return rc;
     int32_t *seg_count = reinterpret_cast<int32_t *>(base);
     int64_t *tmp = reinterpret_cast<int64_t *>(static_cast<unsigned char *>(base) + NOALLOC_COUNT_BYTES);
-    k_export_count<<<blocks_for(n * 32, 256), 256, 0, s>>>(n, C, c->nbr_off, c->nbr, c->pos4, c->user_of, seg_count);
+    k_export_count<<<blocks_for(n * 32, 256), 256, 0, s>>>(n, C, c->nbr_off, list_view(c), c->pos4, c->user_of, seg_count);
     exclusive_scan<int32_t, int64_t>(seg_count, seg_ptr, n * C, tmp, s);
     MLIP_CUDA_TRY(c, cudaMemcpyAsync(c->total_host, seg_ptr + n * C, sizeof(int64_t), cudaMemcpyDeviceToHost, s));
     MLIP_CUDA_TRY(c, cudaStreamSynchronize(s));
@@ -779,7 +836,7 @@ int launch_export_noalloc(mlip_ctx *c, int64_t *seg_ptr, int32_t *nbr, int64_t c
         c->err = "neighbor export: capacity too small";
         return MLIP_ERR_NEIGHBOR_OVERFLOW;
     }
-    k_export_fill<<<blocks_for(n * 32, 256), 256, 0, s>>>(n, C, c->nbr_off, c->nbr, c->pos4, c->user_of, seg_ptr, nbr);
+    k_export_fill<<<blocks_for(n * 32, 256), 256, 0, s>>>(n, C, c->nbr_off, list_view(c), c->pos4, c->user_of, seg_ptr, nbr);
     c->launches += 1;
     MLIP_CUDA_TRY(c, cudaStreamSynchronize(s));
     return MLIP_OK;

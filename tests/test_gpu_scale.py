@@ -146,12 +146,19 @@ def test_benchmark_size_blocks_of_atoms_and_sampled_lists_match_oracle():
     pot.close()
 
 
-def test_list_offsets_beyond_32_bits_match_oracle():
-    """33,957,312 atoms: 4.55e9 list entries, so the offsets of the upper rows pass 2^31 and 2^32."""
+@functools.lru_cache(maxsize=1)
+def _workload_34m():
+    return wl.make_workload(5, n_cells=204, with_velocities=False)
+
+
+@pytest.mark.parametrize("list_format", [0, 1])
+def test_list_offsets_beyond_32_bits_match_oracle(list_format):
+    """33,957,312 atoms: 4.55e9 list entries, so the offsets of the upper rows pass 2^31 and 2^32 -- with plain indices and
+    with the 16-bit cell-relative codes."""
     import paper_2608_16329_b200 as mlip
-    w = wl.make_workload(5, n_cells=204, with_velocities=False)
+    w = _workload_34m()
     enc, head = wl.workload_weights(5, w.n_species)
-    pot = mlip.Potential(w.n_species, w.r_cut, w.skin, enc, head, w.masses)
+    pot = mlip.Potential(w.n_species, w.r_cut, w.skin, enc, head, w.masses, list_format=list_format)
     pot.build_neighbors(w.pos, w.species, w.box)
     assert mlip.mlip_get_counters(pot.ctx)["list_entries"] > 2 ** 32
     rows = sampled_rows(w.n_atoms, 2000, seed=7)
