@@ -61,6 +61,7 @@ struct TileSmem {
     double dp[2][F64_TILE][F64_YS];         // dE/dpre of the layer being propagated
     union {
         double st[32][ST];                  // encoding hand-over
+        double dv[16 * (10 + 16 * ((D + 7) / 8))];   // derivation staging of the tensor form: 16 pairs x (b, b', offset | V, T)
         double w[D * K];                    // W_i = dE_i/dP_i (Eq. 7), derivation
     } pw[F64_TILE];
     int q[F64_TILE][64];                    // compacted neighbor indices
@@ -312,48 +313,107 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
         }
         __syncwarp();
 
-        // ---------------- Derivation (Eq. 8-10), lane = pair ----------------
+        // ---------------- Derivation (Eq. 8-10) ----------------
+        // The pairs inside r_cut are compacted into a ring of neighbor indices and taken NB at a time.
+        //   closed-form shapes (TENSOR): [V; T] = [G; G'] W^T (Eq. 9 and the re-associated Eq. 8 term) on the fp64 tensor
+        //     pipe, 8 pairs per m8n8k4 tile: lane (g, t) evaluates g, g' of pair g at channels 4 ks + t straight into the A
+        //     operand (the quad reads one 32-byte sector of each table row), W_i sits in registers as B fragments, the
+        //     accumulators return through shared memory to lane = pair for the projection.  16 pairs per batch: the
+        //     staging rows share the hand-over buffer with W_i's shared-memory copy, which is dead once the fragments are loaded.
+        //   other shapes: lane = pair throughout, plain DFMA against W_i in shared memory, 32 pairs per batch.
+        constexpr bool TENSOR = CLOSED;
+        constexpr int NB = TENSOR ? 16 : 32;
+        constexpr int NT = (D + 7) / 8;            // n-tiles of the tensor form
+        constexpr int BS = 10, VTS = 2 * 8 * NT;   // staging rows: 4 b, 4 b', table offset | V then T
+        static_assert(!TENSOR || NB * (BS + VTS) * sizeof(double) <= sizeof(sm.pw[0]), "derivation staging must fit the hand-over buffer");
         double fx = 0.0, fy = 0.0, fz = 0.0;
-        int nq = 0;
+        int nq = 0, qh = 0;                        // ring: nq indices from position qh
         int *queue = sm.q[wid];
-        for (int64_t base = beg; base < end || nq > 0; base += 32) {
-            if (base < end) {   // compact the entries inside r_cut into the warp's queue
-                const int64_t e = base + lane;
-                bool valid = false;
-                int j = entry(e, e < end);
-                if (e < end) {
-                    const double4 pj = k.pos4[j];
-                    const double dx = min_image(pj.x - pi.x, k.grid.box[0], k.grid.half[0]);
-                    const double dy = min_image(pj.y - pi.y, k.grid.box[1], k.grid.half[1]);
-                    const double dz = min_image(pj.z - pi.z, k.grid.box[2], k.grid.half[2]);
-                    valid = dx * dx + dy * dy + dz * dz < k.rc2;
-                }
-                const unsigned m = __ballot_sync(0xffffffffu, valid);
-                if (valid) queue[nq + __popc(m & ((1u << lane) - 1u))] = j;
-                nq += __popc(m);
-                __syncwarp();
-                if (nq < 32 && base + 32 < end) continue;
-            }
-            const int nb = min(nq, 32);
+        double Bf[TENSOR ? NT : 1][TENSOR ? K / 4 : 1];
+        if (TENSOR) {
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int ks = 0; ks < K / 4; ++ks) Bf[nt][ks] = (8 * nt + g < D) ? wi[(8 * nt + g) * K + 4 * ks + t] : 0.0;
+            __syncwarp();   // from here on the buffer that held W_i is staging space
+        }
+        double *bs = reinterpret_cast<double *>(&sm.pw[wid]), *vt = bs + NB * BS;
+
+        auto process = [&](int nb) {
+            const int j = lane < nb ? queue[(qh + lane) & 63] : 0;
+            double x = 0.0, y = 0.0, z = 0.0, rinv = 0.0, ux = 0.0, uy = 0.0, uz = 0.0;
+            double b[4] = {0.0, 0.0, 0.0, 0.0}, db[4] = {0.0, 0.0, 0.0, 0.0};
+            const double *cf = k.coef;
             if (lane < nb) {
-                const int j = queue[lane];
                 const double4 pj = k.pos4[j];
-                const double x = min_image(pj.x - pi.x, k.grid.box[0], k.grid.half[0]);
-                const double y = min_image(pj.y - pi.y, k.grid.box[1], k.grid.half[1]);
-                const double z = min_image(pj.z - pi.z, k.grid.box[2], k.grid.half[2]);
-                const double r = sqrt(x * x + y * y + z * z), rinv = 1.0 / r;
-                const double ux = x * rinv, uy = y * rinv, uz = z * rinv;
-                double b[4], db[4];
+                x = min_image(pj.x - pi.x, k.grid.box[0], k.grid.half[0]);
+                y = min_image(pj.y - pi.y, k.grid.box[1], k.grid.half[1]);
+                z = min_image(pj.z - pi.z, k.grid.box[2], k.grid.half[2]);
+                const double r = sqrt(x * x + y * y + z * z);
+                rinv = 1.0 / r;
+                ux = x * rinv; uy = y * rinv; uz = z * rinv;
                 const int iv = spline_basis<true, double>(r, k.r_min, k.inv_h, k.knots, b, db, k.status);
-                const double *cf = k.coef + ((size_t)(si * C + (int)pj.w) * (k.knots + 3) + iv) * K;
-                // v = W g and t = W g' (Eq. 9 and the re-associated Eq. 8 term) for the rows of the angular degrees L0 .. L1,
-                // projected at once; wide bases go through in two degree ranges so that v and t stay in registers
-                double s = 0.0, tx = 0.0, ty = 0.0, tz = 0.0, tu = 0.0;
+                cf = k.coef + ((size_t)(si * C + (int)pj.w) * (k.knots + 3) + iv) * K;
+            }
+            double s = 0.0, tx = 0.0, ty = 0.0, tz = 0.0, tu = 0.0;
+            if constexpr (TENSOR) {
+                if (lane < NB) {   // hand the spline weights and the table row to the tile's lanes
+                    double *row = bs + lane * BS;
+#pragma unroll
+                    for (int m = 0; m < 4; ++m) { row[m] = b[m]; row[4 + m] = db[m]; }
+                    row[8] = __longlong_as_double((long long)(cf - k.coef));
+                }
+                __syncwarp();
+#pragma unroll 1
+                for (int grp = 0; grp < NB / 8; ++grp) {
+                    if (8 * grp >= nb) break;
+                    const double *row = bs + (8 * grp + g) * BS;
+                    double wb[4], wd[4];
+#pragma unroll
+                    for (int m = 0; m < 4; ++m) { wb[m] = row[m]; wd[m] = row[4 + m]; }
+                    const double *ct = k.coef + __double_as_longlong(row[8]) + t;
+                    double V[NT][2], T[NT][2];
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) { V[nt][0] = V[nt][1] = T[nt][0] = T[nt][1] = 0.0; }
+#pragma unroll
+                    for (int ks = 0; ks < K / 4; ++ks) {
+                        double gv = 0.0, dg = 0.0;
+#pragma unroll
+                        for (int m = 0; m < 4; ++m) {
+                            const double cm = __ldg(ct + m * K + 4 * ks);
+                            gv = fma(wb[m], cm, gv);
+                            dg = fma(wd[m], cm, dg);
+                        }
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            dmma(V[nt][0], V[nt][1], gv, Bf[nt][ks]);
+                            dmma(T[nt][0], T[nt][1], dg, Bf[nt][ks]);
+                        }
+                    }
+                    double *out = vt + (8 * grp + g) * VTS + 2 * t;
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        *reinterpret_cast<double2 *>(out + 8 * nt) = make_double2(V[nt][0], V[nt][1]);
+                        *reinterpret_cast<double2 *>(out + 8 * NT + 8 * nt) = make_double2(T[nt][0], T[nt][1]);
+                    }
+                }
+                __syncwarp();
+                if (lane < nb) {
+                    double v[D_ANG], tt[D_ANG];   // components beyond d are zero and drop out of the projection
+                    const double *rowv = vt + lane * VTS;
+#pragma unroll
+                    for (int a = 0; a < D_ANG; ++a) { v[a] = a < 8 * NT ? rowv[a] : 0.0; tt[a] = a < 8 * NT ? rowv[8 * NT + a] : 0.0; }
+                    harmonics_project(ux, uy, uz, v, tt, s, tx, ty, tz, tu);
+                }
+                __syncwarp();
+            } else if (lane < nb) {
+                // v = W g and t = W g' for the rows of the angular degrees L0 .. L1, projected at once; wide bases go
+                // through in two degree ranges so that v and t stay in registers
                 auto rows_of = [&](auto l0c, auto l1c) {
                     constexpr int L0 = decltype(l0c)::value, L1 = decltype(l1c)::value;
-                    constexpr int A0 = CLOSED ? 0 : Shape::begin(L0), A1 = CLOSED ? D : Shape::begin(L1 + 1);
-                    constexpr int DV = CLOSED ? D_ANG : A1 - A0;
-                    double v[DV], tt[DV];   // (closed forms: components beyond d stay zero and drop out of the projection)
+                    constexpr int A0 = Shape::begin(L0), A1 = Shape::begin(L1 + 1);
+                    constexpr int DV = A1 - A0;
+                    double v[DV], tt[DV];
 #pragma unroll
                     for (int a = 0; a < DV; ++a) { v[a] = 0.0; tt[a] = 0.0; }
 #pragma unroll 1
@@ -376,16 +436,17 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                         }
                     }
                     double ps, px, py, pz, pu;
-                    if (CLOSED) harmonics_project(ux, uy, uz, v, tt, ps, px, py, pz, pu);
-                    else angular_project<LMAX, BASIS, L0, L1>(ux, uy, uz, v, tt, ps, px, py, pz, pu);
+                    angular_project<LMAX, BASIS, L0, L1>(ux, uy, uz, v, tt, ps, px, py, pz, pu);
                     s += ps; tx += px; ty += py; tz += pz; tu += pu;
                 };
-                if constexpr (!CLOSED && D > 25) {
+                if constexpr (D > 25) {
                     rows_of(std::integral_constant<int, 0>{}, std::integral_constant<int, 3>{});
                     rows_of(std::integral_constant<int, 4>{}, std::integral_constant<int, LMAX>{});
                 } else {
                     rows_of(std::integral_constant<int, 0>{}, std::integral_constant<int, LMAX>{});
                 }
+            }
+            if (lane < nb) {
                 // f_ij = (g' . u_ij) r^ + J_ang^T v_ij,  J_ang = (grad_u h)(I - u u^T) / r
                 const double qx = s * ux + (tx - tu * ux) * rinv;
                 const double qy = s * uy + (ty - tu * uy) * rinv;
@@ -398,15 +459,28 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                 vir[3] -= y * qx; vir[4] -= y * qy; vir[5] -= y * qz;
                 vir[6] -= z * qx; vir[7] -= z * qy; vir[8] -= z * qz;
             }
+            qh = (qh + nb) & 63;
+            nq -= nb;
+        };
+
+        for (int64_t base = beg; base < end; base += 32) {   // compact the entries inside r_cut into the ring
+            const int64_t e = base + lane;
+            bool valid = false;
+            const int j = entry(e, e < end);
+            if (e < end) {
+                const double4 pj = k.pos4[j];
+                const double dx = min_image(pj.x - pi.x, k.grid.box[0], k.grid.half[0]);
+                const double dy = min_image(pj.y - pi.y, k.grid.box[1], k.grid.half[1]);
+                const double dz = min_image(pj.z - pi.z, k.grid.box[2], k.grid.half[2]);
+                valid = dx * dx + dy * dy + dz * dz < k.rc2;
+            }
+            const unsigned m = __ballot_sync(0xffffffffu, valid);
+            if (valid) queue[(qh + nq + __popc(m & ((1u << lane) - 1u))) & 63] = j;
+            nq += __popc(m);
             __syncwarp();
-            // move what is left of the queue to its front
-            const int rest = nq - nb;
-            const int keep = lane < rest ? queue[nb + lane] : 0;
-            __syncwarp();
-            if (lane < rest) queue[lane] = keep;
-            nq = rest;
-            __syncwarp();
+            while (nq >= NB) { process(NB); __syncwarp(); }
         }
+        while (nq > 0) { process(min(nq, NB)); __syncwarp(); }
 #pragma unroll
         for (int o = 16; o; o >>= 1) {
             fx += __shfl_xor_sync(0xffffffffu, fx, o);
