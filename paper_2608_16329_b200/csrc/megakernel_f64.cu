@@ -61,7 +61,7 @@ struct TileSmem {
     double dp[2][F64_TILE][F64_YS];         // dE/dpre of the layer being propagated
     union {
         double st[32][ST];                  // encoding hand-over
-        double dv[16 * (10 + 16 * ((D + 7) / 8))];   // derivation staging of the tensor form: 16 pairs x (b, b', offset | V, T)
+        double dv[16 * (12 + 16 * ((D + 7) / 8))];   // derivation staging of the tensor form: 16 pairs x (b, b', offset | V, T, pad)
         double w[D * K];                    // W_i = dE_i/dP_i (Eq. 7), derivation
     } pw[F64_TILE];
     int q[F64_TILE][64];                    // compacted neighbor indices
@@ -324,7 +324,8 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
         constexpr bool TENSOR = CLOSED;
         constexpr int NB = TENSOR ? 16 : 32;
         constexpr int NT = (D + 7) / 8;            // n-tiles of the tensor form
-        constexpr int BS = 10, VTS = 2 * 8 * NT;   // staging rows: 4 b, 4 b', table offset | V then T
+        constexpr int BS = 10, VTS = 2 * 8 * NT + 2;   // staging rows: 4 b, 4 b', table offset | V then T (+ 2: lane = pair reads 16
+                                                       // bytes at a 68-word stride, eight lanes on 32 different banks)
         static_assert(!TENSOR || NB * (BS + VTS) * sizeof(double) <= sizeof(sm.pw[0]), "derivation staging must fit the hand-over buffer");
         double fx = 0.0, fy = 0.0, fz = 0.0;
         int nq = 0, qh = 0;                        // ring: nq indices from position qh
@@ -334,7 +335,8 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                for (int ks = 0; ks < K / 4; ++ks) Bf[nt][ks] = (8 * nt + g < D) ? wi[(8 * nt + g) * K + 4 * ks + t] : 0.0;
+                for (int ks = 0; ks < K / 4; ++ks)   // k-step ks = 4 h + u contracts channel 16 h + 4 t + u (see the loads below)
+                    Bf[nt][ks] = (8 * nt + g < D) ? wi[(8 * nt + g) * K + 16 * (ks >> 2) + 4 * t + (ks & 3)] : 0.0;
             __syncwarp();   // from here on the buffer that held W_i is staging space
         }
         double *bs = reinterpret_cast<double *>(&sm.pw[wid]), *vt = bs + NB * BS;
@@ -371,24 +373,30 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                     double wb[4], wd[4];
 #pragma unroll
                     for (int m = 0; m < 4; ++m) { wb[m] = row[m]; wd[m] = row[4 + m]; }
-                    const double *ct = k.coef + __double_as_longlong(row[8]) + t;
+                    const double *ct = k.coef + __double_as_longlong(row[8]) + 4 * t;
                     double V[NT][2], T[NT][2];
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) { V[nt][0] = V[nt][1] = T[nt][0] = T[nt][1] = 0.0; }
+                    // the channel <-> k-index assignment is free (both operands use it); with lane t on channels
+                    // 16 h + 4 t .. + 3 the quad reads 128 contiguous bytes of a table row per load
 #pragma unroll
-                    for (int ks = 0; ks < K / 4; ++ks) {
-                        double gv = 0.0, dg = 0.0;
+                    for (int h = 0; h < K / 16; ++h) {
+                        double gv[4] = {0.0, 0.0, 0.0, 0.0}, dg[4] = {0.0, 0.0, 0.0, 0.0};
 #pragma unroll
                         for (int m = 0; m < 4; ++m) {
-                            const double cm = __ldg(ct + m * K + 4 * ks);
-                            gv = fma(wb[m], cm, gv);
-                            dg = fma(wd[m], cm, dg);
+                            double cc[4];
+                            asm volatile("ld.global.nc.v4.f64 {%0,%1,%2,%3}, [%4];"
+                                         : "=d"(cc[0]), "=d"(cc[1]), "=d"(cc[2]), "=d"(cc[3]) : "l"(ct + m * K + 16 * h));
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) { gv[u] = fma(wb[m], cc[u], gv[u]); dg[u] = fma(wd[m], cc[u], dg[u]); }
                         }
 #pragma unroll
-                        for (int nt = 0; nt < NT; ++nt) {
-                            dmma(V[nt][0], V[nt][1], gv, Bf[nt][ks]);
-                            dmma(T[nt][0], T[nt][1], dg, Bf[nt][ks]);
-                        }
+                        for (int u = 0; u < 4; ++u)
+#pragma unroll
+                            for (int nt = 0; nt < NT; ++nt) {
+                                dmma(V[nt][0], V[nt][1], gv[u], Bf[nt][4 * h + u]);
+                                dmma(T[nt][0], T[nt][1], dg[u], Bf[nt][4 * h + u]);
+                            }
                     }
                     double *out = vt + (8 * grp + g) * VTS + 2 * t;
 #pragma unroll
@@ -402,7 +410,11 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                     double v[D_ANG], tt[D_ANG];   // components beyond d are zero and drop out of the projection
                     const double *rowv = vt + lane * VTS;
 #pragma unroll
-                    for (int a = 0; a < D_ANG; ++a) { v[a] = a < 8 * NT ? rowv[a] : 0.0; tt[a] = a < 8 * NT ? rowv[8 * NT + a] : 0.0; }
+                    for (int a = 0; a < D_ANG; a += 2) {
+                        double2 pv = make_double2(0.0, 0.0), pt = pv;
+                        if (a < 8 * NT) { pv = *reinterpret_cast<const double2 *>(rowv + a); pt = *reinterpret_cast<const double2 *>(rowv + 8 * NT + a); }
+                        v[a] = pv.x; v[a + 1] = pv.y; tt[a] = pt.x; tt[a + 1] = pt.y;
+                    }
                     harmonics_project(ux, uy, uz, v, tt, s, tx, ty, tz, tu);
                 }
                 __syncwarp();
