@@ -212,4 +212,21 @@ __device__ __forceinline__ double min_image(double d, double box, double half) {
     return d;
 }
 
+// Optional per-phase cycle counters (profiling builds only: -DMLIP_PHASE_CLOCKS).  Slots 16.. of
+// the accumulator array receive the summed clock64 ticks of lane 0 of every warp.
+#ifdef MLIP_PHASE_CLOCKS
+struct PhaseClock {
+    long long t, acc[16];
+    __device__ __forceinline__ void start() { t = clock64(); for (int q = 0; q < 16; ++q) acc[q] = 0; }
+    __device__ __forceinline__ void mark(int slot) { const long long now = clock64(); acc[slot] += now - t; t = now; }
+    __device__ __forceinline__ void flush(double *a, int lane) { if (lane == 0) for (int q = 0; q < 16; ++q) atomicAdd(&a[16 + q], (double)acc[q]); }
+};
+#else
+struct PhaseClock {
+    __device__ __forceinline__ void start() {}
+    __device__ __forceinline__ void mark(int) {}
+    __device__ __forceinline__ void flush(double *, int) {}
+};
+#endif
+
 }  // namespace mlip

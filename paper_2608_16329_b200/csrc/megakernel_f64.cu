@@ -35,15 +35,17 @@
 namespace mlip {
 
 constexpr int F64_TILE = 8;         // atoms per tile = warps per CTA = columns of the tensor-pipe tile
-constexpr int F64_YS = HEAD_H + 4;  // activation row stride: 4 mod 16 keeps the B-fragment reads conflict-free
+constexpr int F64_YS = HEAD_H + 2;  // activation row stride: 2 mod 4 doubles keeps the 16-byte B-operand reads conflict-free
 
 // per-species head block (doubles) for n_inv inputs: the caller's row-major matrices, then biases and output layer
 struct Head64 {
-    int w0, wl, bias, wout, total;
+    int w0, wl, w0t, wlt, bias, wout, total;
     __host__ __device__ constexpr explicit Head64(int n_inv)
         : w0(0),                                            // [64][n_inv]
           wl(HEAD_H * n_inv),                               // 3 x [64][64]
-          bias(wl + (HEAD_L - 1) * HEAD_H * HEAD_H),        // [4][64]
+          w0t(wl + (HEAD_L - 1) * HEAD_H * HEAD_H),         // [n_inv][64]: the transposes feed the reverse pass rows too
+          wlt(w0t + HEAD_H * n_inv),                        // 3 x [64][64]
+          bias(wlt + (HEAD_L - 1) * HEAD_H * HEAD_H),       // [4][64]
           wout(bias + HEAD_L * HEAD_H),                     // [64] + b_out
           total(wout + HEAD_H + 8) {}
 };
@@ -54,7 +56,7 @@ struct TileSmem {
     static constexpr int D = Shape::D;
     static constexpr int ST = (D + 6) & ~1;   // hand-over row: D angular values, 4 spline weights, table offset, pad
     static constexpr int NINV = (LMAX + 1) * K;
-    static constexpr int XS = (NINV + 31) / 32 * 32 + 4;
+    static constexpr int XS = (NINV + 31) / 32 * 32 + 2;
     double x[F64_TILE][XS];                 // invariants, then dE/dG
     double y[2][F64_TILE][F64_YS];          // activations of the previous / current layer
     double sd[HEAD_L][F64_TILE][F64_YS];    // SiLU'(pre-activation) per layer
@@ -62,7 +64,8 @@ struct TileSmem {
     union {
         double st[32][ST];                  // encoding hand-over
         double dv[16 * (12 + 16 * ((D + 7) / 8))];   // derivation staging of the tensor form: 16 pairs x (b, b', offset | V, T, pad)
-        double w[D * K];                    // W_i = dE_i/dP_i (Eq. 7), derivation
+        double w[D * K];                    // W_i = dE_i/dP_i (Eq. 7), derivation; P_i on its way from fragments to lane = channel
+        double te[(D + 5) * 36];            // encoding hand-over of the tensor form: D rows of h, 4 of b, table offsets, 32 pairs (+ 4 pad) each
     } pw[F64_TILE];
     int q[F64_TILE][64];                    // compacted neighbor indices
 };
@@ -104,6 +107,29 @@ __device__ __forceinline__ void dmma(double &c0, double &c1, double a, double b)
     asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};" : "+d"(c0), "+d"(c1) : "d"(a), "d"(b));
 }
 
+// One row block of a head layer on the tensor pipe: c += A[8 x 16 NH] B[16 NH x 8].  The k-index <-> input assignment
+// is free as long as both operands use it: k-step 4 h + u contracts input 16 h + 4 t + u, so a quad reads 128
+// contiguous bytes of its weight row per load and a lane's four activations are two 16-byte shared-memory reads.
+// wrow = the lane's weight row + 4 t, xrow = the activations of atom g + 4 t.  Two accumulator chains.
+template <int NH>
+__device__ __forceinline__ void head_dot(double &c0, double &c1, const double *__restrict__ wrow, const double *xrow) {
+    double w[NH][4];
+#pragma unroll
+    for (int h = 0; h < NH; ++h)
+        asm volatile("ld.global.nc.v4.f64 {%0,%1,%2,%3}, [%4];" : "=d"(w[h][0]), "=d"(w[h][1]), "=d"(w[h][2]), "=d"(w[h][3]) : "l"(wrow + 16 * h));
+    double a0 = 0.0, a1 = 0.0;
+#pragma unroll
+    for (int h = 0; h < NH; ++h) {
+        const double2 x01 = *reinterpret_cast<const double2 *>(xrow + 16 * h), x23 = *reinterpret_cast<const double2 *>(xrow + 16 * h + 2);
+        if (h & 1) {
+            dmma(a0, a1, w[h][0], x01.x); dmma(a0, a1, w[h][1], x01.y); dmma(a0, a1, w[h][2], x23.x); dmma(a0, a1, w[h][3], x23.y);
+        } else {
+            dmma(c0, c1, w[h][0], x01.x); dmma(c0, c1, w[h][1], x01.y); dmma(c0, c1, w[h][2], x23.x); dmma(c0, c1, w[h][3], x23.y);
+        }
+    }
+    c0 += a0; c1 += a1;
+}
+
 #ifndef MLIP_F64_TWO_PER_SM_MAX_D
 #define MLIP_F64_TWO_PER_SM_MAX_D 20
 #endif
@@ -134,6 +160,8 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
     for (int s = 0; s < C; ++s) total_tiles += (s_start[s + 1] - s_start[s] + F64_TILE - 1) / F64_TILE;
     double e_sum = 0.0, vir[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
     unsigned long long n_pairs = 0;
+    PhaseClock pc;
+    pc.start();
 
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
         int si = 0, tl = tile;
@@ -162,62 +190,161 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
             return live ? (int)MLIP_CHECK_INDEX(base + (code & L16_MASK), k.n, k.status) : 0;
         };
 
-        // ---------------- Encoding: P = H^T G (Eq. 4), lane = channel ----------------
+        // ---------------- Encoding: P = H^T G (Eq. 4) ----------------
+        // closed-form shapes (TENSOR): four pairs per m8n8k4 step on the fp64 tensor pipe.  A = H^T (rows = angular
+        //   components, k = pair), B = G (k = pair, columns = channels): lane (g, t) evaluates g of pair t at the K / 8
+        //   contiguous channels K/8 * g .., so the eight lanes of a pair read a whole table row per load and four rows are in
+        //   flight per step; the accumulators go through shared memory to lane = channel afterwards.
+        // other shapes: one pair at a time, lane = channel, plain DFMA.
+        constexpr bool TENSOR = CLOSED;
+        constexpr int MT = (D + 7) / 8, NTK = K / 8, PS = 36;   // PS = 4 mod 16 doubles: the A-fragment reads fall on 32 different banks
         double P[D][CPL];
 #pragma unroll
         for (int a = 0; a < D; ++a)
 #pragma unroll
             for (int q = 0; q < CPL; ++q) P[a][q] = 0.0;
-        for (int64_t base = beg; base < end; base += 32) {
-            const int64_t e = base + lane;
-            bool valid = false;
-            const int j_e = entry(e, e < end);
-            if (e < end) {
-                const int j = j_e;
-                const double4 pj = k.pos4[j];
-                const double dx = min_image(pj.x - pi.x, k.grid.box[0], k.grid.half[0]);
-                const double dy = min_image(pj.y - pi.y, k.grid.box[1], k.grid.half[1]);
-                const double dz = min_image(pj.z - pi.z, k.grid.box[2], k.grid.half[2]);
-                const double d2 = dx * dx + dy * dy + dz * dz;
-                valid = d2 < k.rc2;
-                if (valid) {
-                    const double r = sqrt(d2), rinv = 1.0 / r;
-                    double h[CLOSED ? D_ANG : D], b[4];
-                    if (CLOSED) harmonics(dx * rinv, dy * rinv, dz * rinv, h);
-                    else angular_values<LMAX, BASIS>(dx * rinv, dy * rinv, dz * rinv, h);
-                    const int iv = spline_basis<false, double>(r, k.r_min, k.inv_h, k.knots, b, nullptr, k.status);
-                    double *row = sm.pw[wid].st[lane];
+        if constexpr (TENSOR) {
+            double Pc[MT][NTK][2];
 #pragma unroll
-                    for (int a = 0; a < D; ++a) row[a] = h[a];
+            for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-                    for (int m = 0; m < 4; ++m) row[D + m] = b[m];
-                    const long long off = ((long long)(si * C + (int)pj.w) * (k.knots + 3) + iv) * K;
-                    row[D + 4] = __longlong_as_double(off);
+                for (int nt = 0; nt < NTK; ++nt) Pc[mt][nt][0] = Pc[mt][nt][1] = 0.0;
+            double *hs = sm.pw[wid].te, *bq = hs + D * PS, *offs = bq + 4 * PS;
+            for (int64_t base = beg; base < end; base += 32) {
+                const int64_t e = base + lane;
+                const int j_e = entry(e, e < end);
+                bool valid = false;
+                double dx = 0.0, dy = 0.0, dz = 0.0, d2 = 1.0;
+                int sj = 0;
+                if (e < end) {
+                    const double4 pj = k.pos4[j_e];
+                    dx = min_image(pj.x - pi.x, k.grid.box[0], k.grid.half[0]);
+                    dy = min_image(pj.y - pi.y, k.grid.box[1], k.grid.half[1]);
+                    dz = min_image(pj.z - pi.z, k.grid.box[2], k.grid.half[2]);
+                    d2 = dx * dx + dy * dy + dz * dz;
+                    sj = (int)pj.w;
+                    valid = d2 < k.rc2;
                 }
-            }
-            unsigned mask = __ballot_sync(0xffffffffu, valid);
-            n_pairs += __popc(mask);
-            __syncwarp();
-            while (mask) {
-                const int p = __ffs(mask) - 1;
-                mask &= mask - 1;
-                const double *row = sm.pw[wid].st[p];
-                const double *cf = k.coef + __double_as_longlong(row[D + 4]);
+                const unsigned mask = __ballot_sync(0xffffffffu, valid);
+                const int nv = __popc(mask);
+                n_pairs += nv;
+                if (valid) {   // the pairs inside r_cut take consecutive columns of the hand-over rows
+                    const int col = __popc(mask & ((1u << lane) - 1u));
+                    const double r = sqrt(d2), rinv = 1.0 / r;
+                    double h[D_ANG], b[4];
+                    harmonics(dx * rinv, dy * rinv, dz * rinv, h);
+                    const int iv = spline_basis<false, double>(r, k.r_min, k.inv_h, k.knots, b, nullptr, k.status);
 #pragma unroll
-                for (int q = 0; q < CPL; ++q) {
-                    const int c = lane + 32 * q;
-                    double gq = 0.0;
-                    if (c < K) {
-                        gq = row[D] * cf[c];
-                        gq = fma(row[D + 1], cf[K + c], gq);
-                        gq = fma(row[D + 2], cf[2 * K + c], gq);
-                        gq = fma(row[D + 3], cf[3 * K + c], gq);
+                    for (int a = 0; a < D; ++a) hs[a * PS + col] = h[a];
+#pragma unroll
+                    for (int m = 0; m < 4; ++m) bq[m * PS + col] = b[m];
+                    offs[col] = __longlong_as_double(((long long)(si * C + sj) * (k.knots + 3) + iv) * K);
+                }
+                __syncwarp();
+                pc.mark(0);
+                for (int p0 = 0; p0 < nv; p0 += 4) {
+                    const int p = p0 + t;
+                    const bool live = p < nv;   // a step past the last pair contracts zeros against the table's first rows
+                    const double *cf = k.coef + (live ? __double_as_longlong(offs[p]) : 0ll) + NTK * g;
+                    double gq[NTK];
+#pragma unroll
+                    for (int nt = 0; nt < NTK; ++nt) gq[nt] = 0.0;
+#pragma unroll
+                    for (int m = 0; m < 4; ++m) {
+                        const double bm = live ? bq[m * PS + p] : 0.0;
+                        double cc[NTK];
+                        if constexpr (NTK == 2) {
+                            asm volatile("ld.global.nc.v2.f64 {%0,%1}, [%2];" : "=d"(cc[0]), "=d"(cc[1]) : "l"(cf + m * K));
+                        } else {
+#pragma unroll
+                            for (int v = 0; v < NTK; v += 4)
+                                asm volatile("ld.global.nc.v4.f64 {%0,%1,%2,%3}, [%4];"
+                                             : "=d"(cc[v]), "=d"(cc[v + 1]), "=d"(cc[v + 2]), "=d"(cc[v + 3]) : "l"(cf + m * K + v));
+                        }
+#pragma unroll
+                        for (int nt = 0; nt < NTK; ++nt) gq[nt] = fma(bm, cc[nt], gq[nt]);
                     }
 #pragma unroll
-                    for (int a = 0; a < D; ++a) P[a][q] = fma(row[a], gq, P[a][q]);
+                    for (int mt = 0; mt < MT; ++mt) {
+                        const double av = (live && 8 * mt + g < D) ? hs[(8 * mt + g) * PS + p] : 0.0;
+#pragma unroll
+                        for (int nt = 0; nt < NTK; ++nt) dmma(Pc[mt][nt][0], Pc[mt][nt][1], av, gq[nt]);
+                    }
+                }
+                __syncwarp();
+                pc.mark(1);
+            }
+            // fragments -> lane = channel: column n of n-tile nt is channel NTK n + nt
+            double *pm = sm.pw[wid].w;
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int nt = 0; nt < NTK; ++nt)
+#pragma unroll
+                    for (int u = 0; u < 2; ++u)
+                        if (8 * mt + g < D) pm[(8 * mt + g) * K + NTK * (2 * t + u) + nt] = Pc[mt][nt][u];
+            __syncwarp();
+#pragma unroll
+            for (int q = 0; q < CPL; ++q) {
+                const int c = lane + 32 * q;
+                if (c < K) {
+#pragma unroll
+                    for (int a = 0; a < D; ++a) P[a][q] = pm[a * K + c];
                 }
             }
-            __syncwarp();
+            __syncwarp();   // W_i is written over the same buffer below
+        } else {
+            for (int64_t base = beg; base < end; base += 32) {
+                const int64_t e = base + lane;
+                bool valid = false;
+                const int j_e = entry(e, e < end);
+                if (e < end) {
+                    const int j = j_e;
+                    const double4 pj = k.pos4[j];
+                    const double dx = min_image(pj.x - pi.x, k.grid.box[0], k.grid.half[0]);
+                    const double dy = min_image(pj.y - pi.y, k.grid.box[1], k.grid.half[1]);
+                    const double dz = min_image(pj.z - pi.z, k.grid.box[2], k.grid.half[2]);
+                    const double d2 = dx * dx + dy * dy + dz * dz;
+                    valid = d2 < k.rc2;
+                    if (valid) {
+                        const double r = sqrt(d2), rinv = 1.0 / r;
+                        double h[CLOSED ? D_ANG : D], b[4];
+                        if (CLOSED) harmonics(dx * rinv, dy * rinv, dz * rinv, h);
+                        else angular_values<LMAX, BASIS>(dx * rinv, dy * rinv, dz * rinv, h);
+                        const int iv = spline_basis<false, double>(r, k.r_min, k.inv_h, k.knots, b, nullptr, k.status);
+                        double *row = sm.pw[wid].st[lane];
+    #pragma unroll
+                        for (int a = 0; a < D; ++a) row[a] = h[a];
+    #pragma unroll
+                        for (int m = 0; m < 4; ++m) row[D + m] = b[m];
+                        const long long off = ((long long)(si * C + (int)pj.w) * (k.knots + 3) + iv) * K;
+                        row[D + 4] = __longlong_as_double(off);
+                    }
+                }
+                unsigned mask = __ballot_sync(0xffffffffu, valid);
+                n_pairs += __popc(mask);
+                __syncwarp();
+                while (mask) {
+                    const int p = __ffs(mask) - 1;
+                    mask &= mask - 1;
+                    const double *row = sm.pw[wid].st[p];
+                    const double *cf = k.coef + __double_as_longlong(row[D + 4]);
+    #pragma unroll
+                    for (int q = 0; q < CPL; ++q) {
+                        const int c = lane + 32 * q;
+                        double gq = 0.0;
+                        if (c < K) {
+                            gq = row[D] * cf[c];
+                            gq = fma(row[D + 1], cf[K + c], gq);
+                            gq = fma(row[D + 2], cf[2 * K + c], gq);
+                            gq = fma(row[D + 3], cf[3 * K + c], gq);
+                        }
+    #pragma unroll
+                        for (int a = 0; a < D; ++a) P[a][q] = fma(row[a], gq, P[a][q]);
+                    }
+                }
+                __syncwarp();
+            }
         }
 
         // ---------------- Invariants (Eq. 5: p^T C_l p); an empty slot of a ragged tile feeds zeros ----------------
@@ -235,7 +362,9 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                 }
             }
         }
+        pc.mark(2);
         __syncthreads();
+        pc.mark(3);
 
         // ---------------- Regression (Eq. 6) and its reverse pass: the CTA on the tile ----------------
         {
@@ -243,10 +372,11 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
             double y0, y1, d0, d1;
             {   // layer 0: pre[64 x 8] = W0 [64 x NINV] X^T
                 double c0 = hd[H.bias + n], c1 = c0;
-                const double *wrow = hd + H.w0 + (size_t)n * NINV + t;
-                const double *xb = &sm.x[g][t];
-#pragma unroll 8
-                for (int ks = 0; ks < NINV / 4; ++ks) dmma(c0, c1, wrow[4 * ks], xb[4 * ks]);
+                const double *wrow = hd + H.w0 + (size_t)n * NINV + 4 * t;
+                const double *xb = &sm.x[g][4 * t];
+                constexpr int HS = (NINV / 16) % 2 == 0 ? 2 : 1;   // 16-input blocks per call
+#pragma unroll 1
+                for (int h0 = 0; h0 < NINV / 16; h0 += HS) head_dot<HS>(c0, c1, wrow + 16 * h0, xb + 16 * h0);
                 y0 = silu_d(c0, d0); y1 = silu_d(c1, d1);
                 sm.y[0][2 * t][n] = y0; sm.y[0][2 * t + 1][n] = y1;
                 sm.sd[0][2 * t][n] = d0; sm.sd[0][2 * t + 1][n] = d1;
@@ -255,10 +385,7 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
 #pragma unroll 1
             for (int L = 1; L < HEAD_L; ++L) {
                 double c0 = hd[H.bias + L * HEAD_H + n], c1 = c0;
-                const double *wrow = hd + H.wl + (L - 1) * HEAD_H * HEAD_H + n * HEAD_H + t;
-                const double *xb = &sm.y[(L - 1) & 1][g][t];
-#pragma unroll
-                for (int ks = 0; ks < HEAD_H / 4; ++ks) dmma(c0, c1, wrow[4 * ks], xb[4 * ks]);
+                head_dot<HEAD_H / 16>(c0, c1, hd + H.wl + (L - 1) * HEAD_H * HEAD_H + n * HEAD_H + 4 * t, &sm.y[(L - 1) & 1][g][4 * t]);
                 y0 += silu_d(c0, d0); y1 += silu_d(c1, d1);
                 sm.y[L & 1][2 * t][n] = y0; sm.y[L & 1][2 * t + 1][n] = y1;
                 sm.sd[L][2 * t][n] = d0; sm.sd[L][2 * t + 1][n] = d1;
@@ -272,17 +399,15 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                 e_i += hd[H.wout + HEAD_H];
                 if (lane == 0 && have) { k.e_atom[i] = e_i; e_sum += e_i; }
             }
-            // reverse: this lane keeps dE/dy[n] of atoms 2t, 2t + 1; each hidden layer adds W^T (dE/dy . SiLU') through its skip
+            // reverse: this lane keeps dE/dy[n] of atoms 2t, 2t + 1; each hidden layer adds W^T (dE/dy . SiLU') through its
+            // skip.  The transposed copies make the reverse pass read weight rows exactly as the forward pass does.
             double g0 = hd[H.wout + n], g1 = g0;
             sm.dp[(HEAD_L - 1) & 1][2 * t][n] = g0 * sm.sd[HEAD_L - 1][2 * t][n];
             sm.dp[(HEAD_L - 1) & 1][2 * t + 1][n] = g1 * sm.sd[HEAD_L - 1][2 * t + 1][n];
             __syncthreads();
 #pragma unroll 1
             for (int L = HEAD_L - 1; L >= 1; --L) {
-                const double *wcol = hd + H.wl + (L - 1) * HEAD_H * HEAD_H + t * HEAD_H + n;   // A[n][o] = W[o][n]
-                const double *xb = &sm.dp[L & 1][g][t];
-#pragma unroll
-                for (int ks = 0; ks < HEAD_H / 4; ++ks) dmma(g0, g1, wcol[4 * ks * HEAD_H], xb[4 * ks]);
+                head_dot<HEAD_H / 16>(g0, g1, hd + H.wlt + (L - 1) * HEAD_H * HEAD_H + n * HEAD_H + 4 * t, &sm.dp[L & 1][g][4 * t]);
                 sm.dp[(L - 1) & 1][2 * t][n] = g0 * sm.sd[L - 1][2 * t][n];
                 sm.dp[(L - 1) & 1][2 * t + 1][n] = g1 * sm.sd[L - 1][2 * t + 1][n];
                 __syncthreads();
@@ -291,15 +416,13 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
 #pragma unroll 1
             for (int m = wid; m < NINV / 8; m += F64_TILE) {
                 double c0 = 0.0, c1 = 0.0;
-                const double *wcol = hd + H.w0 + (size_t)t * NINV + 8 * m + g;
-                const double *xb = &sm.dp[0][g][t];
-#pragma unroll
-                for (int ks = 0; ks < HEAD_H / 4; ++ks) dmma(c0, c1, wcol[(size_t)4 * ks * NINV], xb[4 * ks]);
+                head_dot<HEAD_H / 16>(c0, c1, hd + H.w0t + (size_t)(8 * m + g) * HEAD_H + 4 * t, &sm.dp[0][g][4 * t]);
                 sm.x[2 * t][8 * m + g] = c0; sm.x[2 * t + 1][8 * m + g] = c1;
             }
             __syncthreads();
         }
 
+        pc.mark(4);
         // W_i = dE_i/dP_i (Eq. 7)
         double *wi = sm.pw[wid].w;
 #pragma unroll
@@ -321,7 +444,6 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
         //     accumulators return through shared memory to lane = pair for the projection.  16 pairs per batch: the
         //     staging rows share the hand-over buffer with W_i's shared-memory copy, which is dead once the fragments are loaded.
         //   other shapes: lane = pair throughout, plain DFMA against W_i in shared memory, 32 pairs per batch.
-        constexpr bool TENSOR = CLOSED;
         constexpr int NB = TENSOR ? 16 : 32;
         constexpr int NT = (D + 7) / 8;            // n-tiles of the tensor form
         constexpr int BS = 10, VTS = 2 * 8 * NT + 2;   // staging rows: 4 b, 4 b', table offset | V then T (+ 2: lane = pair reads 16
@@ -341,7 +463,9 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
         }
         double *bs = reinterpret_cast<double *>(&sm.pw[wid]), *vt = bs + NB * BS;
 
+        pc.mark(5);
         auto process = [&](int nb) {
+            pc.mark(6);
             const int j = lane < nb ? queue[(qh + lane) & 63] : 0;
             double x = 0.0, y = 0.0, z = 0.0, rinv = 0.0, ux = 0.0, uy = 0.0, uz = 0.0;
             double b[4] = {0.0, 0.0, 0.0, 0.0}, db[4] = {0.0, 0.0, 0.0, 0.0};
@@ -366,6 +490,7 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                     row[8] = __longlong_as_double((long long)(cf - k.coef));
                 }
                 __syncwarp();
+                pc.mark(7);
 #pragma unroll 1
                 for (int grp = 0; grp < NB / 8; ++grp) {
                     if (8 * grp >= nb) break;
@@ -406,6 +531,7 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                     }
                 }
                 __syncwarp();
+                pc.mark(8);
                 if (lane < nb) {
                     double v[D_ANG], tt[D_ANG];   // components beyond d are zero and drop out of the projection
                     const double *rowv = vt + lane * VTS;
@@ -473,6 +599,7 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
             }
             qh = (qh + nb) & 63;
             nq -= nb;
+            pc.mark(9);
         };
 
         for (int64_t base = beg; base < end; base += 32) {   // compact the entries inside r_cut into the ring
@@ -504,8 +631,11 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
             atomicAdd(&k.force[3 * (size_t)i + 1], fy);
             atomicAdd(&k.force[3 * (size_t)i + 2], fz);
         }
+        pc.mark(6);
         __syncthreads();   // the next tile's encoding reuses the hand-over rows that alias W_i, and x
+        pc.mark(10);
     }
+    pc.flush(k.acc, lane);
 
 #pragma unroll
     for (int q = 0; q < 9; ++q) {
@@ -542,6 +672,9 @@ int upload_head_f64(mlip_ctx *c, const double *w) {
         for (int L = 0; L < HEAD_L; ++L) {
             double *row = L == 0 ? hp + H.w0 : hp + H.wl + (L - 1) * HEAD_H * HEAD_H;
             memcpy(row, src, sizeof(double) * HEAD_H * in);
+            double *tr = L == 0 ? hp + H.w0t : hp + H.wlt + (L - 1) * HEAD_H * HEAD_H;   // [in][64]
+            for (int o = 0; o < HEAD_H; ++o)
+                for (int q = 0; q < in; ++q) tr[(size_t)q * HEAD_H + o] = src[(size_t)o * in + q];
             memcpy(hp + H.bias + L * HEAD_H, src + in * HEAD_H, sizeof(double) * HEAD_H);
             src += in * HEAD_H + HEAD_H;
             in = HEAD_H;
