@@ -34,6 +34,7 @@
 
 namespace mlip {
 
+constexpr int F64_QCAP = 128;       // pairs per atom kept between the phases (more: the derivation scans the list again)
 constexpr int F64_TILE = 8;         // atoms per tile = warps per CTA = columns of the tensor-pipe tile
 constexpr int F64_YS = HEAD_H + 2;  // activation row stride: 2 mod 4 doubles keeps the 16-byte B-operand reads conflict-free
 
@@ -67,7 +68,7 @@ struct TileSmem {
         double w[D * K];                    // W_i = dE_i/dP_i (Eq. 7), derivation; P_i on its way from fragments to lane = channel
         double te[(D + 5) * 36];            // encoding hand-over of the tensor form: D rows of h, 4 of b, table offsets, 32 pairs (+ 4 pad) each
     } pw[F64_TILE];
-    int q[F64_TILE][64];                    // compacted neighbor indices
+    int q[F64_TILE][F64_QCAP];              // neighbor indices of the pairs inside r_cut: kept from the encoding to the derivation
 };
 
 struct F64Args {
@@ -203,6 +204,7 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
         for (int a = 0; a < D; ++a)
 #pragma unroll
             for (int q = 0; q < CPL; ++q) P[a][q] = 0.0;
+        int n_mine = 0;   // pairs of this warp's atom inside r_cut
         if constexpr (TENSOR) {
             double Pc[MT][NTK][2];
 #pragma unroll
@@ -227,9 +229,9 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                 }
                 const unsigned mask = __ballot_sync(0xffffffffu, valid);
                 const int nv = __popc(mask);
-                n_pairs += nv;
                 if (valid) {   // the pairs inside r_cut take consecutive columns of the hand-over rows
                     const int col = __popc(mask & ((1u << lane) - 1u));
+                    if (n_mine + col < F64_QCAP) sm.q[wid][n_mine + col] = j_e;
                     const double r = sqrt(d2), rinv = 1.0 / r;
                     double h[D_ANG], b[4];
                     harmonics(dx * rinv, dy * rinv, dz * rinv, h);
@@ -240,6 +242,7 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                     for (int m = 0; m < 4; ++m) bq[m * PS + col] = b[m];
                     offs[col] = __longlong_as_double(((long long)(si * C + sj) * (k.knots + 3) + iv) * K);
                 }
+                n_mine += nv;
                 __syncwarp();
                 pc.mark(0);
                 for (int p0 = 0; p0 < nv; p0 += 4) {
@@ -322,7 +325,11 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                     }
                 }
                 unsigned mask = __ballot_sync(0xffffffffu, valid);
-                n_pairs += __popc(mask);
+                if (valid) {
+                    const int col = __popc(mask & ((1u << lane) - 1u));
+                    if (n_mine + col < F64_QCAP) sm.q[wid][n_mine + col] = j_e;
+                }
+                n_mine += __popc(mask);
                 __syncwarp();
                 while (mask) {
                     const int p = __ffs(mask) - 1;
@@ -347,6 +354,7 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
             }
         }
 
+        n_pairs += n_mine;
         // ---------------- Invariants (Eq. 5: p^T C_l p); an empty slot of a ragged tile feeds zeros ----------------
 #pragma unroll
         for (int q = 0; q < CPL; ++q) {
@@ -466,7 +474,7 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
         pc.mark(5);
         auto process = [&](int nb) {
             pc.mark(6);
-            const int j = lane < nb ? queue[(qh + lane) & 63] : 0;
+            const int j = lane < nb ? queue[(qh + lane) & (F64_QCAP - 1)] : 0;
             double x = 0.0, y = 0.0, z = 0.0, rinv = 0.0, ux = 0.0, uy = 0.0, uz = 0.0;
             double b[4] = {0.0, 0.0, 0.0, 0.0}, db[4] = {0.0, 0.0, 0.0, 0.0};
             const double *cf = k.coef;
@@ -597,27 +605,31 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                 vir[3] -= y * qx; vir[4] -= y * qy; vir[5] -= y * qz;
                 vir[6] -= z * qx; vir[7] -= z * qy; vir[8] -= z * qz;
             }
-            qh = (qh + nb) & 63;
+            qh = (qh + nb) & (F64_QCAP - 1);
             nq -= nb;
             pc.mark(9);
         };
 
-        for (int64_t base = beg; base < end; base += 32) {   // compact the entries inside r_cut into the ring
-            const int64_t e = base + lane;
-            bool valid = false;
-            const int j = entry(e, e < end);
-            if (e < end) {
-                const double4 pj = k.pos4[j];
-                const double dx = min_image(pj.x - pi.x, k.grid.box[0], k.grid.half[0]);
-                const double dy = min_image(pj.y - pi.y, k.grid.box[1], k.grid.half[1]);
-                const double dz = min_image(pj.z - pi.z, k.grid.box[2], k.grid.half[2]);
-                valid = dx * dx + dy * dy + dz * dz < k.rc2;
+        if (n_mine <= F64_QCAP) {
+            nq = n_mine;   // the encoding left every pair of this atom in the queue
+        } else {
+            for (int64_t base = beg; base < end; base += 32) {   // compact the entries inside r_cut into the ring
+                const int64_t e = base + lane;
+                bool valid = false;
+                const int j = entry(e, e < end);
+                if (e < end) {
+                    const double4 pj = k.pos4[j];
+                    const double dx = min_image(pj.x - pi.x, k.grid.box[0], k.grid.half[0]);
+                    const double dy = min_image(pj.y - pi.y, k.grid.box[1], k.grid.half[1]);
+                    const double dz = min_image(pj.z - pi.z, k.grid.box[2], k.grid.half[2]);
+                    valid = dx * dx + dy * dy + dz * dz < k.rc2;
+                }
+                const unsigned m = __ballot_sync(0xffffffffu, valid);
+                if (valid) queue[(qh + nq + __popc(m & ((1u << lane) - 1u))) & (F64_QCAP - 1)] = j;
+                nq += __popc(m);
+                __syncwarp();
+                while (nq >= NB) { process(NB); __syncwarp(); }
             }
-            const unsigned m = __ballot_sync(0xffffffffu, valid);
-            if (valid) queue[(qh + nq + __popc(m & ((1u << lane) - 1u))) & 63] = j;
-            nq += __popc(m);
-            __syncwarp();
-            while (nq >= NB) { process(NB); __syncwarp(); }
         }
         while (nq > 0) { process(min(nq, NB)); __syncwarp(); }
 #pragma unroll

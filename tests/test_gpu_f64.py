@@ -100,6 +100,28 @@ def test_fp64_dense_neighborhood_matches_oracle():
     assert np.abs(out["forces"].cpu().numpy() - ref["forces"]).max() <= F_ATOL_F64
 
 
+@pytest.mark.parametrize("basis", [0, 1])
+def test_fp64_more_pairs_than_the_kept_queue_holds_matches_oracle(basis):
+    """A lattice compressed to ~150 pairs per atom: the derivation cannot take the pairs from the encoding's queue
+    (128 entries) and scans the list again.  Both the tensor-pipe form (basis 0) and the general form (canonical basis)."""
+    import paper_2608_16329_b200 as mlip
+    import workloads as wl
+    w = wl.make_workload(1, n_cells=5)
+    enc, head = wl.workload_weights(1, w.n_species)
+    model = oracle.Model(w.n_species, w.r_cut, enc, head, basis=basis)
+    pot = mlip.Potential(w.n_species, w.r_cut, 1.0, enc, head, w.masses, precision=1, basis=basis)
+    pos, box = 0.8 * w.pos, 0.8 * np.asarray(w.box)
+    pot.build_neighbors(pos, w.species, box)
+    out = pot.compute(want_e_atom=True)
+    pot.sync_status()
+    ref = oracle.evaluate(model, pos, w.species, box)
+    assert mlip.mlip_get_counters(pot.ctx)["pairs_in_cutoff"] > 140 * w.n_atoms
+    f = out["forces"].cpu().numpy()
+    assert abs(float(out["energy"].cpu()) - ref["energy"]) <= E_RTOL_F64 * abs(ref["energy"])
+    assert np.abs(f - ref["forces"]).max() <= F_ATOL_F64 * max(1.0, np.abs(ref["forces"]).max())
+    assert np.abs(out["e_atom"].cpu().numpy() - ref["e_atom"]).max() <= 1e-9 * max(1.0, np.abs(ref["e_atom"]).max())
+
+
 @pytest.mark.parametrize("k,l_max", [(16, 3), (64, 3), (32, 1), (32, 2), (16, 2), (64, 1)])
 def test_fp64_descriptor_shape_variants_match_oracle(k, l_max):
     """Radial width k and angular order l_max of the paper's ablations (Tables 6 and 7, Fig. 4(c)); the fp64 kernel is
