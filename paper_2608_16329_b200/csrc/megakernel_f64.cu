@@ -5,16 +5,20 @@
 // and for runs that want that accuracy.
 //
 //   CTA = 8 warps = a tile of 8 atoms of one central species (atoms in (species, cell) order)
-//   encoding    one warp per atom: lane = list entry for geometry, harmonics and spline basis; then
-//               lane = channel for g (Eq. 2) and the moment P (Eq. 4), the pair's h / basis handed
-//               over in shared memory; plain DFMA
+//   encoding    one warp per atom: lane = list entry for geometry, angular values and spline basis; then the
+//               moment P = H^T G (Eq. 4) on the fp64 tensor pipe (mma.sync m8n8k4, IEEE fp64 FMA chains), four
+//               pairs per step, with g (Eq. 2) evaluated straight into the B operand
 //   regression  the whole CTA on the tile: every layer is W [64 x in] times the tile's activations
-//               [in x 8 atoms] on the fp64 tensor pipe (mma.sync m8n8k4, IEEE fp64 FMA chains), warp =
-//               8 rows of W, so each weight is read from L2 once per tile instead of once per atom;
-//               the reverse pass uses the same row-major weights as the transposed operand
-//   derivation  one warp per atom, lane = pair after compacting the pairs inside r_cut: v = W g,
-//               t = W g' against W_i in shared memory, projection onto the pair vector, fp64
-//               atomics for f_j; table rows are read a 32-byte sector at a time
+//               [in x 8 atoms] on the fp64 tensor pipe, warp = 8 rows of W, so each weight is read from L2 once
+//               per tile instead of once per atom; the reverse pass reads transposed copies the same way
+//   derivation  one warp per atom: [V; T] = [G; G'] W^T (Eq. 9 and the re-associated Eq. 8 term) on the tensor
+//               pipe, eight pairs per tile, then lane = pair for the projection onto the pair vector and fp64
+//               atomics for f_j
+//
+// What bounds this kernel is the L1 / shared-memory data pipe and L2 latency, not fp64 arithmetic: every global
+// load is therefore shaped so that a quad or an eight-lane group reads 128 or 256 contiguous bytes (the k-index <->
+// channel assignment of a contraction is free), and the staging rows in shared memory are padded against bank
+// conflicts.
 //
 // The radial tables are the same clamped cubic B-splines as in the fp32 path but with fp64
 // coefficients and enough knots for ~1e-11 relative error; they stay in global memory (L2).
@@ -55,7 +59,6 @@ template <int K, int LMAX, int BASIS>
 struct TileSmem {
     using Shape = AngShape<LMAX, BASIS>;
     static constexpr int D = Shape::D;
-    static constexpr int ST = (D + 6) & ~1;   // hand-over row: D angular values, 4 spline weights, table offset, pad
     static constexpr int NINV = (LMAX + 1) * K;
     static constexpr int XS = (NINV + 31) / 32 * 32 + 2;
     double x[F64_TILE][XS];                 // invariants, then dE/dG
@@ -63,7 +66,6 @@ struct TileSmem {
     double sd[HEAD_L][F64_TILE][F64_YS];    // SiLU'(pre-activation) per layer
     double dp[2][F64_TILE][F64_YS];         // dE/dpre of the layer being propagated
     union {
-        double st[32][ST];                  // encoding hand-over
         double dv[16 * (12 + 16 * ((D + 7) / 8))];   // derivation staging of the tensor form: 16 pairs x (b, b', offset | V, T, pad)
         double w[D * K];                    // W_i = dE_i/dP_i (Eq. 7), derivation; P_i on its way from fragments to lane = channel
         double te[(D + 5) * 36];            // encoding hand-over of the tensor form: D rows of h, 4 of b, table offsets, 32 pairs (+ 4 pad) each
@@ -192,12 +194,10 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
         };
 
         // ---------------- Encoding: P = H^T G (Eq. 4) ----------------
-        // closed-form shapes (TENSOR): four pairs per m8n8k4 step on the fp64 tensor pipe.  A = H^T (rows = angular
-        //   components, k = pair), B = G (k = pair, columns = channels): lane (g, t) evaluates g of pair t at the K / 8
-        //   contiguous channels K/8 * g .., so the eight lanes of a pair read a whole table row per load and four rows are in
-        //   flight per step; the accumulators go through shared memory to lane = channel afterwards.
-        // other shapes: one pair at a time, lane = channel, plain DFMA.
-        constexpr bool TENSOR = CLOSED;
+        // Four pairs per m8n8k4 step on the fp64 tensor pipe.  A = H^T (rows = angular components, k = pair), B = G
+        // (k = pair, columns = channels): lane (g, t) evaluates g of pair t at the K / 8 contiguous channels K/8 * g ..,
+        // so the eight lanes of a pair read a whole table row per load and four rows are in flight per step; the
+        // accumulators go through shared memory to lane = channel afterwards.
         constexpr int MT = (D + 7) / 8, NTK = K / 8, PS = 36;   // PS = 4 mod 16 doubles: the A-fragment reads fall on 32 different banks
         double P[D][CPL];
 #pragma unroll
@@ -205,11 +205,11 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
 #pragma unroll
             for (int q = 0; q < CPL; ++q) P[a][q] = 0.0;
         int n_mine = 0;   // pairs of this warp's atom inside r_cut
-        if constexpr (TENSOR) {
+        {
             double Pc[MT][NTK][2];
-#pragma unroll
+    #pragma unroll
             for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
+    #pragma unroll
                 for (int nt = 0; nt < NTK; ++nt) Pc[mt][nt][0] = Pc[mt][nt][1] = 0.0;
             double *hs = sm.pw[wid].te, *bq = hs + D * PS, *offs = bq + 4 * PS;
             for (int64_t base = beg; base < end; base += 32) {
@@ -233,12 +233,13 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                     const int col = __popc(mask & ((1u << lane) - 1u));
                     if (n_mine + col < F64_QCAP) sm.q[wid][n_mine + col] = j_e;
                     const double r = sqrt(d2), rinv = 1.0 / r;
-                    double h[D_ANG], b[4];
-                    harmonics(dx * rinv, dy * rinv, dz * rinv, h);
+                    double h[D > D_ANG ? D : D_ANG], b[4];
+                    if (CLOSED) harmonics(dx * rinv, dy * rinv, dz * rinv, h);
+                    else angular_values<LMAX, BASIS>(dx * rinv, dy * rinv, dz * rinv, h);
                     const int iv = spline_basis<false, double>(r, k.r_min, k.inv_h, k.knots, b, nullptr, k.status);
-#pragma unroll
+    #pragma unroll
                     for (int a = 0; a < D; ++a) hs[a * PS + col] = h[a];
-#pragma unroll
+    #pragma unroll
                     for (int m = 0; m < 4; ++m) bq[m * PS + col] = b[m];
                     offs[col] = __longlong_as_double(((long long)(si * C + sj) * (k.knots + 3) + iv) * K);
                 }
@@ -250,27 +251,27 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                     const bool live = p < nv;   // a step past the last pair contracts zeros against the table's first rows
                     const double *cf = k.coef + (live ? __double_as_longlong(offs[p]) : 0ll) + NTK * g;
                     double gq[NTK];
-#pragma unroll
+    #pragma unroll
                     for (int nt = 0; nt < NTK; ++nt) gq[nt] = 0.0;
-#pragma unroll
+    #pragma unroll
                     for (int m = 0; m < 4; ++m) {
                         const double bm = live ? bq[m * PS + p] : 0.0;
                         double cc[NTK];
                         if constexpr (NTK == 2) {
                             asm volatile("ld.global.nc.v2.f64 {%0,%1}, [%2];" : "=d"(cc[0]), "=d"(cc[1]) : "l"(cf + m * K));
                         } else {
-#pragma unroll
+    #pragma unroll
                             for (int v = 0; v < NTK; v += 4)
                                 asm volatile("ld.global.nc.v4.f64 {%0,%1,%2,%3}, [%4];"
                                              : "=d"(cc[v]), "=d"(cc[v + 1]), "=d"(cc[v + 2]), "=d"(cc[v + 3]) : "l"(cf + m * K + v));
                         }
-#pragma unroll
+    #pragma unroll
                         for (int nt = 0; nt < NTK; ++nt) gq[nt] = fma(bm, cc[nt], gq[nt]);
                     }
-#pragma unroll
+    #pragma unroll
                     for (int mt = 0; mt < MT; ++mt) {
                         const double av = (live && 8 * mt + g < D) ? hs[(8 * mt + g) * PS + p] : 0.0;
-#pragma unroll
+    #pragma unroll
                         for (int nt = 0; nt < NTK; ++nt) dmma(Pc[mt][nt][0], Pc[mt][nt][1], av, gq[nt]);
                     }
                 }
@@ -279,79 +280,23 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
             }
             // fragments -> lane = channel: column n of n-tile nt is channel NTK n + nt
             double *pm = sm.pw[wid].w;
-#pragma unroll
+    #pragma unroll
             for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
+    #pragma unroll
                 for (int nt = 0; nt < NTK; ++nt)
-#pragma unroll
+    #pragma unroll
                     for (int u = 0; u < 2; ++u)
                         if (8 * mt + g < D) pm[(8 * mt + g) * K + NTK * (2 * t + u) + nt] = Pc[mt][nt][u];
             __syncwarp();
-#pragma unroll
+    #pragma unroll
             for (int q = 0; q < CPL; ++q) {
                 const int c = lane + 32 * q;
                 if (c < K) {
-#pragma unroll
+    #pragma unroll
                     for (int a = 0; a < D; ++a) P[a][q] = pm[a * K + c];
                 }
             }
             __syncwarp();   // W_i is written over the same buffer below
-        } else {
-            for (int64_t base = beg; base < end; base += 32) {
-                const int64_t e = base + lane;
-                bool valid = false;
-                const int j_e = entry(e, e < end);
-                if (e < end) {
-                    const int j = j_e;
-                    const double4 pj = k.pos4[j];
-                    const double dx = min_image(pj.x - pi.x, k.grid.box[0], k.grid.half[0]);
-                    const double dy = min_image(pj.y - pi.y, k.grid.box[1], k.grid.half[1]);
-                    const double dz = min_image(pj.z - pi.z, k.grid.box[2], k.grid.half[2]);
-                    const double d2 = dx * dx + dy * dy + dz * dz;
-                    valid = d2 < k.rc2;
-                    if (valid) {
-                        const double r = sqrt(d2), rinv = 1.0 / r;
-                        double h[CLOSED ? D_ANG : D], b[4];
-                        if (CLOSED) harmonics(dx * rinv, dy * rinv, dz * rinv, h);
-                        else angular_values<LMAX, BASIS>(dx * rinv, dy * rinv, dz * rinv, h);
-                        const int iv = spline_basis<false, double>(r, k.r_min, k.inv_h, k.knots, b, nullptr, k.status);
-                        double *row = sm.pw[wid].st[lane];
-    #pragma unroll
-                        for (int a = 0; a < D; ++a) row[a] = h[a];
-    #pragma unroll
-                        for (int m = 0; m < 4; ++m) row[D + m] = b[m];
-                        const long long off = ((long long)(si * C + (int)pj.w) * (k.knots + 3) + iv) * K;
-                        row[D + 4] = __longlong_as_double(off);
-                    }
-                }
-                unsigned mask = __ballot_sync(0xffffffffu, valid);
-                if (valid) {
-                    const int col = __popc(mask & ((1u << lane) - 1u));
-                    if (n_mine + col < F64_QCAP) sm.q[wid][n_mine + col] = j_e;
-                }
-                n_mine += __popc(mask);
-                __syncwarp();
-                while (mask) {
-                    const int p = __ffs(mask) - 1;
-                    mask &= mask - 1;
-                    const double *row = sm.pw[wid].st[p];
-                    const double *cf = k.coef + __double_as_longlong(row[D + 4]);
-    #pragma unroll
-                    for (int q = 0; q < CPL; ++q) {
-                        const int c = lane + 32 * q;
-                        double gq = 0.0;
-                        if (c < K) {
-                            gq = row[D] * cf[c];
-                            gq = fma(row[D + 1], cf[K + c], gq);
-                            gq = fma(row[D + 2], cf[2 * K + c], gq);
-                            gq = fma(row[D + 3], cf[3 * K + c], gq);
-                        }
-    #pragma unroll
-                        for (int a = 0; a < D; ++a) P[a][q] = fma(row[a], gq, P[a][q]);
-                    }
-                }
-                __syncwarp();
-            }
         }
 
         n_pairs += n_mine;
@@ -445,23 +390,23 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
         __syncwarp();
 
         // ---------------- Derivation (Eq. 8-10) ----------------
-        // The pairs inside r_cut are compacted into a ring of neighbor indices and taken NB at a time.
-        //   closed-form shapes (TENSOR): [V; T] = [G; G'] W^T (Eq. 9 and the re-associated Eq. 8 term) on the fp64 tensor
-        //     pipe, 8 pairs per m8n8k4 tile: lane (g, t) evaluates g, g' of pair g at channels 4 ks + t straight into the A
-        //     operand (the quad reads one 32-byte sector of each table row), W_i sits in registers as B fragments, the
-        //     accumulators return through shared memory to lane = pair for the projection.  16 pairs per batch: the
-        //     staging rows share the hand-over buffer with W_i's shared-memory copy, which is dead once the fragments are loaded.
-        //   other shapes: lane = pair throughout, plain DFMA against W_i in shared memory, 32 pairs per batch.
-        constexpr int NB = TENSOR ? 16 : 32;
+        // The pairs inside r_cut wait in the queue the encoding filled (a longer list is scanned again into a ring) and are
+        // taken NB at a time.
+        //   [V; T] = [G; G'] W^T (Eq. 9 and the re-associated Eq. 8 term) on the fp64 tensor pipe, 8 pairs per m8n8k4 tile:
+        //   lane (g, t) evaluates g, g' of pair g at channels 16 h + 4 t .. + 3 straight into the A operand (the quad reads
+        //   128 contiguous bytes of each table row), W_i sits in registers as B fragments, the accumulators return through
+        //   shared memory to lane = pair for the projection.  16 pairs per batch: the staging rows share the hand-over
+        //   buffer with W_i's shared-memory copy, which is dead once the fragments are loaded.
+        constexpr int NB = 16;
         constexpr int NT = (D + 7) / 8;            // n-tiles of the tensor form
         constexpr int BS = 10, VTS = 2 * 8 * NT + 2;   // staging rows: 4 b, 4 b', table offset | V then T (+ 2: lane = pair reads 16
                                                        // bytes at a 68-word stride, eight lanes on 32 different banks)
-        static_assert(!TENSOR || NB * (BS + VTS) * sizeof(double) <= sizeof(sm.pw[0]), "derivation staging must fit the hand-over buffer");
+        static_assert(NB * (BS + VTS) * sizeof(double) <= sizeof(sm.pw[0]), "derivation staging must fit the hand-over buffer");
         double fx = 0.0, fy = 0.0, fz = 0.0;
         int nq = 0, qh = 0;                        // ring: nq indices from position qh
         int *queue = sm.q[wid];
-        double Bf[TENSOR ? NT : 1][TENSOR ? K / 4 : 1];
-        if (TENSOR) {
+        double Bf[NT][K / 4];
+        {
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
@@ -490,7 +435,7 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                 cf = k.coef + ((size_t)(si * C + (int)pj.w) * (k.knots + 3) + iv) * K;
             }
             double s = 0.0, tx = 0.0, ty = 0.0, tz = 0.0, tu = 0.0;
-            if constexpr (TENSOR) {
+            {
                 if (lane < NB) {   // hand the spline weights and the table row to the tile's lanes
                     double *row = bs + lane * BS;
 #pragma unroll
@@ -541,56 +486,40 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                 __syncwarp();
                 pc.mark(8);
                 if (lane < nb) {
-                    double v[D_ANG], tt[D_ANG];   // components beyond d are zero and drop out of the projection
-                    const double *rowv = vt + lane * VTS;
+                    if constexpr (CLOSED) {
+                        double v[D_ANG], tt[D_ANG];   // components beyond d are zero and drop out of the projection
+                        const double *rowv = vt + lane * VTS;
 #pragma unroll
-                    for (int a = 0; a < D_ANG; a += 2) {
-                        double2 pv = make_double2(0.0, 0.0), pt = pv;
-                        if (a < 8 * NT) { pv = *reinterpret_cast<const double2 *>(rowv + a); pt = *reinterpret_cast<const double2 *>(rowv + 8 * NT + a); }
-                        v[a] = pv.x; v[a + 1] = pv.y; tt[a] = pt.x; tt[a + 1] = pt.y;
+                        for (int a = 0; a < D_ANG; a += 2) {
+                            double2 pv = make_double2(0.0, 0.0), pt = pv;
+                            if (a < 8 * NT) { pv = *reinterpret_cast<const double2 *>(rowv + a); pt = *reinterpret_cast<const double2 *>(rowv + 8 * NT + a); }
+                            v[a] = pv.x; v[a + 1] = pv.y; tt[a] = pt.x; tt[a + 1] = pt.y;
+                        }
+                        harmonics_project(ux, uy, uz, v, tt, s, tx, ty, tz, tu);
+                    } else {
+                        // the rows of the angular degrees L0 .. L1 projected at once; wide bases go through in two degree
+                        // ranges so that v and t stay in registers
+                        const double *rowv = vt + lane * VTS;
+                        auto rows_of = [&](auto l0c, auto l1c) {
+                            constexpr int L0 = decltype(l0c)::value, L1 = decltype(l1c)::value;
+                            constexpr int A0 = Shape::begin(L0), A1 = Shape::begin(L1 + 1);
+                            constexpr int DV = A1 - A0;
+                            double v[DV], tt[DV];
+#pragma unroll
+                            for (int a = 0; a < DV; ++a) { v[a] = rowv[A0 + a]; tt[a] = rowv[8 * NT + A0 + a]; }
+                            double ps, px, py, pz, pu;
+                            angular_project<LMAX, BASIS, L0, L1>(ux, uy, uz, v, tt, ps, px, py, pz, pu);
+                            s += ps; tx += px; ty += py; tz += pz; tu += pu;
+                        };
+                        if constexpr (D > 25) {
+                            rows_of(std::integral_constant<int, 0>{}, std::integral_constant<int, 3>{});
+                            rows_of(std::integral_constant<int, 4>{}, std::integral_constant<int, LMAX>{});
+                        } else {
+                            rows_of(std::integral_constant<int, 0>{}, std::integral_constant<int, LMAX>{});
+                        }
                     }
-                    harmonics_project(ux, uy, uz, v, tt, s, tx, ty, tz, tu);
                 }
                 __syncwarp();
-            } else if (lane < nb) {
-                // v = W g and t = W g' for the rows of the angular degrees L0 .. L1, projected at once; wide bases go
-                // through in two degree ranges so that v and t stay in registers
-                auto rows_of = [&](auto l0c, auto l1c) {
-                    constexpr int L0 = decltype(l0c)::value, L1 = decltype(l1c)::value;
-                    constexpr int A0 = Shape::begin(L0), A1 = Shape::begin(L1 + 1);
-                    constexpr int DV = A1 - A0;
-                    double v[DV], tt[DV];
-#pragma unroll
-                    for (int a = 0; a < DV; ++a) { v[a] = 0.0; tt[a] = 0.0; }
-#pragma unroll 1
-                    for (int c = 0; c < K; c += 4) {   // four channels = one 32-byte sector per table row
-                        double gv[4] = {0.0, 0.0, 0.0, 0.0}, dg[4] = {0.0, 0.0, 0.0, 0.0};
-#pragma unroll
-                        for (int m = 0; m < 4; ++m) {
-                            double cc[4];
-                            asm volatile("ld.global.nc.v4.f64 {%0,%1,%2,%3}, [%4];"
-                                         : "=d"(cc[0]), "=d"(cc[1]), "=d"(cc[2]), "=d"(cc[3]) : "l"(cf + m * K + c));
-#pragma unroll
-                            for (int u = 0; u < 4; ++u) { gv[u] = fma(b[m], cc[u], gv[u]); dg[u] = fma(db[m], cc[u], dg[u]); }
-                        }
-#pragma unroll
-                        for (int a = A0; a < A1; ++a) {
-                            const double2 w0 = *reinterpret_cast<const double2 *>(&wi[a * K + c]);
-                            const double2 w1 = *reinterpret_cast<const double2 *>(&wi[a * K + c + 2]);
-                            v[a - A0] = fma(w0.x, gv[0], fma(w0.y, gv[1], fma(w1.x, gv[2], fma(w1.y, gv[3], v[a - A0]))));
-                            tt[a - A0] = fma(w0.x, dg[0], fma(w0.y, dg[1], fma(w1.x, dg[2], fma(w1.y, dg[3], tt[a - A0]))));
-                        }
-                    }
-                    double ps, px, py, pz, pu;
-                    angular_project<LMAX, BASIS, L0, L1>(ux, uy, uz, v, tt, ps, px, py, pz, pu);
-                    s += ps; tx += px; ty += py; tz += pz; tu += pu;
-                };
-                if constexpr (D > 25) {
-                    rows_of(std::integral_constant<int, 0>{}, std::integral_constant<int, 3>{});
-                    rows_of(std::integral_constant<int, 4>{}, std::integral_constant<int, LMAX>{});
-                } else {
-                    rows_of(std::integral_constant<int, 0>{}, std::integral_constant<int, LMAX>{});
-                }
             }
             if (lane < nb) {
                 // f_ij = (g' . u_ij) r^ + J_ang^T v_ij,  J_ang = (grad_u h)(I - u u^T) / r
@@ -610,10 +539,11 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
             pc.mark(9);
         };
 
-        if (n_mine <= F64_QCAP) {
-            nq = n_mine;   // the encoding left every pair of this atom in the queue
-        } else {
-            for (int64_t base = beg; base < end; base += 32) {   // compact the entries inside r_cut into the ring
+        // one loop for both cases: with every pair already queued there is nothing to scan
+        const bool kept = n_mine <= F64_QCAP;
+        if (kept) nq = n_mine;
+        for (int64_t base = kept ? end : beg;;) {
+            if (base < end) {   // compact the next 32 list entries' pairs inside r_cut into the ring
                 const int64_t e = base + lane;
                 bool valid = false;
                 const int j = entry(e, e < end);
@@ -627,11 +557,13 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                 const unsigned m = __ballot_sync(0xffffffffu, valid);
                 if (valid) queue[(qh + nq + __popc(m & ((1u << lane) - 1u))) & (F64_QCAP - 1)] = j;
                 nq += __popc(m);
+                base += 32;
                 __syncwarp();
-                while (nq >= NB) { process(NB); __syncwarp(); }
             }
+            const bool last = base >= end;
+            while (nq >= NB || (last && nq > 0)) { process(min(nq, NB)); __syncwarp(); }
+            if (last) break;
         }
-        while (nq > 0) { process(min(nq, NB)); __syncwarp(); }
 #pragma unroll
         for (int o = 16; o; o >>= 1) {
             fx += __shfl_xor_sync(0xffffffffu, fx, o);
