@@ -195,8 +195,8 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
 
         // ---------------- Encoding: P = H^T G (Eq. 4) ----------------
         // Four pairs per m8n8k4 step on the fp64 tensor pipe.  A = H^T (rows = angular components, k = pair), B = G
-        // (k = pair, columns = channels): lane (g, t) evaluates g of pair t at the K / 8 contiguous channels K/8 * g ..,
-        // so the eight lanes of a pair read a whole table row per load and four rows are in flight per step; the
+        // (k = pair, columns = channels): lane (g, t) evaluates g of pair t at channels 16 q + 2 g, + 1 (q < K / 16), so the
+        // eight lanes of a pair read 128 contiguous bytes of a table row per load and four rows are in flight per step; the
         // accumulators go through shared memory to lane = channel afterwards.
         constexpr int MT = (D + 7) / 8, NTK = K / 8, PS = 36;   // PS = 4 mod 16 doubles: the A-fragment reads fall on 32 different banks
         double P[D][CPL];
@@ -249,26 +249,21 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                 for (int p0 = 0; p0 < nv; p0 += 4) {
                     const int p = p0 + t;
                     const bool live = p < nv;   // a step past the last pair contracts zeros against the table's first rows
-                    const double *cf = k.coef + (live ? __double_as_longlong(offs[p]) : 0ll) + NTK * g;
+                    const double *cf = k.coef + (live ? __double_as_longlong(offs[p]) : 0ll) + 2 * g;
                     double gq[NTK];
-    #pragma unroll
+#pragma unroll
                     for (int nt = 0; nt < NTK; ++nt) gq[nt] = 0.0;
-    #pragma unroll
+#pragma unroll
                     for (int m = 0; m < 4; ++m) {
                         const double bm = live ? bq[m * PS + p] : 0.0;
                         double cc[NTK];
-                        if constexpr (NTK == 2) {
-                            asm volatile("ld.global.nc.v2.f64 {%0,%1}, [%2];" : "=d"(cc[0]), "=d"(cc[1]) : "l"(cf + m * K));
-                        } else {
-    #pragma unroll
-                            for (int v = 0; v < NTK; v += 4)
-                                asm volatile("ld.global.nc.v4.f64 {%0,%1,%2,%3}, [%4];"
-                                             : "=d"(cc[v]), "=d"(cc[v + 1]), "=d"(cc[v + 2]), "=d"(cc[v + 3]) : "l"(cf + m * K + v));
-                        }
-    #pragma unroll
+#pragma unroll
+                        for (int v = 0; v < NTK; v += 2)   // 16 bytes per lane: the eight lanes of a pair read 128 contiguous bytes
+                            asm volatile("ld.global.nc.v2.f64 {%0,%1}, [%2];" : "=d"(cc[v]), "=d"(cc[v + 1]) : "l"(cf + m * K + 8 * v));
+#pragma unroll
                         for (int nt = 0; nt < NTK; ++nt) gq[nt] = fma(bm, cc[nt], gq[nt]);
                     }
-    #pragma unroll
+#pragma unroll
                     for (int mt = 0; mt < MT; ++mt) {
                         const double av = (live && 8 * mt + g < D) ? hs[(8 * mt + g) * PS + p] : 0.0;
     #pragma unroll
@@ -278,7 +273,7 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                 __syncwarp();
                 pc.mark(1);
             }
-            // fragments -> lane = channel: column n of n-tile nt is channel NTK n + nt
+            // fragments -> lane = channel: column n of n-tile nt is channel 16 (nt / 2) + 2 n + nt % 2
             double *pm = sm.pw[wid].w;
     #pragma unroll
             for (int mt = 0; mt < MT; ++mt)
@@ -286,7 +281,7 @@ __global__ void __launch_bounds__(F64_TILE * 32, f64_ctas_per_sm<K, LMAX, BASIS>
                 for (int nt = 0; nt < NTK; ++nt)
     #pragma unroll
                     for (int u = 0; u < 2; ++u)
-                        if (8 * mt + g < D) pm[(8 * mt + g) * K + NTK * (2 * t + u) + nt] = Pc[mt][nt][u];
+                        if (8 * mt + g < D) pm[(8 * mt + g) * K + 16 * (nt >> 1) + 2 * (2 * t + u) + (nt & 1)] = Pc[mt][nt][u];
             __syncwarp();
     #pragma unroll
             for (int q = 0; q < CPL; ++q) {
