@@ -113,7 +113,7 @@ struct mlip_ctx {
     int64_t *nbr_off = nullptr;    // [N + 1]
     int32_t *nbr = nullptr;        // list entries: int32 indices, or uint16 cell-relative codes when list16
     bool list16 = false;           // format of the current lists (mlip_config.list_format = 1 on a grid of >= 3 cells per edge)
-    int32_t *cell_id = nullptr;    // [N] build-time cell of each atom, internal order (allocated for list_format = 1)
+    int32_t *cell_id = nullptr;    // [N] build-time cell of each atom as packed coordinates, internal order (allocated for list_format = 1)
     unsigned long long *tile_state = nullptr;   // [ceil(N / 64) + 1] look-back words of the one-pass rebuild
     int *tile_ticket = nullptr;
     int64_t nbr_cap = 0, n_entries = 0;
@@ -195,8 +195,15 @@ int launch_get_state(mlip_ctx *c, double *pos, double *vel, cudaStream_t s);
 
 // Compact list entries (neighbor.cu): cell number in the 27-cell traversal order << L16_SHIFT | position inside that cell.
 constexpr int L16_SHIFT = 11, L16_MASK = (1 << L16_SHIFT) - 1;
+// cell_id[] holds an atom's build-time cell as packed coordinates (10 bits each: no division on the way to the 27 cell
+// bases an atom's list needs); grids with more than 1,024 cells along a dimension keep int32 lists.
+constexpr int CELL_PACK_BITS = 10, CELL_PACK_MAX = 1 << CELL_PACK_BITS;
+__host__ __device__ inline int pack_cell(const CellGrid &g, int linear) {
+    const int cz = linear % g.n[2], cy = (linear / g.n[2]) % g.n[1], cx = linear / (g.n[2] * g.n[1]);
+    return cx | (cy << CELL_PACK_BITS) | (cz << (2 * CELL_PACK_BITS));
+}
 __host__ __device__ inline int neighbor_cell(const CellGrid &g, int cid, int it) {
-    const int cz = cid % g.n[2], cy = (cid / g.n[2]) % g.n[1], cx = cid / (g.n[2] * g.n[1]);
+    const int cx = cid & (CELL_PACK_MAX - 1), cy = (cid >> CELL_PACK_BITS) & (CELL_PACK_MAX - 1), cz = cid >> (2 * CELL_PACK_BITS);
     int x = cx + it / 9 - 1, y = cy + (it / 3) % 3 - 1, z = cz + it % 3 - 1;
     x = x < 0 ? x + g.n[0] : (x >= g.n[0] ? x - g.n[0] : x);
     y = y < 0 ? y + g.n[1] : (y >= g.n[1] ? y - g.n[1] : y);

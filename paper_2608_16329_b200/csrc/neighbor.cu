@@ -102,11 +102,11 @@ __global__ void k_sort_cells(int n_cells, int n_species, const int32_t *__restri
 __global__ void k_gather(int64_t n, const int32_t *__restrict__ slot_src, const double4 *__restrict__ pos4_src,
                          const double *__restrict__ vel_src, const int32_t *__restrict__ user_src,
                          double4 *__restrict__ pos4, double *__restrict__ vel, int32_t *__restrict__ user_of,
-                         float *__restrict__ disp, const int32_t *__restrict__ cell_of, int32_t *__restrict__ cell_id) {
+                         float *__restrict__ disp, const int32_t *__restrict__ cell_of, int32_t *__restrict__ cell_id, CellGrid g) {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     int src = slot_src[i];
-    if (cell_id) cell_id[i] = cell_of[src];   // build-time cell of the atom in the internal order (compact lists)
+    if (cell_id) cell_id[i] = pack_cell(g, cell_of[src]);   // build-time cell of the atom in the internal order (compact lists)
     pos4[i] = pos4_src[src];
     user_of[i] = user_src[src];
     for (int a = 0; a < 3; ++a) {
@@ -636,7 +636,7 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
     int32_t *slot_src = c->nbr_count;
     k_place<<<blocks_for(n, 256), 256, 0, s>>>(c->cell_of, n, c->cell_start, c->cell_fill, slot_src);
     k_sort_cells<<<blocks_for(g.n_cells, 128), 128, 0, s>>>(g.n_cells, C, c->cell_start, slot_src, c->pos4_src, c->user_src, c->bin_count, c->status, (int32_t)c->n_owned);
-    k_gather<<<blocks_for(n, 256), 256, 0, s>>>(n, slot_src, c->pos4_src, c->vel_src, c->user_src, c->pos4, c->vel, c->user_of, c->disp, c->cell_of, c->cell_id);
+    k_gather<<<blocks_for(n, 256), 256, 0, s>>>(n, slot_src, c->pos4_src, c->vel_src, c->user_src, c->pos4, c->vel, c->user_of, c->disp, c->cell_of, c->cell_id, g);
     exclusive_scan<int32_t, int32_t>(c->bin_count, c->bin_start, (int64_t)C * g.n_cells, c->scan_tmp, s);
     int nthreads_co = g.n_cells > C + 1 ? g.n_cells : C + 1;
     k_center_order<<<blocks_for(nthreads_co, 128), 128, 0, s>>>(g.n_cells, C, c->cell_start, c->pos4, c->bin_start, c->center_order, c->species_start, c->user_of, (int32_t)c->n_owned);
@@ -645,7 +645,7 @@ int launch_build(mlip_ctx *c, bool allow_sync_grow, cudaStream_t s) {
     float4 *relpos = c->force;
     // entry format of this build: 16-bit cell-relative codes if asked for and the grid has 27 distinct cells around every
     // cell, else plain indices.  A change of format gives up the old array (its capacity is counted in entries).
-    const bool list16 = c->cfg.list_format == 1 && rel;
+    const bool list16 = c->cfg.list_format == 1 && rel && std::max(g.n[0], std::max(g.n[1], g.n[2])) <= CELL_PACK_MAX;
     if (list16 != c->list16 && c->nbr) {
         cudaFree(c->nbr);
         c->resident -= (c->list16 ? sizeof(uint16_t) : sizeof(int32_t)) * c->nbr_cap;
