@@ -69,6 +69,7 @@ constexpr int HB_PART = HB_DP + TILE * 2 * Z_STRIDE;       // split-K partials  
 constexpr int HB_WORDS = HB_PART + 2 * TILE * Z_STRIDE;
 static_assert(HB_WORDS <= TILE * SCR_WORDS, "head buffers alias the scratch of the group's warps");
 constexpr int HC_WORDS = HEAD_L * HEAD_H + HEAD_H + 16;         // biases, w_out, b_out of the current species
+constexpr int64_t STAGGER_BELOW_ATOMS = 200000;                 // systems below this size start their CTAs on different species
 constexpr int PF_IDX = 160;                                     // neighbor indices prefetched per warp for its next atom
 constexpr int PF_CS = 96;                                       // compact lists: the codes take 81 words at most, the 27 cell bases sit here
 static_assert(PF_IDX / 2 + 1 <= PF_CS && PF_CS + 27 <= PF_IDX, "prefetch buffer layout for compact lists");
@@ -899,7 +900,7 @@ __device__ __forceinline__ void head_tile(const KernelArgs &k, float *sX, float 
     group_sync(group);
 }
 
-template <bool TAB_SMEM, bool DET, bool L16>
+template <bool TAB_SMEM, bool DET, bool L16, bool STAGGER>
 __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words) {
     extern __shared__ __align__(16) float smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -940,11 +941,19 @@ __global__ void __launch_bounds__(NW * 32, 1) k_mega(KernelArgs k, int tab_words
     PhaseClock pc;
     pc.start();
 
-    for (int species = 0; species < k.n_species; ++species) {
+    // STAGGER (small systems): the CTAs start on different central species, so that the species are worked on side by
+    // side rather than one after the other by mostly idle SMs (864 atoms: 64 instead of 92 us).  Large systems keep the
+    // plain loop: one front through the cell-ordered atoms, and a loop counter as the species costs 1 % less than a
+    // computed one.  Either way a species whose tiles are all claimed already is passed over: staging its tables would
+    // be the only thing left to do.
+    for (int ss = 0; ss < k.n_species; ++ss) {
+        const int species = STAGGER ? (int)((ss + blockIdx.x) % (unsigned)k.n_species) : ss;
         const int s_beg = __ldg(k.species_start + species), s_end = __ldg(k.species_start + species + 1);
         const int n_tiles = (s_end - s_beg + TILE - 1) / TILE;
         if (n_tiles == 0) continue;
+        if (threadIdx.x == 0) ctl[6 + (ss & 1)] = *reinterpret_cast<volatile int *>(k.tile_counter + species);
         __syncthreads();   // both groups are done with the previous species' tables
+        if (ctl[6 + (ss & 1)] >= n_tiles) continue;
         if (TAB_SMEM) {
             const float4 *src = reinterpret_cast<const float4 *>(k.tab.coef + (size_t)species * k.n_species * rows * K_RADIAL);
             const int n4 = k.n_species * rows * (K_RADIAL / 4);
@@ -1188,12 +1197,16 @@ int launch_megakernel(mlip_ctx *c, cudaStream_t s) {
     const bool in_smem = tables_fit_smem(c);
     const int tab_words = in_smem ? table_smem_words(c) : 0;
     const size_t smem_bytes = sizeof(float) * (size_t)(FIXED_WORDS + tab_words);
-    // instantiations: tables in shared / global memory x floating-point / integer scatter x int32 / 16-bit lists
+    // instantiations: tables in shared / global memory x floating-point / integer scatter x int32 / 16-bit lists, and the
+    // shared-memory ones again with staggered species for small systems
     using Kernel = void (*)(KernelArgs, int);
-    static const Kernel kernels[8] = {k_mega<false, false, false>, k_mega<false, false, true>, k_mega<false, true, false>, k_mega<false, true, true>,
-                                      k_mega<true, false, false>,  k_mega<true, false, true>,  k_mega<true, true, false>,  k_mega<true, true, true>};
+    static const Kernel kernels[12] = {k_mega<false, false, false, false>, k_mega<false, false, true, false>, k_mega<false, true, false, false>,
+                                       k_mega<false, true, true, false>,   k_mega<true, false, false, false>, k_mega<true, false, true, false>,
+                                       k_mega<true, true, false, false>,   k_mega<true, true, true, false>,   k_mega<true, false, false, true>,
+                                       k_mega<true, false, true, true>,    k_mega<true, true, false, true>,   k_mega<true, true, true, true>};
+    const bool stagger = in_smem && n < STAGGER_BELOW_ATOMS;
     if (!c->kernel_ready) {
-        for (int q = 0; q < 8; ++q) {
+        for (int q = 0; q < 12; ++q) {
             const size_t bytes = sizeof(float) * (size_t)(FIXED_WORDS + (q >= 4 ? tab_words : 0));
             cudaError_t e = cudaFuncSetAttribute((const void *)kernels[q], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
             if (e != cudaSuccess) { c->err = std::string("fused kernel shared memory: ") + cudaGetErrorString(e); return MLIP_ERR_CUDA; }
@@ -1209,7 +1222,7 @@ int launch_megakernel(mlip_ctx *c, cudaStream_t s) {
     k.acc = c->acc; k.pair_counter = c->pair_counter; k.status = c->status; k.tile_counter = c->tile_counter;
     const int slot = (int)(c->ev_count % mlip_ctx::EV_POOL);
     MLIP_CUDA_TRY(c, cudaEventRecord(c->ev[2 * slot], s));
-    kernels[(in_smem ? 4 : 0) + (det ? 2 : 0) + (c->list16 ? 1 : 0)]<<<blocks, NW * 32, smem_bytes, s>>>(k, tab_words);
+    kernels[(stagger ? 8 : in_smem ? 4 : 0) + (det ? 2 : 0) + (c->list16 ? 1 : 0)]<<<blocks, NW * 32, smem_bytes, s>>>(k, tab_words);
     if (det) {
         k_fixed_finish<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(n, c->force_fx, c->acc_fx, c->force, c->acc);
         c->launches += 1;
