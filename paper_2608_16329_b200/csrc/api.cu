@@ -240,15 +240,16 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
     c->n_sm = prop.multiProcessorCount;
     do {
         if ((rc = dev_alloc(c, &c->mass, (size_t)cfg->n_species)) != MLIP_OK) break;
-        if ((rc = dev_alloc(c, &c->acc, (size_t)ACC_COUNT)) != MLIP_OK) break;
-        if ((rc = dev_alloc(c, &c->pair_counter, 1)) != MLIP_OK) break;
+        if ((rc = dev_alloc(c, &c->launch_block, (size_t)LB_COUNT)) != MLIP_OK) break;
+        c->tile_counter = reinterpret_cast<int *>(c->launch_block);
+        c->pair_counter = reinterpret_cast<unsigned long long *>(c->launch_block + LB_PAIR);
+        c->acc_fx = reinterpret_cast<long long *>(c->launch_block + LB_ACC_FX);
+        c->acc = c->launch_block + LB_ACC;
         if ((rc = dev_alloc(c, &c->status, 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->rebuild_flag, 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->far_flag, 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->nhc, 8)) != MLIP_OK) break;
-        if ((rc = dev_alloc(c, &c->acc_fx, 10)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->tile_ticket, 2)) != MLIP_OK) break;   // ticket, private overflow flag
-        if ((rc = dev_alloc(c, &c->tile_counter, (size_t)MAX_SPECIES)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->species_start, (size_t)MAX_SPECIES + 1)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->stage_out, 10)) != MLIP_OK) break;
         if ((rc = dev_alloc(c, &c->kin_part, 1184)) != MLIP_OK) break;
@@ -264,7 +265,7 @@ int mlip_create(mlip_ctx **out, const mlip_config *cfg, const double *enc_w, siz
         if (!ev_ok) { rc = MLIP_ERR_CUDA; c->err = "event creation failed"; break; }
         if (cudaMemcpy(c->mass, mass, sizeof(double) * cfg->n_species, cudaMemcpyHostToDevice) != cudaSuccess ||
             cudaMemset(c->status, 0, sizeof(int)) != cudaSuccess || cudaMemset(c->rebuild_flag, 0, sizeof(int)) != cudaSuccess ||
-            cudaMemset(c->nhc, 0, sizeof(double) * 8) != cudaSuccess || cudaMemset(c->acc, 0, sizeof(double) * ACC_COUNT) != cudaSuccess) {
+            cudaMemset(c->nhc, 0, sizeof(double) * 8) != cudaSuccess || cudaMemset(c->launch_block, 0, sizeof(double) * LB_COUNT) != cudaSuccess) {
             rc = MLIP_ERR_CUDA; c->err = "initial upload failed"; break;
         }
         if ((rc = f64 ? upload_head_f64(c, head_w) : upload_head(c, head_w)) != MLIP_OK) break;
@@ -685,7 +686,7 @@ void mlip_destroy(mlip_ctx *c) {
     free_cells(c);
     cudaFree(c->nbr); cudaFree(c->scan_tmp); cudaFree(c->head_w); cudaFree(c->table); cudaFree(c->mass);
     cudaFree(c->head_w_d); cudaFree(c->table_d);
-    cudaFree(c->acc); cudaFree(c->pair_counter); cudaFree(c->status); cudaFree(c->rebuild_flag); cudaFree(c->far_flag); cudaFree(c->nhc); cudaFree(c->acc_fx); cudaFree(c->tile_ticket); cudaFree(c->tile_counter);
+    cudaFree(c->launch_block); cudaFree(c->status); cudaFree(c->rebuild_flag); cudaFree(c->far_flag); cudaFree(c->nhc); cudaFree(c->tile_ticket);
     cudaFree(c->species_start); cudaFree(c->stage_pos); cudaFree(c->stage_species); cudaFree(c->stage_force);
     cudaFree(c->stage_out); cudaFree(c->kin_part);
     if (c->status_host) cudaFreeHost(c->status_host);

@@ -44,6 +44,11 @@ enum : int {
 
 // accumulator slots (double)
 enum : int { ACC_ENERGY = 0, ACC_VIRIAL = 1, ACC_KINETIC = 10, ACC_COUNT = 32 };
+// launch_block in doubles: [0, 4) tile_counter (MAX_SPECIES ints), [4] pair_counter, [5, 15) acc_fx, [16, 16 + ACC_COUNT) acc;
+// everything up to the kinetic-energy slot of acc is cleared before every fused-kernel launch
+constexpr int LB_PAIR = 4, LB_ACC_FX = 5, LB_ACC = 16, LB_COUNT = LB_ACC + ACC_COUNT;
+constexpr size_t LAUNCH_CLEAR_BYTES = sizeof(double) * (LB_ACC + ACC_KINETIC);
+static_assert(MAX_SPECIES * sizeof(int) <= LB_PAIR * sizeof(double), "tile counters must fit before the pair counter");
 
 struct CellGrid {
     int n[3];          // cells per dimension
@@ -120,7 +125,9 @@ struct mlip_ctx {
     // scratch
     int64_t *scan_tmp = nullptr;   // block sums for the scans
     int64_t scan_tmp_cap = 0;
-    double *acc = nullptr;         // [ACC_COUNT]
+    double *launch_block = nullptr;   // one allocation: tile_counter, pair_counter, acc_fx, acc back to back, so that a launch
+                                      // clears its counters and accumulators with a single memset (LAUNCH_CLEAR_BYTES)
+    double *acc = nullptr;         // [ACC_COUNT] (inside launch_block)
     double *kin_part = nullptr;    // [1184] per-block kinetic-energy sums (integrate.cu)
     unsigned long long *pair_counter = nullptr;
     int *status = nullptr;         // device status word

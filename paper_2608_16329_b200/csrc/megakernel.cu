@@ -1184,14 +1184,9 @@ __global__ void k_fixed_finish(int64_t n, const long long *__restrict__ force_fx
 int launch_megakernel(mlip_ctx *c, cudaStream_t s) {
     const int64_t n = c->n;
     const bool det = c->cfg.force_mode == 1;
-    if (det) {
-        MLIP_CUDA_TRY(c, cudaMemsetAsync(c->force_fx, 0, sizeof(long long) * 3 * n, s));
-        MLIP_CUDA_TRY(c, cudaMemsetAsync(c->acc_fx, 0, sizeof(long long) * 10, s));
-    }
+    if (det) MLIP_CUDA_TRY(c, cudaMemsetAsync(c->force_fx, 0, sizeof(long long) * 3 * n, s));
     MLIP_CUDA_TRY(c, cudaMemsetAsync(c->force, 0, sizeof(float4) * n, s));
-    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->acc, 0, sizeof(double) * ACC_KINETIC, s));
-    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->pair_counter, 0, sizeof(unsigned long long), s));
-    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->tile_counter, 0, sizeof(int) * MAX_SPECIES, s));
+    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->launch_block, 0, LAUNCH_CLEAR_BYTES, s));   // tile and pair counters, integer and fp64 accumulators
     const int64_t tiles_max = (n + TILE - 1) / TILE + c->cfg.n_species;
     const int blocks = (int)std::min<int64_t>(tiles_max, (int64_t)c->n_sm);
     const bool in_smem = tables_fit_smem(c);

@@ -662,8 +662,7 @@ bool f64_shape_supported(int k, int l_max, int basis) {
 int launch_megakernel_f64(mlip_ctx *c, cudaStream_t s) {
     const int64_t n = c->n;
     MLIP_CUDA_TRY(c, cudaMemsetAsync(c->force_d, 0, sizeof(double) * 3 * n, s));
-    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->acc, 0, sizeof(double) * ACC_KINETIC, s));
-    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->pair_counter, 0, sizeof(unsigned long long), s));
+    MLIP_CUDA_TRY(c, cudaMemsetAsync(c->launch_block, 0, LAUNCH_CLEAR_BYTES, s));   // pair counter and accumulators
     F64Args k;
     k.n = n; k.n_species = c->cfg.n_species; k.grid = c->grid; k.rc2 = c->cfg.r_cut * c->cfg.r_cut;
     k.coef = c->table_d; k.knots = c->cfg.table_knots; k.r_min = c->cfg.table_r_min;
