@@ -2,6 +2,7 @@
 import os
 import socket
 
+import pytest
 import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
@@ -126,3 +127,11 @@ def test_traffic_record_is_tied_to_the_kernel_sources(tmp_path, monkeypatch):
     rec.write_text("kernel_revision: 0123456789abcdef\ndram_bytes_per_atom: 700.5\n")
     value, why = bench.recorded_traffic()
     assert value is None and "revision" in why
+
+
+def test_time_step_shrinks_for_runs_beyond_the_stable_horizon_of_the_synthetic_potential():
+    """The default run keeps the benchmark's 1 fs; a longer run covers the same simulated time in more, smaller steps."""
+    import bench
+    assert bench.time_step_fs(3 + 20) == 1.0
+    assert bench.time_step_fs(5 + 100) == pytest.approx(bench.SAFE_TRAJECTORY_FS / 105)
+    assert bench.time_step_fs(0) == 1.0
