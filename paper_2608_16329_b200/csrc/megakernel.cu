@@ -636,14 +636,16 @@ __device__ __forceinline__ void tmem_fill_role(uint32_t region, const float *__r
         const float4 v = __ldg(rec + lane);
         tmem_st4(region + col, __float_as_uint(v.x), __float_as_uint(v.y), __float_as_uint(v.z), __float_as_uint(v.w));
     };
-#pragma unroll 1
+    // (the loops are unrolled so that a warp has 8 to 16 loads in flight: one L2 round trip per group of records instead of
+    // one per record, which is what a small system's kernel time is made of)
+#pragma unroll
     for (int q = 0; q < 8; ++q) {
         as_is(TM_FWD0 + 4 * q, fwd + (size_t)(mt4 * KS0 + kh * 8 + q) * 32);
         as_is(TM_BWD0 + 4 * q, bwd + (size_t)(wg * 8 + q) * 32);
     }
 #pragma unroll 1
     for (int b = 0; b < HEAD_L - 1; ++b)
-#pragma unroll 1
+#pragma unroll
         for (int q = 0; q < 4; ++q) {
             {   // forward: hi, lo of the rounded split
                 const float4 v = __ldg(fwd + (size_t)(4 * KS0 + b * 4 * KS1 + mt4 * KS1 + kh * 4 + q) * 32 + lane);
