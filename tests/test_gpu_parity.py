@@ -503,3 +503,25 @@ def test_smaller_descriptor_shapes_run_in_the_fp32_kernel(k, l_max):
     assert abs(float(out["energy"].cpu()) - ref["energy"]) <= E_RTOL * abs(ref["energy"])
     assert np.abs(out["forces"].cpu().numpy() - ref["forces"]).max() <= F_ATOL * f_scale
     assert np.abs(out["e_atom"].cpu().numpy() - ref["e_atom"]).max() <= 2e-5 * max(1.0, np.abs(ref["e_atom"]).max())
+
+
+@pytest.mark.parametrize("precision,list_format", [(0, 0), (0, 1), (1, 0)])
+def test_eight_species_the_maximum_count_match_oracle(precision, list_format):
+    """Eight species: 64 encoders, whose tables no longer fit shared memory, so the fused kernel reads them from global
+    memory (its other table path); species drawn at random over the 500-atom lattice."""
+    import paper_2608_16329_b200 as mlip
+    import workloads as wl
+    n_species = 8
+    w = wl.make_workload(1, n_cells=5)
+    species = np.random.default_rng(3).integers(0, n_species, w.n_atoms).astype(np.int32)
+    enc, head = wl.make_weights(n_species, 77, wl.ENC_OUT_SCALE[1], wl.HEAD_OUT_SCALE[1])
+    model = oracle.Model(n_species, w.r_cut, enc, head)
+    pot = mlip.Potential(n_species, w.r_cut, 1.0, enc, head, np.linspace(20.0, 90.0, n_species), precision=precision, list_format=list_format)
+    pot.build_neighbors(w.pos, species, w.box)
+    out = pot.compute(want_e_atom=True)
+    pot.sync_status()
+    ref = oracle.evaluate(model, w.pos, species, w.box)
+    e_tol, f_tol = (1e-10, 2e-9) if precision else (1e-6, 1e-4)
+    assert abs(float(out["energy"].cpu()) - ref["energy"]) <= e_tol * abs(ref["energy"])
+    assert np.abs(out["forces"].cpu().numpy() - ref["forces"]).max() <= f_tol
+    assert np.abs(out["e_atom"].cpu().numpy() - ref["e_atom"]).max() <= (1e-9 if precision else 2e-5) * max(1.0, np.abs(ref["e_atom"]).max())
