@@ -525,3 +525,28 @@ def test_eight_species_the_maximum_count_match_oracle(precision, list_format):
     assert abs(float(out["energy"].cpu()) - ref["energy"]) <= e_tol * abs(ref["energy"])
     assert np.abs(out["forces"].cpu().numpy() - ref["forces"]).max() <= f_tol
     assert np.abs(out["e_atom"].cpu().numpy() - ref["e_atom"]).max() <= (1e-9 if precision else 2e-5) * max(1.0, np.abs(ref["e_atom"]).max())
+
+
+@pytest.mark.parametrize("precision", [0, 1])
+def test_absent_species_and_a_species_with_one_atom_match_oracle(precision):
+    """Four species declared, two of them without atoms and one with a single atom: empty species ranges and a ragged
+    one-atom tile, followed by a few steps with an in-step rebuild."""
+    import paper_2608_16329_b200 as mlip
+    import workloads as wl
+    n_species = 4
+    w = wl.make_workload(1, n_cells=4)
+    species = np.where(np.arange(w.n_atoms) % 3 == 0, 0, 2).astype(np.int32)
+    species[7] = 3
+    enc, head = wl.make_weights(n_species, 78, wl.ENC_OUT_SCALE[1], wl.HEAD_OUT_SCALE[1])
+    model = oracle.Model(n_species, w.r_cut, enc, head)
+    pot = mlip.Potential(n_species, w.r_cut, 1.0, enc, head, np.linspace(20.0, 90.0, n_species), precision=precision)
+    pot.build_neighbors(w.pos, species, w.box)
+    out = pot.compute()
+    pot.sync_status()
+    ref = oracle.evaluate(model, w.pos, species, w.box)
+    e_tol, f_tol = (1e-10, 2e-9) if precision else (1e-6, 1e-4)
+    assert abs(float(out["energy"].cpu()) - ref["energy"]) <= e_tol * abs(ref["energy"])
+    assert np.abs(out["forces"].cpu().numpy() - ref["forces"]).max() <= f_tol
+    pot.set_velocities(np.zeros_like(w.pos))
+    pot.step(12, 0.5, 5)
+    pot.sync_status()
